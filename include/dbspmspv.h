@@ -1,0 +1,222 @@
+/*
+ * dbspmspv.h -- C ABI of the B200 (sm_100a) DB-SpMSpV library.
+ *
+ * y = A * x with a sparse matrix A held in fixed 16 x 16 blocks and a sparse vector x
+ * (problem statement: Section 2.1).  One block payload is stored once; a block-level CSR view
+ * (entry point of the pull path) and a block-level CSC view (entry point of the push path)
+ * index it (Section 3.2.1).  Per call the input vector is cut into aligned 16-element vector
+ * blocks with a 16-bit nonzero mask each (Section 3.2.2), the ratio of nonempty vector blocks
+ * selects push or pull (Section 3.3.1), every visited block picks a microkernel from its class
+ * and the local mask (Sections 3.3.1, 3.3.3), and results are reduced in the warp and in shared
+ * memory before they reach global memory (Section 3.3.3).
+ *
+ * Conventions
+ *   - Every array argument is a DEVICE pointer owned by the caller unless stated otherwise.
+ *   - `stream` is a cudaStream_t (passed as an opaque pointer; NULL = the legacy default
+ *     stream).  dbspmspv_run / db_bfs / dbspmspv_decode only enqueue work on it: they allocate
+ *     nothing, never synchronise, and return as soon as the kernels are queued.  Calls on the
+ *     same handle must be stream ordered (the handle owns one workspace).
+ *   - Functions return a dbspmspv_status_t.  Argument errors are reported synchronously.
+ *     Conditions detected on the device (output capacity, a bounded wait that ran out) are
+ *     recorded in the handle and returned by the next dbspmspv_get_stats; a kernel never traps.
+ *   - Bit k of every 16-bit mask is local index k, least significant bit first (Figure 4
+ *     caption: mask value 10 = 0b1010 = positions 1 and 3).
+ *   - A stored entry A[i][j] is the graph edge j -> i (what y = A*x propagates from x_j).
+ *   - "Structural" output: row i is reported iff some stored A[i][j] meets some listed x_j,
+ *     whatever the numeric sum is.
+ */
+#ifndef DBSPMSPV_H
+#define DBSPMSPV_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dbspmspv_handle_s *dbspmspv_handle_t;
+typedef void *dbspmspv_stream_t; /* cudaStream_t */
+
+typedef enum {
+    DBSPMSPV_OK = 0,
+    DBSPMSPV_ERR_INVALID_ARG = 1, /* null pointer, negative size, index out of range, ... */
+    DBSPMSPV_ERR_UNSUPPORTED = 2, /* block size other than 16, semiring/dtype mismatch    */
+    DBSPMSPV_ERR_ALLOC = 3,       /* device or host allocation failed (create only)       */
+    DBSPMSPV_ERR_CUDA = 4,        /* a CUDA runtime call failed                           */
+    DBSPMSPV_ERR_CAPACITY = 5,    /* y_capacity too small; nothing was written out of bounds */
+    DBSPMSPV_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out                   */
+    DBSPMSPV_ERR_BOUNDS = 7       /* validate=1: an x index was out of range              */
+} dbspmspv_status_t;
+
+typedef enum {
+    DBSPMSPV_F32 = 0,    /* fp32 values, fp32 accumulation                                 */
+    DBSPMSPV_BF16 = 1,   /* bf16 values and bf16 x, fp32 accumulation (Section 4.3 layers) */
+    DBSPMSPV_PATTERN = 2 /* no values: Boolean matrices (Section 4.2 graphs)               */
+} dbspmspv_dtype_t;
+
+typedef enum {
+    DBSPMSPV_PLUS_TIMES = 0,
+    DBSPMSPV_OR_AND = 1 /* Boolean: only reachability is computed (Section 4.2)            */
+} dbspmspv_semiring_t;
+
+enum { DBSPMSPV_PATH_AUTO = 0, DBSPMSPV_PATH_PUSH = 1, DBSPMSPV_PATH_PULL = 2 };
+enum { DBSPMSPV_FORMAT_AUTO = 0, DBSPMSPV_FORMAT_COO = 1, DBSPMSPV_FORMAT_CSR = 2 };
+
+/* Block classes (Section 3.2.1).  INLINE is this library's sub-case of COO: a block whose few
+ * entries fit in its view entry and therefore has no payload at all.                        */
+enum {
+    DBSPMSPV_BLK_INLINE = 0,
+    DBSPMSPV_BLK_COO = 1,
+    DBSPMSPV_BLK_FCSR = 2,
+    DBSPMSPV_BLK_FCSC = 3,
+    DBSPMSPV_BLK_CSR = 4,
+    DBSPMSPV_BLK_DENSE = 5,
+    DBSPMSPV_BLK_NCLASS = 6
+};
+
+/* Options of the format build.  Zero-initialise, then call dbspmspv_default_create_opts.    */
+typedef struct {
+    int32_t th0;             /* blocks with fewer than th0 entries use packed COO   (32)     */
+    int32_t th1;             /* blocks with more than th1 entries use Dense         (128)    */
+    float th2;               /* directional skew ratio for ForceCSR / ForceCSC      (2.0)    */
+    int32_t seg_cut;         /* a pull segment closes when its weight reaches this  (64)     */
+    int32_t w_dense;         /* pull segment weight of a Dense block                (4)      */
+    int32_t w_mid;           /* ... of a ForceCSR / ForceCSC / CSR block            (2)      */
+    int32_t w_coo;           /* ... of a COO block                                  (1)      */
+    int32_t force_format;    /* DBSPMSPV_FORMAT_*: ablation knob (Section 5.4)               */
+    int32_t input_on_host;   /* 1: the create arrays are HOST pointers (copied once)         */
+    int32_t reserved[7];
+} dbspmspv_create_opts;
+
+/* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
+typedef struct {
+    float th3;               /* push iff nonempty-vector-block ratio < th3 (0.01 in the paper;
+                                the default here is the crossover measured on B200)          */
+    int32_t force_path;      /* DBSPMSPV_PATH_*                                              */
+    int32_t popc_threshold;  /* CSR-class blocks: popc(mask) >= this -> row-driven (pull-style)
+                                microkernel, below -> column-driven (push-style)             */
+    int32_t validate;        /* 1: range-check x indices on the device (ERR_BOUNDS)          */
+    int32_t reserved[12];
+} dbspmspv_run_opts;
+
+#define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64
+
+typedef struct {
+    /* matrix / format (fixed at create) */
+    int64_t m, n, nnz;             /* nnz after merging duplicates                            */
+    int64_t n_blocks;              /* nonempty 16 x 16 blocks                                 */
+    int64_t class_blocks[DBSPMSPV_BLK_NCLASS]; /* per DBSPMSPV_BLK_* class                    */
+    int64_t class_nnz[DBSPMSPV_BLK_NCLASS];
+    int64_t n_row_blocks, n_col_blocks;        /* ceil(m/16), ceil(n/16)                      */
+    int64_t n_segments;            /* pull segments                                           */
+    int64_t payload_bytes;         /* the single block payload                                */
+    int64_t csr_view_bytes;        /* block-CSR view: row pointers + per-block entries        */
+    int64_t csc_view_bytes;        /* block-CSC view: column pointers + per-block entries     */
+    int64_t segment_bytes;
+    int64_t workspace_bytes;       /* per-call scratch owned by the handle                    */
+    /* last dbspmspv_run / dbspmspv_decode */
+    int32_t last_path;             /* DBSPMSPV_PATH_PUSH or _PULL                             */
+    int32_t last_n_nzblk;          /* nonempty vector blocks                                  */
+    int32_t last_n_tasks;          /* push worklist length                                    */
+    int32_t last_y_nnz;
+    /* last db_bfs */
+    int32_t bfs_levels;            /* number of expansion steps executed                      */
+    int32_t bfs_reached;           /* vertices with level >= 0                                */
+    int32_t bfs_level_path[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];  /* per level DBSPMSPV_PATH_*   */
+    int32_t bfs_level_nzblk[DBSPMSPV_MAX_BFS_LEVELS_RECORDED]; /* frontier vector blocks      */
+    /* deferred device status of the last call (DBSPMSPV_OK if none) */
+    int32_t device_status;
+    int32_t reserved[7];
+} dbspmspv_stats;
+
+/* Paper defaults (th0 = 32, th1 = 128, th2 = 2.0; segment weights 4 / 2 / 1; Sections 3.2.1,
+ * 3.3.2) and this library's measured run-time defaults.                                      */
+void dbspmspv_default_create_opts(dbspmspv_create_opts *opts);
+void dbspmspv_default_run_opts(dbspmspv_run_opts *opts);
+
+/*
+ * Build the dual-view blocked format from CSR (Section 3.2.1).  Runs on the GPU and
+ * synchronises `stream` before returning (it is the offline step, Section 5.5).
+ *   m, n     matrix shape (1 <= m, n < 2^31); nnz >= 0 stored entries (< 2^31)
+ *   row_ptr  m+1 int64 offsets; col_idx nnz int32 columns (any order within a row)
+ *   val      nnz values of type `dtype` (float or bf16 bit patterns); ignored for PATTERN
+ *   Duplicate (i, j) entries are summed (PATTERN: merged); explicitly stored zeros are kept as
+ *   structural entries.  block_size must be 16 (the only size the paper evaluates).
+ *   opts     NULL = defaults.  The input arrays are not referenced after return.
+ * Errors: INVALID_ARG (null/negative/out-of-range index), UNSUPPORTED, ALLOC, CUDA.
+ */
+int dbspmspv_create_csr(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz,
+                        const int64_t *row_ptr, const int32_t *col_idx, const void *val,
+                        int dtype, int block_size, const dbspmspv_create_opts *opts,
+                        dbspmspv_stream_t stream);
+
+/* Same from coordinate triples (row[k], col[k], val[k]), any order.                          */
+int dbspmspv_create_coo(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz,
+                        const int32_t *row, const int32_t *col, const void *val, int dtype,
+                        int block_size, const dbspmspv_create_opts *opts,
+                        dbspmspv_stream_t stream);
+
+/*
+ * One SpMSpV call y = A * x (Sections 3.3, 4.1): vector blocking, path selection, worklist,
+ * block microkernels, writeback and compaction, all enqueued on `stream`.
+ *   x_idx    nnz_x distinct indices in [0, n), any order; x_val nnz_x values of the handle's
+ *            dtype (float, or bf16 bit patterns; ignored/NULL for OR_AND).  Both must stay
+ *            valid and unchanged until the call has finished on the stream.
+ *   semiring PLUS_TIMES (F32/BF16 handles) or OR_AND (any handle; values are then 1.0f)
+ *   y_idx    out: row indices of the structural result, ascending; y_val out: fp32 sums
+ *            (may be NULL for OR_AND); both with room for y_capacity entries
+ *   y_nnz    out: one int32 on the device, the number of result entries (the full count even
+ *            when it exceeds y_capacity; then only the first y_capacity are written and the
+ *            deferred status is ERR_CAPACITY)
+ * nnz_x = 0 gives y_nnz = 0.  Errors: INVALID_ARG, UNSUPPORTED synchronously.
+ */
+int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
+                 int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity,
+                 int32_t *y_nnz, dbspmspv_stream_t stream);
+
+/*
+ * DB-BFS (Section 4.2, Algorithm 5): level-synchronous BFS in which each level is one Boolean
+ * SpMSpV with the frontier masks as x, visited vertices stripped, and push or pull chosen per
+ * level by the same vector-block ratio.  The whole traversal runs in one cooperative launch.
+ *   src      source vertex in [0, n); the matrix must be square (any dtype; values ignored)
+ *   levels   out: n int32 on the device; source 0, unreachable -1
+ */
+int db_bfs(dbspmspv_handle_t h, int32_t src, int32_t *levels, dbspmspv_stream_t stream);
+
+/*
+ * Single-token linear layer (Section 4.3): dense x in, dense y out.  The nonzero mask of x is
+ * generated on the GPU by warp ballot (Section 4.1) and drives the same engine.
+ *   x        n values of the handle's dtype (F32 or BF16 handles); zeros (+0.0 and -0.0) are
+ *            structurally absent
+ *   y        out: m fp32 values; rows without a structural hit are exactly 0
+ */
+int dbspmspv_decode(dbspmspv_handle_t h, const void *x, float *y, dbspmspv_stream_t stream);
+
+/* Synchronises `stream`-ordered work of the handle (cudaDeviceSynchronize) and copies the
+ * statistics to the HOST struct `out`.  Returns the deferred device status of the last call. */
+int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out);
+
+/* Test hook: decode the blocked format back to coordinates.  row/col/val: device arrays with
+ * room for stats.nnz entries (val may be NULL; element type = the handle's dtype).  Order is
+ * block-major; sort before comparing.  Synchronises.                                         */
+int dbspmspv_export_coo(dbspmspv_handle_t h, int32_t *row, int32_t *col, void *val);
+
+/* Test hook: copy the per-block class codes (DBSPMSPV_BLK_*) in primary (block-CSR) order and
+ * the block coordinates to device arrays of stats.n_blocks entries (any may be NULL).        */
+int dbspmspv_export_blocks(dbspmspv_handle_t h, int32_t *block_row, int32_t *block_col,
+                           int32_t *block_class, int32_t *block_nnz);
+
+/* Test hook: copy the dual view out: csr_row_ptr (n_row_blocks+1), csc_col_ptr
+ * (n_col_blocks+1), csc_row (n_blocks: row block of every CSC-view position), csc2csr
+ * (n_blocks: CSC-view position -> primary block id).  Device int32 arrays; any may be NULL. */
+int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *csc_col_ptr,
+                          int32_t *csc_row, int32_t *csc2csr);
+
+int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts);
+int dbspmspv_destroy(dbspmspv_handle_t h);
+const char *dbspmspv_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DBSPMSPV_H */

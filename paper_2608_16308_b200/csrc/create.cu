@@ -1,0 +1,633 @@
+// Blocked preprocessing (Section 3.2.1): partition A into 16 x 16 blocks, classify each block,
+// encode one payload, and build the block-CSR and block-CSC views plus the pull segments
+// (Section 3.3.2).  Offline step (Section 5.5): runs on the GPU, may allocate and synchronise.
+// Radix sort and prefix sums are CUB library primitives; everything else is written here.
+#include <cub/cub.cuh>
+
+#include <new>
+#include <vector>
+
+#include "internal.cuh"
+
+namespace dbs {
+namespace {
+
+struct TempPool {  // device scratch of the build, released when the build returns
+    std::vector<void *> ptrs;
+    ~TempPool() { for (void *p : ptrs) cudaFree(p); }
+    template <typename T> bool get(T **out, size_t count) {
+        void *p = nullptr;
+        if (cudaMalloc(&p, (count ? count : 1) * sizeof(T)) != cudaSuccess) { *out = nullptr; return false; }
+        ptrs.push_back(p);
+        *out = static_cast<T *>(p);
+        return true;
+    }
+    void release(void *p) {
+        for (auto &q : ptrs) if (q == p) { cudaFree(p); q = nullptr; }
+    }
+};
+
+constexpr int TPB = 256;
+inline int grid_for(int64_t n, int tpb = TPB) {
+    int64_t g = (n + tpb - 1) / tpb;
+    return (int)(g < 1 ? 1 : g);
+}
+
+// ---- step 1: one 64-bit key per stored entry: (row block, col block, local row, local col)
+__global__ void k_keys_from_csr(int64_t m, int64_t n, int64_t nnz, const int64_t *row_ptr,
+                                const int32_t *col_idx, uint64_t *keys, uint32_t *src,
+                                int *bad) {
+    int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (e == 0 && (row_ptr[0] != 0 || row_ptr[m] != nnz)) *bad = 1;
+    if (e >= nnz) return;
+    int64_t lo = 0, hi = m;  // largest i with row_ptr[i] <= e
+    while (hi - lo > 1) {
+        int64_t mid = (lo + hi) >> 1;
+        if (row_ptr[mid] <= e) lo = mid; else hi = mid;
+    }
+    int64_t i = lo;
+    if (!(row_ptr[i] <= e && e < row_ptr[i + 1])) { *bad = 1; keys[e] = 0; src[e] = (uint32_t)e; return; }
+    int64_t j = col_idx[e];
+    if (j < 0 || j >= n) { *bad = 1; j = 0; }
+    keys[e] = ((uint64_t)(i >> 4) << 35) | ((uint64_t)(j >> 4) << 8) | ((uint64_t)(i & 15) << 4) | (uint64_t)(j & 15);
+    src[e] = (uint32_t)e;
+}
+
+__global__ void k_keys_from_coo(int64_t m, int64_t n, int64_t nnz, const int32_t *row,
+                                const int32_t *col, uint64_t *keys, uint32_t *src, int *bad) {
+    int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (e >= nnz) return;
+    int64_t i = row[e], j = col[e];
+    if (i < 0 || i >= m || j < 0 || j >= n) { *bad = 1; i = 0; j = 0; }
+    keys[e] = ((uint64_t)(i >> 4) << 35) | ((uint64_t)(j >> 4) << 8) | ((uint64_t)(i & 15) << 4) | (uint64_t)(j & 15);
+    src[e] = (uint32_t)e;
+}
+
+// ---- step 2: merge duplicates, find block boundaries
+__global__ void k_flag_new_key(int64_t n, const uint64_t *keys, int shift, int32_t *flag) {
+    int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (e >= n) return;
+    flag[e] = (e == 0 || (keys[e] >> shift) != (keys[e - 1] >> shift)) ? 1 : 0;
+}
+
+template <int DT>
+__global__ void k_merge_duplicates(int64_t nnz, const uint64_t *keys, const uint32_t *src,
+                                   const int32_t *flag, const int32_t *rank, const void *val,
+                                   uint64_t *ukey, void *uval) {
+    int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (e >= nnz || !flag[e]) return;
+    int64_t u = rank[e] - 1;
+    uint64_t k = keys[e];
+    ukey[u] = k;
+    if (DT == DBSPMSPV_F32) {
+        const float *v = static_cast<const float *>(val);
+        float s = v[src[e]];
+        for (int64_t q = e + 1; q < nnz && keys[q] == k; ++q) s += v[src[q]];
+        static_cast<float *>(uval)[u] = s;
+    } else if (DT == DBSPMSPV_BF16) {
+        const __nv_bfloat16 *v = static_cast<const __nv_bfloat16 *>(val);
+        if (e + 1 < nnz && keys[e + 1] == k) {
+            float s = __bfloat162float(v[src[e]]);
+            for (int64_t q = e + 1; q < nnz && keys[q] == k; ++q) s += __bfloat162float(v[src[q]]);
+            static_cast<__nv_bfloat16 *>(uval)[u] = __float2bfloat16_rn(s);
+        } else {
+            static_cast<__nv_bfloat16 *>(uval)[u] = v[src[e]];
+        }
+    }
+}
+
+__global__ void k_block_starts(int64_t nnzu, const int32_t *flag, const int32_t *rank,
+                               int32_t *blk_start, int32_t n_blocks) {
+    int64_t u = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (u == 0) blk_start[n_blocks] = (int32_t)nnzu;
+    if (u >= nnzu || !flag[u]) return;
+    blk_start[rank[u] - 1] = (int32_t)u;
+}
+
+// ---- step 3: classify (Section 3.2.1) and size every block.  One warp per block.
+struct ClassifyParams {
+    int th0, th1;
+    float th2;
+    int force_format;
+    int dtype;
+};
+
+__device__ __forceinline__ int payload_words(int type, int nnz, int vsize) {
+    switch (type) {
+        case DBSPMSPV_BLK_INLINE: return 0;
+        case DBSPMSPV_BLK_COO: return (nnz + 3) / 4 + (nnz * vsize + 3) / 4;
+        case DBSPMSPV_BLK_DENSE: return 8 + (256 * vsize) / 4;
+        default: return vsize ? HDR_BYTES / 4 + (nnz * vsize + 3) / 4 : 8;
+    }
+}
+
+__global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
+                           ClassifyParams cp, uint8_t *type_out, uint32_t *size_out,
+                           int32_t *brow, int32_t *bcol, unsigned long long *class_blocks,
+                           unsigned long long *class_nnz) {
+    __shared__ uint32_t s_row[TPB / 32][16], s_col[TPB / 32][16];
+    __shared__ unsigned int s_cb[DBSPMSPV_BLK_NCLASS], s_cn[DBSPMSPV_BLK_NCLASS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x < DBSPMSPV_BLK_NCLASS) { s_cb[threadIdx.x] = 0; s_cn[threadIdx.x] = 0; }
+    __syncthreads();
+    int64_t b = blockIdx.x * (int64_t)(TPB / 32) + warp;
+    if (b < n_blocks) {
+        if (lane < 16) { s_row[warp][lane] = 0; s_col[warp][lane] = 0; }
+        __syncwarp();
+        const int s = blk_start[b], nnz = blk_start[b + 1] - s;
+        for (int k = lane; k < nnz; k += 32) {
+            uint32_t rc = (uint32_t)(ukey[s + k] & 0xFF);
+            atomicOr(&s_row[warp][rc >> 4], 1u << (rc & 15));
+            atomicOr(&s_col[warp][rc & 15], 1u << (rc >> 4));
+        }
+        __syncwarp();
+        int rcount = lane < 16 ? __popc(s_row[warp][lane]) : 0;
+        int ccount = lane < 16 ? __popc(s_col[warp][lane]) : 0;
+        for (int o = 8; o; o >>= 1) {
+            rcount = max(rcount, __shfl_xor_sync(0xFFFFFFFFu, rcount, o));
+            ccount = max(ccount, __shfl_xor_sync(0xFFFFFFFFu, ccount, o));
+        }
+        if (lane == 0) {
+            int type;
+            if (cp.force_format == DBSPMSPV_FORMAT_COO) type = DBSPMSPV_BLK_COO;
+            else if (cp.force_format == DBSPMSPV_FORMAT_CSR) type = DBSPMSPV_BLK_CSR;
+            else if (nnz < cp.th0) {
+                const int inline_cap = cp.dtype == DBSPMSPV_PATTERN ? 4 : 1;
+                type = nnz <= inline_cap ? DBSPMSPV_BLK_INLINE : DBSPMSPV_BLK_COO;
+            } else if (nnz > cp.th1) type = DBSPMSPV_BLK_DENSE;
+            // skew_c / skew_r = (max column count) / (max row count): the denominators of
+            // the two axis skews are identical for square blocks
+            else if ((float)ccount > cp.th2 * (float)rcount) type = DBSPMSPV_BLK_FCSC;
+            else if ((float)rcount > cp.th2 * (float)ccount) type = DBSPMSPV_BLK_FCSR;
+            else type = DBSPMSPV_BLK_CSR;
+            const int vsize = cp.dtype == DBSPMSPV_F32 ? 4 : cp.dtype == DBSPMSPV_BF16 ? 2 : 0;
+            type_out[b] = (uint8_t)type;
+            size_out[b] = (uint32_t)payload_words(type, nnz, vsize);
+            uint64_t k0 = ukey[s];
+            brow[b] = (int32_t)(k0 >> 35);
+            bcol[b] = (int32_t)((k0 >> 8) & IDX_MASK);
+            atomicAdd(&s_cb[type], 1u);
+            atomicAdd(&s_cn[type], (unsigned)nnz);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < DBSPMSPV_BLK_NCLASS && s_cb[threadIdx.x]) {
+        atomicAdd(&class_blocks[threadIdx.x], (unsigned long long)s_cb[threadIdx.x]);
+        atomicAdd(&class_nnz[threadIdx.x], (unsigned long long)s_cn[threadIdx.x]);
+    }
+}
+
+// ---- step 4: encode payload + primary (block-CSR) view entries.  One warp per block.
+template <int DT>
+__device__ __forceinline__ void store_value(uint8_t *vals, int pos, const void *uval, int64_t u) {
+    if (DT == DBSPMSPV_F32) reinterpret_cast<float *>(vals)[pos] = static_cast<const float *>(uval)[u];
+    else if (DT == DBSPMSPV_BF16) reinterpret_cast<uint16_t *>(vals)[pos] = static_cast<const uint16_t *>(uval)[u];
+}
+
+template <int DT>
+__global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
+                         const void *uval, const uint8_t *type_in, const uint64_t *poff,
+                         const int32_t *bcol, uint8_t *payload, uint32_t *v_idx, uint32_t *v_w,
+                         uint8_t *v_aux) {
+    constexpr int V = Val<DT>::SIZE;
+    __shared__ uint32_t s_row[TPB / 32][16], s_col[TPB / 32][16];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int64_t b = blockIdx.x * (int64_t)(TPB / 32) + warp;
+    if (b >= n_blocks) return;
+    const int s = blk_start[b], nnz = blk_start[b + 1] - s;
+    const int type = type_in[b];
+    const uint64_t off_words = poff[b];
+    uint8_t *base = payload + off_words * 4;
+    if (lane == 0) {
+        v_idx[b] = (uint32_t)bcol[b] | ((uint32_t)type << TYPE_SHIFT);
+        if (type == DBSPMSPV_BLK_INLINE) {
+            if (DT == DBSPMSPV_PATTERN) {
+                uint32_t w = 0;
+                for (int k = 0; k < nnz; ++k) w |= (uint32_t)(ukey[s + k] & 0xFF) << (8 * k);
+                v_w[b] = w;
+                v_aux[b] = (uint8_t)(nnz - 1);
+            } else {
+                v_w[b] = DT == DBSPMSPV_F32 ? __float_as_uint(static_cast<const float *>(uval)[s])
+                                            : (uint32_t) static_cast<const uint16_t *>(uval)[s];
+                v_aux[b] = (uint8_t)(ukey[s] & 0xFF);
+            }
+        } else {
+            v_w[b] = (uint32_t)off_words;
+            v_aux[b] = (uint8_t)(nnz - 1);
+        }
+    }
+    if (type == DBSPMSPV_BLK_INLINE) return;
+    if (type == DBSPMSPV_BLK_COO) {
+        uint8_t *vals = base + ((nnz + 3) & ~3);
+        for (int k = lane; k < ((nnz + 3) & ~3); k += 32)
+            base[k] = k < nnz ? (uint8_t)(ukey[s + k] & 0xFF) : 0;
+        for (int k = lane; k < nnz; k += 32) store_value<DT>(vals, k, uval, s + k);
+        if (DT == DBSPMSPV_BF16 && (nnz & 1) && lane == 0) reinterpret_cast<uint16_t *>(vals)[nnz] = 0;
+        return;
+    }
+    // mask-based classes
+    if (lane < 16) { s_row[warp][lane] = 0; s_col[warp][lane] = 0; }
+    __syncwarp();
+    for (int k = lane; k < nnz; k += 32) {
+        uint32_t rc = (uint32_t)(ukey[s + k] & 0xFF);
+        atomicOr(&s_row[warp][rc >> 4], 1u << (rc & 15));
+        atomicOr(&s_col[warp][rc & 15], 1u << (rc >> 4));
+    }
+    __syncwarp();
+    const bool row_major = (type == DBSPMSPV_BLK_FCSR || type == DBSPMSPV_BLK_CSR);
+    uint32_t mine = lane < 16 ? (row_major ? s_row[warp][lane] : s_col[warp][lane]) : 0;
+    int start = __popc(mine);  // exclusive prefix over lanes 0..15
+    for (int o = 1; o < 16; o <<= 1) {
+        int t = __shfl_up_sync(0xFFFFFFFFu, start, o);
+        if (lane >= o) start += t;
+    }
+    start -= __popc(mine);
+    uint16_t *masks = reinterpret_cast<uint16_t *>(base);
+    if (lane < 16) masks[lane] = (uint16_t)mine;
+    if (type == DBSPMSPV_BLK_DENSE) {
+        if (V) {
+            uint8_t *vals = base + 32;
+            uint32_t *z = reinterpret_cast<uint32_t *>(vals);
+            for (int k = lane; k < 256 * V / 4; k += 32) z[k] = 0;
+            __syncwarp();
+            for (int k = lane; k < nnz; k += 32) {
+                uint32_t rc = (uint32_t)(ukey[s + k] & 0xFF);
+                store_value<DT>(vals, (rc & 15) * 16 + (rc >> 4), uval, s + k);
+            }
+        }
+        return;
+    }
+    if (!V) return;  // pattern: masks only
+    if (lane < 16) base[32 + lane] = (uint8_t)start;
+    uint8_t *vals = base + HDR_BYTES;
+    if (row_major) {
+        for (int k = lane; k < nnz; k += 32) store_value<DT>(vals, k, uval, s + k);
+    } else {
+        // column-major position of (r, c): start of column c + entries of c above row r
+        __shared__ uint8_t s_start[TPB / 32][16];
+        if (lane < 16) s_start[warp][lane] = (uint8_t)start;
+        __syncwarp();
+        for (int k = lane; k < nnz; k += 32) {
+            uint32_t rc = (uint32_t)(ukey[s + k] & 0xFF);
+            int r = rc >> 4, c = rc & 15;
+            int pos = s_start[warp][c] + __popc(s_col[warp][c] & ((1u << r) - 1));
+            store_value<DT>(vals, pos, uval, s + k);
+        }
+    }
+    if (DT == DBSPMSPV_BF16 && (nnz & 1) && lane == 0) reinterpret_cast<uint16_t *>(vals)[nnz] = 0;
+}
+
+// first position p in a sorted int array with a[p] >= v, for v = 0..count (pointer arrays)
+__global__ void k_lower_bounds(int32_t count, const int32_t *sorted, int32_t n, int32_t *ptr) {
+    int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (v > count) return;
+    int32_t lo = 0, hi = n;
+    while (lo < hi) {
+        int32_t mid = lo + ((hi - lo) >> 1);
+        if (sorted[mid] < v) lo = mid + 1; else hi = mid;
+    }
+    ptr[v] = lo;
+}
+
+__global__ void k_csc_keys(int32_t n_blocks, const int32_t *brow, const int32_t *bcol,
+                           uint64_t *keys, int32_t *ids) {
+    int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (b >= n_blocks) return;
+    keys[b] = ((uint64_t)bcol[b] << 27) | (uint64_t)brow[b];
+    ids[b] = (int32_t)b;
+}
+
+__global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
+                             const int32_t *csc2csr, const uint32_t *csr_idx,
+                             const uint32_t *csr_w, const uint8_t *csr_aux, uint32_t *csc_idx,
+                             uint32_t *csc_w, uint8_t *csc_aux, int32_t *bcol_sorted) {
+    int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p >= n_blocks) return;
+    int32_t b = csc2csr[p];
+    uint64_t k = keys_sorted[p];
+    csc_idx[p] = (uint32_t)(k & IDX_MASK) | (csr_idx[b] & ~IDX_MASK);
+    csc_w[p] = csr_w[b];
+    csc_aux[p] = csr_aux[b];
+    bcol_sorted[p] = (int32_t)(k >> 27);
+}
+
+// ---- pull segments (Section 3.3.2): greedy walk along each row block; a segment closes
+// when its accumulated weight reaches the cut.  One thread per row block, two passes.
+struct SegParams { int cut, w_dense, w_mid, w_coo; };
+
+__device__ __forceinline__ int seg_weight(uint32_t idx, const SegParams &sp) {
+    int t = idx >> TYPE_SHIFT;
+    return t == DBSPMSPV_BLK_DENSE ? sp.w_dense : (t <= DBSPMSPV_BLK_COO ? sp.w_coo : sp.w_mid);
+}
+
+__global__ void k_seg_count(int32_t mb, const int32_t *row_ptr, const uint32_t *idx,
+                            SegParams sp, int32_t *count) {
+    int64_t rb = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (rb >= mb) return;
+    int acc = 0, c = 0;
+    for (int p = row_ptr[rb]; p < row_ptr[rb + 1]; ++p) {
+        acc += seg_weight(idx[p], sp);
+        if (acc >= sp.cut) { ++c; acc = 0; }
+    }
+    if (acc > 0) ++c;
+    count[rb] = c;
+}
+
+__global__ void k_seg_write(int32_t mb, const int32_t *row_ptr, const uint32_t *idx,
+                            SegParams sp, const int32_t *seg_off, Segment *segs) {
+    int64_t rb = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (rb >= mb) return;
+    int acc = 0, first = row_ptr[rb];
+    const int end = row_ptr[rb + 1];
+    int o = seg_off[rb];
+    for (int p = first; p < end; ++p) {
+        acc += seg_weight(idx[p], sp);
+        if (acc >= sp.cut || p + 1 == end) {
+            Segment s;
+            s.row_block = (int32_t)rb;
+            s.start = first;
+            s.count = (p + 1 - first) | ((first == row_ptr[rb] && p + 1 == end) ? (int32_t)0x80000000 : 0);
+            segs[o++] = s;
+            first = p + 1;
+            acc = 0;
+        }
+    }
+}
+
+template <typename T>
+int exclusive_sum(TempPool &tp, const T *in, T *out, int64_t n, cudaStream_t st) {
+    size_t bytes = 0;
+    DBS_CUDA(cub::DeviceScan::ExclusiveSum(nullptr, bytes, in, out, n, st));
+    void *tmp;
+    if (!tp.get((uint8_t **)&tmp, bytes)) return DBSPMSPV_ERR_ALLOC;
+    DBS_CUDA(cub::DeviceScan::ExclusiveSum(tmp, bytes, in, out, n, st));
+    DBS_CUDA(cudaStreamSynchronize(st));
+    tp.release(tmp);
+    return DBSPMSPV_OK;
+}
+
+int inclusive_sum_i32(TempPool &tp, const int32_t *in, int32_t *out, int64_t n, cudaStream_t st) {
+    size_t bytes = 0;
+    DBS_CUDA(cub::DeviceScan::InclusiveSum(nullptr, bytes, in, out, n, st));
+    void *tmp;
+    if (!tp.get((uint8_t **)&tmp, bytes)) return DBSPMSPV_ERR_ALLOC;
+    DBS_CUDA(cub::DeviceScan::InclusiveSum(tmp, bytes, in, out, n, st));
+    DBS_CUDA(cudaStreamSynchronize(st));
+    tp.release(tmp);
+    return DBSPMSPV_OK;
+}
+
+template <typename K, typename V>
+int sort_pairs(TempPool &tp, K *&keys, K *&keys_alt, V *&vals, V *&vals_alt, int64_t n,
+               int end_bit, cudaStream_t st) {
+    cub::DoubleBuffer<K> dk(keys, keys_alt);
+    cub::DoubleBuffer<V> dv(vals, vals_alt);
+    size_t bytes = 0;
+    DBS_CUDA(cub::DeviceRadixSort::SortPairs(nullptr, bytes, dk, dv, n, 0, end_bit, st));
+    void *tmp;
+    if (!tp.get((uint8_t **)&tmp, bytes)) return DBSPMSPV_ERR_ALLOC;
+    DBS_CUDA(cub::DeviceRadixSort::SortPairs(tmp, bytes, dk, dv, n, 0, end_bit, st));
+    DBS_CUDA(cudaStreamSynchronize(st));
+    tp.release(tmp);
+    if (dk.Current() != keys) { K *t = keys; keys = keys_alt; keys_alt = t; }
+    if (dv.Current() != vals) { V *t = vals; vals = vals_alt; vals_alt = t; }
+    return DBSPMSPV_OK;
+}
+
+struct Widen {  // uint32 block sizes as uint64, with one extra zero so the scan yields the total
+    const uint32_t *in;
+    int32_t n;
+    __host__ __device__ uint64_t operator()(int64_t i) const { return i < n ? in[i] : 0; }
+};
+
+int bits_for(uint64_t v) { int b = 0; while (v) { ++b; v >>= 1; } return b ? b : 1; }
+
+#define DBS_TRY(expr) do { int s__ = (expr); if (s__ != DBSPMSPV_OK) return s__; } while (0)
+#define DBS_GET(ptr, count) do { if (!tp.get(&(ptr), (size_t)(count))) return DBSPMSPV_ERR_ALLOC; } while (0)
+#define DBS_KEEP(ptr, count) do { void *p__ = nullptr; \
+        if (cudaMalloc(&p__, ((count) ? (size_t)(count) : 1) * sizeof(*(ptr))) != cudaSuccess) return DBSPMSPV_ERR_ALLOC; \
+        (ptr) = static_cast<decltype(ptr)>(p__); } while (0)
+
+int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t *row_ptr,
+          const int32_t *rows, const int32_t *cols, const void *val, cudaStream_t st) {
+    TempPool tp;
+    Device &d = h->d;
+    const int dt = d.dtype;
+    const int vsize = dt == DBSPMSPV_F32 ? 4 : dt == DBSPMSPV_BF16 ? 2 : 0;
+    d.m = m; d.n = n;
+    d.mb = (int32_t)((m + B - 1) / B);
+    d.nb = (int32_t)((n + B - 1) / B);
+
+    // inputs on the host: copy once
+    if (h->copts.input_on_host) {
+        if (row_ptr) { int64_t *t; DBS_GET(t, m + 1); DBS_CUDA(cudaMemcpyAsync(t, row_ptr, (m + 1) * 8, cudaMemcpyHostToDevice, st)); row_ptr = t; }
+        if (rows) { int32_t *t; DBS_GET(t, nnz); DBS_CUDA(cudaMemcpyAsync(t, rows, nnz * 4, cudaMemcpyHostToDevice, st)); rows = t; }
+        { int32_t *t; DBS_GET(t, nnz); DBS_CUDA(cudaMemcpyAsync(t, cols, nnz * 4, cudaMemcpyHostToDevice, st)); cols = t; }
+        if (vsize) { uint8_t *t; DBS_GET(t, nnz * vsize); DBS_CUDA(cudaMemcpyAsync(t, val, nnz * vsize, cudaMemcpyHostToDevice, st)); val = t; }
+    }
+
+    int *bad;
+    DBS_GET(bad, 1);
+    DBS_CUDA(cudaMemsetAsync(bad, 0, sizeof(int), st));
+
+    uint64_t *keys, *keys_alt;
+    uint32_t *src, *src_alt;
+    DBS_GET(keys, nnz); DBS_GET(keys_alt, nnz); DBS_GET(src, nnz); DBS_GET(src_alt, nnz);
+    if (nnz > 0) {
+        if (row_ptr) k_keys_from_csr<<<grid_for(nnz), TPB, 0, st>>>(m, n, nnz, row_ptr, cols, keys, src, bad);
+        else k_keys_from_coo<<<grid_for(nnz), TPB, 0, st>>>(m, n, nnz, rows, cols, keys, src, bad);
+    }
+    int bad_h = 0;
+    DBS_CUDA(cudaMemcpyAsync(&bad_h, bad, sizeof(int), cudaMemcpyDeviceToHost, st));
+    DBS_CUDA(cudaStreamSynchronize(st));
+    if (bad_h) return DBSPMSPV_ERR_INVALID_ARG;
+
+    int64_t nnzu = 0;
+    uint64_t *ukey = nullptr;
+    void *uval = nullptr;
+    int32_t n_blocks = 0;
+    int32_t *blk_start = nullptr;
+    if (nnz > 0) {
+        DBS_TRY(sort_pairs(tp, keys, keys_alt, src, src_alt, nnz, 35 + bits_for((uint64_t)d.mb), st));
+        tp.release(keys_alt); tp.release(src_alt);
+        int32_t *flag, *rank;
+        DBS_GET(flag, nnz); DBS_GET(rank, nnz);
+        k_flag_new_key<<<grid_for(nnz), TPB, 0, st>>>(nnz, keys, 0, flag);
+        DBS_TRY(inclusive_sum_i32(tp, flag, rank, nnz, st));
+        int32_t last;
+        DBS_CUDA(cudaMemcpy(&last, rank + nnz - 1, 4, cudaMemcpyDeviceToHost));
+        nnzu = last;
+        DBS_GET(ukey, nnzu);
+        { uint8_t *t; DBS_GET(t, nnzu * (vsize ? vsize : 1)); uval = t; }
+        if (dt == DBSPMSPV_F32) k_merge_duplicates<DBSPMSPV_F32><<<grid_for(nnz), TPB, 0, st>>>(nnz, keys, src, flag, rank, val, ukey, uval);
+        else if (dt == DBSPMSPV_BF16) k_merge_duplicates<DBSPMSPV_BF16><<<grid_for(nnz), TPB, 0, st>>>(nnz, keys, src, flag, rank, val, ukey, uval);
+        else k_merge_duplicates<DBSPMSPV_PATTERN><<<grid_for(nnz), TPB, 0, st>>>(nnz, keys, src, flag, rank, val, ukey, uval);
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(keys); tp.release(src);
+        k_flag_new_key<<<grid_for(nnzu), TPB, 0, st>>>(nnzu, ukey, 8, flag);
+        DBS_TRY(inclusive_sum_i32(tp, flag, rank, nnzu, st));
+        DBS_CUDA(cudaMemcpy(&last, rank + nnzu - 1, 4, cudaMemcpyDeviceToHost));
+        n_blocks = last;
+        DBS_GET(blk_start, (int64_t)n_blocks + 1);
+        k_block_starts<<<grid_for(nnzu), TPB, 0, st>>>(nnzu, flag, rank, blk_start, n_blocks);
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(flag); tp.release(rank);
+    }
+    h->nnz = nnzu;
+    d.n_blocks = n_blocks;
+
+    // classify + size
+    uint8_t *type;
+    uint32_t *psize;
+    uint64_t *poff;
+    int32_t *bcol;
+    unsigned long long *cls;
+    DBS_GET(type, n_blocks); DBS_GET(psize, n_blocks); DBS_GET(bcol, n_blocks);
+    DBS_GET(cls, 2 * DBSPMSPV_BLK_NCLASS);
+    DBS_KEEP(h->block_row, n_blocks);
+    DBS_CUDA(cudaMemsetAsync(cls, 0, 2 * DBSPMSPV_BLK_NCLASS * sizeof(unsigned long long), st));
+    ClassifyParams cp{h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt};
+    if (n_blocks) k_classify<<<grid_for(n_blocks, TPB / 32), TPB, 0, st>>>(n_blocks, blk_start, ukey, cp, type, psize, h->block_row, bcol, cls, cls + DBSPMSPV_BLK_NCLASS);
+    // 64-bit offsets for the scan (the total may exceed 2^32 words only beyond 16 GB)
+    DBS_GET(poff, (int64_t)n_blocks + 1);
+    {
+        auto it = cub::TransformInputIterator<uint64_t, Widen, cub::CountingInputIterator<int64_t>>(cub::CountingInputIterator<int64_t>(0), Widen{psize, n_blocks});
+        size_t bytes = 0;
+        DBS_CUDA(cub::DeviceScan::ExclusiveSum(nullptr, bytes, it, poff, (int64_t)n_blocks + 1, st));
+        uint8_t *tmp; DBS_GET(tmp, bytes);
+        DBS_CUDA(cub::DeviceScan::ExclusiveSum(tmp, bytes, it, poff, (int64_t)n_blocks + 1, st));
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(tmp);
+    }
+    uint64_t total_words = 0;
+    DBS_CUDA(cudaMemcpy(&total_words, poff + n_blocks, 8, cudaMemcpyDeviceToHost));
+    if (total_words >= (1ull << 32)) return DBSPMSPV_ERR_UNSUPPORTED;
+    h->payload_bytes = (int64_t)total_words * 4;
+    {
+        uint8_t *p; DBS_KEEP(p, h->payload_bytes + 256);  // slack: staged copies may over-read
+        DBS_CUDA(cudaMemsetAsync(p, 0, h->payload_bytes + 256, st));
+        h->payload_alloc = p; d.payload = p;
+    }
+    DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_blocks); DBS_KEEP(d.csr.w, n_blocks); DBS_KEEP(d.csr.aux, n_blocks);
+    DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_blocks); DBS_KEEP(d.csc.w, n_blocks); DBS_KEEP(d.csc.aux, n_blocks);
+    DBS_KEEP(h->csc2csr, n_blocks);
+    if (n_blocks) {
+        uint8_t *pl = static_cast<uint8_t *>(h->payload_alloc);
+        const int g = grid_for(n_blocks, TPB / 32);
+        if (dt == DBSPMSPV_F32) k_encode<DBSPMSPV_F32><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux);
+        else if (dt == DBSPMSPV_BF16) k_encode<DBSPMSPV_BF16><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux);
+        else k_encode<DBSPMSPV_PATTERN><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux);
+    }
+    k_lower_bounds<<<grid_for(d.mb + 1), TPB, 0, st>>>(d.mb, h->block_row, n_blocks, d.csr.ptr);
+    DBS_CUDA(cudaStreamSynchronize(st));
+    tp.release(ukey); tp.release(uval); tp.release(blk_start); tp.release(poff); tp.release(psize);
+
+    // block-CSC view: sort primary ids by (column block, row block)
+    {
+        uint64_t *k2, *k2_alt;
+        int32_t *ids, *ids_alt, *bcol_sorted;
+        DBS_GET(k2, n_blocks); DBS_GET(k2_alt, n_blocks); DBS_GET(ids, n_blocks); DBS_GET(ids_alt, n_blocks);
+        DBS_GET(bcol_sorted, n_blocks);
+        if (n_blocks) {
+            k_csc_keys<<<grid_for(n_blocks), TPB, 0, st>>>(n_blocks, h->block_row, bcol, k2, ids);
+            DBS_TRY(sort_pairs(tp, k2, k2_alt, ids, ids_alt, (int64_t)n_blocks, 27 + bits_for((uint64_t)d.nb), st));
+            DBS_CUDA(cudaMemcpyAsync(h->csc2csr, ids, (size_t)n_blocks * 4, cudaMemcpyDeviceToDevice, st));
+            k_csc_gather<<<grid_for(n_blocks), TPB, 0, st>>>(n_blocks, k2, h->csc2csr, d.csr.idx, d.csr.w, d.csr.aux, d.csc.idx, d.csc.w, d.csc.aux, bcol_sorted);
+        }
+        k_lower_bounds<<<grid_for(d.nb + 1), TPB, 0, st>>>(d.nb, bcol_sorted, n_blocks, d.csc.ptr);
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(k2); tp.release(k2_alt); tp.release(ids); tp.release(ids_alt); tp.release(bcol_sorted);
+    }
+
+    // pull segments
+    {
+        SegParams sp{h->copts.seg_cut, h->copts.w_dense, h->copts.w_mid, h->copts.w_coo};
+        int32_t *cnt, *off;
+        DBS_GET(cnt, (int64_t)d.mb + 1); DBS_GET(off, (int64_t)d.mb + 1);
+        DBS_CUDA(cudaMemsetAsync(cnt, 0, ((size_t)d.mb + 1) * 4, st));
+        k_seg_count<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, cnt);
+        DBS_TRY(exclusive_sum(tp, cnt, off, (int64_t)d.mb + 1, st));
+        int32_t nseg = 0;
+        DBS_CUDA(cudaMemcpy(&nseg, off + d.mb, 4, cudaMemcpyDeviceToHost));
+        d.n_segments = nseg;
+        Segment *segs; DBS_KEEP(segs, nseg);
+        k_seg_write<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, off, segs);
+        d.segments = segs;
+        DBS_CUDA(cudaStreamSynchronize(st));
+    }
+
+    // statistics
+    unsigned long long cls_h[2 * DBSPMSPV_BLK_NCLASS];
+    DBS_CUDA(cudaMemcpy(cls_h, cls, sizeof(cls_h), cudaMemcpyDeviceToHost));
+    dbspmspv_stats &s = h->stats;
+    s.m = m; s.n = n; s.nnz = nnzu; s.n_blocks = n_blocks;
+    for (int c = 0; c < DBSPMSPV_BLK_NCLASS; ++c) { s.class_blocks[c] = (int64_t)cls_h[c]; s.class_nnz[c] = (int64_t)cls_h[DBSPMSPV_BLK_NCLASS + c]; }
+    s.n_row_blocks = d.mb; s.n_col_blocks = d.nb; s.n_segments = d.n_segments;
+    s.payload_bytes = h->payload_bytes;
+    s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)n_blocks * 9;
+    s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)n_blocks * 9;
+    s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment);
+    DBS_CUDA(cudaGetLastError());
+    return DBSPMSPV_OK;
+}
+
+}  // namespace
+
+int allocate_workspace(dbspmspv_handle_s *h);  // run.cu
+
+int create_common(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz, const int64_t *row_ptr,
+                  const int32_t *rows, const int32_t *cols, const void *val, int dtype, int block_size,
+                  const dbspmspv_create_opts *opts, dbspmspv_stream_t stream) {
+    if (!out) return DBSPMSPV_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (m < 1 || n < 1 || nnz < 0 || m >= (1ll << 31) || n >= (1ll << 31) || nnz >= (1ll << 31)) return DBSPMSPV_ERR_INVALID_ARG;
+    if ((!row_ptr && !rows) || (nnz > 0 && !cols)) return DBSPMSPV_ERR_INVALID_ARG;
+    if (dtype != DBSPMSPV_F32 && dtype != DBSPMSPV_BF16 && dtype != DBSPMSPV_PATTERN) return DBSPMSPV_ERR_INVALID_ARG;
+    if (dtype != DBSPMSPV_PATTERN && nnz > 0 && !val) return DBSPMSPV_ERR_INVALID_ARG;
+    if (block_size != B) return DBSPMSPV_ERR_UNSUPPORTED;
+    dbspmspv_handle_s *h = new (std::nothrow) dbspmspv_handle_s();
+    if (!h) return DBSPMSPV_ERR_ALLOC;
+    if (opts) h->copts = *opts; else dbspmspv_default_create_opts(&h->copts);
+    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.w_coo < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
+    dbspmspv_default_run_opts(&h->ropts);
+    h->d.dtype = dtype;
+    if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return DBSPMSPV_ERR_CUDA; }
+    cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+    int st = build(h, m, n, nnz, row_ptr, rows, cols, val, static_cast<cudaStream_t>(stream));
+    if (st == DBSPMSPV_OK) st = allocate_workspace(h);
+    if (st != DBSPMSPV_OK) { cudaGetLastError(); dbspmspv_destroy(h); return st; }
+    *out = h;
+    return DBSPMSPV_OK;
+}
+
+}  // namespace dbs
+
+extern "C" {
+
+void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
+    if (!o) return;
+    *o = dbspmspv_create_opts();
+    o->th0 = 32; o->th1 = 128; o->th2 = 2.0f;
+    o->seg_cut = 64; o->w_dense = 4; o->w_mid = 2; o->w_coo = 1;
+    o->force_format = DBSPMSPV_FORMAT_AUTO;
+    o->input_on_host = 0;
+}
+
+int dbspmspv_create_csr(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz,
+                        const int64_t *row_ptr, const int32_t *col_idx, const void *val,
+                        int dtype, int block_size, const dbspmspv_create_opts *opts,
+                        dbspmspv_stream_t stream) {
+    if (!row_ptr) return DBSPMSPV_ERR_INVALID_ARG;
+    return dbs::create_common(out, m, n, nnz, row_ptr, nullptr, col_idx, val, dtype, block_size, opts, stream);
+}
+
+int dbspmspv_create_coo(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz,
+                        const int32_t *row, const int32_t *col, const void *val, int dtype,
+                        int block_size, const dbspmspv_create_opts *opts,
+                        dbspmspv_stream_t stream) {
+    if (!row && nnz > 0) return DBSPMSPV_ERR_INVALID_ARG;
+    static const int32_t dummy = 0;
+    return dbs::create_common(out, m, n, nnz, nullptr, row ? row : &dummy, col, val, dtype, block_size, opts, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,150 @@
+// Internal definitions shared by the .cu files of libdbspmspv: the in-memory block format,
+// the handle, and small device helpers.  Nothing here is part of the public ABI.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dbspmspv.h"
+
+namespace dbs {
+
+// ---------------------------------------------------------------------------------------
+// Block format (the dual-view storage of Section 3.2.1, laid out for B200)
+//
+// A "view" is three parallel arrays with one entry per nonempty block:
+//   idx[p]  bits 0..26  the block's index along the *other* dimension (column block in the
+//                       block-CSR view, row block in the block-CSC view)
+//           bits 29..31 block class (DBSPMSPV_BLK_*)
+//   w[p]    payload offset in 4-byte words -- or, for INLINE blocks, the data itself:
+//             valued matrices : the single value (fp32 bits, or bf16 bits in the low half)
+//             pattern matrices: up to four packed local coordinates, one per byte
+//   aux[p]  nnz-1 -- or, for valued INLINE blocks, the packed local coordinate
+// A packed local coordinate is one byte: (row << 4) | col.
+// Both views carry the same (w, aux) for a block, so either traversal direction reaches the
+// payload in one hop; the payload itself is stored once, in block-CSR ("primary") order.
+//
+// Payload per class (V = value size: 4 fp32, 2 bf16, 0 pattern; every block starts on a
+// 4-byte boundary):
+//   COO    nnz coordinate bytes, padded to 4 | nnz values
+//   FCSR   16 x u16 row masks | 16 x u8 row starts | values row-major          (Alg. 2)
+//   CSR    same encoding as FCSR (balanced blocks; column access by mask arithmetic)
+//   FCSC   16 x u16 column masks | 16 x u8 column starts | values column-major (Alg. 3)
+//   DENSE  16 x u16 column masks | 256 values column-major (absent entries 0)
+// Pattern matrices keep only the masks (and coordinate bytes).
+// ---------------------------------------------------------------------------------------
+constexpr int B = 16;                       // block edge
+constexpr uint32_t IDX_MASK = 0x07FFFFFFu;  // 27 bits
+constexpr int TYPE_SHIFT = 29;
+constexpr int PUSH_CHUNK = 32;              // CSC-view entries per push task (one per lane)
+constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-class block
+
+struct View {
+    int32_t *ptr;    // nb_major + 1
+    uint32_t *idx;   // n_blocks
+    uint32_t *w;     // n_blocks
+    uint8_t *aux;    // n_blocks
+};
+
+struct Segment {     // pull work unit: a run of consecutive blocks inside one row block
+    int32_t row_block;
+    int32_t start;   // first position in the block-CSR view
+    int32_t count;   // bit 31: the segment covers its whole row block (plain stores allowed)
+};
+
+struct Counters {    // device-resident scalars of one call
+    int32_t n_nzblk;      // nonempty vector blocks
+    int32_t n_tasks;      // push worklist length
+    int32_t path;         // chosen path of the call (DBSPMSPV_PATH_PUSH / _PULL)
+    int32_t y_nnz;
+    int32_t status;       // deferred device status
+    int32_t last_n_nzblk, last_n_tasks, last_path, last_y_nnz;
+    int32_t bfs_levels, bfs_reached;
+    int32_t pad;
+    int32_t bfs_level_path[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
+    int32_t bfs_level_nzblk[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
+};
+
+struct Workspace {
+    float *x_dense;       // n (padded to a multiple of 32): dense copy of x (Section 3.2.2)
+    uint32_t *x_mask32;   // vector-block masks, two 16-bit masks per word
+    uint2 *tasks;         // push worklist: (column block, first CSC-view position)
+    float *y_acc;         // m (padded): dense accumulator, all zero between calls
+    uint32_t *y_mask32;   // structural-hit masks per row block, two per word, zero between calls
+    int32_t *tile_count;  // compaction: result entries per tile of row blocks
+    uint32_t *visited32;  // BFS: visited masks
+    Counters *ctr;
+    int64_t task_capacity;
+    int32_t n_tiles;
+};
+
+struct Device {           // everything the kernels need, passed by value
+    int64_t m, n;
+    int32_t mb, nb;       // row blocks, column blocks
+    int32_t n_blocks;
+    int32_t n_segments;
+    int32_t dtype;
+    View csr, csc;
+    const uint8_t *payload;
+    const Segment *segments;
+    Workspace ws;
+};
+
+}  // namespace dbs
+
+struct dbspmspv_handle_s {
+    dbs::Device d;
+    int device;                 // CUDA device ordinal the handle lives on
+    int sm_count;
+    int64_t nnz;
+    int32_t *csc2csr;           // CSC-view position -> primary block id (Section 3.2.1)
+    int32_t *block_row;         // primary order: row block of every block
+    dbspmspv_create_opts copts;
+    dbspmspv_run_opts ropts;
+    dbspmspv_stats stats;       // host copy of the static part
+    void *payload_alloc;
+    int64_t payload_bytes;
+    int bfs_grid;               // co-resident grid size of the BFS kernel
+};
+
+namespace dbs {
+
+#define DBS_CUDA(call)                                      \
+    do {                                                    \
+        cudaError_t e__ = (call);                           \
+        if (e__ != cudaSuccess) return DBSPMSPV_ERR_CUDA;   \
+    } while (0)
+
+template <typename T>
+__host__ __device__ inline T ceil_div(T a, T b) { return (a + b - 1) / b; }
+
+__device__ __forceinline__ uint32_t mask_of(const uint32_t *mask32, int blk) {
+    return (mask32[blk >> 1] >> ((blk & 1) * 16)) & 0xFFFFu;
+}
+
+// value loads from the payload, widened to fp32
+template <int DT> struct Val;
+template <> struct Val<DBSPMSPV_F32> {
+    static constexpr int SIZE = 4;
+    __device__ static __forceinline__ float load(const uint8_t *base, int k) {
+        return reinterpret_cast<const float *>(base)[k];
+    }
+    __device__ static __forceinline__ float inline_value(uint32_t w) { return __uint_as_float(w); }
+};
+template <> struct Val<DBSPMSPV_BF16> {
+    static constexpr int SIZE = 2;
+    __device__ static __forceinline__ float load(const uint8_t *base, int k) {
+        return __uint_as_float(uint32_t(reinterpret_cast<const uint16_t *>(base)[k]) << 16);
+    }
+    __device__ static __forceinline__ float inline_value(uint32_t w) {
+        return __uint_as_float((w & 0xFFFFu) << 16);
+    }
+};
+template <> struct Val<DBSPMSPV_PATTERN> {
+    static constexpr int SIZE = 0;
+    __device__ static __forceinline__ float load(const uint8_t *, int) { return 1.0f; }
+    __device__ static __forceinline__ float inline_value(uint32_t) { return 1.0f; }
+};
+
+}  // namespace dbs

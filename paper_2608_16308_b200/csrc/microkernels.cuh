@@ -1,0 +1,181 @@
+// Per-block microkernels (Sections 3.3.1 and 3.3.3).  A visited block picks one of these from
+// its class and from popc of the local vector-block mask:
+//   INLINE / small COO   one lane owns the whole block (hypersparse blocks dominate power-law
+//                        matrices, so 32 blocks are processed per warp step)
+//   larger COO           one lane per stored entry, shared-memory accumulation
+//   ForceCSR, CSR (dense mask)   row-driven, two lanes per row (Algorithm 2)
+//   CSR (sparse mask)    column-driven over the active columns, row masks give the positions
+//   ForceCSC             column-driven, half-warps split the columns (Algorithm 3)
+//   Dense                column-major values, half-warp per active column (role of Algorithm 4)
+// All warp-cooperative kernels leave the partial sum of row (lane & 15) in lanes 0..15 and
+// return the 16-bit mask of rows that received a structural product.
+#pragma once
+
+#include "internal.cuh"
+
+namespace dbs {
+
+constexpr unsigned FULL = 0xFFFFFFFFu;
+constexpr int COO_SERIAL_MAX = 6;   // COO blocks up to this size are handled by one lane
+
+__device__ __forceinline__ uint32_t below(int k) { return (1u << k) - 1u; }
+
+// Row-driven kernel for row-mask encodings (Algorithm 2): lane = (row, sub-lane); the two
+// sub-lanes of a row take alternate active entries; value position = row start + number of
+// stored entries left of the column.
+template <int DT>
+__device__ __forceinline__ float mk_row_pull(const uint8_t *blk, uint32_t xm, const float *s_x,
+                                             int lane, uint32_t &hits) {
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    const int row = lane >> 1, sub = lane & 1;
+    const uint32_t rm = masks[row];
+    const int rp = blk[32 + row];
+    const uint8_t *vals = blk + HDR_BYTES;
+    uint32_t active = rm & xm;
+    float sum = 0.f;
+    int nz = 0;
+    while (active) {
+        const int c = __ffs(active) - 1;
+        if ((nz & 1) == sub) sum += Val<DT>::load(vals, rp + __popc(rm & below(c))) * s_x[c];
+        active &= active - 1;
+        ++nz;
+    }
+    sum += __shfl_xor_sync(FULL, sum, 1);
+    hits = __ballot_sync(FULL, lane < 16 && (masks[lane & 15] & xm) != 0);
+    return __shfl_sync(FULL, sum, (lane & 15) * 2);
+}
+
+// Column-driven kernel for row-mask encodings (the push access of the patched-CSR class,
+// Section 3.3.3): walk the active columns only, two at a time (one per half-warp); lane =
+// row tests its own row mask, so no separate column index is stored.
+template <int DT>
+__device__ __forceinline__ float mk_row_push(const uint8_t *blk, uint32_t xm, const float *s_x,
+                                             int lane, uint32_t &hits) {
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    const int row = lane & 15, half = lane >> 4;
+    const uint32_t rm = masks[row];
+    const int rp = blk[32 + row];
+    const uint8_t *vals = blk + HDR_BYTES;
+    uint32_t act = xm;
+    float sum = 0.f;
+    while (act) {
+        const int c0 = __ffs(act) - 1;
+        act &= act - 1;
+        int c1 = -1;
+        if (act) { c1 = __ffs(act) - 1; act &= act - 1; }
+        const int c = half ? c1 : c0;
+        if (c >= 0 && ((rm >> c) & 1u)) sum += Val<DT>::load(vals, rp + __popc(rm & below(c))) * s_x[c];
+    }
+    sum += __shfl_xor_sync(FULL, sum, 16);
+    hits = __ballot_sync(FULL, lane < 16 && (rm & xm) != 0);
+    return sum;
+}
+
+// Column-driven kernel for column-mask encodings (Algorithm 3): lane = row, the two
+// half-warps take columns 0..7 and 8..15.
+template <int DT>
+__device__ __forceinline__ float mk_col_push(const uint8_t *blk, uint32_t xm, const float *s_x,
+                                             int lane, uint32_t &hits) {
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    const int row = lane & 15, part = lane >> 4;
+    const uint8_t *vals = blk + HDR_BYTES;
+    uint32_t active = xm & (part ? 0xFF00u : 0x00FFu);
+    uint32_t hm = 0;
+    float sum = 0.f;
+    while (active) {
+        const int c = __ffs(active) - 1;
+        const uint32_t cm = masks[c];
+        hm |= cm;
+        if ((cm >> row) & 1u) sum += Val<DT>::load(vals, blk[32 + c] + __popc(cm & below(row))) * s_x[c];
+        active &= active - 1;
+    }
+    sum += __shfl_xor_sync(FULL, sum, 16);
+    hits = hm | __shfl_xor_sync(FULL, hm, 16);
+    return sum;
+}
+
+// Dense class: 16 column masks then 256 values column-major.  Same lane map as Algorithm 3;
+// a padding zero never contributes (its mask bit is clear), so hits stay structural.
+template <int DT>
+__device__ __forceinline__ float mk_dense(const uint8_t *blk, uint32_t xm, const float *s_x,
+                                          int lane, uint32_t &hits) {
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    const int row = lane & 15, part = lane >> 4;
+    const uint8_t *vals = blk + 32;
+    uint32_t active = xm & (part ? 0xFF00u : 0x00FFu);
+    uint32_t hm = 0;
+    float sum = 0.f;
+    while (active) {
+        const int c = __ffs(active) - 1;
+        const uint32_t cm = masks[c];
+        hm |= cm;
+        if ((cm >> row) & 1u) sum += Val<DT>::load(vals, c * 16 + row) * s_x[c];
+        active &= active - 1;
+    }
+    sum += __shfl_xor_sync(FULL, sum, 16);
+    hits = hm | __shfl_xor_sync(FULL, hm, 16);
+    return sum;
+}
+
+// Larger COO blocks: one lane per stored entry, accumulation in a 16-float shared scratch.
+template <int DT>
+__device__ __forceinline__ float mk_coo_warp(const uint8_t *blk, int nnz, uint32_t xm,
+                                             const float *s_x, float *s_tmp, int lane,
+                                             uint32_t &hits) {
+    if (lane < 16) s_tmp[lane] = 0.f;
+    __syncwarp();
+    const uint8_t *vals = blk + ((nnz + 3) & ~3);
+    uint32_t hm = 0;
+    for (int k = lane; k < nnz; k += 32) {
+        const uint32_t rc = blk[k];
+        const int c = rc & 15, r = rc >> 4;
+        if ((xm >> c) & 1u) {
+            atomicAdd(&s_tmp[r], Val<DT>::load(vals, k) * s_x[c]);
+            hm |= 1u << r;
+        }
+    }
+    hits = __reduce_or_sync(FULL, hm);
+    __syncwarp();
+    return s_tmp[lane & 15];
+}
+
+// Dispatch of the warp-cooperative kernels: block class x popc(vector-block mask).
+template <int DT>
+__device__ __forceinline__ float warp_block(int type, const uint8_t *blk, int nnz, uint32_t xm,
+                                            const float *s_x, float *s_tmp, int lane,
+                                            int popc_threshold, uint32_t &hits) {
+    switch (type) {
+        case DBSPMSPV_BLK_COO: return mk_coo_warp<DT>(blk, nnz, xm, s_x, s_tmp, lane, hits);
+        case DBSPMSPV_BLK_FCSR: return mk_row_pull<DT>(blk, xm, s_x, lane, hits);
+        case DBSPMSPV_BLK_CSR:
+            return __popc(xm) >= popc_threshold ? mk_row_pull<DT>(blk, xm, s_x, lane, hits)
+                                                : mk_row_push<DT>(blk, xm, s_x, lane, hits);
+        case DBSPMSPV_BLK_FCSC: return mk_col_push<DT>(blk, xm, s_x, lane, hits);
+        default: return mk_dense<DT>(blk, xm, s_x, lane, hits);
+    }
+}
+
+// ---- Boolean forms (Section 4.2, Algorithm 5): only reachability; values are never read.
+// Returns the mask of rows with a stored entry in an active column.
+template <int DT>
+__device__ __forceinline__ uint32_t warp_block_bool(int type, const uint8_t *blk, int nnz,
+                                                    uint32_t xm, int lane) {
+    constexpr bool HAS_STARTS = Val<DT>::SIZE != 0;
+    (void)HAS_STARTS;
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    if (type == DBSPMSPV_BLK_COO) {
+        uint32_t hm = 0;
+        for (int k = lane; k < nnz; k += 32) {
+            const uint32_t rc = blk[k];
+            if ((xm >> (rc & 15)) & 1u) hm |= 1u << (rc >> 4);
+        }
+        return __reduce_or_sync(FULL, hm);
+    }
+    if (type == DBSPMSPV_BLK_FCSR || type == DBSPMSPV_BLK_CSR)
+        return __ballot_sync(FULL, lane < 16 && (masks[lane & 15] & xm) != 0);
+    // column masks: OR of the active columns' masks
+    uint32_t hm = (lane < 16 && ((xm >> lane) & 1u)) ? masks[lane] : 0u;
+    return __reduce_or_sync(FULL, hm);
+}
+
+}  // namespace dbs

@@ -1,0 +1,544 @@
+// One SpMSpV call (Sections 3.3 and 4.1): vector blocking + push worklist, device-side path
+// selection, push / pull traversal with per-block microkernels, hierarchical writeback, and
+// compaction of the dense accumulator into a sorted sparse y.  Also the dense-in / dense-out
+// decode entry (Section 4.3).  Nothing here allocates or synchronises.
+#include "internal.cuh"
+#include "microkernels.cuh"
+
+namespace dbs {
+
+constexpr int CTA = 128;            // four warps per thread block (Section 3.3.2)
+constexpr int WARPS = CTA / 32;
+constexpr int CMP_TPB = 256;        // compaction: threads per tile
+constexpr int CMP_WORDS = 4;        // 32-bit mask words per thread
+constexpr int TILE_WORDS = CMP_TPB * CMP_WORDS;
+
+// ------------------------------------------------------------------------------------------
+// Vector blocking (Section 3.2.2) fused with the push worklist (Section 3.3.2).
+// Sparse input: one thread per listed nonzero scatters the value into the dense copy and sets
+// its mask bit; the thread that turns a vector block from empty to nonempty emits the block's
+// push tasks (runs of <= 32 entries of its block-CSC column).  Space in the worklist is
+// claimed with one warp scan and one atomic per warp; the count of nonempty vector blocks is
+// aggregated the same way (Section 4.1).
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int lane) {
+    int first = 0, nchunks = 0;
+    if (newly) {
+        first = d.csc.ptr[jb];
+        nchunks = (d.csc.ptr[jb + 1] - first + PUSH_CHUNK - 1) / PUSH_CHUNK;
+    }
+    int incl = nchunks;
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(FULL, incl, o);
+        if (lane >= o) incl += t;
+    }
+    const int total = __shfl_sync(FULL, incl, 31);
+    const int n_new = __popc(__ballot_sync(FULL, newly));
+    int base = 0;
+    if (lane == 0 && n_new) {
+        if (total) base = atomicAdd(&d.ws.ctr->n_tasks, total);
+        atomicAdd(&d.ws.ctr->n_nzblk, n_new);
+    }
+    base = __shfl_sync(FULL, base, 0) + incl - nchunks;
+    for (int k = 0; k < nchunks; ++k) d.ws.tasks[base + k] = make_uint2((uint32_t)jb, (uint32_t)(first + k * PUSH_CHUNK));
+}
+
+template <int DT>
+__global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, const void *__restrict__ x_val,
+                                int32_t nnz_x, int validate) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    bool newly = false;
+    int jb = 0;
+    if (t < nnz_x) {
+        const int j = x_idx[t];
+        if (validate && (j < 0 || j >= d.n)) {
+            d.ws.ctr->status = DBSPMSPV_ERR_BOUNDS;
+        } else {
+            float v = 1.0f;
+            if (x_val) {
+                if (DT == DBSPMSPV_BF16) v = __bfloat162float(static_cast<const __nv_bfloat16 *>(x_val)[t]);
+                else v = static_cast<const float *>(x_val)[t];
+            }
+            d.ws.x_dense[j] = v;
+            const int sh = ((j >> 4) & 1) * 16;
+            const uint32_t old = atomicOr(&d.ws.x_mask32[j >> 5], 1u << ((j & 15) + sh));
+            newly = ((old >> sh) & 0xFFFFu) == 0;
+            jb = j >> 4;
+        }
+    }
+    emit_tasks(d, newly, jb, lane);
+}
+
+// Dense input (Sections 4.1, 4.3): every warp reads 32 elements, one ballot gives the two
+// 16-bit masks of its two vector blocks.  Also clears the dense output.
+template <int DT>
+__global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__restrict__ y) {
+    const int lane = threadIdx.x & 31;
+    const int64_t padded = (int64_t)((d.nb + 1) / 2) * 32;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < padded; j += stride) {
+        float v = 0.f;
+        if (j < d.n) v = DT == DBSPMSPV_BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(x)[j])
+                                             : static_cast<const float *>(x)[j];
+        if (j < (int64_t)d.nb * 16) d.ws.x_dense[j] = v;
+        const uint32_t bits = __ballot_sync(FULL, v != 0.0f);
+        if (lane == 0) d.ws.x_mask32[j >> 5] = bits;
+        const bool newly = (lane == 0 && (bits & 0xFFFFu)) || (lane == 16 && (bits >> 16));
+        emit_tasks(d, newly, (int)(j >> 4), lane);
+    }
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < d.m; i += stride) y[i] = 0.f;
+}
+
+// ------------------------------------------------------------------------------------------
+// Traversal.  Output goes through `Out`: the sparse path accumulates into the handle's dense
+// accumulator and structural-hit masks; the decode path adds straight into the caller's y.
+// ------------------------------------------------------------------------------------------
+struct OutSparse {
+    float *acc;
+    uint32_t *mask32;
+    static constexpr bool MASKS = true;
+};
+struct OutDense {
+    float *acc;
+    uint32_t *mask32;
+    static constexpr bool MASKS = false;
+};
+
+// One lane owns one hypersparse block (INLINE or small COO).  `emit(r, v)` receives every
+// product; returns the structural-hit row mask.
+template <int DT, typename Emit>
+__device__ __forceinline__ uint32_t lane_block(int type, uint32_t w, uint32_t aux, uint32_t xm,
+                                               const float *xb, const uint8_t *payload, Emit emit) {
+    uint32_t hit = 0;
+    if (type == DBSPMSPV_BLK_INLINE) {
+        if (DT == DBSPMSPV_PATTERN) {
+            for (uint32_t k = 0; k <= aux; ++k) {
+                const uint32_t rc = (w >> (8 * k)) & 0xFFu;
+                if ((xm >> (rc & 15)) & 1u) hit |= 1u << (rc >> 4);
+            }
+        } else {
+            const int c = aux & 15, r = aux >> 4;
+            if ((xm >> c) & 1u) { emit(r, Val<DT>::inline_value(w) * xb[c]); hit = 1u << r; }
+        }
+    } else {  // small COO, row-major: products of one row are summed before they are emitted
+        const int nnz = (int)aux + 1;
+        const uint8_t *blk = payload + (size_t)w * 4;
+        const uint8_t *vals = blk + ((nnz + 3) & ~3);
+        int cur = -1;
+        float s = 0.f;
+        for (int k = 0; k < nnz; ++k) {
+            const uint32_t rc = blk[k];
+            const int c = rc & 15, r = rc >> 4;
+            if ((xm >> c) & 1u) {
+                if (DT != DBSPMSPV_PATTERN) {
+                    if (r != cur) { if (cur >= 0) emit(cur, s); cur = r; s = 0.f; }
+                    s += Val<DT>::load(vals, k) * xb[c];
+                }
+                hit |= 1u << r;
+            }
+        }
+        if (DT != DBSPMSPV_PATTERN && cur >= 0) emit(cur, s);
+    }
+    return hit;
+}
+
+// Push (Section 3.3.2): every warp takes one task = up to 32 consecutive block-CSC entries of
+// one active column block; the vector block is staged once per task (Section 3.3.3).  Lanes
+// own hypersparse blocks; heavier blocks are then processed by the whole warp one at a time.
+// Writeback: warp-level reduction, then one global atomic per touched row and one atomicOr on
+// the row block's hit mask.
+template <int DT, typename Out>
+__device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp) {
+    const int lane = threadIdx.x & 31;
+    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int n_tasks = d.ws.ctr->n_tasks;
+    for (int t = gwarp; t < n_tasks; t += nwarps) {
+        const uint2 task = d.ws.tasks[t];
+        const int jb = (int)task.x;
+        const int start = (int)task.y;
+        const int end = min(start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
+        const uint32_t xm = mask_of(d.ws.x_mask32, jb);
+        if (lane < 16) s_x[lane] = d.ws.x_dense[jb * 16 + lane];
+        __syncwarp();
+        const int p = start + lane;
+        bool heavy = false;
+        uint32_t idx = 0, w = 0, aux = 0;
+        if (p < end) {
+            idx = d.csc.idx[p]; w = d.csc.w[p]; aux = d.csc.aux[p];
+            const int type = idx >> TYPE_SHIFT;
+            const int brow = idx & IDX_MASK;
+            if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX)) {
+                float *row0 = out.acc + (size_t)brow * 16;
+                const uint32_t hit = lane_block<DT>(type, w, aux, xm, s_x, d.payload,
+                                                    [&](int r, float v) { atomicAdd(row0 + r, v); });
+                if (Out::MASKS && hit) atomicOr(&out.mask32[brow >> 1], hit << ((brow & 1) * 16));
+            } else {
+                heavy = true;
+            }
+        }
+        uint32_t hv = __ballot_sync(FULL, heavy);
+        while (hv) {
+            const int src = __ffs(hv) - 1;
+            hv &= hv - 1;
+            const uint32_t bidx = __shfl_sync(FULL, idx, src);
+            const uint32_t bw = __shfl_sync(FULL, w, src);
+            const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
+            const int type = bidx >> TYPE_SHIFT;
+            const int brow = bidx & IDX_MASK;
+            const uint8_t *blk = d.payload + (size_t)bw * 4;
+            uint32_t hits;
+            if (DT == DBSPMSPV_PATTERN) {
+                hits = warp_block_bool<DT>(type, blk, nnz, xm, lane);
+            } else {
+                const float sum = warp_block<DT>(type, blk, nnz, xm, s_x, s_tmp, lane, popc_threshold, hits);
+                if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(out.acc + (size_t)brow * 16 + lane, sum);
+            }
+            if (Out::MASKS && lane == 0 && hits) atomicOr(&out.mask32[brow >> 1], hits << ((brow & 1) * 16));
+        }
+        __syncwarp();
+    }
+}
+
+// Pull (Section 3.3.2): every warp takes one load-weighted segment of a row block and keeps
+// the 16 partial sums of that row block in shared memory; blocks whose vector block is empty
+// are skipped on their mask.  A segment that covers its whole row block writes with plain
+// stores; split row blocks fall back to atomics.
+template <int DT, typename Out>
+__device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp,
+                          float *s_y) {
+    const int lane = threadIdx.x & 31;
+    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (int sg = gwarp; sg < d.n_segments; sg += nwarps) {
+        const Segment seg = d.segments[sg];
+        const int rb = seg.row_block;
+        const bool whole = seg.count < 0;
+        const int end = seg.start + (seg.count & 0x7FFFFFFF);
+        if (lane < 16) s_y[lane] = 0.f;
+        __syncwarp();
+        uint32_t hit = 0;
+        for (int base = seg.start; base < end; base += 32) {
+            const int p = base + lane;
+            bool heavy = false;
+            uint32_t idx = 0, w = 0, aux = 0, xm = 0;
+            if (p < end) {
+                idx = d.csr.idx[p];
+                const int bcol = idx & IDX_MASK;
+                xm = mask_of(d.ws.x_mask32, bcol);
+                if (xm) {
+                    w = d.csr.w[p]; aux = d.csr.aux[p];
+                    const int type = idx >> TYPE_SHIFT;
+                    if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX)) {
+                        hit |= lane_block<DT>(type, w, aux, xm, d.ws.x_dense + (size_t)bcol * 16, d.payload,
+                                              [&](int r, float v) { atomicAdd(&s_y[r], v); });
+                    } else {
+                        heavy = true;
+                    }
+                }
+            }
+            uint32_t hv = __ballot_sync(FULL, heavy);
+            while (hv) {
+                const int src = __ffs(hv) - 1;
+                hv &= hv - 1;
+                const uint32_t bidx = __shfl_sync(FULL, idx, src);
+                const uint32_t bw = __shfl_sync(FULL, w, src);
+                const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
+                const uint32_t bxm = __shfl_sync(FULL, xm, src);
+                const int type = bidx >> TYPE_SHIFT;
+                const int bcol = bidx & IDX_MASK;
+                const uint8_t *blk = d.payload + (size_t)bw * 4;
+                uint32_t hits;
+                if (DT == DBSPMSPV_PATTERN) {
+                    hits = warp_block_bool<DT>(type, blk, nnz, bxm, lane);
+                } else {
+                    __syncwarp();
+                    if (lane < 16) s_x[lane] = d.ws.x_dense[(size_t)bcol * 16 + lane];
+                    __syncwarp();
+                    const float sum = warp_block<DT>(type, blk, nnz, bxm, s_x, s_tmp, lane, popc_threshold, hits);
+                    if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(&s_y[lane], sum);
+                }
+                hit |= hits;
+            }
+        }
+        hit = __reduce_or_sync(FULL, hit);
+        __syncwarp();
+        if (DT != DBSPMSPV_PATTERN && lane < 16 && ((hit >> lane) & 1u)) {
+            float *dst = out.acc + (size_t)rb * 16 + lane;
+            if (whole) *dst = s_y[lane]; else atomicAdd(dst, s_y[lane]);
+        }
+        if (Out::MASKS && lane == 0 && hit) {
+            if (whole) reinterpret_cast<uint16_t *>(out.mask32)[rb] = (uint16_t)hit;
+            else atomicOr(&out.mask32[rb >> 1], hit << ((rb & 1) * 16));
+        }
+        __syncwarp();
+    }
+}
+
+// Global selector (Section 3.3.1): s_b = N_nzblk / N_blk; push iff s_b < th3.  Evaluated on
+// the device by every thread block from the counter the blocking kernel produced.
+__device__ __forceinline__ int select_path(const Device &d, float th3, int force_path) {
+    if (force_path == DBSPMSPV_PATH_PUSH || force_path == DBSPMSPV_PATH_PULL) return force_path;
+    const float sb = (float)d.ws.ctr->n_nzblk / (float)d.nb;
+    return sb < th3 ? DBSPMSPV_PATH_PUSH : DBSPMSPV_PATH_PULL;
+}
+
+template <int DT, typename Out>
+__global__ void __launch_bounds__(CTA) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
+    __shared__ float s_x[WARPS][16], s_tmp[WARPS][16], s_y[WARPS][16];
+    const int warp = threadIdx.x >> 5;
+    const int path = select_path(d, th3, force_path);
+    if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
+    if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp]);
+    else pull_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp]);
+}
+
+// ------------------------------------------------------------------------------------------
+// Output compaction: the hit masks of the row blocks are scanned in order, so y comes out
+// sorted.  Pass 1 counts per tile, pass 2 places the entries, clears the accumulator and the
+// masks it read, clears the vector-block state of this call's x, and rolls the counters over.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(CMP_TPB) k_compact_count(Device d) {
+    __shared__ int s_red[CMP_TPB / 32];
+    const int n_words = (d.mb + 1) / 2;
+    const int w0 = (blockIdx.x * CMP_TPB + threadIdx.x) * CMP_WORDS;
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < CMP_WORDS; ++k)
+        if (w0 + k < n_words) c += __popc(d.ws.y_mask32[w0 + k]);
+    c = __reduce_add_sync(FULL, c);
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int k = 0; k < CMP_TPB / 32; ++k) t += s_red[k];
+        d.ws.tile_count[blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__restrict__ y_idx, float *__restrict__ y_val,
+                                                           int64_t y_capacity, int32_t *__restrict__ y_nnz, int boolean,
+                                                           const int32_t *__restrict__ x_idx, int32_t nnz_x) {
+    __shared__ int s_red[CMP_TPB / 32];
+    __shared__ int s_base;
+    const int n_tiles = d.ws.n_tiles;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if ((int)blockIdx.x < n_tiles) {
+        // entries in all earlier tiles
+        int before = 0;
+        for (int k = threadIdx.x; k < (int)blockIdx.x; k += CMP_TPB) before += d.ws.tile_count[k];
+        before = __reduce_add_sync(FULL, before);
+        if (lane == 0) s_red[warp] = before;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int t = 0;
+            for (int k = 0; k < CMP_TPB / 32; ++k) t += s_red[k];
+            s_base = t;
+        }
+        __syncthreads();
+        const int n_words = (d.mb + 1) / 2;
+        const int w0 = (blockIdx.x * CMP_TPB + threadIdx.x) * CMP_WORDS;
+        uint32_t words[CMP_WORDS];
+        int c = 0;
+#pragma unroll
+        for (int k = 0; k < CMP_WORDS; ++k) {
+            words[k] = w0 + k < n_words ? d.ws.y_mask32[w0 + k] : 0u;
+            c += __popc(words[k]);
+        }
+        int incl = c;
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(FULL, incl, o);
+            if (lane >= o) incl += t;
+        }
+        __syncthreads();
+        if (lane == 31) s_red[warp] = incl;
+        __syncthreads();
+        int pos = s_base + incl - c;
+        for (int k = 0; k < warp; ++k) pos += s_red[k];
+        if (c) {
+#pragma unroll
+            for (int k = 0; k < CMP_WORDS; ++k) {
+                uint32_t wd = words[k];
+                if (wd) d.ws.y_mask32[w0 + k] = 0u;
+                while (wd) {
+                    const int bit = __ffs(wd) - 1;
+                    wd &= wd - 1;
+                    const int row = (w0 + k) * 32 + bit;
+                    const float v = d.ws.y_acc[row];
+                    d.ws.y_acc[row] = 0.f;
+                    if (pos < y_capacity) {
+                        y_idx[pos] = row;
+                        if (y_val) y_val[pos] = boolean ? 1.0f : v;
+                    }
+                    ++pos;
+                }
+            }
+        }
+        if ((int)blockIdx.x == n_tiles - 1 && threadIdx.x == CMP_TPB - 1) {
+            Counters *c2 = d.ws.ctr;
+            *y_nnz = pos;
+            if (pos > y_capacity) c2->status = DBSPMSPV_ERR_CAPACITY;
+            c2->last_y_nnz = pos;
+            c2->last_n_nzblk = c2->n_nzblk;
+            c2->last_n_tasks = c2->n_tasks;
+            c2->last_path = c2->path;
+            c2->n_nzblk = 0;
+            c2->n_tasks = 0;
+        }
+    }
+    // vector-block state of this call's x: clear the masks (the dense copy may keep stale
+    // values; it is only ever read under a mask bit)
+    const int stride = gridDim.x * CMP_TPB;
+    for (int k = blockIdx.x * CMP_TPB + threadIdx.x; k < nnz_x; k += stride) {
+        const int j = x_idx[k];
+        if (j >= 0 && j < d.n) d.ws.x_mask32[j >> 5] = 0u;
+    }
+}
+
+__global__ void k_decode_cleanup(Device d) {
+    const int n_words = (d.nb + 1) / 2;
+    const int stride = gridDim.x * blockDim.x;
+    for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n_words; k += stride) d.ws.x_mask32[k] = 0u;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        Counters *c = d.ws.ctr;
+        c->last_n_nzblk = c->n_nzblk;
+        c->last_n_tasks = c->n_tasks;
+        c->last_path = c->path;
+        c->last_y_nnz = (int32_t)d.m;
+        c->n_nzblk = 0;
+        c->n_tasks = 0;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+template <typename T> static int dev_alloc_zero(T **p, size_t count, int64_t *total) {
+    void *q = nullptr;
+    size_t bytes = (count ? count : 1) * sizeof(T);
+    if (cudaMalloc(&q, bytes) != cudaSuccess) return DBSPMSPV_ERR_ALLOC;
+    if (cudaMemset(q, 0, bytes) != cudaSuccess) return DBSPMSPV_ERR_CUDA;
+    *p = static_cast<T *>(q);
+    *total += (int64_t)bytes;
+    return DBSPMSPV_OK;
+}
+
+template <int DT, typename Out> static int compute_grid(int sm_count) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_compute<DT, Out>, CTA, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    return sm_count * per_sm;
+}
+
+int allocate_workspace(dbspmspv_handle_s *h) {
+    Device &d = h->d;
+    Workspace &ws = d.ws;
+    int64_t total = 0;
+    const size_t xwords = (size_t)(d.nb + 1) / 2 + 4, ywords = (size_t)(d.mb + 1) / 2 + 4;
+    ws.task_capacity = (int64_t)d.n_blocks / PUSH_CHUNK + d.nb + 32;
+    ws.n_tiles = (int32_t)ceil_div<int64_t>((d.mb + 1) / 2, TILE_WORDS);
+    if (ws.n_tiles < 1) ws.n_tiles = 1;
+#define DBS_WS(expr) do { int s__ = (expr); if (s__ != DBSPMSPV_OK) return s__; } while (0)
+    DBS_WS(dev_alloc_zero(&ws.x_dense, xwords * 32, &total));
+    DBS_WS(dev_alloc_zero(&ws.x_mask32, xwords, &total));
+    DBS_WS(dev_alloc_zero(&ws.tasks, (size_t)ws.task_capacity, &total));
+    DBS_WS(dev_alloc_zero(&ws.y_acc, ywords * 32, &total));
+    DBS_WS(dev_alloc_zero(&ws.y_mask32, ywords, &total));
+    DBS_WS(dev_alloc_zero(&ws.tile_count, (size_t)ws.n_tiles, &total));
+    DBS_WS(dev_alloc_zero(&ws.visited32, d.m == d.n ? ywords : 1, &total));
+    DBS_WS(dev_alloc_zero(&ws.ctr, 1, &total));
+#undef DBS_WS
+    h->stats.workspace_bytes = total;
+    return DBSPMSPV_OK;
+}
+
+template <int DT>
+static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
+                     int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
+                     cudaStream_t st) {
+    const Device &d = h->d;
+    static int grid = 0;
+    if (!grid) grid = compute_grid<DT, OutSparse>(h->sm_count);
+    if (nnz_x > 0) k_xblock_sparse<DT><<<(nnz_x + 255) / 256, 256, 0, st>>>(d, x_idx, semiring == DBSPMSPV_OR_AND ? nullptr : x_val, nnz_x, h->ropts.validate);
+    OutSparse out{d.ws.y_acc, d.ws.y_mask32};
+    if (nnz_x > 0 && d.n_blocks > 0) k_compute<DT, OutSparse><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold);
+    const int nt = d.ws.n_tiles;
+    k_compact_count<<<nt, CMP_TPB, 0, st>>>(d);
+    int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
+    if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
+    k_compact_write<<<nt + extra, CMP_TPB, 0, st>>>(d, y_idx, y_val, y_capacity, y_nnz, semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN, x_idx, nnz_x);
+    DBS_CUDA(cudaGetLastError());
+    return DBSPMSPV_OK;
+}
+
+template <int DT>
+static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStream_t st) {
+    const Device &d = h->d;
+    static int grid = 0;
+    if (!grid) grid = compute_grid<DT, OutDense>(h->sm_count);
+    const int64_t padded = (int64_t)((d.nb + 1) / 2) * 32;
+    int64_t work = padded > d.m ? padded : d.m;
+    int g = (int)((work + 255) / 256);
+    if (g > 8 * h->sm_count) g = 8 * h->sm_count;
+    k_xblock_dense<DT><<<g, 256, 0, st>>>(d, x, y);
+    OutDense out{y, nullptr};
+    if (d.n_blocks > 0) k_compute<DT, OutDense><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold);
+    int gc = ((d.nb + 1) / 2 + 255) / 256;
+    if (gc > h->sm_count) gc = h->sm_count;
+    k_decode_cleanup<<<gc, 256, 0, st>>>(d);
+    DBS_CUDA(cudaGetLastError());
+    return DBSPMSPV_OK;
+}
+
+}  // namespace dbs
+
+extern "C" {
+
+void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
+    if (!o) return;
+    *o = dbspmspv_run_opts();
+    o->th3 = 0.01f;
+    o->force_path = DBSPMSPV_PATH_AUTO;
+    o->popc_threshold = 8;
+    o->validate = 0;
+}
+
+int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts) {
+    if (!h || !opts) return DBSPMSPV_ERR_INVALID_ARG;
+    if (opts->force_path < DBSPMSPV_PATH_AUTO || opts->force_path > DBSPMSPV_PATH_PULL) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!(opts->th3 >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
+    h->ropts = *opts;
+    return DBSPMSPV_OK;
+}
+
+int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
+                 int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
+                 dbspmspv_stream_t stream) {
+    if (!h || nnz_x < 0 || y_capacity < 0 || !y_nnz) return DBSPMSPV_ERR_INVALID_ARG;
+    if (nnz_x > 0 && !x_idx) return DBSPMSPV_ERR_INVALID_ARG;
+    if (y_capacity > 0 && !y_idx) return DBSPMSPV_ERR_INVALID_ARG;
+    if (semiring != DBSPMSPV_PLUS_TIMES && semiring != DBSPMSPV_OR_AND) return DBSPMSPV_ERR_INVALID_ARG;
+    if (semiring == DBSPMSPV_PLUS_TIMES) {
+        if (h->d.dtype == DBSPMSPV_PATTERN) return DBSPMSPV_ERR_UNSUPPORTED;
+        if ((nnz_x > 0 && !x_val) || (y_capacity > 0 && !y_val)) return DBSPMSPV_ERR_INVALID_ARG;
+    }
+    if ((int64_t)nnz_x > h->d.n) return DBSPMSPV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (h->d.dtype) {
+        case DBSPMSPV_F32: return dbs::run_typed<DBSPMSPV_F32>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
+        case DBSPMSPV_BF16: return dbs::run_typed<DBSPMSPV_BF16>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
+        default: return dbs::run_typed<DBSPMSPV_PATTERN>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
+    }
+}
+
+int dbspmspv_decode(dbspmspv_handle_t h, const void *x, float *y, dbspmspv_stream_t stream) {
+    if (!h || !x || !y) return DBSPMSPV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (h->d.dtype) {
+        case DBSPMSPV_F32: return dbs::decode_typed<DBSPMSPV_F32>(h, x, y, st);
+        case DBSPMSPV_BF16: return dbs::decode_typed<DBSPMSPV_BF16>(h, x, y, st);
+        default: return DBSPMSPV_ERR_UNSUPPORTED;
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,220 @@
+"""GPU parity of dbspmspv_run against the CPU oracle: structural index set identical, values
+within 2e-5 * sum|a x|, for forced push, forced pull and the automatic selector, every block
+format variant and every value type, including empty and ragged inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_16308_b200 import binding as B
+from paper_2608_16308_b200 import workloads as wl
+from gpu_util import Handle, check_against_oracle, ref_matrix
+from test_gpu_format import mixed_matrix
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [B.PATH_AUTO, B.PATH_PUSH, B.PATH_PULL]
+
+
+def dense_x(n, seed, frac):
+    k = max(1, int(n * frac))
+    return wl.sparse_x(seed, 0, n, k)
+
+
+MATS = [
+    ("uniform300x200", lambda: wl.random_sparse(300, 200, 4000, 1)),
+    ("ragged77x131", lambda: wl.random_sparse(77, 131, 900, 2)),
+    ("mixed", lambda: mixed_matrix(96, 112, 3)),
+    ("rmat12", lambda: wl.rmat(12, 16, seed=1)),
+    ("stencil16", lambda: wl.stencil27(16, seed=2)),
+    ("wide", lambda: wl.random_sparse(40, 5000, 6000, 5)),
+    ("tall", lambda: wl.random_sparse(5000, 40, 6000, 6)),
+]
+
+
+@pytest.mark.parametrize("name,make", MATS, ids=[m[0] for m in MATS])
+@pytest.mark.parametrize("dtype", [B.F32, B.BF16])
+def test_parity_all_paths(name, make, dtype):
+    csr = make()
+    h = Handle(csr, dtype)
+    A = ref_matrix(csr, bf16=dtype == B.BF16)
+    for frac in (0.002, 0.05, 0.5, 1.0):
+        x = dense_x(csr.n, 7, frac)
+        if dtype == B.BF16:
+            x.val = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x.val))
+        want = oracle.ref_pull(A, x.idx, x.val)
+        for path in PATHS:
+            for thr in (1, 8, 17):
+                h.set_opts(force_path=path, popc_threshold=thr)
+                check_against_oracle(h.run(x), want)
+                st = h.get_stats()
+                if path != B.PATH_AUTO:
+                    assert st.last_path == path
+                assert st.last_n_nzblk == np.unique(x.idx >> 4).size
+                assert st.last_y_nnz == want[0].size
+    h.close()
+
+
+@pytest.mark.parametrize("fmt", [B.FORMAT_COO, B.FORMAT_CSR])
+def test_forced_single_format_equals_auto(fmt):
+    csr = mixed_matrix(96, 112, 3)
+    o = B.default_create_opts()
+    o.force_format = fmt
+    h = Handle(csr, B.F32, opts=o)
+    A = ref_matrix(csr)
+    for frac in (0.05, 0.6):
+        x = dense_x(csr.n, 11, frac)
+        want = oracle.ref_pull(A, x.idx, x.val)
+        for path in (B.PATH_PUSH, B.PATH_PULL):
+            h.set_opts(force_path=path)
+            check_against_oracle(h.run(x), want)
+    h.close()
+
+
+def test_selector_follows_the_block_ratio_rule():
+    """push iff N_nzblk / N_blk < th3, evaluated in fp32 from the same integers."""
+    csr = wl.random_sparse(4096, 4096, 30000, 3)
+    h = Handle(csr, B.F32)
+    nblk = (csr.n + 15) // 16
+    for k in (1, 2, 3, 5, 40, 400):
+        x = wl.sparse_x(50 + k, 0, csr.n, k)
+        nz = np.unique(x.idx >> 4).size
+        for th3 in (0.01, 0.005, 0.5):
+            h.set_opts(th3=th3)
+            h.run(x)
+            st = h.get_stats()
+            assert st.last_n_nzblk == nz
+            want = B.PATH_PUSH if np.float32(nz) / np.float32(nblk) < np.float32(th3) else B.PATH_PULL
+            assert st.last_path == want
+    h.close()
+
+
+def test_boolean_semiring_on_pattern_and_valued_handles():
+    csr = wl.rmat(11, 8, seed=5)
+    A = ref_matrix(csr)
+    x = dense_x(csr.n, 3, 0.03)
+    want = oracle.ref_pull(A, x.idx, None)
+    for dtype in (B.PATTERN, B.F32):
+        h = Handle(csr, dtype)
+        for path in PATHS:
+            h.set_opts(force_path=path)
+            check_against_oracle(h.run(x, semiring=B.OR_AND), want, boolean=True)
+        h.close()
+    h = Handle(csr, B.PATTERN)
+    xi = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.DbSpmspvError) as e:
+        B.dbspmspv_run(h.h, xi, xi.float(), 4, B.PLUS_TIMES, h.y_idx, h.y_val, 10, h.y_nnz)
+    assert e.value.status == B.ERR_UNSUPPORTED
+    h.close()
+
+
+def test_empty_x_and_empty_matrix_and_isolated_columns():
+    csr = wl.random_sparse(100, 100, 300, 8)
+    h = Handle(csr, B.F32)
+    yi, yv, k = h.run(wl.SparseVec(100, np.zeros(0, np.int32), np.zeros(0, np.float32)))
+    assert k == 0 and yi.size == 0
+    # x listed only on columns that hold no entry
+    empty_cols = np.setdiff1d(np.arange(100), csr.col_idx)[:5].astype(np.int32)
+    assert empty_cols.size > 0
+    for path in PATHS:
+        h.set_opts(force_path=path)
+        yi, yv, k = h.run(wl.SparseVec(100, empty_cols, np.ones(empty_cols.size, np.float32)))
+        assert k == 0
+    h.close()
+    e = wl.CSR(50, 60, np.zeros(51, np.int64), np.zeros(0, np.int32), np.zeros(0, np.float32))
+    h = Handle(e, B.F32)
+    assert h.stats.n_blocks == 0
+    yi, yv, k = h.run(wl.sparse_x(1, 0, 60, 10))
+    assert k == 0
+    h.close()
+
+
+def test_state_is_clean_between_calls():
+    """Back-to-back calls with different x on one handle: nothing leaks from the previous call
+    (accumulator, hit masks, vector-block masks, worklist)."""
+    csr = wl.rmat(12, 16, seed=2)
+    h = Handle(csr, B.F32)
+    A = ref_matrix(csr)
+    for rep, (frac, path) in enumerate([(0.3, B.PATH_PUSH), (0.001, B.PATH_PULL), (0.02, B.PATH_PUSH),
+                                        (0.5, B.PATH_PULL), (0.0005, B.PATH_PUSH)]):
+        x = dense_x(csr.n, 20 + rep, frac)
+        h.set_opts(force_path=path)
+        check_against_oracle(h.run(x), oracle.ref_pull(A, x.idx, x.val))
+    h.close()
+
+
+def test_capacity_overflow_is_reported_not_written():
+    csr = wl.random_sparse(500, 500, 5000, 4)
+    h = Handle(csr, B.F32)
+    x = dense_x(csr.n, 5, 0.2)
+    want = oracle.ref_pull(ref_matrix(csr), x.idx, x.val)
+    cap = want[0].size // 2
+    h.y_idx.fill_(-1)
+    yi, yv, k = h.run(x, capacity=cap)
+    assert k == want[0].size                                  # full count is still reported
+    assert np.array_equal(yi, want[0][:cap])
+    assert (h.y_idx[cap:].cpu().numpy() == -1).all()          # nothing beyond capacity
+    st = h.get_stats(raise_on_device_status=False)
+    assert st.device_status == B.ERR_CAPACITY
+    assert h.get_stats().device_status == B.OK                # reported once, then cleared
+    check_against_oracle(h.run(x), want)                      # the handle stays usable
+    h.close()
+
+
+def test_validate_flags_out_of_range_index():
+    csr = wl.random_sparse(100, 100, 300, 8)
+    h = Handle(csr, B.F32)
+    h.set_opts(validate=1)
+    x = wl.SparseVec(100, np.array([1, 5000, 7], np.int32), np.ones(3, np.float32))
+    h.run(x)
+    assert h.get_stats(raise_on_device_status=False).device_status == B.ERR_BOUNDS
+    h.close()
+
+
+def test_identity_permutation_and_block_diagonal_dense():
+    n = 333
+    eye = wl.CSR(n, n, np.arange(n + 1, dtype=np.int64), np.arange(n, dtype=np.int32), np.ones(n, np.float32))
+    h = Handle(eye, B.F32)
+    x = wl.sparse_x(3, 0, n, 50)
+    order = np.argsort(x.idx)
+    for path in PATHS:
+        h.set_opts(force_path=path)
+        yi, yv, k = h.run(x)
+        assert np.array_equal(yi, x.idx[order]) and np.array_equal(yv, x.val[order])   # bit exact
+    h.close()
+    # block-diagonal matrix of dense 16 x 16 blocks == a small dense GEMV per block
+    nb = 6
+    a = np.zeros((16 * nb, 16 * nb), dtype=np.float32)
+    for b in range(nb):
+        a[16 * b:16 * b + 16, 16 * b:16 * b + 16] = wl.rand_f32(5, b, np.arange(256, dtype=np.uint64)).reshape(16, 16) + 0.1
+    csr = wl.csr_from_dense(a)
+    h = Handle(csr, B.F32)
+    assert h.stats.class_blocks[B.BLK_DENSE] == nb
+    x = wl.sparse_x(8, 0, 16 * nb, 40)
+    xd = np.zeros(16 * nb)
+    xd[x.idx] = x.val
+    want = a.astype(np.float64) @ xd
+    for path in PATHS:
+        h.set_opts(force_path=path)
+        yi, yv, k = h.run(x)
+        assert np.allclose(yv, want[yi], rtol=0, atol=2e-5 * (np.abs(a) @ np.abs(xd)).max())
+    h.close()
+
+
+def test_stencil_unit_values_give_integer_neighbour_counts():
+    """0/1-valued stencil with x = ones on a full grid line: y counts neighbours on the line
+    (exact in fp32)."""
+    d = 16
+    csr = wl.stencil27(d, values=False)
+    csr.val = np.ones(csr.nnz, dtype=np.float32)
+    h = Handle(csr, B.F32)
+    line = (np.arange(d) + d * (5 + d * 7)).astype(np.int32)        # y = 5, z = 7
+    x = wl.SparseVec(csr.n, line, np.ones(d, np.float32))
+    for path in PATHS:
+        h.set_opts(force_path=path)
+        yi, yv, k = h.run(x)
+        assert k == 9 * d                                           # the 3 x 3 tube around the line
+        xs = yi % d
+        want = 3 - (xs == 0) - (xs == d - 1)
+        assert np.array_equal(yv, want.astype(np.float32))
+    h.close()
