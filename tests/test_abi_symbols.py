@@ -44,7 +44,7 @@ def test_struct_layouts_match_the_header():
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     for cname, cls in (("dbspmspv_create_opts", B.CreateOpts), ("dbspmspv_run_opts", B.RunOpts),
                        ("dbspmspv_stats", B.Stats)):
-        body = re.search(r"typedef struct \{(.*?)\}\s*" + cname + ";", text, flags=re.S).group(1)
+        body = re.search(r"typedef struct \{([^}]*)\}\s*" + cname + ";", text).group(1)
         fields = []
         for decl in body.split(";"):
             decl = decl.strip()
