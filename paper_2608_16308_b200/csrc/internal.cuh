@@ -62,6 +62,7 @@ struct Counters {    // device-resident scalars of one call
     int32_t last_n_nzblk, last_n_tasks, last_path, last_y_nnz;
     int32_t bfs_levels, bfs_reached;
     int32_t pad;
+    int32_t bfs_cnt[2][2];  // BFS: {nonempty frontier blocks, tasks}, double buffered by level
     int32_t bfs_level_path[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
     int32_t bfs_level_nzblk[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
 };

@@ -4,6 +4,7 @@
 // decode entry (Section 4.3).  Nothing here allocates or synchronises.
 #include "internal.cuh"
 #include "microkernels.cuh"
+#include "worklist.cuh"
 
 namespace dbs {
 
@@ -21,28 +22,6 @@ constexpr int TILE_WORDS = CMP_TPB * CMP_WORDS;
 // claimed with one warp scan and one atomic per warp; the count of nonempty vector blocks is
 // aggregated the same way (Section 4.1).
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int lane) {
-    int first = 0, nchunks = 0;
-    if (newly) {
-        first = d.csc.ptr[jb];
-        nchunks = (d.csc.ptr[jb + 1] - first + PUSH_CHUNK - 1) / PUSH_CHUNK;
-    }
-    int incl = nchunks;
-    for (int o = 1; o < 32; o <<= 1) {
-        int t = __shfl_up_sync(FULL, incl, o);
-        if (lane >= o) incl += t;
-    }
-    const int total = __shfl_sync(FULL, incl, 31);
-    const int n_new = __popc(__ballot_sync(FULL, newly));
-    int base = 0;
-    if (lane == 0 && n_new) {
-        if (total) base = atomicAdd(&d.ws.ctr->n_tasks, total);
-        atomicAdd(&d.ws.ctr->n_nzblk, n_new);
-    }
-    base = __shfl_sync(FULL, base, 0) + incl - nchunks;
-    for (int k = 0; k < nchunks; ++k) d.ws.tasks[base + k] = make_uint2((uint32_t)jb, (uint32_t)(first + k * PUSH_CHUNK));
-}
-
 template <int DT>
 __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, const void *__restrict__ x_val,
                                 int32_t nnz_x, int validate) {
@@ -67,7 +46,7 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
             jb = j >> 4;
         }
     }
-    emit_tasks(d, newly, jb, lane);
+    emit_tasks(d, newly, jb, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
 }
 
 // Dense input (Sections 4.1, 4.3): every warp reads 32 elements, one ballot gives the two
@@ -85,7 +64,7 @@ __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__re
         const uint32_t bits = __ballot_sync(FULL, v != 0.0f);
         if (lane == 0) d.ws.x_mask32[j >> 5] = bits;
         const bool newly = (lane == 0 && (bits & 0xFFFFu)) || (lane == 16 && (bits >> 16));
-        emit_tasks(d, newly, (int)(j >> 4), lane);
+        emit_tasks(d, newly, (int)(j >> 4), lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
     }
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < d.m; i += stride) y[i] = 0.f;
 }

@@ -1,0 +1,38 @@
+// Push worklist (Section 3.3.2): the work of the active column blocks is flattened into
+// block-level tasks, each a run of at most PUSH_CHUNK consecutive entries of one block-CSC
+// column, so that a long column block is spread over many warps.
+#pragma once
+
+#include "internal.cuh"
+
+namespace dbs {
+
+// Called by a full warp.  Lanes with `newly` set own a vector block `jb` that has just become
+// nonempty; each appends that block's tasks.  Space is claimed with one warp scan and one
+// atomic per warp; the count of nonempty vector blocks is aggregated the same way
+// (hierarchical counting, Section 4.1).
+__device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int lane,
+                                           int32_t *n_tasks, int32_t *n_nzblk) {
+    int first = 0, nchunks = 0;
+    if (newly) {
+        first = d.csc.ptr[jb];
+        nchunks = (d.csc.ptr[jb + 1] - first + PUSH_CHUNK - 1) / PUSH_CHUNK;
+    }
+    int incl = nchunks;
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    const int n_new = __popc(__ballot_sync(0xFFFFFFFFu, newly));
+    int base = 0;
+    if (lane == 0 && n_new) {
+        if (total) base = atomicAdd(n_tasks, total);
+        atomicAdd(n_nzblk, n_new);
+    }
+    base = __shfl_sync(0xFFFFFFFFu, base, 0) + incl - nchunks;
+    for (int k = 0; k < nchunks; ++k)
+        d.ws.tasks[base + k] = make_uint2((uint32_t)jb, (uint32_t)(first + k * PUSH_CHUNK));
+}
+
+}  // namespace dbs

@@ -1,0 +1,87 @@
+"""GPU parity of dbspmspv_decode (dense bf16/fp32 x in, dense fp32 y out) against the oracle's
+dense-output loop on the bf16-rounded operands."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_16308_b200 import binding as B
+from paper_2608_16308_b200 import workloads as wl
+from gpu_util import Handle, ref_matrix, DEV, TOL
+
+pytestmark = pytest.mark.gpu
+PATHS = [B.PATH_AUTO, B.PATH_PUSH, B.PATH_PULL]
+
+
+def decode(h, x_f32):
+    if h.dtype == B.BF16:
+        xd = torch.from_numpy(wl.f32_to_bf16_bits(x_f32).view(np.int16)).to(DEV)
+    else:
+        xd = torch.from_numpy(np.ascontiguousarray(x_f32, dtype=np.float32)).to(DEV)
+    y = torch.full((h.csr.m,), 123.0, dtype=torch.float32, device=DEV)
+    B.dbspmspv_decode(h.h, xd, y)
+    torch.cuda.synchronize()
+    return y.cpu().numpy()
+
+
+def check(y, want, scale):
+    err = np.abs(y.astype(np.float64) - want)
+    assert (err <= TOL * scale).all(), f"worst {np.max(err / np.maximum(scale, 1e-300)):.3e}"
+    assert (y[scale == 0] == 0.0).all()            # rows without a structural hit are exactly 0
+
+
+@pytest.mark.parametrize("shape", [(192, 256), (1000, 333), (333, 1000)])
+@pytest.mark.parametrize("prune,zf", [(0.5, 0.7), (0.5, 0.9), (0.7, 0.9)])
+def test_decode_parity_bf16(shape, prune, zf):
+    m, n = shape
+    w = wl.pruned_weight(m, n, prune, seed=5, stream=m)
+    x = wl.relu_activation(n, zf, seed=5, stream=60)
+    h = Handle(w, B.BF16)
+    want, scale = oracle.ref_decode(ref_matrix(w), x)
+    for p in PATHS:
+        for thr in (1, 8):
+            h.set_opts(force_path=p, popc_threshold=thr)
+            check(decode(h, x), want, scale)
+    assert h.get_stats().last_n_nzblk == int((x.reshape(-1)[: (n // 16) * 16].reshape(-1, 16) != 0).any(axis=1).sum()
+                                             + (1 if n % 16 and (x[(n // 16) * 16:] != 0).any() else 0))
+    h.close()
+
+
+def test_decode_fp32_handle_small_integers_exact_and_negative_zero():
+    a = (wl.rand_below(3, 0, np.arange(64 * 48, dtype=np.uint64), 7).reshape(64, 48) - 3).astype(np.float32)
+    w = wl.csr_from_dense(a)
+    x = (wl.rand_below(3, 1, np.arange(48, dtype=np.uint64), 5) - 2).astype(np.float32)
+    x[5] = -0.0
+    for dtype in (B.F32, B.BF16):
+        h = Handle(w, dtype)
+        want, _ = oracle.ref_decode(ref_matrix(w), x)
+        for p in PATHS:
+            h.set_opts(force_path=p)
+            assert np.array_equal(decode(h, x).astype(np.float64), want)
+        h.close()
+
+
+def test_decode_all_zero_x_and_interleaving_with_run():
+    w = wl.pruned_weight(128, 160, 0.5, seed=5, stream=7)
+    h = Handle(w, B.BF16)
+    y = decode(h, np.zeros(160, dtype=np.float32))
+    assert (y == 0).all()
+    x = wl.relu_activation(160, 0.7, seed=5, stream=61)
+    want, scale = oracle.ref_decode(ref_matrix(w), x)
+    check(decode(h, x), want, scale)
+    # a sparse-output call on the same handle right after a decode call, and back
+    from gpu_util import check_against_oracle
+    xs = wl.sparse_x(4, 0, 160, 12)
+    xs.val = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(xs.val))
+    check_against_oracle(h.run(xs), oracle.ref_pull(ref_matrix(w), xs.idx, xs.val))
+    check(decode(h, x), want, scale)
+    h.close()
+
+
+def test_decode_rejects_pattern_handles():
+    h = Handle(wl.random_sparse(32, 32, 50, 1, values=False), B.PATTERN)
+    t = torch.zeros(32, device=DEV)
+    with pytest.raises(B.DbSpmspvError) as e:
+        B.dbspmspv_decode(h.h, t, t)
+    assert e.value.status == B.ERR_UNSUPPORTED
+    h.close()
