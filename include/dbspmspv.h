@@ -79,7 +79,7 @@ typedef struct {
     int32_t th0;             /* blocks with fewer than th0 entries use packed COO   (32)     */
     int32_t th1;             /* blocks with more than th1 entries use Dense         (128)    */
     float th2;               /* directional skew ratio for ForceCSR / ForceCSC      (2.0)    */
-    int32_t seg_cut;         /* a pull segment closes when its weight reaches this  (64)     */
+    int32_t seg_cut;         /* a pull segment closes when its weight reaches this  (128)    */
     int32_t w_dense;         /* pull segment weight of a Dense block                (4)      */
     int32_t w_mid;           /* ... of a ForceCSR / ForceCSC / CSR block            (2)      */
     int32_t w_coo;           /* ... of a COO block                                  (1)      */

@@ -57,13 +57,13 @@ __device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int dept
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
     for (int t = gwarp; t < n_tasks; t += nwarps) {
         const uint2 task = d.ws.tasks[t];
-        const int jb = (int)task.x, start = (int)task.y;
-        const int end = min(start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
+        const int jb = (int)(task.x & IDX_MASK);
+        const int cnt = (int)(task.x >> 27) + 1;
         const uint32_t xm = mask_of(d.ws.x_mask32, jb);
-        const int p = start + lane;
+        const int p = (int)task.y + lane;
         bool heavy = false;
         uint32_t idx = 0, w = 0, aux = 0;
-        if (p < end) {
+        if (lane < cnt) {
             idx = d.csc.idx[p];
             const int type = idx >> TYPE_SHIFT, brow = idx & IDX_MASK;
             const uint32_t need = ~mask_of(d.ws.visited32, brow) & 0xFFFFu;

@@ -608,7 +608,7 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     if (!o) return;
     *o = dbspmspv_create_opts();
     o->th0 = 32; o->th1 = 128; o->th2 = 2.0f;
-    o->seg_cut = 64; o->w_dense = 4; o->w_mid = 2; o->w_coo = 1;
+    o->seg_cut = 128; o->w_dense = 4; o->w_mid = 2; o->w_coo = 1;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
 }

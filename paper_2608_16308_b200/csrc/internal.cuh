@@ -70,7 +70,7 @@ struct Counters {    // device-resident scalars of one call
 struct Workspace {
     float *x_dense;       // n (padded to a multiple of 32): dense copy of x (Section 3.2.2)
     uint32_t *x_mask32;   // vector-block masks, two 16-bit masks per word
-    uint2 *tasks;         // push worklist: (column block, first CSC-view position)
+    uint2 *tasks;         // push worklist: (column block | (entries-1) << 27, first CSC-view position)
     float *y_acc;         // m (padded): dense accumulator, all zero between calls
     uint32_t *y_mask32;   // structural-hit masks per row block, two per word, zero between calls
     int32_t *tile_count;  // compaction: result entries per tile of row blocks

@@ -16,7 +16,7 @@
 namespace dbs {
 
 constexpr unsigned FULL = 0xFFFFFFFFu;
-constexpr int COO_SERIAL_MAX = 6;   // COO blocks up to this size are handled by one lane
+constexpr int COO_SERIAL_MAX = 32;  // COO blocks up to this many entries are handled by one lane
 
 __device__ __forceinline__ uint32_t below(int k) { return (1u << k) - 1u; }
 

@@ -11,8 +11,7 @@ namespace dbs {
 constexpr int CTA = 128;            // four warps per thread block (Section 3.3.2)
 constexpr int WARPS = CTA / 32;
 constexpr int CMP_TPB = 256;        // compaction: threads per tile
-constexpr int CMP_WORDS = 4;        // 32-bit mask words per thread
-constexpr int TILE_WORDS = CMP_TPB * CMP_WORDS;
+constexpr int TILE_WORDS = CMP_TPB;  // one 32-bit mask word (two row blocks) per thread
 
 // ------------------------------------------------------------------------------------------
 // Vector blocking (Section 3.2.2) fused with the push worklist (Section 3.3.2).
@@ -84,11 +83,15 @@ struct OutDense {
     static constexpr bool MASKS = false;
 };
 
-// One lane owns one hypersparse block (INLINE or small COO).  `emit(r, v)` receives every
-// product; returns the structural-hit row mask.
+// One lane owns one hypersparse block (INLINE or COO).  `emit(r, v)` receives the products,
+// already summed per row where the entries of a row are adjacent (COO is stored row-major);
+// `xin` is the x entry of an INLINE block's single column (fetched by the caller in parallel
+// with the mask); `xb` points at the 16 x entries of the block's vector block.  Returns the
+// structural-hit row mask.
 template <int DT, typename Emit>
 __device__ __forceinline__ uint32_t lane_block(int type, uint32_t w, uint32_t aux, uint32_t xm,
-                                               const float *xb, const uint8_t *payload, Emit emit) {
+                                               float xin, const float *xb, const uint8_t *payload,
+                                               Emit emit) {
     uint32_t hit = 0;
     if (type == DBSPMSPV_BLK_INLINE) {
         if (DT == DBSPMSPV_PATTERN) {
@@ -96,25 +99,29 @@ __device__ __forceinline__ uint32_t lane_block(int type, uint32_t w, uint32_t au
                 const uint32_t rc = (w >> (8 * k)) & 0xFFu;
                 if ((xm >> (rc & 15)) & 1u) hit |= 1u << (rc >> 4);
             }
-        } else {
-            const int c = aux & 15, r = aux >> 4;
-            if ((xm >> c) & 1u) { emit(r, Val<DT>::inline_value(w) * xb[c]); hit = 1u << r; }
+        } else if ((xm >> (aux & 15)) & 1u) {
+            emit((int)(aux >> 4), Val<DT>::inline_value(w) * xin);
+            hit = 1u << (aux >> 4);
         }
-    } else {  // small COO, row-major: products of one row are summed before they are emitted
+    } else {
         const int nnz = (int)aux + 1;
         const uint8_t *blk = payload + (size_t)w * 4;
+        const uint32_t *cw = reinterpret_cast<const uint32_t *>(blk);
         const uint8_t *vals = blk + ((nnz + 3) & ~3);
         int cur = -1;
         float s = 0.f;
-        for (int k = 0; k < nnz; ++k) {
-            const uint32_t rc = blk[k];
-            const int c = rc & 15, r = rc >> 4;
-            if ((xm >> c) & 1u) {
-                if (DT != DBSPMSPV_PATTERN) {
-                    if (r != cur) { if (cur >= 0) emit(cur, s); cur = r; s = 0.f; }
-                    s += Val<DT>::load(vals, k) * xb[c];
+        for (int k0 = 0; k0 < nnz; k0 += 4) {
+            uint32_t word = cw[k0 >> 2];
+            const int lim = min(4, nnz - k0);
+            for (int j = 0; j < lim; ++j, word >>= 8) {
+                const int c = word & 15, r = (word >> 4) & 15;
+                if ((xm >> c) & 1u) {
+                    if (DT != DBSPMSPV_PATTERN) {
+                        if (r != cur) { if (cur >= 0) emit(cur, s); cur = r; s = 0.f; }
+                        s += Val<DT>::load(vals, k0 + j) * xb[c];
+                    }
+                    hit |= 1u << r;
                 }
-                hit |= 1u << r;
             }
         }
         if (DT != DBSPMSPV_PATTERN && cur >= 0) emit(cur, s);
@@ -122,11 +129,16 @@ __device__ __forceinline__ uint32_t lane_block(int type, uint32_t w, uint32_t au
     return hit;
 }
 
+__device__ __forceinline__ bool lane_owned(int type, uint32_t aux) {
+    return type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX);
+}
+
 // Push (Section 3.3.2): every warp takes one task = up to 32 consecutive block-CSC entries of
 // one active column block; the vector block is staged once per task (Section 3.3.3).  Lanes
 // own hypersparse blocks; heavier blocks are then processed by the whole warp one at a time.
 // Writeback: warp-level reduction, then one global atomic per touched row and one atomicOr on
-// the row block's hit mask.
+// the row block's hit mask.  The task record carries its length, so the view entries, the mask
+// and the x block are all fetched in one round of independent loads.
 template <int DT, typename Out>
 __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp) {
     const int lane = threadIdx.x & 31;
@@ -135,22 +147,22 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
     const int n_tasks = d.ws.ctr->n_tasks;
     for (int t = gwarp; t < n_tasks; t += nwarps) {
         const uint2 task = d.ws.tasks[t];
-        const int jb = (int)task.x;
-        const int start = (int)task.y;
-        const int end = min(start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
+        const int jb = (int)(task.x & IDX_MASK);
+        const int cnt = (int)(task.x >> 27) + 1;
+        const int p = (int)task.y + lane;
+        const bool have = lane < cnt;
+        uint32_t idx = 0, w = 0, aux = 0;
+        if (have) { idx = d.csc.idx[p]; w = d.csc.w[p]; aux = d.csc.aux[p]; }
         const uint32_t xm = mask_of(d.ws.x_mask32, jb);
         if (lane < 16) s_x[lane] = d.ws.x_dense[jb * 16 + lane];
         __syncwarp();
-        const int p = start + lane;
         bool heavy = false;
-        uint32_t idx = 0, w = 0, aux = 0;
-        if (p < end) {
-            idx = d.csc.idx[p]; w = d.csc.w[p]; aux = d.csc.aux[p];
+        if (have) {
             const int type = idx >> TYPE_SHIFT;
             const int brow = idx & IDX_MASK;
-            if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX)) {
+            if (lane_owned(type, aux)) {
                 float *row0 = out.acc + (size_t)brow * 16;
-                const uint32_t hit = lane_block<DT>(type, w, aux, xm, s_x, d.payload,
+                const uint32_t hit = lane_block<DT>(type, w, aux, xm, s_x[aux & 15], s_x, d.payload,
                                                     [&](int r, float v) { atomicAdd(row0 + r, v); });
                 if (Out::MASKS && hit) atomicOr(&out.mask32[brow >> 1], hit << ((brow & 1) * 16));
             } else {
@@ -183,7 +195,11 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
 // Pull (Section 3.3.2): every warp takes one load-weighted segment of a row block and keeps
 // the 16 partial sums of that row block in shared memory; blocks whose vector block is empty
 // are skipped on their mask.  A segment that covers its whole row block writes with plain
-// stores; split row blocks fall back to atomics.
+// stores; split row blocks fall back to atomics.  PULL_UNROLL x 32 view entries are fetched
+// per step, then their masks and (for INLINE blocks) x entries, so that each lane keeps
+// several independent loads in flight.
+constexpr int PULL_UNROLL = 4;
+
 template <int DT, typename Out>
 __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp,
                           float *s_y) {
@@ -198,47 +214,58 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
         if (lane < 16) s_y[lane] = 0.f;
         __syncwarp();
         uint32_t hit = 0;
-        for (int base = seg.start; base < end; base += 32) {
-            const int p = base + lane;
-            bool heavy = false;
-            uint32_t idx = 0, w = 0, aux = 0, xm = 0;
-            if (p < end) {
-                idx = d.csr.idx[p];
-                const int bcol = idx & IDX_MASK;
-                xm = mask_of(d.ws.x_mask32, bcol);
-                if (xm) {
-                    w = d.csr.w[p]; aux = d.csr.aux[p];
-                    const int type = idx >> TYPE_SHIFT;
-                    if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX)) {
-                        hit |= lane_block<DT>(type, w, aux, xm, d.ws.x_dense + (size_t)bcol * 16, d.payload,
-                                              [&](int r, float v) { atomicAdd(&s_y[r], v); });
-                    } else {
-                        heavy = true;
-                    }
-                }
+        for (int base = seg.start; base < end; base += 32 * PULL_UNROLL) {
+            uint32_t idx[PULL_UNROLL], w[PULL_UNROLL], aux[PULL_UNROLL], xm[PULL_UNROLL];
+            float xin[PULL_UNROLL];
+#pragma unroll
+            for (int u = 0; u < PULL_UNROLL; ++u) {
+                const int p = base + u * 32 + lane;
+                idx[u] = 0; w[u] = 0; aux[u] = 0;
+                if (p < end) { idx[u] = d.csr.idx[p]; w[u] = d.csr.w[p]; aux[u] = d.csr.aux[p]; }
             }
-            uint32_t hv = __ballot_sync(FULL, heavy);
-            while (hv) {
-                const int src = __ffs(hv) - 1;
-                hv &= hv - 1;
-                const uint32_t bidx = __shfl_sync(FULL, idx, src);
-                const uint32_t bw = __shfl_sync(FULL, w, src);
-                const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
-                const uint32_t bxm = __shfl_sync(FULL, xm, src);
-                const int type = bidx >> TYPE_SHIFT;
-                const int bcol = bidx & IDX_MASK;
-                const uint8_t *blk = d.payload + (size_t)bw * 4;
-                uint32_t hits;
-                if (DT == DBSPMSPV_PATTERN) {
-                    hits = warp_block_bool<DT>(type, blk, nnz, bxm, lane);
-                } else {
-                    __syncwarp();
-                    if (lane < 16) s_x[lane] = d.ws.x_dense[(size_t)bcol * 16 + lane];
-                    __syncwarp();
-                    const float sum = warp_block<DT>(type, blk, nnz, bxm, s_x, s_tmp, lane, popc_threshold, hits);
-                    if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(&s_y[lane], sum);
+#pragma unroll
+            for (int u = 0; u < PULL_UNROLL; ++u) {
+                const int bcol = idx[u] & IDX_MASK;
+                const bool have = base + u * 32 + lane < end;
+                xm[u] = have ? mask_of(d.ws.x_mask32, bcol) : 0u;
+                xin[u] = (have && DT != DBSPMSPV_PATTERN) ? d.ws.x_dense[(size_t)bcol * 16 + (aux[u] & 15)] : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < PULL_UNROLL; ++u) {
+                if (base + u * 32 >= end) break;   // warp-uniform
+                bool heavy = false;
+                if (xm[u]) {
+                    const int type = idx[u] >> TYPE_SHIFT;
+                    const int bcol = idx[u] & IDX_MASK;
+                    if (lane_owned(type, aux[u]))
+                        hit |= lane_block<DT>(type, w[u], aux[u], xm[u], xin[u], d.ws.x_dense + (size_t)bcol * 16,
+                                              d.payload, [&](int r, float v) { atomicAdd(&s_y[r], v); });
+                    else
+                        heavy = true;
                 }
-                hit |= hits;
+                uint32_t hv = __ballot_sync(FULL, heavy);
+                while (hv) {
+                    const int src = __ffs(hv) - 1;
+                    hv &= hv - 1;
+                    const uint32_t bidx = __shfl_sync(FULL, idx[u], src);
+                    const uint32_t bw = __shfl_sync(FULL, w[u], src);
+                    const int nnz = (int)__shfl_sync(FULL, aux[u], src) + 1;
+                    const uint32_t bxm = __shfl_sync(FULL, xm[u], src);
+                    const int type = bidx >> TYPE_SHIFT;
+                    const int bcol = bidx & IDX_MASK;
+                    const uint8_t *blk = d.payload + (size_t)bw * 4;
+                    uint32_t hits;
+                    if (DT == DBSPMSPV_PATTERN) {
+                        hits = warp_block_bool<DT>(type, blk, nnz, bxm, lane);
+                    } else {
+                        __syncwarp();
+                        if (lane < 16) s_x[lane] = d.ws.x_dense[(size_t)bcol * 16 + lane];
+                        __syncwarp();
+                        const float sum = warp_block<DT>(type, blk, nnz, bxm, s_x, s_tmp, lane, popc_threshold, hits);
+                        if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(&s_y[lane], sum);
+                    }
+                    hit |= hits;
+                }
             }
         }
         hit = __reduce_or_sync(FULL, hit);
@@ -281,11 +308,8 @@ __global__ void __launch_bounds__(CTA) k_compute(Device d, Out out, float th3, i
 __global__ void __launch_bounds__(CMP_TPB) k_compact_count(Device d) {
     __shared__ int s_red[CMP_TPB / 32];
     const int n_words = (d.mb + 1) / 2;
-    const int w0 = (blockIdx.x * CMP_TPB + threadIdx.x) * CMP_WORDS;
-    int c = 0;
-#pragma unroll
-    for (int k = 0; k < CMP_WORDS; ++k)
-        if (w0 + k < n_words) c += __popc(d.ws.y_mask32[w0 + k]);
+    const int wi = blockIdx.x * CMP_TPB + threadIdx.x;
+    int c = wi < n_words ? __popc(d.ws.y_mask32[wi]) : 0;
     c = __reduce_add_sync(FULL, c);
     if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = c;
     __syncthreads();
@@ -317,14 +341,9 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
         }
         __syncthreads();
         const int n_words = (d.mb + 1) / 2;
-        const int w0 = (blockIdx.x * CMP_TPB + threadIdx.x) * CMP_WORDS;
-        uint32_t words[CMP_WORDS];
-        int c = 0;
-#pragma unroll
-        for (int k = 0; k < CMP_WORDS; ++k) {
-            words[k] = w0 + k < n_words ? d.ws.y_mask32[w0 + k] : 0u;
-            c += __popc(words[k]);
-        }
+        const int wi = blockIdx.x * CMP_TPB + threadIdx.x;     // one 32-row mask word per thread
+        const uint32_t word = wi < n_words ? d.ws.y_mask32[wi] : 0u;
+        const int c = __popc(word);
         int incl = c;
         for (int o = 1; o < 32; o <<= 1) {
             int t = __shfl_up_sync(FULL, incl, o);
@@ -333,32 +352,34 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
         __syncthreads();
         if (lane == 31) s_red[warp] = incl;
         __syncthreads();
-        int pos = s_base + incl - c;
-        for (int k = 0; k < warp; ++k) pos += s_red[k];
-        if (c) {
-#pragma unroll
-            for (int k = 0; k < CMP_WORDS; ++k) {
-                uint32_t wd = words[k];
-                if (wd) d.ws.y_mask32[w0 + k] = 0u;
-                while (wd) {
-                    const int bit = __ffs(wd) - 1;
-                    wd &= wd - 1;
-                    const int row = (w0 + k) * 32 + bit;
-                    const float v = d.ws.y_acc[row];
-                    d.ws.y_acc[row] = 0.f;
-                    if (pos < y_capacity) {
-                        y_idx[pos] = row;
-                        if (y_val) y_val[pos] = boolean ? 1.0f : v;
-                    }
-                    ++pos;
+        int wbase = s_base;
+        for (int k = 0; k < warp; ++k) wbase += s_red[k];
+        // the warp walks its 32 words; lanes are the 32 rows of a word, so the accumulator is
+        // read and cleared with coalesced accesses and y is written in ascending order
+        uint32_t todo = __ballot_sync(FULL, word != 0);
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const uint32_t wd = __shfl_sync(FULL, word, src);
+            const int off = __shfl_sync(FULL, incl - c, src);
+            if ((wd >> lane) & 1u) {
+                const int row = (wi - lane + src) * 32 + lane;
+                const int64_t pos = (int64_t)wbase + off + __popc(wd & below(lane));
+                const float v = d.ws.y_acc[row];
+                d.ws.y_acc[row] = 0.f;
+                if (pos < y_capacity) {
+                    y_idx[pos] = row;
+                    if (y_val) y_val[pos] = boolean ? 1.0f : v;
                 }
             }
         }
+        if (word) d.ws.y_mask32[wi] = 0u;
         if ((int)blockIdx.x == n_tiles - 1 && threadIdx.x == CMP_TPB - 1) {
             Counters *c2 = d.ws.ctr;
-            *y_nnz = pos;
-            if (pos > y_capacity) c2->status = DBSPMSPV_ERR_CAPACITY;
-            c2->last_y_nnz = pos;
+            const int total = wbase + incl;
+            *y_nnz = total;
+            if (total > y_capacity) c2->status = DBSPMSPV_ERR_CAPACITY;
+            c2->last_y_nnz = total;
             c2->last_n_nzblk = c2->n_nzblk;
             c2->last_n_tasks = c2->n_tasks;
             c2->last_path = c2->path;

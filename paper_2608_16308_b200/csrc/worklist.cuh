@@ -13,11 +13,12 @@ namespace dbs {
 // (hierarchical counting, Section 4.1).
 __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int lane,
                                            int32_t *n_tasks, int32_t *n_nzblk) {
-    int first = 0, nchunks = 0;
+    int first = 0, deg = 0;
     if (newly) {
         first = d.csc.ptr[jb];
-        nchunks = (d.csc.ptr[jb + 1] - first + PUSH_CHUNK - 1) / PUSH_CHUNK;
+        deg = d.csc.ptr[jb + 1] - first;
     }
+    const int nchunks = (deg + PUSH_CHUNK - 1) / PUSH_CHUNK;
     int incl = nchunks;
     for (int o = 1; o < 32; o <<= 1) {
         int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
@@ -31,8 +32,29 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
         atomicAdd(n_nzblk, n_new);
     }
     base = __shfl_sync(0xFFFFFFFFu, base, 0) + incl - nchunks;
-    for (int k = 0; k < nchunks; ++k)
-        d.ws.tasks[base + k] = make_uint2((uint32_t)jb, (uint32_t)(first + k * PUSH_CHUNK));
+    // task record: column block in bits 0..26, (entries - 1) in bits 27..31, first position.
+    // Short columns are written by their own lane; a long column block (a hub) is written by
+    // the whole warp so that one lane does not serialise thousands of stores.
+    constexpr int SMALL = 4;
+    if (nchunks <= SMALL)
+        for (int k = 0; k < nchunks; ++k) {
+            const int cnt = min(PUSH_CHUNK, deg - k * PUSH_CHUNK);
+            d.ws.tasks[base + k] = make_uint2((uint32_t)jb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(first + k * PUSH_CHUNK));
+        }
+    uint32_t big = __ballot_sync(0xFFFFFFFFu, nchunks > SMALL);
+    while (big) {
+        const int src = __ffs(big) - 1;
+        big &= big - 1;
+        const int bjb = __shfl_sync(0xFFFFFFFFu, jb, src);
+        const int bfirst = __shfl_sync(0xFFFFFFFFu, first, src);
+        const int bdeg = __shfl_sync(0xFFFFFFFFu, deg, src);
+        const int bbase = __shfl_sync(0xFFFFFFFFu, base, src);
+        const int bn = (bdeg + PUSH_CHUNK - 1) / PUSH_CHUNK;
+        for (int k = lane; k < bn; k += 32) {
+            const int cnt = min(PUSH_CHUNK, bdeg - k * PUSH_CHUNK);
+            d.ws.tasks[bbase + k] = make_uint2((uint32_t)bjb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(bfirst + k * PUSH_CHUNK));
+        }
+    }
 }
 
 }  // namespace dbs
