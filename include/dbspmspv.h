@@ -85,7 +85,9 @@ typedef struct {
     int32_t w_coo;           /* ... of a COO block                                  (1)      */
     int32_t force_format;    /* DBSPMSPV_FORMAT_*: ablation knob (Section 5.4)               */
     int32_t input_on_host;   /* 1: the create arrays are HOST pointers (copied once)         */
-    int32_t reserved[7];
+    int32_t inline_max;      /* valued matrices: a block with at most this many entries keeps
+                                them in its view entries, one entry per element       (4)    */
+    int32_t reserved[6];
 } dbspmspv_create_opts;
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
@@ -105,6 +107,8 @@ typedef struct {
     /* matrix / format (fixed at create) */
     int64_t m, n, nnz;             /* nnz after merging duplicates                            */
     int64_t n_blocks;              /* nonempty 16 x 16 blocks                                 */
+    int64_t n_view_entries;        /* entries per view (>= n_blocks: INLINE blocks of valued
+                                      matrices hold one entry per stored element)            */
     int64_t class_blocks[DBSPMSPV_BLK_NCLASS]; /* per DBSPMSPV_BLK_* class                    */
     int64_t class_nnz[DBSPMSPV_BLK_NCLASS];
     int64_t n_row_blocks, n_col_blocks;        /* ceil(m/16), ceil(n/16)                      */
@@ -201,14 +205,16 @@ int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out);
  * block-major; sort before comparing.  Synchronises.                                         */
 int dbspmspv_export_coo(dbspmspv_handle_t h, int32_t *row, int32_t *col, void *val);
 
-/* Test hook: copy the per-block class codes (DBSPMSPV_BLK_*) in primary (block-CSR) order and
- * the block coordinates to device arrays of stats.n_blocks entries (any may be NULL).        */
+/* Test hook: per view entry, in primary (block-CSR) order: block coordinates, class code
+ * (DBSPMSPV_BLK_*) and stored elements of the entry.  Device arrays of stats.n_view_entries
+ * int32 (any may be NULL).  The entries of one INLINE block are adjacent.                    */
 int dbspmspv_export_blocks(dbspmspv_handle_t h, int32_t *block_row, int32_t *block_col,
                            int32_t *block_class, int32_t *block_nnz);
 
 /* Test hook: copy the dual view out: csr_row_ptr (n_row_blocks+1), csc_col_ptr
- * (n_col_blocks+1), csc_row (n_blocks: row block of every CSC-view position), csc2csr
- * (n_blocks: CSC-view position -> primary block id).  Device int32 arrays; any may be NULL. */
+ * (n_col_blocks+1), csc_row (n_view_entries: row block of every CSC-view position), csc2csr
+ * (n_view_entries: CSC-view position -> primary entry id).  Device int32 arrays; any may be
+ * NULL.                                                                                      */
 int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *csc_col_ptr,
                           int32_t *csc_row, int32_t *csc2csr);
 

@@ -35,7 +35,8 @@ class CreateOpts(ctypes.Structure):
     _fields_ = [("th0", ctypes.c_int32), ("th1", ctypes.c_int32), ("th2", ctypes.c_float),
                 ("seg_cut", ctypes.c_int32), ("w_dense", ctypes.c_int32), ("w_mid", ctypes.c_int32),
                 ("w_coo", ctypes.c_int32), ("force_format", ctypes.c_int32),
-                ("input_on_host", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7)]
+                ("input_on_host", ctypes.c_int32), ("inline_max", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 6)]
 
 
 class RunOpts(ctypes.Structure):
@@ -46,7 +47,7 @@ class RunOpts(ctypes.Structure):
 
 class Stats(ctypes.Structure):
     _fields_ = [("m", ctypes.c_int64), ("n", ctypes.c_int64), ("nnz", ctypes.c_int64),
-                ("n_blocks", ctypes.c_int64), ("class_blocks", ctypes.c_int64 * 6),
+                ("n_blocks", ctypes.c_int64), ("n_view_entries", ctypes.c_int64), ("class_blocks", ctypes.c_int64 * 6),
                 ("class_nnz", ctypes.c_int64 * 6), ("n_row_blocks", ctypes.c_int64),
                 ("n_col_blocks", ctypes.c_int64), ("n_segments", ctypes.c_int64),
                 ("payload_bytes", ctypes.c_int64), ("csr_view_bytes", ctypes.c_int64),

@@ -15,7 +15,7 @@ __device__ __forceinline__ int block_nnz(int dtype, uint32_t idx, uint32_t aux) 
 
 __global__ void k_block_nnz(Device d, int32_t *out) {
     int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (b < d.n_blocks) out[b] = block_nnz(d.dtype, d.csr.idx[b], d.csr.aux[b]);
+    if (b < d.n_entries) out[b] = block_nnz(d.dtype, d.csr.idx[b], d.csr.aux[b]);
 }
 
 template <int DT>
@@ -33,7 +33,7 @@ __global__ void k_export(Device d, const int32_t *block_row, const int32_t *elem
                          int32_t *col, void *val) {
     const int lane = threadIdx.x & 31;
     int64_t b = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
-    if (b >= d.n_blocks) return;
+    if (b >= d.n_entries) return;
     const uint32_t idx = d.csr.idx[b], w = d.csr.w[b], aux = d.csr.aux[b];
     const int type = idx >> TYPE_SHIFT;
     const int r0 = block_row[b] * 16, c0 = (int)(idx & IDX_MASK) * 16;
@@ -87,7 +87,7 @@ __global__ void k_export(Device d, const int32_t *block_row, const int32_t *elem
 __global__ void k_export_blocks(Device d, const int32_t *brow, int32_t *block_row, int32_t *block_col,
                                 int32_t *block_class, int32_t *nnz) {
     int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (b >= d.n_blocks) return;
+    if (b >= d.n_entries) return;
     const uint32_t idx = d.csr.idx[b];
     if (block_row) block_row[b] = brow[b];
     if (block_col) block_col[b] = (int32_t)(idx & IDX_MASK);
@@ -97,7 +97,7 @@ __global__ void k_export_blocks(Device d, const int32_t *brow, int32_t *block_ro
 
 __global__ void k_export_csc_rows(Device d, int32_t *csc_row) {
     int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (p < d.n_blocks) csc_row[p] = (int32_t)(d.csc.idx[p] & IDX_MASK);
+    if (p < d.n_entries) csc_row[p] = (int32_t)(d.csc.idx[p] & IDX_MASK);
 }
 
 }  // namespace
@@ -132,12 +132,12 @@ int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out) {
 int dbspmspv_export_coo(dbspmspv_handle_t h, int32_t *row, int32_t *col, void *val) {
     if (!h || !row || !col) return DBSPMSPV_ERR_INVALID_ARG;
     const dbs::Device &d = h->d;
-    if (d.n_blocks == 0) return DBSPMSPV_OK;
+    if (d.n_entries == 0) return DBSPMSPV_OK;
     int32_t *cnt = nullptr, *start = nullptr;
     void *tmp = nullptr;
     size_t bytes = 0;
     int status = DBSPMSPV_OK;
-    const int nb = d.n_blocks;
+    const int nb = d.n_entries;
     if (cudaMalloc(&cnt, (size_t)nb * 4) != cudaSuccess || cudaMalloc(&start, (size_t)nb * 4) != cudaSuccess) status = DBSPMSPV_ERR_ALLOC;
     if (status == DBSPMSPV_OK) {
         dbs::k_block_nnz<<<(nb + 255) / 256, 256>>>(d, cnt);
@@ -160,7 +160,7 @@ int dbspmspv_export_blocks(dbspmspv_handle_t h, int32_t *block_row, int32_t *blo
                            int32_t *block_class, int32_t *block_nnz) {
     if (!h) return DBSPMSPV_ERR_INVALID_ARG;
     const dbs::Device &d = h->d;
-    if (d.n_blocks) dbs::k_export_blocks<<<(d.n_blocks + 255) / 256, 256>>>(d, h->block_row, block_row, block_col, block_class, block_nnz);
+    if (d.n_entries) dbs::k_export_blocks<<<(d.n_entries + 255) / 256, 256>>>(d, h->block_row, block_row, block_col, block_class, block_nnz);
     DBS_CUDA(cudaDeviceSynchronize());
     return DBSPMSPV_OK;
 }
@@ -171,8 +171,8 @@ int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *cs
     const dbs::Device &d = h->d;
     if (csr_row_ptr) DBS_CUDA(cudaMemcpy(csr_row_ptr, d.csr.ptr, ((size_t)d.mb + 1) * 4, cudaMemcpyDeviceToDevice));
     if (csc_col_ptr) DBS_CUDA(cudaMemcpy(csc_col_ptr, d.csc.ptr, ((size_t)d.nb + 1) * 4, cudaMemcpyDeviceToDevice));
-    if (csc_row && d.n_blocks) dbs::k_export_csc_rows<<<(d.n_blocks + 255) / 256, 256>>>(d, csc_row);
-    if (csc2csr && d.n_blocks) DBS_CUDA(cudaMemcpy(csc2csr, h->csc2csr, (size_t)d.n_blocks * 4, cudaMemcpyDeviceToDevice));
+    if (csc_row && d.n_entries) dbs::k_export_csc_rows<<<(d.n_entries + 255) / 256, 256>>>(d, csc_row);
+    if (csc2csr && d.n_entries) DBS_CUDA(cudaMemcpy(csc2csr, h->csc2csr, (size_t)d.n_entries * 4, cudaMemcpyDeviceToDevice));
     DBS_CUDA(cudaDeviceSynchronize());
     return DBSPMSPV_OK;
 }

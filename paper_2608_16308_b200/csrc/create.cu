@@ -110,6 +110,7 @@ struct ClassifyParams {
     float th2;
     int force_format;
     int dtype;
+    int inline_max;   // valued matrices: blocks with at most this many entries are stored inline
 };
 
 __device__ __forceinline__ int payload_words(int type, int nnz, int vsize) {
@@ -123,7 +124,7 @@ __device__ __forceinline__ int payload_words(int type, int nnz, int vsize) {
 
 __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
                            ClassifyParams cp, uint8_t *type_out, uint32_t *size_out,
-                           int32_t *brow, int32_t *bcol, unsigned long long *class_blocks,
+                           int32_t *ecount, int32_t *brow, int32_t *bcol, unsigned long long *class_blocks,
                            unsigned long long *class_nnz) {
     __shared__ uint32_t s_row[TPB / 32][16], s_col[TPB / 32][16];
     __shared__ unsigned int s_cb[DBSPMSPV_BLK_NCLASS], s_cn[DBSPMSPV_BLK_NCLASS];
@@ -152,7 +153,9 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
             if (cp.force_format == DBSPMSPV_FORMAT_COO) type = DBSPMSPV_BLK_COO;
             else if (cp.force_format == DBSPMSPV_FORMAT_CSR) type = DBSPMSPV_BLK_CSR;
             else if (nnz < cp.th0) {
-                const int inline_cap = cp.dtype == DBSPMSPV_PATTERN ? 4 : 1;
+                // pattern: up to four coordinates fit in one view entry; valued: one view
+                // entry per stored element, up to inline_max of them
+                const int inline_cap = cp.dtype == DBSPMSPV_PATTERN ? 4 : cp.inline_max;
                 type = nnz <= inline_cap ? DBSPMSPV_BLK_INLINE : DBSPMSPV_BLK_COO;
             } else if (nnz > cp.th1) type = DBSPMSPV_BLK_DENSE;
             // skew_c / skew_r = (max column count) / (max row count): the denominators of
@@ -163,6 +166,7 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
             const int vsize = cp.dtype == DBSPMSPV_F32 ? 4 : cp.dtype == DBSPMSPV_BF16 ? 2 : 0;
             type_out[b] = (uint8_t)type;
             size_out[b] = (uint32_t)payload_words(type, nnz, vsize);
+            ecount[b] = (type == DBSPMSPV_BLK_INLINE && cp.dtype != DBSPMSPV_PATTERN) ? nnz : 1;
             uint64_t k0 = ukey[s];
             brow[b] = (int32_t)(k0 >> 35);
             bcol[b] = (int32_t)((k0 >> 8) & IDX_MASK);
@@ -187,8 +191,9 @@ __device__ __forceinline__ void store_value(uint8_t *vals, int pos, const void *
 template <int DT>
 __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
                          const void *uval, const uint8_t *type_in, const uint64_t *poff,
-                         const int32_t *bcol, uint8_t *payload, uint32_t *v_idx, uint32_t *v_w,
-                         uint8_t *v_aux) {
+                         const int32_t *eoff, const int32_t *brow, const int32_t *bcol,
+                         uint8_t *payload, uint32_t *v_idx, uint32_t *v_w, uint8_t *v_aux,
+                         int32_t *entry_row) {
     constexpr int V = Val<DT>::SIZE;
     __shared__ uint32_t s_row[TPB / 32][16], s_col[TPB / 32][16];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -198,23 +203,30 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
     const int type = type_in[b];
     const uint64_t off_words = poff[b];
     uint8_t *base = payload + off_words * 4;
-    if (lane == 0) {
-        v_idx[b] = (uint32_t)bcol[b] | ((uint32_t)type << TYPE_SHIFT);
-        if (type == DBSPMSPV_BLK_INLINE) {
-            if (DT == DBSPMSPV_PATTERN) {
-                uint32_t w = 0;
-                for (int k = 0; k < nnz; ++k) w |= (uint32_t)(ukey[s + k] & 0xFF) << (8 * k);
-                v_w[b] = w;
-                v_aux[b] = (uint8_t)(nnz - 1);
-            } else {
-                v_w[b] = DT == DBSPMSPV_F32 ? __float_as_uint(static_cast<const float *>(uval)[s])
-                                            : (uint32_t) static_cast<const uint16_t *>(uval)[s];
-                v_aux[b] = (uint8_t)(ukey[s] & 0xFF);
-            }
-        } else {
-            v_w[b] = (uint32_t)off_words;
-            v_aux[b] = (uint8_t)(nnz - 1);
+    const int e0 = eoff[b];
+    const uint32_t tagged = (uint32_t)bcol[b] | ((uint32_t)type << TYPE_SHIFT);
+    if (type == DBSPMSPV_BLK_INLINE && DT != DBSPMSPV_PATTERN) {
+        // one view entry per stored element: value in w, packed coordinate in aux
+        for (int k = lane; k < nnz; k += 32) {
+            v_idx[e0 + k] = tagged;
+            v_w[e0 + k] = DT == DBSPMSPV_F32 ? __float_as_uint(static_cast<const float *>(uval)[s + k])
+                                             : (uint32_t) static_cast<const uint16_t *>(uval)[s + k];
+            v_aux[e0 + k] = (uint8_t)(ukey[s + k] & 0xFF);
+            entry_row[e0 + k] = brow[b];
         }
+        return;
+    }
+    if (lane == 0) {
+        v_idx[e0] = tagged;
+        entry_row[e0] = brow[b];
+        if (type == DBSPMSPV_BLK_INLINE) {
+            uint32_t w = 0;
+            for (int k = 0; k < nnz; ++k) w |= (uint32_t)(ukey[s + k] & 0xFF) << (8 * k);
+            v_w[e0] = w;
+        } else {
+            v_w[e0] = (uint32_t)off_words;
+        }
+        v_aux[e0] = (uint8_t)(nnz - 1);
     }
     if (type == DBSPMSPV_BLK_INLINE) return;
     if (type == DBSPMSPV_BLK_COO) {
@@ -289,11 +301,11 @@ __global__ void k_lower_bounds(int32_t count, const int32_t *sorted, int32_t n, 
     ptr[v] = lo;
 }
 
-__global__ void k_csc_keys(int32_t n_blocks, const int32_t *brow, const int32_t *bcol,
+__global__ void k_csc_keys(int32_t n_entries, const int32_t *entry_row, const uint32_t *csr_idx,
                            uint64_t *keys, int32_t *ids) {
     int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (b >= n_blocks) return;
-    keys[b] = ((uint64_t)bcol[b] << 27) | (uint64_t)brow[b];
+    if (b >= n_entries) return;
+    keys[b] = ((uint64_t)(csr_idx[b] & IDX_MASK) << 27) | (uint64_t)entry_row[b];
     ids[b] = (int32_t)b;
 }
 
@@ -474,20 +486,25 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         tp.release(flag); tp.release(rank);
     }
     h->nnz = nnzu;
-    d.n_blocks = n_blocks;
 
     // classify + size
     uint8_t *type;
     uint32_t *psize;
     uint64_t *poff;
-    int32_t *bcol;
+    int32_t *brow, *bcol, *ecount, *eoff;
     unsigned long long *cls;
-    DBS_GET(type, n_blocks); DBS_GET(psize, n_blocks); DBS_GET(bcol, n_blocks);
+    DBS_GET(type, n_blocks); DBS_GET(psize, n_blocks); DBS_GET(brow, n_blocks); DBS_GET(bcol, n_blocks);
+    DBS_GET(ecount, (int64_t)n_blocks + 1); DBS_GET(eoff, (int64_t)n_blocks + 1);
     DBS_GET(cls, 2 * DBSPMSPV_BLK_NCLASS);
-    DBS_KEEP(h->block_row, n_blocks);
     DBS_CUDA(cudaMemsetAsync(cls, 0, 2 * DBSPMSPV_BLK_NCLASS * sizeof(unsigned long long), st));
-    ClassifyParams cp{h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt};
-    if (n_blocks) k_classify<<<grid_for(n_blocks, TPB / 32), TPB, 0, st>>>(n_blocks, blk_start, ukey, cp, type, psize, h->block_row, bcol, cls, cls + DBSPMSPV_BLK_NCLASS);
+    DBS_CUDA(cudaMemsetAsync(ecount, 0, ((size_t)n_blocks + 1) * 4, st));
+    ClassifyParams cp{h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt, h->copts.inline_max};
+    if (n_blocks) k_classify<<<grid_for(n_blocks, TPB / 32), TPB, 0, st>>>(n_blocks, blk_start, ukey, cp, type, psize, ecount, brow, bcol, cls, cls + DBSPMSPV_BLK_NCLASS);
+    // view entries: a small valued block contributes one entry per stored element
+    DBS_TRY(exclusive_sum(tp, ecount, eoff, (int64_t)n_blocks + 1, st));
+    int32_t n_entries = 0;
+    DBS_CUDA(cudaMemcpy(&n_entries, eoff + n_blocks, 4, cudaMemcpyDeviceToHost));
+    d.n_entries = n_entries;
     // 64-bit offsets for the scan (the total may exceed 2^32 words only beyond 16 GB)
     DBS_GET(poff, (int64_t)n_blocks + 1);
     {
@@ -508,33 +525,36 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         DBS_CUDA(cudaMemsetAsync(p, 0, h->payload_bytes + 256, st));
         h->payload_alloc = p; d.payload = p;
     }
-    DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_blocks); DBS_KEEP(d.csr.w, n_blocks); DBS_KEEP(d.csr.aux, n_blocks);
-    DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_blocks); DBS_KEEP(d.csc.w, n_blocks); DBS_KEEP(d.csc.aux, n_blocks);
-    DBS_KEEP(h->csc2csr, n_blocks);
+    DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_entries); DBS_KEEP(d.csr.w, n_entries); DBS_KEEP(d.csr.aux, n_entries);
+    DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_entries); DBS_KEEP(d.csc.w, n_entries); DBS_KEEP(d.csc.aux, n_entries);
+    DBS_KEEP(h->csc2csr, n_entries);
+    DBS_KEEP(h->block_row, n_entries);
     if (n_blocks) {
         uint8_t *pl = static_cast<uint8_t *>(h->payload_alloc);
         const int g = grid_for(n_blocks, TPB / 32);
-        if (dt == DBSPMSPV_F32) k_encode<DBSPMSPV_F32><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux);
-        else if (dt == DBSPMSPV_BF16) k_encode<DBSPMSPV_BF16><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux);
-        else k_encode<DBSPMSPV_PATTERN><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux);
+        if (dt == DBSPMSPV_F32) k_encode<DBSPMSPV_F32><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row);
+        else if (dt == DBSPMSPV_BF16) k_encode<DBSPMSPV_BF16><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row);
+        else k_encode<DBSPMSPV_PATTERN><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row);
     }
-    k_lower_bounds<<<grid_for(d.mb + 1), TPB, 0, st>>>(d.mb, h->block_row, n_blocks, d.csr.ptr);
+    k_lower_bounds<<<grid_for(d.mb + 1), TPB, 0, st>>>(d.mb, h->block_row, n_entries, d.csr.ptr);
     DBS_CUDA(cudaStreamSynchronize(st));
     tp.release(ukey); tp.release(uval); tp.release(blk_start); tp.release(poff); tp.release(psize);
+    tp.release(brow); tp.release(bcol); tp.release(ecount); tp.release(eoff); tp.release(type);
 
-    // block-CSC view: sort primary ids by (column block, row block)
+    // block-CSC view: sort the primary entries by (column block, row block); the radix sort is
+    // stable, so the entries of one block stay together and in order
     {
         uint64_t *k2, *k2_alt;
         int32_t *ids, *ids_alt, *bcol_sorted;
-        DBS_GET(k2, n_blocks); DBS_GET(k2_alt, n_blocks); DBS_GET(ids, n_blocks); DBS_GET(ids_alt, n_blocks);
-        DBS_GET(bcol_sorted, n_blocks);
-        if (n_blocks) {
-            k_csc_keys<<<grid_for(n_blocks), TPB, 0, st>>>(n_blocks, h->block_row, bcol, k2, ids);
-            DBS_TRY(sort_pairs(tp, k2, k2_alt, ids, ids_alt, (int64_t)n_blocks, 27 + bits_for((uint64_t)d.nb), st));
-            DBS_CUDA(cudaMemcpyAsync(h->csc2csr, ids, (size_t)n_blocks * 4, cudaMemcpyDeviceToDevice, st));
-            k_csc_gather<<<grid_for(n_blocks), TPB, 0, st>>>(n_blocks, k2, h->csc2csr, d.csr.idx, d.csr.w, d.csr.aux, d.csc.idx, d.csc.w, d.csc.aux, bcol_sorted);
+        DBS_GET(k2, n_entries); DBS_GET(k2_alt, n_entries); DBS_GET(ids, n_entries); DBS_GET(ids_alt, n_entries);
+        DBS_GET(bcol_sorted, n_entries);
+        if (n_entries) {
+            k_csc_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, h->block_row, d.csr.idx, k2, ids);
+            DBS_TRY(sort_pairs(tp, k2, k2_alt, ids, ids_alt, (int64_t)n_entries, 27 + bits_for((uint64_t)d.nb), st));
+            DBS_CUDA(cudaMemcpyAsync(h->csc2csr, ids, (size_t)n_entries * 4, cudaMemcpyDeviceToDevice, st));
+            k_csc_gather<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, k2, h->csc2csr, d.csr.idx, d.csr.w, d.csr.aux, d.csc.idx, d.csc.w, d.csc.aux, bcol_sorted);
         }
-        k_lower_bounds<<<grid_for(d.nb + 1), TPB, 0, st>>>(d.nb, bcol_sorted, n_blocks, d.csc.ptr);
+        k_lower_bounds<<<grid_for(d.nb + 1), TPB, 0, st>>>(d.nb, bcol_sorted, n_entries, d.csc.ptr);
         DBS_CUDA(cudaStreamSynchronize(st));
         tp.release(k2); tp.release(k2_alt); tp.release(ids); tp.release(ids_alt); tp.release(bcol_sorted);
     }
@@ -564,8 +584,9 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     for (int c = 0; c < DBSPMSPV_BLK_NCLASS; ++c) { s.class_blocks[c] = (int64_t)cls_h[c]; s.class_nnz[c] = (int64_t)cls_h[DBSPMSPV_BLK_NCLASS + c]; }
     s.n_row_blocks = d.mb; s.n_col_blocks = d.nb; s.n_segments = d.n_segments;
     s.payload_bytes = h->payload_bytes;
-    s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)n_blocks * 9;
-    s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)n_blocks * 9;
+    s.n_view_entries = d.n_entries;
+    s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)d.n_entries * 9;
+    s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.n_entries * 9;
     s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment);
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
@@ -588,7 +609,7 @@ int create_common(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz, con
     dbspmspv_handle_s *h = new (std::nothrow) dbspmspv_handle_s();
     if (!h) return DBSPMSPV_ERR_ALLOC;
     if (opts) h->copts = *opts; else dbspmspv_default_create_opts(&h->copts);
-    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.w_coo < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
+    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.w_coo < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 16) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
     dbspmspv_default_run_opts(&h->ropts);
     h->d.dtype = dtype;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return DBSPMSPV_ERR_CUDA; }
@@ -611,6 +632,7 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     o->seg_cut = 128; o->w_dense = 4; o->w_mid = 2; o->w_coo = 1;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
+    o->inline_max = 4;
 }
 
 int dbspmspv_create_csr(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz,

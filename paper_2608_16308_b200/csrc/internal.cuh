@@ -42,9 +42,9 @@ constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-cl
 
 struct View {
     int32_t *ptr;    // nb_major + 1
-    uint32_t *idx;   // n_blocks
-    uint32_t *w;     // n_blocks
-    uint8_t *aux;    // n_blocks
+    uint32_t *idx;   // n_entries
+    uint32_t *w;     // n_entries
+    uint8_t *aux;    // n_entries
 };
 
 struct Segment {     // pull work unit: a run of consecutive blocks inside one row block
@@ -83,7 +83,7 @@ struct Workspace {
 struct Device {           // everything the kernels need, passed by value
     int64_t m, n;
     int32_t mb, nb;       // row blocks, column blocks
-    int32_t n_blocks;
+    int32_t n_entries;    // view entries (>= nonempty blocks: a small block is one entry per stored element)
     int32_t n_segments;
     int32_t dtype;
     View csr, csc;

@@ -133,6 +133,43 @@ __device__ __forceinline__ bool lane_owned(int type, uint32_t aux) {
     return type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX);
 }
 
+// The COO blocks held by the 32 lanes of a warp, processed as ONE flat list of stored entries:
+// a warp scan of the per-lane entry counts lays the entries out, then every lane takes one
+// entry per step and finds its owner block by a shuffle binary search over the scan.  This
+// keeps all lanes busy whatever the mix of block sizes (a lane looping over its own block
+// would make the whole warp wait for the largest block).  `cnt` is the lane's entry count
+// (0 = no COO block here), `tag` a per-block value handed back to `emit(tag, r, c, value, xm)`.
+template <int DT, typename Emit>
+__device__ __forceinline__ void warp_flat_coo(int cnt, uint32_t w, uint32_t xm, uint32_t tag,
+                                              const uint8_t *payload, int lane, Emit emit) {
+    int incl = cnt;
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(FULL, incl, o);
+        if (lane >= o) incl += t;
+    }
+    const int total = __shfl_sync(FULL, incl, 31);
+    for (int e0 = 0; e0 < total; e0 += 32) {
+        const int e = e0 + lane;
+        int o = 0;
+#pragma unroll
+        for (int s = 16; s; s >>= 1) {
+            const int v = __shfl_sync(FULL, incl, o + s - 1);
+            if (v <= e) o += s;
+        }
+        const int bn = __shfl_sync(FULL, cnt, o);
+        const int k = e - (__shfl_sync(FULL, incl, o) - bn);
+        const uint32_t bw = __shfl_sync(FULL, w, o);
+        const uint32_t bxm = __shfl_sync(FULL, xm, o);
+        const uint32_t btag = __shfl_sync(FULL, tag, o);
+        if (e < total) {
+            const uint8_t *blk = payload + (size_t)bw * 4;
+            const uint32_t rc = blk[k];
+            const int c = rc & 15, r = rc >> 4;
+            if ((bxm >> c) & 1u) emit(btag, r, c, Val<DT>::load(blk + ((bn + 3) & ~3), k), o);
+        }
+    }
+}
+
 // Push (Section 3.3.2): every warp takes one task = up to 32 consecutive block-CSC entries of
 // one active column block; the vector block is staged once per task (Section 3.3.3).  Lanes
 // own hypersparse blocks; heavier blocks are then processed by the whole warp one at a time.
@@ -157,17 +194,33 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
         if (lane < 16) s_x[lane] = d.ws.x_dense[jb * 16 + lane];
         __syncwarp();
         bool heavy = false;
+        int coo_cnt = 0;
+        const int type = idx >> TYPE_SHIFT;
+        const int brow = idx & IDX_MASK;
         if (have) {
-            const int type = idx >> TYPE_SHIFT;
-            const int brow = idx & IDX_MASK;
-            if (lane_owned(type, aux)) {
+            if (type == DBSPMSPV_BLK_INLINE) {
                 float *row0 = out.acc + (size_t)brow * 16;
                 const uint32_t hit = lane_block<DT>(type, w, aux, xm, s_x[aux & 15], s_x, d.payload,
                                                     [&](int r, float v) { atomicAdd(row0 + r, v); });
                 if (Out::MASKS && hit) atomicOr(&out.mask32[brow >> 1], hit << ((brow & 1) * 16));
+            } else if (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX) {
+                coo_cnt = (int)aux + 1;
             } else {
                 heavy = true;
             }
+        }
+        if (__any_sync(FULL, coo_cnt)) {
+            s_tmp[lane] = 0.f;   // per-owner-lane hit masks (bit patterns), 32 slots
+            __syncwarp();
+            uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_tmp);
+            warp_flat_coo<DT>(coo_cnt, w, xm, (uint32_t)brow, d.payload, lane,
+                              [&](uint32_t tag, int r, int c, float a, int owner) {
+                                  if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)tag * 16 + r, a * s_x[c]);
+                                  if (Out::MASKS) atomicOr(&s_hit[owner], 1u << r);
+                              });
+            __syncwarp();
+            if (Out::MASKS && coo_cnt && s_hit[lane]) atomicOr(&out.mask32[brow >> 1], s_hit[lane] << ((brow & 1) * 16));
+            __syncwarp();
         }
         uint32_t hv = __ballot_sync(FULL, heavy);
         while (hv) {
@@ -176,17 +229,17 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
             const uint32_t bidx = __shfl_sync(FULL, idx, src);
             const uint32_t bw = __shfl_sync(FULL, w, src);
             const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
-            const int type = bidx >> TYPE_SHIFT;
-            const int brow = bidx & IDX_MASK;
+            const int btype = bidx >> TYPE_SHIFT;
+            const int bbrow = bidx & IDX_MASK;
             const uint8_t *blk = d.payload + (size_t)bw * 4;
             uint32_t hits;
             if (DT == DBSPMSPV_PATTERN) {
-                hits = warp_block_bool<DT>(type, blk, nnz, xm, lane);
+                hits = warp_block_bool<DT>(btype, blk, nnz, xm, lane);
             } else {
-                const float sum = warp_block<DT>(type, blk, nnz, xm, s_x, s_tmp, lane, popc_threshold, hits);
-                if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(out.acc + (size_t)brow * 16 + lane, sum);
+                const float sum = warp_block<DT>(btype, blk, nnz, xm, s_x, s_tmp, lane, popc_threshold, hits);
+                if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(out.acc + (size_t)bbrow * 16 + lane, sum);
             }
-            if (Out::MASKS && lane == 0 && hits) atomicOr(&out.mask32[brow >> 1], hits << ((brow & 1) * 16));
+            if (Out::MASKS && lane == 0 && hits) atomicOr(&out.mask32[bbrow >> 1], hits << ((bbrow & 1) * 16));
         }
         __syncwarp();
     }
@@ -234,15 +287,24 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
             for (int u = 0; u < PULL_UNROLL; ++u) {
                 if (base + u * 32 >= end) break;   // warp-uniform
                 bool heavy = false;
+                int coo_cnt = 0;
+                const int bcol_l = idx[u] & IDX_MASK;
                 if (xm[u]) {
                     const int type = idx[u] >> TYPE_SHIFT;
-                    const int bcol = idx[u] & IDX_MASK;
-                    if (lane_owned(type, aux[u]))
-                        hit |= lane_block<DT>(type, w[u], aux[u], xm[u], xin[u], d.ws.x_dense + (size_t)bcol * 16,
-                                              d.payload, [&](int r, float v) { atomicAdd(&s_y[r], v); });
+                    if (type == DBSPMSPV_BLK_INLINE)
+                        hit |= lane_block<DT>(type, w[u], aux[u], xm[u], xin[u], nullptr, d.payload,
+                                              [&](int r, float v) { atomicAdd(&s_y[r], v); });
+                    else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX)
+                        coo_cnt = (int)aux[u] + 1;
                     else
                         heavy = true;
                 }
+                if (__any_sync(FULL, coo_cnt))
+                    warp_flat_coo<DT>(coo_cnt, w[u], xm[u], (uint32_t)bcol_l, d.payload, lane,
+                                      [&](uint32_t tag, int r, int c, float a, int) {
+                                          if (DT != DBSPMSPV_PATTERN) atomicAdd(&s_y[r], a * d.ws.x_dense[(size_t)tag * 16 + c]);
+                                          hit |= 1u << r;
+                                      });
                 uint32_t hv = __ballot_sync(FULL, heavy);
                 while (hv) {
                     const int src = __ffs(hv) - 1;
@@ -292,7 +354,7 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
 
 template <int DT, typename Out>
 __global__ void __launch_bounds__(CTA) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
-    __shared__ float s_x[WARPS][16], s_tmp[WARPS][16], s_y[WARPS][16];
+    __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16];
     const int warp = threadIdx.x >> 5;
     const int path = select_path(d, th3, force_path);
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
@@ -435,7 +497,7 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     Workspace &ws = d.ws;
     int64_t total = 0;
     const size_t xwords = (size_t)(d.nb + 1) / 2 + 4, ywords = (size_t)(d.mb + 1) / 2 + 4;
-    ws.task_capacity = (int64_t)d.n_blocks / PUSH_CHUNK + d.nb + 32;
+    ws.task_capacity = (int64_t)d.n_entries / PUSH_CHUNK + d.nb + 32;
     ws.n_tiles = (int32_t)ceil_div<int64_t>((d.mb + 1) / 2, TILE_WORDS);
     if (ws.n_tiles < 1) ws.n_tiles = 1;
 #define DBS_WS(expr) do { int s__ = (expr); if (s__ != DBSPMSPV_OK) return s__; } while (0)
@@ -461,7 +523,7 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     if (!grid) grid = compute_grid<DT, OutSparse>(h->sm_count);
     if (nnz_x > 0) k_xblock_sparse<DT><<<(nnz_x + 255) / 256, 256, 0, st>>>(d, x_idx, semiring == DBSPMSPV_OR_AND ? nullptr : x_val, nnz_x, h->ropts.validate);
     OutSparse out{d.ws.y_acc, d.ws.y_mask32};
-    if (nnz_x > 0 && d.n_blocks > 0) k_compute<DT, OutSparse><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold);
+    if (nnz_x > 0 && d.n_entries > 0) k_compute<DT, OutSparse><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold);
     const int nt = d.ws.n_tiles;
     k_compact_count<<<nt, CMP_TPB, 0, st>>>(d);
     int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
@@ -482,7 +544,7 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
     if (g > 8 * h->sm_count) g = 8 * h->sm_count;
     k_xblock_dense<DT><<<g, 256, 0, st>>>(d, x, y);
     OutDense out{y, nullptr};
-    if (d.n_blocks > 0) k_compute<DT, OutDense><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold);
+    if (d.n_entries > 0) k_compute<DT, OutDense><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold);
     int gc = ((d.nb + 1) / 2 + 255) / 256;
     if (gc > h->sm_count) gc = h->sm_count;
     k_decode_cleanup<<<gc, 256, 0, st>>>(d);

@@ -80,7 +80,7 @@ class Handle:
         return r[order], c[order], (None if v is None else v[order])
 
     def export_blocks(self):
-        nb = int(self.stats.n_blocks)
+        nb = int(self.stats.n_view_entries)
         out = [torch.empty(max(nb, 1), dtype=torch.int32, device=DEV) for _ in range(4)]
         B.dbspmspv_export_blocks(self.h, *out)
         return [t[:nb].cpu().numpy() for t in out]
@@ -89,10 +89,10 @@ class Handle:
         s = self.stats
         a = torch.empty(s.n_row_blocks + 1, dtype=torch.int32, device=DEV)
         b = torch.empty(s.n_col_blocks + 1, dtype=torch.int32, device=DEV)
-        c = torch.empty(max(s.n_blocks, 1), dtype=torch.int32, device=DEV)
-        d = torch.empty(max(s.n_blocks, 1), dtype=torch.int32, device=DEV)
+        c = torch.empty(max(s.n_view_entries, 1), dtype=torch.int32, device=DEV)
+        d = torch.empty(max(s.n_view_entries, 1), dtype=torch.int32, device=DEV)
         B.dbspmspv_export_views(self.h, a, b, c, d)
-        nb = int(s.n_blocks)
+        nb = int(s.n_view_entries)
         return a.cpu().numpy(), b.cpu().numpy(), c[:nb].cpu().numpy(), d[:nb].cpu().numpy()
 
     def get_stats(self, **kw):

@@ -20,7 +20,7 @@ def cpu_classify(rows, cols, dtype, th0=32, th1=128, th2=2.0):
     key, rows, cols = key[order], rows[order], cols[order]
     ub, start, cnt = np.unique(key, return_index=True, return_counts=True)
     cls = np.empty(ub.size, dtype=np.int32)
-    cap = 4 if dtype == B.PATTERN else 1
+    cap = 4          # default inline_max; pattern entries hold up to four coordinates
     for b in range(ub.size):
         n = cnt[b]
         if n < th0:
@@ -87,24 +87,38 @@ def test_export_equals_input_and_census(name, make, dtype):
         assert np.array_equal(v.view(np.uint32), csr.val.view(np.uint32))      # bit exact
     elif dtype == B.BF16:
         assert np.array_equal(v.view(np.uint16), to_bf16_bits(csr.val))
-    br, bc, cls, bn = h.export_blocks()
+    er, ec, ecls, en = h.export_blocks()                 # per view entry, primary order
     wr, wc, wcls, wn = cpu_classify(csr.rows(), csr.col_idx, dtype)
-    assert np.array_equal(br, wr) and np.array_equal(bc, wc)                    # primary order
+    # entries -> blocks: the entries of one block are adjacent
+    ekey = er.astype(np.int64) << 32 | ec
+    assert (np.diff(ekey) >= 0).all()                                           # primary order
+    first = np.r_[True, np.diff(ekey) != 0]
+    br, bc, cls = er[first], ec[first], ecls[first]
+    bn = np.add.reduceat(en, np.flatnonzero(first)) if en.size else en
+    assert np.array_equal(br, wr) and np.array_equal(bc, wc)
     assert np.array_equal(bn, wn) and int(bn.sum()) == csr.nnz
     assert np.array_equal(cls, wcls)
+    if dtype == B.PATTERN:
+        assert first.all()                                                      # one entry per block
+    else:
+        assert (en[ecls == B.BLK_INLINE] == 1).all() and first[ecls != B.BLK_INLINE].all()
+    assert s.n_blocks == wr.size and s.n_view_entries == er.size
     for k in range(6):
         assert s.class_blocks[k] == int((wcls == k).sum())
         assert s.class_nnz[k] == int(wn[wcls == k].sum())
-    # dual view: same block set, CSC order, consistent pointers
+    # dual view: same entry set, CSC order, consistent pointers
     rp, cp, crow, c2r = h.export_views()
-    nb = br.size
-    assert rp[0] == 0 and rp[-1] == nb and cp[0] == 0 and cp[-1] == nb
-    assert np.array_equal(np.diff(rp), np.bincount(br, minlength=s.n_row_blocks))
-    assert np.array_equal(np.diff(cp), np.bincount(bc, minlength=s.n_col_blocks))
-    assert np.array_equal(np.sort(c2r), np.arange(nb))                          # a permutation
-    assert np.array_equal(crow, br[c2r])
-    ccol = bc[c2r]
-    assert (np.diff(ccol.astype(np.int64) * (1 << 32) + crow) > 0).all()        # sorted by (col, row)
+    ne = er.size
+    assert rp[0] == 0 and rp[-1] == ne and cp[0] == 0 and cp[-1] == ne
+    assert np.array_equal(np.diff(rp), np.bincount(er, minlength=s.n_row_blocks))
+    assert np.array_equal(np.diff(cp), np.bincount(ec, minlength=s.n_col_blocks))
+    assert np.array_equal(np.sort(c2r), np.arange(ne))                          # a permutation
+    assert np.array_equal(crow, er[c2r])
+    ccol = ec[c2r]
+    ckey = ccol.astype(np.int64) * (1 << 32) + crow
+    assert (np.diff(ckey) >= 0).all()                                           # sorted by (col, row)
+    same = np.diff(ckey) == 0
+    assert (np.diff(c2r)[same] == 1).all()                                      # a block's entries stay in order
     h.close()
 
 
@@ -134,7 +148,8 @@ def test_threshold_edges():
     assert cls_of(full[:128]) != B.BLK_DENSE
     assert cls_of(full[:129]) == B.BLK_DENSE
     assert cls_of(full[:1]) == B.BLK_INLINE
-    assert cls_of(full[:2]) == B.BLK_COO
+    assert cls_of(full[:4]) == B.BLK_INLINE
+    assert cls_of(full[:5]) == B.BLK_COO
     # 32 entries as two full rows: max row 16, max col 2 -> ForceCSR
     assert cls_of(full[:32]) == B.BLK_FCSR
     assert cls_of([(c, r) for r, c in full[:32]]) == B.BLK_FCSC
@@ -178,7 +193,7 @@ def test_forced_formats_round_trip(fmt):
     o.force_format = fmt
     h = Handle(csr, B.F32, opts=o)
     want = B.BLK_COO if fmt == B.FORMAT_COO else B.BLK_CSR
-    assert (h.export_blocks()[2] == want).all()
+    assert (h.export_blocks()[2] == want).all() and h.stats.n_view_entries == h.stats.n_blocks
     r, c, v = h.export_coo()
     assert np.array_equal(r, csr.rows()) and np.array_equal(c, csr.col_idx)
     assert np.array_equal(v.view(np.uint32), csr.val.view(np.uint32))
