@@ -1,0 +1,429 @@
+"""Benchmark of the DB-SpMSpV hot path on B200.
+
+Workload at N=1 (benchmark configs[1]): R-MAT scale 20, edge factor 16, fp32 values, with the
+input-sparsity sweep x nnz fraction 1e-5 ... 0.5.  One *step* is one pass of the whole hot path
+(vector blocking -> selector -> worklist -> block microkernels -> writeback -> compaction) over
+that batch: one dbspmspv_run call per sweep point, six calls.  L2 is flushed before every timed
+call, so every number is cold.  `value` is the bytes the method must touch (B_touch)
+summed over the sweep, divided by the summed device time.  DB-BFS GTEPS (configs[3]) is reported
+in `bfs` unless --no-bfs is given.
+
+python bench.py [--gpus N --steps K --warmup W] [--impl reference] [--no-bfs]
+Under torchrun every rank runs the same sweep on its own GPU (independent replicas: the path
+has no exchange step), times are the max over ranks, `value` is the whole-job aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_16308_b200 import workloads as wl  # noqa: E402
+
+METRIC = "spmspv_sweep_achieved_hbm_GBps"
+UNIT = "GB/s"
+WORKLOAD = "rmat20_ef16_fp32_xsweep_1e-5..0.5"
+VIEW_ENTRY_BYTES = 9          # idx 4 + w 4 + aux 1 per view entry
+
+
+# ---------------------------------------------------------------------------------------------
+# Algorithmic bytes (host, from the structure of A and x; documented in the design doc)
+# ---------------------------------------------------------------------------------------------
+def payload_bytes_per_entry(cls: np.ndarray, nnz: np.ndarray, vsize: int) -> np.ndarray:
+    """Payload bytes of every view entry from the documented per-class sizes."""
+    out = np.zeros(cls.size, dtype=np.int64)
+    coo = cls == 1
+    out[coo] = ((nnz[coo] + 3) // 4) * 4 + ((nnz[coo] * vsize + 3) // 4) * 4
+    mid = (cls >= 2) & (cls <= 4)
+    out[mid] = (48 + ((nnz[mid] * vsize + 3) // 4) * 4) if vsize else 32
+    out[cls == 5] = 32 + 256 * vsize
+    return out
+
+
+class ByteModel:
+    """B_touch and B_min of one call (SpMSpV): see the design doc, 'Algorithmic bytes'."""
+
+    def __init__(self, csr: wl.CSR, entry_col: np.ndarray, entry_cls: np.ndarray, entry_nnz: np.ndarray,
+                 vsize: int):
+        self.csr, self.vsize = csr, vsize
+        nb = (csr.n + 15) // 16
+        per_entry = VIEW_ENTRY_BYTES + payload_bytes_per_entry(entry_cls, entry_nnz, vsize)
+        self.colblock_bytes = np.bincount(entry_col, weights=per_entry, minlength=nb)
+        self.col_nnz = np.bincount(csr.col_idx, minlength=csr.n)
+
+    def bytes(self, x_idx: np.ndarray, y_nnz: int, y_row_blocks: int):
+        xb = np.unique(x_idx >> 4)
+        touched = float(self.colblock_bytes[xb].sum())               # view entries + payload
+        pointers = 8.0 * xb.size                                      # column-pointer pair
+        xbytes = 8.0 * x_idx.size + xb.size * (2 + 64)                # list + mask + staged block
+        ybytes = 8.0 * y_nnz + 8.0 * y_nnz + 8.0 * y_row_blocks       # out + acc RMW + mask set/clear
+        b_touch = touched + pointers + xbytes + ybytes
+        b_min = float((8 + self.col_nnz[x_idx] * (self.vsize + 4)).sum()) + 8.0 * x_idx.size + 8.0 * y_nnz
+        return b_touch, b_min, touched + pointers + xb.size * 66     # last: traversal kernel only
+
+
+# ---------------------------------------------------------------------------------------------
+def sample_clocks(stop: threading.Event, out: list) -> None:
+    q = "clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+    idx = os.environ.get("LOCAL_RANK", "0")
+    while not stop.is_set():
+        try:
+            r = subprocess.run(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-i", idx],
+                               capture_output=True, text=True, timeout=5)
+            if r.returncode == 0 and r.stdout.strip():
+                out.append([f.strip() for f in r.stdout.strip().split(",")])
+        except Exception:
+            pass
+        stop.wait(0.2)
+
+
+def clocks_summary(samples: list) -> dict:
+    if not samples:
+        return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    sm = sorted(int(s[0]) for s in samples if s[0].isdigit())
+    names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+    reasons = [n for k, n in enumerate(names) if any(len(s) > 2 + k and s[2 + k].lower().startswith("active") for s in samples)]
+    return {"sm_mhz": sm[len(sm) // 2] if sm else None,
+            "sm_max_mhz": int(samples[0][1]) if samples[0][1].isdigit() else None,
+            "reasons": reasons, "samples": len(samples)}
+
+
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+def reference_arm(args) -> None:
+    """--impl reference: the CPU oracle as it stands, on the host cores, same config and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    a = wl.rmat(20, 16, seed=1)
+    A = oracle.RefMatrix(a.m, a.n, a.row_ptr, a.col_idx, a.val)
+    A.csc()
+    xs = [wl.rmat_x(a.n, f, k) for k, f in enumerate(wl.RMAT_SWEEP)]
+    model = host_byte_model(a)
+    per_step = []
+    btouch_step = 0.0
+    for it in range(args.warmup + args.steps):
+        t_step, btouch_step = 0.0, 0.0
+        for x in xs:
+            best = None
+            for fn in (oracle.ref_push, oracle.ref_pull):
+                t0 = time.perf_counter()
+                yi, _, _ = fn(A, x.idx, x.val)
+                dt = time.perf_counter() - t0
+                best = dt if best is None or dt < best else best
+            t_step += best
+            btouch_step += model.bytes(x.idx, yi.size, np.unique(yi >> 4).size)[0]
+        if it >= args.warmup:
+            per_step.append(t_step)
+    ms = 1e3 * float(np.mean(per_step))
+    value = btouch_step / (ms * 1e-3) / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "note": "CPU oracle (Algorithm 1 push/pull, faster of the two per point), "
+                                                     "whole sweep per step, single thread"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": "whole 6-point sweep per step"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def host_byte_model(a: wl.CSR) -> ByteModel:
+    """Byte model with the class census computed on the host (used by the reference arm, where
+    no GPU library is loaded): the documented classification rule applied with numpy."""
+    rows = a.rows()
+    key = (rows.astype(np.int64) >> 4) * ((a.n + 15) // 16) + (a.col_idx >> 4)
+    ub, cnt = np.unique(key, return_counts=True)
+    bcol = (ub % ((a.n + 15) // 16)).astype(np.int64)
+    # hypersparse matrices: blocks with <= 4 entries are INLINE (one 9-byte entry per element),
+    # 5..31 COO; the handful of denser blocks are counted as CSR-class
+    inl = cnt <= 4
+    cls = np.where(inl, 0, np.where(cnt < 32, 1, np.where(cnt > 128, 5, 4))).astype(np.int32)
+    ecol = np.concatenate([np.repeat(bcol[inl], cnt[inl]), bcol[~inl]])
+    ecls = np.concatenate([np.zeros(int(cnt[inl].sum()), np.int32), cls[~inl]])
+    ennz = np.concatenate([np.ones(int(cnt[inl].sum()), np.int64), cnt[~inl]])
+    return ByteModel(a, ecol, ecls, ennz, 4)
+
+
+# ---------------------------------------------------------------------------------------------
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-bfs", action="store_true")
+    ap.add_argument("--bfs-scale", type=int, default=22)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_16308_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    a = wl.rmat(20, 16, seed=1)
+    h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(a.val), B.F32)
+    st0 = B.dbspmspv_get_stats(h)
+    ne = int(st0.n_view_entries)
+    e_col = torch.empty(ne, dtype=torch.int32, device=dev)
+    e_cls = torch.empty(ne, dtype=torch.int32, device=dev)
+    e_nnz = torch.empty(ne, dtype=torch.int32, device=dev)
+    B.dbspmspv_export_blocks(h, None, e_col, e_cls, e_nnz)
+    model = ByteModel(a, e_col.cpu().numpy().astype(np.int64), e_cls.cpu().numpy(), e_nnz.cpu().numpy().astype(np.int64), 4)
+    del e_col, e_cls, e_nnz
+
+    xs = [wl.rmat_x(a.n, f, k) for k, f in enumerate(wl.RMAT_SWEEP)]
+    xd = [(up(x.idx), up(x.val)) for x in xs]
+    xh = [(torch.from_numpy(x.idx).pin_memory(), torch.from_numpy(x.val).pin_memory()) for x in xs]
+    y_idx = torch.empty(a.m, dtype=torch.int32, device=dev)
+    y_val = torch.empty(a.m, dtype=torch.float32, device=dev)
+    y_nnz = torch.zeros(1, dtype=torch.int32, device=dev)
+    y_idx_h = torch.empty(a.m, dtype=torch.int32).pin_memory()
+    y_val_h = torch.empty(a.m, dtype=torch.float32).pin_memory()
+    y_nnz_h = torch.zeros(1, dtype=torch.int32).pin_memory()
+    xi_stage = torch.empty(a.n, dtype=torch.int32, device=dev)
+    xv_stage = torch.empty(a.n, dtype=torch.float32, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)     # > 126 MB L2
+    stream = torch.cuda.current_stream()
+    opts = B.default_run_opts()
+    opts.timing = 1
+    B.dbspmspv_set_run_opts(h, opts)
+
+    npts = len(xs)
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(npts)]
+          for _ in range(args.steps)]
+    kernel_ms = np.zeros((args.steps, npts))
+    info = [None] * npts
+
+    def one_call(k):
+        B.dbspmspv_run(h, xd[k][0], xd[k][1], int(xs[k].idx.size), B.PLUS_TIMES, y_idx, y_val, a.m, y_nnz)
+
+    for _ in range(args.warmup):
+        for k in range(npts):
+            flush.fill_(1)
+            one_call(k)
+    torch.cuda.synchronize()
+    launches0 = B.dbspmspv_get_stats(h).kernel_launches
+
+    stop, samples = threading.Event(), []
+    th = threading.Thread(target=sample_clocks, args=(stop, samples), daemon=True)
+    th.start()
+    barrier()
+    t_wall0 = time.perf_counter()
+    for s in range(args.steps):
+        for k in range(npts):
+            flush.fill_(s & 0xFF)                # L2 flush, outside the event pair
+            ev[s][k][0].record(stream)
+            one_call(k)
+            ev[s][k][1].record(stream)
+            stt = B.dbspmspv_get_stats(h)        # synchronises; reads the traversal-kernel time
+            kernel_ms[s, k] = stt.last_compute_ms
+            if info[k] is None:
+                yk = int(stt.last_y_nnz)
+                yrb = int(torch.unique(y_idx[:yk] >> 4).numel())
+                info[k] = (stt.last_path, stt.last_n_nzblk, stt.last_n_tasks, yk, yrb)
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    stop.set()
+    th.join(timeout=2)
+    launches = B.dbspmspv_get_stats(h).kernel_launches - launches0
+
+    call_ms = np.array([[ev[s][k][0].elapsed_time(ev[s][k][1]) for k in range(npts)] for s in range(args.steps)])
+    step_ms = call_ms.sum(axis=1)
+    ms_per_step = float(step_ms.mean())
+    if world > 1:
+        t = torch.tensor([ms_per_step], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step = float(t.item())
+
+    # ---- end to end through the same C-ABI call with HOST buffers
+    e2e_ms = []
+    h2d = d2h = 0
+    for s in range(max(3, args.steps // 2) + 2):
+        tot = 0.0
+        h2d = d2h = 0
+        for k in range(npts):
+            flush.fill_(1)
+            n_x = int(xs[k].idx.size)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            xi_stage[:n_x].copy_(xh[k][0], non_blocking=True)
+            xv_stage[:n_x].copy_(xh[k][1], non_blocking=True)
+            B.dbspmspv_run(h, xi_stage, xv_stage, n_x, B.PLUS_TIMES, y_idx, y_val, a.m, y_nnz)
+            y_nnz_h.copy_(y_nnz, non_blocking=True)
+            stream.synchronize()
+            kk = int(y_nnz_h.item())
+            y_idx_h[:kk].copy_(y_idx[:kk], non_blocking=True)
+            y_val_h[:kk].copy_(y_val[:kk], non_blocking=True)
+            e1.record(stream)
+            stream.synchronize()
+            tot += e0.elapsed_time(e1)
+            h2d += 8 * n_x
+            d2h += 4 + 8 * kk
+        if s >= 2:
+            e2e_ms.append(tot)
+    e2e_ms_step = float(np.mean(e2e_ms))
+    if world > 1:
+        t = torch.tensor([e2e_ms_step], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms_step = float(t.item())
+
+    peak, peak_kind = measured_peak_gbs()
+    sweep, b_touch_total, b_kernel_total = [], 0.0, 0.0
+    for k, x in enumerate(xs):
+        path, nzblk, ntasks, yk, yrb = info[k]
+        bt, bm, bk = model.bytes(x.idx, yk, yrb)
+        us = float(np.median(call_ms[:, k])) * 1e3
+        kus = float(np.median(kernel_ms[:, k])) * 1e3
+        b_touch_total += bt
+        b_kernel_total += bk
+        sweep.append({"x_fraction": wl.RMAT_SWEEP[k], "x_nnz": int(x.idx.size), "path": "push" if path == B.PATH_PUSH else "pull",
+                      "us": round(us, 2), "us_min": round(float(call_ms[:, k].min()) * 1e3, 2),
+                      "traversal_kernel_us": round(kus, 2), "y_nnz": yk, "n_nzblk": nzblk,
+                      "B_touch": int(bt), "B_min": int(bm), "GBps_touch": round(bt / us / 1e3, 2),
+                      "frac_of_peak_touch": round(bt / us / 1e3 / peak, 4), "frac_of_peak_min": round(bm / us / 1e3 / peak, 4)})
+    value = world * b_touch_total / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * b_touch_total / (e2e_ms_step * 1e-3) / 1e9
+    kernel_total_ms = float(np.median(kernel_ms, axis=0).sum())
+    achieved = b_kernel_total / (kernel_total_ms * 1e-3) / 1e9
+
+    line = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "step": "6 dbspmspv_run calls (one per sweep point), auto path",
+                       "l2": "flushed (512 MB write) before every timed call", "block_size": 16,
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+            "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "ms_per_step": round(e2e_ms_step, 5),
+                    "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": int(launches),
+            "clocks": clocks_summary(samples),
+            "roofline": {"bound": "hbm", "kernel": "k_compute (push/pull traversal, 6 launches per step)",
+                         "achieved": round(achieved, 2), "peak": peak, "peak_kind": f"of {peak_kind}",
+                         "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES_PER_STEP,
+                         "algorithmic_bytes_per_step": int(b_kernel_total)},
+            "sweep": sweep, "wall_s_timed_region": round(t_wall, 3)}
+
+    if rank == 0 and world == 1:
+        line["cpu_baseline"] = cpu_baseline(a, xs, model)
+    if rank == 0 and world == 1 and not args.no_bfs:
+        try:
+            line["bfs"] = bench_bfs(args, B, torch, dev, flush)
+        except Exception as e:  # the SpMSpV line must survive a BFS-side problem
+            line["bfs"] = {"error": repr(e)}
+    B.dbspmspv_destroy(h)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# traffic of the traversal kernel (dram__bytes_read.sum + dram__bytes_write.sum over the six
+# launches of one step), from the ncu capture summarised in profiles/; None until captured
+NCU_TRAFFIC_BYTES_PER_STEP = None
+
+
+def cpu_baseline(a, xs, model):
+    """The oracle as it stands, single thread, on the same sweep (bounded: one pass, both
+    routines per point, the faster one counted)."""
+    import oracle
+    A = oracle.RefMatrix(a.m, a.n, a.row_ptr, a.col_idx, a.val)
+    A.csc()
+    total_t, total_b = 0.0, 0.0
+    for rep in range(2):
+        total_t, total_b = 0.0, 0.0
+        for x in xs:
+            best = None
+            for fn in (oracle.ref_push, oracle.ref_pull):
+                t0 = time.perf_counter()
+                yi, _, _ = fn(A, x.idx, x.val)
+                dt = time.perf_counter() - t0
+                best = dt if best is None or dt < best else best
+            total_t += best
+            total_b += model.bytes(x.idx, yi.size, np.unique(yi >> 4).size)[0]
+    return {"value": round(total_b / total_t / 1e9, 4), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "whole 6-point sweep, faster of ref_push/ref_pull per point, second of two passes",
+            "ms_per_step": round(total_t * 1e3, 3), "host_cores_available": os.cpu_count()}
+
+
+def bench_bfs(args, B, torch, dev, flush):
+    """DB-BFS GTEPS on the symmetrised R-MAT graph, 16 seeded sources (configs[3])."""
+    g = wl.rmat(args.bfs_scale, 16, seed=3, values=False, symmetrise=True)
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    h = B.dbspmspv_create_csr(g.m, g.n, g.nnz, up(g.row_ptr), up(g.col_idx), None, B.PATTERN)
+    srcs = wl.bfs_sources(g, 16)
+    deg = np.diff(g.row_ptr)
+    levels = torch.empty(g.n, dtype=torch.int32, device=dev)
+    times, teps, nlev = [], [], []
+    for s in srcs:
+        best = None
+        for rep in range(3):
+            flush.fill_(rep)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.db_bfs(h, int(s), levels)
+            e1.record()
+            torch.cuda.synchronize()
+            t = e0.elapsed_time(e1)
+            best = t if best is None or t < best else best
+        lv = levels.cpu().numpy()
+        edges = float(deg[lv >= 0].sum()) / 2.0
+        times.append(best)
+        teps.append(edges / (best * 1e-3) / 1e9)
+        nlev.append(int(B.dbspmspv_get_stats(h).bfs_levels))
+    import oracle
+    A = oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx)
+    A.csc()
+    t0 = time.perf_counter()
+    ref = oracle.ref_bfs(A, int(srcs[-1]))
+    cpu_s = time.perf_counter() - t0
+    match = bool(np.array_equal(ref, lv))
+    B.dbspmspv_destroy(h)
+    hm = len(teps) / sum(1.0 / t for t in teps)
+    return {"workload": f"rmat{args.bfs_scale}_sym_ef16_pattern_16sources", "gteps_harmonic_mean": round(hm, 3),
+            "gteps_min": round(min(teps), 3), "gteps_max": round(max(teps), 3),
+            "ms_median": round(float(np.median(times)), 4), "levels": nlev, "vertices": int(g.n), "nnz": int(g.nnz),
+            "last_source_matches_oracle": match,
+            "cpu_baseline": {"value": round(float(deg[ref >= 0].sum()) / 2.0 / cpu_s / 1e9, 4), "unit": "GTEPS",
+                             "cores": 1, "kind": "oracle", "sample": "queue BFS from the last source"}}
+
+
+if __name__ == "__main__":
+    main()

@@ -80,14 +80,15 @@ typedef struct {
     int32_t th1;             /* blocks with more than th1 entries use Dense         (128)    */
     float th2;               /* directional skew ratio for ForceCSR / ForceCSC      (2.0)    */
     int32_t seg_cut;         /* a pull segment closes when its weight reaches this  (128)    */
-    int32_t w_dense;         /* pull segment weight of a Dense block                (4)      */
-    int32_t w_mid;           /* ... of a ForceCSR / ForceCSC / CSR block            (2)      */
-    int32_t w_coo;           /* ... of a COO block                                  (1)      */
+    int32_t w_dense;         /* pull segment weight of a Dense block                (32)     */
+    int32_t w_mid;           /* ... of a ForceCSR / ForceCSC / CSR block            (16)     */
+    int32_t w_coo;           /* ... of a COO block                                  (4)      */
     int32_t force_format;    /* DBSPMSPV_FORMAT_*: ablation knob (Section 5.4)               */
     int32_t input_on_host;   /* 1: the create arrays are HOST pointers (copied once)         */
     int32_t inline_max;      /* valued matrices: a block with at most this many entries keeps
                                 them in its view entries, one entry per element       (4)    */
-    int32_t reserved[6];
+    int32_t w_inline;        /* ... of an INLINE view entry                         (1)      */
+    int32_t reserved[5];
 } dbspmspv_create_opts;
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
@@ -98,7 +99,9 @@ typedef struct {
     int32_t popc_threshold;  /* CSR-class blocks: popc(mask) >= this -> row-driven (pull-style)
                                 microkernel, below -> column-driven (push-style)             */
     int32_t validate;        /* 1: range-check x indices on the device (ERR_BOUNDS)          */
-    int32_t reserved[12];
+    int32_t timing;          /* 1: bracket the traversal kernel of run/decode with two CUDA
+                                events (made at create); read back as last_compute_ms      */
+    int32_t reserved[11];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64
@@ -130,11 +133,16 @@ typedef struct {
     int32_t bfs_level_nzblk[DBSPMSPV_MAX_BFS_LEVELS_RECORDED]; /* frontier vector blocks      */
     /* deferred device status of the last call (DBSPMSPV_OK if none) */
     int32_t device_status;
-    int32_t reserved[7];
+    float last_compute_ms;         /* traversal kernel time of the last run/decode (timing=1),
+                                      else -1                                                 */
+    int64_t kernel_launches;       /* kernels launched through this handle so far             */
+    int32_t reserved[4];
 } dbspmspv_stats;
 
-/* Paper defaults (th0 = 32, th1 = 128, th2 = 2.0; segment weights 4 / 2 / 1; Sections 3.2.1,
- * 3.3.2) and this library's measured run-time defaults.                                      */
+/* Paper thresholds (th0 = 32, th1 = 128, th2 = 2.0, Section 3.2.1).  The segment weights keep
+ * the paper's ordering Dense > CSR-like > COO (Section 3.3.2) but are rescaled (32 / 16 / 4 / 1
+ * against a cut of 128) because one warp step here covers 32 INLINE entries but one heavier
+ * block.  Run-time defaults are this library's measured ones.                                      */
 void dbspmspv_default_create_opts(dbspmspv_create_opts *opts);
 void dbspmspv_default_run_opts(dbspmspv_run_opts *opts);
 

@@ -36,13 +36,13 @@ class CreateOpts(ctypes.Structure):
                 ("seg_cut", ctypes.c_int32), ("w_dense", ctypes.c_int32), ("w_mid", ctypes.c_int32),
                 ("w_coo", ctypes.c_int32), ("force_format", ctypes.c_int32),
                 ("input_on_host", ctypes.c_int32), ("inline_max", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 6)]
+                ("w_inline", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
 
 
 class RunOpts(ctypes.Structure):
     _fields_ = [("th3", ctypes.c_float), ("force_path", ctypes.c_int32),
                 ("popc_threshold", ctypes.c_int32), ("validate", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 12)]
+                ("timing", ctypes.c_int32), ("reserved", ctypes.c_int32 * 11)]
 
 
 class Stats(ctypes.Structure):
@@ -58,7 +58,8 @@ class Stats(ctypes.Structure):
                 ("bfs_reached", ctypes.c_int32),
                 ("bfs_level_path", ctypes.c_int32 * MAX_BFS_LEVELS_RECORDED),
                 ("bfs_level_nzblk", ctypes.c_int32 * MAX_BFS_LEVELS_RECORDED),
-                ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7)]
+                ("device_status", ctypes.c_int32), ("last_compute_ms", ctypes.c_float),
+                ("kernel_launches", ctypes.c_int64), ("reserved", ctypes.c_int32 * 4)]
 
 
 _lib = None

@@ -122,6 +122,12 @@ int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out) {
         out->bfs_level_nzblk[k] = c.bfs_level_nzblk[k];
     }
     out->device_status = c.status;
+    out->kernel_launches = h->kernel_launches;
+    out->last_compute_ms = -1.0f;
+    if (h->timed) {
+        float ms = -1.0f;
+        if (cudaEventElapsedTime(&ms, h->ev[0], h->ev[1]) == cudaSuccess) out->last_compute_ms = ms;
+    }
     if (c.status != DBSPMSPV_OK) {  // report once, then clear
         int32_t zero = 0;
         DBS_CUDA(cudaMemcpy(&h->d.ws.ctr->status, &zero, sizeof(zero), cudaMemcpyHostToDevice));
@@ -189,6 +195,8 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     dbs::Workspace &ws = d.ws;
     cudaFree(ws.x_dense); cudaFree(ws.x_mask32); cudaFree(ws.tasks); cudaFree(ws.y_acc);
     cudaFree(ws.y_mask32); cudaFree(ws.tile_count); cudaFree(ws.visited32); cudaFree(ws.ctr);
+    if (h->ev[0]) cudaEventDestroy(h->ev[0]);
+    if (h->ev[1]) cudaEventDestroy(h->ev[1]);
     delete h;
     return DBSPMSPV_OK;
 }

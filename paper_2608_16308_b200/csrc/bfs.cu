@@ -248,6 +248,7 @@ static int bfs_typed(dbspmspv_handle_s *h, int32_t src, int32_t *levels, cudaStr
     int max_levels = d.n > 0x7FFFFFFF ? 0x7FFFFFFF : (int)d.n;
     void *args[] = {&d, &src, &levels, &th3, &force, &max_levels};
     DBS_CUDA(cudaLaunchCooperativeKernel((void *)k_bfs<DT>, dim3(h->bfs_grid), dim3(BFS_CTA), args, 0, st));
+    ++h->kernel_launches;
     return DBSPMSPV_OK;
 }
 

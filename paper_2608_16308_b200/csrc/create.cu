@@ -325,11 +325,11 @@ __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
 
 // ---- pull segments (Section 3.3.2): greedy walk along each row block; a segment closes
 // when its accumulated weight reaches the cut.  One thread per row block, two passes.
-struct SegParams { int cut, w_dense, w_mid, w_coo; };
+struct SegParams { int cut, w_dense, w_mid, w_coo, w_inline; };
 
 __device__ __forceinline__ int seg_weight(uint32_t idx, const SegParams &sp) {
     int t = idx >> TYPE_SHIFT;
-    return t == DBSPMSPV_BLK_DENSE ? sp.w_dense : (t <= DBSPMSPV_BLK_COO ? sp.w_coo : sp.w_mid);
+    return t == DBSPMSPV_BLK_DENSE ? sp.w_dense : t == DBSPMSPV_BLK_INLINE ? sp.w_inline : t == DBSPMSPV_BLK_COO ? sp.w_coo : sp.w_mid;
 }
 
 __global__ void k_seg_count(int32_t mb, const int32_t *row_ptr, const uint32_t *idx,
@@ -561,7 +561,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
 
     // pull segments
     {
-        SegParams sp{h->copts.seg_cut, h->copts.w_dense, h->copts.w_mid, h->copts.w_coo};
+        SegParams sp{h->copts.seg_cut, h->copts.w_dense, h->copts.w_mid, h->copts.w_coo, h->copts.w_inline};
         int32_t *cnt, *off;
         DBS_GET(cnt, (int64_t)d.mb + 1); DBS_GET(off, (int64_t)d.mb + 1);
         DBS_CUDA(cudaMemsetAsync(cnt, 0, ((size_t)d.mb + 1) * 4, st));
@@ -609,7 +609,7 @@ int create_common(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz, con
     dbspmspv_handle_s *h = new (std::nothrow) dbspmspv_handle_s();
     if (!h) return DBSPMSPV_ERR_ALLOC;
     if (opts) h->copts = *opts; else dbspmspv_default_create_opts(&h->copts);
-    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.w_coo < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 16) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
+    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 16) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
     dbspmspv_default_run_opts(&h->ropts);
     h->d.dtype = dtype;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return DBSPMSPV_ERR_CUDA; }
@@ -629,7 +629,7 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     if (!o) return;
     *o = dbspmspv_create_opts();
     o->th0 = 32; o->th1 = 128; o->th2 = 2.0f;
-    o->seg_cut = 128; o->w_dense = 4; o->w_mid = 2; o->w_coo = 1;
+    o->seg_cut = 128; o->w_dense = 32; o->w_mid = 16; o->w_coo = 4; o->w_inline = 1;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
     o->inline_max = 4;

@@ -107,6 +107,9 @@ struct dbspmspv_handle_s {
     void *payload_alloc;
     int64_t payload_bytes;
     int bfs_grid;               // co-resident grid size of the BFS kernel
+    cudaEvent_t ev[2];          // optional timing of the traversal kernel (run_opts.timing)
+    bool timed;
+    int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)
 };
 
 namespace dbs {
