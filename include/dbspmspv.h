@@ -79,14 +79,14 @@ typedef struct {
     int32_t th0;             /* blocks with fewer than th0 entries use packed COO   (32)     */
     int32_t th1;             /* blocks with more than th1 entries use Dense         (128)    */
     float th2;               /* directional skew ratio for ForceCSR / ForceCSC      (2.0)    */
-    int32_t seg_cut;         /* a pull segment closes when its weight reaches this  (128)    */
+    int32_t seg_cut;         /* a pull segment closes when its weight reaches this  (128, max)*/
     int32_t w_dense;         /* pull segment weight of a Dense block                (32)     */
     int32_t w_mid;           /* ... of a ForceCSR / ForceCSC / CSR block            (16)     */
     int32_t w_coo;           /* ... of a COO block                                  (4)      */
     int32_t force_format;    /* DBSPMSPV_FORMAT_*: ablation knob (Section 5.4)               */
     int32_t input_on_host;   /* 1: the create arrays are HOST pointers (copied once)         */
     int32_t inline_max;      /* valued matrices: a block with at most this many entries keeps
-                                them in its view entries, one entry per element       (4)    */
+                                them in its view entries, one entry per element       (8)    */
     int32_t w_inline;        /* ... of an INLINE view entry                         (1)      */
     int32_t reserved[5];
 } dbspmspv_create_opts;

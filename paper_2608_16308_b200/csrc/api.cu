@@ -191,6 +191,8 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     cudaFree(d.csc.ptr); cudaFree(d.csc.idx); cudaFree(d.csc.w); cudaFree(d.csc.aux);
     cudaFree(h->payload_alloc);
     cudaFree(const_cast<dbs::Segment *>(d.segments));
+    cudaFree(const_cast<int2 *>(d.chunks));
+    cudaFree(const_cast<int32_t *>(d.seg_rb));
     cudaFree(h->csc2csr); cudaFree(h->block_row);
     dbs::Workspace &ws = d.ws;
     cudaFree(ws.x_dense); cudaFree(ws.x_mask32); cudaFree(ws.tasks); cudaFree(ws.y_acc);

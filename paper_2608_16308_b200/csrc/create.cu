@@ -345,8 +345,8 @@ __global__ void k_seg_count(int32_t mb, const int32_t *row_ptr, const uint32_t *
     count[rb] = c;
 }
 
-__global__ void k_seg_write(int32_t mb, const int32_t *row_ptr, const uint32_t *idx,
-                            SegParams sp, const int32_t *seg_off, Segment *segs) {
+__global__ void k_seg_write(int32_t mb, const int32_t *row_ptr, uint32_t *idx,
+                            SegParams sp, const int32_t *seg_off, Segment *segs, int32_t *seg_rb) {
     int64_t rb = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (rb >= mb) return;
     int acc = 0, first = row_ptr[rb];
@@ -359,11 +359,36 @@ __global__ void k_seg_write(int32_t mb, const int32_t *row_ptr, const uint32_t *
             s.row_block = (int32_t)rb;
             s.start = first;
             s.count = (p + 1 - first) | ((first == row_ptr[rb] && p + 1 == end) ? (int32_t)0x80000000 : 0);
+            s.weight = acc;
+            seg_rb[o] = (int32_t)rb;
             segs[o++] = s;
+            idx[first] |= 1u << 28;   // first entry of a segment (bits 27, 28 of idx are spare)
             first = p + 1;
             acc = 0;
         }
     }
+}
+
+// pull chunks: consecutive segments grouped by accumulated weight; chunk k starts at the first
+// segment whose exclusive weight prefix is >= k * PULL_CH
+__global__ void k_seg_weights(int32_t n_segments, const Segment *segs, int32_t *w) {
+    int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (k < n_segments) w[k] = segs[k].weight;
+    if (k == n_segments) w[k] = 0;
+}
+
+__global__ void k_chunks(int32_t n_chunks, const Segment *segs, const int32_t *wprefix, int32_t n_segments,
+                         int32_t n_entries, int2 *chunks) {
+    int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (k > n_chunks) return;
+    if (k == n_chunks) { chunks[k] = make_int2(n_segments, n_entries); return; }
+    const int64_t target = k * (int64_t)PULL_CH;
+    int32_t lo = 0, hi = n_segments;
+    while (lo < hi) {
+        int32_t mid = lo + ((hi - lo) >> 1);
+        if (wprefix[mid] < target) lo = mid + 1; else hi = mid;
+    }
+    chunks[k] = make_int2(lo, lo < n_segments ? segs[lo].start : n_entries);
 }
 
 template <typename T>
@@ -525,7 +550,8 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         DBS_CUDA(cudaMemsetAsync(p, 0, h->payload_bytes + 256, st));
         h->payload_alloc = p; d.payload = p;
     }
-    DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_entries); DBS_KEEP(d.csr.w, n_entries); DBS_KEEP(d.csr.aux, n_entries);
+    DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_entries + VIEW_PAD); DBS_KEEP(d.csr.w, n_entries + VIEW_PAD); DBS_KEEP(d.csr.aux, n_entries + VIEW_PAD);
+    DBS_CUDA(cudaMemsetAsync(d.csr.idx + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.aux + n_entries, 0, VIEW_PAD, st));
     DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_entries); DBS_KEEP(d.csc.w, n_entries); DBS_KEEP(d.csc.aux, n_entries);
     DBS_KEEP(h->csc2csr, n_entries);
     DBS_KEEP(h->block_row, n_entries);
@@ -571,8 +597,21 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         DBS_CUDA(cudaMemcpy(&nseg, off + d.mb, 4, cudaMemcpyDeviceToHost));
         d.n_segments = nseg;
         Segment *segs; DBS_KEEP(segs, nseg);
-        k_seg_write<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, off, segs);
+        int32_t *seg_rb; DBS_KEEP(seg_rb, (int64_t)nseg + 1);
+        k_seg_write<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, off, segs, seg_rb);
+        d.seg_rb = seg_rb;
         d.segments = segs;
+        int32_t *segw, *segpre;
+        DBS_GET(segw, (int64_t)nseg + 1); DBS_GET(segpre, (int64_t)nseg + 1);
+        k_seg_weights<<<grid_for((int64_t)nseg + 1), TPB, 0, st>>>(nseg, segs, segw);
+        DBS_TRY(exclusive_sum(tp, segw, segpre, (int64_t)nseg + 1, st));
+        int32_t total_w = 0;
+        DBS_CUDA(cudaMemcpy(&total_w, segpre + nseg, 4, cudaMemcpyDeviceToHost));
+        if (total_w < 0) return DBSPMSPV_ERR_UNSUPPORTED;
+        d.n_chunks = (int32_t)(((int64_t)total_w + PULL_CH - 1) / PULL_CH);
+        int2 *chunks; DBS_KEEP(chunks, (int64_t)d.n_chunks + 1);
+        k_chunks<<<grid_for((int64_t)d.n_chunks + 1), TPB, 0, st>>>(d.n_chunks, segs, segpre, nseg, d.n_entries, chunks);
+        d.chunks = chunks;
         DBS_CUDA(cudaStreamSynchronize(st));
     }
 
@@ -587,7 +626,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     s.n_view_entries = d.n_entries;
     s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)d.n_entries * 9;
     s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.n_entries * 9;
-    s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment);
+    s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment) + ((int64_t)d.n_chunks + 1) * 8 + (int64_t)d.n_segments * 4;
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }
@@ -609,7 +648,7 @@ int create_common(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz, con
     dbspmspv_handle_s *h = new (std::nothrow) dbspmspv_handle_s();
     if (!h) return DBSPMSPV_ERR_ALLOC;
     if (opts) h->copts = *opts; else dbspmspv_default_create_opts(&h->copts);
-    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 16) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
+    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.seg_cut > MAX_SEG_ENTRIES || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 16) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
     dbspmspv_default_run_opts(&h->ropts);
     h->d.dtype = dtype;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return DBSPMSPV_ERR_CUDA; }
@@ -632,7 +671,7 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     o->seg_cut = 128; o->w_dense = 32; o->w_mid = 16; o->w_coo = 4; o->w_inline = 1;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
-    o->inline_max = 4;
+    o->inline_max = 8;
 }
 
 int dbspmspv_create_csr(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz,

@@ -16,6 +16,7 @@ namespace dbs {
 // A "view" is three parallel arrays with one entry per nonempty block:
 //   idx[p]  bits 0..26  the block's index along the *other* dimension (column block in the
 //                       block-CSR view, row block in the block-CSC view)
+//           bit  28     block-CSR view only: first entry of a pull segment
 //           bits 29..31 block class (DBSPMSPV_BLK_*)
 //   w[p]    payload offset in 4-byte words -- or, for INLINE blocks, the data itself:
 //             valued matrices : the single value (fp32 bits, or bf16 bits in the low half)
@@ -47,11 +48,25 @@ struct View {
     uint8_t *aux;    // n_entries
 };
 
-struct Segment {     // pull work unit: a run of consecutive blocks inside one row block
+struct Segment {     // pull work unit: a run of consecutive view entries inside one row block
     int32_t row_block;
     int32_t start;   // first position in the block-CSR view
     int32_t count;   // bit 31: the segment covers its whole row block (plain stores allowed)
+    int32_t weight;  // accumulated cost weight (Section 3.3.2)
 };
+
+// Pull streams the block-CSR view through shared memory in chunks: chunk k owns the consecutive
+// segments whose exclusive weight prefix lies in [k * PULL_CH, (k+1) * PULL_CH).  Every entry
+// weighs at least 1 and a segment has at most MAX_SEG_ENTRIES entries, so a chunk spans fewer
+// than PULL_CH + MAX_SEG_ENTRIES entries, and equal weight per chunk balances the warps.
+constexpr int PULL_CH = 256;
+constexpr int MAX_SEG_ENTRIES = 128;
+constexpr int STAGE_CAP = PULL_CH + MAX_SEG_ENTRIES + 32;   // + alignment slack (16 each side)
+constexpr int VIEW_PAD = 64;                                // view arrays are over-allocated by this
+
+// Dense-x marker for "not listed": a NaN bit pattern that listed values never take (listed
+// NaNs are stored as the canonical quiet NaN), so one gather yields presence and value.
+constexpr uint32_t X_ABSENT = 0x7FFFFFFFu;
 
 struct Counters {    // device-resident scalars of one call
     int32_t n_nzblk;      // nonempty vector blocks
@@ -89,6 +104,9 @@ struct Device {           // everything the kernels need, passed by value
     View csr, csc;
     const uint8_t *payload;
     const Segment *segments;
+    const int32_t *seg_rb;  // row block of every segment (compact copy for the pull kernel)
+    const int2 *chunks;   // n_chunks + 1: {first segment, first entry} of every pull chunk
+    int32_t n_chunks;
     Workspace ws;
 };
 

@@ -4,6 +4,7 @@
 // decode entry (Section 4.3).  Nothing here allocates or synchronises.
 #include "internal.cuh"
 #include "microkernels.cuh"
+#include "staging.cuh"
 #include "worklist.cuh"
 
 namespace dbs {
@@ -38,7 +39,9 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
                 if (DT == DBSPMSPV_BF16) v = __bfloat162float(static_cast<const __nv_bfloat16 *>(x_val)[t]);
                 else v = static_cast<const float *>(x_val)[t];
             }
-            d.ws.x_dense[j] = v;
+            // a listed NaN that happens to carry the marker's bit pattern is stored as the
+            // canonical quiet NaN, so the marker itself never appears as data
+            d.ws.x_dense[j] = __float_as_uint(v) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v;
             const int sh = ((j >> 4) & 1) * 16;
             const uint32_t old = atomicOr(&d.ws.x_mask32[j >> 5], 1u << ((j & 15) + sh));
             newly = ((old >> sh) & 0xFFFFu) == 0;
@@ -59,7 +62,9 @@ __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__re
         float v = 0.f;
         if (j < d.n) v = DT == DBSPMSPV_BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(x)[j])
                                              : static_cast<const float *>(x)[j];
-        if (j < (int64_t)d.nb * 16) d.ws.x_dense[j] = v;
+        if (j < (int64_t)d.nb * 16)
+            d.ws.x_dense[j] = v != 0.0f ? (__float_as_uint(v) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v)
+                                        : __uint_as_float(X_ABSENT);
         const uint32_t bits = __ballot_sync(FULL, v != 0.0f);
         if (lane == 0) d.ws.x_mask32[j >> 5] = bits;
         const bool newly = (lane == 0 && (bits & 0xFFFFu)) || (lane == 16 && (bits >> 16));
@@ -138,9 +143,10 @@ __device__ __forceinline__ bool lane_owned(int type, uint32_t aux) {
 // entry per step and finds its owner block by a shuffle binary search over the scan.  This
 // keeps all lanes busy whatever the mix of block sizes (a lane looping over its own block
 // would make the whole warp wait for the largest block).  `cnt` is the lane's entry count
-// (0 = no COO block here), `tag` a per-block value handed back to `emit(tag, r, c, value, xm)`.
+// (0 = no COO block here); `tag0`, `tag1` are per-block values handed back to
+// `emit(tag0, tag1, r, c, value, owner_lane)` for every entry whose column is active.
 template <int DT, typename Emit>
-__device__ __forceinline__ void warp_flat_coo(int cnt, uint32_t w, uint32_t xm, uint32_t tag,
+__device__ __forceinline__ void warp_flat_coo(int cnt, uint32_t w, uint32_t xm, uint32_t tag0, uint32_t tag1,
                                               const uint8_t *payload, int lane, Emit emit) {
     int incl = cnt;
     for (int o = 1; o < 32; o <<= 1) {
@@ -160,12 +166,13 @@ __device__ __forceinline__ void warp_flat_coo(int cnt, uint32_t w, uint32_t xm, 
         const int k = e - (__shfl_sync(FULL, incl, o) - bn);
         const uint32_t bw = __shfl_sync(FULL, w, o);
         const uint32_t bxm = __shfl_sync(FULL, xm, o);
-        const uint32_t btag = __shfl_sync(FULL, tag, o);
+        const uint32_t bt0 = __shfl_sync(FULL, tag0, o);
+        const uint32_t bt1 = __shfl_sync(FULL, tag1, o);
         if (e < total) {
             const uint8_t *blk = payload + (size_t)bw * 4;
             const uint32_t rc = blk[k];
             const int c = rc & 15, r = rc >> 4;
-            if ((bxm >> c) & 1u) emit(btag, r, c, Val<DT>::load(blk + ((bn + 3) & ~3), k), o);
+            if ((bxm >> c) & 1u) emit(bt0, bt1, r, c, Val<DT>::load(blk + ((bn + 3) & ~3), k), o);
         }
     }
 }
@@ -213,8 +220,8 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
             s_tmp[lane] = 0.f;   // per-owner-lane hit masks (bit patterns), 32 slots
             __syncwarp();
             uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_tmp);
-            warp_flat_coo<DT>(coo_cnt, w, xm, (uint32_t)brow, d.payload, lane,
-                              [&](uint32_t tag, int r, int c, float a, int owner) {
+            warp_flat_coo<DT>(coo_cnt, w, xm, (uint32_t)brow, 0u, d.payload, lane,
+                              [&](uint32_t tag, uint32_t, int r, int c, float a, int owner) {
                                   if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)tag * 16 + r, a * s_x[c]);
                                   if (Out::MASKS) atomicOr(&s_hit[owner], 1u << r);
                               });
@@ -245,66 +252,175 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
     }
 }
 
-// Pull (Section 3.3.2): every warp takes one load-weighted segment of a row block and keeps
-// the 16 partial sums of that row block in shared memory; blocks whose vector block is empty
-// are skipped on their mask.  A segment that covers its whole row block writes with plain
-// stores; split row blocks fall back to atomics.  PULL_UNROLL x 32 view entries are fetched
-// per step, then their masks and (for INLINE blocks) x entries, so that each lane keeps
-// several independent loads in flight.
+// Pull (Section 3.3.2).  The block-CSR view is streamed through shared memory: every warp owns
+// a double-buffered stage (Section 3.3.3) that one lane fills with three bulk copies (index,
+// word and aux arrays of one chunk of consecutive segments) while the warp works on the other
+// stage.  Inside a chunk the lanes run over the entries 32 at a time, whatever segment they
+// belong to: the first entry of every segment carries a flag bit, so a ballot and a popcount
+// give each lane its segment, hence its row block.  Writeback is hierarchical where it pays:
+// the segment the warp is currently "in" accumulates its 16 partial sums in shared memory
+// (long hub row blocks stay there over many steps); products of the other, short segments met
+// in the same step go straight to global atomics.  INLINE entries need one gather only: the
+// dense copy of x carries a "not listed" marker, so presence and value come from one load.
+struct PullStage {
+    uint32_t idx[STAGE_CAP];
+    uint32_t w[STAGE_CAP];
+    uint8_t aux[STAGE_CAP];
+};
+struct PullWarp {
+    PullStage stage[2];
+    uint64_t bar[2];
+};
 constexpr int PULL_UNROLL = 4;
+constexpr uint32_t SEG_FLAG = 1u << 28;   // view entry starts a pull segment (block-CSR view only)
+
+// lane 0 issues the copies of the chunk [e0, e1) into stage st
+__device__ __forceinline__ void pull_issue(const Device &d, int e0, int e1, PullStage *st, uint64_t *bar, int lane) {
+    const int a0 = e0 & ~15, a1 = (e1 + 15) & ~15;
+    if (lane == 0 && a1 > a0) {
+        const uint32_t n = (uint32_t)(a1 - a0);
+        fence_proxy_async_smem();
+        mbar_arrive_expect_tx(bar, n * 9u);
+        bulk_copy_g2s(st->idx, d.csr.idx + a0, n * 4u, bar);
+        bulk_copy_g2s(st->w, d.csr.w + a0, n * 4u, bar);
+        bulk_copy_g2s(st->aux, d.csr.aux + a0, n, bar);
+    }
+}
+
+// Writeback of one block handled outside the shared-memory accumulator: one global atomic per
+// touched row plus one atomicOr on the row block's structural-hit mask.
+template <typename Out>
+__device__ __forceinline__ void flush_rows(Out out, int rb, uint32_t hits, float v, int lane) {
+    if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(out.acc + (size_t)rb * 16 + lane, v);
+    if (Out::MASKS && lane == 0 && hits) atomicOr(&out.mask32[rb >> 1], hits << ((rb & 1) * 16));
+}
 
 template <int DT, typename Out>
 __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp,
-                          float *s_y) {
+                          float *s_y, PullWarp *pw) {
     const int lane = threadIdx.x & 31;
+    const uint32_t le_mask = 0xFFFFFFFFu >> (31 - lane);
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
-    for (int sg = gwarp; sg < d.n_segments; sg += nwarps) {
-        const Segment seg = d.segments[sg];
-        const int rb = seg.row_block;
-        const bool whole = seg.count < 0;
-        const int end = seg.start + (seg.count & 0x7FFFFFFF);
-        if (lane < 16) s_y[lane] = 0.f;
-        __syncwarp();
+    if (lane == 0) { mbar_init(&pw->bar[0], 1); mbar_init(&pw->bar[1], 1); fence_barrier_init(); }
+    if (lane < 16) s_y[lane] = 0.f;
+    __syncwarp();
+    uint32_t parity = 0u;             // bit s: phase parity of stage s
+    int cur = 0;
+    bool next_in_flight = false;
+    int2 c0 = make_int2(0, 0), c1 = c0, n0 = c0, n1 = c0;
+    if (gwarp < d.n_chunks) {
+        c0 = d.chunks[gwarp]; c1 = d.chunks[gwarp + 1];
+        pull_issue(d, c0.y, c1.y, &pw->stage[0], &pw->bar[0], lane);
+    }
+    if (gwarp + nwarps < d.n_chunks) { n0 = d.chunks[gwarp + nwarps]; n1 = d.chunks[gwarp + nwarps + 1]; }
+    for (int c = gwarp; c < d.n_chunks; c += nwarps) {
+        const int e0 = c0.y, e1 = c1.y, a0 = e0 & ~15;
+        int ord_base = c0.x - 1;          // segment of the entry just before the current step
+        // prefetch: next chunk's copies, and the descriptor of the one after
+        const int cn = c + nwarps;
+        next_in_flight = cn < d.n_chunks;
+        if (next_in_flight) pull_issue(d, n0.y, n1.y, &pw->stage[cur ^ 1], &pw->bar[cur ^ 1], lane);
+        c0 = n0; c1 = n1;
+        if (cn + nwarps < d.n_chunks) { n0 = d.chunks[cn + nwarps]; n1 = d.chunks[cn + nwarps + 1]; }
+        if (e1 > e0) {
+            if (!mbar_wait_bounded(&pw->bar[cur], (parity >> cur) & 1u)) {
+                d.ws.ctr->status = DBSPMSPV_ERR_TIMEOUT;
+                break;
+            }
+            parity ^= 1u << cur;
+        }
+        const PullStage *st = &pw->stage[cur];
+        int cur_ord = -1, cur_rb = 0;     // segment held in the shared accumulator
         uint32_t hit = 0;
-        for (int base = seg.start; base < end; base += 32 * PULL_UNROLL) {
-            uint32_t idx[PULL_UNROLL], w[PULL_UNROLL], aux[PULL_UNROLL], xm[PULL_UNROLL];
+        for (int base = e0; base < e1; base += 32 * PULL_UNROLL) {
+            uint32_t idx[PULL_UNROLL], w[PULL_UNROLL], aux[PULL_UNROLL];
             float xin[PULL_UNROLL];
 #pragma unroll
             for (int u = 0; u < PULL_UNROLL; ++u) {
                 const int p = base + u * 32 + lane;
                 idx[u] = 0; w[u] = 0; aux[u] = 0;
-                if (p < end) { idx[u] = d.csr.idx[p]; w[u] = d.csr.w[p]; aux[u] = d.csr.aux[p]; }
+                if (p < e1) { const int o = p - a0; idx[u] = st->idx[o]; w[u] = st->w[o]; aux[u] = st->aux[o]; }
             }
 #pragma unroll
             for (int u = 0; u < PULL_UNROLL; ++u) {
-                const int bcol = idx[u] & IDX_MASK;
-                const bool have = base + u * 32 + lane < end;
-                xm[u] = have ? mask_of(d.ws.x_mask32, bcol) : 0u;
-                xin[u] = (have && DT != DBSPMSPV_PATTERN) ? d.ws.x_dense[(size_t)bcol * 16 + (aux[u] & 15)] : 0.f;
+                const bool have = base + u * 32 + lane < e1;
+                xin[u] = (have && DT != DBSPMSPV_PATTERN)
+                             ? d.ws.x_dense[(size_t)(idx[u] & IDX_MASK) * 16 + (aux[u] & 15)]
+                             : __uint_as_float(X_ABSENT);
             }
 #pragma unroll
             for (int u = 0; u < PULL_UNROLL; ++u) {
-                if (base + u * 32 >= end) break;   // warp-uniform
+                if (base + u * 32 >= e1) break;   // warp-uniform
+                const bool have = base + u * 32 + lane < e1;
+                const uint32_t fb = __ballot_sync(FULL, have && (idx[u] & SEG_FLAG));
+                const int ord = ord_base + __popc(fb & le_mask);
+                ord_base += __popc(fb);
+                const int rb = have ? d.seg_rb[ord] : 0;
+                // the shared accumulator follows the segment of the step's first entry
+                const int ord0 = __shfl_sync(FULL, ord, 0);
+                if (ord0 != cur_ord) {
+                    hit = __reduce_or_sync(FULL, hit);
+                    __syncwarp();
+                    if (lane < 16) {
+                        if (DT != DBSPMSPV_PATTERN && ((hit >> lane) & 1u)) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+                        s_y[lane] = 0.f;
+                    }
+                    if (Out::MASKS && lane == 0 && hit) atomicOr(&out.mask32[cur_rb >> 1], hit << ((cur_rb & 1) * 16));
+                    hit = 0;
+                    cur_ord = ord0;
+                    cur_rb = __shfl_sync(FULL, rb, 0);
+                    __syncwarp();
+                }
+                const int type = idx[u] >> TYPE_SHIFT;
+                bool other = false;
+                if (have) {
+                    if (type == DBSPMSPV_BLK_INLINE && DT != DBSPMSPV_PATTERN) {
+                        if (__float_as_uint(xin[u]) != X_ABSENT) {
+                            const float v = Val<DT>::inline_value(w[u]) * xin[u];
+                            const int r = aux[u] >> 4;
+                            if (ord == cur_ord) {
+                                atomicAdd(&s_y[r], v);
+                                hit |= 1u << r;
+                            } else {
+                                atomicAdd(out.acc + (size_t)rb * 16 + r, v);
+                                if (Out::MASKS) atomicOr(&out.mask32[rb >> 1], 1u << (r + (rb & 1) * 16));
+                            }
+                        }
+                    } else {
+                        other = true;
+                    }
+                }
+                if (!__any_sync(FULL, other)) continue;
+                // classes that go through the vector-block mask; they write straight to global
+                const int bcol_l = idx[u] & IDX_MASK;
+                const uint32_t xm = other ? mask_of(d.ws.x_mask32, bcol_l) : 0u;
                 bool heavy = false;
                 int coo_cnt = 0;
-                const int bcol_l = idx[u] & IDX_MASK;
-                if (xm[u]) {
-                    const int type = idx[u] >> TYPE_SHIFT;
-                    if (type == DBSPMSPV_BLK_INLINE)
-                        hit |= lane_block<DT>(type, w[u], aux[u], xm[u], xin[u], nullptr, d.payload,
-                                              [&](int r, float v) { atomicAdd(&s_y[r], v); });
-                    else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX)
+                if (xm) {
+                    if (type == DBSPMSPV_BLK_INLINE) {             // pattern: up to four coordinates
+                        const uint32_t hb = lane_block<DT>(type, w[u], aux[u], xm, 0.f, nullptr, d.payload, [](int, float) {});
+                        if (Out::MASKS && hb) atomicOr(&out.mask32[rb >> 1], hb << ((rb & 1) * 16));
+                    } else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
                         coo_cnt = (int)aux[u] + 1;
-                    else
+                    } else {
                         heavy = true;
+                    }
                 }
-                if (__any_sync(FULL, coo_cnt))
-                    warp_flat_coo<DT>(coo_cnt, w[u], xm[u], (uint32_t)bcol_l, d.payload, lane,
-                                      [&](uint32_t tag, int r, int c, float a, int) {
-                                          if (DT != DBSPMSPV_PATTERN) atomicAdd(&s_y[r], a * d.ws.x_dense[(size_t)tag * 16 + c]);
-                                          hit |= 1u << r;
+                if (__any_sync(FULL, coo_cnt)) {
+                    uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_tmp);   // per-owner-lane hit masks
+                    s_hit[lane] = 0u;
+                    __syncwarp();
+                    warp_flat_coo<DT>(coo_cnt, w[u], xm, (uint32_t)rb, (uint32_t)bcol_l, d.payload, lane,
+                                      [&](uint32_t trb, uint32_t tcol, int r, int c, float a, int owner) {
+                                          if (DT != DBSPMSPV_PATTERN)
+                                              atomicAdd(out.acc + (size_t)trb * 16 + r, a * d.ws.x_dense[(size_t)tcol * 16 + c]);
+                                          if (Out::MASKS) atomicOr(&s_hit[owner], 1u << r);
                                       });
+                    __syncwarp();
+                    if (Out::MASKS && coo_cnt && s_hit[lane]) atomicOr(&out.mask32[rb >> 1], s_hit[lane] << ((rb & 1) * 16));
+                    __syncwarp();
+                }
                 uint32_t hv = __ballot_sync(FULL, heavy);
                 while (hv) {
                     const int src = __ffs(hv) - 1;
@@ -312,36 +428,40 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                     const uint32_t bidx = __shfl_sync(FULL, idx[u], src);
                     const uint32_t bw = __shfl_sync(FULL, w[u], src);
                     const int nnz = (int)__shfl_sync(FULL, aux[u], src) + 1;
-                    const uint32_t bxm = __shfl_sync(FULL, xm[u], src);
-                    const int type = bidx >> TYPE_SHIFT;
+                    const uint32_t bxm = __shfl_sync(FULL, xm, src);
+                    const int brb = __shfl_sync(FULL, rb, src);
+                    const int btype = bidx >> TYPE_SHIFT;
                     const int bcol = bidx & IDX_MASK;
                     const uint8_t *blk = d.payload + (size_t)bw * 4;
                     uint32_t hits;
+                    float sum = 0.f;
                     if (DT == DBSPMSPV_PATTERN) {
-                        hits = warp_block_bool<DT>(type, blk, nnz, bxm, lane);
+                        hits = warp_block_bool<DT>(btype, blk, nnz, bxm, lane);
                     } else {
                         __syncwarp();
                         if (lane < 16) s_x[lane] = d.ws.x_dense[(size_t)bcol * 16 + lane];
                         __syncwarp();
-                        const float sum = warp_block<DT>(type, blk, nnz, bxm, s_x, s_tmp, lane, popc_threshold, hits);
-                        if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(&s_y[lane], sum);
+                        sum = warp_block<DT>(btype, blk, nnz, bxm, s_x, s_tmp, lane, popc_threshold, hits);
                     }
-                    hit |= hits;
+                    flush_rows(out, brb, hits, sum, lane);
                 }
             }
         }
+        // end of the chunk: flush what the shared accumulator still holds
         hit = __reduce_or_sync(FULL, hit);
         __syncwarp();
-        if (DT != DBSPMSPV_PATTERN && lane < 16 && ((hit >> lane) & 1u)) {
-            float *dst = out.acc + (size_t)rb * 16 + lane;
-            if (whole) *dst = s_y[lane]; else atomicAdd(dst, s_y[lane]);
+        if (lane < 16) {
+            if (DT != DBSPMSPV_PATTERN && ((hit >> lane) & 1u)) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+            s_y[lane] = 0.f;
         }
-        if (Out::MASKS && lane == 0 && hit) {
-            if (whole) reinterpret_cast<uint16_t *>(out.mask32)[rb] = (uint16_t)hit;
-            else atomicOr(&out.mask32[rb >> 1], hit << ((rb & 1) * 16));
-        }
+        if (Out::MASKS && lane == 0 && hit) atomicOr(&out.mask32[cur_rb >> 1], hit << ((cur_rb & 1) * 16));
         __syncwarp();
+        cur ^= 1;
+        next_in_flight = false;
     }
+    // left early on a timeout: let the copy still in flight land before the stage memory is
+    // given back (bounded, like every wait here)
+    if (next_in_flight) mbar_wait_bounded(&pw->bar[cur ^ 1], (parity >> (cur ^ 1)) & 1u);
 }
 
 // Global selector (Section 3.3.1): s_b = N_nzblk / N_blk; push iff s_b < th3.  Evaluated on
@@ -355,11 +475,12 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
 template <int DT, typename Out>
 __global__ void __launch_bounds__(CTA) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
     __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16];
+    __shared__ __align__(128) PullWarp s_pull[WARPS];
     const int warp = threadIdx.x >> 5;
     const int path = select_path(d, th3, force_path);
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
     if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp]);
-    else pull_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp]);
+    else pull_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], &s_pull[warp]);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -457,7 +578,7 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
     const int stride = gridDim.x * CMP_TPB;
     for (int k = blockIdx.x * CMP_TPB + threadIdx.x; k < nnz_x; k += stride) {
         const int j = x_idx[k];
-        if (j >= 0 && j < d.n) d.ws.x_mask32[j >> 5] = 0u;
+        if (j >= 0 && j < d.n) { d.ws.x_mask32[j >> 5] = 0u; d.ws.x_dense[j] = __uint_as_float(X_ABSENT); }
     }
 }
 
@@ -465,6 +586,8 @@ __global__ void k_decode_cleanup(Device d) {
     const int n_words = (d.nb + 1) / 2;
     const int stride = gridDim.x * blockDim.x;
     for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n_words; k += stride) d.ws.x_mask32[k] = 0u;
+    for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < (int64_t)d.nb * 16; j += stride)
+        d.ws.x_dense[j] = __uint_as_float(X_ABSENT);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         Counters *c = d.ws.ctr;
         c->last_n_nzblk = c->n_nzblk;
@@ -474,6 +597,10 @@ __global__ void k_decode_cleanup(Device d) {
         c->n_nzblk = 0;
         c->n_tasks = 0;
     }
+}
+
+__global__ void k_fill_u32(uint32_t *p, int64_t n, uint32_t v) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = v;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -514,6 +641,12 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     DBS_WS(dev_alloc_zero(&ws.ctr, 1, &total));
 #undef DBS_WS
     h->stats.workspace_bytes = total;
+    if (cudaMemset(ws.x_dense, 0xFF, xwords * 32 * sizeof(float)) != cudaSuccess) return DBSPMSPV_ERR_CUDA;
+    {   // 0xFFFFFFFF -> the marker pattern 0x7FFFFFFF needs a kernel; a tiny fill does it
+        uint32_t *p = reinterpret_cast<uint32_t *>(ws.x_dense);
+        k_fill_u32<<<256, 256>>>(p, (int64_t)xwords * 32, X_ABSENT);
+        if (cudaDeviceSynchronize() != cudaSuccess) return DBSPMSPV_ERR_CUDA;
+    }
     // events for the optional kernel timing are made here so that run-time calls create nothing
     if (cudaEventCreate(&h->ev[0]) != cudaSuccess || cudaEventCreate(&h->ev[1]) != cudaSuccess) return DBSPMSPV_ERR_CUDA;
     return DBSPMSPV_OK;

@@ -20,7 +20,7 @@ def cpu_classify(rows, cols, dtype, th0=32, th1=128, th2=2.0):
     key, rows, cols = key[order], rows[order], cols[order]
     ub, start, cnt = np.unique(key, return_index=True, return_counts=True)
     cls = np.empty(ub.size, dtype=np.int32)
-    cap = 4          # default inline_max; pattern entries hold up to four coordinates
+    cap = 4 if dtype == B.PATTERN else 8   # pattern: four coordinates per entry; valued: inline_max
     for b in range(ub.size):
         n = cnt[b]
         if n < th0:
@@ -148,8 +148,8 @@ def test_threshold_edges():
     assert cls_of(full[:128]) != B.BLK_DENSE
     assert cls_of(full[:129]) == B.BLK_DENSE
     assert cls_of(full[:1]) == B.BLK_INLINE
-    assert cls_of(full[:4]) == B.BLK_INLINE
-    assert cls_of(full[:5]) == B.BLK_COO
+    assert cls_of(full[:8]) == B.BLK_INLINE
+    assert cls_of(full[:9]) == B.BLK_COO
     # 32 entries as two full rows: max row 16, max col 2 -> ForceCSR
     assert cls_of(full[:32]) == B.BLK_FCSR
     assert cls_of([(c, r) for r, c in full[:32]]) == B.BLK_FCSC
