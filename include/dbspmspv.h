@@ -45,7 +45,8 @@ typedef enum {
     DBSPMSPV_ERR_CUDA = 4,        /* a CUDA runtime call failed                           */
     DBSPMSPV_ERR_CAPACITY = 5,    /* y_capacity too small; nothing was written out of bounds */
     DBSPMSPV_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out                   */
-    DBSPMSPV_ERR_BOUNDS = 7       /* validate=1: an x index was out of range              */
+    DBSPMSPV_ERR_BOUNDS = 7,      /* validate=1: an x index was out of range              */
+    DBSPMSPV_ERR_TOO_LARGE = 8    /* dbspmspv_compact_noalloc: more rows than its fixed scratch covers */
 } dbspmspv_status_t;
 
 typedef enum {
@@ -225,6 +226,36 @@ int dbspmspv_export_blocks(dbspmspv_handle_t h, int32_t *block_row, int32_t *blo
  * NULL.                                                                                      */
 int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *csc_col_ptr,
                           int32_t *csc_row, int32_t *csc2csr);
+
+/*
+ * Output compaction without any allocation.  (The paper has no counterpart: it returns a dense
+ * y.  This entry point exists for callers that may not allocate device memory at the point of
+ * the call -- real-time loops that must stay out of the allocator, hosts that own the whole
+ * device heap, phases of a larger program with a frozen memory budget -- and that already hold
+ * a dense result plus a row-hit bitmap, for instance from their own kernels.)
+ *
+ *   acc         m fp32 values (device); only rows whose bit is set are read
+ *   hit_bitmap  ceil(m/32) uint32 words (device): bit (i & 31) of word (i >> 5) set iff row i
+ *               belongs to the result; bits at or beyond m must be clear
+ *   y_idx/y_val out: the set rows in ascending order and their values, room for y_capacity
+ *               entries (y_val may be NULL); y_nnz out: one int32 on the device, the full count
+ *   Inputs are not modified.  Handles are not involved.
+ *
+ * Scratch: one counter per 8192 rows, kept in a fixed 16 KB __device__ array inside the
+ * library (every GPU that loads the library holds it until the process exits).  Hence
+ *   - m may be at most 33,554,432 rows; larger m returns DBSPMSPV_ERR_TOO_LARGE and does nothing;
+ *   - the array is shared by every call and keeps the previous call's contents; each call
+ *     overwrites every counter it will read before reading it, so nothing has to be cleared;
+ *   - two calls whose kernels overlap on the GPU (different streams, or threads) race on it:
+ *     serialise calls to this entry point on one device;
+ *   - the first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress); make that first call before any stream capture begins.
+ * It calls no cudaMalloc / cudaFree or other allocating routine, enqueues two kernels on
+ * `stream` and returns without synchronising.
+ */
+int dbspmspv_compact_noalloc(const float *acc, const uint32_t *hit_bitmap, int64_t m,
+                             int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
+                             dbspmspv_stream_t stream);
 
 int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts);
 int dbspmspv_destroy(dbspmspv_handle_t h);

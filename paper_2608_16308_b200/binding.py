@@ -14,7 +14,7 @@ from typing import Optional
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libdbspmspv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_CAPACITY, ERR_TIMEOUT, ERR_BOUNDS = range(8)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_CAPACITY, ERR_TIMEOUT, ERR_BOUNDS, ERR_TOO_LARGE = range(9)
 F32, BF16, PATTERN = 0, 1, 2
 PLUS_TIMES, OR_AND = 0, 1
 PATH_AUTO, PATH_PUSH, PATH_PULL = 0, 1, 2
@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "dbspmspv_default_create_opts", "dbspmspv_default_run_opts", "dbspmspv_create_csr",
     "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "dbspmspv_decode", "dbspmspv_get_stats",
     "dbspmspv_export_coo", "dbspmspv_export_blocks", "dbspmspv_export_views",
-    "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror",
+    "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror", "dbspmspv_compact_noalloc",
 )
 
 
@@ -89,6 +89,7 @@ def lib() -> ctypes.CDLL:
         L.dbspmspv_export_coo.argtypes = [vp, vp, vp, vp]
         L.dbspmspv_export_blocks.argtypes = [vp, vp, vp, vp, vp]
         L.dbspmspv_export_views.argtypes = [vp, vp, vp, vp, vp]
+        L.dbspmspv_compact_noalloc.argtypes = [vp, vp, i64, vp, vp, i64, vp, vp]
         L.dbspmspv_set_run_opts.argtypes = [vp, ctypes.POINTER(RunOpts)]
         L.dbspmspv_destroy.argtypes = [vp]
         L.dbspmspv_strerror.argtypes = [ctypes.c_int]
@@ -195,6 +196,16 @@ def dbspmspv_export_blocks(h, block_row, block_col, block_class, block_nnz) -> N
 def dbspmspv_export_views(h, csr_row_ptr, csc_col_ptr, csc_row, csc2csr) -> None:
     _check(lib().dbspmspv_export_views(h, _ptr(csr_row_ptr), _ptr(csc_col_ptr), _ptr(csc_row),
                                        _ptr(csc2csr)), "dbspmspv_export_views")
+
+
+def dbspmspv_compact_noalloc(acc, hit_bitmap, m, y_idx, y_val, y_capacity, y_nnz,
+                             stream: Optional[int] = None) -> None:
+    """Marshals to dbspmspv_compact_noalloc: compaction of (dense values, row-hit bitmap) into a
+    sorted sparse vector for callers that may not allocate device memory (the library keeps the
+    16 KB of scratch it needs in a fixed device array; at most 33,554,432 rows per call)."""
+    _check(lib().dbspmspv_compact_noalloc(_ptr(acc), _ptr(hit_bitmap), m, _ptr(y_idx), _ptr(y_val),
+                                          y_capacity, _ptr(y_nnz), _stream() if stream is None else stream),
+           "dbspmspv_compact_noalloc")
 
 
 def dbspmspv_set_run_opts(h, opts: RunOpts) -> None:

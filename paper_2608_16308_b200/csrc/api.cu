@@ -213,6 +213,7 @@ const char *dbspmspv_strerror(int status) {
         case DBSPMSPV_ERR_CAPACITY: return "output capacity too small";
         case DBSPMSPV_ERR_TIMEOUT: return "bounded device wait ran out";
         case DBSPMSPV_ERR_BOUNDS: return "x index out of range";
+        case DBSPMSPV_ERR_TOO_LARGE: return "more rows than the fixed scratch of the no-allocation entry point covers";
         default: return "unknown status";
     }
 }
