@@ -58,43 +58,46 @@ __device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int dept
     for (int t = gwarp; t < n_tasks; t += nwarps) {
         const uint2 task = d.ws.tasks[t];
         const int jb = (int)(task.x & IDX_MASK);
-        const int cnt = (int)(task.x >> 27) + 1;
+        const int start = (int)task.y;
+        const int end = min(start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
         const uint32_t xm = mask_of(d.ws.x_mask32, jb);
-        const int p = (int)task.y + lane;
-        bool heavy = false;
-        uint32_t idx = 0, w = 0, aux = 0;
-        if (lane < cnt) {
-            idx = d.csc.idx[p];
-            const int type = idx >> TYPE_SHIFT, brow = idx & IDX_MASK;
-            const uint32_t need = ~mask_of(d.ws.visited32, brow) & 0xFFFFu;
-            if (need) {
-                w = d.csc.w[p]; aux = d.csc.aux[p];
-                if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX)) {
-                    const uint32_t hit = lane_block_bool<DT>(type, w, aux, xm, d.payload) & need;
-                    if (hit) {
-                        const int sh = (brow & 1) * 16;
-                        const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hit << sh);
-                        write_levels(levels, brow, hit & ~(old >> sh), depth);
+        for (int base = start; base < end; base += 32) {
+            const int p = base + lane;
+            bool heavy = false;
+            uint32_t idx = 0, w = 0, aux = 0;
+            if (p < end) {
+                idx = d.csc.idx[p];
+                const int type = idx >> TYPE_SHIFT, brow = idx & IDX_MASK;
+                const uint32_t need = ~mask_of(d.ws.visited32, brow) & 0xFFFFu;
+                if (need) {
+                    w = d.csc.w[p]; aux = d.csc.aux[p];
+                    if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX)) {
+                        const uint32_t hit = lane_block_bool<DT>(type, w, aux, xm, d.payload) & need;
+                        if (hit) {
+                            const int sh = (brow & 1) * 16;
+                            const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hit << sh);
+                            write_levels(levels, brow, hit & ~(old >> sh), depth);
+                        }
+                    } else {
+                        heavy = true;
                     }
-                } else {
-                    heavy = true;
                 }
             }
-        }
-        uint32_t hv = __ballot_sync(FULL, heavy);
-        while (hv) {
-            const int src = __ffs(hv) - 1;
-            hv &= hv - 1;
-            const uint32_t bidx = __shfl_sync(FULL, idx, src);
-            const uint32_t bw = __shfl_sync(FULL, w, src);
-            const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
-            const int type = bidx >> TYPE_SHIFT, brow = bidx & IDX_MASK;
-            uint32_t hits = warp_block_bool<DT>(type, d.payload + (size_t)bw * 4, nnz, xm, lane);
-            hits &= ~mask_of(d.ws.visited32, brow);
-            if (lane == 0 && hits) {
-                const int sh = (brow & 1) * 16;
-                const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hits << sh);
-                write_levels(levels, brow, hits & ~(old >> sh), depth);
+            uint32_t hv = __ballot_sync(FULL, heavy);
+            while (hv) {
+                const int src = __ffs(hv) - 1;
+                hv &= hv - 1;
+                const uint32_t bidx = __shfl_sync(FULL, idx, src);
+                const uint32_t bw = __shfl_sync(FULL, w, src);
+                const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
+                const int type = bidx >> TYPE_SHIFT, brow = bidx & IDX_MASK;
+                uint32_t hits = warp_block_bool<DT>(type, d.payload + (size_t)bw * 4, nnz, xm, lane);
+                hits &= ~mask_of(d.ws.visited32, brow);
+                if (lane == 0 && hits) {
+                    const int sh = (brow & 1) * 16;
+                    const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hits << sh);
+                    write_levels(levels, brow, hits & ~(old >> sh), depth);
+                }
             }
         }
     }

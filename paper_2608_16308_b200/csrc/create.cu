@@ -552,7 +552,8 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     }
     DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_entries + VIEW_PAD); DBS_KEEP(d.csr.w, n_entries + VIEW_PAD); DBS_KEEP(d.csr.aux, n_entries + VIEW_PAD);
     DBS_CUDA(cudaMemsetAsync(d.csr.idx + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.aux + n_entries, 0, VIEW_PAD, st));
-    DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_entries); DBS_KEEP(d.csc.w, n_entries); DBS_KEEP(d.csc.aux, n_entries);
+    DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_entries + VIEW_PAD); DBS_KEEP(d.csc.w, n_entries + VIEW_PAD); DBS_KEEP(d.csc.aux, n_entries + VIEW_PAD);
+    DBS_CUDA(cudaMemsetAsync(d.csc.idx + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csc.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csc.aux + n_entries, 0, VIEW_PAD, st));
     DBS_KEEP(h->csc2csr, n_entries);
     DBS_KEEP(h->block_row, n_entries);
     if (n_blocks) {

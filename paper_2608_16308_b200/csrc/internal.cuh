@@ -38,7 +38,10 @@ namespace dbs {
 constexpr int B = 16;                       // block edge
 constexpr uint32_t IDX_MASK = 0x07FFFFFFu;  // 27 bits
 constexpr int TYPE_SHIFT = 29;
-constexpr int PUSH_CHUNK = 32;              // CSC-view entries per push task (one per lane)
+#ifndef DBS_PUSH_CHUNK
+#define DBS_PUSH_CHUNK 32
+#endif
+constexpr int PUSH_CHUNK = DBS_PUSH_CHUNK;   // CSC-view entries per push task (32 per warp step)
 constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-class block
 
 struct View {
@@ -59,7 +62,10 @@ struct Segment {     // pull work unit: a run of consecutive view entries inside
 // segments whose exclusive weight prefix lies in [k * PULL_CH, (k+1) * PULL_CH).  Every entry
 // weighs at least 1 and a segment has at most MAX_SEG_ENTRIES entries, so a chunk spans fewer
 // than PULL_CH + MAX_SEG_ENTRIES entries, and equal weight per chunk balances the warps.
-constexpr int PULL_CH = 256;
+#ifndef DBS_PULL_CH
+#define DBS_PULL_CH 256
+#endif
+constexpr int PULL_CH = DBS_PULL_CH;
 constexpr int MAX_SEG_ENTRIES = 128;
 constexpr int STAGE_CAP = PULL_CH + MAX_SEG_ENTRIES + 32;   // + alignment slack (16 each side)
 constexpr int VIEW_PAD = 64;                                // view arrays are over-allocated by this
@@ -85,9 +91,10 @@ struct Counters {    // device-resident scalars of one call
 struct Workspace {
     float *x_dense;       // n (padded to a multiple of 32): dense copy of x (Section 3.2.2)
     uint32_t *x_mask32;   // vector-block masks, two 16-bit masks per word
-    uint2 *tasks;         // push worklist: (column block | (entries-1) << 27, first CSC-view position)
+    uint2 *tasks;         // push worklist: (column block | (ceil(entries/4)-1) << 27, first CSC-view position)
     float *y_acc;         // m (padded): dense accumulator, all zero between calls
-    uint32_t *y_mask32;   // structural-hit masks per row block, two per word, zero between calls
+    uint32_t *y_mask32;   // run: hit masks packed by the compaction pass; BFS: next-frontier masks
+    uint8_t *y_hit8;      // run: one structural-hit flag byte per row, all zero between calls
     int32_t *tile_count;  // compaction: result entries per tile of row blocks
     uint32_t *visited32;  // BFS: visited masks
     Counters *ctr;
@@ -140,6 +147,14 @@ namespace dbs {
 
 template <typename T>
 __host__ __device__ inline T ceil_div(T a, T b) { return (a + b - 1) / b; }
+
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start while its predecessor drains; `pdl_wait` blocks until the predecessor has completed and
+// its writes are visible (a no-op for a normally launched kernel), `pdl_launch_dependents`
+// lets the successor's launch proceed early.  This hides the launch latency between the short
+// kernels of one call.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t mask_of(const uint32_t *mask32, int blk) {
     return (mask32[blk >> 1] >> ((blk & 1) * 16)) & 0xFFFFu;

@@ -25,6 +25,7 @@ constexpr int TILE_WORDS = CMP_TPB;  // one 32-bit mask word (two row blocks) pe
 template <int DT>
 __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, const void *__restrict__ x_val,
                                 int32_t nnz_x, int validate) {
+    pdl_launch_dependents();
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = threadIdx.x & 31;
     bool newly = false;
@@ -79,12 +80,12 @@ __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__re
 // ------------------------------------------------------------------------------------------
 struct OutSparse {
     float *acc;
-    uint32_t *mask32;
+    uint8_t *hit8;     // one byte per row: 1 = structurally hit (plain idempotent stores, no atomics)
     static constexpr bool MASKS = true;
 };
 struct OutDense {
     float *acc;
-    uint32_t *mask32;
+    uint8_t *hit8;
     static constexpr bool MASKS = false;
 };
 
@@ -177,14 +178,36 @@ __device__ __forceinline__ void warp_flat_coo(int cnt, uint32_t w, uint32_t xm, 
     }
 }
 
-// Push (Section 3.3.2): every warp takes one task = up to 32 consecutive block-CSC entries of
-// one active column block; the vector block is staged once per task (Section 3.3.3).  Lanes
+// Structural-hit marking: one byte per output row, set with a plain store.  Stores of the same
+// value to the same byte need no atomic and no read, so hub rows that are hit by thousands of
+// products per call cost nothing extra; the compaction pass packs the bytes into masks.
+__device__ __forceinline__ void mark_rows(uint8_t *hit8, int rb, uint32_t rows16) {
+    uint8_t *base = hit8 + (size_t)rb * 16;
+    while (rows16) {
+        base[__ffs(rows16) - 1] = 1;
+        rows16 &= rows16 - 1;
+    }
+}
+
+// Writeback of one block handled outside the shared-memory accumulator: lanes 0..15 own the 16
+// rows; one global atomic and one flag store per touched row.
+template <typename Out>
+__device__ __forceinline__ void flush_rows(Out out, int rb, uint32_t hits, float v, int lane) {
+    if (lane < 16 && ((hits >> lane) & 1u)) {
+        atomicAdd(out.acc + (size_t)rb * 16 + lane, v);
+        if (Out::MASKS) out.hit8[(size_t)rb * 16 + lane] = 1;
+    }
+}
+
+// Push (Section 3.3.2): every warp takes one task = up to PUSH_CHUNK consecutive block-CSC
+// entries of one active column block (32 per step, all fetched up front); the vector block is staged once per task (Section 3.3.3).  Lanes
 // own hypersparse blocks; heavier blocks are then processed by the whole warp one at a time.
 // Writeback: warp-level reduction, then one global atomic per touched row and one atomicOr on
 // the row block's hit mask.  The task record carries its length, so the view entries, the mask
 // and the x block are all fetched in one round of independent loads.
 template <int DT, typename Out>
 __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp) {
+    constexpr int U = PUSH_CHUNK / 32;
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -192,61 +215,68 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
     for (int t = gwarp; t < n_tasks; t += nwarps) {
         const uint2 task = d.ws.tasks[t];
         const int jb = (int)(task.x & IDX_MASK);
-        const int cnt = (int)(task.x >> 27) + 1;
-        const int p = (int)task.y + lane;
-        const bool have = lane < cnt;
-        uint32_t idx = 0, w = 0, aux = 0;
-        if (have) { idx = d.csc.idx[p]; w = d.csc.w[p]; aux = d.csc.aux[p]; }
+        const int upper = ((int)(task.x >> 27) + 1) * 4;      // entries of the task, rounded up to 4
+        const int start = (int)task.y;
+        // one round of independent loads: view entries, exact end, mask, x block
+        uint32_t idx[U], w[U], aux[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            idx[u] = 0; w[u] = 0; aux[u] = 0;
+            if (u * 32 + lane < upper) { const int p = start + u * 32 + lane; idx[u] = d.csc.idx[p]; w[u] = d.csc.w[p]; aux[u] = d.csc.aux[p]; }
+        }
+        const int end = min(start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
         const uint32_t xm = mask_of(d.ws.x_mask32, jb);
         if (lane < 16) s_x[lane] = d.ws.x_dense[jb * 16 + lane];
         __syncwarp();
-        bool heavy = false;
-        int coo_cnt = 0;
-        const int type = idx >> TYPE_SHIFT;
-        const int brow = idx & IDX_MASK;
-        if (have) {
-            if (type == DBSPMSPV_BLK_INLINE) {
-                float *row0 = out.acc + (size_t)brow * 16;
-                const uint32_t hit = lane_block<DT>(type, w, aux, xm, s_x[aux & 15], s_x, d.payload,
-                                                    [&](int r, float v) { atomicAdd(row0 + r, v); });
-                if (Out::MASKS && hit) atomicOr(&out.mask32[brow >> 1], hit << ((brow & 1) * 16));
-            } else if (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX) {
-                coo_cnt = (int)aux + 1;
-            } else {
-                heavy = true;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (start + u * 32 >= end) break;                 // warp-uniform
+            const bool have = start + u * 32 + lane < end;
+            bool heavy = false;
+            int coo_cnt = 0;
+            const int type = idx[u] >> TYPE_SHIFT;
+            const int brow = idx[u] & IDX_MASK;
+            if (have) {
+                if (type == DBSPMSPV_BLK_INLINE) {
+                    float *row0 = out.acc + (size_t)brow * 16;
+                    const uint32_t hit = lane_block<DT>(type, w[u], aux[u], xm, s_x[aux[u] & 15], s_x, d.payload,
+                                                        [&](int r, float v) { atomicAdd(row0 + r, v); });
+                    if (Out::MASKS && hit) mark_rows(out.hit8, brow, hit);
+                } else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
+                    coo_cnt = (int)aux[u] + 1;
+                } else {
+                    heavy = true;
+                }
             }
-        }
-        if (__any_sync(FULL, coo_cnt)) {
-            s_tmp[lane] = 0.f;   // per-owner-lane hit masks (bit patterns), 32 slots
-            __syncwarp();
-            uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_tmp);
-            warp_flat_coo<DT>(coo_cnt, w, xm, (uint32_t)brow, 0u, d.payload, lane,
-                              [&](uint32_t tag, uint32_t, int r, int c, float a, int owner) {
-                                  if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)tag * 16 + r, a * s_x[c]);
-                                  if (Out::MASKS) atomicOr(&s_hit[owner], 1u << r);
-                              });
-            __syncwarp();
-            if (Out::MASKS && coo_cnt && s_hit[lane]) atomicOr(&out.mask32[brow >> 1], s_hit[lane] << ((brow & 1) * 16));
-            __syncwarp();
-        }
-        uint32_t hv = __ballot_sync(FULL, heavy);
-        while (hv) {
-            const int src = __ffs(hv) - 1;
-            hv &= hv - 1;
-            const uint32_t bidx = __shfl_sync(FULL, idx, src);
-            const uint32_t bw = __shfl_sync(FULL, w, src);
-            const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
-            const int btype = bidx >> TYPE_SHIFT;
-            const int bbrow = bidx & IDX_MASK;
-            const uint8_t *blk = d.payload + (size_t)bw * 4;
-            uint32_t hits;
-            if (DT == DBSPMSPV_PATTERN) {
-                hits = warp_block_bool<DT>(btype, blk, nnz, xm, lane);
-            } else {
-                const float sum = warp_block<DT>(btype, blk, nnz, xm, s_x, s_tmp, lane, popc_threshold, hits);
-                if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(out.acc + (size_t)bbrow * 16 + lane, sum);
+            if (__any_sync(FULL, coo_cnt)) {
+                uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_tmp);   // per-owner-lane hit masks
+                s_hit[lane] = 0u;
+                __syncwarp();
+                warp_flat_coo<DT>(coo_cnt, w[u], xm, (uint32_t)brow, 0u, d.payload, lane,
+                                  [&](uint32_t tag, uint32_t, int r, int c, float a, int owner) {
+                                      if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)tag * 16 + r, a * s_x[c]);
+                                      if (Out::MASKS) atomicOr(&s_hit[owner], 1u << r);
+                                  });
+                __syncwarp();
+                if (Out::MASKS && coo_cnt && s_hit[lane]) mark_rows(out.hit8, brow, s_hit[lane]);
+                __syncwarp();
             }
-            if (Out::MASKS && lane == 0 && hits) atomicOr(&out.mask32[bbrow >> 1], hits << ((bbrow & 1) * 16));
+            uint32_t hv = __ballot_sync(FULL, heavy);
+            while (hv) {
+                const int src = __ffs(hv) - 1;
+                hv &= hv - 1;
+                const uint32_t bidx = __shfl_sync(FULL, idx[u], src);
+                const uint32_t bw = __shfl_sync(FULL, w[u], src);
+                const int nnz = (int)__shfl_sync(FULL, aux[u], src) + 1;
+                const int btype = bidx >> TYPE_SHIFT;
+                const int bbrow = bidx & IDX_MASK;
+                const uint8_t *blk = d.payload + (size_t)bw * 4;
+                uint32_t hits;
+                float sum = 0.f;
+                if (DT == DBSPMSPV_PATTERN) hits = warp_block_bool<DT>(btype, blk, nnz, xm, lane);
+                else sum = warp_block<DT>(btype, blk, nnz, xm, s_x, s_tmp, lane, popc_threshold, hits);
+                flush_rows(out, bbrow, hits, sum, lane);
+            }
         }
         __syncwarp();
     }
@@ -271,13 +301,16 @@ struct PullWarp {
     PullStage stage[2];
     uint64_t bar[2];
 };
-constexpr int PULL_UNROLL = 4;
+#ifndef DBS_PULL_UNROLL
+#define DBS_PULL_UNROLL 2
+#endif
+constexpr int PULL_UNROLL = DBS_PULL_UNROLL;
 constexpr uint32_t SEG_FLAG = 1u << 28;   // view entry starts a pull segment (block-CSR view only)
 
 // lane 0 issues the copies of the chunk [e0, e1) into stage st
 __device__ __forceinline__ void pull_issue(const Device &d, int e0, int e1, PullStage *st, uint64_t *bar, int lane) {
     const int a0 = e0 & ~15, a1 = (e1 + 15) & ~15;
-    if (lane == 0 && a1 > a0) {
+    if (lane == 0 && e1 > e0) {      // same condition as the consumer's wait
         const uint32_t n = (uint32_t)(a1 - a0);
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(bar, n * 9u);
@@ -285,14 +318,6 @@ __device__ __forceinline__ void pull_issue(const Device &d, int e0, int e1, Pull
         bulk_copy_g2s(st->w, d.csr.w + a0, n * 4u, bar);
         bulk_copy_g2s(st->aux, d.csr.aux + a0, n, bar);
     }
-}
-
-// Writeback of one block handled outside the shared-memory accumulator: one global atomic per
-// touched row plus one atomicOr on the row block's structural-hit mask.
-template <typename Out>
-__device__ __forceinline__ void flush_rows(Out out, int rb, uint32_t hits, float v, int lane) {
-    if (lane < 16 && ((hits >> lane) & 1u)) atomicAdd(out.acc + (size_t)rb * 16 + lane, v);
-    if (Out::MASKS && lane == 0 && hits) atomicOr(&out.mask32[rb >> 1], hits << ((rb & 1) * 16));
 }
 
 template <int DT, typename Out>
@@ -363,10 +388,12 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                     hit = __reduce_or_sync(FULL, hit);
                     __syncwarp();
                     if (lane < 16) {
-                        if (DT != DBSPMSPV_PATTERN && ((hit >> lane) & 1u)) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+                        if ((hit >> lane) & 1u) {
+                            if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+                            if (Out::MASKS) out.hit8[(size_t)cur_rb * 16 + lane] = 1;
+                        }
                         s_y[lane] = 0.f;
                     }
-                    if (Out::MASKS && lane == 0 && hit) atomicOr(&out.mask32[cur_rb >> 1], hit << ((cur_rb & 1) * 16));
                     hit = 0;
                     cur_ord = ord0;
                     cur_rb = __shfl_sync(FULL, rb, 0);
@@ -384,7 +411,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                                 hit |= 1u << r;
                             } else {
                                 atomicAdd(out.acc + (size_t)rb * 16 + r, v);
-                                if (Out::MASKS) atomicOr(&out.mask32[rb >> 1], 1u << (r + (rb & 1) * 16));
+                                if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
                             }
                         }
                     } else {
@@ -400,7 +427,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                 if (xm) {
                     if (type == DBSPMSPV_BLK_INLINE) {             // pattern: up to four coordinates
                         const uint32_t hb = lane_block<DT>(type, w[u], aux[u], xm, 0.f, nullptr, d.payload, [](int, float) {});
-                        if (Out::MASKS && hb) atomicOr(&out.mask32[rb >> 1], hb << ((rb & 1) * 16));
+                        if (Out::MASKS && hb) mark_rows(out.hit8, rb, hb);
                     } else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
                         coo_cnt = (int)aux[u] + 1;
                     } else {
@@ -418,7 +445,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                                           if (Out::MASKS) atomicOr(&s_hit[owner], 1u << r);
                                       });
                     __syncwarp();
-                    if (Out::MASKS && coo_cnt && s_hit[lane]) atomicOr(&out.mask32[rb >> 1], s_hit[lane] << ((rb & 1) * 16));
+                    if (Out::MASKS && coo_cnt && s_hit[lane]) mark_rows(out.hit8, rb, s_hit[lane]);
                     __syncwarp();
                 }
                 uint32_t hv = __ballot_sync(FULL, heavy);
@@ -451,10 +478,12 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
         hit = __reduce_or_sync(FULL, hit);
         __syncwarp();
         if (lane < 16) {
-            if (DT != DBSPMSPV_PATTERN && ((hit >> lane) & 1u)) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+            if ((hit >> lane) & 1u) {
+                if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+                if (Out::MASKS) out.hit8[(size_t)cur_rb * 16 + lane] = 1;
+            }
             s_y[lane] = 0.f;
         }
-        if (Out::MASKS && lane == 0 && hit) atomicOr(&out.mask32[cur_rb >> 1], hit << ((cur_rb & 1) * 16));
         __syncwarp();
         cur ^= 1;
         next_in_flight = false;
@@ -472,11 +501,16 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
     return sb < th3 ? DBSPMSPV_PATH_PUSH : DBSPMSPV_PATH_PULL;
 }
 
+#ifndef DBS_MIN_CTAS
+#define DBS_MIN_CTAS 1
+#endif
 template <int DT, typename Out>
-__global__ void __launch_bounds__(CTA) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
+__global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
     __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16];
     __shared__ __align__(128) PullWarp s_pull[WARPS];
     const int warp = threadIdx.x >> 5;
+    pdl_wait();
+    pdl_launch_dependents();
     const int path = select_path(d, th3, force_path);
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
     if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp]);
@@ -490,9 +524,26 @@ __global__ void __launch_bounds__(CTA) k_compute(Device d, Out out, float th3, i
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(CMP_TPB) k_compact_count(Device d) {
     __shared__ int s_red[CMP_TPB / 32];
+    pdl_wait();
+    pdl_launch_dependents();
     const int n_words = (d.mb + 1) / 2;
     const int wi = blockIdx.x * CMP_TPB + threadIdx.x;
-    int c = wi < n_words ? __popc(d.ws.y_mask32[wi]) : 0;
+    int c = 0;
+    if (wi < n_words) {
+        // 32 row flags (bytes, 0 or 1) -> one mask word; the flags are cleared for the next call
+        uint4 *f4 = reinterpret_cast<uint4 *>(d.ws.y_hit8 + (size_t)wi * 32);
+        const uint4 a = f4[0], b = f4[1];
+        const uint32_t v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        uint32_t word = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) word |= (((v[q] & 0x01010101u) * 0x01020408u) >> 24 & 0xFu) << (4 * q);
+        if (word) {
+            f4[0] = make_uint4(0u, 0u, 0u, 0u);
+            f4[1] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        d.ws.y_mask32[wi] = word;
+        c = __popc(word);
+    }
     c = __reduce_add_sync(FULL, c);
     if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = c;
     __syncthreads();
@@ -510,6 +561,7 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
     __shared__ int s_base;
     const int n_tiles = d.ws.n_tiles;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_wait();
     if ((int)blockIdx.x < n_tiles) {
         // entries in all earlier tiles
         int before = 0;
@@ -559,7 +611,6 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
                 }
             }
         }
-        if (word) d.ws.y_mask32[wi] = 0u;
         if ((int)blockIdx.x == n_tiles - 1 && threadIdx.x == CMP_TPB - 1) {
             Counters *c2 = d.ws.ctr;
             const int total = wbase + incl;
@@ -616,6 +667,23 @@ template <typename T> static int dev_alloc_zero(T **p, size_t count, int64_t *to
     return DBSPMSPV_OK;
 }
 
+// Launch with the programmatic-stream-serialisation attribute (see pdl_wait): the kernel may be
+// scheduled while its predecessor in the stream is still draining.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 template <int DT, typename Out> static int compute_grid(int sm_count) {
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_compute<DT, Out>, CTA, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
@@ -636,6 +704,7 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     DBS_WS(dev_alloc_zero(&ws.tasks, (size_t)ws.task_capacity, &total));
     DBS_WS(dev_alloc_zero(&ws.y_acc, ywords * 32, &total));
     DBS_WS(dev_alloc_zero(&ws.y_mask32, ywords, &total));
+    DBS_WS(dev_alloc_zero(&ws.y_hit8, ywords * 32, &total));
     DBS_WS(dev_alloc_zero(&ws.tile_count, (size_t)ws.n_tiles, &total));
     DBS_WS(dev_alloc_zero(&ws.visited32, d.m == d.n ? ywords : 1, &total));
     DBS_WS(dev_alloc_zero(&ws.ctr, 1, &total));
@@ -660,16 +729,17 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     static int grid = 0;
     if (!grid) grid = compute_grid<DT, OutSparse>(h->sm_count);
     if (nnz_x > 0) { k_xblock_sparse<DT><<<(nnz_x + 255) / 256, 256, 0, st>>>(d, x_idx, semiring == DBSPMSPV_OR_AND ? nullptr : x_val, nnz_x, h->ropts.validate); ++h->kernel_launches; }
-    OutSparse out{d.ws.y_acc, d.ws.y_mask32};
+    OutSparse out{d.ws.y_acc, d.ws.y_hit8};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
-    if (nnz_x > 0 && d.n_entries > 0) { k_compute<DT, OutSparse><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold); ++h->kernel_launches; }
+    if (nnz_x > 0 && d.n_entries > 0) { DBS_CUDA(launch_pdl(k_compute<DT, OutSparse>, grid, CTA, st, d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold)); ++h->kernel_launches; }
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
     h->kernel_launches += 2;
     const int nt = d.ws.n_tiles;
-    k_compact_count<<<nt, CMP_TPB, 0, st>>>(d);
+    DBS_CUDA(launch_pdl(k_compact_count, nt, CMP_TPB, st, d));
     int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
     if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
-    k_compact_write<<<nt + extra, CMP_TPB, 0, st>>>(d, y_idx, y_val, y_capacity, y_nnz, semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN, x_idx, nnz_x);
+    DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, st, d, y_idx, y_val, y_capacity, y_nnz,
+                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x));
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }

@@ -32,14 +32,15 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
         atomicAdd(n_nzblk, n_new);
     }
     base = __shfl_sync(0xFFFFFFFFu, base, 0) + incl - nchunks;
-    // task record: column block in bits 0..26, (entries - 1) in bits 27..31, first position.
+    // task record: column block in bits 0..26, ceil(entries / 4) - 1 in bits 27..31 (the exact
+    // end comes from the column pointer), first position.
     // Short columns are written by their own lane; a long column block (a hub) is written by
     // the whole warp so that one lane does not serialise thousands of stores.
     constexpr int SMALL = 4;
     if (nchunks <= SMALL)
         for (int k = 0; k < nchunks; ++k) {
             const int cnt = min(PUSH_CHUNK, deg - k * PUSH_CHUNK);
-            d.ws.tasks[base + k] = make_uint2((uint32_t)jb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(first + k * PUSH_CHUNK));
+            d.ws.tasks[base + k] = make_uint2((uint32_t)jb | ((uint32_t)((cnt + 3) / 4 - 1) << 27), (uint32_t)(first + k * PUSH_CHUNK));
         }
     uint32_t big = __ballot_sync(0xFFFFFFFFu, nchunks > SMALL);
     while (big) {
@@ -52,7 +53,7 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
         const int bn = (bdeg + PUSH_CHUNK - 1) / PUSH_CHUNK;
         for (int k = lane; k < bn; k += 32) {
             const int cnt = min(PUSH_CHUNK, bdeg - k * PUSH_CHUNK);
-            d.ws.tasks[bbase + k] = make_uint2((uint32_t)bjb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(bfirst + k * PUSH_CHUNK));
+            d.ws.tasks[bbase + k] = make_uint2((uint32_t)bjb | ((uint32_t)((cnt + 3) / 4 - 1) << 27), (uint32_t)(bfirst + k * PUSH_CHUNK));
         }
     }
 }
