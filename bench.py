@@ -43,11 +43,11 @@ def payload_bytes_per_entry(cls: np.ndarray, nnz: np.ndarray, vsize: int) -> np.
     """Payload bytes of every view entry from the documented per-class sizes."""
     out = np.zeros(cls.size, dtype=np.int64)
     coo = cls == 1
-    out[coo] = ((nnz[coo] + 3) // 4) * 4 + ((nnz[coo] * vsize + 3) // 4) * 4
+    out[coo] = ((nnz[coo] + 3) // 4) * 4 + nnz[coo] * vsize
     mid = (cls >= 2) & (cls <= 4)
-    out[mid] = (48 + ((nnz[mid] * vsize + 3) // 4) * 4) if vsize else 32
+    out[mid] = (48 + nnz[mid] * vsize) if vsize else 32
     out[cls == 5] = 32 + 256 * vsize
-    return out
+    return ((out + 15) // 16) * 16          # every block is padded to 16 bytes
 
 
 class ByteModel:
@@ -175,10 +175,15 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-bfs", action="store_true")
     ap.add_argument("--bfs-scale", type=int, default=22)
+    ap.add_argument("--crossover", action="store_true",
+                    help="print the measured push/pull crossover table (forced paths) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         reference_arm(args)
+        return
+    if args.crossover:
+        crossover_table()
         return
 
     import torch
@@ -371,6 +376,58 @@ def main() -> None:
 # DRAM traffic of that launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
 # summarised in profiles/k_compute_pull_rmat20_x50pct.txt
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 156198400
+
+
+def crossover_table() -> None:
+    """Forced push vs forced pull, whole dbspmspv_run call, cold L2, median of 15: the data
+    behind the default th3 (Section 3.3.1's selector, crossover re-measured on B200)."""
+    import torch
+    from paper_2608_16308_b200 import binding as B
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(h, x, m, path):
+        o = B.default_run_opts()
+        o.force_path = path
+        B.dbspmspv_set_run_opts(h, o)
+        xi, xv = up(x.idx), up(x.val)
+        y_idx = torch.empty(m, dtype=torch.int32, device=dev)
+        y_val = torch.empty(m, dtype=torch.float32, device=dev)
+        y_nnz = torch.zeros(1, dtype=torch.int32, device=dev)
+        ts = []
+        for it in range(18):
+            flush.fill_(it)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.dbspmspv_run(h, xi, xv, int(x.idx.size), B.PLUS_TIMES, y_idx, y_val, m, y_nnz)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts[3:]))
+
+    print("| matrix | x | s_b = N_nzblk/N_blk | push us | pull us | faster |")
+    print("|---|---|---|---|---|---|")
+    cases = []
+    a = wl.uniform_rows()
+    cases.append(("uniform 16384^2, 8/row", a, [("164 nnz", wl.sparse_x(0, 1, a.n, 164))] +
+                  [(f"{f:g}", wl.sparse_x(40 + i, 0, a.n, int(a.n * f))) for i, f in enumerate((0.05, 0.2, 0.5, 1.0))]))
+    a2 = wl.rmat(20, 16, seed=1)
+    fr = list(wl.RMAT_SWEEP) + [0.2, 0.3, 0.7, 1.0]
+    cases.append(("R-MAT scale 20", a2, [(f"{f:g}", wl.rmat_x(a2.n, f, k) if k < 6 else wl.sparse_x(200 + k, 0, a2.n, int(a2.n * f)))
+                                         for k, f in enumerate(fr)]))
+    a3 = wl.stencil27(160, seed=2)
+    cases.append(("27-pt stencil 160^3, runs of 64", a3, [(f"{r * 64 / a3.n:.3g}", wl.clustered_x(a3.n, r))
+                                                          for r in (64, 3200, 12800, 32000)]))
+    for name, mat, xs in cases:
+        h = B.dbspmspv_create_csr(mat.m, mat.n, mat.nnz, up(mat.row_ptr), up(mat.col_idx), up(mat.val), B.F32)
+        nblk = (mat.n + 15) // 16
+        for label, x in sorted(xs, key=lambda t: t[1].idx.size):
+            sb = np.unique(x.idx >> 4).size / nblk
+            tp, tl = timed(h, x, mat.m, B.PATH_PUSH), timed(h, x, mat.m, B.PATH_PULL)
+            print(f"| {name} | {label} | {sb:.4f} | {tp:.1f} | {tl:.1f} | {'push' if tp < tl else 'pull'} |")
+        B.dbspmspv_destroy(h)
 
 
 def cpu_baseline(a, xs, model):

@@ -81,8 +81,8 @@ typedef struct {
     int32_t th1;             /* blocks with more than th1 entries use Dense         (128)    */
     float th2;               /* directional skew ratio for ForceCSR / ForceCSC      (2.0)    */
     int32_t seg_cut;         /* a pull segment closes when its weight reaches this  (128, max)*/
-    int32_t w_dense;         /* pull segment weight of a Dense block                (32)     */
-    int32_t w_mid;           /* ... of a ForceCSR / ForceCSC / CSR block            (16)     */
+    int32_t w_dense;         /* pull segment weight of a Dense block                (16)     */
+    int32_t w_mid;           /* ... of a ForceCSR / ForceCSC / CSR block            (8)      */
     int32_t w_coo;           /* ... of a COO block                                  (4)      */
     int32_t force_format;    /* DBSPMSPV_FORMAT_*: ablation knob (Section 5.4)               */
     int32_t input_on_host;   /* 1: the create arrays are HOST pointers (copied once)         */
@@ -94,15 +94,18 @@ typedef struct {
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
 typedef struct {
-    float th3;               /* push iff nonempty-vector-block ratio < th3 (0.01 in the paper;
-                                the default here is the crossover measured on B200)          */
+    float th3;               /* dbspmspv_run / decode: push iff the nonempty-vector-block ratio is
+                                below th3.  0.01 in the paper; default 0.9, the crossover
+                                measured on B200 (profiles/selector_crossover.md)            */
     int32_t force_path;      /* DBSPMSPV_PATH_*                                              */
     int32_t popc_threshold;  /* CSR-class blocks: popc(mask) >= this -> row-driven (pull-style)
                                 microkernel, below -> column-driven (push-style)             */
     int32_t validate;        /* 1: range-check x indices on the device (ERR_BOUNDS)          */
     int32_t timing;          /* 1: bracket the traversal kernel of run/decode with two CUDA
                                 events (made at create); read back as last_compute_ms      */
-    int32_t reserved[11];
+    float th3_bfs;           /* db_bfs: same rule per level (pull levels skip finished row
+                                blocks and stop early, so the crossover is lower; 0.01)    */
+    int32_t reserved[10];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64
@@ -141,7 +144,7 @@ typedef struct {
 } dbspmspv_stats;
 
 /* Paper thresholds (th0 = 32, th1 = 128, th2 = 2.0, Section 3.2.1).  The segment weights keep
- * the paper's ordering Dense > CSR-like > COO (Section 3.3.2) but are rescaled (32 / 16 / 4 / 1
+ * the paper's ordering Dense > CSR-like > COO (Section 3.3.2) but are rescaled (16 / 8 / 4 / 1
  * against a cut of 128) because one warp step here covers 32 INLINE entries but one heavier
  * block.  Run-time defaults are this library's measured ones.                                      */
 void dbspmspv_default_create_opts(dbspmspv_create_opts *opts);

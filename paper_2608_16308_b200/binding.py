@@ -42,7 +42,8 @@ class CreateOpts(ctypes.Structure):
 class RunOpts(ctypes.Structure):
     _fields_ = [("th3", ctypes.c_float), ("force_path", ctypes.c_int32),
                 ("popc_threshold", ctypes.c_int32), ("validate", ctypes.c_int32),
-                ("timing", ctypes.c_int32), ("reserved", ctypes.c_int32 * 11)]
+                ("timing", ctypes.c_int32), ("th3_bfs", ctypes.c_float),
+                ("reserved", ctypes.c_int32 * 10)]
 
 
 class Stats(ctypes.Structure):

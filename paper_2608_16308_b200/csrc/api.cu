@@ -64,7 +64,7 @@ __global__ void k_export(Device d, const int32_t *block_row, const int32_t *elem
     }
     start -= __popc(mine);
     if (lane >= 16) return;
-    const bool row_major = type == DBSPMSPV_BLK_FCSR || type == DBSPMSPV_BLK_CSR;
+    const bool row_major = type == DBSPMSPV_BLK_FCSR;
     if (type == DBSPMSPV_BLK_DENSE) {
         const uint8_t *vals = blk + 32;
         int k = 0;

@@ -246,7 +246,7 @@ static int bfs_typed(dbspmspv_handle_s *h, int32_t src, int32_t *levels, cudaStr
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_bfs<DT>, BFS_CTA, 0) != cudaSuccess || per_sm < 1) return DBSPMSPV_ERR_CUDA;
         h->bfs_grid = per_sm * h->sm_count;
     }
-    float th3 = h->ropts.th3;
+    float th3 = h->ropts.th3_bfs;
     int force = h->ropts.force_path;
     int max_levels = d.n > 0x7FFFFFFF ? 0x7FFFFFFF : (int)d.n;
     void *args[] = {&d, &src, &levels, &th3, &force, &max_levels};

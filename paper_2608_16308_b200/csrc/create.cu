@@ -113,15 +113,6 @@ struct ClassifyParams {
     int inline_max;   // valued matrices: blocks with at most this many entries are stored inline
 };
 
-__device__ __forceinline__ int payload_words(int type, int nnz, int vsize) {
-    switch (type) {
-        case DBSPMSPV_BLK_INLINE: return 0;
-        case DBSPMSPV_BLK_COO: return (nnz + 3) / 4 + (nnz * vsize + 3) / 4;
-        case DBSPMSPV_BLK_DENSE: return 8 + (256 * vsize) / 4;
-        default: return vsize ? HDR_BYTES / 4 + (nnz * vsize + 3) / 4 : 8;
-    }
-}
-
 __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
                            ClassifyParams cp, uint8_t *type_out, uint32_t *size_out,
                            int32_t *ecount, int32_t *brow, int32_t *bcol, unsigned long long *class_blocks,
@@ -246,7 +237,7 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
         atomicOr(&s_col[warp][rc & 15], 1u << (rc >> 4));
     }
     __syncwarp();
-    const bool row_major = (type == DBSPMSPV_BLK_FCSR || type == DBSPMSPV_BLK_CSR);
+    const bool row_major = (type == DBSPMSPV_BLK_FCSR);
     uint32_t mine = lane < 16 ? (row_major ? s_row[warp][lane] : s_col[warp][lane]) : 0;
     int start = __popc(mine);  // exclusive prefix over lanes 0..15
     for (int o = 1; o < 16; o <<= 1) {
@@ -623,6 +614,11 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     s.m = m; s.n = n; s.nnz = nnzu; s.n_blocks = n_blocks;
     for (int c = 0; c < DBSPMSPV_BLK_NCLASS; ++c) { s.class_blocks[c] = (int64_t)cls_h[c]; s.class_nnz[c] = (int64_t)cls_h[DBSPMSPV_BLK_NCLASS + c]; }
     s.n_row_blocks = d.mb; s.n_col_blocks = d.nb; s.n_segments = d.n_segments;
+    {
+        int64_t heavy_nnz = 0;
+        for (int c = DBSPMSPV_BLK_FCSR; c <= DBSPMSPV_BLK_DENSE; ++c) heavy_nnz += s.class_nnz[c];
+        h->heavy_stage = heavy_nnz * 2 > nnzu;
+    }
     s.payload_bytes = h->payload_bytes;
     s.n_view_entries = d.n_entries;
     s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)d.n_entries * 9;
@@ -669,7 +665,7 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     if (!o) return;
     *o = dbspmspv_create_opts();
     o->th0 = 32; o->th1 = 128; o->th2 = 2.0f;
-    o->seg_cut = 128; o->w_dense = 32; o->w_mid = 16; o->w_coo = 4; o->w_inline = 1;
+    o->seg_cut = 128; o->w_dense = 16; o->w_mid = 8; o->w_coo = 4; o->w_inline = 1;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
     o->inline_max = 8;

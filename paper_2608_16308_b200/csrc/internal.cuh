@@ -27,11 +27,11 @@ namespace dbs {
 // payload in one hop; the payload itself is stored once, in block-CSR ("primary") order.
 //
 // Payload per class (V = value size: 4 fp32, 2 bf16, 0 pattern; every block starts on a
-// 4-byte boundary):
+// 16-byte boundary and is padded to a multiple of 16 bytes):
 //   COO    nnz coordinate bytes, padded to 4 | nnz values
 //   FCSR   16 x u16 row masks | 16 x u8 row starts | values row-major          (Alg. 2)
-//   CSR    same encoding as FCSR (balanced blocks; column access by mask arithmetic)
 //   FCSC   16 x u16 column masks | 16 x u8 column starts | values column-major (Alg. 3)
+//   CSR    same encoding as FCSC (balanced blocks; row access by mask arithmetic)
 //   DENSE  16 x u16 column masks | 256 values column-major (absent entries 0)
 // Pattern matrices keep only the masks (and coordinate bytes).
 // ---------------------------------------------------------------------------------------
@@ -43,6 +43,20 @@ constexpr int TYPE_SHIFT = 29;
 #endif
 constexpr int PUSH_CHUNK = DBS_PUSH_CHUNK;   // CSC-view entries per push task (32 per warp step)
 constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-class block
+constexpr int PAY_CAP = 8192;               // bytes of block payload one warp stages at a time
+
+// Payload size in 4-byte words; every block is padded to 16 bytes so that it can be moved with
+// one bulk copy.  vsize = bytes per value (4 fp32, 2 bf16, 0 pattern).
+__host__ __device__ inline int payload_words(int type, int nnz, int vsize) {
+    int bytes;
+    switch (type) {
+        case DBSPMSPV_BLK_INLINE: return 0;
+        case DBSPMSPV_BLK_COO: bytes = ((nnz + 3) & ~3) + nnz * vsize; break;
+        case DBSPMSPV_BLK_DENSE: bytes = 32 + 256 * vsize; break;
+        default: bytes = vsize ? HDR_BYTES + nnz * vsize : 32; break;
+    }
+    return ((bytes + 15) & ~15) / 4;
+}
 
 struct View {
     int32_t *ptr;    // nb_major + 1
@@ -132,6 +146,7 @@ struct dbspmspv_handle_s {
     void *payload_alloc;
     int64_t payload_bytes;
     int bfs_grid;               // co-resident grid size of the BFS kernel
+    bool heavy_stage;           // most stored elements sit in mask-based blocks: pull stages payloads
     cudaEvent_t ev[2];          // optional timing of the traversal kernel (run_opts.timing)
     bool timed;
     int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)

@@ -3,9 +3,9 @@
 //   INLINE / small COO   one lane owns the whole block (hypersparse blocks dominate power-law
 //                        matrices, so 32 blocks are processed per warp step)
 //   larger COO           one lane per stored entry, shared-memory accumulation
-//   ForceCSR, CSR (dense mask)   row-driven, two lanes per row (Algorithm 2)
-//   CSR (sparse mask)    column-driven over the active columns, row masks give the positions
-//   ForceCSC             column-driven, half-warps split the columns (Algorithm 3)
+//   ForceCSR             row-driven, two lanes per row (Algorithm 2)
+//   CSR (dense mask)     row-driven on the column-major block (row masks rebuilt from the column masks)
+//   CSR (sparse mask), ForceCSC   column-driven, half-warps split the columns (Algorithm 3)
 //   Dense                column-major values, half-warp per active column (role of Algorithm 4)
 // All warp-cooperative kernels leave the partial sum of row (lane & 15) in lanes 0..15 and
 // return the 16-bit mask of rows that received a structural product.
@@ -45,30 +45,36 @@ __device__ __forceinline__ float mk_row_pull(const uint8_t *blk, uint32_t xm, co
     return __shfl_sync(FULL, sum, (lane & 15) * 2);
 }
 
-// Column-driven kernel for row-mask encodings (the push access of the patched-CSR class,
-// Section 3.3.3): walk the active columns only, two at a time (one per half-warp); lane =
-// row tests its own row mask, so no separate column index is stored.
+// Row-driven kernel for column-mask encodings: the pull-style access of the balanced (CSR)
+// class (Section 3.3.3: a relatively dense vector block is reduced by rows).  The block is
+// stored column-major so that sparse masks touch few bytes; here every lane first rebuilds the
+// mask of its own row from the 16 column masks (staged in shared memory), then walks it like
+// Algorithm 2, two lanes per row.  Value position = column start + stored entries above the row.
 template <int DT>
-__device__ __forceinline__ float mk_row_push(const uint8_t *blk, uint32_t xm, const float *s_x,
-                                             int lane, uint32_t &hits) {
+__device__ __forceinline__ float mk_col_pull(const uint8_t *blk, uint32_t xm, const float *s_x,
+                                             uint32_t *s_hdr, int lane, uint32_t &hits) {
     const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
-    const int row = lane & 15, half = lane >> 4;
-    const uint32_t rm = masks[row];
-    const int rp = blk[32 + row];
+    __syncwarp();
+    if (lane < 16) { s_hdr[lane] = masks[lane]; s_hdr[16 + lane] = blk[32 + lane]; }
+    __syncwarp();
+    const int row = lane >> 1, sub = lane & 1;
     const uint8_t *vals = blk + HDR_BYTES;
-    uint32_t act = xm;
+    uint32_t rm = 0;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) rm |= ((s_hdr[c] >> row) & 1u) << c;
+    uint32_t active = rm & xm;
     float sum = 0.f;
-    while (act) {
-        const int c0 = __ffs(act) - 1;
-        act &= act - 1;
-        int c1 = -1;
-        if (act) { c1 = __ffs(act) - 1; act &= act - 1; }
-        const int c = half ? c1 : c0;
-        if (c >= 0 && ((rm >> c) & 1u)) sum += Val<DT>::load(vals, rp + __popc(rm & below(c))) * s_x[c];
+    int nz = 0;
+    while (active) {
+        const int c = __ffs(active) - 1;
+        if ((nz & 1) == sub) sum += Val<DT>::load(vals, s_hdr[16 + c] + __popc(s_hdr[c] & below(row))) * s_x[c];
+        active &= active - 1;
+        ++nz;
     }
-    sum += __shfl_xor_sync(FULL, sum, 16);
-    hits = __ballot_sync(FULL, lane < 16 && (rm & xm) != 0);
-    return sum;
+    sum += __shfl_xor_sync(FULL, sum, 1);
+    uint32_t hm = (lane < 16 && ((xm >> lane) & 1u)) ? s_hdr[lane] : 0u;
+    hits = __reduce_or_sync(FULL, hm);
+    return __shfl_sync(FULL, sum, (lane & 15) * 2);
 }
 
 // Column-driven kernel for column-mask encodings (Algorithm 3): lane = row, the two
@@ -147,12 +153,60 @@ __device__ __forceinline__ float warp_block(int type, const uint8_t *blk, int nn
     switch (type) {
         case DBSPMSPV_BLK_COO: return mk_coo_warp<DT>(blk, nnz, xm, s_x, s_tmp, lane, hits);
         case DBSPMSPV_BLK_FCSR: return mk_row_pull<DT>(blk, xm, s_x, lane, hits);
-        case DBSPMSPV_BLK_CSR:
-            return __popc(xm) >= popc_threshold ? mk_row_pull<DT>(blk, xm, s_x, lane, hits)
-                                                : mk_row_push<DT>(blk, xm, s_x, lane, hits);
+        case DBSPMSPV_BLK_CSR:   // balanced blocks: the local mask decides (Section 3.3.3)
+            return __popc(xm) >= popc_threshold
+                       ? mk_col_pull<DT>(blk, xm, s_x, reinterpret_cast<uint32_t *>(s_tmp), lane, hits)
+                       : mk_col_push<DT>(blk, xm, s_x, lane, hits);
         case DBSPMSPV_BLK_FCSC: return mk_col_push<DT>(blk, xm, s_x, lane, hits);
         default: return mk_dense<DT>(blk, xm, s_x, lane, hits);
     }
+}
+
+// ---- Lane-owned form of the mask-based classes.  When many heavier blocks sit side by side
+// (layers of a pruned model, banded matrices) a warp that took them one at a time would wait
+// out two dependent memory round trips per block; instead every lane walks its own block and
+// the warp keeps 32 blocks in flight.  Products are added into the lane's private column of a
+// shared 16 x 33 scratch (`acc` points at it, stride 33 floats: conflict free), so no atomics
+// are needed; the caller then folds the column into the row block's result.
+constexpr int LANE_ACC_STRIDE = 33;
+template <int DT>
+__device__ __forceinline__ uint32_t lane_heavy(int type, const uint8_t *blk, uint32_t xm,
+                                               const float *xb, float *acc) {
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    uint32_t hit = 0;
+    if (type == DBSPMSPV_BLK_FCSR) {            // row masks, row-major values
+        const uint8_t *vals = blk + HDR_BYTES;
+        for (int r = 0; r < 16; ++r) {
+            const uint32_t full = masks[r];
+            uint32_t act = full & xm;
+            if (!act) continue;
+            const int base = blk[32 + r];
+            float s = 0.f;
+            for (; act; act &= act - 1) {
+                const int c = __ffs(act) - 1;
+                s += Val<DT>::load(vals, base + __popc(full & below(c))) * xb[c];
+            }
+            acc[r * LANE_ACC_STRIDE] += s;
+            hit |= 1u << r;
+        }
+        return hit;
+    }
+    const bool dense = type == DBSPMSPV_BLK_DENSE;
+    const uint8_t *vals = blk + (dense ? 32 : HDR_BYTES);
+    for (uint32_t act = xm; act; act &= act - 1) {   // column masks, column-major values
+        const int c = __ffs(act) - 1;
+        uint32_t cm = masks[c];
+        if (!cm) continue;
+        hit |= cm;
+        const float xc = xb[c];
+        int k = dense ? c * 16 : blk[32 + c];
+        if (dense) {
+            for (; cm; cm &= cm - 1) { const int r = __ffs(cm) - 1; acc[r * LANE_ACC_STRIDE] += Val<DT>::load(vals, k + r) * xc; }
+        } else {
+            for (; cm; cm &= cm - 1, ++k) { const int r = __ffs(cm) - 1; acc[r * LANE_ACC_STRIDE] += Val<DT>::load(vals, k) * xc; }
+        }
+    }
+    return hit;
 }
 
 // ---- Boolean forms (Section 4.2, Algorithm 5): only reachability; values are never read.
@@ -171,11 +225,25 @@ __device__ __forceinline__ uint32_t warp_block_bool(int type, const uint8_t *blk
         }
         return __reduce_or_sync(FULL, hm);
     }
-    if (type == DBSPMSPV_BLK_FCSR || type == DBSPMSPV_BLK_CSR)
+    if (type == DBSPMSPV_BLK_FCSR)
         return __ballot_sync(FULL, lane < 16 && (masks[lane & 15] & xm) != 0);
     // column masks: OR of the active columns' masks
     uint32_t hm = (lane < 16 && ((xm >> lane) & 1u)) ? masks[lane] : 0u;
     return __reduce_or_sync(FULL, hm);
 }
+
+// Lane-owned Boolean form: rows of one mask-based block reached from the active columns.
+__device__ __forceinline__ uint32_t lane_heavy_bool(int type, const uint8_t *blk, uint32_t xm) {
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    uint32_t hit = 0;
+    if (type == DBSPMSPV_BLK_FCSR) {
+        for (int r = 0; r < 16; ++r) hit |= (masks[r] & xm) ? (1u << r) : 0u;
+    } else {
+        for (uint32_t act = xm; act; act &= act - 1) hit |= masks[__ffs(act) - 1];
+    }
+    return hit;
+}
+
+constexpr int HEAVY_LANE_MIN = 4;   // this many mask-based blocks in one warp step -> lane-owned form
 
 }  // namespace dbs

@@ -206,7 +206,7 @@ __device__ __forceinline__ void flush_rows(Out out, int rb, uint32_t hits, float
 // the row block's hit mask.  The task record carries its length, so the view entries, the mask
 // and the x block are all fetched in one round of independent loads.
 template <int DT, typename Out>
-__device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp) {
+__device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp, float *s_lacc) {
     constexpr int U = PUSH_CHUNK / 32;
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -262,6 +262,29 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                 __syncwarp();
             }
             uint32_t hv = __ballot_sync(FULL, heavy);
+            const uint32_t hv_mask = __ballot_sync(FULL, heavy && type != DBSPMSPV_BLK_COO);
+            if (__popc(hv_mask) >= HEAVY_LANE_MIN) {
+                // many mask-based blocks side by side: every lane walks its own block
+                if (heavy && type != DBSPMSPV_BLK_COO) {
+                    const uint8_t *blk = d.payload + (size_t)w[u] * 4;
+                    float *acc = s_lacc + lane;
+                    uint32_t hits;
+                    if (DT == DBSPMSPV_PATTERN) {
+                        hits = lane_heavy_bool(type, blk, xm);
+                    } else {
+#pragma unroll
+                        for (int r = 0; r < 16; ++r) acc[r * LANE_ACC_STRIDE] = 0.f;
+                        hits = lane_heavy<DT>(type, blk, xm, s_x, acc);
+                    }
+                    for (uint32_t hh = hits; hh; hh &= hh - 1) {
+                        const int r = __ffs(hh) - 1;
+                        if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)brow * 16 + r, acc[r * LANE_ACC_STRIDE]);
+                        if (Out::MASKS) out.hit8[(size_t)brow * 16 + r] = 1;
+                    }
+                }
+                __syncwarp();
+                hv &= ~hv_mask;   // oversized COO blocks (forced format) stay with the warp form
+            }
             while (hv) {
                 const int src = __ffs(hv) - 1;
                 hv &= hv - 1;
@@ -322,7 +345,7 @@ __device__ __forceinline__ void pull_issue(const Device &d, int e0, int e1, Pull
 
 template <int DT, typename Out>
 __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp,
-                          float *s_y, PullWarp *pw) {
+                          float *s_y, float *s_lacc, PullWarp *pw) {
     const int lane = threadIdx.x & 31;
     const uint32_t le_mask = 0xFFFFFFFFu >> (31 - lane);
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -356,7 +379,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
             parity ^= 1u << cur;
         }
         const PullStage *st = &pw->stage[cur];
-        int cur_ord = -1, cur_rb = 0;     // segment held in the shared accumulator
+        int cur_rb = -1;                  // row block held in the shared accumulator
         uint32_t hit = 0;
         for (int base = e0; base < e1; base += 32 * PULL_UNROLL) {
             uint32_t idx[PULL_UNROLL], w[PULL_UNROLL], aux[PULL_UNROLL];
@@ -382,9 +405,10 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                 const int ord = ord_base + __popc(fb & le_mask);
                 ord_base += __popc(fb);
                 const int rb = have ? d.seg_rb[ord] : 0;
-                // the shared accumulator follows the segment of the step's first entry
-                const int ord0 = __shfl_sync(FULL, ord, 0);
-                if (ord0 != cur_ord) {
+                // the shared accumulator follows the row block of the step's first entry (a long
+                // row block keeps it over all its segments of the chunk)
+                const int rb0 = __shfl_sync(FULL, rb, 0);
+                if (rb0 != cur_rb) {
                     hit = __reduce_or_sync(FULL, hit);
                     __syncwarp();
                     if (lane < 16) {
@@ -395,8 +419,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                         s_y[lane] = 0.f;
                     }
                     hit = 0;
-                    cur_ord = ord0;
-                    cur_rb = __shfl_sync(FULL, rb, 0);
+                    cur_rb = rb0;
                     __syncwarp();
                 }
                 const int type = idx[u] >> TYPE_SHIFT;
@@ -406,7 +429,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                         if (__float_as_uint(xin[u]) != X_ABSENT) {
                             const float v = Val<DT>::inline_value(w[u]) * xin[u];
                             const int r = aux[u] >> 4;
-                            if (ord == cur_ord) {
+                            if (rb == cur_rb) {
                                 atomicAdd(&s_y[r], v);
                                 hit |= 1u << r;
                             } else {
@@ -449,6 +472,44 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                     __syncwarp();
                 }
                 uint32_t hv = __ballot_sync(FULL, heavy);
+                const uint32_t hv_mask = __ballot_sync(FULL, heavy && type != DBSPMSPV_BLK_COO);
+                if (__popc(hv_mask) >= HEAVY_LANE_MIN) {
+                    // many mask-based blocks side by side: every lane walks its own block and
+                    // leaves 16 partial sums in its private scratch column.  Blocks of the row
+                    // block held in the shared accumulator are then summed across lanes by 16
+                    // lanes (no atomics); blocks of other row blocks go straight to global.
+                    const bool mine = heavy && type != DBSPMSPV_BLK_COO;
+                    float *acc = s_lacc + lane;
+                    uint32_t hits = 0;
+                    if (mine) {
+                        const uint8_t *blk = d.payload + (size_t)w[u] * 4;
+                        if (DT == DBSPMSPV_PATTERN) {
+                            hits = lane_heavy_bool(type, blk, xm);
+                        } else {
+#pragma unroll
+                            for (int r = 0; r < 16; ++r) acc[r * LANE_ACC_STRIDE] = 0.f;
+                            hits = lane_heavy<DT>(type, blk, xm, d.ws.x_dense + (size_t)bcol_l * 16, acc);
+                        }
+                    }
+                    const bool in_cur = mine && rb == cur_rb;
+                    const uint32_t members = __ballot_sync(FULL, in_cur);
+                    __syncwarp();
+                    if (in_cur) hit |= hits;
+                    if (DT != DBSPMSPV_PATTERN && members && lane < 16) {
+                        float t = 0.f;
+                        for (uint32_t mm = members; mm; mm &= mm - 1) t += s_lacc[lane * LANE_ACC_STRIDE + __ffs(mm) - 1];
+                        s_y[lane] += t;
+                    }
+                    if (mine && !in_cur) {
+                        for (uint32_t hh = hits; hh; hh &= hh - 1) {
+                            const int r = __ffs(hh) - 1;
+                            if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)rb * 16 + r, acc[r * LANE_ACC_STRIDE]);
+                            if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
+                        }
+                    }
+                    __syncwarp();
+                    hv &= ~hv_mask;
+                }
                 while (hv) {
                     const int src = __ffs(hv) - 1;
                     hv &= hv - 1;
@@ -507,14 +568,15 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
 template <int DT, typename Out>
 __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
     __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16];
+    __shared__ float s_lacc[WARPS][16 * LANE_ACC_STRIDE];
     __shared__ __align__(128) PullWarp s_pull[WARPS];
     const int warp = threadIdx.x >> 5;
     pdl_wait();
     pdl_launch_dependents();
     const int path = select_path(d, th3, force_path);
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
-    if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp]);
-    else pull_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], &s_pull[warp]);
+    if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_lacc[warp]);
+    else pull_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], s_lacc[warp], &s_pull[warp]);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -773,7 +835,8 @@ extern "C" {
 void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
-    o->th3 = 0.01f;
+    o->th3 = 0.9f;
+    o->th3_bfs = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;
     o->popc_threshold = 8;
     o->validate = 0;
@@ -782,7 +845,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
 int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts) {
     if (!h || !opts) return DBSPMSPV_ERR_INVALID_ARG;
     if (opts->force_path < DBSPMSPV_PATH_AUTO || opts->force_path > DBSPMSPV_PATH_PULL) return DBSPMSPV_ERR_INVALID_ARG;
-    if (!(opts->th3 >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!(opts->th3 >= 0.f) || !(opts->th3_bfs >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
     h->ropts = *opts;
     return DBSPMSPV_OK;
 }

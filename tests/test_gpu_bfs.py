@@ -123,7 +123,7 @@ def test_chebyshev_closed_form_and_valued_handle():
 def test_auto_switches_direction_across_levels():
     g = wl.rmat(14, 16, seed=4, values=False, symmetrise=True)
     h = Handle(g, B.PATTERN)
-    h.set_opts(th3=0.01)
+    h.set_opts(th3_bfs=0.01)
     src = int(wl.bfs_sources(g, 1, seed=9)[0])
     bfs(h, src)
     st = h.get_stats()
