@@ -94,7 +94,7 @@ typedef struct {
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
 typedef struct {
-    float th3;               /* dbspmspv_run / decode: push iff the nonempty-vector-block ratio is
+    float th3;               /* dbspmspv_run: push iff the nonempty-vector-block ratio is
                                 below th3.  0.01 in the paper; default 0.9, the crossover
                                 measured on B200 (profiles/selector_crossover.md)            */
     int32_t force_path;      /* DBSPMSPV_PATH_*                                              */
@@ -105,7 +105,9 @@ typedef struct {
                                 events (made at create); read back as last_compute_ms      */
     float th3_bfs;           /* db_bfs: same rule per level (pull levels skip finished row
                                 blocks and stop early, so the crossover is lower; 0.01)    */
-    int32_t reserved[10];
+    float th3_decode;        /* dbspmspv_decode: same rule; the output is dense and every row block
+                                takes part, so pull wins much earlier (0.01, the paper's value) */
+    int32_t reserved[9];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64

@@ -64,7 +64,7 @@ __global__ void k_export(Device d, const int32_t *block_row, const int32_t *elem
     }
     start -= __popc(mine);
     if (lane >= 16) return;
-    const bool row_major = type == DBSPMSPV_BLK_FCSR;
+    const bool row_major = is_row_major(type);
     if (type == DBSPMSPV_BLK_DENSE) {
         const uint8_t *vals = blk + 32;
         int k = 0;
@@ -91,7 +91,7 @@ __global__ void k_export_blocks(Device d, const int32_t *brow, int32_t *block_ro
     const uint32_t idx = d.csr.idx[b];
     if (block_row) block_row[b] = brow[b];
     if (block_col) block_col[b] = (int32_t)(idx & IDX_MASK);
-    if (block_class) block_class[b] = (int32_t)(idx >> TYPE_SHIFT);
+    if (block_class) block_class[b] = (int32_t)public_class((int)(idx >> TYPE_SHIFT));
     if (nnz) nnz[b] = block_nnz(d.dtype, idx, d.csr.aux[b]);
 }
 

@@ -153,7 +153,7 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
             // the two axis skews are identical for square blocks
             else if ((float)ccount > cp.th2 * (float)rcount) type = DBSPMSPV_BLK_FCSC;
             else if ((float)rcount > cp.th2 * (float)ccount) type = DBSPMSPV_BLK_FCSR;
-            else type = DBSPMSPV_BLK_CSR;
+            else type = rcount <= CSR_SHORT_ROW ? BLK_CSR_ROWMAJOR : DBSPMSPV_BLK_CSR;
             const int vsize = cp.dtype == DBSPMSPV_F32 ? 4 : cp.dtype == DBSPMSPV_BF16 ? 2 : 0;
             type_out[b] = (uint8_t)type;
             size_out[b] = (uint32_t)payload_words(type, nnz, vsize);
@@ -161,8 +161,8 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
             uint64_t k0 = ukey[s];
             brow[b] = (int32_t)(k0 >> 35);
             bcol[b] = (int32_t)((k0 >> 8) & IDX_MASK);
-            atomicAdd(&s_cb[type], 1u);
-            atomicAdd(&s_cn[type], (unsigned)nnz);
+            atomicAdd(&s_cb[public_class(type)], 1u);
+            atomicAdd(&s_cn[public_class(type)], (unsigned)nnz);
         }
     }
     __syncthreads();
@@ -237,7 +237,7 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
         atomicOr(&s_col[warp][rc & 15], 1u << (rc >> 4));
     }
     __syncwarp();
-    const bool row_major = (type == DBSPMSPV_BLK_FCSR);
+    const bool row_major = is_row_major(type);
     uint32_t mine = lane < 16 ? (row_major ? s_row[warp][lane] : s_col[warp][lane]) : 0;
     int start = __popc(mine);  // exclusive prefix over lanes 0..15
     for (int o = 1; o < 16; o <<= 1) {

@@ -31,11 +31,20 @@ namespace dbs {
 //   COO    nnz coordinate bytes, padded to 4 | nnz values
 //   FCSR   16 x u16 row masks | 16 x u8 row starts | values row-major          (Alg. 2)
 //   FCSC   16 x u16 column masks | 16 x u8 column starts | values column-major (Alg. 3)
-//   CSR    same encoding as FCSC (balanced blocks; row access by mask arithmetic)
+//   CSR    balanced blocks: same encoding as FCSC (column-major suits sparse vector blocks;
+//          row access by mask arithmetic) -- except blocks whose longest row has at most
+//          CSR_SHORT_ROW entries (banded/stencil blocks), which use the FCSR encoding: two
+//          lanes per row then finish in one or two steps (internal code BLK_CSR_ROWMAJOR)
 //   DENSE  16 x u16 column masks | 256 values column-major (absent entries 0)
 // Pattern matrices keep only the masks (and coordinate bytes).
 // ---------------------------------------------------------------------------------------
 constexpr int B = 16;                       // block edge
+// Internal class code 6: a balanced (CSR-class) block whose rows are short, stored row-major
+// like ForceCSR; statistics and exports report it as DBSPMSPV_BLK_CSR.
+constexpr int BLK_CSR_ROWMAJOR = 6;
+constexpr int CSR_SHORT_ROW = 4;            // longest row at most this -> row-major sub-form
+__host__ __device__ inline bool is_row_major(int type) { return type == DBSPMSPV_BLK_FCSR || type == BLK_CSR_ROWMAJOR; }
+__host__ __device__ inline int public_class(int type) { return type == BLK_CSR_ROWMAJOR ? DBSPMSPV_BLK_CSR : type; }
 constexpr uint32_t IDX_MASK = 0x07FFFFFFu;  // 27 bits
 constexpr int TYPE_SHIFT = 29;
 #ifndef DBS_PUSH_CHUNK

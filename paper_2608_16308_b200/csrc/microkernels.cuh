@@ -152,7 +152,8 @@ __device__ __forceinline__ float warp_block(int type, const uint8_t *blk, int nn
                                             int popc_threshold, uint32_t &hits) {
     switch (type) {
         case DBSPMSPV_BLK_COO: return mk_coo_warp<DT>(blk, nnz, xm, s_x, s_tmp, lane, hits);
-        case DBSPMSPV_BLK_FCSR: return mk_row_pull<DT>(blk, xm, s_x, lane, hits);
+        case DBSPMSPV_BLK_FCSR:
+        case BLK_CSR_ROWMAJOR: return mk_row_pull<DT>(blk, xm, s_x, lane, hits);
         case DBSPMSPV_BLK_CSR:   // balanced blocks: the local mask decides (Section 3.3.3)
             return __popc(xm) >= popc_threshold
                        ? mk_col_pull<DT>(blk, xm, s_x, reinterpret_cast<uint32_t *>(s_tmp), lane, hits)
@@ -174,7 +175,7 @@ __device__ __forceinline__ uint32_t lane_heavy(int type, const uint8_t *blk, uin
                                                const float *xb, float *acc) {
     const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
     uint32_t hit = 0;
-    if (type == DBSPMSPV_BLK_FCSR) {            // row masks, row-major values
+    if (is_row_major(type)) {                   // row masks, row-major values
         const uint8_t *vals = blk + HDR_BYTES;
         for (int r = 0; r < 16; ++r) {
             const uint32_t full = masks[r];
@@ -225,7 +226,7 @@ __device__ __forceinline__ uint32_t warp_block_bool(int type, const uint8_t *blk
         }
         return __reduce_or_sync(FULL, hm);
     }
-    if (type == DBSPMSPV_BLK_FCSR)
+    if (is_row_major(type))
         return __ballot_sync(FULL, lane < 16 && (masks[lane & 15] & xm) != 0);
     // column masks: OR of the active columns' masks
     uint32_t hm = (lane < 16 && ((xm >> lane) & 1u)) ? masks[lane] : 0u;
@@ -236,7 +237,7 @@ __device__ __forceinline__ uint32_t warp_block_bool(int type, const uint8_t *blk
 __device__ __forceinline__ uint32_t lane_heavy_bool(int type, const uint8_t *blk, uint32_t xm) {
     const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
     uint32_t hit = 0;
-    if (type == DBSPMSPV_BLK_FCSR) {
+    if (is_row_major(type)) {
         for (int r = 0; r < 16; ++r) hit |= (masks[r] & xm) ? (1u << r) : 0u;
     } else {
         for (uint32_t act = xm; act; act &= act - 1) hit |= masks[__ffs(act) - 1];

@@ -205,7 +205,7 @@ __device__ __forceinline__ void flush_rows(Out out, int rb, uint32_t hits, float
 // Writeback: warp-level reduction, then one global atomic per touched row and one atomicOr on
 // the row block's hit mask.  The task record carries its length, so the view entries, the mask
 // and the x block are all fetched in one round of independent loads.
-template <int DT, typename Out>
+template <int DT, typename Out, bool HV>
 __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp, float *s_lacc) {
     constexpr int U = PUSH_CHUNK / 32;
     const int lane = threadIdx.x & 31;
@@ -262,10 +262,13 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                 __syncwarp();
             }
             uint32_t hv = __ballot_sync(FULL, heavy);
-            const uint32_t hv_mask = __ballot_sync(FULL, heavy && type != DBSPMSPV_BLK_COO);
-            if (__popc(hv_mask) >= HEAVY_LANE_MIN) {
+            // sparse local mask -> lane-owned form; dense local mask -> warp form (Section 3.3.3:
+            // the number of active entries of the vector block picks the microkernel)
+            const bool lane_form = heavy && type != DBSPMSPV_BLK_COO && __popc(xm) < popc_threshold;
+            const uint32_t hv_mask = HV ? __ballot_sync(FULL, lane_form) : 0u;
+            if (HV && __popc(hv_mask) >= HEAVY_LANE_MIN) {
                 // many mask-based blocks side by side: every lane walks its own block
-                if (heavy && type != DBSPMSPV_BLK_COO) {
+                if (lane_form) {
                     const uint8_t *blk = d.payload + (size_t)w[u] * 4;
                     float *acc = s_lacc + lane;
                     uint32_t hits;
@@ -343,16 +346,22 @@ __device__ __forceinline__ void pull_issue(const Device &d, int e0, int e1, Pull
     }
 }
 
-template <int DT, typename Out>
+template <int DT, typename Out, bool HV, bool HS>
 __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp,
-                          float *s_y, float *s_lacc, PullWarp *pw) {
+                          float *s_y, float *s_lacc, PullWarp *pw, uint8_t *s_pay, uint64_t *pay_bar) {
     const int lane = threadIdx.x & 31;
     const uint32_t le_mask = 0xFFFFFFFFu >> (31 - lane);
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
-    if (lane == 0) { mbar_init(&pw->bar[0], 1); mbar_init(&pw->bar[1], 1); fence_barrier_init(); }
+    if (lane == 0) {
+        mbar_init(&pw->bar[0], 1); mbar_init(&pw->bar[1], 1);
+        if (HS) mbar_init(pay_bar, 1);
+        fence_barrier_init();
+    }
     if (lane < 16) s_y[lane] = 0.f;
     __syncwarp();
+    uint32_t pay_parity = 0u;
+    bool failed = false;              // a bounded wait ran out: stop, report, leave cleanly
     uint32_t parity = 0u;             // bit s: phase parity of stage s
     int cur = 0;
     bool next_in_flight = false;
@@ -381,7 +390,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
         const PullStage *st = &pw->stage[cur];
         int cur_rb = -1;                  // row block held in the shared accumulator
         uint32_t hit = 0;
-        for (int base = e0; base < e1; base += 32 * PULL_UNROLL) {
+        for (int base = e0; base < e1 && !failed; base += 32 * PULL_UNROLL) {
             uint32_t idx[PULL_UNROLL], w[PULL_UNROLL], aux[PULL_UNROLL];
             float xin[PULL_UNROLL];
 #pragma unroll
@@ -472,42 +481,80 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                     __syncwarp();
                 }
                 uint32_t hv = __ballot_sync(FULL, heavy);
-                const uint32_t hv_mask = __ballot_sync(FULL, heavy && type != DBSPMSPV_BLK_COO);
-                if (__popc(hv_mask) >= HEAVY_LANE_MIN) {
-                    // many mask-based blocks side by side: every lane walks its own block and
-                    // leaves 16 partial sums in its private scratch column.  Blocks of the row
+                // sparse local mask -> lane-owned form; dense local mask -> warp form
+                const bool lane_form = heavy && type != DBSPMSPV_BLK_COO && __popc(xm) < popc_threshold;
+                const uint32_t hv_mask = HV ? __ballot_sync(FULL, lane_form) : 0u;
+                if (HV && ((HS && hv_mask) || __popc(hv_mask) >= HEAVY_LANE_MIN)) {
+                    // Mask-based blocks side by side (layers of a pruned model, banded matrices):
+                    // every lane walks its own block and leaves 16 partial sums in its private
+                    // scratch column, so the warp keeps up to 32 blocks going.  Blocks of the row
                     // block held in the shared accumulator are then summed across lanes by 16
                     // lanes (no atomics); blocks of other row blocks go straight to global.
-                    const bool mine = heavy && type != DBSPMSPV_BLK_COO;
+                    // HS variant (matrices made of such blocks): the payloads of the touched
+                    // blocks are first staged in shared memory by bulk copies, one per block,
+                    // issued by the lane that holds the block (Section 3.3.3), in groups that fit
+                    // the stage, and the lanes then read their block from shared memory.
+                    const bool mine = lane_form;
                     float *acc = s_lacc + lane;
-                    uint32_t hits = 0;
-                    if (mine) {
+                    int bytes = 0, incl = 0;
+                    if (HS) {
+                        bytes = mine ? payload_words(type, (int)aux[u] + 1, Val<DT>::SIZE) * 4 : 0;
+                        incl = bytes;
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const int t = __shfl_up_sync(FULL, incl, o);
+                            if (lane >= o) incl += t;
+                        }
+                    }
+                    const int off = incl - bytes;
+                    uint32_t remaining = hv_mask;
+                    while (remaining) {
+                        uint32_t grp = remaining;
                         const uint8_t *blk = d.payload + (size_t)w[u] * 4;
-                        if (DT == DBSPMSPV_PATTERN) {
-                            hits = lane_heavy_bool(type, blk, xm);
-                        } else {
+                        if (HS) {
+                            const int gbase = __shfl_sync(FULL, off, __ffs(remaining) - 1);
+                            const bool fits = ((remaining >> lane) & 1u) && (incl - gbase <= PAY_CAP);
+                            grp = __ballot_sync(FULL, fits);
+                            const int total = __shfl_sync(FULL, incl, 31 - __clz(grp)) - gbase;
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == __ffs(grp) - 1) mbar_arrive_expect_tx(pay_bar, (uint32_t)total);
+                            __syncwarp();
+                            if (fits) bulk_copy_g2s(s_pay + (off - gbase), blk, (uint32_t)bytes, pay_bar);
+                            blk = s_pay + (off - gbase);
+                        }
+                        const bool in_grp = (grp >> lane) & 1u;
+                        if (in_grp && DT != DBSPMSPV_PATTERN) {
 #pragma unroll
                             for (int r = 0; r < 16; ++r) acc[r * LANE_ACC_STRIDE] = 0.f;
-                            hits = lane_heavy<DT>(type, blk, xm, d.ws.x_dense + (size_t)bcol_l * 16, acc);
                         }
-                    }
-                    const bool in_cur = mine && rb == cur_rb;
-                    const uint32_t members = __ballot_sync(FULL, in_cur);
-                    __syncwarp();
-                    if (in_cur) hit |= hits;
-                    if (DT != DBSPMSPV_PATTERN && members && lane < 16) {
-                        float t = 0.f;
-                        for (uint32_t mm = members; mm; mm &= mm - 1) t += s_lacc[lane * LANE_ACC_STRIDE + __ffs(mm) - 1];
-                        s_y[lane] += t;
-                    }
-                    if (mine && !in_cur) {
-                        for (uint32_t hh = hits; hh; hh &= hh - 1) {
-                            const int r = __ffs(hh) - 1;
-                            if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)rb * 16 + r, acc[r * LANE_ACC_STRIDE]);
-                            if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
+                        if (HS) {
+                            if (!mbar_wait_bounded(pay_bar, pay_parity)) { failed = true; break; }
+                            pay_parity ^= 1u;
                         }
+                        uint32_t hits = 0;
+                        if (in_grp)
+                            hits = DT == DBSPMSPV_PATTERN ? lane_heavy_bool(type, blk, xm)
+                                                          : lane_heavy<DT>(type, blk, xm, d.ws.x_dense + (size_t)bcol_l * 16, acc);
+                        const bool in_cur = in_grp && rb == cur_rb;
+                        const uint32_t members = __ballot_sync(FULL, in_cur);
+                        __syncwarp();
+                        if (in_cur) hit |= hits;
+                        if (DT != DBSPMSPV_PATTERN && members && lane < 16) {
+                            float t = 0.f;
+                            for (uint32_t mm = members; mm; mm &= mm - 1) t += s_lacc[lane * LANE_ACC_STRIDE + __ffs(mm) - 1];
+                            s_y[lane] += t;
+                        }
+                        if (in_grp && !in_cur) {
+                            for (uint32_t hh = hits; hh; hh &= hh - 1) {
+                                const int r = __ffs(hh) - 1;
+                                if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)rb * 16 + r, acc[r * LANE_ACC_STRIDE]);
+                                if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
+                            }
+                        }
+                        remaining &= ~grp;
+                        __syncwarp();
                     }
-                    __syncwarp();
+                    if (failed) break;
                     hv &= ~hv_mask;
                 }
                 while (hv) {
@@ -535,6 +582,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                 }
             }
         }
+        if (failed) { d.ws.ctr->status = DBSPMSPV_ERR_TIMEOUT; break; }
         // end of the chunk: flush what the shared accumulator still holds
         hit = __reduce_or_sync(FULL, hit);
         __syncwarp();
@@ -552,6 +600,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
     // left early on a timeout: let the copy still in flight land before the stage memory is
     // given back (bounded, like every wait here)
     if (next_in_flight) mbar_wait_bounded(&pw->bar[cur ^ 1], (parity >> (cur ^ 1)) & 1u);
+    if (HS && failed) mbar_wait_bounded(pay_bar, pay_parity);
 }
 
 // Global selector (Section 3.3.1): s_b = N_nzblk / N_blk; push iff s_b < th3.  Evaluated on
@@ -565,18 +614,35 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
 #ifndef DBS_MIN_CTAS
 #define DBS_MIN_CTAS 1
 #endif
-template <int DT, typename Out>
+// Variants of the traversal kernel, chosen per handle from the class census at create:
+//   MODE 0  hypersparse matrices (power-law graphs): no lane-owned code, smallest footprint
+//   MODE 1  matrices whose elements sit mostly in mask-based blocks: lane-owned microkernels
+//   MODE 2  the same plus payload staging in shared memory (used by the decode entry)
+// Dynamic shared memory: per-warp pull stages | lane scratch (MODE >= 1) | payload stage and
+// its barrier (MODE 2).
+template <int MODE> constexpr size_t compute_dyn_smem() {
+    return WARPS * sizeof(PullWarp) + (MODE >= 1 ? WARPS * 16 * LANE_ACC_STRIDE * sizeof(float) : 0) +
+           (MODE == 2 ? WARPS * (size_t)PAY_CAP + WARPS * sizeof(uint64_t) : 0);
+}
+
+template <int DT, typename Out, int MODE>
 __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
+    constexpr bool HV = MODE >= 1, HS = MODE == 2;
     __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16];
-    __shared__ float s_lacc[WARPS][16 * LANE_ACC_STRIDE];
-    __shared__ __align__(128) PullWarp s_pull[WARPS];
+    extern __shared__ __align__(128) uint8_t s_dyn[];
+    PullWarp *s_pull = reinterpret_cast<PullWarp *>(s_dyn);
+    float *s_lacc = reinterpret_cast<float *>(s_dyn + WARPS * sizeof(PullWarp));
+    uint8_t *s_pay = reinterpret_cast<uint8_t *>(s_lacc + WARPS * 16 * LANE_ACC_STRIDE);
+    uint64_t *s_pay_bar = reinterpret_cast<uint64_t *>(s_pay + WARPS * (size_t)PAY_CAP);
     const int warp = threadIdx.x >> 5;
     pdl_wait();
     pdl_launch_dependents();
     const int path = select_path(d, th3, force_path);
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
-    if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_lacc[warp]);
-    else pull_body<DT, Out>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], s_lacc[warp], &s_pull[warp]);
+    float *lacc = HV ? s_lacc + warp * 16 * LANE_ACC_STRIDE : nullptr;
+    if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], lacc);
+    else pull_body<DT, Out, HV, HS>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], lacc, &s_pull[warp],
+                                    HS ? s_pay + warp * (size_t)PAY_CAP : nullptr, HS ? s_pay_bar + warp : nullptr);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -732,11 +798,11 @@ template <typename T> static int dev_alloc_zero(T **p, size_t count, int64_t *to
 // Launch with the programmatic-stream-serialisation attribute (see pdl_wait): the kernel may be
 // scheduled while its predecessor in the stream is still draining.
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, cudaStream_t st, Args... args) {
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)block);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -746,10 +812,28 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, cud
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-template <int DT, typename Out> static int compute_grid(int sm_count) {
+// Persistent grid of the traversal kernel: as many thread blocks as fit (0 on error).
+template <int DT, typename Out, int MODE> static int compute_grid(int sm_count) {
+    const size_t smem = compute_dyn_smem<MODE>();
+    if (cudaFuncSetAttribute(k_compute<DT, Out, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_compute<DT, Out>, CTA, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_compute<DT, Out, MODE>, CTA, smem) != cudaSuccess || per_sm < 1) return 0;
     return sm_count * per_sm;
+}
+
+template <int DT, typename Out, int MODE>
+static int launch_compute(dbspmspv_handle_s *h, Out out, float th3, bool pdl, cudaStream_t st) {
+    static int grid = 0;
+    if (!grid) grid = compute_grid<DT, Out, MODE>(h->sm_count);
+    if (!grid) return DBSPMSPV_ERR_CUDA;
+    const size_t smem = compute_dyn_smem<MODE>();
+    if (pdl) {
+        DBS_CUDA(launch_pdl(k_compute<DT, Out, MODE>, grid, CTA, smem, st, h->d, out, th3, h->ropts.force_path, h->ropts.popc_threshold));
+    } else {
+        k_compute<DT, Out, MODE><<<grid, CTA, smem, st>>>(h->d, out, th3, h->ropts.force_path, h->ropts.popc_threshold);
+    }
+    ++h->kernel_launches;
+    return DBSPMSPV_OK;
 }
 
 int allocate_workspace(dbspmspv_handle_s *h) {
@@ -788,19 +872,23 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
                      int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
                      cudaStream_t st) {
     const Device &d = h->d;
-    static int grid = 0;
-    if (!grid) grid = compute_grid<DT, OutSparse>(h->sm_count);
     if (nnz_x > 0) { k_xblock_sparse<DT><<<(nnz_x + 255) / 256, 256, 0, st>>>(d, x_idx, semiring == DBSPMSPV_OR_AND ? nullptr : x_val, nnz_x, h->ropts.validate); ++h->kernel_launches; }
     OutSparse out{d.ws.y_acc, d.ws.y_hit8};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
-    if (nnz_x > 0 && d.n_entries > 0) { DBS_CUDA(launch_pdl(k_compute<DT, OutSparse>, grid, CTA, st, d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold)); ++h->kernel_launches; }
+    if (nnz_x > 0 && d.n_entries > 0) {
+        // (payload staging, MODE 2, is kept for the decode entry: its larger shared-memory
+        // footprint costs the push path more occupancy than staging gains on sparse x)
+        const int s = h->heavy_stage ? launch_compute<DT, OutSparse, 1>(h, out, h->ropts.th3, true, st)
+                                     : launch_compute<DT, OutSparse, 0>(h, out, h->ropts.th3, true, st);
+        if (s != DBSPMSPV_OK) return s;
+    }
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
     h->kernel_launches += 2;
     const int nt = d.ws.n_tiles;
-    DBS_CUDA(launch_pdl(k_compact_count, nt, CMP_TPB, st, d));
+    DBS_CUDA(launch_pdl(k_compact_count, nt, CMP_TPB, 0, st, d));
     int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
     if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
-    DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, st, d, y_idx, y_val, y_capacity, y_nnz,
+    DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, 0, st, d, y_idx, y_val, y_capacity, y_nnz,
                         (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x));
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
@@ -809,8 +897,6 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
 template <int DT>
 static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStream_t st) {
     const Device &d = h->d;
-    static int grid = 0;
-    if (!grid) grid = compute_grid<DT, OutDense>(h->sm_count);
     const int64_t padded = (int64_t)((d.nb + 1) / 2) * 32;
     int64_t work = padded > d.m ? padded : d.m;
     int g = (int)((work + 255) / 256);
@@ -818,7 +904,11 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
     k_xblock_dense<DT><<<g, 256, 0, st>>>(d, x, y);
     OutDense out{y, nullptr};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
-    if (d.n_entries > 0) { k_compute<DT, OutDense><<<grid, CTA, 0, st>>>(d, out, h->ropts.th3, h->ropts.force_path, h->ropts.popc_threshold); ++h->kernel_launches; }
+    if (d.n_entries > 0) {
+        const int s = h->heavy_stage ? launch_compute<DT, OutDense, 2>(h, out, h->ropts.th3_decode, false, st)
+                                     : launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, false, st);
+        if (s != DBSPMSPV_OK) return s;
+    }
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
     h->kernel_launches += 2;
     int gc = ((d.nb + 1) / 2 + 255) / 256;
@@ -837,6 +927,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     *o = dbspmspv_run_opts();
     o->th3 = 0.9f;
     o->th3_bfs = 0.01f;
+    o->th3_decode = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;
     o->popc_threshold = 8;
     o->validate = 0;
@@ -845,7 +936,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
 int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts) {
     if (!h || !opts) return DBSPMSPV_ERR_INVALID_ARG;
     if (opts->force_path < DBSPMSPV_PATH_AUTO || opts->force_path > DBSPMSPV_PATH_PULL) return DBSPMSPV_ERR_INVALID_ARG;
-    if (!(opts->th3 >= 0.f) || !(opts->th3_bfs >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!(opts->th3 >= 0.f) || !(opts->th3_bfs >= 0.f) || !(opts->th3_decode >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
     h->ropts = *opts;
     return DBSPMSPV_OK;
 }
