@@ -119,34 +119,45 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
         const bool whole = seg.count < 0;
         const int end = seg.start + (seg.count & 0x7FFFFFFF);
         uint32_t hit = 0;
-        for (int base = seg.start; base < end; base += 32) {
-            const int p = base + lane;
-            bool heavy = false;
-            uint32_t idx = 0, w = 0, aux = 0, xm = 0;
-            if (p < end) {
-                idx = d.csr.idx[p];
-                xm = mask_of(d.ws.x_mask32, idx & IDX_MASK);
-                if (xm) {
-                    w = d.csr.w[p]; aux = d.csr.aux[p];
-                    const int type = idx >> TYPE_SHIFT;
-                    if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX))
-                        hit |= lane_block_bool<DT>(type, w, aux, xm, d.payload);
+        // up to four warp steps of view entries are fetched at once, then their frontier masks,
+        // so that every lane keeps several independent loads in flight
+        constexpr int U = 4;
+        bool done = false;
+        for (int base = seg.start; base < end && !done; base += 32 * U) {
+            uint32_t idx[U], w[U], aux[U], xm[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int p = base + u * 32 + lane;
+                idx[u] = 0; w[u] = 0; aux[u] = 0;
+                if (p < end) { idx[u] = d.csr.idx[p]; w[u] = d.csr.w[p]; aux[u] = d.csr.aux[p]; }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                xm[u] = base + u * 32 + lane < end ? mask_of(d.ws.x_mask32, idx[u] & IDX_MASK) : 0u;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (base + u * 32 >= end) break;
+                bool heavy = false;
+                if (xm[u]) {
+                    const int type = idx[u] >> TYPE_SHIFT;
+                    if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX))
+                        hit |= lane_block_bool<DT>(type, w[u], aux[u], xm[u], d.payload);
                     else
                         heavy = true;
                 }
+                uint32_t hv = __ballot_sync(FULL, heavy);
+                while (hv) {
+                    const int src = __ffs(hv) - 1;
+                    hv &= hv - 1;
+                    const uint32_t bidx = __shfl_sync(FULL, idx[u], src);
+                    const uint32_t bw = __shfl_sync(FULL, w[u], src);
+                    const int nnz = (int)__shfl_sync(FULL, aux[u], src) + 1;
+                    const uint32_t bxm = __shfl_sync(FULL, xm[u], src);
+                    hit |= warp_block_bool<DT>(bidx >> TYPE_SHIFT, d.payload + (size_t)bw * 4, nnz, bxm, lane);
+                }
+                hit = __reduce_or_sync(FULL, hit);
+                if ((hit & need) == need) { done = true; break; }
             }
-            uint32_t hv = __ballot_sync(FULL, heavy);
-            while (hv) {
-                const int src = __ffs(hv) - 1;
-                hv &= hv - 1;
-                const uint32_t bidx = __shfl_sync(FULL, idx, src);
-                const uint32_t bw = __shfl_sync(FULL, w, src);
-                const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
-                const uint32_t bxm = __shfl_sync(FULL, xm, src);
-                hit |= warp_block_bool<DT>(bidx >> TYPE_SHIFT, d.payload + (size_t)bw * 4, nnz, bxm, lane);
-            }
-            hit = __reduce_or_sync(FULL, hit);
-            if ((hit & need) == need) break;
         }
         hit &= need;
         if (hit) {
