@@ -99,6 +99,25 @@ def clocks_summary(samples: list) -> dict:
             "reasons": reasons, "samples": len(samples)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Max of a per-rank time over all ranks (the whole job is as slow as its slowest rank);
+    identity without a process group.  Works on NCCL (device tensor) and gloo (CPU tensor)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(units_per_rank: float, ms_per_step_local: float, world: int, device=None):
+    """Whole-job throughput of independent replicas: every rank processes `units_per_rank`
+    per step, the step takes the max over ranks.  Returns (units per second, ms)."""
+    ms = max_over_ranks(ms_per_step_local, device)
+    return world * units_per_rank / (ms * 1e-3), ms
+
+
 def measured_peak_gbs():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -282,11 +301,7 @@ def main() -> None:
 
     call_ms = np.array([[ev[s][k][0].elapsed_time(ev[s][k][1]) for k in range(npts)] for s in range(args.steps)])
     step_ms = call_ms.sum(axis=1)
-    ms_per_step = float(step_ms.mean())
-    if world > 1:
-        t = torch.tensor([ms_per_step], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t.item())
+    ms_per_step = max_over_ranks(float(step_ms.mean()), dev)
 
     # ---- end to end through the same C-ABI call with HOST buffers
     e2e_ms = []
@@ -314,11 +329,7 @@ def main() -> None:
             d2h += 4 + 8 * kk
         if s >= 2:
             e2e_ms.append(tot)
-    e2e_ms_step = float(np.mean(e2e_ms))
-    if world > 1:
-        t = torch.tensor([e2e_ms_step], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms_step = float(t.item())
+    e2e_ms_step = max_over_ranks(float(np.mean(e2e_ms)), dev)
 
     peak, peak_kind = measured_peak_gbs()
     sweep, b_touch_total = [], 0.0
@@ -360,6 +371,7 @@ def main() -> None:
             "sweep": sweep, "wall_s_timed_region": round(t_wall, 3)}
 
     if rank == 0 and world == 1:
+        line["cusparse_spmv_reference"] = cusparse_reference(a, torch, dev, flush)
         line["cpu_baseline"] = cpu_baseline(a, xs, model)
     if rank == 0 and world == 1 and not args.no_bfs:
         try:
@@ -428,6 +440,30 @@ def crossover_table() -> None:
             tp, tl = timed(h, x, mat.m, B.PATH_PUSH), timed(h, x, mat.m, B.PATH_PULL)
             print(f"| {name} | {label} | {sb:.4f} | {tp:.1f} | {tl:.1f} | {'push' if tp < tl else 'pull'} |")
         B.dbspmspv_destroy(h)
+
+
+def cusparse_reference(a, torch, dev, flush):
+    """Same-box library reference: CSR SpMV on x densified to length n (torch's sparse CSR
+    matmul, which calls cuSPARSE).  One time serves every sweep point: a dense x makes the
+    library read the whole matrix whatever x holds.  Harness only; the library never links it."""
+    try:
+        A = torch.sparse_csr_tensor(torch.from_numpy(a.row_ptr).to(dev), torch.from_numpy(a.col_idx.astype(np.int64)).to(dev),
+                                    torch.from_numpy(a.val).to(dev), size=(a.m, a.n))
+        xd = torch.zeros(a.n, 1, dtype=torch.float32, device=dev)
+        xd[:: 7] = 1.0
+        ts = []
+        for it in range(13):
+            flush.fill_(it)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            y = A @ xd
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return {"us": round(float(np.median(ts[3:])), 2), "what": "torch sparse CSR (cuSPARSE) SpMV, fp32, dense x, cold L2",
+                "csr_bytes": int(a.nnz * 8 + (a.m + 1) * 8)}
+    except Exception as e:
+        return {"error": repr(e)}
 
 
 def cpu_baseline(a, xs, model):
