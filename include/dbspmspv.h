@@ -87,9 +87,11 @@ typedef struct {
     int32_t force_format;    /* DBSPMSPV_FORMAT_*: ablation knob (Section 5.4)               */
     int32_t input_on_host;   /* 1: the create arrays are HOST pointers (copied once)         */
     int32_t inline_max;      /* valued matrices: a block with at most this many entries keeps
-                                them in its view entries, one entry per element       (8)    */
+                                them in its view entries, one entry per element      (31)    */
     int32_t w_inline;        /* ... of an INLINE view entry                         (1)      */
-    int32_t reserved[5];
+    int32_t w_dense_sparse;  /* Dense / CSR-like weights used instead when such blocks are a */
+    int32_t w_mid_sparse;    /* minority of the matrix (hypersparse matrices)  (128 / 64)    */
+    int32_t reserved[3];
 } dbspmspv_create_opts;
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */

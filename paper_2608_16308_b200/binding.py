@@ -36,7 +36,8 @@ class CreateOpts(ctypes.Structure):
                 ("seg_cut", ctypes.c_int32), ("w_dense", ctypes.c_int32), ("w_mid", ctypes.c_int32),
                 ("w_coo", ctypes.c_int32), ("force_format", ctypes.c_int32),
                 ("input_on_host", ctypes.c_int32), ("inline_max", ctypes.c_int32),
-                ("w_inline", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
+                ("w_inline", ctypes.c_int32), ("w_dense_sparse", ctypes.c_int32),
+                ("w_mid_sparse", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
 
 
 class RunOpts(ctypes.Structure):

@@ -577,9 +577,21 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         tp.release(k2); tp.release(k2_alt); tp.release(ids); tp.release(ids_alt); tp.release(bcol_sorted);
     }
 
-    // pull segments
+    // class census -> which kernel variant the handle uses, hence what a mask-based block costs
+    unsigned long long cls_h[2 * DBSPMSPV_BLK_NCLASS];
+    DBS_CUDA(cudaMemcpy(cls_h, cls, sizeof(cls_h), cudaMemcpyDeviceToHost));
     {
-        SegParams sp{h->copts.seg_cut, h->copts.w_dense, h->copts.w_mid, h->copts.w_coo, h->copts.w_inline};
+        unsigned long long heavy_nnz = 0;
+        for (int c = DBSPMSPV_BLK_FCSR; c <= DBSPMSPV_BLK_DENSE; ++c) heavy_nnz += cls_h[DBSPMSPV_BLK_NCLASS + c];
+        h->heavy_stage = heavy_nnz * 2 > (unsigned long long)nnzu;
+    }
+
+    // pull segments.  Where mask-based blocks are the bulk of the matrix the lanes of a warp each
+    // own one (cheap per block); where they are a minority a whole warp takes them one at a
+    // time, which costs about as much as a few hundred INLINE entries: the weights differ.
+    {
+        SegParams sp{h->copts.seg_cut, h->heavy_stage ? h->copts.w_dense : h->copts.w_dense_sparse,
+                     h->heavy_stage ? h->copts.w_mid : h->copts.w_mid_sparse, h->copts.w_coo, h->copts.w_inline};
         int32_t *cnt, *off;
         DBS_GET(cnt, (int64_t)d.mb + 1); DBS_GET(off, (int64_t)d.mb + 1);
         DBS_CUDA(cudaMemsetAsync(cnt, 0, ((size_t)d.mb + 1) * 4, st));
@@ -608,17 +620,10 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     }
 
     // statistics
-    unsigned long long cls_h[2 * DBSPMSPV_BLK_NCLASS];
-    DBS_CUDA(cudaMemcpy(cls_h, cls, sizeof(cls_h), cudaMemcpyDeviceToHost));
     dbspmspv_stats &s = h->stats;
     s.m = m; s.n = n; s.nnz = nnzu; s.n_blocks = n_blocks;
     for (int c = 0; c < DBSPMSPV_BLK_NCLASS; ++c) { s.class_blocks[c] = (int64_t)cls_h[c]; s.class_nnz[c] = (int64_t)cls_h[DBSPMSPV_BLK_NCLASS + c]; }
     s.n_row_blocks = d.mb; s.n_col_blocks = d.nb; s.n_segments = d.n_segments;
-    {
-        int64_t heavy_nnz = 0;
-        for (int c = DBSPMSPV_BLK_FCSR; c <= DBSPMSPV_BLK_DENSE; ++c) heavy_nnz += s.class_nnz[c];
-        h->heavy_stage = heavy_nnz * 2 > nnzu;
-    }
     s.payload_bytes = h->payload_bytes;
     s.n_view_entries = d.n_entries;
     s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)d.n_entries * 9;
@@ -645,7 +650,7 @@ int create_common(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz, con
     dbspmspv_handle_s *h = new (std::nothrow) dbspmspv_handle_s();
     if (!h) return DBSPMSPV_ERR_ALLOC;
     if (opts) h->copts = *opts; else dbspmspv_default_create_opts(&h->copts);
-    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.seg_cut > MAX_SEG_ENTRIES || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 16) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
+    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.seg_cut > MAX_SEG_ENTRIES || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid_sparse < 1 || h->copts.w_dense_sparse < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 31) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
     dbspmspv_default_run_opts(&h->ropts);
     h->d.dtype = dtype;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return DBSPMSPV_ERR_CUDA; }
@@ -666,9 +671,10 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     *o = dbspmspv_create_opts();
     o->th0 = 32; o->th1 = 128; o->th2 = 2.0f;
     o->seg_cut = 128; o->w_dense = 16; o->w_mid = 8; o->w_coo = 4; o->w_inline = 1;
+    o->w_dense_sparse = 128; o->w_mid_sparse = 64;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
-    o->inline_max = 8;
+    o->inline_max = 31;
 }
 
 int dbspmspv_create_csr(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz,

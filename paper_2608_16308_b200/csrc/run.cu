@@ -12,7 +12,7 @@ namespace dbs {
 constexpr int CTA = 128;            // four warps per thread block (Section 3.3.2)
 constexpr int WARPS = CTA / 32;
 constexpr int CMP_TPB = 256;        // compaction: threads per tile
-constexpr int TILE_WORDS = CMP_TPB;  // one 32-bit mask word (two row blocks) per thread
+constexpr int TILE_WORDS = CMP_TPB / 4;  // a tile: 64 mask words = 2048 rows; placement uses 8 rows per thread
 
 // ------------------------------------------------------------------------------------------
 // Vector blocking (Section 3.2.2) fused with the push worklist (Section 3.3.2).
@@ -650,12 +650,12 @@ __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out
 // sorted.  Pass 1 counts per tile, pass 2 places the entries, clears the accumulator and the
 // masks it read, clears the vector-block state of this call's x, and rolls the counters over.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(CMP_TPB) k_compact_count(Device d) {
-    __shared__ int s_red[CMP_TPB / 32];
+__global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d) {
+    __shared__ int s_red[TILE_WORDS / 32];
     pdl_wait();
     pdl_launch_dependents();
     const int n_words = (d.mb + 1) / 2;
-    const int wi = blockIdx.x * CMP_TPB + threadIdx.x;
+    const int wi = blockIdx.x * TILE_WORDS + threadIdx.x;
     int c = 0;
     if (wi < n_words) {
         // 32 row flags (bytes, 0 or 1) -> one mask word; the flags are cleared for the next call
@@ -677,7 +677,7 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_count(Device d) {
     __syncthreads();
     if (threadIdx.x == 0) {
         int t = 0;
-        for (int k = 0; k < CMP_TPB / 32; ++k) t += s_red[k];
+        for (int k = 0; k < TILE_WORDS / 32; ++k) t += s_red[k];
         d.ws.tile_count[blockIdx.x] = t;
     }
 }
@@ -704,9 +704,13 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
         }
         __syncthreads();
         const int n_words = (d.mb + 1) / 2;
-        const int wi = blockIdx.x * CMP_TPB + threadIdx.x;     // one 32-row mask word per thread
+        // every thread owns 8 consecutive rows (a quarter of a mask word): two independent
+        // 16-byte loads fetch their accumulator entries, which are cleared and written out
+        const int wi = blockIdx.x * TILE_WORDS + (threadIdx.x >> 2);
+        const int sub = threadIdx.x & 3;
         const uint32_t word = wi < n_words ? d.ws.y_mask32[wi] : 0u;
-        const int c = __popc(word);
+        const uint32_t bits = (word >> (8 * sub)) & 0xFFu;
+        const int c = __popc(bits);
         int incl = c;
         for (int o = 1; o < 32; o <<= 1) {
             int t = __shfl_up_sync(FULL, incl, o);
@@ -717,22 +721,20 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
         __syncthreads();
         int wbase = s_base;
         for (int k = 0; k < warp; ++k) wbase += s_red[k];
-        // every lane owns one 32-row word: it fetches the 32 accumulator entries with eight
-        // independent 16-byte loads, clears them, and writes its run of result entries
-        if (word) {
-            float4 *acc4 = reinterpret_cast<float4 *>(d.ws.y_acc + (size_t)wi * 32);
-            float4 v4[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) v4[q] = acc4[q];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) acc4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (bits) {
+            const int row0 = wi * 32 + sub * 8;
+            float4 *acc4 = reinterpret_cast<float4 *>(d.ws.y_acc + row0);
+            float4 v4[2];
+            v4[0] = acc4[0]; v4[1] = acc4[1];
+            acc4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+            acc4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
             const float *v = reinterpret_cast<const float *>(v4);
             int64_t pos = (int64_t)wbase + incl - c;
 #pragma unroll
-            for (int bit = 0; bit < 32; ++bit) {
-                if ((word >> bit) & 1u) {
+            for (int bit = 0; bit < 8; ++bit) {
+                if ((bits >> bit) & 1u) {
                     if (pos < y_capacity) {
-                        y_idx[pos] = wi * 32 + bit;
+                        y_idx[pos] = row0 + bit;
                         if (y_val) y_val[pos] = boolean ? 1.0f : v[bit];
                     }
                     ++pos;
@@ -885,7 +887,7 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
     h->kernel_launches += 2;
     const int nt = d.ws.n_tiles;
-    DBS_CUDA(launch_pdl(k_compact_count, nt, CMP_TPB, 0, st, d));
+    DBS_CUDA(launch_pdl(k_compact_count, nt, TILE_WORDS, 0, st, d));
     int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
     if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
     DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, 0, st, d, y_idx, y_val, y_capacity, y_nnz,

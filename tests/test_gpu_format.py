@@ -20,7 +20,7 @@ def cpu_classify(rows, cols, dtype, th0=32, th1=128, th2=2.0):
     key, rows, cols = key[order], rows[order], cols[order]
     ub, start, cnt = np.unique(key, return_index=True, return_counts=True)
     cls = np.empty(ub.size, dtype=np.int32)
-    cap = 4 if dtype == B.PATTERN else 8   # pattern: four coordinates per entry; valued: inline_max
+    cap = 4 if dtype == B.PATTERN else 31  # pattern: four coordinates per entry; valued: inline_max
     for b in range(ub.size):
         n = cnt[b]
         if n < th0:
@@ -123,8 +123,16 @@ def test_export_equals_input_and_census(name, make, dtype):
 
 
 def test_every_class_occurs_in_mixed():
-    h = Handle(mixed_matrix(96, 112, 3), B.F32)
+    """With the packed-COO class enabled for small blocks (inline_max below th0) the planted
+    matrix exercises all six classes; with the default (every block under th0 inline) all but COO."""
+    o = B.default_create_opts()
+    o.inline_max = 4
+    h = Handle(mixed_matrix(96, 112, 3), B.F32, opts=o)
     assert all(h.stats.class_blocks[k] > 0 for k in range(6))
+    h.close()
+    h = Handle(mixed_matrix(96, 112, 3), B.F32)
+    assert h.stats.class_blocks[B.BLK_COO] == 0
+    assert all(h.stats.class_blocks[k] > 0 for k in range(6) if k != B.BLK_COO)
     h.close()
 
 
@@ -143,13 +151,16 @@ def test_threshold_edges():
         h.close()
         return c
     full = [(r, c) for r in range(16) for c in range(16)]
-    assert cls_of(full[:31]) == B.BLK_COO
     assert cls_of(full[:32]) in (B.BLK_FCSR, B.BLK_CSR, B.BLK_FCSC)
     assert cls_of(full[:128]) != B.BLK_DENSE
     assert cls_of(full[:129]) == B.BLK_DENSE
     assert cls_of(full[:1]) == B.BLK_INLINE
-    assert cls_of(full[:8]) == B.BLK_INLINE
-    assert cls_of(full[:9]) == B.BLK_COO
+    assert cls_of(full[:31]) == B.BLK_INLINE          # default inline_max = 31 = th0 - 1
+    o = B.default_create_opts()
+    o.inline_max = 8
+    h = Handle(_block(full[:9]), B.F32, opts=o)       # above inline_max, below th0 -> packed COO
+    assert h.export_blocks()[2][0] == B.BLK_COO
+    h.close()
     # 32 entries as two full rows: max row 16, max col 2 -> ForceCSR
     assert cls_of(full[:32]) == B.BLK_FCSR
     assert cls_of([(c, r) for r, c in full[:32]]) == B.BLK_FCSC

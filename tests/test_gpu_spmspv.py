@@ -33,10 +33,12 @@ MATS = [
 
 
 @pytest.mark.parametrize("name,make", MATS, ids=[m[0] for m in MATS])
-@pytest.mark.parametrize("dtype", [B.F32, B.BF16])
-def test_parity_all_paths(name, make, dtype):
+@pytest.mark.parametrize("dtype,inline_max", [(B.F32, 31), (B.BF16, 31), (B.F32, 4), (B.BF16, 2)])
+def test_parity_all_paths(name, make, dtype, inline_max):
     csr = make()
-    h = Handle(csr, dtype)
+    o = B.default_create_opts()
+    o.inline_max = inline_max          # below th0 - 1 the packed-COO class comes into play
+    h = Handle(csr, dtype, opts=o)
     A = ref_matrix(csr, bf16=dtype == B.BF16)
     for frac in (0.002, 0.05, 0.5, 1.0):
         x = dense_x(csr.n, 7, frac)
