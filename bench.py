@@ -426,7 +426,7 @@ def crossover_table() -> None:
     cases.append(("uniform 16384^2, 8/row", a, [("164 nnz", wl.sparse_x(0, 1, a.n, 164))] +
                   [(f"{f:g}", wl.sparse_x(40 + i, 0, a.n, int(a.n * f))) for i, f in enumerate((0.05, 0.2, 0.5, 1.0))]))
     a2 = wl.rmat(20, 16, seed=1)
-    fr = list(wl.RMAT_SWEEP) + [0.2, 0.3, 0.7, 1.0]
+    fr = list(wl.RMAT_SWEEP) + [0.03, 0.05, 0.2, 0.3, 0.7, 1.0]
     cases.append(("R-MAT scale 20", a2, [(f"{f:g}", wl.rmat_x(a2.n, f, k) if k < 6 else wl.sparse_x(200 + k, 0, a2.n, int(a2.n * f)))
                                          for k, f in enumerate(fr)]))
     a3 = wl.stencil27(160, seed=2)

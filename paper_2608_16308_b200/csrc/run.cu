@@ -927,7 +927,7 @@ extern "C" {
 void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
-    o->th3 = 0.9f;
+    o->th3 = 0.65f;
     o->th3_bfs = 0.01f;
     o->th3_decode = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;
