@@ -52,7 +52,6 @@ constexpr int TYPE_SHIFT = 29;
 #endif
 constexpr int PUSH_CHUNK = DBS_PUSH_CHUNK;   // CSC-view entries per push task (32 per warp step)
 constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-class block
-constexpr int PAY_CAP = 8192;               // bytes of block payload one warp stages at a time
 
 // Payload size in 4-byte words; every block is padded to 16 bytes so that it can be moved with
 // one bulk copy.  vsize = bytes per value (4 fp32, 2 bf16, 0 pattern).
@@ -155,7 +154,7 @@ struct dbspmspv_handle_s {
     void *payload_alloc;
     int64_t payload_bytes;
     int bfs_grid;               // co-resident grid size of the BFS kernel
-    bool heavy_stage;           // most stored elements sit in mask-based blocks: pull stages payloads
+    bool heavy_stage;           // most stored elements sit in mask-based blocks: MODE 1 kernels
     cudaEvent_t ev[2];          // optional timing of the traversal kernel (run_opts.timing)
     bool timed;
     int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)

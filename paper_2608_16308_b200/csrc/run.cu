@@ -346,22 +346,16 @@ __device__ __forceinline__ void pull_issue(const Device &d, int e0, int e1, Pull
     }
 }
 
-template <int DT, typename Out, bool HV, bool HS>
+template <int DT, typename Out, bool HV>
 __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp,
-                          float *s_y, float *s_lacc, PullWarp *pw, uint8_t *s_pay, uint64_t *pay_bar) {
+                          float *s_y, float *s_lacc, PullWarp *pw) {
     const int lane = threadIdx.x & 31;
     const uint32_t le_mask = 0xFFFFFFFFu >> (31 - lane);
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
-    if (lane == 0) {
-        mbar_init(&pw->bar[0], 1); mbar_init(&pw->bar[1], 1);
-        if (HS) mbar_init(pay_bar, 1);
-        fence_barrier_init();
-    }
+    if (lane == 0) { mbar_init(&pw->bar[0], 1); mbar_init(&pw->bar[1], 1); fence_barrier_init(); }
     if (lane < 16) s_y[lane] = 0.f;
     __syncwarp();
-    uint32_t pay_parity = 0u;
-    bool failed = false;              // a bounded wait ran out: stop, report, leave cleanly
     uint32_t parity = 0u;             // bit s: phase parity of stage s
     int cur = 0;
     bool next_in_flight = false;
@@ -390,7 +384,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
         const PullStage *st = &pw->stage[cur];
         int cur_rb = -1;                  // row block held in the shared accumulator
         uint32_t hit = 0;
-        for (int base = e0; base < e1 && !failed; base += 32 * PULL_UNROLL) {
+        for (int base = e0; base < e1; base += 32 * PULL_UNROLL) {
             uint32_t idx[PULL_UNROLL], w[PULL_UNROLL], aux[PULL_UNROLL];
             float xin[PULL_UNROLL];
 #pragma unroll
@@ -480,81 +474,64 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                     if (Out::MASKS && coo_cnt && s_hit[lane]) mark_rows(out.hit8, rb, s_hit[lane]);
                     __syncwarp();
                 }
+                // runs of column-mask blocks (pruned layers): half-warp streaming form
+                if (HV && DT != DBSPMSPV_PATTERN) {
+                    const bool colmask = heavy && (type == DBSPMSPV_BLK_FCSC || type == DBSPMSPV_BLK_CSR || type == DBSPMSPV_BLK_DENSE);
+                    const uint32_t cs = __ballot_sync(FULL, colmask);
+                    if (__popc(cs) >= HEAVY_LANE_MIN) {
+                        half_stream<DT>(d.payload, d.ws.x_dense, idx[u], w[u], xm, rb, cs, lane,
+                                        [&](int erb, int erow, float esum) {
+                                            if (erb == cur_rb) {
+                                                atomicAdd(&s_y[erow], esum);
+                                                hit |= 1u << erow;
+                                            } else {
+                                                atomicAdd(out.acc + (size_t)erb * 16 + erow, esum);
+                                                if (Out::MASKS) out.hit8[(size_t)erb * 16 + erow] = 1;
+                                            }
+                                        });
+                        if (colmask) heavy = false;
+                        __syncwarp();
+                    }
+                }
                 uint32_t hv = __ballot_sync(FULL, heavy);
                 // sparse local mask -> lane-owned form; dense local mask -> warp form
                 const bool lane_form = heavy && type != DBSPMSPV_BLK_COO && __popc(xm) < popc_threshold;
                 const uint32_t hv_mask = HV ? __ballot_sync(FULL, lane_form) : 0u;
-                if (HV && ((HS && hv_mask) || __popc(hv_mask) >= HEAVY_LANE_MIN)) {
-                    // Mask-based blocks side by side (layers of a pruned model, banded matrices):
-                    // every lane walks its own block and leaves 16 partial sums in its private
-                    // scratch column, so the warp keeps up to 32 blocks going.  Blocks of the row
-                    // block held in the shared accumulator are then summed across lanes by 16
-                    // lanes (no atomics); blocks of other row blocks go straight to global.
-                    // HS variant (matrices made of such blocks): the payloads of the touched
-                    // blocks are first staged in shared memory by bulk copies, one per block,
-                    // issued by the lane that holds the block (Section 3.3.3), in groups that fit
-                    // the stage, and the lanes then read their block from shared memory.
-                    const bool mine = lane_form;
+                if (HV && __popc(hv_mask) >= HEAVY_LANE_MIN) {
+                    // Mask-based blocks side by side under sparse local masks (banded matrices at
+                    // run ends): every lane walks its own block and leaves 16 partial sums in its
+                    // private scratch column, so the warp keeps up to 32 blocks going.  Blocks of
+                    // the row block held in the shared accumulator are then summed across lanes
+                    // by 16 lanes (no atomics); blocks of other row blocks go straight to global.
                     float *acc = s_lacc + lane;
-                    int bytes = 0, incl = 0;
-                    if (HS) {
-                        bytes = mine ? payload_words(type, (int)aux[u] + 1, Val<DT>::SIZE) * 4 : 0;
-                        incl = bytes;
-                        for (int o = 1; o < 32; o <<= 1) {
-                            const int t = __shfl_up_sync(FULL, incl, o);
-                            if (lane >= o) incl += t;
-                        }
-                    }
-                    const int off = incl - bytes;
-                    uint32_t remaining = hv_mask;
-                    while (remaining) {
-                        uint32_t grp = remaining;
+                    uint32_t hits = 0;
+                    if (lane_form) {
                         const uint8_t *blk = d.payload + (size_t)w[u] * 4;
-                        if (HS) {
-                            const int gbase = __shfl_sync(FULL, off, __ffs(remaining) - 1);
-                            const bool fits = ((remaining >> lane) & 1u) && (incl - gbase <= PAY_CAP);
-                            grp = __ballot_sync(FULL, fits);
-                            const int total = __shfl_sync(FULL, incl, 31 - __clz(grp)) - gbase;
-                            fence_proxy_async_smem();
-                            __syncwarp();
-                            if (lane == __ffs(grp) - 1) mbar_arrive_expect_tx(pay_bar, (uint32_t)total);
-                            __syncwarp();
-                            if (fits) bulk_copy_g2s(s_pay + (off - gbase), blk, (uint32_t)bytes, pay_bar);
-                            blk = s_pay + (off - gbase);
-                        }
-                        const bool in_grp = (grp >> lane) & 1u;
-                        if (in_grp && DT != DBSPMSPV_PATTERN) {
+                        if (DT == DBSPMSPV_PATTERN) {
+                            hits = lane_heavy_bool(type, blk, xm);
+                        } else {
 #pragma unroll
                             for (int r = 0; r < 16; ++r) acc[r * LANE_ACC_STRIDE] = 0.f;
+                            hits = lane_heavy<DT>(type, blk, xm, d.ws.x_dense + (size_t)bcol_l * 16, acc);
                         }
-                        if (HS) {
-                            if (!mbar_wait_bounded(pay_bar, pay_parity)) { failed = true; break; }
-                            pay_parity ^= 1u;
-                        }
-                        uint32_t hits = 0;
-                        if (in_grp)
-                            hits = DT == DBSPMSPV_PATTERN ? lane_heavy_bool(type, blk, xm)
-                                                          : lane_heavy<DT>(type, blk, xm, d.ws.x_dense + (size_t)bcol_l * 16, acc);
-                        const bool in_cur = in_grp && rb == cur_rb;
-                        const uint32_t members = __ballot_sync(FULL, in_cur);
-                        __syncwarp();
-                        if (in_cur) hit |= hits;
-                        if (DT != DBSPMSPV_PATTERN && members && lane < 16) {
-                            float t = 0.f;
-                            for (uint32_t mm = members; mm; mm &= mm - 1) t += s_lacc[lane * LANE_ACC_STRIDE + __ffs(mm) - 1];
-                            s_y[lane] += t;
-                        }
-                        if (in_grp && !in_cur) {
-                            for (uint32_t hh = hits; hh; hh &= hh - 1) {
-                                const int r = __ffs(hh) - 1;
-                                if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)rb * 16 + r, acc[r * LANE_ACC_STRIDE]);
-                                if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
-                            }
-                        }
-                        remaining &= ~grp;
-                        __syncwarp();
                     }
-                    if (failed) break;
+                    const bool in_cur = lane_form && rb == cur_rb;
+                    const uint32_t members = __ballot_sync(FULL, in_cur);
+                    __syncwarp();
+                    if (in_cur) hit |= hits;
+                    if (DT != DBSPMSPV_PATTERN && members && lane < 16) {
+                        float t = 0.f;
+                        for (uint32_t mm = members; mm; mm &= mm - 1) t += s_lacc[lane * LANE_ACC_STRIDE + __ffs(mm) - 1];
+                        s_y[lane] += t;
+                    }
+                    if (lane_form && !in_cur) {
+                        for (uint32_t hh = hits; hh; hh &= hh - 1) {
+                            const int r = __ffs(hh) - 1;
+                            if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)rb * 16 + r, acc[r * LANE_ACC_STRIDE]);
+                            if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
+                        }
+                    }
+                    __syncwarp();
                     hv &= ~hv_mask;
                 }
                 while (hv) {
@@ -582,7 +559,6 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                 }
             }
         }
-        if (failed) { d.ws.ctr->status = DBSPMSPV_ERR_TIMEOUT; break; }
         // end of the chunk: flush what the shared accumulator still holds
         hit = __reduce_or_sync(FULL, hit);
         __syncwarp();
@@ -600,7 +576,6 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
     // left early on a timeout: let the copy still in flight land before the stage memory is
     // given back (bounded, like every wait here)
     if (next_in_flight) mbar_wait_bounded(&pw->bar[cur ^ 1], (parity >> (cur ^ 1)) & 1u);
-    if (HS && failed) mbar_wait_bounded(pay_bar, pay_parity);
 }
 
 // Global selector (Section 3.3.1): s_b = N_nzblk / N_blk; push iff s_b < th3.  Evaluated on
@@ -615,25 +590,22 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
 #define DBS_MIN_CTAS 1
 #endif
 // Variants of the traversal kernel, chosen per handle from the class census at create:
-//   MODE 0  hypersparse matrices (power-law graphs): no lane-owned code, smallest footprint
-//   MODE 1  matrices whose elements sit mostly in mask-based blocks: lane-owned microkernels
-//   MODE 2  the same plus payload staging in shared memory (used by the decode entry)
-// Dynamic shared memory: per-warp pull stages | lane scratch (MODE >= 1) | payload stage and
-// its barrier (MODE 2).
+//   MODE 0  hypersparse matrices (power-law graphs): no lane-owned / streaming code, smallest
+//           footprint
+//   MODE 1  matrices whose elements sit mostly in mask-based blocks (pruned layers, banded
+//           matrices): half-warp streaming and lane-owned microkernels
+// Dynamic shared memory: per-warp pull stages | lane scratch of the lane-owned form (MODE 1).
 template <int MODE> constexpr size_t compute_dyn_smem() {
-    return WARPS * sizeof(PullWarp) + (MODE >= 1 ? WARPS * 16 * LANE_ACC_STRIDE * sizeof(float) : 0) +
-           (MODE == 2 ? WARPS * (size_t)PAY_CAP + WARPS * sizeof(uint64_t) : 0);
+    return WARPS * sizeof(PullWarp) + (MODE >= 1 ? WARPS * 16 * LANE_ACC_STRIDE * sizeof(float) : 0);
 }
 
 template <int DT, typename Out, int MODE>
 __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
-    constexpr bool HV = MODE >= 1, HS = MODE == 2;
+    constexpr bool HV = MODE >= 1;
     __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16];
     extern __shared__ __align__(128) uint8_t s_dyn[];
     PullWarp *s_pull = reinterpret_cast<PullWarp *>(s_dyn);
     float *s_lacc = reinterpret_cast<float *>(s_dyn + WARPS * sizeof(PullWarp));
-    uint8_t *s_pay = reinterpret_cast<uint8_t *>(s_lacc + WARPS * 16 * LANE_ACC_STRIDE);
-    uint64_t *s_pay_bar = reinterpret_cast<uint64_t *>(s_pay + WARPS * (size_t)PAY_CAP);
     const int warp = threadIdx.x >> 5;
     pdl_wait();
     pdl_launch_dependents();
@@ -641,8 +613,7 @@ __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
     float *lacc = HV ? s_lacc + warp * 16 * LANE_ACC_STRIDE : nullptr;
     if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], lacc);
-    else pull_body<DT, Out, HV, HS>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], lacc, &s_pull[warp],
-                                    HS ? s_pay + warp * (size_t)PAY_CAP : nullptr, HS ? s_pay_bar + warp : nullptr);
+    else pull_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], lacc, &s_pull[warp]);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -878,8 +849,6 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     OutSparse out{d.ws.y_acc, d.ws.y_hit8};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
     if (nnz_x > 0 && d.n_entries > 0) {
-        // (payload staging, MODE 2, is kept for the decode entry: its larger shared-memory
-        // footprint costs the push path more occupancy than staging gains on sparse x)
         const int s = h->heavy_stage ? launch_compute<DT, OutSparse, 1>(h, out, h->ropts.th3, true, st)
                                      : launch_compute<DT, OutSparse, 0>(h, out, h->ropts.th3, true, st);
         if (s != DBSPMSPV_OK) return s;
@@ -907,7 +876,7 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
     OutDense out{y, nullptr};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
     if (d.n_entries > 0) {
-        const int s = h->heavy_stage ? launch_compute<DT, OutDense, 2>(h, out, h->ropts.th3_decode, false, st)
+        const int s = h->heavy_stage ? launch_compute<DT, OutDense, 1>(h, out, h->ropts.th3_decode, false, st)
                                      : launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, false, st);
         if (s != DBSPMSPV_OK) return s;
     }
