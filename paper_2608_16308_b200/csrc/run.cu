@@ -11,6 +11,7 @@ namespace dbs {
 
 constexpr int CTA = 128;            // four warps per thread block (Section 3.3.2)
 constexpr int WARPS = CTA / 32;
+constexpr int XB_TPB = 512;         // vector blocking of a sparse x: threads per block
 constexpr int CMP_TPB = 256;        // compaction: threads per tile
 constexpr int TILE_WORDS = CMP_TPB / 4;  // a tile: 64 mask words = 2048 rows; placement uses 8 rows per thread
 
@@ -19,8 +20,8 @@ constexpr int TILE_WORDS = CMP_TPB / 4;  // a tile: 64 mask words = 2048 rows; p
 // Sparse input: one thread per listed nonzero scatters the value into the dense copy and sets
 // its mask bit; the thread that turns a vector block from empty to nonempty emits the block's
 // push tasks (runs of <= 32 entries of its block-CSC column).  Space in the worklist is
-// claimed with one warp scan and one atomic per warp; the count of nonempty vector blocks is
-// aggregated the same way (Section 4.1).
+// claimed with a warp scan, a sum over the thread block's warps and one atomic per thread
+// block; the count of nonempty vector blocks is aggregated the same way (Section 4.1).
 // ------------------------------------------------------------------------------------------
 template <int DT>
 __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, const void *__restrict__ x_val,
@@ -49,7 +50,7 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
             jb = j >> 4;
         }
     }
-    emit_tasks(d, newly, jb, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+    emit_tasks<true>(d, newly, jb, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
 }
 
 // Dense input (Sections 4.1, 4.3): every warp reads 32 elements, one ballot gives the two
@@ -331,6 +332,10 @@ struct PullWarp {
 #define DBS_PULL_UNROLL 2
 #endif
 constexpr int PULL_UNROLL = DBS_PULL_UNROLL;
+#ifndef DBS_SY_COPIES
+#define DBS_SY_COPIES 4
+#endif
+constexpr int SY_COPIES = DBS_SY_COPIES;  // copies of the pull accumulator per warp (power of two, <= 32)
 constexpr uint32_t SEG_FLAG = 1u << 28;   // view entry starts a pull segment (block-CSR view only)
 
 // lane 0 issues the copies of the chunk [e0, e1) into stage st
@@ -354,7 +359,10 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
     if (lane == 0) { mbar_init(&pw->bar[0], 1); mbar_init(&pw->bar[1], 1); fence_barrier_init(); }
-    if (lane < 16) s_y[lane] = 0.f;
+    // the shared accumulator is kept in SY_COPIES copies, each fed by its own group of lanes:
+    // fewer lanes per address means fewer retries of the shared-memory fp32 atomic
+    for (int k = lane; k < 16 * SY_COPIES; k += 32) s_y[k] = 0.f;
+    float *const my_y = s_y + (lane / (32 / SY_COPIES)) * 16;
     __syncwarp();
     uint32_t parity = 0u;             // bit s: phase parity of stage s
     int cur = 0;
@@ -383,6 +391,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
         }
         const PullStage *st = &pw->stage[cur];
         int cur_rb = -1;                  // row block held in the shared accumulator
+        int last_rb = -1;                 // row block of segment ord_base
         uint32_t hit = 0;
         for (int base = e0; base < e1; base += 32 * PULL_UNROLL) {
             uint32_t idx[PULL_UNROLL], w[PULL_UNROLL], aux[PULL_UNROLL];
@@ -404,46 +413,55 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
             for (int u = 0; u < PULL_UNROLL; ++u) {
                 if (base + u * 32 >= e1) break;   // warp-uniform
                 const bool have = base + u * 32 + lane < e1;
-                const uint32_t fb = __ballot_sync(FULL, have && (idx[u] & SEG_FLAG));
-                const int ord = ord_base + __popc(fb & le_mask);
-                ord_base += __popc(fb);
-                const int rb = have ? d.seg_rb[ord] : 0;
+                const uint32_t fb = __ballot_sync(FULL, (idx[u] & SEG_FLAG) != 0u);   // idx is 0 past the end
+                // Most steps lie inside one segment (long row blocks are cut into segments of whole
+                // steps): then the row block is warp-uniform and known without a per-lane lookup.
+                const bool one_seg = (fb & ~1u) == 0u;
+                int rb, rb0;
+                if (one_seg) {
+                    if (fb) last_rb = d.seg_rb[++ord_base];
+                    rb = rb0 = last_rb;
+                } else {
+                    const int ord = ord_base + __popc(fb & le_mask);
+                    ord_base += __popc(fb);
+                    rb = have ? d.seg_rb[ord] : 0;
+                    rb0 = __shfl_sync(FULL, rb, 0);
+                    last_rb = __shfl_sync(FULL, rb, 31);   // (past the end only in the chunk's last step)
+                }
                 // the shared accumulator follows the row block of the step's first entry (a long
                 // row block keeps it over all its segments of the chunk)
-                const int rb0 = __shfl_sync(FULL, rb, 0);
                 if (rb0 != cur_rb) {
                     hit = __reduce_or_sync(FULL, hit);
                     __syncwarp();
                     if (lane < 16) {
                         if ((hit >> lane) & 1u) {
-                            if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+                            if (DT != DBSPMSPV_PATTERN) {
+                                float t = 0.f;
+#pragma unroll
+                                for (int k = 0; k < SY_COPIES; ++k) { t += s_y[k * 16 + lane]; s_y[k * 16 + lane] = 0.f; }
+                                atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, t);
+                            }
                             if (Out::MASKS) out.hit8[(size_t)cur_rb * 16 + lane] = 1;
                         }
-                        s_y[lane] = 0.f;
                     }
                     hit = 0;
                     cur_rb = rb0;
                     __syncwarp();
                 }
                 const int type = idx[u] >> TYPE_SHIFT;
-                bool other = false;
-                if (have) {
-                    if (type == DBSPMSPV_BLK_INLINE && DT != DBSPMSPV_PATTERN) {
-                        if (__float_as_uint(xin[u]) != X_ABSENT) {
-                            const float v = Val<DT>::inline_value(w[u]) * xin[u];
-                            const int r = aux[u] >> 4;
-                            if (rb == cur_rb) {
-                                atomicAdd(&s_y[r], v);
-                                hit |= 1u << r;
-                            } else {
-                                atomicAdd(out.acc + (size_t)rb * 16 + r, v);
-                                if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
-                            }
-                        }
+                const bool inl = type == DBSPMSPV_BLK_INLINE && DT != DBSPMSPV_PATTERN;
+                if (inl && __float_as_uint(xin[u]) != X_ABSENT) {    // absent also covers "past the end"
+                    const float v = Val<DT>::inline_value(w[u]) * xin[u];
+                    const int r = aux[u] >> 4;
+                    if (one_seg || rb == cur_rb) {
+                        atomicAdd(&my_y[r], v);
+                        hit |= 1u << r;
                     } else {
-                        other = true;
+                        atomicAdd(out.acc + (size_t)rb * 16 + r, v);
+                        if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
                     }
                 }
+                const bool other = have && !inl;
                 if (!__any_sync(FULL, other)) continue;
                 // classes that go through the vector-block mask; they write straight to global
                 const int bcol_l = idx[u] & IDX_MASK;
@@ -482,7 +500,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                         half_stream<DT>(d.payload, d.ws.x_dense, idx[u], w[u], xm, rb, cs, lane,
                                         [&](int erb, int erow, float esum) {
                                             if (erb == cur_rb) {
-                                                atomicAdd(&s_y[erow], esum);
+                                                atomicAdd(&my_y[erow], esum);
                                                 hit |= 1u << erow;
                                             } else {
                                                 atomicAdd(out.acc + (size_t)erb * 16 + erow, esum);
@@ -564,10 +582,14 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
         __syncwarp();
         if (lane < 16) {
             if ((hit >> lane) & 1u) {
-                if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, s_y[lane]);
+                if (DT != DBSPMSPV_PATTERN) {
+                    float t = 0.f;
+#pragma unroll
+                    for (int k = 0; k < SY_COPIES; ++k) { t += s_y[k * 16 + lane]; s_y[k * 16 + lane] = 0.f; }
+                    atomicAdd(out.acc + (size_t)cur_rb * 16 + lane, t);
+                }
                 if (Out::MASKS) out.hit8[(size_t)cur_rb * 16 + lane] = 1;
             }
-            s_y[lane] = 0.f;
         }
         __syncwarp();
         cur ^= 1;
@@ -602,7 +624,7 @@ template <int MODE> constexpr size_t compute_dyn_smem() {
 template <int DT, typename Out, int MODE>
 __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
     constexpr bool HV = MODE >= 1;
-    __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16];
+    __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16 * SY_COPIES];
     extern __shared__ __align__(128) uint8_t s_dyn[];
     PullWarp *s_pull = reinterpret_cast<PullWarp *>(s_dyn);
     float *s_lacc = reinterpret_cast<float *>(s_dyn + WARPS * sizeof(PullWarp));
@@ -656,65 +678,75 @@ __global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d) {
 __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__restrict__ y_idx, float *__restrict__ y_val,
                                                            int64_t y_capacity, int32_t *__restrict__ y_nnz, int boolean,
                                                            const int32_t *__restrict__ x_idx, int32_t nnz_x) {
-    __shared__ int s_red[CMP_TPB / 32];
-    __shared__ int s_base;
+    __shared__ int s_before[CMP_TPB / 32], s_cnt[CMP_TPB / 32];
+    __shared__ int32_t s_oidx[TILE_WORDS * 32];
+    __shared__ float s_oval[TILE_WORDS * 32];
     const int n_tiles = d.ws.n_tiles;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     pdl_wait();
+    // The kernel is a chain of dependent loads, not bandwidth: everything that can be fetched
+    // up front is fetched before the first barrier.
+    const int stride = gridDim.x * CMP_TPB;
+    const int k0 = blockIdx.x * CMP_TPB + threadIdx.x;
+    const int j0 = k0 < nnz_x ? x_idx[k0] : -1;
     if ((int)blockIdx.x < n_tiles) {
-        // entries in all earlier tiles
-        int before = 0;
-        for (int k = threadIdx.x; k < (int)blockIdx.x; k += CMP_TPB) before += d.ws.tile_count[k];
-        before = __reduce_add_sync(FULL, before);
-        if (lane == 0) s_red[warp] = before;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            int t = 0;
-            for (int k = 0; k < CMP_TPB / 32; ++k) t += s_red[k];
-            s_base = t;
-        }
-        __syncthreads();
         const int n_words = (d.mb + 1) / 2;
-        // every thread owns 8 consecutive rows (a quarter of a mask word): two independent
-        // 16-byte loads fetch their accumulator entries, which are cleared and written out
+        // every thread owns 8 consecutive rows (a quarter of a mask word)
         const int wi = blockIdx.x * TILE_WORDS + (threadIdx.x >> 2);
         const int sub = threadIdx.x & 3;
         const uint32_t word = wi < n_words ? d.ws.y_mask32[wi] : 0u;
+        int before = 0;               // entries in all earlier tiles
+        for (int k = threadIdx.x; k < (int)blockIdx.x; k += CMP_TPB) before += d.ws.tile_count[k];
         const uint32_t bits = (word >> (8 * sub)) & 0xFFu;
         const int c = __popc(bits);
+        const int row0 = wi * 32 + sub * 8;
+        float4 v4[2];
+        if (bits) {                   // two independent 16-byte loads fetch the 8 accumulator entries
+            float4 *acc4 = reinterpret_cast<float4 *>(d.ws.y_acc + row0);
+            v4[0] = acc4[0]; v4[1] = acc4[1];
+            acc4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+            acc4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         int incl = c;
         for (int o = 1; o < 32; o <<= 1) {
             int t = __shfl_up_sync(FULL, incl, o);
             if (lane >= o) incl += t;
         }
+        before = __reduce_add_sync(FULL, before);
+        if (lane == 31) s_cnt[warp] = incl;
+        if (lane == 0) s_before[warp] = before;
         __syncthreads();
-        if (lane == 31) s_red[warp] = incl;
-        __syncthreads();
-        int wbase = s_base;
-        for (int k = 0; k < warp; ++k) wbase += s_red[k];
+        int base = 0, local = 0, tile_total = 0;
+#pragma unroll
+        for (int k = 0; k < CMP_TPB / 32; ++k) {
+            base += s_before[k];
+            if (k < warp) local += s_cnt[k];
+            tile_total += s_cnt[k];
+        }
+        // the tile's entries are gathered in shared memory, then written out in whole lines
         if (bits) {
-            const int row0 = wi * 32 + sub * 8;
-            float4 *acc4 = reinterpret_cast<float4 *>(d.ws.y_acc + row0);
-            float4 v4[2];
-            v4[0] = acc4[0]; v4[1] = acc4[1];
-            acc4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-            acc4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
             const float *v = reinterpret_cast<const float *>(v4);
-            int64_t pos = (int64_t)wbase + incl - c;
+            int pos = local + incl - c;
 #pragma unroll
             for (int bit = 0; bit < 8; ++bit) {
                 if ((bits >> bit) & 1u) {
-                    if (pos < y_capacity) {
-                        y_idx[pos] = row0 + bit;
-                        if (y_val) y_val[pos] = boolean ? 1.0f : v[bit];
-                    }
+                    s_oidx[pos] = row0 + bit;
+                    s_oval[pos] = boolean ? 1.0f : v[bit];
                     ++pos;
                 }
             }
         }
-        if ((int)blockIdx.x == n_tiles - 1 && threadIdx.x == CMP_TPB - 1) {
+        __syncthreads();
+        for (int k = threadIdx.x; k < tile_total; k += CMP_TPB) {
+            const int64_t pos = (int64_t)base + k;
+            if (pos < y_capacity) {
+                y_idx[pos] = s_oidx[k];
+                if (y_val) y_val[pos] = s_oval[k];
+            }
+        }
+        if ((int)blockIdx.x == n_tiles - 1 && threadIdx.x == 0) {
             Counters *c2 = d.ws.ctr;
-            const int total = wbase + incl;
+            const int total = base + tile_total;
             *y_nnz = total;
             if (total > y_capacity) c2->status = DBSPMSPV_ERR_CAPACITY;
             c2->last_y_nnz = total;
@@ -725,10 +757,9 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
             c2->n_tasks = 0;
         }
     }
-    // vector-block state of this call's x: clear the masks (the dense copy may keep stale
-    // values; it is only ever read under a mask bit)
-    const int stride = gridDim.x * CMP_TPB;
-    for (int k = blockIdx.x * CMP_TPB + threadIdx.x; k < nnz_x; k += stride) {
+    // vector-block state of this call's x: clear the masks and put the "not listed" marker back
+    if (j0 >= 0 && j0 < d.n) { d.ws.x_mask32[j0 >> 5] = 0u; d.ws.x_dense[j0] = __uint_as_float(X_ABSENT); }
+    for (int k = k0 + stride; k < nnz_x; k += stride) {
         const int j = x_idx[k];
         if (j >= 0 && j < d.n) { d.ws.x_mask32[j >> 5] = 0u; d.ws.x_dense[j] = __uint_as_float(X_ABSENT); }
     }
@@ -845,7 +876,7 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
                      int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
                      cudaStream_t st) {
     const Device &d = h->d;
-    if (nnz_x > 0) { k_xblock_sparse<DT><<<(nnz_x + 255) / 256, 256, 0, st>>>(d, x_idx, semiring == DBSPMSPV_OR_AND ? nullptr : x_val, nnz_x, h->ropts.validate); ++h->kernel_launches; }
+    if (nnz_x > 0) { k_xblock_sparse<DT><<<(nnz_x + XB_TPB - 1) / XB_TPB, XB_TPB, 0, st>>>(d, x_idx, semiring == DBSPMSPV_OR_AND ? nullptr : x_val, nnz_x, h->ropts.validate); ++h->kernel_launches; }
     OutSparse out{d.ws.y_acc, d.ws.y_hit8};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
     if (nnz_x > 0 && d.n_entries > 0) {

@@ -7,10 +7,13 @@
 
 namespace dbs {
 
-// Called by a full warp.  Lanes with `newly` set own a vector block `jb` that has just become
-// nonempty; each appends that block's tasks.  Space is claimed with one warp scan and one
-// atomic per warp; the count of nonempty vector blocks is aggregated the same way
-// (hierarchical counting, Section 4.1).
+// Called by a full warp -- or, with CTA_WIDE, by every thread of the thread block.  Lanes with
+// `newly` set own a vector block `jb` that has just become nonempty; each appends that block's
+// tasks.  Space is claimed hierarchically (Section 4.1): a warp scan, then either one atomic per
+// warp or -- CTA_WIDE -- a sum over the block's warps in shared memory and one atomic per thread
+// block (thousands of warps queueing on one counter serialise in L2 otherwise).  The count of
+// nonempty vector blocks is aggregated the same way.
+template <bool CTA_WIDE = false>
 __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int lane,
                                            int32_t *n_tasks, int32_t *n_nzblk) {
     int first = 0, deg = 0;
@@ -27,7 +30,25 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
     const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
     const int n_new = __popc(__ballot_sync(0xFFFFFFFFu, newly));
     int base = 0;
-    if (lane == 0 && n_new) {
+    if (CTA_WIDE) {
+        __shared__ int s_tot[32], s_new[32], s_base;
+        const int warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+        if (lane == 0) { s_tot[warp] = total; s_new[warp] = n_new; }
+        __syncthreads();
+        if (warp == 0) {
+            const int t = lane < nw ? s_tot[lane] : 0, c = lane < nw ? s_new[lane] : 0;
+            const int tsum = __reduce_add_sync(0xFFFFFFFFu, t), csum = __reduce_add_sync(0xFFFFFFFFu, c);
+            if (lane == 0) {
+                s_base = tsum ? atomicAdd(n_tasks, tsum) : 0;
+                if (csum) atomicAdd(n_nzblk, csum);
+            }
+        }
+        __syncthreads();
+        if (lane == 0) {
+            base = s_base;
+            for (int k = 0; k < warp; ++k) base += s_tot[k];
+        }
+    } else if (lane == 0 && n_new) {
         if (total) base = atomicAdd(n_tasks, total);
         atomicAdd(n_nzblk, n_new);
     }
