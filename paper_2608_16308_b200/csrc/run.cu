@@ -677,7 +677,7 @@ __global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d) {
 
 __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__restrict__ y_idx, float *__restrict__ y_val,
                                                            int64_t y_capacity, int32_t *__restrict__ y_nnz, int boolean,
-                                                           const int32_t *__restrict__ x_idx, int32_t nnz_x) {
+                                                           const int32_t *__restrict__ x_idx, int32_t nnz_x, int clear_all) {
     __shared__ int s_before[CMP_TPB / 32], s_cnt[CMP_TPB / 32];
     __shared__ int32_t s_oidx[TILE_WORDS * 32];
     __shared__ float s_oval[TILE_WORDS * 32];
@@ -688,7 +688,7 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
     // up front is fetched before the first barrier.
     const int stride = gridDim.x * CMP_TPB;
     const int k0 = blockIdx.x * CMP_TPB + threadIdx.x;
-    const int j0 = k0 < nnz_x ? x_idx[k0] : -1;
+    const int j0 = (!clear_all && k0 < nnz_x) ? x_idx[k0] : -1;
     if ((int)blockIdx.x < n_tiles) {
         const int n_words = (d.mb + 1) / 2;
         // every thread owns 8 consecutive rows (a quarter of a mask word)
@@ -758,6 +758,16 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
         }
     }
     // vector-block state of this call's x: clear the masks and put the "not listed" marker back
+    // -- entry by entry, or, for an x that lists a good part of all columns, by streaming over
+    // the whole dense copy (full-line stores instead of scattered 4-byte ones)
+    if (clear_all) {
+        const int n_words = (d.nb + 1) / 2;
+        const uint32_t mk = X_ABSENT;
+        uint4 *xd4 = reinterpret_cast<uint4 *>(d.ws.x_dense);
+        for (int k = k0; k < n_words * 8; k += stride) xd4[k] = make_uint4(mk, mk, mk, mk);
+        for (int k = k0; k < n_words; k += stride) d.ws.x_mask32[k] = 0u;
+        return;
+    }
     if (j0 >= 0 && j0 < d.n) { d.ws.x_mask32[j0 >> 5] = 0u; d.ws.x_dense[j0] = __uint_as_float(X_ABSENT); }
     for (int k = k0 + stride; k < nnz_x; k += stride) {
         const int j = x_idx[k];
@@ -890,8 +900,9 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     DBS_CUDA(launch_pdl(k_compact_count, nt, TILE_WORDS, 0, st, d));
     int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
     if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
+    const int clear_all = (int64_t)nnz_x * 8 > d.n;     // scattered clears cost more than a full sweep
     DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, 0, st, d, y_idx, y_val, y_capacity, y_nnz,
-                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x));
+                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x, clear_all));
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }
