@@ -91,7 +91,11 @@ typedef struct {
     int32_t w_inline;        /* ... of an INLINE view entry                         (1)      */
     int32_t w_dense_sparse;  /* Dense / CSR-like weights used instead when such blocks are a */
     int32_t w_mid_sparse;    /* minority of the matrix (hypersparse matrices)  (128 / 64)    */
-    int32_t reserved[3];
+    int32_t th0_pattern;     /* pattern matrices: th0 used in place of th0 (32).  Lower values
+                                turn coordinate lists of th0_pattern..31 entries into 32-byte
+                                bit-mask blocks (measured slower for BFS on power-law graphs:
+                                four times the payload traffic)                              */
+    int32_t reserved[2];
 } dbspmspv_create_opts;
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */

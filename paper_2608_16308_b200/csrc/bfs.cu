@@ -23,9 +23,10 @@ __device__ __forceinline__ uint32_t lane_block_bool(int type, uint32_t w, uint32
     uint32_t hit = 0;
     if (type == DBSPMSPV_BLK_INLINE) {
         if (DT == DBSPMSPV_PATTERN) {
-            for (uint32_t k = 0; k <= aux; ++k) {
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) {      // up to four packed coordinates, no branch
                 const uint32_t rc = (w >> (8 * k)) & 0xFFu;
-                if ((xm >> (rc & 15)) & 1u) hit |= 1u << (rc >> 4);
+                hit |= (k <= aux ? (xm >> (rc & 15)) & 1u : 0u) << (rc >> 4);
             }
         } else if ((xm >> (aux & 15)) & 1u) {
             hit = 1u << (aux >> 4);
@@ -71,8 +72,11 @@ __device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int dept
                 const uint32_t need = ~mask_of(d.ws.visited32, brow) & 0xFFFFu;
                 if (need) {
                     w = d.csc.w[p]; aux = d.csc.aux[p];
-                    if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux < COO_SERIAL_MAX)) {
-                        const uint32_t hit = lane_block_bool<DT>(type, w, aux, xm, d.payload) & need;
+                    if (type != DBSPMSPV_BLK_COO || aux < COO_SERIAL_MAX) {
+                        // one lane per block: hypersparse blocks from their coordinates,
+                        // mask-based blocks from their 16 masks
+                        const uint32_t hit = need & (type <= DBSPMSPV_BLK_COO ? lane_block_bool<DT>(type, w, aux, xm, d.payload)
+                                                                             : lane_heavy_bool(type, d.payload + (size_t)w * 4, xm));
                         if (hit) {
                             const int sh = (brow & 1) * 16;
                             const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hit << sh);
@@ -111,10 +115,22 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    // the descriptor and the visited mask of the warp's next segment are fetched while the
+    // current one is processed (two of the four dependent loads per segment leave the chain)
+    Segment seg_n = Segment{0, 0, 0, 0};
+    uint32_t need_n = 0;
+    if (gwarp < d.n_segments) {
+        seg_n = d.segments[gwarp];
+        need_n = ~mask_of(d.ws.visited32, seg_n.row_block) & 0xFFFFu;
+    }
     for (int sg = gwarp; sg < d.n_segments; sg += nwarps) {
-        const Segment seg = d.segments[sg];
+        const Segment seg = seg_n;
+        const uint32_t need = need_n;
+        if (sg + nwarps < d.n_segments) {
+            seg_n = d.segments[sg + nwarps];
+            need_n = ~mask_of(d.ws.visited32, seg_n.row_block) & 0xFFFFu;
+        }
         const int rb = seg.row_block;
-        const uint32_t need = ~mask_of(d.ws.visited32, rb) & 0xFFFFu;
         if (!need) continue;
         const bool whole = seg.count < 0;
         const int end = seg.start + (seg.count & 0x7FFFFFFF);
@@ -140,10 +156,12 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
                 bool heavy = false;
                 if (xm[u]) {
                     const int type = idx[u] >> TYPE_SHIFT;
-                    if (type == DBSPMSPV_BLK_INLINE || (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX))
-                        hit |= lane_block_bool<DT>(type, w[u], aux[u], xm[u], d.payload);
-                    else
-                        heavy = true;
+                    if (type <= DBSPMSPV_BLK_COO) {
+                        if (type == DBSPMSPV_BLK_INLINE || aux[u] < COO_SERIAL_MAX) hit |= lane_block_bool<DT>(type, w[u], aux[u], xm[u], d.payload);
+                        else heavy = true;
+                    } else {
+                        hit |= lane_heavy_bool(type, d.payload + (size_t)w[u] * 4, xm[u]);
+                    }
                 }
                 uint32_t hv = __ballot_sync(FULL, heavy);
                 while (hv) {
@@ -173,6 +191,12 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
     }
 }
 
+// Per-level selector (Section 3.3.1): push iff N_nzblk / N_blk < th3.  Monotone in n_nzblk.
+__device__ __forceinline__ int bfs_path(int n_nzblk, int nb, float th3, int force_path) {
+    if (force_path == DBSPMSPV_PATH_PUSH || force_path == DBSPMSPV_PATH_PULL) return force_path;
+    return ((float)n_nzblk / (float)nb < th3) ? DBSPMSPV_PATH_PUSH : DBSPMSPV_PATH_PULL;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t *levels, float th3,
                                                  int force_path, int max_levels) {
@@ -184,7 +208,10 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
     Counters *ctr = d.ws.ctr;
 
     for (int64_t v = tid; v < d.n; v += nthreads) levels[v] = -1;
-    for (int k = tid; k < n_words; k += nthreads) { d.ws.visited32[k] = 0u; d.ws.x_mask32[k] = 0u; d.ws.y_mask32[k] = 0u; }
+    // rows without a stored element can never be reached through a pull: they start out as
+    // "visited", so that a row block is skipped (and a segment left early) once every row that
+    // can be found has been found
+    for (int k = tid; k < n_words; k += nthreads) { d.ws.visited32[k] = ~d.row_present32[k]; d.ws.x_mask32[k] = 0u; d.ws.y_mask32[k] = 0u; }
     if (tid == 0) { ctr->bfs_cnt[0][0] = 0; ctr->bfs_cnt[0][1] = 0; ctr->bfs_cnt[1][0] = 0; ctr->bfs_cnt[1][1] = 0; ctr->bfs_reached = 1; }
     grid.sync();
     // level 0: the source is the first frontier
@@ -194,7 +221,7 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
             levels[src] = 0;
             const uint32_t bit = 1u << ((src & 15) + (jb & 1) * 16);
             d.ws.x_mask32[jb >> 1] = bit;
-            d.ws.visited32[jb >> 1] = bit;
+            d.ws.visited32[jb >> 1] |= bit;
         }
         emit_tasks(d, lane == 0, jb, lane, &ctr->bfs_cnt[0][1], &ctr->bfs_cnt[0][0]);
     }
@@ -206,9 +233,7 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         const int n_tasks = ctr->bfs_cnt[cur][1];
         if (n_nzblk == 0) break;
         ++depth;
-        int path = force_path;
-        if (path != DBSPMSPV_PATH_PUSH && path != DBSPMSPV_PATH_PULL)
-            path = ((float)n_nzblk / (float)d.nb < th3) ? DBSPMSPV_PATH_PUSH : DBSPMSPV_PATH_PULL;
+        const int path = bfs_path(n_nzblk, d.nb, th3, force_path);
         if (tid == 0) {
             ctr->bfs_cnt[cur ^ 1][0] = 0;
             ctr->bfs_cnt[cur ^ 1][1] = 0;
@@ -221,7 +246,11 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         else bfs_pull<DT>(d, levels, depth);
         grid.sync();
         // next frontier: masks produced above become the vector-block masks of the next level;
-        // visited is updated; the push worklist and block statistics are rebuilt on the fly
+        // visited is updated; the push worklist and block statistics are rebuilt on the fly.
+        // The worklist is only needed if the next level is a push: the running count of nonempty
+        // blocks only grows, so once it has reached the selector's threshold the next level is
+        // known to be a pull and the remaining warps just count (a push is only ever chosen
+        // when no warp has skipped).
         int found = 0;
         for (int k0 = (tid & ~31); k0 < n_words; k0 += nthreads) {
             const int k = k0 + lane;
@@ -235,8 +264,17 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
                 }
                 if (nm || d.ws.x_mask32[k]) d.ws.x_mask32[k] = nm;
             }
-            emit_tasks(d, (nm & 0xFFFFu) != 0, 2 * k, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->bfs_cnt[cur ^ 1][0]);
-            emit_tasks(d, (nm >> 16) != 0, 2 * k + 1, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->bfs_cnt[cur ^ 1][0]);
+            const bool lo = (nm & 0xFFFFu) != 0, hi = (nm >> 16) != 0;
+            int seen = 0;     // read by one lane: the branch below must be warp-uniform
+            if (lane == 0) seen = *reinterpret_cast<volatile int32_t *>(&ctr->bfs_cnt[cur ^ 1][0]);
+            seen = __shfl_sync(FULL, seen, 0);
+            if (bfs_path(seen, d.nb, th3, force_path) == DBSPMSPV_PATH_PULL) {
+                const int nz = __popc(__ballot_sync(FULL, lo)) + __popc(__ballot_sync(FULL, hi));
+                if (lane == 0 && nz) atomicAdd(&ctr->bfs_cnt[cur ^ 1][0], nz);
+            } else {
+                emit_tasks(d, lo, 2 * k, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->bfs_cnt[cur ^ 1][0]);
+                emit_tasks(d, hi, 2 * k + 1, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->bfs_cnt[cur ^ 1][0]);
+            }
         }
         found = __reduce_add_sync(FULL, found);
         if (lane == 0 && found) atomicAdd(&ctr->bfs_reached, found);

@@ -63,6 +63,17 @@ __global__ void k_keys_from_coo(int64_t m, int64_t n, int64_t nnz, const int32_t
     src[e] = (uint32_t)e;
 }
 
+// rows that hold at least one stored element, as 16-bit masks per row block (two per word)
+__global__ void k_row_presence(int64_t nnzu, const uint64_t *ukey, uint32_t *row_present32) {
+    int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (e >= nnzu) return;
+    const uint64_t k = ukey[e];
+    const int64_t rb = (int64_t)(k >> 35);
+    const uint32_t bit = 1u << (((uint32_t)(k >> 4) & 15u) + (uint32_t)(rb & 1) * 16u);
+    uint32_t *word = row_present32 + (rb >> 1);
+    if (!(*word & bit)) atomicOr(word, bit);
+}
+
 // ---- step 2: merge duplicates, find block boundaries
 __global__ void k_flag_new_key(int64_t n, const uint64_t *keys, int shift, int32_t *flag) {
     int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
@@ -445,6 +456,11 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     d.m = m; d.n = n;
     d.mb = (int32_t)((m + B - 1) / B);
     d.nb = (int32_t)((n + B - 1) / B);
+    {
+        uint32_t *rp; DBS_KEEP(rp, (d.mb + 1) / 2);
+        d.row_present32 = rp;
+        DBS_CUDA(cudaMemsetAsync(rp, 0, (size_t)((d.mb + 1) / 2) * 4, st));
+    }
 
     // inputs on the host: copy once
     if (h->copts.input_on_host) {
@@ -490,6 +506,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         if (dt == DBSPMSPV_F32) k_merge_duplicates<DBSPMSPV_F32><<<grid_for(nnz), TPB, 0, st>>>(nnz, keys, src, flag, rank, val, ukey, uval);
         else if (dt == DBSPMSPV_BF16) k_merge_duplicates<DBSPMSPV_BF16><<<grid_for(nnz), TPB, 0, st>>>(nnz, keys, src, flag, rank, val, ukey, uval);
         else k_merge_duplicates<DBSPMSPV_PATTERN><<<grid_for(nnz), TPB, 0, st>>>(nnz, keys, src, flag, rank, val, ukey, uval);
+        k_row_presence<<<grid_for(nnzu), TPB, 0, st>>>(nnzu, ukey, const_cast<uint32_t *>(d.row_present32));
         DBS_CUDA(cudaStreamSynchronize(st));
         tp.release(keys); tp.release(src);
         k_flag_new_key<<<grid_for(nnzu), TPB, 0, st>>>(nnzu, ukey, 8, flag);
@@ -514,7 +531,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     DBS_GET(cls, 2 * DBSPMSPV_BLK_NCLASS);
     DBS_CUDA(cudaMemsetAsync(cls, 0, 2 * DBSPMSPV_BLK_NCLASS * sizeof(unsigned long long), st));
     DBS_CUDA(cudaMemsetAsync(ecount, 0, ((size_t)n_blocks + 1) * 4, st));
-    ClassifyParams cp{h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt, h->copts.inline_max};
+    ClassifyParams cp{dt == DBSPMSPV_PATTERN ? h->copts.th0_pattern : h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt, h->copts.inline_max};
     if (n_blocks) k_classify<<<grid_for(n_blocks, TPB / 32), TPB, 0, st>>>(n_blocks, blk_start, ukey, cp, type, psize, ecount, brow, bcol, cls, cls + DBSPMSPV_BLK_NCLASS);
     // view entries: a small valued block contributes one entry per stored element
     DBS_TRY(exclusive_sum(tp, ecount, eoff, (int64_t)n_blocks + 1, st));
@@ -650,7 +667,7 @@ int create_common(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz, con
     dbspmspv_handle_s *h = new (std::nothrow) dbspmspv_handle_s();
     if (!h) return DBSPMSPV_ERR_ALLOC;
     if (opts) h->copts = *opts; else dbspmspv_default_create_opts(&h->copts);
-    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.seg_cut > MAX_SEG_ENTRIES || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid_sparse < 1 || h->copts.w_dense_sparse < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 31) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
+    if (h->copts.th0 < 1 || h->copts.th0_pattern < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.seg_cut > MAX_SEG_ENTRIES || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid_sparse < 1 || h->copts.w_dense_sparse < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 31) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
     dbspmspv_default_run_opts(&h->ropts);
     h->d.dtype = dtype;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return DBSPMSPV_ERR_CUDA; }
@@ -671,7 +688,7 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     *o = dbspmspv_create_opts();
     o->th0 = 32; o->th1 = 128; o->th2 = 2.0f;
     o->seg_cut = 128; o->w_dense = 16; o->w_mid = 8; o->w_coo = 4; o->w_inline = 1;
-    o->w_dense_sparse = 128; o->w_mid_sparse = 64;
+    o->w_dense_sparse = 128; o->w_mid_sparse = 64; o->th0_pattern = 32;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
     o->inline_max = 31;

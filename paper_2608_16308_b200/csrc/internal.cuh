@@ -136,6 +136,7 @@ struct Device {           // everything the kernels need, passed by value
     const int32_t *seg_rb;  // row block of every segment (compact copy for the pull kernel)
     const int2 *chunks;   // n_chunks + 1: {first segment, first entry} of every pull chunk
     int32_t n_chunks;
+    const uint32_t *row_present32;  // per row block: rows that hold a stored element (two 16-bit masks per word)
     Workspace ws;
 };
 

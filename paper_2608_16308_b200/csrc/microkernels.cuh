@@ -317,14 +317,28 @@ __device__ __forceinline__ void half_stream(const uint8_t *payload, const float 
     if (touched) emit(srb, row, sum);
 }
 
-// Lane-owned Boolean form: rows of one mask-based block reached from the active columns.
+// Lane-owned Boolean form: rows of one mask-based block reached from the active columns.  The 16
+// masks (the first 32 bytes of every mask-based block, 16-byte aligned) come in with two
+// 16-byte loads and are tested in registers without a data-dependent branch.
 __device__ __forceinline__ uint32_t lane_heavy_bool(int type, const uint8_t *blk, uint32_t xm) {
-    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    const uint4 *m4 = reinterpret_cast<const uint4 *>(blk);
+    const uint4 a = m4[0], b = m4[1];
+    const uint32_t wd[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};   // two masks per word
     uint32_t hit = 0;
     if (is_row_major(type)) {
-        for (int r = 0; r < 16; ++r) hit |= (masks[r] & xm) ? (1u << r) : 0u;
+        const uint32_t xx = xm | (xm << 16);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t t = wd[i] & xx;
+            hit |= ((t & 0xFFFFu) ? 1u : 0u) << (2 * i);
+            hit |= ((t >> 16) ? 1u : 0u) << (2 * i + 1);
+        }
     } else {
-        for (uint32_t act = xm; act; act &= act - 1) hit |= masks[__ffs(act) - 1];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t lo = 0u - ((xm >> (2 * i)) & 1u), hi = 0u - ((xm >> (2 * i + 1)) & 1u);
+            hit |= (wd[i] & 0xFFFFu & lo) | ((wd[i] >> 16) & hi);
+        }
     }
     return hit;
 }

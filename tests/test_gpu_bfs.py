@@ -38,9 +38,12 @@ GRAPHS = [
 
 @pytest.mark.parametrize("name,make", GRAPHS, ids=[g[0] for g in GRAPHS])
 @pytest.mark.parametrize("path", PATHS)
-def test_levels_bit_exact(name, make, path):
+@pytest.mark.parametrize("th0_pattern", [32, 5], ids=["coo_lists", "bitmaps"])
+def test_levels_bit_exact(name, make, path, th0_pattern):
     g = make()
-    h = Handle(g, B.PATTERN)
+    o = B.default_create_opts()
+    o.th0_pattern = th0_pattern          # 5: pattern blocks of 5..31 entries become bit-mask blocks
+    h = Handle(g, B.PATTERN, opts=o)
     h.set_opts(force_path=path)
     A = ref_matrix(g)
     deg = np.diff(g.row_ptr)
