@@ -86,16 +86,12 @@ typedef struct {
     int32_t w_coo;           /* ... of a COO block                                  (4)      */
     int32_t force_format;    /* DBSPMSPV_FORMAT_*: ablation knob (Section 5.4)               */
     int32_t input_on_host;   /* 1: the create arrays are HOST pointers (copied once)         */
-    int32_t inline_max;      /* valued matrices: a block with at most this many entries keeps
+    int32_t inline_max;      /* a block with at most this many entries keeps
                                 them in its view entries, one entry per element      (31)    */
     int32_t w_inline;        /* ... of an INLINE view entry                         (1)      */
     int32_t w_dense_sparse;  /* Dense / CSR-like weights used instead when such blocks are a */
     int32_t w_mid_sparse;    /* minority of the matrix (hypersparse matrices)  (128 / 64)    */
-    int32_t th0_pattern;     /* pattern matrices: th0 used in place of th0 (32).  Lower values
-                                turn coordinate lists of th0_pattern..31 entries into 32-byte
-                                bit-mask blocks (measured slower for BFS on power-law graphs:
-                                four times the payload traffic)                              */
-    int32_t reserved[2];
+    int32_t reserved[3];
 } dbspmspv_create_opts;
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
@@ -109,8 +105,10 @@ typedef struct {
     int32_t validate;        /* 1: range-check x indices on the device (ERR_BOUNDS)          */
     int32_t timing;          /* 1: bracket the traversal kernel of run/decode with two CUDA
                                 events (made at create); read back as last_compute_ms      */
-    float th3_bfs;           /* db_bfs: same rule per level (pull levels skip finished row
-                                blocks and stop early, so the crossover is lower; 0.01)    */
+    float th3_bfs;           /* db_bfs: same rule per level.  Default 0.1, measured on the
+                                symmetrised R-MAT scale 22 graph (0.05 .. 0.2 are within 1 %;
+                                a pull level skips finished row blocks, a push level pays one
+                                atomic per reached entry)                                   */
     float th3_decode;        /* dbspmspv_decode: same rule; the output is dense and every row block
                                 takes part, so pull wins much earlier (0.01, the paper's value) */
     int32_t reserved[9];

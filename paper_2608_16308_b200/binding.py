@@ -37,8 +37,7 @@ class CreateOpts(ctypes.Structure):
                 ("w_coo", ctypes.c_int32), ("force_format", ctypes.c_int32),
                 ("input_on_host", ctypes.c_int32), ("inline_max", ctypes.c_int32),
                 ("w_inline", ctypes.c_int32), ("w_dense_sparse", ctypes.c_int32),
-                ("w_mid_sparse", ctypes.c_int32), ("th0_pattern", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 2)]
+                ("w_mid_sparse", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
 
 
 class RunOpts(ctypes.Structure):

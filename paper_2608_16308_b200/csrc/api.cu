@@ -9,7 +9,7 @@ namespace {
 
 __device__ __forceinline__ int block_nnz(int dtype, uint32_t idx, uint32_t aux) {
     const int type = idx >> TYPE_SHIFT;
-    if (type == DBSPMSPV_BLK_INLINE && dtype != DBSPMSPV_PATTERN) return 1;
+    if (type == DBSPMSPV_BLK_INLINE) return 1;
     return (int)aux + 1;
 }
 
@@ -39,9 +39,7 @@ __global__ void k_export(Device d, const int32_t *block_row, const int32_t *elem
     const int r0 = block_row[b] * 16, c0 = (int)(idx & IDX_MASK) * 16;
     const int64_t o = elem_start[b];
     if (type == DBSPMSPV_BLK_INLINE) {
-        if (DT == DBSPMSPV_PATTERN) {
-            if (lane <= (int)aux) { uint32_t rc = (w >> (8 * lane)) & 0xFF; row[o + lane] = r0 + (rc >> 4); col[o + lane] = c0 + (rc & 15); }
-        } else if (lane == 0) {
+        if (lane == 0) {
             row[o] = r0 + (aux >> 4); col[o] = c0 + (aux & 15);
             if (val && DT == DBSPMSPV_F32) static_cast<uint32_t *>(val)[o] = w;
             if (val && DT == DBSPMSPV_BF16) static_cast<uint16_t *>(val)[o] = (uint16_t)w;

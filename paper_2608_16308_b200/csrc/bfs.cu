@@ -22,15 +22,7 @@ __device__ __forceinline__ uint32_t lane_block_bool(int type, uint32_t w, uint32
                                                     const uint8_t *payload) {
     uint32_t hit = 0;
     if (type == DBSPMSPV_BLK_INLINE) {
-        if (DT == DBSPMSPV_PATTERN) {
-#pragma unroll
-            for (uint32_t k = 0; k < 4; ++k) {      // up to four packed coordinates, no branch
-                const uint32_t rc = (w >> (8 * k)) & 0xFFu;
-                hit |= (k <= aux ? (xm >> (rc & 15)) & 1u : 0u) << (rc >> 4);
-            }
-        } else if ((xm >> (aux & 15)) & 1u) {
-            hit = 1u << (aux >> 4);
-        }
+        hit = ((xm >> (aux & 15)) & 1u) << (aux >> 4);
     } else {
         const uint8_t *blk = payload + (size_t)w * 4;
         for (uint32_t k = 0; k <= aux; ++k) {
@@ -49,42 +41,66 @@ __device__ __forceinline__ void write_levels(int32_t *levels, int rb, uint32_t f
     }
 }
 
-// Boolean push: tasks of the active frontier blocks; newly reached rows are claimed with one
-// atomicOr per block on the next-frontier masks (the winner writes the level).
+// Boolean push: tasks of the active frontier blocks (a task is at most PUSH_CHUNK = 32 view
+// entries: one warp step); newly reached rows are claimed with one atomicOr per entry on the
+// next-frontier masks (the winner writes the level).  Like the pull, the loop is software-
+// pipelined: while task k is evaluated, the visited masks of k+1, the view entries of k+2 and
+// the task record of k+3 (in this warp's stride) are in flight.
 template <int DT>
 __device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int depth) {
+    static_assert(PUSH_CHUNK == 32, "one warp step per task");
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint2 none = make_uint2(0u, 0u);
+    struct Entries { uint32_t idx, aux, xm; int n; };   // n: entries of the task (0 = no task)
+    auto entries_of = [&](int t, const uint2 &task) {
+        Entries e{0u, 0u, 0u, 0};
+        if (t < n_tasks) {
+            const int jb = (int)(task.x & IDX_MASK), start = (int)task.y;
+            // the record holds ceil(n / 4) - 1: load under that bound (the view arrays are padded),
+            // the exact end comes from the column pointer
+            const int approx = (int)((task.x >> 27) + 1) * 4;
+            if (lane < approx) { e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane]; }
+            e.xm = mask_of(d.ws.x_mask32, jb);
+            e.n = min(PUSH_CHUNK, d.csc.ptr[jb + 1] - start);
+        }
+        return e;
+    };
+    auto need_of = [&](const Entries &e) { return lane < e.n ? ~mask_of(d.ws.visited32, e.idx & IDX_MASK) & 0xFFFFu : 0u; };
+    uint2 t1 = gwarp + nwarps < n_tasks ? d.ws.tasks[gwarp + nwarps] : none;
+    uint2 t2 = gwarp + 2 * nwarps < n_tasks ? d.ws.tasks[gwarp + 2 * nwarps] : none;
+    Entries e0 = entries_of(gwarp, gwarp < n_tasks ? d.ws.tasks[gwarp] : none);
+    Entries e1 = entries_of(gwarp + nwarps, t1);
+    uint32_t need0 = need_of(e0);
     for (int t = gwarp; t < n_tasks; t += nwarps) {
-        const uint2 task = d.ws.tasks[t];
-        const int jb = (int)(task.x & IDX_MASK);
-        const int start = (int)task.y;
-        const int end = min(start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
-        const uint32_t xm = mask_of(d.ws.x_mask32, jb);
-        for (int base = start; base < end; base += 32) {
-            const int p = base + lane;
+        const uint2 t3 = t + 3 * nwarps < n_tasks ? d.ws.tasks[t + 3 * nwarps] : none;   // stage 1
+        const Entries e2 = entries_of(t + 2 * nwarps, t2);                                // stage 2
+        const uint32_t need1 = need_of(e1);                                               // stage 3
+        // stage 4: evaluate task t
+        {
+            const uint32_t idx = e0.idx, aux = e0.aux, xm = e0.xm;
+            const int type = idx >> TYPE_SHIFT, brow = idx & IDX_MASK;
             bool heavy = false;
-            uint32_t idx = 0, w = 0, aux = 0;
-            if (p < end) {
-                idx = d.csc.idx[p];
-                const int type = idx >> TYPE_SHIFT, brow = idx & IDX_MASK;
-                const uint32_t need = ~mask_of(d.ws.visited32, brow) & 0xFFFFu;
-                if (need) {
-                    w = d.csc.w[p]; aux = d.csc.aux[p];
-                    if (type != DBSPMSPV_BLK_COO || aux < COO_SERIAL_MAX) {
-                        // one lane per block: hypersparse blocks from their coordinates,
-                        // mask-based blocks from their 16 masks
-                        const uint32_t hit = need & (type <= DBSPMSPV_BLK_COO ? lane_block_bool<DT>(type, w, aux, xm, d.payload)
-                                                                             : lane_heavy_bool(type, d.payload + (size_t)w * 4, xm));
-                        if (hit) {
-                            const int sh = (brow & 1) * 16;
-                            const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hit << sh);
-                            write_levels(levels, brow, hit & ~(old >> sh), depth);
-                        }
+            uint32_t w = 0;
+            if (need0) {
+                uint32_t hit = 0;
+                if (type == DBSPMSPV_BLK_INLINE) {
+                    hit = ((xm >> (aux & 15)) & 1u) << (aux >> 4);
+                } else {
+                    w = d.csc.w[(int)d.ws.tasks[t].y + lane];
+                    if (type == DBSPMSPV_BLK_COO) {
+                        if (aux < COO_SERIAL_MAX) hit = lane_block_bool<DT>(type, w, aux, xm, d.payload);
+                        else heavy = true;
                     } else {
-                        heavy = true;
+                        hit = lane_heavy_bool(type, d.payload + (size_t)w * 4, xm);
                     }
+                }
+                hit &= need0;
+                if (hit) {
+                    const int sh = (brow & 1) * 16;
+                    const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hit << sh);
+                    write_levels(levels, brow, hit & ~(old >> sh), depth);
                 }
             }
             uint32_t hv = __ballot_sync(FULL, heavy);
@@ -94,100 +110,117 @@ __device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int dept
                 const uint32_t bidx = __shfl_sync(FULL, idx, src);
                 const uint32_t bw = __shfl_sync(FULL, w, src);
                 const int nnz = (int)__shfl_sync(FULL, aux, src) + 1;
-                const int type = bidx >> TYPE_SHIFT, brow = bidx & IDX_MASK;
-                uint32_t hits = warp_block_bool<DT>(type, d.payload + (size_t)bw * 4, nnz, xm, lane);
-                hits &= ~mask_of(d.ws.visited32, brow);
+                const int btype = bidx >> TYPE_SHIFT, bbrow = bidx & IDX_MASK;
+                uint32_t hits = warp_block_bool<DT>(btype, d.payload + (size_t)bw * 4, nnz, xm, lane);
+                hits &= ~mask_of(d.ws.visited32, bbrow);
                 if (lane == 0 && hits) {
-                    const int sh = (brow & 1) * 16;
-                    const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hits << sh);
-                    write_levels(levels, brow, hits & ~(old >> sh), depth);
+                    const int sh = (bbrow & 1) * 16;
+                    const uint32_t old = atomicOr(&d.ws.y_mask32[bbrow >> 1], hits << sh);
+                    write_levels(levels, bbrow, hits & ~(old >> sh), depth);
                 }
             }
         }
+        // rotate the pipeline
+        e0 = e1; e1 = e2; need0 = need1; t2 = t3;
     }
 }
 
-// Boolean pull: one warp per row-block segment; row blocks with nothing left to discover are
-// skipped, and a segment stops as soon as all its unvisited rows are found (the early exit of
-// Algorithm 5 lifted to the row block).
+// Boolean pull: one warp per row-block segment (a segment has at most MAX_SEG_ENTRIES = 4 x 32
+// view entries, so one round of four warp steps covers it); row blocks with nothing left to
+// discover are skipped.  A segment costs a chain of dependent loads (descriptor -> visited mask
+// -> view entries -> frontier masks); the loop is software-pipelined four deep so that only the
+// last link is waited for: while segment k is evaluated, the entries of k+1, the visited mask
+// of k+2 and the descriptor of k+3 (k counted in this warp's stride) are already in flight.
 template <int DT>
 __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
+    constexpr int U = MAX_SEG_ENTRIES / 32;
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
-    // the descriptor and the visited mask of the warp's next segment are fetched while the
-    // current one is processed (two of the four dependent loads per segment leave the chain)
-    Segment seg_n = Segment{0, 0, 0, 0};
-    uint32_t need_n = 0;
-    if (gwarp < d.n_segments) {
-        seg_n = d.segments[gwarp];
-        need_n = ~mask_of(d.ws.visited32, seg_n.row_block) & 0xFFFFu;
+    const int nseg = d.n_segments;
+    const Segment none = Segment{0, 0, 0, 0};
+    auto need_of = [&](const Segment &sg) { return (sg.count & 0x7FFFFFFF) ? ~mask_of(d.ws.visited32, sg.row_block) & 0xFFFFu : 0u; };
+    // prologue: fill the pipeline
+    Segment s0 = gwarp < nseg ? d.segments[gwarp] : none;
+    Segment s1 = gwarp + nwarps < nseg ? d.segments[gwarp + nwarps] : none;
+    Segment s2 = gwarp + 2 * nwarps < nseg ? d.segments[gwarp + 2 * nwarps] : none;
+    uint32_t need0 = need_of(s0), need1 = need_of(s1);
+    uint32_t idx0[U], aux0[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int k = u * 32 + lane;
+        idx0[u] = 0; aux0[u] = 0;
+        if (need0 && k < (s0.count & 0x7FFFFFFF)) { idx0[u] = d.csr.idx[s0.start + k]; aux0[u] = d.csr.aux[s0.start + k]; }
     }
-    for (int sg = gwarp; sg < d.n_segments; sg += nwarps) {
-        const Segment seg = seg_n;
-        const uint32_t need = need_n;
-        if (sg + nwarps < d.n_segments) {
-            seg_n = d.segments[sg + nwarps];
-            need_n = ~mask_of(d.ws.visited32, seg_n.row_block) & 0xFFFFu;
+    for (int sg = gwarp; sg < nseg; sg += nwarps) {
+        // stage 1: descriptor three strides ahead
+        const Segment s3 = sg + 3 * nwarps < nseg ? d.segments[sg + 3 * nwarps] : none;
+        // stage 2: visited mask two strides ahead
+        const uint32_t need2 = need_of(s2);
+        // stage 3: view entries one stride ahead
+        uint32_t idx1[U], aux1[U];
+        const int cnt1 = s1.count & 0x7FFFFFFF;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int k = u * 32 + lane;
+            idx1[u] = 0; aux1[u] = 0;
+            if (need1 && k < cnt1) { idx1[u] = d.csr.idx[s1.start + k]; aux1[u] = d.csr.aux[s1.start + k]; }
         }
-        const int rb = seg.row_block;
-        if (!need) continue;
-        const bool whole = seg.count < 0;
-        const int end = seg.start + (seg.count & 0x7FFFFFFF);
-        uint32_t hit = 0;
-        // up to four warp steps of view entries are fetched at once, then their frontier masks,
-        // so that every lane keeps several independent loads in flight
-        constexpr int U = 4;
-        bool done = false;
-        for (int base = seg.start; base < end && !done; base += 32 * U) {
-            uint32_t idx[U], w[U], aux[U], xm[U];
+        // stage 4: evaluate this segment
+        if (need0) {
+            const int cnt0 = s0.count & 0x7FFFFFFF;
+            const int rb = s0.row_block;
+            uint32_t xm[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) xm[u] = u * 32 + lane < cnt0 ? mask_of(d.ws.x_mask32, idx0[u] & IDX_MASK) : 0u;
+            uint32_t hit = 0;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int p = base + u * 32 + lane;
-                idx[u] = 0; w[u] = 0; aux[u] = 0;
-                if (p < end) { idx[u] = d.csr.idx[p]; w[u] = d.csr.w[p]; aux[u] = d.csr.aux[p]; }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-                xm[u] = base + u * 32 + lane < end ? mask_of(d.ws.x_mask32, idx[u] & IDX_MASK) : 0u;
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (base + u * 32 >= end) break;
+                if (u * 32 >= cnt0) break;      // warp-uniform
+                const int type = idx0[u] >> TYPE_SHIFT;
                 bool heavy = false;
+                uint32_t w = 0;
                 if (xm[u]) {
-                    const int type = idx[u] >> TYPE_SHIFT;
-                    if (type <= DBSPMSPV_BLK_COO) {
-                        if (type == DBSPMSPV_BLK_INLINE || aux[u] < COO_SERIAL_MAX) hit |= lane_block_bool<DT>(type, w[u], aux[u], xm[u], d.payload);
-                        else heavy = true;
+                    if (type == DBSPMSPV_BLK_INLINE) {
+                        hit |= ((xm[u] >> (aux0[u] & 15)) & 1u) << (aux0[u] >> 4);
                     } else {
-                        hit |= lane_heavy_bool(type, d.payload + (size_t)w[u] * 4, xm[u]);
+                        w = d.csr.w[s0.start + u * 32 + lane];
+                        if (type == DBSPMSPV_BLK_COO) {
+                            if (aux0[u] < COO_SERIAL_MAX) hit |= lane_block_bool<DT>(type, w, aux0[u], xm[u], d.payload);
+                            else heavy = true;
+                        } else {
+                            hit |= lane_heavy_bool(type, d.payload + (size_t)w * 4, xm[u]);
+                        }
                     }
                 }
                 uint32_t hv = __ballot_sync(FULL, heavy);
                 while (hv) {
                     const int src = __ffs(hv) - 1;
                     hv &= hv - 1;
-                    const uint32_t bidx = __shfl_sync(FULL, idx[u], src);
-                    const uint32_t bw = __shfl_sync(FULL, w[u], src);
-                    const int nnz = (int)__shfl_sync(FULL, aux[u], src) + 1;
+                    const uint32_t bidx = __shfl_sync(FULL, idx0[u], src);
+                    const uint32_t bw = __shfl_sync(FULL, w, src);
+                    const int nnz = (int)__shfl_sync(FULL, aux0[u], src) + 1;
                     const uint32_t bxm = __shfl_sync(FULL, xm[u], src);
                     hit |= warp_block_bool<DT>(bidx >> TYPE_SHIFT, d.payload + (size_t)bw * 4, nnz, bxm, lane);
                 }
-                hit = __reduce_or_sync(FULL, hit);
-                if ((hit & need) == need) { done = true; break; }
+            }
+            hit = __reduce_or_sync(FULL, hit) & need0;
+            if (hit) {
+                if (s0.count < 0) {          // the segment is its whole row block: plain stores
+                    if (lane == 0) reinterpret_cast<uint16_t *>(d.ws.y_mask32)[rb] = (uint16_t)hit;
+                    if (lane < 16 && ((hit >> lane) & 1u)) levels[rb * 16 + lane] = depth;
+                } else if (lane == 0) {
+                    const int sh = (rb & 1) * 16;
+                    const uint32_t old = atomicOr(&d.ws.y_mask32[rb >> 1], hit << sh);
+                    write_levels(levels, rb, hit & ~(old >> sh), depth);
+                }
             }
         }
-        hit &= need;
-        if (hit) {
-            if (whole) {
-                if (lane == 0) reinterpret_cast<uint16_t *>(d.ws.y_mask32)[rb] = (uint16_t)hit;
-                if (lane < 16 && ((hit >> lane) & 1u)) levels[rb * 16 + lane] = depth;
-            } else if (lane == 0) {
-                const int sh = (rb & 1) * 16;
-                const uint32_t old = atomicOr(&d.ws.y_mask32[rb >> 1], hit << sh);
-                write_levels(levels, rb, hit & ~(old >> sh), depth);
-            }
-        }
+        // rotate the pipeline
+        s0 = s1; s1 = s2; s2 = s3;
+        need0 = need1; need1 = need2;
+#pragma unroll
+        for (int u = 0; u < U; ++u) { idx0[u] = idx1[u]; aux0[u] = aux1[u]; }
     }
 }
 
@@ -245,40 +278,35 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         if (path == DBSPMSPV_PATH_PUSH) bfs_push<DT>(d, n_tasks, levels, depth);
         else bfs_pull<DT>(d, levels, depth);
         grid.sync();
-        // next frontier: masks produced above become the vector-block masks of the next level;
-        // visited is updated; the push worklist and block statistics are rebuilt on the fly.
-        // The worklist is only needed if the next level is a push: the running count of nonempty
-        // blocks only grows, so once it has reached the selector's threshold the next level is
-        // known to be a pull and the remaining warps just count (a push is only ever chosen
-        // when no warp has skipped).
-        int found = 0;
-        for (int k0 = (tid & ~31); k0 < n_words; k0 += nthreads) {
-            const int k = k0 + lane;
-            uint32_t nm = 0;
-            if (k < n_words) {
-                nm = d.ws.y_mask32[k];
-                if (nm) {
-                    d.ws.y_mask32[k] = 0u;
-                    d.ws.visited32[k] |= nm;
-                    found += __popc(nm);
-                }
-                if (nm || d.ws.x_mask32[k]) d.ws.x_mask32[k] = nm;
+        // next frontier: masks produced above become the vector-block masks of the next level,
+        // visited is updated and the nonempty blocks are counted (one atomic per warp)
+        int found = 0, nz = 0;
+        for (int k = tid; k < n_words; k += nthreads) {
+            const uint32_t nm = d.ws.y_mask32[k];
+            if (nm) {
+                d.ws.y_mask32[k] = 0u;
+                d.ws.visited32[k] |= nm;
+                found += __popc(nm);
+                nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
             }
-            const bool lo = (nm & 0xFFFFu) != 0, hi = (nm >> 16) != 0;
-            int seen = 0;     // read by one lane: the branch below must be warp-uniform
-            if (lane == 0) seen = *reinterpret_cast<volatile int32_t *>(&ctr->bfs_cnt[cur ^ 1][0]);
-            seen = __shfl_sync(FULL, seen, 0);
-            if (bfs_path(seen, d.nb, th3, force_path) == DBSPMSPV_PATH_PULL) {
-                const int nz = __popc(__ballot_sync(FULL, lo)) + __popc(__ballot_sync(FULL, hi));
-                if (lane == 0 && nz) atomicAdd(&ctr->bfs_cnt[cur ^ 1][0], nz);
-            } else {
-                emit_tasks(d, lo, 2 * k, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->bfs_cnt[cur ^ 1][0]);
-                emit_tasks(d, hi, 2 * k + 1, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->bfs_cnt[cur ^ 1][0]);
-            }
+            if (nm || d.ws.x_mask32[k]) d.ws.x_mask32[k] = nm;
         }
         found = __reduce_add_sync(FULL, found);
-        if (lane == 0 && found) atomicAdd(&ctr->bfs_reached, found);
+        nz = __reduce_add_sync(FULL, nz);
+        if (lane == 0 && found) { atomicAdd(&ctr->bfs_reached, found); atomicAdd(&ctr->bfs_cnt[cur ^ 1][0], nz); }
         grid.sync();
+        // the push worklist is rebuilt only if the next level is a push (the selector's input is
+        // known now); its block count goes to a scratch counter
+        const int next_n = ctr->bfs_cnt[cur ^ 1][0];
+        if (next_n && bfs_path(next_n, d.nb, th3, force_path) == DBSPMSPV_PATH_PUSH) {
+            for (int k0 = (tid & ~31); k0 < n_words; k0 += nthreads) {
+                const int k = k0 + lane;
+                const uint32_t nm = k < n_words ? d.ws.x_mask32[k] : 0u;
+                emit_tasks(d, (nm & 0xFFFFu) != 0, 2 * k, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad);
+                emit_tasks(d, (nm >> 16) != 0, 2 * k + 1, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad);
+            }
+            grid.sync();
+        }
         cur ^= 1;
     }
     // leave the shared workspace as dbspmspv_run expects it: all masks clear

@@ -155,10 +155,8 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
             if (cp.force_format == DBSPMSPV_FORMAT_COO) type = DBSPMSPV_BLK_COO;
             else if (cp.force_format == DBSPMSPV_FORMAT_CSR) type = DBSPMSPV_BLK_CSR;
             else if (nnz < cp.th0) {
-                // pattern: up to four coordinates fit in one view entry; valued: one view
-                // entry per stored element, up to inline_max of them
-                const int inline_cap = cp.dtype == DBSPMSPV_PATTERN ? 4 : cp.inline_max;
-                type = nnz <= inline_cap ? DBSPMSPV_BLK_INLINE : DBSPMSPV_BLK_COO;
+                // one view entry per stored element, up to inline_max of them
+                type = nnz <= cp.inline_max ? DBSPMSPV_BLK_INLINE : DBSPMSPV_BLK_COO;
             } else if (nnz > cp.th1) type = DBSPMSPV_BLK_DENSE;
             // skew_c / skew_r = (max column count) / (max row count): the denominators of
             // the two axis skews are identical for square blocks
@@ -168,7 +166,7 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
             const int vsize = cp.dtype == DBSPMSPV_F32 ? 4 : cp.dtype == DBSPMSPV_BF16 ? 2 : 0;
             type_out[b] = (uint8_t)type;
             size_out[b] = (uint32_t)payload_words(type, nnz, vsize);
-            ecount[b] = (type == DBSPMSPV_BLK_INLINE && cp.dtype != DBSPMSPV_PATTERN) ? nnz : 1;
+            ecount[b] = type == DBSPMSPV_BLK_INLINE ? nnz : 1;
             uint64_t k0 = ukey[s];
             brow[b] = (int32_t)(k0 >> 35);
             bcol[b] = (int32_t)((k0 >> 8) & IDX_MASK);
@@ -207,12 +205,14 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
     uint8_t *base = payload + off_words * 4;
     const int e0 = eoff[b];
     const uint32_t tagged = (uint32_t)bcol[b] | ((uint32_t)type << TYPE_SHIFT);
-    if (type == DBSPMSPV_BLK_INLINE && DT != DBSPMSPV_PATTERN) {
-        // one view entry per stored element: value in w, packed coordinate in aux
+    if (type == DBSPMSPV_BLK_INLINE) {
+        // one view entry per stored element: value in w (unused for pattern matrices), packed
+        // coordinate in aux
         for (int k = lane; k < nnz; k += 32) {
             v_idx[e0 + k] = tagged;
-            v_w[e0 + k] = DT == DBSPMSPV_F32 ? __float_as_uint(static_cast<const float *>(uval)[s + k])
-                                             : (uint32_t) static_cast<const uint16_t *>(uval)[s + k];
+            v_w[e0 + k] = DT == DBSPMSPV_F32    ? __float_as_uint(static_cast<const float *>(uval)[s + k])
+                          : DT == DBSPMSPV_BF16 ? (uint32_t) static_cast<const uint16_t *>(uval)[s + k]
+                                                : 0u;
             v_aux[e0 + k] = (uint8_t)(ukey[s + k] & 0xFF);
             entry_row[e0 + k] = brow[b];
         }
@@ -221,16 +221,9 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
     if (lane == 0) {
         v_idx[e0] = tagged;
         entry_row[e0] = brow[b];
-        if (type == DBSPMSPV_BLK_INLINE) {
-            uint32_t w = 0;
-            for (int k = 0; k < nnz; ++k) w |= (uint32_t)(ukey[s + k] & 0xFF) << (8 * k);
-            v_w[e0] = w;
-        } else {
-            v_w[e0] = (uint32_t)off_words;
-        }
+        v_w[e0] = (uint32_t)off_words;
         v_aux[e0] = (uint8_t)(nnz - 1);
     }
-    if (type == DBSPMSPV_BLK_INLINE) return;
     if (type == DBSPMSPV_BLK_COO) {
         uint8_t *vals = base + ((nnz + 3) & ~3);
         for (int k = lane; k < ((nnz + 3) & ~3); k += 32)
@@ -531,7 +524,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     DBS_GET(cls, 2 * DBSPMSPV_BLK_NCLASS);
     DBS_CUDA(cudaMemsetAsync(cls, 0, 2 * DBSPMSPV_BLK_NCLASS * sizeof(unsigned long long), st));
     DBS_CUDA(cudaMemsetAsync(ecount, 0, ((size_t)n_blocks + 1) * 4, st));
-    ClassifyParams cp{dt == DBSPMSPV_PATTERN ? h->copts.th0_pattern : h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt, h->copts.inline_max};
+    ClassifyParams cp{h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt, h->copts.inline_max};
     if (n_blocks) k_classify<<<grid_for(n_blocks, TPB / 32), TPB, 0, st>>>(n_blocks, blk_start, ukey, cp, type, psize, ecount, brow, bcol, cls, cls + DBSPMSPV_BLK_NCLASS);
     // view entries: a small valued block contributes one entry per stored element
     DBS_TRY(exclusive_sum(tp, ecount, eoff, (int64_t)n_blocks + 1, st));
@@ -667,7 +660,7 @@ int create_common(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nnz, con
     dbspmspv_handle_s *h = new (std::nothrow) dbspmspv_handle_s();
     if (!h) return DBSPMSPV_ERR_ALLOC;
     if (opts) h->copts = *opts; else dbspmspv_default_create_opts(&h->copts);
-    if (h->copts.th0 < 1 || h->copts.th0_pattern < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.seg_cut > MAX_SEG_ENTRIES || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid_sparse < 1 || h->copts.w_dense_sparse < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 31) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
+    if (h->copts.th0 < 1 || h->copts.th1 > 256 || h->copts.seg_cut < 1 || h->copts.seg_cut > MAX_SEG_ENTRIES || h->copts.w_coo < 1 || h->copts.w_inline < 1 || h->copts.w_mid_sparse < 1 || h->copts.w_dense_sparse < 1 || h->copts.w_mid < 1 || h->copts.w_dense < 1 || h->copts.inline_max < 0 || h->copts.inline_max > 31) { delete h; return DBSPMSPV_ERR_INVALID_ARG; }
     dbspmspv_default_run_opts(&h->ropts);
     h->d.dtype = dtype;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return DBSPMSPV_ERR_CUDA; }
@@ -688,7 +681,7 @@ void dbspmspv_default_create_opts(dbspmspv_create_opts *o) {
     *o = dbspmspv_create_opts();
     o->th0 = 32; o->th1 = 128; o->th2 = 2.0f;
     o->seg_cut = 128; o->w_dense = 16; o->w_mid = 8; o->w_coo = 4; o->w_inline = 1;
-    o->w_dense_sparse = 128; o->w_mid_sparse = 64; o->th0_pattern = 32;
+    o->w_dense_sparse = 128; o->w_mid_sparse = 64;
     o->force_format = DBSPMSPV_FORMAT_AUTO;
     o->input_on_host = 0;
     o->inline_max = 31;

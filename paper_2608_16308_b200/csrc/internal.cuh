@@ -18,10 +18,11 @@ namespace dbs {
 //                       block-CSR view, row block in the block-CSC view)
 //           bit  28     block-CSR view only: first entry of a pull segment
 //           bits 29..31 block class (DBSPMSPV_BLK_*)
-//   w[p]    payload offset in 4-byte words -- or, for INLINE blocks, the data itself:
-//             valued matrices : the single value (fp32 bits, or bf16 bits in the low half)
-//             pattern matrices: up to four packed local coordinates, one per byte
-//   aux[p]  nnz-1 -- or, for valued INLINE blocks, the packed local coordinate
+//   w[p]    payload offset in 4-byte words -- or, for INLINE entries, the stored value itself
+//           (fp32 bits, or bf16 bits in the low half; unused for pattern matrices)
+//   aux[p]  nnz-1 -- or, for INLINE entries, the packed local coordinate
+// A block with at most inline_max stored elements has no payload: it is one INLINE view entry
+// per element (adjacent in both views).
 // A packed local coordinate is one byte: (row << 4) | col.
 // Both views carry the same (w, aux) for a block, so either traversal direction reaches the
 // payload in one hop; the payload itself is stored once, in block-CSR ("primary") order.

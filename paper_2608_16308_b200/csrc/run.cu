@@ -101,13 +101,8 @@ __device__ __forceinline__ uint32_t lane_block(int type, uint32_t w, uint32_t au
                                                Emit emit) {
     uint32_t hit = 0;
     if (type == DBSPMSPV_BLK_INLINE) {
-        if (DT == DBSPMSPV_PATTERN) {
-            for (uint32_t k = 0; k <= aux; ++k) {
-                const uint32_t rc = (w >> (8 * k)) & 0xFFu;
-                if ((xm >> (rc & 15)) & 1u) hit |= 1u << (rc >> 4);
-            }
-        } else if ((xm >> (aux & 15)) & 1u) {
-            emit((int)(aux >> 4), Val<DT>::inline_value(w) * xin);
+        if ((xm >> (aux & 15)) & 1u) {
+            if (DT != DBSPMSPV_PATTERN) emit((int)(aux >> 4), Val<DT>::inline_value(w) * xin);
             hit = 1u << (aux >> 4);
         }
     } else {
@@ -405,8 +400,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
 #pragma unroll
             for (int u = 0; u < PULL_UNROLL; ++u) {
                 const bool have = base + u * 32 + lane < e1;
-                xin[u] = (have && DT != DBSPMSPV_PATTERN)
-                             ? d.ws.x_dense[(size_t)(idx[u] & IDX_MASK) * 16 + (aux[u] & 15)]
+                xin[u] = have ? d.ws.x_dense[(size_t)(idx[u] & IDX_MASK) * 16 + (aux[u] & 15)]
                              : __uint_as_float(X_ABSENT);
             }
 #pragma unroll
@@ -449,15 +443,15 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                     __syncwarp();
                 }
                 const int type = idx[u] >> TYPE_SHIFT;
-                const bool inl = type == DBSPMSPV_BLK_INLINE && DT != DBSPMSPV_PATTERN;
+                const bool inl = type == DBSPMSPV_BLK_INLINE;
                 if (inl && __float_as_uint(xin[u]) != X_ABSENT) {    // absent also covers "past the end"
                     const float v = Val<DT>::inline_value(w[u]) * xin[u];
                     const int r = aux[u] >> 4;
                     if (one_seg || rb == cur_rb) {
-                        atomicAdd(&my_y[r], v);
+                        if (DT != DBSPMSPV_PATTERN) atomicAdd(&my_y[r], v);
                         hit |= 1u << r;
                     } else {
-                        atomicAdd(out.acc + (size_t)rb * 16 + r, v);
+                        if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)rb * 16 + r, v);
                         if (Out::MASKS) out.hit8[(size_t)rb * 16 + r] = 1;
                     }
                 }
@@ -469,10 +463,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                 bool heavy = false;
                 int coo_cnt = 0;
                 if (xm) {
-                    if (type == DBSPMSPV_BLK_INLINE) {             // pattern: up to four coordinates
-                        const uint32_t hb = lane_block<DT>(type, w[u], aux[u], xm, 0.f, nullptr, d.payload, [](int, float) {});
-                        if (Out::MASKS && hb) mark_rows(out.hit8, rb, hb);
-                    } else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
+                    if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
                         coo_cnt = (int)aux[u] + 1;
                     } else {
                         heavy = true;
@@ -939,7 +930,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
     o->th3 = 0.65f;
-    o->th3_bfs = 0.01f;
+    o->th3_bfs = 0.1f;
     o->th3_decode = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;
     o->popc_threshold = 8;

@@ -30,7 +30,6 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
 def test_host_only_entry_points():
     o = B.default_create_opts()
     assert (o.th0, o.th1, o.th2) == (32, 128, 2.0)          # Section 3.2.1 thresholds
-    assert o.th0_pattern == 32
     assert o.w_dense > o.w_mid > o.w_coo >= o.w_inline >= 1   # Section 3.3.2 ordering of segment weights
     r = B.default_run_opts()
     assert r.force_path == B.PATH_AUTO and r.th3 > 0

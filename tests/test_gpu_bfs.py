@@ -38,11 +38,11 @@ GRAPHS = [
 
 @pytest.mark.parametrize("name,make", GRAPHS, ids=[g[0] for g in GRAPHS])
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("th0_pattern", [32, 5], ids=["coo_lists", "bitmaps"])
-def test_levels_bit_exact(name, make, path, th0_pattern):
+@pytest.mark.parametrize("inline_max", [31, 3], ids=["inline", "coo_lists"])
+def test_levels_bit_exact(name, make, path, inline_max):
     g = make()
     o = B.default_create_opts()
-    o.th0_pattern = th0_pattern          # 5: pattern blocks of 5..31 entries become bit-mask blocks
+    o.inline_max = inline_max            # 3: blocks of 4..31 entries become packed coordinate lists
     h = Handle(g, B.PATTERN, opts=o)
     h.set_opts(force_path=path)
     A = ref_matrix(g)

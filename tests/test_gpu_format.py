@@ -20,7 +20,7 @@ def cpu_classify(rows, cols, dtype, th0=32, th1=128, th2=2.0):
     key, rows, cols = key[order], rows[order], cols[order]
     ub, start, cnt = np.unique(key, return_index=True, return_counts=True)
     cls = np.empty(ub.size, dtype=np.int32)
-    cap = 4 if dtype == B.PATTERN else 31  # pattern: four coordinates per entry; valued: inline_max
+    cap = 31                               # inline_max: one view entry per stored element
     for b in range(ub.size):
         n = cnt[b]
         if n < th0:
@@ -98,10 +98,7 @@ def test_export_equals_input_and_census(name, make, dtype):
     assert np.array_equal(br, wr) and np.array_equal(bc, wc)
     assert np.array_equal(bn, wn) and int(bn.sum()) == csr.nnz
     assert np.array_equal(cls, wcls)
-    if dtype == B.PATTERN:
-        assert first.all()                                                      # one entry per block
-    else:
-        assert (en[ecls == B.BLK_INLINE] == 1).all() and first[ecls != B.BLK_INLINE].all()
+    assert (en[ecls == B.BLK_INLINE] == 1).all() and first[ecls != B.BLK_INLINE].all()
     assert s.n_blocks == wr.size and s.n_view_entries == er.size
     for k in range(6):
         assert s.class_blocks[k] == int((wcls == k).sum())
