@@ -207,22 +207,37 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    static_assert(U == 1, "one warp step per task");
     const int n_tasks = d.ws.ctr->n_tasks;
-    for (int t = gwarp; t < n_tasks; t += nwarps) {
-        const uint2 task = d.ws.tasks[t];
-        const int jb = (int)(task.x & IDX_MASK);
-        const int upper = ((int)(task.x >> 27) + 1) * 4;      // entries of the task, rounded up to 4
-        const int start = (int)task.y;
-        // one round of independent loads: view entries, exact end, mask, x block
-        uint32_t idx[U], w[U], aux[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            idx[u] = 0; w[u] = 0; aux[u] = 0;
-            if (u * 32 + lane < upper) { const int p = start + u * 32 + lane; idx[u] = d.csc.idx[p]; w[u] = d.csc.w[p]; aux[u] = d.csc.aux[p]; }
+    // A task is a chain of dependent loads (record -> entries, column end, mask, x block); the
+    // loop is software-pipelined: while task k is evaluated, the loads of k+1 and the record of
+    // k+2 (in this warp's stride) are in flight.
+    struct Loads { uint32_t idx, w, aux, xm; float xv; int start, end; };
+    auto loads_of = [&](int t, const uint2 &task) {
+        Loads l{0u, 0u, 0u, 0u, 0.f, 0, 0};
+        if (t < n_tasks) {
+            const int jb = (int)(task.x & IDX_MASK);
+            const int upper = ((int)(task.x >> 27) + 1) * 4;      // entries of the task, rounded up to 4
+            l.start = (int)task.y;
+            if (lane < upper) { const int p = l.start + lane; l.idx = d.csc.idx[p]; l.w = d.csc.w[p]; l.aux = d.csc.aux[p]; }
+            l.end = min(l.start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
+            l.xm = mask_of(d.ws.x_mask32, jb);
+            if (lane < 16) l.xv = d.ws.x_dense[jb * 16 + lane];
         }
-        const int end = min(start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
-        const uint32_t xm = mask_of(d.ws.x_mask32, jb);
-        if (lane < 16) s_x[lane] = d.ws.x_dense[jb * 16 + lane];
+        return l;
+    };
+    const uint2 none = make_uint2(0u, 0u);
+    uint2 rec1 = gwarp + nwarps < n_tasks ? d.ws.tasks[gwarp + nwarps] : none;
+    Loads cur = loads_of(gwarp, gwarp < n_tasks ? d.ws.tasks[gwarp] : none);
+    for (int t = gwarp; t < n_tasks; t += nwarps) {
+        const uint2 rec2 = t + 2 * nwarps < n_tasks ? d.ws.tasks[t + 2 * nwarps] : none;
+        const Loads nxt = loads_of(t + nwarps, rec1);
+        rec1 = rec2;
+        uint32_t idx[U] = {cur.idx}, w[U] = {cur.w}, aux[U] = {cur.aux};
+        const int start = cur.start, end = cur.end;
+        const uint32_t xm = cur.xm;
+        if (lane < 16) s_x[lane] = cur.xv;
+        cur = nxt;
         __syncwarp();
 #pragma unroll
         for (int u = 0; u < U; ++u) {
