@@ -194,6 +194,8 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-bfs", action="store_true")
     ap.add_argument("--bfs-scale", type=int, default=22)
+    ap.add_argument("--bfs-only", action="store_true",
+                    help="run only the DB-BFS leg and print its record (the command ncu captures k_bfs from)")
     ap.add_argument("--crossover", action="store_true",
                     help="print the measured push/pull crossover table (forced paths) and exit")
     args = ap.parse_args()
@@ -214,6 +216,11 @@ def main() -> None:
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
+    if args.bfs_only:
+        if rank == 0:
+            flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+            print(json.dumps(bench_bfs(args, B, torch, dev, flush)))
+        return
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
