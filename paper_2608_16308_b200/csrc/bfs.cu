@@ -145,13 +145,20 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
     Segment s1 = gwarp + nwarps < nseg ? d.segments[gwarp + nwarps] : none;
     Segment s2 = gwarp + 2 * nwarps < nseg ? d.segments[gwarp + 2 * nwarps] : none;
     uint32_t need0 = need_of(s0), need1 = need_of(s1);
-    uint32_t idx0[U], aux0[U];
+    // the entries of a segment: lane l takes positions l, l + 32, ... (constant offsets from one
+    // pointer per array, one comparison per step)
+    auto fetch = [&](const Segment &sg, uint32_t need, uint32_t (&idx)[U], uint32_t (&aux)[U]) {
+        const uint32_t *ip = d.csr.idx + sg.start + lane;
+        const uint8_t *ap = d.csr.aux + sg.start + lane;
+        const int rem = need ? (sg.count & 0x7FFFFFFF) - lane : 0;
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-        const int k = u * 32 + lane;
-        idx0[u] = 0; aux0[u] = 0;
-        if (need0 && k < (s0.count & 0x7FFFFFFF)) { idx0[u] = d.csr.idx[s0.start + k]; aux0[u] = d.csr.aux[s0.start + k]; }
-    }
+        for (int u = 0; u < U; ++u) {
+            idx[u] = 0; aux[u] = 0;
+            if (rem > u * 32) { idx[u] = ip[u * 32]; aux[u] = ap[u * 32]; }
+        }
+    };
+    uint32_t idx0[U], aux0[U];
+    fetch(s0, need0, idx0, aux0);
     for (int sg = gwarp; sg < nseg; sg += nwarps) {
         // stage 1: descriptor three strides ahead
         const Segment s3 = sg + 3 * nwarps < nseg ? d.segments[sg + 3 * nwarps] : none;
@@ -159,31 +166,36 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
         const uint32_t need2 = need_of(s2);
         // stage 3: view entries one stride ahead
         uint32_t idx1[U], aux1[U];
-        const int cnt1 = s1.count & 0x7FFFFFFF;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int k = u * 32 + lane;
-            idx1[u] = 0; aux1[u] = 0;
-            if (need1 && k < cnt1) { idx1[u] = d.csr.idx[s1.start + k]; aux1[u] = d.csr.aux[s1.start + k]; }
-        }
+        fetch(s1, need1, idx1, aux1);
         // stage 4: evaluate this segment
         if (need0) {
             const int cnt0 = s0.count & 0x7FFFFFFF;
             const int rb = s0.row_block;
+            // frontier masks: only for entries that can still contribute -- past-the-end entries
+            // are all-zero (INLINE, row 0); an INLINE entry whose row is not wanted is skipped
+            // (late pull levels want one or two rows of a row block: most gathers fall away)
+            const int rem0 = cnt0 - lane;
             uint32_t xm[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) xm[u] = u * 32 + lane < cnt0 ? mask_of(d.ws.x_mask32, idx0[u] & IDX_MASK) : 0u;
-            uint32_t hit = 0;
+            bool heavy_any = false;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (u * 32 >= cnt0) break;      // warp-uniform
-                const int type = idx0[u] >> TYPE_SHIFT;
-                bool heavy = false;
-                uint32_t w = 0;
-                if (xm[u]) {
-                    if (type == DBSPMSPV_BLK_INLINE) {
-                        hit |= ((xm[u] >> (aux0[u] & 15)) & 1u) << (aux0[u] >> 4);
-                    } else {
+                const bool inl = (idx0[u] >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE;
+                const bool want = rem0 > u * 32 && (!inl || ((need0 >> (aux0[u] >> 4)) & 1u));
+                xm[u] = want ? mask_of(d.ws.x_mask32, idx0[u] & IDX_MASK) : 0u;
+                heavy_any |= want && !inl;
+            }
+            uint32_t hit = 0;
+#pragma unroll
+            for (int u = 0; u < U; ++u)        // INLINE entries: branch-free (xm is 0 where not wanted)
+                hit |= ((idx0[u] >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE ? (xm[u] >> (aux0[u] & 15)) & 1u : 0u) << (aux0[u] >> 4);
+            if (__any_sync(FULL, heavy_any)) {   // rare: packed-COO and mask-based blocks
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (u * 32 >= cnt0) break;      // warp-uniform
+                    const int type = idx0[u] >> TYPE_SHIFT;
+                    bool heavy = false;
+                    uint32_t w = 0;
+                    if (xm[u] && type != DBSPMSPV_BLK_INLINE) {
                         w = d.csr.w[s0.start + u * 32 + lane];
                         if (type == DBSPMSPV_BLK_COO) {
                             if (aux0[u] < COO_SERIAL_MAX) hit |= lane_block_bool<DT>(type, w, aux0[u], xm[u], d.payload);
@@ -192,16 +204,16 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
                             hit |= lane_heavy_bool(type, d.payload + (size_t)w * 4, xm[u]);
                         }
                     }
-                }
-                uint32_t hv = __ballot_sync(FULL, heavy);
-                while (hv) {
-                    const int src = __ffs(hv) - 1;
-                    hv &= hv - 1;
-                    const uint32_t bidx = __shfl_sync(FULL, idx0[u], src);
-                    const uint32_t bw = __shfl_sync(FULL, w, src);
-                    const int nnz = (int)__shfl_sync(FULL, aux0[u], src) + 1;
-                    const uint32_t bxm = __shfl_sync(FULL, xm[u], src);
-                    hit |= warp_block_bool<DT>(bidx >> TYPE_SHIFT, d.payload + (size_t)bw * 4, nnz, bxm, lane);
+                    uint32_t hv = __ballot_sync(FULL, heavy);
+                    while (hv) {
+                        const int src = __ffs(hv) - 1;
+                        hv &= hv - 1;
+                        const uint32_t bidx = __shfl_sync(FULL, idx0[u], src);
+                        const uint32_t bw = __shfl_sync(FULL, w, src);
+                        const int nnz = (int)__shfl_sync(FULL, aux0[u], src) + 1;
+                        const uint32_t bxm = __shfl_sync(FULL, xm[u], src);
+                        hit |= warp_block_bool<DT>(bidx >> TYPE_SHIFT, d.payload + (size_t)bw * 4, nnz, bxm, lane);
+                    }
                 }
             }
             hit = __reduce_or_sync(FULL, hit) & need0;

@@ -181,8 +181,11 @@ __host__ __device__ inline T ceil_div(T a, T b) { return (a + b - 1) / b; }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// 16-bit mask of one block.  The mask arrays are updated as 32-bit words (two blocks per word,
+// the even block in the low half: atomics need the word) but read as the halfword itself: one
+// 16-bit load instead of a word load plus shift and mask (the GPU is little-endian).
 __device__ __forceinline__ uint32_t mask_of(const uint32_t *mask32, int blk) {
-    return (mask32[blk >> 1] >> ((blk & 1) * 16)) & 0xFFFFu;
+    return reinterpret_cast<const uint16_t *>(mask32)[blk];
 }
 
 // value loads from the payload, widened to fp32
