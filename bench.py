@@ -250,8 +250,6 @@ def main() -> None:
     y_idx_h = torch.empty(a.m, dtype=torch.int32).pin_memory()
     y_val_h = torch.empty(a.m, dtype=torch.float32).pin_memory()
     y_nnz_h = torch.zeros(1, dtype=torch.int32).pin_memory()
-    xi_stage = torch.empty(a.n, dtype=torch.int32, device=dev)
-    xv_stage = torch.empty(a.n, dtype=torch.float32, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)     # > 126 MB L2
     stream = torch.cuda.current_stream()
     opts = B.default_run_opts()
@@ -310,7 +308,9 @@ def main() -> None:
     step_ms = call_ms.sum(axis=1)
     ms_per_step = max_over_ranks(float(step_ms.mean()), dev)
 
-    # ---- end to end through the same C-ABI call with HOST buffers
+    # ---- end to end through the same C-ABI call with HOST buffers: x and y live in page-locked
+    # host memory that the device addresses directly, so the call's own kernels read x and write
+    # y (and the count) across PCIe -- no staging copy, one synchronisation per call
     e2e_ms = []
     h2d = d2h = 0
     for s in range(max(3, args.steps // 2) + 2):
@@ -321,18 +321,14 @@ def main() -> None:
             n_x = int(xs[k].idx.size)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            xi_stage[:n_x].copy_(xh[k][0], non_blocking=True)
-            xv_stage[:n_x].copy_(xh[k][1], non_blocking=True)
-            B.dbspmspv_run(h, xi_stage, xv_stage, n_x, B.PLUS_TIMES, y_idx, y_val, a.m, y_nnz)
-            y_nnz_h.copy_(y_nnz, non_blocking=True)
-            stream.synchronize()
-            kk = int(y_nnz_h.item())
-            y_idx_h[:kk].copy_(y_idx[:kk], non_blocking=True)
-            y_val_h[:kk].copy_(y_val[:kk], non_blocking=True)
+            B.dbspmspv_run(h, xh[k][0], xh[k][1], n_x, B.PLUS_TIMES, y_idx_h, y_val_h, a.m, y_nnz_h)
             e1.record(stream)
             stream.synchronize()
+            kk = int(y_nnz_h.item())
             tot += e0.elapsed_time(e1)
-            h2d += 8 * n_x
+            # x is read once by the blocking kernel; its indices once more by the clean-up pass
+            # unless the dense copy is cleared wholesale (x lists more than n / 8 columns)
+            h2d += 8 * n_x + (0 if 8 * n_x > a.n else 4 * n_x)
             d2h += 4 + 8 * kk
         if s >= 2:
             e2e_ms.append(tot)

@@ -187,9 +187,13 @@ int dbspmspv_create_coo(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nn
  *   semiring PLUS_TIMES (F32/BF16 handles) or OR_AND (any handle; values are then 1.0f)
  *   y_idx    out: row indices of the structural result, ascending; y_val out: fp32 sums
  *            (may be NULL for OR_AND); both with room for y_capacity entries
- *   y_nnz    out: one int32 on the device, the number of result entries (the full count even
- *            when it exceeds y_capacity; then only the first y_capacity are written and the
- *            deferred status is ERR_CAPACITY)
+ *   y_nnz    out: one int32, the number of result entries (the full count even when it
+ *            exceeds y_capacity; then only the first y_capacity are written and the deferred
+ *            status is ERR_CAPACITY)
+ * x_idx, x_val, y_idx, y_val and y_nnz are device pointers -- or page-locked host memory that
+ * the device addresses directly (cudaHostAlloc / cudaHostRegister under unified addressing):
+ * the call's kernels then read x and write y across the bus themselves, with no staging copy
+ * (x_idx is read a second time by the clean-up pass unless x lists more than n / 8 columns).
  * nnz_x = 0 gives y_nnz = 0.  Errors: INVALID_ARG, UNSUPPORTED synchronously.
  */
 int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
