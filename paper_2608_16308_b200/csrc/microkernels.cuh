@@ -233,15 +233,22 @@ __device__ __forceinline__ uint32_t warp_block_bool(int type, const uint8_t *blk
     return __reduce_or_sync(FULL, hm);
 }
 
-// Half-warp streaming form for runs of column-mask blocks (ForceCSC, column-major CSR, Dense):
-// the lane map of Algorithm 3 (lane = row), but the two half-warps take two different blocks, so
-// no cross-lane reduction is needed and a row's sum stays in a register while consecutive blocks
-// belong to the same row block.  Lane `row` of a half holds column mask, column start and x entry
-// number `row` of its block in registers; the column loop broadcasts them by shuffle, and up to
-// four columns' value loads are issued before their products are added, so several loads per
-// lane are in flight (two per round was measured 25 % slower: the kernel is latency bound).  The header of the next block pair is fetched before the current one is
-// worked on.  `emit(rb, row, sum)` is called by a lane when its row block changes and at the end.
-template <int DT, typename Emit>
+// Half-warp streaming form for runs of mask-based blocks: lane = row, and the two half-warps take
+// two different blocks, so no cross-lane reduction is needed and a row's sum stays in a register
+// while consecutive blocks belong to the same row block.  Lane `row` of a half holds mask, start
+// and x entry number `row` of its block in registers.
+//   column-major blocks (ForceCSC, CSR, Dense; the lane map of Algorithm 3): the half walks the
+//     active columns together; mask and start of a column are broadcast by shuffle and every
+//     lane picks its row's element of that column, if any;
+//   row-major blocks (ForceCSR, short-row CSR; Algorithm 2 with one lane per row): every lane
+//     walks the active entries of its own row; only the x entry comes by shuffle.
+// Up to four value loads are issued before their products are added, so several loads per lane
+// are in flight (two per round was measured 25 % slower: the walk is latency bound), and the
+// header of the next block pair is fetched before the current one is worked on.
+// One call takes blocks of one layout (ROWS: row-major), so the loop is specialised at compile
+// time and both halves stay converged.
+// `emit(rb, row, sum)` is called by a lane when its row block changes and at the end.
+template <int DT, bool ROWS, typename Emit>
 __device__ __forceinline__ void half_stream(const uint8_t *payload, const float *x_dense, uint32_t idx_l,
                                             uint32_t w_l, uint32_t xm_l, int rb_l, uint32_t todo, int lane,
                                             Emit emit) {
@@ -250,8 +257,8 @@ __device__ __forceinline__ void half_stream(const uint8_t *payload, const float 
     float sum = 0.f;
     bool touched = false;
     int srb = -1;
-    // header of one block for this lane: column mask | column start << 16, and x entry, of column `row`
-    auto fetch = [&](uint32_t rem, uint32_t &bxm, int &brb, bool &dense, const uint8_t *&vals,
+    // header of one block for this lane: mask | start << 16, and x entry, number `row`
+    auto fetch = [&](uint32_t rem, uint32_t &bxm, int &brb, int &kind, const uint8_t *&vals,
                      uint32_t &hdr, float &xr) -> uint32_t {
         const int l0 = __ffs(rem) - 1;
         rem &= rem - 1;
@@ -265,54 +272,78 @@ __device__ __forceinline__ void half_stream(const uint8_t *payload, const float 
         brb = __shfl_sync(FULL, rb_l, sl);
         if (src < 0) { bxm = 0u; brb = -1; }
         const uint8_t *blk = payload + (size_t)bw * 4;
-        dense = (bidx >> TYPE_SHIFT) == DBSPMSPV_BLK_DENSE;
-        vals = blk + (dense ? 32 : HDR_BYTES);
-        const uint32_t st = dense ? row * 16 : (Val<DT>::SIZE ? blk[32 + row] : 0);
+        const int type = bidx >> TYPE_SHIFT;
+        kind = type == DBSPMSPV_BLK_DENSE ? 2 : (is_row_major(type) ? 1 : 0);   // 0 column-major, 1 row-major, 2 dense
+        vals = blk + (kind == 2 ? 32 : HDR_BYTES);
+        const uint32_t st = kind == 2 ? row * 16 : (Val<DT>::SIZE ? blk[32 + row] : 0);
         hdr = reinterpret_cast<const uint16_t *>(blk)[row] | (st << 16);
         xr = x_dense[(size_t)(bidx & IDX_MASK) * 16 + row];
         return rem;
     };
-    bool dense;
+    int kind;
     uint32_t bxm, hdr;
     int brb;
     const uint8_t *vals;
     float xr;
-    uint32_t rem = fetch(todo, bxm, brb, dense, vals, hdr, xr);
+    uint32_t rem = fetch(todo, bxm, brb, kind, vals, hdr, xr);
     for (;;) {
         // prefetch the next pair while this one is processed
-        bool n_dense = false;
+        int n_kind = 0;
         uint32_t n_bxm = 0, n_hdr = 0, n_rem = 0;
         int n_brb = -1;
         const uint8_t *n_vals = vals;
         float n_xr = 0.f;
         const bool more = rem != 0;
-        if (more) n_rem = fetch(rem, n_bxm, n_brb, n_dense, n_vals, n_hdr, n_xr);
+        if (more) n_rem = fetch(rem, n_bxm, n_brb, n_kind, n_vals, n_hdr, n_xr);
         if (bxm && brb != srb) {
             if (touched) emit(srb, row, sum);
             sum = 0.f; touched = false; srb = brb;
         }
-        uint32_t a = bxm;
-        while (__any_sync(FULL, a != 0)) {
-            float v[4], xc[4];
+        if (ROWS) {
+            uint32_t a = hdr & 0xFFFFu & bxm;          // my row's entries under active columns
+            while (__any_sync(FULL, a != 0)) {
+                float v[4], xc[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const bool on = a != 0;
-                const int c = on ? __ffs(a) - 1 : 0;
-                a &= a - 1;                           // stays 0 once it is 0
-                const uint32_t hc = __shfl_sync(FULL, hdr, hb | c);
-                const float xs = __shfl_sync(FULL, xr, hb | c);
-                xc[j] = 0.f;                          // (an inactive column's x is the NaN marker)
-                v[j] = 0.f;
-                if (on && ((hc >> row) & 1u)) {
-                    xc[j] = xs;
-                    v[j] = Val<DT>::load(vals, (hc >> 16) + (dense ? row : __popc(hc & below_row)));
-                    touched = true;
+                for (int j = 0; j < 4; ++j) {
+                    const bool on = a != 0;
+                    const int c = on ? __ffs(a) - 1 : 0;
+                    a &= a - 1;                           // stays 0 once it is 0
+                    const float xs = __shfl_sync(FULL, xr, hb | c);
+                    xc[j] = 0.f;
+                    v[j] = 0.f;
+                    if (on) {
+                        xc[j] = xs;
+                        v[j] = Val<DT>::load(vals, (hdr >> 16) + __popc(hdr & 0xFFFFu & below(c)));
+                        touched = true;
+                    }
                 }
+                sum += (v[0] * xc[0] + v[1] * xc[1]) + (v[2] * xc[2] + v[3] * xc[3]);
             }
-            sum += (v[0] * xc[0] + v[1] * xc[1]) + (v[2] * xc[2] + v[3] * xc[3]);
+        } else {
+            const bool dense = kind == 2;
+            uint32_t a = bxm;                          // the active columns
+            while (__any_sync(FULL, a != 0)) {
+                float v[4], xc[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool on = a != 0;
+                    const int c = on ? __ffs(a) - 1 : 0;
+                    a &= a - 1;
+                    const uint32_t hc = __shfl_sync(FULL, hdr, hb | c);
+                    const float xs = __shfl_sync(FULL, xr, hb | c);
+                    xc[j] = 0.f;                          // (an inactive column's x is the NaN marker)
+                    v[j] = 0.f;
+                    if (on && ((hc >> row) & 1u)) {
+                        xc[j] = xs;
+                        v[j] = Val<DT>::load(vals, (hc >> 16) + (dense ? row : __popc(hc & below_row)));
+                        touched = true;
+                    }
+                }
+                sum += (v[0] * xc[0] + v[1] * xc[1]) + (v[2] * xc[2] + v[3] * xc[3]);
+            }
         }
         if (!more) break;
-        rem = n_rem; bxm = n_bxm; brb = n_brb; dense = n_dense; vals = n_vals; hdr = n_hdr; xr = n_xr;
+        rem = n_rem; bxm = n_bxm; brb = n_brb; kind = n_kind; vals = n_vals; hdr = n_hdr; xr = n_xr;
     }
     if (touched) emit(srb, row, sum);
 }

@@ -212,11 +212,12 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
     // A task is a chain of dependent loads (record -> entries, column end, mask, x block); the
     // loop is software-pipelined: while task k is evaluated, the loads of k+1 and the record of
     // k+2 (in this warp's stride) are in flight.
-    struct Loads { uint32_t idx, w, aux, xm; float xv; int start, end; };
+    struct Loads { uint32_t idx, w, aux, xm; float xv; int start, end, jb; };
     auto loads_of = [&](int t, const uint2 &task) {
-        Loads l{0u, 0u, 0u, 0u, 0.f, 0, 0};
+        Loads l{0u, 0u, 0u, 0u, 0.f, 0, 0, 0};
         if (t < n_tasks) {
             const int jb = (int)(task.x & IDX_MASK);
+            l.jb = jb;
             const int upper = ((int)(task.x >> 27) + 1) * 4;      // entries of the task, rounded up to 4
             l.start = (int)task.y;
             if (lane < upper) { const int p = l.start + lane; l.idx = d.csc.idx[p]; l.w = d.csc.w[p]; l.aux = d.csc.aux[p]; }
@@ -234,7 +235,7 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
         const Loads nxt = loads_of(t + nwarps, rec1);
         rec1 = rec2;
         uint32_t idx[U] = {cur.idx}, w[U] = {cur.w}, aux[U] = {cur.aux};
-        const int start = cur.start, end = cur.end;
+        const int start = cur.start, end = cur.end, jb = cur.jb;
         const uint32_t xm = cur.xm;
         if (lane < 16) s_x[lane] = cur.xv;
         cur = nxt;
@@ -271,6 +272,25 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                 __syncwarp();
                 if (Out::MASKS && coo_cnt && s_hit[lane]) mark_rows(out.hit8, brow, s_hit[lane]);
                 __syncwarp();
+            }
+            // dense vector block and several mask-based blocks in the step: half-warp streaming
+            // form (two blocks per warp at a time, next pair prefetched; a warp that takes one
+            // block at a time waits out two dependent loads per block)
+            if (HV && DT != DBSPMSPV_PATTERN && __popc(xm) >= popc_threshold) {
+                const bool mk = heavy && type != DBSPMSPV_BLK_COO;
+                const uint32_t cs = __ballot_sync(FULL, mk);
+                if (__popc(cs) >= HEAVY_LANE_MIN) {
+                    auto emit = [&](int erb, int erow, float esum) {
+                        atomicAdd(out.acc + (size_t)erb * 16 + erow, esum);
+                        if (Out::MASKS) out.hit8[(size_t)erb * 16 + erow] = 1;
+                    };
+                    const uint32_t rows = __ballot_sync(FULL, mk && is_row_major(type));
+                    const uint32_t tagged = (idx[u] & ~IDX_MASK) | (uint32_t)jb;     // class bits + the task's column block
+                    if (cs & ~rows) half_stream<DT, false>(d.payload, d.ws.x_dense, tagged, w[u], xm, brow, cs & ~rows, lane, emit);
+                    if (rows) half_stream<DT, true>(d.payload, d.ws.x_dense, tagged, w[u], xm, brow, rows, lane, emit);
+                    if (mk) heavy = false;
+                    __syncwarp();
+                }
             }
             uint32_t hv = __ballot_sync(FULL, heavy);
             // sparse local mask -> lane-owned form; dense local mask -> warp form (Section 3.3.3:
@@ -498,22 +518,24 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
                     if (Out::MASKS && coo_cnt && s_hit[lane]) mark_rows(out.hit8, rb, s_hit[lane]);
                     __syncwarp();
                 }
-                // runs of column-mask blocks (pruned layers): half-warp streaming form
+                // runs of mask-based blocks (pruned layers, banded matrices): half-warp streaming form
                 if (HV && DT != DBSPMSPV_PATTERN) {
-                    const bool colmask = heavy && (type == DBSPMSPV_BLK_FCSC || type == DBSPMSPV_BLK_CSR || type == DBSPMSPV_BLK_DENSE);
-                    const uint32_t cs = __ballot_sync(FULL, colmask);
+                    const bool mk = heavy && type != DBSPMSPV_BLK_COO;
+                    const uint32_t cs = __ballot_sync(FULL, mk);
                     if (__popc(cs) >= HEAVY_LANE_MIN) {
-                        half_stream<DT>(d.payload, d.ws.x_dense, idx[u], w[u], xm, rb, cs, lane,
-                                        [&](int erb, int erow, float esum) {
-                                            if (erb == cur_rb) {
-                                                atomicAdd(&my_y[erow], esum);
-                                                hit |= 1u << erow;
-                                            } else {
-                                                atomicAdd(out.acc + (size_t)erb * 16 + erow, esum);
-                                                if (Out::MASKS) out.hit8[(size_t)erb * 16 + erow] = 1;
-                                            }
-                                        });
-                        if (colmask) heavy = false;
+                        auto emit = [&](int erb, int erow, float esum) {
+                            if (erb == cur_rb) {
+                                atomicAdd(&my_y[erow], esum);
+                                hit |= 1u << erow;
+                            } else {
+                                atomicAdd(out.acc + (size_t)erb * 16 + erow, esum);
+                                if (Out::MASKS) out.hit8[(size_t)erb * 16 + erow] = 1;
+                            }
+                        };
+                        const uint32_t rows = __ballot_sync(FULL, mk && is_row_major(type));
+                        if (cs & ~rows) half_stream<DT, false>(d.payload, d.ws.x_dense, idx[u], w[u], xm, rb, cs & ~rows, lane, emit);
+                        if (rows) half_stream<DT, true>(d.payload, d.ws.x_dense, idx[u], w[u], xm, rb, rows, lane, emit);
+                        if (mk) heavy = false;
                         __syncwarp();
                     }
                 }
