@@ -319,7 +319,10 @@ __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
 }
 
 // ---- pull segments (Section 3.3.2): greedy walk along each row block; a segment closes
-// when its accumulated weight reaches the cut.  One thread per row block, two passes.
+// when its accumulated weight reaches the cut.  One warp per row block (hub row blocks hold
+// 10^5 entries: a single thread walking them took tens of milliseconds), two passes.  The warp
+// takes 32 entries per step: a scan of their weights, then the cuts inside the step one after
+// the other (each restarts the running weight at zero).
 struct SegParams { int cut, w_dense, w_mid, w_coo, w_inline; };
 
 __device__ __forceinline__ int seg_weight(uint32_t idx, const SegParams &sp) {
@@ -327,41 +330,65 @@ __device__ __forceinline__ int seg_weight(uint32_t idx, const SegParams &sp) {
     return t == DBSPMSPV_BLK_DENSE ? sp.w_dense : t == DBSPMSPV_BLK_INLINE ? sp.w_inline : t == DBSPMSPV_BLK_COO ? sp.w_coo : sp.w_mid;
 }
 
+// Calls close(first, end_exclusive, weight) -- by every lane, with warp-uniform arguments --
+// for each segment of row block rb, in order.
+template <typename Close>
+__device__ __forceinline__ void seg_walk(int begin, int end, const uint32_t *idx, const SegParams &sp, int lane, Close close) {
+    int acc = 0, first = begin;
+    for (int base = begin; base < end; base += 32) {
+        const int p = base + lane;
+        const int w = p < end ? seg_weight(idx[p], sp) : 0;
+        int incl = w;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        int removed = 0;      // weight of this step already closed into segments
+        for (;;) {
+            const uint32_t m = __ballot_sync(0xFFFFFFFFu, p < end && incl > removed && acc + incl - removed >= sp.cut);
+            if (!m) break;
+            const int l = __ffs(m) - 1;
+            const int upto = __shfl_sync(0xFFFFFFFFu, incl, l);
+            close(first, base + l + 1, acc + upto - removed);
+            first = base + l + 1;
+            removed = upto;
+            acc = 0;
+        }
+        acc += __shfl_sync(0xFFFFFFFFu, incl, 31) - removed;
+    }
+    if (first < end) close(first, end, acc);
+}
+
 __global__ void k_seg_count(int32_t mb, const int32_t *row_ptr, const uint32_t *idx,
                             SegParams sp, int32_t *count) {
-    int64_t rb = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t rb = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
     if (rb >= mb) return;
-    int acc = 0, c = 0;
-    for (int p = row_ptr[rb]; p < row_ptr[rb + 1]; ++p) {
-        acc += seg_weight(idx[p], sp);
-        if (acc >= sp.cut) { ++c; acc = 0; }
-    }
-    if (acc > 0) ++c;
-    count[rb] = c;
+    int c = 0;
+    seg_walk(row_ptr[rb], row_ptr[rb + 1], idx, sp, lane, [&](int, int, int) { ++c; });
+    if (lane == 0) count[rb] = c;
 }
 
 __global__ void k_seg_write(int32_t mb, const int32_t *row_ptr, uint32_t *idx,
                             SegParams sp, const int32_t *seg_off, Segment *segs, int32_t *seg_rb) {
-    int64_t rb = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t rb = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
     if (rb >= mb) return;
-    int acc = 0, first = row_ptr[rb];
-    const int end = row_ptr[rb + 1];
+    const int begin = row_ptr[rb], end = row_ptr[rb + 1];
     int o = seg_off[rb];
-    for (int p = first; p < end; ++p) {
-        acc += seg_weight(idx[p], sp);
-        if (acc >= sp.cut || p + 1 == end) {
+    seg_walk(begin, end, idx, sp, lane, [&](int first, int stop, int weight) {
+        if (lane == 0) {
             Segment s;
             s.row_block = (int32_t)rb;
             s.start = first;
-            s.count = (p + 1 - first) | ((first == row_ptr[rb] && p + 1 == end) ? (int32_t)0x80000000 : 0);
-            s.weight = acc;
+            s.count = (stop - first) | ((first == begin && stop == end) ? (int32_t)0x80000000 : 0);
+            s.weight = weight;
             seg_rb[o] = (int32_t)rb;
-            segs[o++] = s;
+            segs[o] = s;
             idx[first] |= 1u << 28;   // first entry of a segment (bits 27, 28 of idx are spare)
-            first = p + 1;
-            acc = 0;
         }
-    }
+        ++o;
+    });
 }
 
 // pull chunks: consecutive segments grouped by accumulated weight; chunk k starts at the first
@@ -605,14 +632,14 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         int32_t *cnt, *off;
         DBS_GET(cnt, (int64_t)d.mb + 1); DBS_GET(off, (int64_t)d.mb + 1);
         DBS_CUDA(cudaMemsetAsync(cnt, 0, ((size_t)d.mb + 1) * 4, st));
-        k_seg_count<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, cnt);
+        k_seg_count<<<grid_for((int64_t)d.mb * 32), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, cnt);
         DBS_TRY(exclusive_sum(tp, cnt, off, (int64_t)d.mb + 1, st));
         int32_t nseg = 0;
         DBS_CUDA(cudaMemcpy(&nseg, off + d.mb, 4, cudaMemcpyDeviceToHost));
         d.n_segments = nseg;
         Segment *segs; DBS_KEEP(segs, nseg);
         int32_t *seg_rb; DBS_KEEP(seg_rb, (int64_t)nseg + 1);
-        k_seg_write<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, off, segs, seg_rb);
+        k_seg_write<<<grid_for((int64_t)d.mb * 32), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, off, segs, seg_rb);
         d.seg_rb = seg_rb;
         d.segments = segs;
         int32_t *segw, *segpre;
