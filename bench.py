@@ -1,12 +1,12 @@
 """Benchmark of the DB-SpMSpV hot path on B200.
 
-Workload at N=1 (benchmark configs[1]): R-MAT scale 20, edge factor 16, fp32 values, with the
+Workload at N=1: R-MAT scale 20, edge factor 16, fp32 values, with the
 input-sparsity sweep x nnz fraction 1e-5 ... 0.5.  One *step* is one pass of the whole hot path
 (vector blocking -> selector -> worklist -> block microkernels -> writeback -> compaction) over
 that batch: one dbspmspv_run call per sweep point, six calls.  L2 is flushed before every timed
-call, so every number is cold.  `value` is the bytes the method must touch (B_touch)
-summed over the sweep, divided by the summed device time.  DB-BFS GTEPS (configs[3]) is reported
-in `bfs` unless --no-bfs is given.
+call, so every number is cold.  `value` is the bytes the method must touch (B_touch, defined at
+ByteModel below) summed over the sweep, divided by the summed device time.  DB-BFS GTEPS on the
+symmetrised R-MAT scale 22 graph is reported in `bfs` unless --no-bfs is given.
 
 python bench.py [--gpus N --steps K --warmup W] [--impl reference] [--no-bfs]
 Under torchrun every rank runs the same sweep on its own GPU (independent replicas: the path
@@ -37,7 +37,7 @@ VIEW_ENTRY_BYTES = 9          # idx 4 + w 4 + aux 1 per view entry
 
 
 # ---------------------------------------------------------------------------------------------
-# Algorithmic bytes (host, from the structure of A and x; documented in the design doc)
+# Algorithmic bytes (host, from the structure of A and x)
 # ---------------------------------------------------------------------------------------------
 def payload_bytes_per_entry(cls: np.ndarray, nnz: np.ndarray, vsize: int) -> np.ndarray:
     """Payload bytes of every view entry from the documented per-class sizes."""
@@ -51,7 +51,13 @@ def payload_bytes_per_entry(cls: np.ndarray, nnz: np.ndarray, vsize: int) -> np.
 
 
 class ByteModel:
-    """B_touch and B_min of one call (SpMSpV): see the design doc, 'Algorithmic bytes'."""
+    """Algorithmic bytes of one SpMSpV call, each distinct byte once.
+    B_touch: what the method must touch -- the view entries (9 bytes each) and payloads of the
+    blocks in active column blocks, a column-pointer pair per active column block, x (8 bytes per
+    listed nonzero, plus mask and staged block per nonempty vector block), y (8 bytes out and an
+    8-byte accumulator read-modify-write per output, 8 bytes of hit flags per touched row block).
+    B_min: the information-theoretic floor of a plain CSC gather -- per listed x_j its column's
+    entries at (value + 4-byte row) each plus a pointer pair, x and y once."""
 
     def __init__(self, csr: wl.CSR, entry_col: np.ndarray, entry_cls: np.ndarray, entry_nnz: np.ndarray,
                  vsize: int):
