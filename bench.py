@@ -181,9 +181,9 @@ def host_byte_model(a: wl.CSR) -> ByteModel:
     key = (rows.astype(np.int64) >> 4) * ((a.n + 15) // 16) + (a.col_idx >> 4)
     ub, cnt = np.unique(key, return_counts=True)
     bcol = (ub % ((a.n + 15) // 16)).astype(np.int64)
-    # hypersparse matrices: blocks with <= 4 entries are INLINE (one 9-byte entry per element),
-    # 5..31 COO; the handful of denser blocks are counted as CSR-class
-    inl = cnt <= 4
+    # blocks with fewer than 32 entries are INLINE (one 9-byte view entry per element, the
+    # library's default); the handful of denser blocks are counted as CSR-class or Dense
+    inl = cnt < 32
     cls = np.where(inl, 0, np.where(cnt < 32, 1, np.where(cnt > 128, 5, 4))).astype(np.int32)
     ecol = np.concatenate([np.repeat(bcol[inl], cnt[inl]), bcol[~inl]])
     ecls = np.concatenate([np.zeros(int(cnt[inl].sum()), np.int32), cls[~inl]])
@@ -384,6 +384,10 @@ def main() -> None:
         line["cpu_baseline"] = cpu_baseline(a, xs, model)
     if rank == 0 and world == 1 and not args.no_bfs:
         try:
+            line["other_configs"] = other_configs(B, torch, dev, flush, peak)
+        except Exception as e:
+            line["other_configs"] = {"error": repr(e)}
+        try:
             line["bfs"] = bench_bfs(args, B, torch, dev, flush)
         except Exception as e:  # the SpMSpV line must survive a BFS-side problem
             line["bfs"] = {"error": repr(e)}
@@ -396,7 +400,7 @@ def main() -> None:
 
 # DRAM traffic of that launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
 # summarised in profiles/k_compute_pull_rmat20_x50pct.txt
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 157396480
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 157449984
 
 
 def crossover_table() -> None:
@@ -449,6 +453,75 @@ def crossover_table() -> None:
             tp, tl = timed(h, x, mat.m, B.PATH_PUSH), timed(h, x, mat.m, B.PATH_PULL)
             print(f"| {name} | {label} | {sb:.4f} | {tp:.1f} | {tl:.1f} | {'push' if tp < tl else 'pull'} |")
         B.dbspmspv_destroy(h)
+
+
+def other_configs(B, torch, dev, flush, peak):
+    """The remaining workload shapes, one record each (whole call, cold L2, median of 12 after 3
+    warm-ups): the uniform matrix with a 1 % x, the 27-point stencil with clustered x at 0.1 %
+    and 5 %, and single-token decode on three pruned layer shapes next to a dense bf16 GEMV of
+    the same shape on the same box."""
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    out = []
+
+    def timed(fn):
+        ts = []
+        for it in range(15):
+            flush.fill_(it)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts[3:]))
+
+    def spmspv_case(name, a, xs):
+        h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(a.val), B.F32)
+        ne = int(B.dbspmspv_get_stats(h).n_view_entries)
+        e_col = torch.empty(ne, dtype=torch.int32, device=dev)
+        e_cls = torch.empty(ne, dtype=torch.int32, device=dev)
+        e_nnz = torch.empty(ne, dtype=torch.int32, device=dev)
+        B.dbspmspv_export_blocks(h, None, e_col, e_cls, e_nnz)
+        model = ByteModel(a, e_col.cpu().numpy().astype(np.int64), e_cls.cpu().numpy(), e_nnz.cpu().numpy().astype(np.int64), 4)
+        y_idx = torch.empty(a.m, dtype=torch.int32, device=dev)
+        y_val = torch.empty(a.m, dtype=torch.float32, device=dev)
+        y_nnz = torch.zeros(1, dtype=torch.int32, device=dev)
+        for label, x in xs:
+            xi, xv = up(x.idx), up(x.val)
+            us = timed(lambda: B.dbspmspv_run(h, xi, xv, int(x.idx.size), B.PLUS_TIMES, y_idx, y_val, a.m, y_nnz))
+            st = B.dbspmspv_get_stats(h)
+            k = int(y_nnz.item())
+            yrb = int(np.unique(y_idx[:k].cpu().numpy() >> 4).size)
+            bt = model.bytes(x.idx, k, yrb)[0]
+            out.append({"workload": name, "x": label, "path": "push" if st.last_path == B.PATH_PUSH else "pull",
+                        "us": round(us, 2), "y_nnz": k, "B_touch": int(bt), "GBps_touch": round(bt / us / 1e3, 2),
+                        "frac_of_peak_touch": round(bt / us / 1e3 / peak, 4)})
+        B.dbspmspv_destroy(h)
+
+    a1 = wl.uniform_rows()
+    spmspv_case("uniform16384_8perrow_fp32", a1, [("164 nnz (1 %)", wl.sparse_x(0, 1, a1.n, 164))])
+    a3 = wl.stencil27(160, seed=2)
+    spmspv_case("stencil27_160cubed_fp32", a3, [("0.1 % in runs of 64", wl.clustered_x(a3.n, 64)),
+                                                 ("5 % in runs of 64", wl.clustered_x(a3.n, 3200))])
+    del a3
+    for (m, n) in wl.DECODE_SHAPES:
+        wgt = wl.pruned_weight(m, n, 0.5)
+        bits = wl.f32_to_bf16_bits(wgt.val).view(np.int16)
+        h = B.dbspmspv_create_csr(wgt.m, wgt.n, wgt.nnz, up(wgt.row_ptr), up(wgt.col_idx), up(bits), B.BF16)
+        x = wl.relu_activation(n, 0.7)
+        xd = up(wl.f32_to_bf16_bits(x).view(np.int16))
+        y = torch.empty(m, dtype=torch.float32, device=dev)
+        us = timed(lambda: B.dbspmspv_decode(h, xd, y))
+        st = B.dbspmspv_get_stats(h)
+        wd = torch.randn(m, n, device=dev, dtype=torch.bfloat16)
+        xb = torch.randn(n, device=dev, dtype=torch.bfloat16)
+        gemv = timed(lambda: torch.mv(wd, xb))
+        out.append({"workload": f"decode_{m}x{n}_bf16_prune50_act70zero", "path": "push" if st.last_path == B.PATH_PUSH else "pull",
+                    "us": round(us, 2), "dense_bf16_gemv_us_same_box": round(gemv, 2),
+                    "format_bytes": int(st.payload_bytes + st.csr_view_bytes)})
+        B.dbspmspv_destroy(h)
+        del wd
+    return out
 
 
 def cusparse_reference(a, torch, dev, flush):

@@ -57,6 +57,7 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
 // 16-bit masks of its two vector blocks.  Also clears the dense output.
 template <int DT>
 __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__restrict__ y) {
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int64_t padded = (int64_t)((d.nb + 1) / 2) * 32;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -804,6 +805,7 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
 }
 
 __global__ void k_decode_cleanup(Device d) {
+    pdl_wait();
     const int n_words = (d.nb + 1) / 2;
     const int stride = gridDim.x * blockDim.x;
     for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n_words; k += stride) d.ws.x_mask32[k] = 0u;
@@ -946,15 +948,15 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
     OutDense out{y, nullptr};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
     if (d.n_entries > 0) {
-        const int s = h->heavy_stage ? launch_compute<DT, OutDense, 1>(h, out, h->ropts.th3_decode, false, st)
-                                     : launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, false, st);
+        const int s = h->heavy_stage ? launch_compute<DT, OutDense, 1>(h, out, h->ropts.th3_decode, true, st)
+                                     : launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, true, st);
         if (s != DBSPMSPV_OK) return s;
     }
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
     h->kernel_launches += 2;
     int gc = ((d.nb + 1) / 2 + 255) / 256;
     if (gc > h->sm_count) gc = h->sm_count;
-    k_decode_cleanup<<<gc, 256, 0, st>>>(d);
+    DBS_CUDA(launch_pdl(k_decode_cleanup, gc, 256, 0, st, d));
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }
