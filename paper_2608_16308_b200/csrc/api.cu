@@ -186,7 +186,7 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     dbs::Device &d = h->d;
     cudaDeviceSynchronize();
     cudaFree(d.csr.ptr); cudaFree(d.csr.idx); cudaFree(d.csr.w); cudaFree(d.csr.aux);
-    cudaFree(d.csc.ptr); cudaFree(d.csc.idx); cudaFree(d.csc.w); cudaFree(d.csc.aux);
+    cudaFree(d.csc.ptr); cudaFree(d.csc.idx); cudaFree(d.csc.w); cudaFree(d.csc.aux); cudaFree(d.csc.colptr);
     cudaFree(h->payload_alloc);
     cudaFree(const_cast<dbs::Segment *>(d.segments));
     cudaFree(const_cast<int2 *>(d.chunks));

@@ -58,12 +58,9 @@ __device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int dept
         Entries e{0u, 0u, 0u, 0};
         if (t < n_tasks) {
             const int jb = (int)(task.x & IDX_MASK), start = (int)task.y;
-            // the record holds ceil(n / 4) - 1: load under that bound (the view arrays are padded),
-            // the exact end comes from the column pointer
-            const int approx = (int)((task.x >> 27) + 1) * 4;
-            if (lane < approx) { e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane]; }
+            e.n = (int)(task.x >> 27) + 1;
+            if (lane < e.n) { e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane]; }
             e.xm = mask_of(d.ws.x_mask32, jb);
-            e.n = min(PUSH_CHUNK, d.csc.ptr[jb + 1] - start);
         }
         return e;
     };
@@ -268,7 +265,10 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
             d.ws.x_mask32[jb >> 1] = bit;
             d.ws.visited32[jb >> 1] |= bit;
         }
-        emit_tasks(d, lane == 0, jb, lane, &ctr->bfs_cnt[0][1], &ctr->bfs_cnt[0][0]);
+        int first = 0, deg = 0;
+        if (lane == 0) column_run(d, src, first, deg);
+        else if (lane == 1) payload_run(d, jb, first, deg);
+        emit_tasks(d, lane == 0, jb, first, deg, lane, &ctr->bfs_cnt[0][1], &ctr->bfs_cnt[0][0]);
     }
     grid.sync();
 
@@ -311,11 +311,31 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         // known now); its block count goes to a scratch counter
         const int next_n = ctr->bfs_cnt[cur ^ 1][0];
         if (next_n && bfs_path(next_n, d.nb, th3, force_path) == DBSPMSPV_PATH_PUSH) {
+            // lane l of a warp step takes vector block 64 * step + l and then + 32: first the
+            // block's entries with a payload, then the INLINE run of every frontier column
             for (int k0 = (tid & ~31); k0 < n_words; k0 += nthreads) {
-                const int k = k0 + lane;
-                const uint32_t nm = k < n_words ? d.ws.x_mask32[k] : 0u;
-                emit_tasks(d, (nm & 0xFFFFu) != 0, 2 * k, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad);
-                emit_tasks(d, (nm >> 16) != 0, 2 * k + 1, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad);
+                const uint32_t word = k0 + (lane >> 1) < n_words ? d.ws.x_mask32[k0 + (lane >> 1)] : 0u;
+                const uint32_t word2 = k0 + 16 + (lane >> 1) < n_words ? d.ws.x_mask32[k0 + 16 + (lane >> 1)] : 0u;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int jb = 2 * k0 + 32 * half + lane;
+                    uint32_t m = ((half ? word2 : word) >> ((lane & 1) * 16)) & 0xFFFFu;
+                    int first = 0, deg = 0;
+                    if (m) payload_run(d, jb, first, deg);
+                    if (__any_sync(FULL, deg > 0)) emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad, d.payload_chunk);
+                    while (__any_sync(FULL, m != 0)) {     // one run of consecutive frontier columns at a time
+                        first = 0; deg = 0;
+                        if (m) {
+                            const int c0 = __ffs(m) - 1;
+                            const int len = __ffs(~(m >> c0)) - 1;
+                            const int32_t *cp = d.csc.colptr + 17 * jb + c0;
+                            first = cp[0];
+                            deg = cp[len] - first;
+                            m &= ~(((1u << len) - 1u) << c0);
+                        }
+                        emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad);
+                    }
+                }
             }
             grid.sync();
         }

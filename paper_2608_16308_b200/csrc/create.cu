@@ -296,12 +296,33 @@ __global__ void k_lower_bounds(int32_t count, const int32_t *sorted, int32_t n, 
     ptr[v] = lo;
 }
 
+// Sort key of the block-CSC view: column block (27 bits) | group (5 bits: 0 = entry with a
+// payload, 16 + c = INLINE element of local column c) | row block (27 bits) | local row (4 bits).
+constexpr int CSC_KEY_GROUP_SHIFT = 31, CSC_KEY_COL_SHIFT = 36;
 __global__ void k_csc_keys(int32_t n_entries, const int32_t *entry_row, const uint32_t *csr_idx,
-                           uint64_t *keys, int32_t *ids) {
+                           const uint8_t *csr_aux, uint64_t *keys, int32_t *ids) {
     int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (b >= n_entries) return;
-    keys[b] = ((uint64_t)(csr_idx[b] & IDX_MASK) << 27) | (uint64_t)entry_row[b];
+    const uint32_t idx = csr_idx[b];
+    const bool inl = (idx >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE;
+    const uint32_t rc = csr_aux[b];
+    const uint64_t group = inl ? 16u + (rc & 15u) : 0u, r = inl ? rc >> 4 : 0u;
+    keys[b] = ((uint64_t)(idx & IDX_MASK) << CSC_KEY_COL_SHIFT) | (group << CSC_KEY_GROUP_SHIFT) |
+              ((uint64_t)entry_row[b] << 4) | r;
     ids[b] = (int32_t)b;
+}
+
+// colptr[17 * jb + k], k = 0..16: first position whose (column block, group) is >= (jb, 16 + k)
+__global__ void k_csc_colptr(int32_t nb, const uint64_t *keys_sorted, int32_t n, int32_t *colptr) {
+    int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (t >= (int64_t)nb * 17) return;
+    const uint64_t target = ((uint64_t)(t / 17) << 5) + (uint64_t)(16 + t % 17);   // k = 16: the next column block
+    int32_t lo = 0, hi = n;
+    while (lo < hi) {
+        int32_t mid = lo + ((hi - lo) >> 1);
+        if ((keys_sorted[mid] >> CSC_KEY_GROUP_SHIFT) < target) lo = mid + 1; else hi = mid;
+    }
+    colptr[t] = lo;
 }
 
 __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
@@ -312,10 +333,10 @@ __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
     if (p >= n_blocks) return;
     int32_t b = csc2csr[p];
     uint64_t k = keys_sorted[p];
-    csc_idx[p] = (uint32_t)(k & IDX_MASK) | (csr_idx[b] & ~IDX_MASK);
+    csc_idx[p] = (uint32_t)((k >> 4) & IDX_MASK) | (csr_idx[b] & ~IDX_MASK);
     csc_w[p] = csr_w[b];
     csc_aux[p] = csr_aux[b];
-    bcol_sorted[p] = (int32_t)(k >> 27);
+    bcol_sorted[p] = (int32_t)(k >> CSC_KEY_COL_SHIFT);
 }
 
 // ---- pull segments (Section 3.3.2): greedy walk along each row block; a segment closes
@@ -580,6 +601,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     }
     DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_entries + VIEW_PAD); DBS_KEEP(d.csr.w, n_entries + VIEW_PAD); DBS_KEEP(d.csr.aux, n_entries + VIEW_PAD);
     DBS_CUDA(cudaMemsetAsync(d.csr.idx + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.aux + n_entries, 0, VIEW_PAD, st));
+    DBS_KEEP(d.csc.colptr, (int64_t)d.nb * 17); d.csr.colptr = nullptr;
     DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_entries + VIEW_PAD); DBS_KEEP(d.csc.w, n_entries + VIEW_PAD); DBS_KEEP(d.csc.aux, n_entries + VIEW_PAD);
     DBS_CUDA(cudaMemsetAsync(d.csc.idx + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csc.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csc.aux + n_entries, 0, VIEW_PAD, st));
     DBS_KEEP(h->csc2csr, n_entries);
@@ -596,20 +618,21 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     tp.release(ukey); tp.release(uval); tp.release(blk_start); tp.release(poff); tp.release(psize);
     tp.release(brow); tp.release(bcol); tp.release(ecount); tp.release(eoff); tp.release(type);
 
-    // block-CSC view: sort the primary entries by (column block, row block); the radix sort is
-    // stable, so the entries of one block stay together and in order
+    // block-CSC view: sort the primary entries by column block, and inside it payload entries
+    // first (by row block), then the INLINE elements column by column
     {
         uint64_t *k2, *k2_alt;
         int32_t *ids, *ids_alt, *bcol_sorted;
         DBS_GET(k2, n_entries); DBS_GET(k2_alt, n_entries); DBS_GET(ids, n_entries); DBS_GET(ids_alt, n_entries);
         DBS_GET(bcol_sorted, n_entries);
         if (n_entries) {
-            k_csc_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, h->block_row, d.csr.idx, k2, ids);
-            DBS_TRY(sort_pairs(tp, k2, k2_alt, ids, ids_alt, (int64_t)n_entries, 27 + bits_for((uint64_t)d.nb), st));
+            k_csc_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, h->block_row, d.csr.idx, d.csr.aux, k2, ids);
+            DBS_TRY(sort_pairs(tp, k2, k2_alt, ids, ids_alt, (int64_t)n_entries, CSC_KEY_COL_SHIFT + bits_for((uint64_t)d.nb), st));
             DBS_CUDA(cudaMemcpyAsync(h->csc2csr, ids, (size_t)n_entries * 4, cudaMemcpyDeviceToDevice, st));
             k_csc_gather<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, k2, h->csc2csr, d.csr.idx, d.csr.w, d.csr.aux, d.csc.idx, d.csc.w, d.csc.aux, bcol_sorted);
         }
         k_lower_bounds<<<grid_for(d.nb + 1), TPB, 0, st>>>(d.nb, bcol_sorted, n_entries, d.csc.ptr);
+        k_csc_colptr<<<grid_for((int64_t)d.nb * 17), TPB, 0, st>>>(d.nb, k2, n_entries, d.csc.colptr);
         DBS_CUDA(cudaStreamSynchronize(st));
         tp.release(k2); tp.release(k2_alt); tp.release(ids); tp.release(ids_alt); tp.release(bcol_sorted);
     }
@@ -664,7 +687,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     s.payload_bytes = h->payload_bytes;
     s.n_view_entries = d.n_entries;
     s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)d.n_entries * 9;
-    s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.n_entries * 9;
+    s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.nb * 17 * 4 + (int64_t)d.n_entries * 9;
     s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment) + ((int64_t)d.n_chunks + 1) * 8 + (int64_t)d.n_segments * 4;
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;

@@ -26,6 +26,8 @@ namespace dbs {
 // A packed local coordinate is one byte: (row << 4) | col.
 // Both views carry the same (w, aux) for a block, so either traversal direction reaches the
 // payload in one hop; the payload itself is stored once, in block-CSR ("primary") order.
+// The block-CSR view is ordered by (row block, column block, local row, local column); the
+// block-CSC view by column block, and inside it as described at View::colptr.
 //
 // Payload per class (V = value size: 4 fp32, 2 bf16, 0 pattern; every block starts on a
 // 16-byte boundary and is padded to a multiple of 16 bytes):
@@ -52,6 +54,7 @@ constexpr int TYPE_SHIFT = 29;
 #define DBS_PUSH_CHUNK 32
 #endif
 constexpr int PUSH_CHUNK = DBS_PUSH_CHUNK;   // CSC-view entries per push task (32 per warp step)
+static_assert(PUSH_CHUNK == 32, "a push task is one warp step; its record stores the exact entry count in 5 bits");
 constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-class block
 
 // Payload size in 4-byte words; every block is padded to 16 bytes so that it can be moved with
@@ -72,6 +75,13 @@ struct View {
     uint32_t *idx;   // n_entries
     uint32_t *w;     // n_entries
     uint8_t *aux;    // n_entries
+    // Block-CSC view only.  Inside a column block the entries are ordered: first the block
+    // entries with a payload (by row block), then the INLINE elements column by column (by row).
+    // colptr[17 * jb + c], c = 0..16, delimits them: the payload run is [ptr[jb], colptr[17 jb]),
+    // the INLINE elements of local column c are [colptr[17 jb + c], colptr[17 jb + c + 1]), and
+    // colptr[17 jb + 16] = ptr[jb + 1].  A push therefore visits only the elements of the columns
+    // x actually lists, not every element of an active column block.
+    int32_t *colptr;
 };
 
 struct Segment {     // pull work unit: a run of consecutive view entries inside one row block
@@ -137,6 +147,7 @@ struct Device {           // everything the kernels need, passed by value
     const int32_t *seg_rb;  // row block of every segment (compact copy for the pull kernel)
     const int2 *chunks;   // n_chunks + 1: {first segment, first entry} of every pull chunk
     int32_t n_chunks;
+    int32_t payload_chunk;  // entries with a payload per push task (see allocate_workspace)
     const uint32_t *row_present32;  // per row block: rows that hold a stored element (two 16-bit masks per word)
     Workspace ws;
 };

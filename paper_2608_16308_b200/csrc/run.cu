@@ -29,8 +29,8 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
     pdl_launch_dependents();
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = threadIdx.x & 31;
-    bool newly = false;
-    int jb = 0;
+    bool newly = false, fresh = false;
+    int jb = 0, jcol = 0;
     if (t < nnz_x) {
         const int j = x_idx[t];
         if (validate && (j < 0 || j >= d.n)) {
@@ -47,10 +47,21 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
             const int sh = ((j >> 4) & 1) * 16;
             const uint32_t old = atomicOr(&d.ws.x_mask32[j >> 5], 1u << ((j & 15) + sh));
             newly = ((old >> sh) & 0xFFFFu) == 0;
+            fresh = ((old >> ((j & 15) + sh)) & 1u) == 0;     // (an index listed twice emits once)
             jb = j >> 4;
+            jcol = j;
         }
     }
-    emit_tasks<true>(d, newly, jb, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+    // push tasks: the INLINE elements of this column; and, by the thread that turned the vector
+    // block nonempty, the column block's entries with a payload
+    int first = 0, deg = 0;
+    if (fresh) column_run(d, jcol, first, deg);
+    merge_column_runs(fresh, jcol, first, deg, lane);
+    emit_tasks<true>(d, newly, jb, first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+    first = 0; deg = 0;
+    if (newly) payload_run(d, jb, first, deg);
+    if (__syncthreads_or(deg > 0))
+        emit_tasks<true>(d, false, jb, first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, d.payload_chunk);
 }
 
 // Dense input (Sections 4.1, 4.3): every warp reads 32 elements, one ballot gives the two
@@ -71,7 +82,15 @@ __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__re
         const uint32_t bits = __ballot_sync(FULL, v != 0.0f);
         if (lane == 0) d.ws.x_mask32[j >> 5] = bits;
         const bool newly = (lane == 0 && (bits & 0xFFFFu)) || (lane == 16 && (bits >> 16));
-        emit_tasks(d, newly, (int)(j >> 4), lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+        int first = 0, deg = 0;
+        const bool listed = v != 0.0f && j < d.n;
+        if (listed) column_run(d, (int)j, first, deg);
+        merge_column_runs(listed, (int)j, first, deg, lane);
+        emit_tasks(d, newly, (int)(j >> 4), first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+        first = 0; deg = 0;
+        if (newly) payload_run(d, (int)(j >> 4), first, deg);
+        if (__any_sync(FULL, deg > 0))
+            emit_tasks(d, false, (int)(j >> 4), first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, d.payload_chunk);
     }
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < d.m; i += stride) y[i] = 0.f;
 }
@@ -219,10 +238,10 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
         if (t < n_tasks) {
             const int jb = (int)(task.x & IDX_MASK);
             l.jb = jb;
-            const int upper = ((int)(task.x >> 27) + 1) * 4;      // entries of the task, rounded up to 4
+            const int cnt = (int)(task.x >> 27) + 1;              // entries of the task
             l.start = (int)task.y;
-            if (lane < upper) { const int p = l.start + lane; l.idx = d.csc.idx[p]; l.w = d.csc.w[p]; l.aux = d.csc.aux[p]; }
-            l.end = min(l.start + PUSH_CHUNK, d.csc.ptr[jb + 1]);
+            if (lane < cnt) { const int p = l.start + lane; l.idx = d.csc.idx[p]; l.w = d.csc.w[p]; l.aux = d.csc.aux[p]; }
+            l.end = l.start + cnt;
             l.xm = mask_of(d.ws.x_mask32, jb);
             if (lane < 16) l.xv = d.ws.x_dense[jb * 16 + lane];
         }
@@ -885,7 +904,13 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     Workspace &ws = d.ws;
     int64_t total = 0;
     const size_t xwords = (size_t)(d.nb + 1) / 2 + 4, ywords = (size_t)(d.mb + 1) / 2 + 4;
-    ws.task_capacity = (int64_t)d.n_entries / PUSH_CHUNK + d.nb + 32;
+    // Entries with a payload per push task: a full warp step where such blocks are the bulk of
+    // the matrix (the lanes then share them out); a few where they are the exception and a warp
+    // takes them one at a time (32 of them in one task would keep one warp busy for tens of
+    // microseconds while the others have long finished).
+    d.payload_chunk = h->heavy_stage ? PUSH_CHUNK : 4;
+    // one partial task at most per column (INLINE run) and per column block (payload run)
+    ws.task_capacity = (int64_t)d.n_entries / d.payload_chunk + 17 * (int64_t)d.nb + 32;
     ws.n_tiles = (int32_t)ceil_div<int64_t>((d.mb + 1) / 2, TILE_WORDS);
     if (ws.n_tiles < 1) ws.n_tiles = 1;
 #define DBS_WS(expr) do { int s__ = (expr); if (s__ != DBSPMSPV_OK) return s__; } while (0)
@@ -968,7 +993,7 @@ extern "C" {
 void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
-    o->th3 = 0.65f;
+    o->th3 = 0.9f;
     o->th3_bfs = 0.1f;
     o->th3_decode = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;

@@ -7,21 +7,17 @@
 
 namespace dbs {
 
-// Called by a full warp -- or, with CTA_WIDE, by every thread of the thread block.  Lanes with
-// `newly` set own a vector block `jb` that has just become nonempty; each appends that block's
-// tasks.  Space is claimed hierarchically (Section 4.1): a warp scan, then either one atomic per
-// warp or -- CTA_WIDE -- a sum over the block's warps in shared memory and one atomic per thread
-// block (thousands of warps queueing on one counter serialise in L2 otherwise).  The count of
-// nonempty vector blocks is aggregated the same way.
+// Called by a full warp -- or, with CTA_WIDE, by every thread of the thread block.  Every lane
+// hands in one run [first, first + deg) of block-CSC positions of column block `jb` (deg = 0:
+// nothing) and appends its tasks, `chunk` entries each (at most PUSH_CHUNK); lanes with `newly`
+// set own a vector block that has just become nonempty (counted).  Space is claimed hierarchically (Section 4.1): a warp scan, then either
+// one atomic per warp or -- CTA_WIDE -- a sum over the block's warps in shared memory and one
+// atomic per thread block (thousands of warps queueing on one counter serialise in L2
+// otherwise).  The count of nonempty vector blocks is aggregated the same way.
 template <bool CTA_WIDE = false>
-__device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int lane,
-                                           int32_t *n_tasks, int32_t *n_nzblk) {
-    int first = 0, deg = 0;
-    if (newly) {
-        first = d.csc.ptr[jb];
-        deg = d.csc.ptr[jb + 1] - first;
-    }
-    const int nchunks = (deg + PUSH_CHUNK - 1) / PUSH_CHUNK;
+__device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int first, int deg, int lane,
+                                           int32_t *n_tasks, int32_t *n_nzblk, int chunk = PUSH_CHUNK) {
+    const int nchunks = (deg + chunk - 1) / chunk;
     int incl = nchunks;
     for (int o = 1; o < 32; o <<= 1) {
         int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
@@ -33,6 +29,7 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
     if (CTA_WIDE) {
         __shared__ int s_tot[32], s_new[32], s_base;
         const int warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+        __syncthreads();                       // (the arrays may still be read by an earlier call)
         if (lane == 0) { s_tot[warp] = total; s_new[warp] = n_new; }
         __syncthreads();
         if (warp == 0) {
@@ -48,20 +45,19 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
             base = s_base;
             for (int k = 0; k < warp; ++k) base += s_tot[k];
         }
-    } else if (lane == 0 && n_new) {
+    } else if (lane == 0) {
         if (total) base = atomicAdd(n_tasks, total);
-        atomicAdd(n_nzblk, n_new);
+        if (n_new) atomicAdd(n_nzblk, n_new);
     }
     base = __shfl_sync(0xFFFFFFFFu, base, 0) + incl - nchunks;
-    // task record: column block in bits 0..26, ceil(entries / 4) - 1 in bits 27..31 (the exact
-    // end comes from the column pointer), first position.
+    // task record: column block in bits 0..26, entries - 1 in bits 27..31, first position.
     // Short columns are written by their own lane; a long column block (a hub) is written by
     // the whole warp so that one lane does not serialise thousands of stores.
     constexpr int SMALL = 4;
     if (nchunks <= SMALL)
         for (int k = 0; k < nchunks; ++k) {
-            const int cnt = min(PUSH_CHUNK, deg - k * PUSH_CHUNK);
-            d.ws.tasks[base + k] = make_uint2((uint32_t)jb | ((uint32_t)((cnt + 3) / 4 - 1) << 27), (uint32_t)(first + k * PUSH_CHUNK));
+            const int cnt = min(chunk, deg - k * chunk);
+            d.ws.tasks[base + k] = make_uint2((uint32_t)jb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(first + k * chunk));
         }
     uint32_t big = __ballot_sync(0xFFFFFFFFu, nchunks > SMALL);
     while (big) {
@@ -71,12 +67,40 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
         const int bfirst = __shfl_sync(0xFFFFFFFFu, first, src);
         const int bdeg = __shfl_sync(0xFFFFFFFFu, deg, src);
         const int bbase = __shfl_sync(0xFFFFFFFFu, base, src);
-        const int bn = (bdeg + PUSH_CHUNK - 1) / PUSH_CHUNK;
+        const int bn = (bdeg + chunk - 1) / chunk;
         for (int k = lane; k < bn; k += 32) {
-            const int cnt = min(PUSH_CHUNK, bdeg - k * PUSH_CHUNK);
-            d.ws.tasks[bbase + k] = make_uint2((uint32_t)bjb | ((uint32_t)((cnt + 3) / 4 - 1) << 27), (uint32_t)(bfirst + k * PUSH_CHUNK));
+            const int cnt = min(chunk, bdeg - k * chunk);
+            d.ws.tasks[bbase + k] = make_uint2((uint32_t)bjb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(bfirst + k * chunk));
         }
     }
+}
+
+// The two kinds of run of a column block in the block-CSC view (see View::colptr).
+__device__ __forceinline__ void payload_run(const Device &d, int jb, int &first, int &deg) {
+    first = d.csc.ptr[jb];
+    deg = d.csc.colptr[17 * jb] - first;
+}
+__device__ __forceinline__ void column_run(const Device &d, int j, int &first, int &deg) {
+    const int32_t *cp = d.csc.colptr + 17 * (j >> 4) + (j & 15);
+    first = cp[0];
+    deg = cp[1] - first;
+}
+
+// Runs of consecutive columns of one column block are adjacent in the view, so lanes that hold
+// consecutive columns (a sorted x with clustered nonzeros; a dense x) are merged into one run
+// owned by the first lane of the chain; the others are left with deg = 0.  Called by a full
+// warp; `has`: the lane holds column j with the run [first, first + deg).
+__device__ __forceinline__ void merge_column_runs(bool has, int j, int &first, int &deg, int lane) {
+    const int pj = __shfl_up_sync(0xFFFFFFFFu, j, 1);
+    const bool phas = __shfl_up_sync(0xFFFFFFFFu, (int)has, 1) != 0;
+    const bool cont = lane > 0 && has && phas && j == pj + 1 && (j >> 4) == (pj >> 4);
+    const uint32_t contm = __ballot_sync(0xFFFFFFFFu, cont);
+    const int end = first + deg;
+    const uint32_t after = ~contm & ~((2u << lane) - 1u);    // lanes behind me that do not continue a chain
+    const int stop = after ? __ffs(after) - 1 : 32;           // my chain is lanes [lane, stop)
+    const int tail_end = __shfl_sync(0xFFFFFFFFu, end, stop - 1);
+    if (cont) deg = 0;
+    else if (has) deg = tail_end - first;
 }
 
 }  // namespace dbs

@@ -103,7 +103,9 @@ def test_export_equals_input_and_census(name, make, dtype):
     for k in range(6):
         assert s.class_blocks[k] == int((wcls == k).sum())
         assert s.class_nnz[k] == int(wn[wcls == k].sum())
-    # dual view: same entry set, CSC order, consistent pointers
+    # dual view: same entry set, consistent pointers, and the block-CSC order: by column block;
+    # inside it the entries with a payload first (by row block), then the INLINE elements column
+    # by column (by row), so that a push can visit single columns
     rp, cp, crow, c2r = h.export_views()
     ne = er.size
     assert rp[0] == 0 and rp[-1] == ne and cp[0] == 0 and cp[-1] == ne
@@ -111,11 +113,16 @@ def test_export_equals_input_and_census(name, make, dtype):
     assert np.array_equal(np.diff(cp), np.bincount(ec, minlength=s.n_col_blocks))
     assert np.array_equal(np.sort(c2r), np.arange(ne))                          # a permutation
     assert np.array_equal(crow, er[c2r])
-    ccol = ec[c2r]
-    ckey = ccol.astype(np.int64) * (1 << 32) + crow
-    assert (np.diff(ckey) >= 0).all()                                           # sorted by (col, row)
-    same = np.diff(ckey) == 0
-    assert (np.diff(c2r)[same] == 1).all()                                      # a block's entries stay in order
+    # the stored elements in primary order: by (row block, column block, local row, local column)
+    prim = np.lexsort((c & 15, r & 15, c >> 4, r >> 4))
+    pr, pc = r[prim], c[prim]
+    elem0 = np.r_[0, np.cumsum(en)[:-1]] if ne else np.zeros(0, np.int64)       # first element of every entry
+    inl = ecls == B.BLK_INLINE
+    lr = np.where(inl, pr[elem0] & 15, 0) if ne else elem0
+    lc = np.where(inl, pc[elem0] & 15, 0) if ne else elem0
+    group = np.where(inl, 16 + lc, 0)
+    key = ((ec.astype(np.int64) << 36) | (group.astype(np.int64) << 31) | (er.astype(np.int64) << 4) | lr)[c2r]
+    assert (np.diff(key) > 0).all()                                             # strictly ascending: the order above
     h.close()
 
 
