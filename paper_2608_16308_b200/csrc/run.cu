@@ -31,6 +31,7 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
     const int lane = threadIdx.x & 31;
     bool newly = false, fresh = false;
     int jb = 0, jcol = 0;
+    int first = 0, deg = 0, pfirst = 0, pdeg = 0;
     if (t < nnz_x) {
         const int j = x_idx[t];
         if (validate && (j < 0 || j >= d.n)) {
@@ -44,6 +45,10 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
             // a listed NaN that happens to carry the marker's bit pattern is stored as the
             // canonical quiet NaN, so the marker itself never appears as data
             d.ws.x_dense[j] = __float_as_uint(v) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v;
+            // the runs this thread may have to turn into tasks are fetched before the atomic
+            // whose result decides it (the loads are independent of it; the chain is shorter)
+            column_run(d, j, first, deg);
+            payload_run(d, j >> 4, pfirst, pdeg);
             const int sh = ((j >> 4) & 1) * 16;
             const uint32_t old = atomicOr(&d.ws.x_mask32[j >> 5], 1u << ((j & 15) + sh));
             newly = ((old >> sh) & 0xFFFFu) == 0;
@@ -54,14 +59,12 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
     }
     // push tasks: the INLINE elements of this column; and, by the thread that turned the vector
     // block nonempty, the column block's entries with a payload
-    int first = 0, deg = 0;
-    if (fresh) column_run(d, jcol, first, deg);
+    if (!fresh) deg = 0;
     merge_column_runs(fresh, jcol, first, deg, lane);
     emit_tasks<true>(d, newly, jb, first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
-    first = 0; deg = 0;
-    if (newly) payload_run(d, jb, first, deg);
-    if (__syncthreads_or(deg > 0))
-        emit_tasks<true>(d, false, jb, first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, d.payload_chunk);
+    if (!newly) pdeg = 0;
+    if (__syncthreads_or(pdeg > 0))
+        emit_tasks<true>(d, false, jb, pfirst, pdeg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, d.payload_chunk);
 }
 
 // Dense input (Sections 4.1, 4.3): every warp reads 32 elements, one ballot gives the two
