@@ -236,7 +236,8 @@ int dbspmspv_export_blocks(dbspmspv_handle_t h, int32_t *block_row, int32_t *blo
 /* Test hook: copy the dual view out: csr_row_ptr (n_row_blocks+1), csc_col_ptr
  * (n_col_blocks+1), csc_row (n_view_entries: row block of every CSC-view position), csc2csr
  * (n_view_entries: CSC-view position -> primary entry id).  Device int32 arrays; any may be
- * NULL.                                                                                      */
+ * NULL.  CSC-view order: by column block; inside a column block the entries with a payload
+ * first (by row block), then the INLINE elements by (local column, row block, local row).    */
 int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *csc_col_ptr,
                           int32_t *csc_row, int32_t *csc2csr);
 
