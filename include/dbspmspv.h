@@ -91,7 +91,10 @@ typedef struct {
     int32_t w_inline;        /* ... of an INLINE view entry                         (1)      */
     int32_t w_dense_sparse;  /* Dense / CSR-like weights used instead when such blocks are a */
     int32_t w_mid_sparse;    /* minority of the matrix (hypersparse matrices)  (128 / 64)    */
-    int32_t reserved[3];
+    int32_t no_bfs_index;    /* 1: do not build the row-run index that square matrices get for
+                                the pull levels of db_bfs (4 bytes per stored element; a pull
+                                level then walks whole row-block segments)          (0)    */
+    int32_t reserved[2];
 } dbspmspv_create_opts;
 
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
@@ -146,7 +149,8 @@ typedef struct {
     float last_compute_ms;         /* traversal kernel time of the last run/decode (timing=1),
                                       else -1                                                 */
     int64_t kernel_launches;       /* kernels launched through this handle so far             */
-    int32_t reserved[4];
+    int64_t bfs_index_bytes;       /* row-run index of DB-BFS (0 when not built)              */
+    int32_t reserved[2];
 } dbspmspv_stats;
 
 /* Paper thresholds (th0 = 32, th1 = 128, th2 = 2.0, Section 3.2.1).  The segment weights keep

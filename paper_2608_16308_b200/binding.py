@@ -37,7 +37,8 @@ class CreateOpts(ctypes.Structure):
                 ("w_coo", ctypes.c_int32), ("force_format", ctypes.c_int32),
                 ("input_on_host", ctypes.c_int32), ("inline_max", ctypes.c_int32),
                 ("w_inline", ctypes.c_int32), ("w_dense_sparse", ctypes.c_int32),
-                ("w_mid_sparse", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
+                ("w_mid_sparse", ctypes.c_int32), ("no_bfs_index", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 2)]
 
 
 class RunOpts(ctypes.Structure):
@@ -61,7 +62,8 @@ class Stats(ctypes.Structure):
                 ("bfs_level_path", ctypes.c_int32 * MAX_BFS_LEVELS_RECORDED),
                 ("bfs_level_nzblk", ctypes.c_int32 * MAX_BFS_LEVELS_RECORDED),
                 ("device_status", ctypes.c_int32), ("last_compute_ms", ctypes.c_float),
-                ("kernel_launches", ctypes.c_int64), ("reserved", ctypes.c_int32 * 4)]
+                ("kernel_launches", ctypes.c_int64), ("bfs_index_bytes", ctypes.c_int64),
+                ("reserved", ctypes.c_int32 * 2)]
 
 
 _lib = None

@@ -192,6 +192,8 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     cudaFree(const_cast<int2 *>(d.chunks));
     cudaFree(const_cast<int32_t *>(d.seg_rb));
     cudaFree(const_cast<uint32_t *>(d.row_present32));
+    cudaFree(const_cast<int32_t *>(d.rowrun_ptr)); cudaFree(const_cast<uint32_t *>(d.rowrun_idx));
+    cudaFree(const_cast<int32_t *>(d.payload_ptr)); cudaFree(const_cast<int32_t *>(d.payload_pos));
     cudaFree(h->csc2csr); cudaFree(h->block_row);
     dbs::Workspace &ws = d.ws;
     cudaFree(ws.x_dense); cudaFree(ws.x_mask32); cudaFree(ws.tasks); cudaFree(ws.y_acc);

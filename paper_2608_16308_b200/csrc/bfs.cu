@@ -233,6 +233,85 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
     }
 }
 
+// Boolean pull over the row-run index (square matrices, unless the index was switched off): a
+// warp takes the 32 rows of one mask word (two row blocks), lane = row.  Entries with a payload
+// are evaluated first, from the per-row-block position list; then every row that is still wanted
+// walks its own INLINE run and stops at its first frontier neighbour -- the early exit of
+// Algorithm 5 per row instead of per row block: in the big levels a row finds a parent within a
+// few entries, so a fraction of the edges is read at all.  Four entries are fetched per round
+// and lane (then their four frontier masks); a row that has not finished after eight rounds is
+// long (a hub with no frontier neighbour so far) and is finished by the whole warp, 32 entries
+// per step.  The warp owns its mask word: plain stores, no atomics.
+template <int DT>
+__device__ void bfs_pull_rows(const Device &d, int32_t *levels, int depth) {
+    const int lane = threadIdx.x & 31;
+    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int n_words = (d.mb + 1) / 2;
+    constexpr uint32_t NONE = 0xFFFFFFFFu;          // no entry: local column 31 never matches a 16-bit mask
+    for (int wd = gwarp; wd < n_words; wd += nwarps) {
+        const uint32_t need = ~d.ws.visited32[wd];   // (rows without stored elements and rows past m count as visited)
+        if (!need) continue;
+        uint32_t found = 0;
+        // entries with a payload, one per lane
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            const int rb = 2 * wd + hf;
+            const uint32_t need16 = (need >> (16 * hf)) & 0xFFFFu;
+            if (rb >= d.mb || !need16) continue;    // warp-uniform
+            const int pbeg = d.payload_ptr[rb], pend = d.payload_ptr[rb + 1];
+            uint32_t hit = 0;
+            for (int q = pbeg + lane; q < pend; q += 32) {
+                const int pos = d.payload_pos[q];
+                const uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
+                const uint32_t xm = mask_of(d.ws.x_mask32, idx & IDX_MASK);
+                if (xm) {
+                    const int type = idx >> TYPE_SHIFT;
+                    const uint32_t w = d.csr.w[pos];
+                    hit |= type == DBSPMSPV_BLK_COO ? lane_block_bool<DT>(type, w, aux, xm, d.payload)
+                                                    : lane_heavy_bool(type, d.payload + (size_t)w * 4, xm);
+                }
+            }
+            if (pend > pbeg) found |= (__reduce_or_sync(FULL, hit) & need16) << (16 * hf);
+        }
+        // row runs
+        const int row = wd * 32 + lane;
+        bool active = ((need & ~found) >> lane) & 1u;
+        int p = 0, e = 0;
+        if (active) { p = d.rowrun_ptr[row]; e = d.rowrun_ptr[row + 1]; active = p < e; }
+        bool got = false;
+        for (int round = 0; round < 8 && __any_sync(FULL, active); ++round) {
+            uint32_t v[4], xm[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = (active && p + j < e) ? d.rowrun_idx[p + j] : NONE;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) xm[j] = v[j] != NONE ? mask_of(d.ws.x_mask32, v[j] & IDX_MASK) : 0u;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) got |= ((xm[j] >> (v[j] >> 27)) & 1u) != 0;
+            p += 4;
+            if (got || p >= e) active = false;
+        }
+        uint32_t longm = __ballot_sync(FULL, active);
+        while (longm) {
+            const int src = __ffs(longm) - 1;
+            longm &= longm - 1;
+            const int lp = __shfl_sync(FULL, p, src), le = __shfl_sync(FULL, e, src);
+            bool hit = false;
+            for (int q = lp; q < le && !hit; q += 32) {
+                const uint32_t v = q + lane < le ? d.rowrun_idx[q + lane] : NONE;
+                const uint32_t xm = v != NONE ? mask_of(d.ws.x_mask32, v & IDX_MASK) : 0u;
+                hit = __any_sync(FULL, (xm >> (v >> 27)) & 1u);
+            }
+            if (lane == src) got = hit;
+        }
+        found = (found | __ballot_sync(FULL, got)) & need;
+        if (found) {
+            if (lane == 0) d.ws.y_mask32[wd] = found;
+            if ((found >> lane) & 1u) levels[row] = depth;
+        }
+    }
+}
+
 // Per-level selector (Section 3.3.1): push iff N_nzblk / N_blk < th3.  Monotone in n_nzblk.
 __device__ __forceinline__ int bfs_path(int n_nzblk, int nb, float th3, int force_path) {
     if (force_path == DBSPMSPV_PATH_PUSH || force_path == DBSPMSPV_PATH_PULL) return force_path;
@@ -288,6 +367,7 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
             }
         }
         if (path == DBSPMSPV_PATH_PUSH) bfs_push<DT>(d, n_tasks, levels, depth);
+        else if (d.rowrun_ptr) bfs_pull_rows<DT>(d, levels, depth);
         else bfs_pull<DT>(d, levels, depth);
         grid.sync();
         // next frontier: masks produced above become the vector-block masks of the next level,

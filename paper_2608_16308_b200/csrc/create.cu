@@ -339,6 +339,39 @@ __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
     bcol_sorted[p] = (int32_t)(k >> CSC_KEY_COL_SHIFT);
 }
 
+// ---- row-run index of the INLINE elements (DB-BFS pull levels)
+__global__ void k_rowrun_keys(int32_t n_entries, int64_t m, const int32_t *entry_row, const uint32_t *csr_idx,
+                              const uint8_t *csr_aux, uint64_t *keys, uint32_t *vals, int32_t *is_payload) {
+    int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p >= n_entries) return;
+    const uint32_t idx = csr_idx[p], rc = csr_aux[p];
+    const bool inl = (idx >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE;
+    const uint64_t row = inl ? (uint64_t)entry_row[p] * 16 + (rc >> 4) : (uint64_t)m;   // others sort behind every row
+    const uint64_t col = inl ? (uint64_t)(idx & IDX_MASK) * 16 + (rc & 15u) : 0u;
+    keys[p] = (row << 31) | col;
+    vals[p] = (idx & IDX_MASK) | ((rc & 15u) << 27);
+    is_payload[p] = inl ? 0 : 1;
+}
+
+// ptr[i] = first position whose row is >= i, i = 0..m
+__global__ void k_rowrun_ptr(int64_t m, const uint64_t *keys_sorted, int32_t n, int32_t *ptr) {
+    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i > m) return;
+    int32_t lo = 0, hi = n;
+    while (lo < hi) {
+        int32_t mid = lo + ((hi - lo) >> 1);
+        if ((keys_sorted[mid] >> 31) < (uint64_t)i) lo = mid + 1; else hi = mid;
+    }
+    ptr[i] = lo;
+}
+
+__global__ void k_payload_list(int32_t n_entries, int32_t mb, const int32_t *is_payload, const int32_t *rank,
+                               const int32_t *csr_ptr, int32_t *payload_pos, int32_t *payload_ptr) {
+    int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p < n_entries && is_payload[p]) payload_pos[rank[p]] = (int32_t)p;
+    if (p <= mb) payload_ptr[p] = rank[csr_ptr[p]];
+}
+
 // ---- pull segments (Section 3.3.2): greedy walk along each row block; a segment closes
 // when its accumulated weight reaches the cut.  One warp per row block (hub row blocks hold
 // 10^5 entries: a single thread walking them took tens of milliseconds), two passes.  The warp
@@ -637,6 +670,36 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         tp.release(k2); tp.release(k2_alt); tp.release(ids); tp.release(ids_alt); tp.release(bcol_sorted);
     }
 
+    // row-run index for the pull levels of DB-BFS
+    d.rowrun_ptr = nullptr; d.rowrun_idx = nullptr; d.payload_ptr = nullptr; d.payload_pos = nullptr;
+    if (m == n && !h->copts.no_bfs_index) {
+        uint64_t *rk, *rk_alt;
+        uint32_t *rv, *rv_alt;
+        int32_t *isp, *rank;
+        DBS_GET(rk, n_entries); DBS_GET(rk_alt, n_entries); DBS_GET(rv, n_entries); DBS_GET(rv_alt, n_entries);
+        DBS_GET(isp, (int64_t)n_entries + 1); DBS_GET(rank, (int64_t)n_entries + 1);
+        DBS_CUDA(cudaMemsetAsync(isp, 0, ((size_t)n_entries + 1) * 4, st));
+        if (n_entries) {
+            k_rowrun_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, m, h->block_row, d.csr.idx, d.csr.aux, rk, rv, isp);
+            DBS_TRY(sort_pairs(tp, rk, rk_alt, rv, rv_alt, (int64_t)n_entries, 31 + bits_for((uint64_t)m), st));
+        }
+        DBS_TRY(exclusive_sum(tp, isp, rank, (int64_t)n_entries + 1, st));
+        int32_t n_payload = 0;
+        DBS_CUDA(cudaMemcpy(&n_payload, rank + n_entries, 4, cudaMemcpyDeviceToHost));
+        const int32_t n_inline = n_entries - n_payload;
+        int32_t *rp, *pp, *ppos;
+        uint32_t *ri;
+        DBS_KEEP(rp, m + 1); DBS_KEEP(ri, n_inline); DBS_KEEP(pp, (int64_t)d.mb + 1); DBS_KEEP(ppos, n_payload);
+        d.rowrun_ptr = rp; d.rowrun_idx = ri; d.payload_ptr = pp; d.payload_pos = ppos;
+        k_rowrun_ptr<<<grid_for(m + 1), TPB, 0, st>>>(m, rk, n_entries, rp);
+        if (n_inline) DBS_CUDA(cudaMemcpyAsync(ri, rv, (size_t)n_inline * 4, cudaMemcpyDeviceToDevice, st));
+        const int64_t span = (int64_t)n_entries > d.mb + 1 ? n_entries : d.mb + 1;
+        k_payload_list<<<grid_for(span), TPB, 0, st>>>(n_entries, d.mb, isp, rank, d.csr.ptr, ppos, pp);
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(rk); tp.release(rk_alt); tp.release(rv); tp.release(rv_alt); tp.release(isp); tp.release(rank);
+        h->bfs_index_bytes = ((int64_t)m + 1) * 4 + (int64_t)n_inline * 4 + ((int64_t)d.mb + 1) * 4 + (int64_t)n_payload * 4;
+    }
+
     // class census -> which kernel variant the handle uses, hence what a mask-based block costs
     unsigned long long cls_h[2 * DBSPMSPV_BLK_NCLASS];
     DBS_CUDA(cudaMemcpy(cls_h, cls, sizeof(cls_h), cudaMemcpyDeviceToHost));
@@ -689,6 +752,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)d.n_entries * 9;
     s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.nb * 17 * 4 + (int64_t)d.n_entries * 9;
     s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment) + ((int64_t)d.n_chunks + 1) * 8 + (int64_t)d.n_segments * 4;
+    s.bfs_index_bytes = h->bfs_index_bytes;
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }

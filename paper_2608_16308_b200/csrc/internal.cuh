@@ -148,6 +148,15 @@ struct Device {           // everything the kernels need, passed by value
     const int2 *chunks;   // n_chunks + 1: {first segment, first entry} of every pull chunk
     int32_t n_chunks;
     int32_t payload_chunk;  // entries with a payload per push task (see allocate_workspace)
+    // Row-run index for the pull levels of DB-BFS (square matrices, unless switched off): the
+    // INLINE elements once more, row by row -- rowrun_idx[k] = column block | local column << 27
+    // for k in [rowrun_ptr[i], rowrun_ptr[i + 1]) -- so that a row can stop at its first frontier
+    // neighbour; and the block-CSR positions of the entries with a payload, per row block
+    // (payload_pos[payload_ptr[rb] .. payload_ptr[rb + 1])).  Null when not built.
+    const int32_t *rowrun_ptr;
+    const uint32_t *rowrun_idx;
+    const int32_t *payload_ptr;
+    const int32_t *payload_pos;
     const uint32_t *row_present32;  // per row block: rows that hold a stored element (two 16-bit masks per word)
     Workspace ws;
 };
@@ -171,6 +180,7 @@ struct dbspmspv_handle_s {
     cudaEvent_t ev[2];          // optional timing of the traversal kernel (run_opts.timing)
     bool timed;
     int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)
+    int64_t bfs_index_bytes;
 };
 
 namespace dbs {

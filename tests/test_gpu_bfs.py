@@ -38,11 +38,12 @@ GRAPHS = [
 
 @pytest.mark.parametrize("name,make", GRAPHS, ids=[g[0] for g in GRAPHS])
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("inline_max", [31, 3], ids=["inline", "coo_lists"])
-def test_levels_bit_exact(name, make, path, inline_max):
+@pytest.mark.parametrize("inline_max,no_index", [(31, 0), (3, 0), (31, 1)], ids=["inline", "coo_lists", "no_row_index"])
+def test_levels_bit_exact(name, make, path, inline_max, no_index):
     g = make()
     o = B.default_create_opts()
     o.inline_max = inline_max            # 3: blocks of 4..31 entries become packed coordinate lists
+    o.no_bfs_index = no_index            # 1: pull levels walk the row-block segments
     h = Handle(g, B.PATTERN, opts=o)
     h.set_opts(force_path=path)
     A = ref_matrix(g)
