@@ -108,10 +108,10 @@ typedef struct {
     int32_t validate;        /* 1: range-check x indices on the device (ERR_BOUNDS)          */
     int32_t timing;          /* 1: bracket the traversal kernel of run/decode with two CUDA
                                 events (made at create); read back as last_compute_ms      */
-    float th3_bfs;           /* db_bfs: same rule per level.  Default 0.1, measured on the
-                                symmetrised R-MAT scale 22 graph (0.05 .. 0.2 are within 1 %;
-                                a pull level skips finished row blocks, a push level pays one
-                                atomic per reached entry)                                   */
+    float th3_bfs;           /* db_bfs: same rule per level.  Default 0.05, measured on the
+                                symmetrised R-MAT scale 22 graph (0.03 .. 0.07 are within 3 %;
+                                a pull level stops every row at its first frontier neighbour,
+                                a push level pays one atomic per reached entry)             */
     float th3_decode;        /* dbspmspv_decode: same rule; the output is dense and every row block
                                 takes part, so pull wins much earlier (0.01, the paper's value) */
     int32_t reserved[9];

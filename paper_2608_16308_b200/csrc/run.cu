@@ -997,7 +997,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
     o->th3 = 0.9f;
-    o->th3_bfs = 0.1f;
+    o->th3_bfs = 0.05f;
     o->th3_decode = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;
     o->popc_threshold = 8;
