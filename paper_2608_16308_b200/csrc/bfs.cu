@@ -47,31 +47,36 @@ __device__ __forceinline__ void write_levels(int32_t *levels, int rb, uint32_t f
 // pipelined: while task k is evaluated, the visited masks of k+1, the view entries of k+2 and
 // the task record of k+3 (in this warp's stride) are in flight.
 template <int DT>
-__device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int depth) {
+__device__ void bfs_push(const Device &d, int n_recs, const int4 *hubs, int n_hubs, int32_t *levels, int depth) {
     static_assert(PUSH_CHUNK == 32, "one warp step per task");
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const HubTable table = load_hub_table(hubs, n_hubs, lane);
+    const int n_tasks = n_recs + table.total;                    // task records, then the steps of the hub runs
+    auto item = [&](int i) { return worklist_item(d.ws.tasks, n_recs, table, i); };
     const uint2 none = make_uint2(0u, 0u);
-    struct Entries { uint32_t idx, aux, xm; int n; };   // n: entries of the task (0 = no task)
+    struct Entries { uint32_t idx, aux, xm; int n, start; };   // n: entries of the task (0 = no task)
     auto entries_of = [&](int t, const uint2 &task) {
-        Entries e{0u, 0u, 0u, 0};
+        Entries e{0u, 0u, 0u, 0, 0};
         if (t < n_tasks) {
             const int jb = (int)(task.x & IDX_MASK), start = (int)task.y;
             e.n = (int)(task.x >> 27) + 1;
+            e.start = start;
             if (lane < e.n) { e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane]; }
             e.xm = mask_of(d.ws.x_mask32, jb);
         }
         return e;
     };
     auto need_of = [&](const Entries &e) { return lane < e.n ? ~mask_of(d.ws.visited32, e.idx & IDX_MASK) & 0xFFFFu : 0u; };
-    uint2 t1 = gwarp + nwarps < n_tasks ? d.ws.tasks[gwarp + nwarps] : none;
-    uint2 t2 = gwarp + 2 * nwarps < n_tasks ? d.ws.tasks[gwarp + 2 * nwarps] : none;
-    Entries e0 = entries_of(gwarp, gwarp < n_tasks ? d.ws.tasks[gwarp] : none);
+    uint2 t1 = gwarp + nwarps < n_tasks ? item(gwarp + nwarps) : none;
+    uint2 t2 = gwarp + 2 * nwarps < n_tasks ? item(gwarp + 2 * nwarps) : none;
+    uint2 t0 = gwarp < n_tasks ? item(gwarp) : none;
+    Entries e0 = entries_of(gwarp, t0);
     Entries e1 = entries_of(gwarp + nwarps, t1);
     uint32_t need0 = need_of(e0);
     for (int t = gwarp; t < n_tasks; t += nwarps) {
-        const uint2 t3 = t + 3 * nwarps < n_tasks ? d.ws.tasks[t + 3 * nwarps] : none;   // stage 1
+        const uint2 t3 = t + 3 * nwarps < n_tasks ? item(t + 3 * nwarps) : none;          // stage 1
         const Entries e2 = entries_of(t + 2 * nwarps, t2);                                // stage 2
         const uint32_t need1 = need_of(e1);                                               // stage 3
         // stage 4: evaluate task t
@@ -85,7 +90,7 @@ __device__ void bfs_push(const Device &d, int n_tasks, int32_t *levels, int dept
                 if (type == DBSPMSPV_BLK_INLINE) {
                     hit = ((xm >> (aux & 15)) & 1u) << (aux >> 4);
                 } else {
-                    w = d.csc.w[(int)d.ws.tasks[t].y + lane];
+                    w = d.csc.w[e0.start + lane];
                     if (type == DBSPMSPV_BLK_COO) {
                         if (aux < COO_SERIAL_MAX) hit = lane_block_bool<DT>(type, w, aux, xm, d.payload);
                         else heavy = true;
@@ -325,6 +330,7 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
     const int tid = blockIdx.x * blockDim.x + threadIdx.x;
     const int nthreads = gridDim.x * blockDim.x;
     const int lane = threadIdx.x & 31;
+    const int gwarp_all = tid >> 5, nwarps_all = nthreads >> 5;
     const int n_words = (d.mb + 1) / 2;
     Counters *ctr = d.ws.ctr;
 
@@ -333,7 +339,7 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
     // "visited", so that a row block is skipped (and a segment left early) once every row that
     // can be found has been found
     for (int k = tid; k < n_words; k += nthreads) { d.ws.visited32[k] = ~d.row_present32[k]; d.ws.x_mask32[k] = 0u; d.ws.y_mask32[k] = 0u; }
-    if (tid == 0) { ctr->bfs_cnt[0][0] = 0; ctr->bfs_cnt[0][1] = 0; ctr->bfs_cnt[1][0] = 0; ctr->bfs_cnt[1][1] = 0; ctr->bfs_reached = 1; }
+    if (tid == 0) { ctr->bfs_cnt[0][0] = 0; ctr->bfs_cnt[0][1] = 0; ctr->bfs_cnt[1][0] = 0; ctr->bfs_cnt[1][1] = 0; ctr->bfs_hubs[0] = 0; ctr->bfs_hubs[1] = 0; ctr->bfs_reached = 1; }
     grid.sync();
     // level 0: the source is the first frontier
     if (blockIdx.x == 0 && threadIdx.x < 32) {
@@ -347,7 +353,7 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         int first = 0, deg = 0;
         if (lane == 0) column_run(d, src, first, deg);
         else if (lane == 1) payload_run(d, jb, first, deg);
-        emit_tasks(d, lane == 0, jb, first, deg, lane, &ctr->bfs_cnt[0][1], &ctr->bfs_cnt[0][0]);
+        emit_tasks(d, lane == 0, jb, first, deg, lane, &ctr->bfs_cnt[0][1], &ctr->bfs_cnt[0][0], PUSH_CHUNK, &ctr->bfs_hubs[0], d.ws.hubs);
     }
     grid.sync();
 
@@ -361,27 +367,41 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         if (tid == 0) {
             ctr->bfs_cnt[cur ^ 1][0] = 0;
             ctr->bfs_cnt[cur ^ 1][1] = 0;
+            ctr->bfs_hubs[cur ^ 1] = 0;
+            ctr->bfs_nwords = 0;
             if (depth <= DBSPMSPV_MAX_BFS_LEVELS_RECORDED) {
                 ctr->bfs_level_path[depth - 1] = path;
                 ctr->bfs_level_nzblk[depth - 1] = n_nzblk;
             }
         }
-        if (path == DBSPMSPV_PATH_PUSH) bfs_push<DT>(d, n_tasks, levels, depth);
+        if (path == DBSPMSPV_PATH_PUSH) bfs_push<DT>(d, n_tasks, d.ws.hubs + cur * HUB_CAP, min(ctr->bfs_hubs[cur], HUB_CAP), levels, depth);
         else if (d.rowrun_ptr) bfs_pull_rows<DT>(d, levels, depth);
         else bfs_pull<DT>(d, levels, depth);
         grid.sync();
         // next frontier: masks produced above become the vector-block masks of the next level,
         // visited is updated and the nonempty blocks are counted (one atomic per warp)
         int found = 0, nz = 0;
-        for (int k = tid; k < n_words; k += nthreads) {
-            const uint32_t nm = d.ws.y_mask32[k];
-            if (nm) {
-                d.ws.y_mask32[k] = 0u;
-                d.ws.visited32[k] |= nm;
-                found += __popc(nm);
-                nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
+        for (int k0 = tid & ~31; k0 < n_words; k0 += nthreads) {
+            const int k = k0 + lane;
+            uint32_t nm = 0;
+            if (k < n_words) {
+                nm = d.ws.y_mask32[k];
+                if (nm) {
+                    d.ws.y_mask32[k] = 0u;
+                    d.ws.visited32[k] |= nm;
+                    found += __popc(nm);
+                    nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
+                }
+                if (nm || d.ws.x_mask32[k]) d.ws.x_mask32[k] = nm;
             }
-            if (nm || d.ws.x_mask32[k]) d.ws.x_mask32[k] = nm;
+            // the nonzero words are listed, so that a worklist rebuild can share them out evenly
+            const uint32_t nzw = __ballot_sync(FULL, nm != 0u);
+            if (nzw) {
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&ctr->bfs_nwords, __popc(nzw));
+                base = __shfl_sync(FULL, base, 0);
+                if (nm) d.ws.bfs_words[base + __popc(nzw & ((1u << lane) - 1u))] = k;
+            }
         }
         found = __reduce_add_sync(FULL, found);
         nz = __reduce_add_sync(FULL, nz);
@@ -391,31 +411,25 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         // known now); its block count goes to a scratch counter
         const int next_n = ctr->bfs_cnt[cur ^ 1][0];
         if (next_n && bfs_path(next_n, d.nb, th3, force_path) == DBSPMSPV_PATH_PUSH) {
-            // lane l of a warp step takes vector block 64 * step + l and then + 32: first the
-            // block's entries with a payload, then the INLINE run of every frontier column
-            for (int k0 = (tid & ~31); k0 < n_words; k0 += nthreads) {
-                const uint32_t word = k0 + (lane >> 1) < n_words ? d.ws.x_mask32[k0 + (lane >> 1)] : 0u;
-                const uint32_t word2 = k0 + 16 + (lane >> 1) < n_words ? d.ws.x_mask32[k0 + 16 + (lane >> 1)] : 0u;
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int jb = 2 * k0 + 32 * half + lane;
-                    uint32_t m = ((half ? word2 : word) >> ((lane & 1) * 16)) & 0xFFFFu;
-                    int first = 0, deg = 0;
-                    if (m) payload_run(d, jb, first, deg);
-                    if (__any_sync(FULL, deg > 0)) emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad, d.payload_chunk);
-                    while (__any_sync(FULL, m != 0)) {     // one run of consecutive frontier columns at a time
-                        first = 0; deg = 0;
-                        if (m) {
-                            const int c0 = __ffs(m) - 1;
-                            const int len = __ffs(~(m >> c0)) - 1;
-                            const int32_t *cp = d.csc.colptr + 17 * jb + c0;
-                            first = cp[0];
-                            deg = cp[len] - first;
-                            m &= ~(((1u << len) - 1u) << c0);
-                        }
-                        emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad);
-                    }
-                }
+            // a warp takes one listed mask word (two vector blocks) at a time, lane = column:
+            // frontier columns emit their INLINE runs (adjacent ones merged), lanes 0 and 16 the
+            // payload runs of the two blocks.  (With the words in index order, the few warps that
+            // held the hub blocks of an early frontier wrote almost the whole worklist.)
+            const int n_listed = ctr->bfs_nwords;
+            for (int i = gwarp_all; i < n_listed; i += nwarps_all) {
+                const int wd = d.ws.bfs_words[i];
+                const uint32_t word = d.ws.x_mask32[wd];
+                const int jb = 2 * wd + (lane >> 4), j = jb * 16 + (lane & 15);
+                const bool listed = (word >> lane) & 1u;
+                int first = 0, deg = 0;
+                if (listed) column_run(d, j, first, deg);
+                merge_column_runs(listed, j, first, deg, lane);
+                emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad, PUSH_CHUNK,
+                           &ctr->bfs_hubs[cur ^ 1], d.ws.hubs + (cur ^ 1) * HUB_CAP);
+                first = 0; deg = 0;
+                if ((lane & 15) == 0 && ((word >> lane) & 0xFFFFu)) payload_run(d, jb, first, deg);
+                if (__any_sync(FULL, deg > 0))
+                    emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad, d.payload_chunk);
             }
             grid.sync();
         }

@@ -55,6 +55,10 @@ constexpr int TYPE_SHIFT = 29;
 #endif
 constexpr int PUSH_CHUNK = DBS_PUSH_CHUNK;   // CSC-view entries per push task (32 per warp step)
 static_assert(PUSH_CHUNK == 32, "a push task is one warp step; its record stores the exact entry count in 5 bits");
+// A run of the push worklist with at least HUB_MIN_ENTRIES entries (a hub column) is not cut
+// into tasks: it is listed once and every warp of the traversal strides over its 32-entry steps.
+constexpr int HUB_MIN_ENTRIES = 8192;
+constexpr int HUB_CAP = 32;
 constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-class block
 
 // Payload size in 4-byte words; every block is padded to 16 bytes so that it can be moved with
@@ -116,6 +120,9 @@ struct Counters {    // device-resident scalars of one call
     int32_t last_n_nzblk, last_n_tasks, last_path, last_y_nnz;
     int32_t bfs_levels, bfs_reached;
     int32_t pad;
+    int32_t n_hubs;         // hub runs of this call's push worklist (may exceed HUB_CAP: the rest became tasks)
+    int32_t bfs_hubs[2];    // BFS: the same per level, double buffered
+    int32_t bfs_nwords;     // BFS: nonzero words of the new frontier's masks (listed in Workspace::bfs_words)
     int32_t bfs_cnt[2][2];  // BFS: {nonempty frontier blocks, tasks}, double buffered by level
     int32_t bfs_level_path[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
     int32_t bfs_level_nzblk[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
@@ -124,12 +131,14 @@ struct Counters {    // device-resident scalars of one call
 struct Workspace {
     float *x_dense;       // n (padded to a multiple of 32): dense copy of x (Section 3.2.2)
     uint32_t *x_mask32;   // vector-block masks, two 16-bit masks per word
-    uint2 *tasks;         // push worklist: (column block | (ceil(entries/4)-1) << 27, first CSC-view position)
+    uint2 *tasks;         // push worklist: (column block | (entries - 1) << 27, first CSC-view position)
+    int4 *hubs;           // 2 x HUB_CAP hub runs (column block, first position, entries, -): see worklist.cuh
     float *y_acc;         // m (padded): dense accumulator, all zero between calls
     uint32_t *y_mask32;   // run: hit masks packed by the compaction pass; BFS: next-frontier masks
     uint8_t *y_hit8;      // run: one structural-hit flag byte per row, all zero between calls
     int32_t *tile_count;  // compaction: result entries per tile of row blocks
     uint32_t *visited32;  // BFS: visited masks
+    int32_t *bfs_words;   // BFS: indices of the nonzero mask words of the new frontier
     Counters *ctr;
     int64_t task_capacity;
     int32_t n_tiles;

@@ -61,7 +61,7 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
     // block nonempty, the column block's entries with a payload
     if (!fresh) deg = 0;
     merge_column_runs(fresh, jcol, first, deg, lane);
-    emit_tasks<true>(d, newly, jb, first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+    emit_tasks<true>(d, newly, jb, first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, PUSH_CHUNK, &d.ws.ctr->n_hubs, d.ws.hubs);
     if (!newly) pdeg = 0;
     if (__syncthreads_or(pdeg > 0))
         emit_tasks<true>(d, false, jb, pfirst, pdeg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, d.payload_chunk);
@@ -89,7 +89,7 @@ __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__re
         const bool listed = v != 0.0f && j < d.n;
         if (listed) column_run(d, (int)j, first, deg);
         merge_column_runs(listed, (int)j, first, deg, lane);
-        emit_tasks(d, newly, (int)(j >> 4), first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+        emit_tasks(d, newly, (int)(j >> 4), first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, PUSH_CHUNK, &d.ws.ctr->n_hubs, d.ws.hubs);
         first = 0; deg = 0;
         if (newly) payload_run(d, (int)(j >> 4), first, deg);
         if (__any_sync(FULL, deg > 0))
@@ -231,7 +231,10 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
     static_assert(U == 1, "one warp step per task");
-    const int n_tasks = d.ws.ctr->n_tasks;
+    const int n_recs = d.ws.ctr->n_tasks, n_hubs = min(d.ws.ctr->n_hubs, HUB_CAP);
+    const HubTable hubs = load_hub_table(d.ws.hubs, n_hubs, lane);
+    const int n_tasks = n_recs + hubs.total;                       // task records, then the steps of the hub runs
+    auto item = [&](int i) { return worklist_item(d.ws.tasks, n_recs, hubs, i); };
     // A task is a chain of dependent loads (record -> entries, column end, mask, x block); the
     // loop is software-pipelined: while task k is evaluated, the loads of k+1 and the record of
     // k+2 (in this warp's stride) are in flight.
@@ -251,10 +254,10 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
         return l;
     };
     const uint2 none = make_uint2(0u, 0u);
-    uint2 rec1 = gwarp + nwarps < n_tasks ? d.ws.tasks[gwarp + nwarps] : none;
-    Loads cur = loads_of(gwarp, gwarp < n_tasks ? d.ws.tasks[gwarp] : none);
+    uint2 rec1 = gwarp + nwarps < n_tasks ? item(gwarp + nwarps) : none;
+    Loads cur = loads_of(gwarp, gwarp < n_tasks ? item(gwarp) : none);
     for (int t = gwarp; t < n_tasks; t += nwarps) {
-        const uint2 rec2 = t + 2 * nwarps < n_tasks ? d.ws.tasks[t + 2 * nwarps] : none;
+        const uint2 rec2 = t + 2 * nwarps < n_tasks ? item(t + 2 * nwarps) : none;
         const Loads nxt = loads_of(t + nwarps, rec1);
         rec1 = rec2;
         uint32_t idx[U] = {cur.idx}, w[U] = {cur.w}, aux[U] = {cur.aux};
@@ -806,6 +809,7 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
             c2->last_path = c2->path;
             c2->n_nzblk = 0;
             c2->n_tasks = 0;
+            c2->n_hubs = 0;
         }
     }
     // vector-block state of this call's x: clear the masks and put the "not listed" marker back
@@ -841,6 +845,7 @@ __global__ void k_decode_cleanup(Device d) {
         c->last_y_nnz = (int32_t)d.m;
         c->n_nzblk = 0;
         c->n_tasks = 0;
+        c->n_hubs = 0;
     }
 }
 
@@ -920,6 +925,8 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     DBS_WS(dev_alloc_zero(&ws.x_dense, xwords * 32, &total));
     DBS_WS(dev_alloc_zero(&ws.x_mask32, xwords, &total));
     DBS_WS(dev_alloc_zero(&ws.tasks, (size_t)ws.task_capacity, &total));
+    DBS_WS(dev_alloc_zero(&ws.hubs, (size_t)2 * HUB_CAP, &total));
+    DBS_WS(dev_alloc_zero(&ws.bfs_words, xwords, &total));
     DBS_WS(dev_alloc_zero(&ws.y_acc, ywords * 32, &total));
     DBS_WS(dev_alloc_zero(&ws.y_mask32, ywords, &total));
     DBS_WS(dev_alloc_zero(&ws.y_hit8, ywords * 32, &total));

@@ -16,7 +16,14 @@ namespace dbs {
 // otherwise).  The count of nonempty vector blocks is aggregated the same way.
 template <bool CTA_WIDE = false>
 __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, int first, int deg, int lane,
-                                           int32_t *n_tasks, int32_t *n_nzblk, int chunk = PUSH_CHUNK) {
+                                           int32_t *n_tasks, int32_t *n_nzblk, int chunk = PUSH_CHUNK,
+                                           int32_t *n_hubs = nullptr, int4 *hubs = nullptr) {
+    // a hub run is listed, not cut up (writing tens of thousands of task records from one warp
+    // took longer than the traversal of the level they belonged to)
+    if (n_hubs && deg >= HUB_MIN_ENTRIES) {
+        const int slot = atomicAdd(n_hubs, 1);
+        if (slot < HUB_CAP) { hubs[slot] = make_int4(jb, first, deg, 0); deg = 0; }
+    }
     const int nchunks = (deg + chunk - 1) / chunk;
     int incl = nchunks;
     for (int o = 1; o < 32; o <<= 1) {
@@ -73,6 +80,42 @@ __device__ __forceinline__ void emit_tasks(const Device &d, bool newly, int jb, 
             d.ws.tasks[bbase + k] = make_uint2((uint32_t)bjb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(bfirst + k * chunk));
         }
     }
+}
+
+// The listed hub runs of one worklist, held by a warp in registers: lane h keeps hub h, the
+// number of its 32-entry steps and the number of steps of the hubs before it.
+struct HubTable {
+    int4 hub;        // (column block, first position, entries, -) of hub number `lane`
+    int start;       // steps of the hubs before this one
+    int steps;       // steps of this one (0: no hub in this lane)
+    int total;       // steps of all hubs (warp-uniform)
+};
+__device__ __forceinline__ HubTable load_hub_table(const int4 *hubs, int n_hubs, int lane) {
+    static_assert(HUB_CAP <= 32, "one hub per lane");
+    HubTable t;
+    t.hub = lane < n_hubs ? hubs[lane] : make_int4(0, 0, 0, 0);
+    t.steps = (t.hub.z + PUSH_CHUNK - 1) / PUSH_CHUNK;
+    int incl = t.steps;
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    t.start = incl - t.steps;
+    t.total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    return t;
+}
+// Item i of a push worklist made of n_tasks task records followed by the steps of the hub runs.
+// Called by a full warp with a warp-uniform i.
+__device__ __forceinline__ uint2 worklist_item(const uint2 *tasks, int n_tasks, const HubTable &t, int i) {
+    if (i < n_tasks) return tasks[i];
+    const int k = i - n_tasks;
+    const uint32_t m = __ballot_sync(0xFFFFFFFFu, k >= t.start && k < t.start + t.steps);
+    if (!m) return make_uint2(0u, 0u);
+    const int src = __ffs(m) - 1;
+    const int jb = __shfl_sync(0xFFFFFFFFu, t.hub.x, src), first = __shfl_sync(0xFFFFFFFFu, t.hub.y, src);
+    const int deg = __shfl_sync(0xFFFFFFFFu, t.hub.z, src), kk = k - __shfl_sync(0xFFFFFFFFu, t.start, src);
+    const int cnt = min(PUSH_CHUNK, deg - kk * PUSH_CHUNK);
+    return make_uint2((uint32_t)jb | ((uint32_t)(cnt - 1) << 27), (uint32_t)(first + kk * PUSH_CHUNK));
 }
 
 // The two kinds of run of a column block in the block-CSC view (see View::colptr).

@@ -138,3 +138,22 @@ def test_auto_switches_direction_across_levels():
         assert p == (B.PATH_PUSH if np.float32(k) / np.float32(nblk) < np.float32(0.01) else B.PATH_PULL)
     assert B.PATH_PUSH in paths and B.PATH_PULL in paths
     h.close()
+
+
+def test_hub_column_goes_through_the_hub_list():
+    """A star with 12,000 leaves: the centre's column holds more INLINE elements than the hub
+    threshold, so its push is not cut into tasks but strided over by all warps."""
+    n = 12001
+    rows = np.r_[np.zeros(n - 1, np.int64), np.arange(1, n)]
+    cols = np.r_[np.arange(1, n), np.zeros(n - 1, np.int64)]
+    order = np.lexsort((cols, rows))
+    rows, cols = rows[order], cols[order]
+    row_ptr = np.r_[0, np.cumsum(np.bincount(rows, minlength=n))].astype(np.int64)
+    g = wl.CSR(n, n, row_ptr, cols.astype(np.int32), None)
+    A = ref_matrix(g)
+    for path in (B.PATH_PUSH, B.PATH_AUTO):
+        h = Handle(g, B.PATTERN)
+        h.set_opts(force_path=path)
+        for s in (5, 0, n - 1):
+            assert np.array_equal(bfs(h, s), oracle.ref_bfs(A, s)), f"source {s}"
+        h.close()

@@ -245,3 +245,22 @@ def test_page_locked_host_buffers_are_read_and_written_in_place(frac):
             check_against_oracle((yi[:k].numpy(), yv[:k].numpy(), k), oracle.ref_pull(A, x.idx, x.val))
             check_against_oracle(h.run(x), oracle.ref_pull(A, x.idx, x.val))      # device buffers, same handle
     h.close()
+
+
+def test_hub_column_goes_through_the_hub_list():
+    """One column with 9,000 stored elements (more than the hub threshold) among sparse ones:
+    its push run is listed once and strided over by all warps instead of being cut into tasks."""
+    m, n = 9000, 64
+    bg = wl.random_sparse(m, n, 3000, 11)
+    dense = np.zeros((m, n), dtype=np.float32)
+    dense[bg.rows(), bg.col_idx] = bg.val
+    dense[:, 7] = np.linspace(0.5, 1.5, m, dtype=np.float32)
+    csr = wl.csr_from_dense(dense)
+    h = Handle(csr, B.F32)
+    A = ref_matrix(csr)
+    for path in PATHS:
+        h.set_opts(force_path=path)
+        for idx in ([7], [3, 7, 40], list(range(0, 64, 3))):
+            x = wl.SparseVec(n, np.array(idx, dtype=np.int32), np.linspace(1.0, 2.0, len(idx), dtype=np.float32))
+            check_against_oracle(h.run(x), oracle.ref_pull(A, x.idx, x.val))
+    h.close()
