@@ -14,7 +14,10 @@ namespace cg = cooperative_groups;
 
 namespace dbs {
 
-constexpr int BFS_CTA = 128;
+#ifndef DBS_BFS_CTA
+#define DBS_BFS_CTA 1024   // one thread block per SM: a grid barrier over 148 blocks costs far less than over a thousand
+#endif
+constexpr int BFS_CTA = DBS_BFS_CTA;
 
 // Rows of one hypersparse block reached from the active columns (one lane per block).
 template <int DT>
