@@ -692,7 +692,7 @@ template <int MODE> constexpr size_t compute_dyn_smem() {
 }
 
 template <int DT, typename Out, int MODE>
-__global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold) {
+__global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold, int pull_done) {
     constexpr bool HV = MODE >= 1;
     __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16 * SY_COPIES];
     extern __shared__ __align__(128) uint8_t s_dyn[];
@@ -704,8 +704,56 @@ __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out
     const int path = select_path(d, th3, force_path);
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
     float *lacc = HV ? s_lacc + warp * 16 * LANE_ACC_STRIDE : nullptr;
+    if (pull_done && path == DBSPMSPV_PATH_PULL) return;     // (the decode entry's own pull kernel has run)
     if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], lacc);
     else pull_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], lacc, &s_pull[warp]);
+}
+
+// Pull of the decode entry for matrices whose elements sit mostly in mask-based blocks (pruned
+// layers): one warp per pull segment, the segment's view entries read straight from global
+// memory, mask-based blocks walked by the half-warp streaming form, sums added to the dense y
+// with one atomic per row and half-warp.  No shared memory and few registers: twice the warps per
+// SM of the general traversal kernel, which is what this latency-bound walk needs.  Does nothing
+// unless the selector says pull; the general kernel, launched next, then only runs the push.
+template <int DT>
+__global__ void __launch_bounds__(CTA) k_decode_pull(Device d, float *__restrict__ y, float th3, int force_path) {
+    pdl_wait();
+    pdl_launch_dependents();
+    if (select_path(d, th3, force_path) != DBSPMSPV_PATH_PULL) return;
+    if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = DBSPMSPV_PATH_PULL;
+    const int lane = threadIdx.x & 31;
+    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    auto emit = [&](int erb, int erow, float esum) { atomicAdd(y + (size_t)erb * 16 + erow, esum); };
+    for (int sg = gwarp; sg < d.n_segments; sg += nwarps) {
+        const Segment seg = d.segments[sg];
+        const int rb = seg.row_block, cnt = seg.count & 0x7FFFFFFF;
+        for (int base = 0; base < cnt; base += 32) {
+            const bool have = base + lane < cnt;
+            const int p = seg.start + base + lane;
+            uint32_t idx = 0, w = 0, aux = 0, xm = 0;
+            if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; xm = mask_of(d.ws.x_mask32, idx & IDX_MASK); }
+            const int type = idx >> TYPE_SHIFT;
+            const bool mk = have && xm && type > DBSPMSPV_BLK_COO;
+            const uint32_t all = __ballot_sync(FULL, mk), rows = __ballot_sync(FULL, mk && is_row_major(type));
+            if (all & ~rows) half_stream<DT, false>(d.payload, d.ws.x_dense, idx, w, xm, rb, all & ~rows, lane, emit);
+            if (rows) half_stream<DT, true>(d.payload, d.ws.x_dense, idx, w, xm, rb, rows, lane, emit);
+            if (have && xm && type <= DBSPMSPV_BLK_COO) {       // the odd hypersparse block: its own lane
+                const float *xb = d.ws.x_dense + (size_t)(idx & IDX_MASK) * 16;
+                float *row0 = y + (size_t)rb * 16;
+                if (type == DBSPMSPV_BLK_INLINE) {
+                    if ((xm >> (aux & 15)) & 1u) atomicAdd(row0 + (aux >> 4), Val<DT>::inline_value(w) * xb[aux & 15]);
+                } else {
+                    const int nnz = (int)aux + 1;
+                    const uint8_t *blk = d.payload + (size_t)w * 4, *vals = blk + ((nnz + 3) & ~3);
+                    for (int k = 0; k < nnz; ++k) {
+                        const int c = blk[k] & 15, r = blk[k] >> 4;
+                        if ((xm >> c) & 1u) atomicAdd(row0 + r, Val<DT>::load(vals, k) * xb[c]);
+                    }
+                }
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -909,15 +957,15 @@ template <int DT, typename Out, int MODE> static int compute_grid(int sm_count) 
 }
 
 template <int DT, typename Out, int MODE>
-static int launch_compute(dbspmspv_handle_s *h, Out out, float th3, bool pdl, cudaStream_t st) {
+static int launch_compute(dbspmspv_handle_s *h, Out out, float th3, bool pdl, cudaStream_t st, int pull_done = 0) {
     static int grid = 0;
     if (!grid) grid = compute_grid<DT, Out, MODE>(h->sm_count);
     if (!grid) return DBSPMSPV_ERR_CUDA;
     const size_t smem = compute_dyn_smem<MODE>();
     if (pdl) {
-        DBS_CUDA(launch_pdl(k_compute<DT, Out, MODE>, grid, CTA, smem, st, h->d, out, th3, h->ropts.force_path, h->ropts.popc_threshold));
+        DBS_CUDA(launch_pdl(k_compute<DT, Out, MODE>, grid, CTA, smem, st, h->d, out, th3, h->ropts.force_path, h->ropts.popc_threshold, pull_done));
     } else {
-        k_compute<DT, Out, MODE><<<grid, CTA, smem, st>>>(h->d, out, th3, h->ropts.force_path, h->ropts.popc_threshold);
+        k_compute<DT, Out, MODE><<<grid, CTA, smem, st>>>(h->d, out, th3, h->ropts.force_path, h->ropts.popc_threshold, pull_done);
     }
     ++h->kernel_launches;
     return DBSPMSPV_OK;
@@ -999,8 +1047,21 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
     OutDense out{y, nullptr};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
     if (d.n_entries > 0) {
-        const int s = h->heavy_stage ? launch_compute<DT, OutDense, 1>(h, out, h->ropts.th3_decode, true, st)
-                                     : launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, true, st);
+        int s;
+        if (h->heavy_stage) {
+            // pull by the lean kernel of its own; the general kernel then only runs a push
+            static int grid = 0;
+            if (!grid) {
+                int per_sm = 0;
+                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_decode_pull<DT>, CTA, 0) != cudaSuccess || per_sm < 1) return DBSPMSPV_ERR_CUDA;
+                grid = per_sm * h->sm_count;
+            }
+            DBS_CUDA(launch_pdl(k_decode_pull<DT>, grid, CTA, 0, st, d, y, h->ropts.th3_decode, h->ropts.force_path));
+            ++h->kernel_launches;
+            s = launch_compute<DT, OutDense, 1>(h, out, h->ropts.th3_decode, true, st, 1);
+        } else {
+            s = launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, true, st);
+        }
         if (s != DBSPMSPV_OK) return s;
     }
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
