@@ -31,7 +31,7 @@ def check(y, want, scale):
 
 
 @pytest.mark.parametrize("shape", [(192, 256), (1000, 333), (333, 1000)])
-@pytest.mark.parametrize("prune,zf", [(0.5, 0.7), (0.5, 0.9), (0.7, 0.9)])
+@pytest.mark.parametrize("prune,zf", [(0.5, 0.7), (0.5, 0.9), (0.7, 0.9), (0.95, 0.7)])
 def test_decode_parity_bf16(shape, prune, zf):
     m, n = shape
     w = wl.pruned_weight(m, n, prune, seed=5, stream=m)
@@ -85,3 +85,22 @@ def test_decode_rejects_pattern_handles():
         B.dbspmspv_decode(h.h, t, t)
     assert e.value.status == B.ERR_UNSUPPORTED
     h.close()
+
+
+@pytest.mark.parametrize("inline_max", [31, 3])
+def test_decode_on_a_matrix_with_every_block_class(inline_max):
+    """Planted dense, row-skewed, column-skewed and banded blocks over a sparse background
+    (with inline_max = 3 also packed-COO blocks): the decode entry's own pull kernel meets every
+    class, row-major and column-major, and the push goes through the general kernel."""
+    from test_gpu_format import mixed_matrix
+    a = mixed_matrix(160, 176, 9)
+    o = B.default_create_opts()
+    o.inline_max = inline_max
+    x = wl.relu_activation(a.n, 0.6, seed=3, stream=61)
+    for dtype in (B.F32, B.BF16):
+        h = Handle(a, dtype, opts=o)
+        want, scale = oracle.ref_decode(ref_matrix(a, bf16=dtype == B.BF16), x if dtype == B.F32 else wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x)))
+        for p in PATHS:
+            h.set_opts(force_path=p)
+            check(decode(h, x), want, scale)
+        h.close()
