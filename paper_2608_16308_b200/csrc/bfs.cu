@@ -50,7 +50,7 @@ __device__ __forceinline__ void write_levels(int32_t *levels, int rb, uint32_t f
 // pipelined: while task k is evaluated, the visited masks of k+1, the view entries of k+2 and
 // the task record of k+3 (in this warp's stride) are in flight.
 template <int DT>
-__device__ void bfs_push(const Device &d, int n_recs, const int4 *hubs, int n_hubs, int32_t *levels, int depth) {
+__device__ void bfs_push(const Device &d, const uint32_t *F, uint32_t *N, int n_recs, const int4 *hubs, int n_hubs, int32_t *levels, int depth) {
     static_assert(PUSH_CHUNK == 32, "one warp step per task");
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -67,7 +67,7 @@ __device__ void bfs_push(const Device &d, int n_recs, const int4 *hubs, int n_hu
             e.n = (int)(task.x >> 27) + 1;
             e.start = start;
             if (lane < e.n) { e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane]; }
-            e.xm = mask_of(d.ws.x_mask32, jb);
+            e.xm = mask_of(F, jb);
         }
         return e;
     };
@@ -104,7 +104,7 @@ __device__ void bfs_push(const Device &d, int n_recs, const int4 *hubs, int n_hu
                 hit &= need0;
                 if (hit) {
                     const int sh = (brow & 1) * 16;
-                    const uint32_t old = atomicOr(&d.ws.y_mask32[brow >> 1], hit << sh);
+                    const uint32_t old = atomicOr(&N[brow >> 1], hit << sh);
                     write_levels(levels, brow, hit & ~(old >> sh), depth);
                 }
             }
@@ -120,7 +120,7 @@ __device__ void bfs_push(const Device &d, int n_recs, const int4 *hubs, int n_hu
                 hits &= ~mask_of(d.ws.visited32, bbrow);
                 if (lane == 0 && hits) {
                     const int sh = (bbrow & 1) * 16;
-                    const uint32_t old = atomicOr(&d.ws.y_mask32[bbrow >> 1], hits << sh);
+                    const uint32_t old = atomicOr(&N[bbrow >> 1], hits << sh);
                     write_levels(levels, bbrow, hits & ~(old >> sh), depth);
                 }
             }
@@ -137,7 +137,7 @@ __device__ void bfs_push(const Device &d, int n_recs, const int4 *hubs, int n_hu
 // last link is waited for: while segment k is evaluated, the entries of k+1, the visited mask
 // of k+2 and the descriptor of k+3 (k counted in this warp's stride) are already in flight.
 template <int DT>
-__device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
+__device__ void bfs_pull(const Device &d, const uint32_t *F, uint32_t *N, int32_t *levels, int depth) {
     constexpr int U = MAX_SEG_ENTRIES / 32;
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -186,7 +186,7 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
             for (int u = 0; u < U; ++u) {
                 const bool inl = (idx0[u] >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE;
                 const bool want = rem0 > u * 32 && (!inl || ((need0 >> (aux0[u] >> 4)) & 1u));
-                xm[u] = want ? mask_of(d.ws.x_mask32, idx0[u] & IDX_MASK) : 0u;
+                xm[u] = want ? mask_of(F, idx0[u] & IDX_MASK) : 0u;
                 heavy_any |= want && !inl;
             }
             uint32_t hit = 0;
@@ -224,11 +224,11 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
             hit = __reduce_or_sync(FULL, hit) & need0;
             if (hit) {
                 if (s0.count < 0) {          // the segment is its whole row block: plain stores
-                    if (lane == 0) reinterpret_cast<uint16_t *>(d.ws.y_mask32)[rb] = (uint16_t)hit;
+                    if (lane == 0) reinterpret_cast<uint16_t *>(N)[rb] = (uint16_t)hit;
                     if (lane < 16 && ((hit >> lane) & 1u)) levels[rb * 16 + lane] = depth;
                 } else if (lane == 0) {
                     const int sh = (rb & 1) * 16;
-                    const uint32_t old = atomicOr(&d.ws.y_mask32[rb >> 1], hit << sh);
+                    const uint32_t old = atomicOr(&N[rb >> 1], hit << sh);
                     write_levels(levels, rb, hit & ~(old >> sh), depth);
                 }
             }
@@ -251,15 +251,30 @@ __device__ void bfs_pull(const Device &d, int32_t *levels, int depth) {
 // long (a hub with no frontier neighbour so far) and is finished by the whole warp, 32 entries
 // per step.  The warp owns its mask word: plain stores, no atomics.
 template <int DT>
-__device__ void bfs_pull_rows(const Device &d, int32_t *levels, int depth) {
+__device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, uint32_t *Z, int32_t *nz_out, int32_t *nwords_out,
+                              int32_t *levels, int depth) {
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
     const int n_words = (d.mb + 1) / 2;
     constexpr uint32_t NONE = 0xFFFFFFFFu;          // no entry: local column 31 never matches a 16-bit mask
+    // This traversal also does the level's bookkeeping for its word (it owns it): the new
+    // frontier word is stored whatever its value (the buffer is not cleared beforehand), the
+    // buffer that comes into use two levels on is cleared, visited is updated, and the nonempty
+    // blocks, the vertices found and the nonzero words are counted / listed (in batches of 32
+    // words per warp) -- so a pull level needs no separate update pass and one grid barrier less.
+    int n_found = 0, n_nz = 0, n_batch = 0, batch_wd = 0;
+    auto flush_batch = [&]() {
+        int base = 0;
+        if (lane == 0) base = atomicAdd(nwords_out, n_batch);
+        base = __shfl_sync(FULL, base, 0);
+        if (lane < n_batch) d.ws.bfs_words[base + lane] = batch_wd;
+        n_batch = 0;
+    };
     for (int wd = gwarp; wd < n_words; wd += nwarps) {
         const uint32_t need = ~d.ws.visited32[wd];   // (rows without stored elements and rows past m count as visited)
-        if (!need) continue;
+        if (lane == 0) Z[wd] = 0u;
+        if (!need) { if (lane == 0) N[wd] = 0u; continue; }
         uint32_t found = 0;
         // entries with a payload, one per lane
 #pragma unroll
@@ -272,7 +287,7 @@ __device__ void bfs_pull_rows(const Device &d, int32_t *levels, int depth) {
             for (int q = pbeg + lane; q < pend; q += 32) {
                 const int pos = d.payload_pos[q];
                 const uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
-                const uint32_t xm = mask_of(d.ws.x_mask32, idx & IDX_MASK);
+                const uint32_t xm = mask_of(F, idx & IDX_MASK);
                 if (xm) {
                     const int type = idx >> TYPE_SHIFT;
                     const uint32_t w = d.csr.w[pos];
@@ -293,7 +308,7 @@ __device__ void bfs_pull_rows(const Device &d, int32_t *levels, int depth) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) v[j] = (active && p + j < e) ? d.rowrun_idx[p + j] : NONE;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) xm[j] = v[j] != NONE ? mask_of(d.ws.x_mask32, v[j] & IDX_MASK) : 0u;
+            for (int j = 0; j < 4; ++j) xm[j] = v[j] != NONE ? mask_of(F, v[j] & IDX_MASK) : 0u;
 #pragma unroll
             for (int j = 0; j < 4; ++j) got |= ((xm[j] >> (v[j] >> 27)) & 1u) != 0;
             p += 4;
@@ -307,17 +322,24 @@ __device__ void bfs_pull_rows(const Device &d, int32_t *levels, int depth) {
             bool hit = false;
             for (int q = lp; q < le && !hit; q += 32) {
                 const uint32_t v = q + lane < le ? d.rowrun_idx[q + lane] : NONE;
-                const uint32_t xm = v != NONE ? mask_of(d.ws.x_mask32, v & IDX_MASK) : 0u;
+                const uint32_t xm = v != NONE ? mask_of(F, v & IDX_MASK) : 0u;
                 hit = __any_sync(FULL, (xm >> (v >> 27)) & 1u);
             }
             if (lane == src) got = hit;
         }
         found = (found | __ballot_sync(FULL, got)) & need;
+        if (lane == 0) N[wd] = found;
         if (found) {
-            if (lane == 0) d.ws.y_mask32[wd] = found;
+            if (lane == 0) d.ws.visited32[wd] |= found;
             if ((found >> lane) & 1u) levels[row] = depth;
+            n_found += __popc(found);
+            n_nz += ((found & 0xFFFFu) != 0) + ((found >> 16) != 0);
+            if (lane == n_batch) batch_wd = wd;
+            if (++n_batch == 32) flush_batch();
         }
     }
+    if (n_batch) flush_batch();
+    if (lane == 0 && n_found) { atomicAdd(&d.ws.ctr->bfs_reached, n_found); atomicAdd(nz_out, n_nz); }
 }
 
 // Per-level selector (Section 3.3.1): push iff N_nzblk / N_blk < th3.  Monotone in n_nzblk.
@@ -341,8 +363,11 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
     // rows without a stored element can never be reached through a pull: they start out as
     // "visited", so that a row block is skipped (and a segment left early) once every row that
     // can be found has been found
-    for (int k = tid; k < n_words; k += nthreads) { d.ws.visited32[k] = ~d.row_present32[k]; d.ws.x_mask32[k] = 0u; d.ws.y_mask32[k] = 0u; }
-    if (tid == 0) { ctr->bfs_cnt[0][0] = 0; ctr->bfs_cnt[0][1] = 0; ctr->bfs_cnt[1][0] = 0; ctr->bfs_cnt[1][1] = 0; ctr->bfs_hubs[0] = 0; ctr->bfs_hubs[1] = 0; ctr->bfs_reached = 1; }
+    for (int k = tid; k < n_words; k += nthreads) { d.ws.visited32[k] = ~d.row_present32[k]; d.ws.x_mask32[k] = 0u; d.ws.y_mask32[k] = 0u; d.ws.z_mask32[k] = 0u; }
+    if (tid == 0) {
+        for (int k = 0; k < 3; ++k) { ctr->bfs_cnt[k][0] = 0; ctr->bfs_cnt[k][1] = 0; ctr->bfs_hubs[k] = 0; ctr->bfs_nwords[k] = 0; }
+        ctr->bfs_reached = 1;
+    }
     grid.sync();
     // level 0: the source is the first frontier
     if (blockIdx.x == 0 && threadIdx.x < 32) {
@@ -360,6 +385,9 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
     }
     grid.sync();
 
+    // Three mask buffers rotate: F holds the frontier, N receives the next one, Z is cleared while
+    // the level runs and becomes N of the next level (the old F becomes Z).
+    uint32_t *F = d.ws.x_mask32, *N = d.ws.y_mask32, *Z = d.ws.z_mask32;
     int cur = 0, depth = 0;
     while (depth < max_levels) {
         const int n_nzblk = ctr->bfs_cnt[cur][0];
@@ -367,80 +395,91 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         if (n_nzblk == 0) break;
         ++depth;
         const int path = bfs_path(n_nzblk, d.nb, th3, force_path);
+        // per-level counters: `cur` holds this level's, `nxt` is accumulated for the next level,
+        // `spare` (the previous level's, read for the last time before the barriers of that
+        // level) is reset now and accumulated into at the next level
+        const int nxt = (cur + 1) % 3, spare = (cur + 2) % 3;
         if (tid == 0) {
-            ctr->bfs_cnt[cur ^ 1][0] = 0;
-            ctr->bfs_cnt[cur ^ 1][1] = 0;
-            ctr->bfs_hubs[cur ^ 1] = 0;
-            ctr->bfs_nwords = 0;
+            ctr->bfs_cnt[spare][0] = 0;
+            ctr->bfs_cnt[spare][1] = 0;
+            ctr->bfs_hubs[spare] = 0;
+            ctr->bfs_nwords[spare] = 0;
             if (depth <= DBSPMSPV_MAX_BFS_LEVELS_RECORDED) {
                 ctr->bfs_level_path[depth - 1] = path;
                 ctr->bfs_level_nzblk[depth - 1] = n_nzblk;
             }
         }
-        if (path == DBSPMSPV_PATH_PUSH) bfs_push<DT>(d, n_tasks, d.ws.hubs + cur * HUB_CAP, min(ctr->bfs_hubs[cur], HUB_CAP), levels, depth);
-        else if (d.rowrun_ptr) bfs_pull_rows<DT>(d, levels, depth);
-        else bfs_pull<DT>(d, levels, depth);
-        grid.sync();
-        // next frontier: masks produced above become the vector-block masks of the next level,
-        // visited is updated and the nonempty blocks are counted (one atomic per warp)
-        int found = 0, nz = 0;
-        for (int k0 = tid & ~31; k0 < n_words; k0 += nthreads) {
-            const int k = k0 + lane;
-            uint32_t nm = 0;
-            if (k < n_words) {
-                nm = d.ws.y_mask32[k];
-                if (nm) {
-                    d.ws.y_mask32[k] = 0u;
-                    d.ws.visited32[k] |= nm;
-                    found += __popc(nm);
-                    nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
+        const bool fused = path != DBSPMSPV_PATH_PUSH && d.rowrun_ptr != nullptr;
+        if (fused) {
+            bfs_pull_rows<DT>(d, F, N, Z, &ctr->bfs_cnt[nxt][0], &ctr->bfs_nwords[nxt], levels, depth);
+            grid.sync();
+        } else {
+            if (path == DBSPMSPV_PATH_PUSH) bfs_push<DT>(d, F, N, n_tasks, d.ws.hubs + cur * HUB_CAP, min(ctr->bfs_hubs[cur], HUB_CAP), levels, depth);
+            else bfs_pull<DT>(d, F, N, levels, depth);
+            grid.sync();
+            // the masks produced above are the next frontier: visited is updated, the nonempty
+            // blocks are counted (one atomic per warp), the nonzero words listed so that a
+            // worklist rebuild can share them out evenly, and the spare buffer is cleared
+            int found = 0, nz = 0;
+            for (int k0 = tid & ~31; k0 < n_words; k0 += nthreads) {
+                const int k = k0 + lane;
+                uint32_t nm = 0;
+                if (k < n_words) {
+                    nm = N[k];
+                    if (nm) {
+                        d.ws.visited32[k] |= nm;
+                        found += __popc(nm);
+                        nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
+                    }
+                    if (Z[k]) Z[k] = 0u;
                 }
-                if (nm || d.ws.x_mask32[k]) d.ws.x_mask32[k] = nm;
+                const uint32_t nzw = __ballot_sync(FULL, nm != 0u);
+                if (nzw) {
+                    int base = 0;
+                    if (lane == 0) base = atomicAdd(&ctr->bfs_nwords[nxt], __popc(nzw));
+                    base = __shfl_sync(FULL, base, 0);
+                    if (nm) d.ws.bfs_words[base + __popc(nzw & ((1u << lane) - 1u))] = k;
+                }
             }
-            // the nonzero words are listed, so that a worklist rebuild can share them out evenly
-            const uint32_t nzw = __ballot_sync(FULL, nm != 0u);
-            if (nzw) {
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&ctr->bfs_nwords, __popc(nzw));
-                base = __shfl_sync(FULL, base, 0);
-                if (nm) d.ws.bfs_words[base + __popc(nzw & ((1u << lane) - 1u))] = k;
-            }
+            found = __reduce_add_sync(FULL, found);
+            nz = __reduce_add_sync(FULL, nz);
+            if (lane == 0 && found) { atomicAdd(&ctr->bfs_reached, found); atomicAdd(&ctr->bfs_cnt[nxt][0], nz); }
+            grid.sync();
         }
-        found = __reduce_add_sync(FULL, found);
-        nz = __reduce_add_sync(FULL, nz);
-        if (lane == 0 && found) { atomicAdd(&ctr->bfs_reached, found); atomicAdd(&ctr->bfs_cnt[cur ^ 1][0], nz); }
-        grid.sync();
+        { uint32_t *t = F; F = N; N = Z; Z = t; }       // rotate: the new frontier is what was written
         // the push worklist is rebuilt only if the next level is a push (the selector's input is
         // known now); its block count goes to a scratch counter
-        const int next_n = ctr->bfs_cnt[cur ^ 1][0];
+        const int next_n = ctr->bfs_cnt[nxt][0];
         if (next_n && bfs_path(next_n, d.nb, th3, force_path) == DBSPMSPV_PATH_PUSH) {
             // a warp takes one listed mask word (two vector blocks) at a time, lane = column:
             // frontier columns emit their INLINE runs (adjacent ones merged), lanes 0 and 16 the
             // payload runs of the two blocks.  (With the words in index order, the few warps that
             // held the hub blocks of an early frontier wrote almost the whole worklist.)
-            const int n_listed = ctr->bfs_nwords;
+            const int n_listed = ctr->bfs_nwords[nxt];
             for (int i = gwarp_all; i < n_listed; i += nwarps_all) {
                 const int wd = d.ws.bfs_words[i];
-                const uint32_t word = d.ws.x_mask32[wd];
+                const uint32_t word = F[wd];
                 const int jb = 2 * wd + (lane >> 4), j = jb * 16 + (lane & 15);
                 const bool listed = (word >> lane) & 1u;
                 int first = 0, deg = 0;
                 if (listed) column_run(d, j, first, deg);
                 merge_column_runs(listed, j, first, deg, lane);
-                emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad, PUSH_CHUNK,
-                           &ctr->bfs_hubs[cur ^ 1], d.ws.hubs + (cur ^ 1) * HUB_CAP);
+                emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[nxt][1], &ctr->pad, PUSH_CHUNK,
+                           &ctr->bfs_hubs[nxt], d.ws.hubs + nxt * HUB_CAP);
                 first = 0; deg = 0;
                 if ((lane & 15) == 0 && ((word >> lane) & 0xFFFFu)) payload_run(d, jb, first, deg);
                 if (__any_sync(FULL, deg > 0))
-                    emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[cur ^ 1][1], &ctr->pad, d.payload_chunk);
+                    emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[nxt][1], &ctr->pad, d.payload_chunk);
             }
             grid.sync();
         }
-        cur ^= 1;
+        cur = nxt;
     }
-    // leave the shared workspace as dbspmspv_run expects it: all masks clear
+    // leave the shared workspace as dbspmspv_run expects it: all masks clear (Z is the last
+    // frontier that was expanded; F is empty unless the level cap ended the search; N is clear)
+    for (int k = tid; k < n_words; k += nthreads) if (Z[k]) Z[k] = 0u;
     if (ctr->bfs_cnt[cur][0] != 0)
-        for (int k = tid; k < n_words; k += nthreads) d.ws.x_mask32[k] = 0u;
+        for (int k = tid; k < n_words; k += nthreads) F[k] = 0u;
     if (tid == 0) ctr->bfs_levels = depth;
 }
 

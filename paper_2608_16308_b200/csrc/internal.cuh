@@ -121,9 +121,11 @@ struct Counters {    // device-resident scalars of one call
     int32_t bfs_levels, bfs_reached;
     int32_t pad;
     int32_t n_hubs;         // hub runs of this call's push worklist (may exceed HUB_CAP: the rest became tasks)
-    int32_t bfs_hubs[2];    // BFS: the same per level, double buffered
-    int32_t bfs_nwords;     // BFS: nonzero words of the new frontier's masks (listed in Workspace::bfs_words)
-    int32_t bfs_cnt[2][2];  // BFS: {nonempty frontier blocks, tasks}, double buffered by level
+    int32_t bfs_hubs[3];    // BFS: the same per level (the per-level counters rotate three ways: the
+                            // level's own, the ones it accumulates for the next level, and a spare
+                            // set that is reset meanwhile)
+    int32_t bfs_nwords[3];  // BFS: nonzero words of the new frontier's masks (listed in Workspace::bfs_words)
+    int32_t bfs_cnt[3][2];  // BFS: {nonempty frontier blocks, tasks}
     int32_t bfs_level_path[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
     int32_t bfs_level_nzblk[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
 };
@@ -132,12 +134,13 @@ struct Workspace {
     float *x_dense;       // n (padded to a multiple of 32): dense copy of x (Section 3.2.2)
     uint32_t *x_mask32;   // vector-block masks, two 16-bit masks per word
     uint2 *tasks;         // push worklist: (column block | (entries - 1) << 27, first CSC-view position)
-    int4 *hubs;           // 2 x HUB_CAP hub runs (column block, first position, entries, -): see worklist.cuh
+    int4 *hubs;           // 3 x HUB_CAP hub runs (column block, first position, entries, -): see worklist.cuh
     float *y_acc;         // m (padded): dense accumulator, all zero between calls
     uint32_t *y_mask32;   // run: hit masks packed by the compaction pass; BFS: next-frontier masks
     uint8_t *y_hit8;      // run: one structural-hit flag byte per row, all zero between calls
     int32_t *tile_count;  // compaction: result entries per tile of row blocks
     uint32_t *visited32;  // BFS: visited masks
+    uint32_t *z_mask32;   // BFS: third mask buffer (frontier / next / being cleared rotate)
     int32_t *bfs_words;   // BFS: indices of the nonzero mask words of the new frontier
     Counters *ctr;
     int64_t task_capacity;

@@ -989,8 +989,9 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     DBS_WS(dev_alloc_zero(&ws.x_dense, xwords * 32, &total));
     DBS_WS(dev_alloc_zero(&ws.x_mask32, xwords, &total));
     DBS_WS(dev_alloc_zero(&ws.tasks, (size_t)ws.task_capacity, &total));
-    DBS_WS(dev_alloc_zero(&ws.hubs, (size_t)2 * HUB_CAP, &total));
+    DBS_WS(dev_alloc_zero(&ws.hubs, (size_t)3 * HUB_CAP, &total));
     DBS_WS(dev_alloc_zero(&ws.bfs_words, xwords, &total));
+    DBS_WS(dev_alloc_zero(&ws.z_mask32, xwords > ywords ? xwords : ywords, &total));
     DBS_WS(dev_alloc_zero(&ws.y_acc, ywords * 32, &total));
     DBS_WS(dev_alloc_zero(&ws.y_mask32, ywords, &total));
     DBS_WS(dev_alloc_zero(&ws.y_hit8, ywords * 32, &total));
