@@ -23,7 +23,10 @@ constexpr int TILE_WORDS = CMP_TPB / 4;  // a tile: 64 mask words = 2048 rows; p
 // claimed with a warp scan, a sum over the thread block's warps and one atomic per thread
 // block; the count of nonempty vector blocks is aggregated the same way (Section 4.1).
 // ------------------------------------------------------------------------------------------
-template <int DT>
+// EMIT = false: only the dense copy, the masks and the count -- the worklist is then built by
+// k_emit_from_masks, and only if the selector chooses the push (used when x is so dense that a
+// pull is likely: the tasks of half a million columns would be written for nothing).
+template <int DT, bool EMIT>
 __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, const void *__restrict__ x_val,
                                 int32_t nnz_x, int validate) {
     pdl_launch_dependents();
@@ -47,8 +50,7 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
             d.ws.x_dense[j] = __float_as_uint(v) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v;
             // the runs this thread may have to turn into tasks are fetched before the atomic
             // whose result decides it (the loads are independent of it; the chain is shorter)
-            column_run(d, j, first, deg);
-            payload_run(d, j >> 4, pfirst, pdeg);
+            if (EMIT) { column_run(d, j, first, deg); payload_run(d, j >> 4, pfirst, pdeg); }
             const int sh = ((j >> 4) & 1) * 16;
             const uint32_t old = atomicOr(&d.ws.x_mask32[j >> 5], 1u << ((j & 15) + sh));
             newly = ((old >> sh) & 0xFFFFu) == 0;
@@ -56,6 +58,10 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
             jb = j >> 4;
             jcol = j;
         }
+    }
+    if (!EMIT) {                                              // count the nonempty vector blocks, nothing else
+        emit_tasks<true>(d, newly, jb, 0, 0, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk);
+        return;
     }
     // push tasks: the INLINE elements of this column; and, by the thread that turned the vector
     // block nonempty, the column block's entries with a payload
@@ -76,6 +82,36 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
     if (!newly) pdeg = 0;
     if (__syncthreads_or(pdeg > 0))
         emit_tasks<true>(d, false, jb, pfirst, pdeg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, d.payload_chunk);
+}
+
+__device__ __forceinline__ int select_path(const Device &d, float th3, int force_path);
+
+// The push worklist from the finished vector-block masks (hypersparse matrices): runs only if
+// the selector chooses the push.  A warp takes one mask word (two vector blocks) at a time,
+// lane = column: listed columns emit their INLINE runs (adjacent ones merged), lanes 0 and 16
+// the payload runs of the two blocks.
+__global__ void k_emit_from_masks(Device d, float th3, int force_path) {
+    pdl_wait();
+    pdl_launch_dependents();
+    if (select_path(d, th3, force_path) != DBSPMSPV_PATH_PUSH) return;
+    const int lane = threadIdx.x & 31;
+    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int n_words = (d.nb + 1) / 2;
+    Counters *ctr = d.ws.ctr;
+    for (int wd = gwarp; wd < n_words; wd += nwarps) {
+        const uint32_t word = d.ws.x_mask32[wd];
+        if (!word) continue;                                   // warp-uniform
+        const int jb = 2 * wd + (lane >> 4), j = jb * 16 + (lane & 15);
+        const bool listed = (word >> lane) & 1u;
+        int first = 0, deg = 0;
+        if (listed) column_run(d, j, first, deg);
+        merge_column_runs(listed, j, first, deg, lane);
+        emit_tasks(d, false, jb, first, deg, lane, &ctr->n_tasks, &ctr->pad, PUSH_CHUNK, &ctr->n_hubs, d.ws.hubs);
+        first = 0; deg = 0;
+        if ((lane & 15) == 0 && ((word >> lane) & 0xFFFFu)) payload_run(d, jb, first, deg);
+        if (__any_sync(FULL, deg > 0)) emit_tasks(d, false, jb, first, deg, lane, &ctr->n_tasks, &ctr->pad, d.payload_chunk);
+    }
 }
 
 // Dense input (Sections 4.1, 4.3): every warp reads 32 elements, one ballot gives the two
@@ -1016,7 +1052,23 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
                      int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
                      cudaStream_t st) {
     const Device &d = h->d;
-    if (nnz_x > 0) { k_xblock_sparse<DT><<<(nnz_x + XB_TPB - 1) / XB_TPB, XB_TPB, 0, st>>>(d, x_idx, semiring == DBSPMSPV_OR_AND ? nullptr : x_val, nnz_x, h->ropts.validate); ++h->kernel_launches; }
+    // x lists a quarter of the columns or more: a pull is likely (on hypersparse matrices), so
+    // the worklist is built afterwards from the masks, and only if the selector does choose the push
+    const bool late_emit = !h->heavy_stage && h->ropts.force_path != DBSPMSPV_PATH_PUSH && (int64_t)nnz_x * 4 >= d.n;
+    const void *xv = semiring == DBSPMSPV_OR_AND ? nullptr : x_val;
+    if (nnz_x > 0) {
+        const int g = (nnz_x + XB_TPB - 1) / XB_TPB;
+        if (late_emit) {
+            k_xblock_sparse<DT, false><<<g, XB_TPB, 0, st>>>(d, x_idx, xv, nnz_x, h->ropts.validate);
+            int ge = ((d.nb + 1) / 2 + 7) / 8;
+            if (ge > 8 * h->sm_count) ge = 8 * h->sm_count;
+            DBS_CUDA(launch_pdl(k_emit_from_masks, ge, 256, 0, st, d, h->ropts.th3, h->ropts.force_path));
+            ++h->kernel_launches;
+        } else {
+            k_xblock_sparse<DT, true><<<g, XB_TPB, 0, st>>>(d, x_idx, xv, nnz_x, h->ropts.validate);
+        }
+        ++h->kernel_launches;
+    }
     OutSparse out{d.ws.y_acc, d.ws.y_hit8};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
     if (nnz_x > 0 && d.n_entries > 0) {

@@ -264,3 +264,24 @@ def test_hub_column_goes_through_the_hub_list():
             x = wl.SparseVec(n, np.array(idx, dtype=np.int32), np.linspace(1.0, 2.0, len(idx), dtype=np.float32))
             check_against_oracle(h.run(x), oracle.ref_pull(A, x.idx, x.val))
     h.close()
+
+
+def test_dense_but_clustered_x_takes_the_push_with_a_late_worklist():
+    """x lists more than a quarter of the columns, so the worklist is not built while x is
+    blocked -- but the listed columns fill only 40 % of the vector blocks, so the selector still
+    chooses the push and the worklist is built from the finished masks."""
+    csr = wl.rmat(12, 16, seed=5)
+    h = Handle(csr, B.F32)
+    A = ref_matrix(csr)
+    k = int(0.4 * csr.n) // 16 * 16
+    idx = np.arange(k, dtype=np.int32)
+    x = wl.SparseVec(csr.n, idx, np.linspace(-1.0, 1.0, k, dtype=np.float32) + 0.25)
+    want = oracle.ref_pull(A, x.idx, x.val)
+    check_against_oracle(h.run(x), want)
+    st = h.get_stats()
+    assert st.last_path == B.PATH_PUSH and st.last_n_nzblk == k // 16 and st.last_n_tasks > 0
+    h.set_opts(force_path=B.PATH_PULL)
+    check_against_oracle(h.run(x), want)
+    h.set_opts()
+    check_against_oracle(h.run(dense_x(csr.n, 3, 0.01)), oracle.ref_pull(A, dense_x(csr.n, 3, 0.01).idx, dense_x(csr.n, 3, 0.01).val))
+    h.close()
