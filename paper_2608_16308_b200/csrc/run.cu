@@ -513,7 +513,8 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
 #pragma unroll
             for (int u = 0; u < PULL_UNROLL; ++u) {
                 const bool have = base + u * 32 + lane < e1;
-                xin[u] = have ? d.ws.x_dense[(size_t)(idx[u] & IDX_MASK) * 16 + (aux[u] & 15)]
+                // (L2-only load: the 4-byte gathers hit L1 one time in ten and only evict each other there)
+                xin[u] = have ? __ldcg(&d.ws.x_dense[(size_t)(idx[u] & IDX_MASK) * 16 + (aux[u] & 15)])
                              : __uint_as_float(X_ABSENT);
             }
 #pragma unroll
