@@ -306,7 +306,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
         for (int round = 0; round < 8 && __any_sync(FULL, active); ++round) {
             uint32_t v[4], xm[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = (active && p + j < e) ? d.rowrun_idx[p + j] : NONE;
+            for (int j = 0; j < 4; ++j) v[j] = (active && p + j < e) ? __ldcs(&d.rowrun_idx[p + j]) : NONE;
 #pragma unroll
             for (int j = 0; j < 4; ++j) xm[j] = v[j] != NONE ? mask_of(F, v[j] & IDX_MASK) : 0u;
 #pragma unroll
