@@ -12,18 +12,38 @@
 namespace dbs {
 namespace {
 
-struct TempPool {  // device scratch of the build, released when the build returns
-    std::vector<void *> ptrs;
-    ~TempPool() { for (void *p : ptrs) cudaFree(p); }
+// Device scratch of the build.  A released block is kept and handed out again to a later request
+// it fits without much waste (the build's buffers come in a few sizes: one per stored entry, per
+// block, per view entry), because cudaMalloc/cudaFree cost more than most of the build's kernels;
+// everything goes back to the driver when the build returns, or earlier if an allocation fails.
+struct TempPool {
+    struct Block { void *p; size_t bytes; bool free; };
+    std::vector<Block> blocks;
+    ~TempPool() { for (auto &b : blocks) cudaFree(b.p); }
+    void trim() {
+        size_t k = 0;
+        for (auto &b : blocks) { if (b.free) cudaFree(b.p); else blocks[k++] = b; }
+        blocks.resize(k);
+    }
     template <typename T> bool get(T **out, size_t count) {
+        const size_t need = (count ? count : 1) * sizeof(T);
+        Block *best = nullptr;
+        for (auto &b : blocks)
+            if (b.free && b.bytes >= need && b.bytes <= need + need / 2 + 4096 && (!best || b.bytes < best->bytes)) best = &b;
+        if (best) { best->free = false; *out = static_cast<T *>(best->p); return true; }
         void *p = nullptr;
-        if (cudaMalloc(&p, (count ? count : 1) * sizeof(T)) != cudaSuccess) { *out = nullptr; return false; }
-        ptrs.push_back(p);
+        if (cudaMalloc(&p, need) != cudaSuccess) {
+            cudaGetLastError();
+            trim();
+            if (cudaMalloc(&p, need) != cudaSuccess) { *out = nullptr; return false; }
+        }
+        blocks.push_back({p, need, false});
         *out = static_cast<T *>(p);
         return true;
     }
+    // the caller has synchronised the stream that used the block
     void release(void *p) {
-        for (auto &q : ptrs) if (q == p) { cudaFree(p); q = nullptr; }
+        for (auto &b : blocks) if (b.p == p) b.free = true;
     }
 };
 
@@ -63,15 +83,19 @@ __global__ void k_keys_from_coo(int64_t m, int64_t n, int64_t nnz, const int32_t
     src[e] = (uint32_t)e;
 }
 
-// rows that hold at least one stored element, as 16-bit masks per row block (two per word)
+// rows that hold at least one stored element, as 16-bit masks per row block (two per word).
+// The keys are sorted by row block, so the lanes of a warp share a few words at most: the bits
+// of one word are combined in the warp and set with one atomic.
 __global__ void k_row_presence(int64_t nnzu, const uint64_t *ukey, uint32_t *row_present32) {
     int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (e >= nnzu) return;
-    const uint64_t k = ukey[e];
+    const bool have = e < nnzu;
+    const uint64_t k = have ? ukey[e] : 0;
     const int64_t rb = (int64_t)(k >> 35);
     const uint32_t bit = 1u << (((uint32_t)(k >> 4) & 15u) + (uint32_t)(rb & 1) * 16u);
-    uint32_t *word = row_present32 + (rb >> 1);
-    if (!(*word & bit)) atomicOr(word, bit);
+    const int word = have ? (int)(rb >> 1) : -1;
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, word);
+    const uint32_t bits = __reduce_or_sync(peers, bit);
+    if (have && (threadIdx.x & 31) == __ffs(peers) - 1) atomicOr(row_present32 + word, bits);
 }
 
 // ---- step 2: merge duplicates, find block boundaries
@@ -518,7 +542,9 @@ int bits_for(uint64_t v) { int b = 0; while (v) { ++b; v >>= 1; } return b ? b :
 #define DBS_TRY(expr) do { int s__ = (expr); if (s__ != DBSPMSPV_OK) return s__; } while (0)
 #define DBS_GET(ptr, count) do { if (!tp.get(&(ptr), (size_t)(count))) return DBSPMSPV_ERR_ALLOC; } while (0)
 #define DBS_KEEP(ptr, count) do { void *p__ = nullptr; \
-        if (cudaMalloc(&p__, ((count) ? (size_t)(count) : 1) * sizeof(*(ptr))) != cudaSuccess) return DBSPMSPV_ERR_ALLOC; \
+        const size_t b__ = ((count) ? (size_t)(count) : 1) * sizeof(*(ptr)); \
+        if (cudaMalloc(&p__, b__) != cudaSuccess) { cudaGetLastError(); tp.trim(); \
+            if (cudaMalloc(&p__, b__) != cudaSuccess) return DBSPMSPV_ERR_ALLOC; } \
         (ptr) = static_cast<decltype(ptr)>(p__); } while (0)
 
 int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t *row_ptr,
