@@ -139,13 +139,16 @@ __global__ void k_block_starts(int64_t nnzu, const int32_t *flag, const int32_t 
     blk_start[rank[u] - 1] = (int32_t)u;
 }
 
-// ---- step 3: classify (Section 3.2.1) and size every block.  One warp per block.
+// ---- step 3: classify (Section 3.2.1) and size every block.  A warp takes 32 consecutive
+// blocks, one per lane: below th0 stored elements (most blocks of a hypersparse matrix) the
+// class follows from the count alone; the blocks that need their row and column occupancy are
+// then walked one after the other by the whole warp.
 struct ClassifyParams {
     int th0, th1;
     float th2;
     int force_format;
     int dtype;
-    int inline_max;   // valued matrices: blocks with at most this many entries are stored inline
+    int inline_max;   // blocks with at most this many entries are stored inline
 };
 
 __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
@@ -157,46 +160,56 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x < DBSPMSPV_BLK_NCLASS) { s_cb[threadIdx.x] = 0; s_cn[threadIdx.x] = 0; }
     __syncthreads();
-    int64_t b = blockIdx.x * (int64_t)(TPB / 32) + warp;
-    if (b < n_blocks) {
+    const int64_t b = (blockIdx.x * (int64_t)(TPB / 32) + warp) * 32 + lane;
+    const bool have = b < n_blocks;
+    const int s = have ? blk_start[b] : 0, nnz = have ? blk_start[b + 1] - s : 0;
+    const bool by_shape = have && cp.force_format == DBSPMSPV_FORMAT_AUTO && nnz >= cp.th0 && nnz <= cp.th1;
+    int rmax = 0, cmax = 0;   // largest row / column count of this lane's block
+    for (uint32_t todo = __ballot_sync(0xFFFFFFFFu, by_shape); todo; todo &= todo - 1) {
+        const int src = __ffs(todo) - 1;
+        const int ss = __shfl_sync(0xFFFFFFFFu, s, src), nn = __shfl_sync(0xFFFFFFFFu, nnz, src);
         if (lane < 16) { s_row[warp][lane] = 0; s_col[warp][lane] = 0; }
         __syncwarp();
-        const int s = blk_start[b], nnz = blk_start[b + 1] - s;
-        for (int k = lane; k < nnz; k += 32) {
-            uint32_t rc = (uint32_t)(ukey[s + k] & 0xFF);
+        for (int k = lane; k < nn; k += 32) {
+            uint32_t rc = (uint32_t)(ukey[ss + k] & 0xFF);
             atomicOr(&s_row[warp][rc >> 4], 1u << (rc & 15));
             atomicOr(&s_col[warp][rc & 15], 1u << (rc >> 4));
         }
         __syncwarp();
         int rcount = lane < 16 ? __popc(s_row[warp][lane]) : 0;
         int ccount = lane < 16 ? __popc(s_col[warp][lane]) : 0;
-        for (int o = 8; o; o >>= 1) {
-            rcount = max(rcount, __shfl_xor_sync(0xFFFFFFFFu, rcount, o));
-            ccount = max(ccount, __shfl_xor_sync(0xFFFFFFFFu, ccount, o));
-        }
-        if (lane == 0) {
-            int type;
-            if (cp.force_format == DBSPMSPV_FORMAT_COO) type = DBSPMSPV_BLK_COO;
-            else if (cp.force_format == DBSPMSPV_FORMAT_CSR) type = DBSPMSPV_BLK_CSR;
-            else if (nnz < cp.th0) {
-                // one view entry per stored element, up to inline_max of them
-                type = nnz <= cp.inline_max ? DBSPMSPV_BLK_INLINE : DBSPMSPV_BLK_COO;
-            } else if (nnz > cp.th1) type = DBSPMSPV_BLK_DENSE;
-            // skew_c / skew_r = (max column count) / (max row count): the denominators of
-            // the two axis skews are identical for square blocks
-            else if ((float)ccount > cp.th2 * (float)rcount) type = DBSPMSPV_BLK_FCSC;
-            else if ((float)rcount > cp.th2 * (float)ccount) type = DBSPMSPV_BLK_FCSR;
-            else type = rcount <= CSR_SHORT_ROW ? BLK_CSR_ROWMAJOR : DBSPMSPV_BLK_CSR;
-            const int vsize = cp.dtype == DBSPMSPV_F32 ? 4 : cp.dtype == DBSPMSPV_BF16 ? 2 : 0;
-            type_out[b] = (uint8_t)type;
-            size_out[b] = (uint32_t)payload_words(type, nnz, vsize);
-            ecount[b] = type == DBSPMSPV_BLK_INLINE ? nnz : 1;
-            uint64_t k0 = ukey[s];
-            brow[b] = (int32_t)(k0 >> 35);
-            bcol[b] = (int32_t)((k0 >> 8) & IDX_MASK);
-            atomicAdd(&s_cb[public_class(type)], 1u);
-            atomicAdd(&s_cn[public_class(type)], (unsigned)nnz);
-        }
+        __syncwarp();
+        rcount = __reduce_max_sync(0xFFFFFFFFu, rcount);
+        ccount = __reduce_max_sync(0xFFFFFFFFu, ccount);
+        if (lane == src) { rmax = rcount; cmax = ccount; }
+    }
+    int type = -1;
+    if (have) {
+        if (cp.force_format == DBSPMSPV_FORMAT_COO) type = DBSPMSPV_BLK_COO;
+        else if (cp.force_format == DBSPMSPV_FORMAT_CSR) type = DBSPMSPV_BLK_CSR;
+        else if (nnz < cp.th0) {
+            // one view entry per stored element, up to inline_max of them
+            type = nnz <= cp.inline_max ? DBSPMSPV_BLK_INLINE : DBSPMSPV_BLK_COO;
+        } else if (nnz > cp.th1) type = DBSPMSPV_BLK_DENSE;
+        // skew_c / skew_r = (max column count) / (max row count): the denominators of
+        // the two axis skews are identical for square blocks
+        else if ((float)cmax > cp.th2 * (float)rmax) type = DBSPMSPV_BLK_FCSC;
+        else if ((float)rmax > cp.th2 * (float)cmax) type = DBSPMSPV_BLK_FCSR;
+        else type = rmax <= CSR_SHORT_ROW ? BLK_CSR_ROWMAJOR : DBSPMSPV_BLK_CSR;
+        const int vsize = cp.dtype == DBSPMSPV_F32 ? 4 : cp.dtype == DBSPMSPV_BF16 ? 2 : 0;
+        type_out[b] = (uint8_t)type;
+        size_out[b] = (uint32_t)payload_words(type, nnz, vsize);
+        ecount[b] = type == DBSPMSPV_BLK_INLINE ? nnz : 1;
+        const uint64_t k0 = ukey[s];
+        brow[b] = (int32_t)(k0 >> 35);
+        bcol[b] = (int32_t)((k0 >> 8) & IDX_MASK);
+    }
+    const int cls = have ? public_class(type) : -1;
+    for (int c = 0; c < DBSPMSPV_BLK_NCLASS; ++c) {
+        const uint32_t mine = __ballot_sync(0xFFFFFFFFu, cls == c);
+        if (!mine) continue;
+        const unsigned total = __reduce_add_sync(0xFFFFFFFFu, cls == c ? (unsigned)nnz : 0u);
+        if (lane == 0) { atomicAdd(&s_cb[c], (unsigned)__popc(mine)); atomicAdd(&s_cn[c], total); }
     }
     __syncthreads();
     if (threadIdx.x < DBSPMSPV_BLK_NCLASS && s_cb[threadIdx.x]) {
@@ -205,43 +218,44 @@ __global__ void k_classify(int32_t n_blocks, const int32_t *blk_start, const uin
     }
 }
 
-// ---- step 4: encode payload + primary (block-CSR) view entries.  One warp per block.
 template <int DT>
 __device__ __forceinline__ void store_value(uint8_t *vals, int pos, const void *uval, int64_t u) {
     if (DT == DBSPMSPV_F32) reinterpret_cast<float *>(vals)[pos] = static_cast<const float *>(uval)[u];
     else if (DT == DBSPMSPV_BF16) reinterpret_cast<uint16_t *>(vals)[pos] = static_cast<const uint16_t *>(uval)[u];
 }
 
+// INLINE blocks: one view entry per stored element (value in w, unused for pattern matrices;
+// packed coordinate in aux).  One thread per stored element; block_of[u] is 1 + its block.
 template <int DT>
-__global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
-                         const void *uval, const uint8_t *type_in, const uint64_t *poff,
-                         const int32_t *eoff, const int32_t *brow, const int32_t *bcol,
-                         uint8_t *payload, uint32_t *v_idx, uint32_t *v_w, uint8_t *v_aux,
-                         int32_t *entry_row) {
+__global__ void k_encode_inline(int64_t nnzu, const int32_t *block_of, const int32_t *blk_start,
+                                const uint64_t *ukey, const void *uval, const uint8_t *type_in,
+                                const int32_t *eoff, const int32_t *brow, const int32_t *bcol,
+                                uint32_t *v_idx, uint32_t *v_w, uint8_t *v_aux, int32_t *entry_row) {
+    const int64_t u = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (u >= nnzu) return;
+    const int32_t b = block_of[u] - 1;
+    if (type_in[b] != DBSPMSPV_BLK_INLINE) return;
+    const int32_t e = eoff[b] + (int32_t)(u - blk_start[b]);
+    v_idx[e] = (uint32_t)bcol[b] | ((uint32_t)DBSPMSPV_BLK_INLINE << TYPE_SHIFT);
+    v_w[e] = DT == DBSPMSPV_F32    ? __float_as_uint(static_cast<const float *>(uval)[u])
+             : DT == DBSPMSPV_BF16 ? (uint32_t) static_cast<const uint16_t *>(uval)[u]
+                                   : 0u;
+    v_aux[e] = (uint8_t)(ukey[u] & 0xFF);
+    entry_row[e] = brow[b];
+}
+
+// One block with a payload, by a whole warp.
+template <int DT>
+__device__ __forceinline__ void encode_block(int32_t b, int s, int nnz, int type, const uint64_t *ukey,
+                                             const void *uval, const uint64_t *poff, const int32_t *eoff,
+                                             const int32_t *brow, const int32_t *bcol, uint8_t *payload,
+                                             uint32_t *v_idx, uint32_t *v_w, uint8_t *v_aux, int32_t *entry_row,
+                                             uint32_t *s_row, uint32_t *s_col, uint8_t *s_start, int lane) {
     constexpr int V = Val<DT>::SIZE;
-    __shared__ uint32_t s_row[TPB / 32][16], s_col[TPB / 32][16];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int64_t b = blockIdx.x * (int64_t)(TPB / 32) + warp;
-    if (b >= n_blocks) return;
-    const int s = blk_start[b], nnz = blk_start[b + 1] - s;
-    const int type = type_in[b];
     const uint64_t off_words = poff[b];
     uint8_t *base = payload + off_words * 4;
     const int e0 = eoff[b];
     const uint32_t tagged = (uint32_t)bcol[b] | ((uint32_t)type << TYPE_SHIFT);
-    if (type == DBSPMSPV_BLK_INLINE) {
-        // one view entry per stored element: value in w (unused for pattern matrices), packed
-        // coordinate in aux
-        for (int k = lane; k < nnz; k += 32) {
-            v_idx[e0 + k] = tagged;
-            v_w[e0 + k] = DT == DBSPMSPV_F32    ? __float_as_uint(static_cast<const float *>(uval)[s + k])
-                          : DT == DBSPMSPV_BF16 ? (uint32_t) static_cast<const uint16_t *>(uval)[s + k]
-                                                : 0u;
-            v_aux[e0 + k] = (uint8_t)(ukey[s + k] & 0xFF);
-            entry_row[e0 + k] = brow[b];
-        }
-        return;
-    }
     if (lane == 0) {
         v_idx[e0] = tagged;
         entry_row[e0] = brow[b];
@@ -257,16 +271,16 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
         return;
     }
     // mask-based classes
-    if (lane < 16) { s_row[warp][lane] = 0; s_col[warp][lane] = 0; }
+    if (lane < 16) { s_row[lane] = 0; s_col[lane] = 0; }
     __syncwarp();
     for (int k = lane; k < nnz; k += 32) {
         uint32_t rc = (uint32_t)(ukey[s + k] & 0xFF);
-        atomicOr(&s_row[warp][rc >> 4], 1u << (rc & 15));
-        atomicOr(&s_col[warp][rc & 15], 1u << (rc >> 4));
+        atomicOr(&s_row[rc >> 4], 1u << (rc & 15));
+        atomicOr(&s_col[rc & 15], 1u << (rc >> 4));
     }
     __syncwarp();
     const bool row_major = is_row_major(type);
-    uint32_t mine = lane < 16 ? (row_major ? s_row[warp][lane] : s_col[warp][lane]) : 0;
+    uint32_t mine = lane < 16 ? (row_major ? s_row[lane] : s_col[lane]) : 0;
     int start = __popc(mine);  // exclusive prefix over lanes 0..15
     for (int o = 1; o < 16; o <<= 1) {
         int t = __shfl_up_sync(0xFFFFFFFFu, start, o);
@@ -295,17 +309,41 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
         for (int k = lane; k < nnz; k += 32) store_value<DT>(vals, k, uval, s + k);
     } else {
         // column-major position of (r, c): start of column c + entries of c above row r
-        __shared__ uint8_t s_start[TPB / 32][16];
-        if (lane < 16) s_start[warp][lane] = (uint8_t)start;
+        if (lane < 16) s_start[lane] = (uint8_t)start;
         __syncwarp();
         for (int k = lane; k < nnz; k += 32) {
             uint32_t rc = (uint32_t)(ukey[s + k] & 0xFF);
             int r = rc >> 4, c = rc & 15;
-            int pos = s_start[warp][c] + __popc(s_col[warp][c] & ((1u << r) - 1));
+            int pos = s_start[c] + __popc(s_col[c] & ((1u << r) - 1));
             store_value<DT>(vals, pos, uval, s + k);
         }
     }
     if (DT == DBSPMSPV_BF16 && (nnz & 1) && lane == 0) reinterpret_cast<uint16_t *>(vals)[nnz] = 0;
+}
+
+// ---- step 4: encode payload + primary (block-CSR) view entries.  A warp takes 32 consecutive
+// blocks and encodes those with a payload one after the other (the INLINE ones are written
+// by k_encode_inline).
+template <int DT>
+__global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint64_t *ukey,
+                         const void *uval, const uint8_t *type_in, const uint64_t *poff,
+                         const int32_t *eoff, const int32_t *brow, const int32_t *bcol,
+                         uint8_t *payload, uint32_t *v_idx, uint32_t *v_w, uint8_t *v_aux,
+                         int32_t *entry_row) {
+    __shared__ uint32_t s_row[TPB / 32][16], s_col[TPB / 32][16];
+    __shared__ uint8_t s_start[TPB / 32][16];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t b = (blockIdx.x * (int64_t)(TPB / 32) + warp) * 32 + lane;
+    const bool have = b < n_blocks;
+    const int s = have ? blk_start[b] : 0, nnz = have ? blk_start[b + 1] - s : 0;
+    const int type = have ? type_in[b] : DBSPMSPV_BLK_INLINE;
+    for (uint32_t todo = __ballot_sync(0xFFFFFFFFu, type != DBSPMSPV_BLK_INLINE); todo; todo &= todo - 1) {
+        const int src = __ffs(todo) - 1;
+        __syncwarp();   // the previous block's use of the shared masks is over
+        encode_block<DT>((int32_t)(b - lane + src), __shfl_sync(0xFFFFFFFFu, s, src), __shfl_sync(0xFFFFFFFFu, nnz, src),
+                         __shfl_sync(0xFFFFFFFFu, type, src), ukey, uval, poff, eoff, brow, bcol, payload,
+                         v_idx, v_w, v_aux, entry_row, s_row[warp], s_col[warp], s_start[warp], lane);
+    }
 }
 
 // first position p in a sorted int array with a[p] >= v, for v = 0..count (pointer arrays)
@@ -397,9 +435,9 @@ __global__ void k_payload_list(int32_t n_entries, int32_t mb, const int32_t *is_
 }
 
 // ---- pull segments (Section 3.3.2): greedy walk along each row block; a segment closes
-// when its accumulated weight reaches the cut.  One warp per row block (hub row blocks hold
-// 10^5 entries: a single thread walking them took tens of milliseconds), two passes.  The warp
-// takes 32 entries per step: a scan of their weights, then the cuts inside the step one after
+// when its accumulated weight reaches the cut.  One warp per stretch of a row block (hub row
+// blocks hold 10^5 entries: a single thread walking them took tens of milliseconds, a single
+// warp milliseconds), two passes.  The warp takes 32 entries per step: a scan of their weights, then the cuts inside the step one after
 // the other (each restarts the running weight at zero).
 struct SegParams { int cut, w_dense, w_mid, w_coo, w_inline; };
 
@@ -437,31 +475,58 @@ __device__ __forceinline__ void seg_walk(int begin, int end, const uint32_t *idx
     if (first < end) close(first, end, acc);
 }
 
-__global__ void k_seg_count(int32_t mb, const int32_t *row_ptr, const uint32_t *idx,
-                            SegParams sp, int32_t *count) {
-    const int64_t rb = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (rb >= mb) return;
-    int c = 0;
-    seg_walk(row_ptr[rb], row_ptr[rb + 1], idx, sp, lane, [&](int, int, int) { ++c; });
-    if (lane == 0) count[rb] = c;
+// A warp walks one stretch of at most SEG_STRETCH entries of a row block, so that the hub row
+// blocks of a power-law matrix are cut by many warps at once; the walk starts afresh at a
+// stretch boundary (no segment spans one).
+constexpr int SEG_STRETCH = 8192;
+
+__global__ void k_seg_units(int32_t mb, const int32_t *row_ptr, int32_t *units) {
+    const int64_t rb = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (rb > mb) return;
+    units[rb] = rb < mb ? (row_ptr[rb + 1] - row_ptr[rb] + SEG_STRETCH - 1) / SEG_STRETCH : 0;
 }
 
-__global__ void k_seg_write(int32_t mb, const int32_t *row_ptr, uint32_t *idx,
-                            SegParams sp, const int32_t *seg_off, Segment *segs, int32_t *seg_rb) {
-    const int64_t rb = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+struct Stretch { int32_t rb, begin, end; };
+__device__ __forceinline__ Stretch stretch_of(int32_t u, int32_t mb, const int32_t *unit_off, const int32_t *row_ptr) {
+    int32_t lo = 0, hi = mb;   // last row block whose first unit is <= u
+    while (hi - lo > 1) {
+        const int32_t mid = lo + ((hi - lo) >> 1);
+        if (unit_off[mid] <= u) lo = mid; else hi = mid;
+    }
+    Stretch s;
+    s.rb = lo;
+    s.begin = row_ptr[lo] + (u - unit_off[lo]) * SEG_STRETCH;
+    s.end = min(row_ptr[lo + 1], s.begin + SEG_STRETCH);
+    return s;
+}
+
+__global__ void k_seg_count(int32_t n_units, int32_t mb, const int32_t *unit_off, const int32_t *row_ptr,
+                            const uint32_t *idx, SegParams sp, int32_t *count) {
+    const int64_t u = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (rb >= mb) return;
-    const int begin = row_ptr[rb], end = row_ptr[rb + 1];
-    int o = seg_off[rb];
-    seg_walk(begin, end, idx, sp, lane, [&](int first, int stop, int weight) {
+    if (u >= n_units) return;
+    const Stretch s = stretch_of((int32_t)u, mb, unit_off, row_ptr);
+    int c = 0;
+    seg_walk(s.begin, s.end, idx, sp, lane, [&](int, int, int) { ++c; });
+    if (lane == 0) count[u] = c;
+}
+
+__global__ void k_seg_write(int32_t n_units, int32_t mb, const int32_t *unit_off, const int32_t *row_ptr,
+                            uint32_t *idx, SegParams sp, const int32_t *seg_off, Segment *segs, int32_t *seg_rb) {
+    const int64_t u = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (u >= n_units) return;
+    const Stretch st = stretch_of((int32_t)u, mb, unit_off, row_ptr);
+    const int begin = row_ptr[st.rb], end = row_ptr[st.rb + 1];
+    int o = seg_off[u];
+    seg_walk(st.begin, st.end, idx, sp, lane, [&](int first, int stop, int weight) {
         if (lane == 0) {
             Segment s;
-            s.row_block = (int32_t)rb;
+            s.row_block = st.rb;
             s.start = first;
             s.count = (stop - first) | ((first == begin && stop == end) ? (int32_t)0x80000000 : 0);
             s.weight = weight;
-            seg_rb[o] = (int32_t)rb;
+            seg_rb[o] = st.rb;
             segs[o] = s;
             idx[first] |= 1u << 28;   // first entry of a segment (bits 27, 28 of idx are spare)
         }
@@ -590,7 +655,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     uint64_t *ukey = nullptr;
     void *uval = nullptr;
     int32_t n_blocks = 0;
-    int32_t *blk_start = nullptr;
+    int32_t *blk_start = nullptr, *block_of = nullptr;   // block_of[u] = 1 + the block of stored element u
     if (nnz > 0) {
         DBS_TRY(sort_pairs(tp, keys, keys_alt, src, src_alt, nnz, 35 + bits_for((uint64_t)d.mb), st));
         tp.release(keys_alt); tp.release(src_alt);
@@ -616,7 +681,8 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         DBS_GET(blk_start, (int64_t)n_blocks + 1);
         k_block_starts<<<grid_for(nnzu), TPB, 0, st>>>(nnzu, flag, rank, blk_start, n_blocks);
         DBS_CUDA(cudaStreamSynchronize(st));
-        tp.release(flag); tp.release(rank);
+        tp.release(flag);
+        block_of = rank;
     }
     h->nnz = nnzu;
 
@@ -632,7 +698,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     DBS_CUDA(cudaMemsetAsync(cls, 0, 2 * DBSPMSPV_BLK_NCLASS * sizeof(unsigned long long), st));
     DBS_CUDA(cudaMemsetAsync(ecount, 0, ((size_t)n_blocks + 1) * 4, st));
     ClassifyParams cp{h->copts.th0, h->copts.th1, h->copts.th2, h->copts.force_format, dt, h->copts.inline_max};
-    if (n_blocks) k_classify<<<grid_for(n_blocks, TPB / 32), TPB, 0, st>>>(n_blocks, blk_start, ukey, cp, type, psize, ecount, brow, bcol, cls, cls + DBSPMSPV_BLK_NCLASS);
+    if (n_blocks) k_classify<<<grid_for(n_blocks, TPB), TPB, 0, st>>>(n_blocks, blk_start, ukey, cp, type, psize, ecount, brow, bcol, cls, cls + DBSPMSPV_BLK_NCLASS);
     // view entries: a small valued block contributes one entry per stored element
     DBS_TRY(exclusive_sum(tp, ecount, eoff, (int64_t)n_blocks + 1, st));
     int32_t n_entries = 0;
@@ -667,14 +733,18 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     DBS_KEEP(h->block_row, n_entries);
     if (n_blocks) {
         uint8_t *pl = static_cast<uint8_t *>(h->payload_alloc);
-        const int g = grid_for(n_blocks, TPB / 32);
-        if (dt == DBSPMSPV_F32) k_encode<DBSPMSPV_F32><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row);
-        else if (dt == DBSPMSPV_BF16) k_encode<DBSPMSPV_BF16><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row);
-        else k_encode<DBSPMSPV_PATTERN><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row);
+        const int g = grid_for(n_blocks, TPB), gi = grid_for(nnzu);
+#define DBS_ENCODE(DT) do { \
+            k_encode_inline<DT><<<gi, TPB, 0, st>>>(nnzu, block_of, blk_start, ukey, uval, type, eoff, brow, bcol, d.csr.idx, d.csr.w, d.csr.aux, h->block_row); \
+            k_encode<DT><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row); } while (0)
+        if (dt == DBSPMSPV_F32) DBS_ENCODE(DBSPMSPV_F32);
+        else if (dt == DBSPMSPV_BF16) DBS_ENCODE(DBSPMSPV_BF16);
+        else DBS_ENCODE(DBSPMSPV_PATTERN);
+#undef DBS_ENCODE
     }
     k_lower_bounds<<<grid_for(d.mb + 1), TPB, 0, st>>>(d.mb, h->block_row, n_entries, d.csr.ptr);
     DBS_CUDA(cudaStreamSynchronize(st));
-    tp.release(ukey); tp.release(uval); tp.release(blk_start); tp.release(poff); tp.release(psize);
+    tp.release(ukey); tp.release(uval); tp.release(blk_start); tp.release(block_of); tp.release(poff); tp.release(psize);
     tp.release(brow); tp.release(bcol); tp.release(ecount); tp.release(eoff); tp.release(type);
 
     // block-CSC view: sort the primary entries by column block, and inside it payload entries
@@ -741,17 +811,23 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     {
         SegParams sp{h->copts.seg_cut, h->heavy_stage ? h->copts.w_dense : h->copts.w_dense_sparse,
                      h->heavy_stage ? h->copts.w_mid : h->copts.w_mid_sparse, h->copts.w_coo, h->copts.w_inline};
+        int32_t *units, *unit_off;
+        DBS_GET(units, (int64_t)d.mb + 1); DBS_GET(unit_off, (int64_t)d.mb + 1);
+        k_seg_units<<<grid_for((int64_t)d.mb + 1), TPB, 0, st>>>(d.mb, d.csr.ptr, units);
+        DBS_TRY(exclusive_sum(tp, units, unit_off, (int64_t)d.mb + 1, st));
+        int32_t n_units = 0;
+        DBS_CUDA(cudaMemcpy(&n_units, unit_off + d.mb, 4, cudaMemcpyDeviceToHost));
         int32_t *cnt, *off;
-        DBS_GET(cnt, (int64_t)d.mb + 1); DBS_GET(off, (int64_t)d.mb + 1);
-        DBS_CUDA(cudaMemsetAsync(cnt, 0, ((size_t)d.mb + 1) * 4, st));
-        k_seg_count<<<grid_for((int64_t)d.mb * 32), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, cnt);
-        DBS_TRY(exclusive_sum(tp, cnt, off, (int64_t)d.mb + 1, st));
+        DBS_GET(cnt, (int64_t)n_units + 1); DBS_GET(off, (int64_t)n_units + 1);
+        DBS_CUDA(cudaMemsetAsync(cnt, 0, ((size_t)n_units + 1) * 4, st));
+        if (n_units) k_seg_count<<<grid_for((int64_t)n_units * 32), TPB, 0, st>>>(n_units, d.mb, unit_off, d.csr.ptr, d.csr.idx, sp, cnt);
+        DBS_TRY(exclusive_sum(tp, cnt, off, (int64_t)n_units + 1, st));
         int32_t nseg = 0;
-        DBS_CUDA(cudaMemcpy(&nseg, off + d.mb, 4, cudaMemcpyDeviceToHost));
+        DBS_CUDA(cudaMemcpy(&nseg, off + n_units, 4, cudaMemcpyDeviceToHost));
         d.n_segments = nseg;
         Segment *segs; DBS_KEEP(segs, nseg);
         int32_t *seg_rb; DBS_KEEP(seg_rb, (int64_t)nseg + 1);
-        k_seg_write<<<grid_for((int64_t)d.mb * 32), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr.idx, sp, off, segs, seg_rb);
+        if (n_units) k_seg_write<<<grid_for((int64_t)n_units * 32), TPB, 0, st>>>(n_units, d.mb, unit_off, d.csr.ptr, d.csr.idx, sp, off, segs, seg_rb);
         d.seg_rb = seg_rb;
         d.segments = segs;
         int32_t *segw, *segpre;
