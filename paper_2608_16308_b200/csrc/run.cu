@@ -747,46 +747,183 @@ __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out
 }
 
 // Pull of the decode entry for matrices whose elements sit mostly in mask-based blocks (pruned
-// layers): one warp per pull segment, the segment's view entries read straight from global
-// memory, mask-based blocks walked by the half-warp streaming form, sums added to the dense y
-// with one atomic per row and half-warp.  No shared memory and few registers: twice the warps per
-// SM of the general traversal kernel, which is what this latency-bound walk needs.  Does nothing
-// unless the selector says pull; the general kernel, launched next, then only runs the push.
+// layers).  A warp takes 32 consecutive entries of the block-CSR view, one block per lane.  A
+// lane walks the active columns of its own column-major or Dense block and keeps the 16 row sums
+// in registers (a Dense column is two 16-byte loads for bf16); with activations 10 % dense a block
+// has one or two active columns, and a step serves 32 blocks with the instructions the half-warp
+// form spends on two.  When the 32 entries share a row block -- always, for the layer shapes of
+// Section 4.3 -- the 32 x 16 sums are folded by 16 shuffles into one atomic per row; otherwise every
+// lane adds its own.  Row-major blocks take the half-warp streaming form, the odd COO/INLINE
+// entry its own lane.  Does nothing unless the selector says pull; the general
+// kernel, launched next, then only runs the push.
+#ifndef DBS_LBC
+#define DBS_LBC 3
+#endif
+constexpr int LBC = DBS_LBC;              // columns of a lane's block per pass of lane_block_columns
+constexpr int LBC_SLOT_BYTES = 48;  // staging slot of a lane: 32 bytes used; the stride keeps 16-byte stores conflict-free
+
+// Active columns of one column-major (or Dense) block, by the lane that owns it: acc[r] += A[r][c] x[c].
+// The loads of up to LBC columns are issued together, level by level (x and header, then the
+// values), so a pass costs two memory latencies whatever the number of columns.  bf16 values
+// come in as two 16-byte loads per column -- with 32 lanes on 32 different cache lines a load
+// instruction costs the same whatever its width, so element-wise loads were 8 times the L1 work.
+// A compressed column (its values packed in row order from a 2-byte aligned start) is then
+// expanded to its rows through the lane's own 48 bytes of shared memory: the 32 aligned bytes
+// that hold it are stored there and each row with a set mask bit reads the next 2 bytes.  No
+// other lane touches the slot, so no barrier is involved.
 template <int DT>
-__global__ void __launch_bounds__(CTA) k_decode_pull(Device d, float *__restrict__ y, float th3, int force_path) {
+__device__ __forceinline__ void lane_block_columns(const uint8_t *blk, bool dense, uint32_t xm, const float *xb,
+                                                   float (&acc)[16], uint4 *slot) {
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    for (uint32_t a = xm; a;) {
+        int c[LBC];
+        bool on[LBC];
+        float xs[LBC];
+        uint32_t mc[LBC];
+        int pos[LBC];
+#pragma unroll
+        for (int j = 0; j < LBC; ++j) { on[j] = a != 0; c[j] = on[j] ? __ffs(a) - 1 : 0; a &= a - 1; }
+#pragma unroll
+        for (int j = 0; j < LBC; ++j) {
+            xs[j] = 0.f; mc[j] = 0u; pos[j] = 0;
+            if (on[j]) {
+                xs[j] = xb[c[j]];
+                if (!dense) { mc[j] = masks[c[j]]; pos[j] = blk[32 + c[j]]; }
+            }
+        }
+        if (DT == DBSPMSPV_BF16) {
+            uint4 lo[LBC], hi[LBC];
+            int off[LBC];          // halfword offset of the column's first value inside lo|hi
+#pragma unroll
+            for (int j = 0; j < LBC; ++j) {
+                lo[j] = make_uint4(0u, 0u, 0u, 0u); hi[j] = lo[j]; off[j] = 0;
+                if (on[j]) {
+                    const int byte0 = dense ? 32 + c[j] * 32 : HDR_BYTES + ((pos[j] * 2) & ~15);
+                    off[j] = dense ? 0 : pos[j] & 7;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(blk + byte0);
+                    lo[j] = src[0]; hi[j] = src[1];       // (the payload has slack behind its last block)
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < LBC; ++j) {
+                if (!on[j]) continue;
+                if (dense) {
+                    // absent elements are stored as zeros: only a non-finite x needs the mask
+                    uint32_t gate = 0xFFFFu;
+                    if ((__float_as_uint(xs[j]) & 0x7F800000u) == 0x7F800000u) gate = masks[c[j]];
+                    const uint32_t u[8] = {lo[j].x, lo[j].y, lo[j].z, lo[j].w, hi[j].x, hi[j].y, hi[j].z, hi[j].w};
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float v0 = __uint_as_float(u[q] << 16), v1 = __uint_as_float(u[q] & 0xFFFF0000u);
+                        if ((gate >> (2 * q)) & 1u) acc[2 * q] += v0 * xs[j];
+                        if ((gate >> (2 * q + 1)) & 1u) acc[2 * q + 1] += v1 * xs[j];
+                    }
+                } else if (off[j] + __popc(mc[j]) <= 16) {
+                    slot[0] = lo[j]; slot[1] = hi[j];
+                    asm volatile("" ::: "memory");
+                    const uint16_t *sv = reinterpret_cast<const uint16_t *>(slot) + off[j];
+                    int i = 0;
+#pragma unroll
+                    for (int r = 0; r < 16; ++r)
+                        if ((mc[j] >> r) & 1u) { acc[r] += __uint_as_float((uint32_t)sv[i] << 16) * xs[j]; ++i; }
+                    asm volatile("" ::: "memory");
+                } else {
+                    // the column straddles the 32 staged bytes: element-wise
+                    const uint8_t *vals = blk + HDR_BYTES;
+                    int i = pos[j];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r)
+                        if ((mc[j] >> r) & 1u) { acc[r] += Val<DT>::load(vals, i) * xs[j]; ++i; }
+                }
+            }
+        } else {
+            const uint8_t *vals = blk + (dense ? 32 : HDR_BYTES);
+#pragma unroll
+            for (int j = 0; j < LBC; ++j) {
+                if (!on[j]) continue;
+                if (dense) {
+                    uint32_t gate = 0xFFFFu;
+                    if ((__float_as_uint(xs[j]) & 0x7F800000u) == 0x7F800000u) gate = masks[c[j]];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r)
+                        if ((gate >> r) & 1u) acc[r] += Val<DT>::load(vals, c[j] * 16 + r) * xs[j];
+                } else {
+                    int i = pos[j];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r)
+                        if ((mc[j] >> r) & 1u) { acc[r] += Val<DT>::load(vals, i) * xs[j]; ++i; }
+                }
+            }
+        }
+    }
+}
+
+// Sum of acc[r] over the 32 lanes, for all 16 rows: afterwards the lane pair (2k, 2k + 1) holds
+// the total of row folded_row(lane).
+__device__ __forceinline__ float fold_rows(const float (&acc)[16], int lane) {
+    float a8[8], a4[4], a2[2];
+    const bool u16 = lane & 16, u8 = lane & 8, u4 = lane & 4, u2 = lane & 2;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a8[i] = (u16 ? acc[i + 8] : acc[i]) + __shfl_xor_sync(FULL, u16 ? acc[i] : acc[i + 8], 16);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) a4[i] = (u8 ? a8[i + 4] : a8[i]) + __shfl_xor_sync(FULL, u8 ? a8[i] : a8[i + 4], 8);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) a2[i] = (u4 ? a4[i + 2] : a4[i]) + __shfl_xor_sync(FULL, u4 ? a4[i] : a4[i + 2], 4);
+    const float a1 = (u2 ? a2[1] : a2[0]) + __shfl_xor_sync(FULL, u2 ? a2[0] : a2[1], 2);
+    return a1 + __shfl_xor_sync(FULL, a1, 1);
+}
+__device__ __forceinline__ int folded_row(int lane) { return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1); }
+
+template <int DT>
+__global__ void __launch_bounds__(CTA) k_decode_pull(Device d, const int32_t *__restrict__ entry_row,
+                                                     float *__restrict__ y, float th3, int force_path) {
+    __shared__ __align__(16) uint8_t s_slots[CTA * LBC_SLOT_BYTES];
     pdl_wait();
     pdl_launch_dependents();
     if (select_path(d, th3, force_path) != DBSPMSPV_PATH_PULL) return;
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = DBSPMSPV_PATH_PULL;
     const int lane = threadIdx.x & 31;
+    uint4 *slot = reinterpret_cast<uint4 *>(s_slots + threadIdx.x * LBC_SLOT_BYTES);
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int n_tasks = (d.n_entries + 31) >> 5;
     auto emit = [&](int erb, int erow, float esum) { atomicAdd(y + (size_t)erb * 16 + erow, esum); };
-    for (int sg = gwarp; sg < d.n_segments; sg += nwarps) {
-        const Segment seg = d.segments[sg];
-        const int rb = seg.row_block, cnt = seg.count & 0x7FFFFFFF;
-        for (int base = 0; base < cnt; base += 32) {
-            const bool have = base + lane < cnt;
-            const int p = seg.start + base + lane;
-            uint32_t idx = 0, w = 0, aux = 0, xm = 0;
-            if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; xm = mask_of(d.ws.x_mask32, idx & IDX_MASK); }
-            const int type = idx >> TYPE_SHIFT;
-            const bool mk = have && xm && type > DBSPMSPV_BLK_COO;
-            const uint32_t all = __ballot_sync(FULL, mk), rows = __ballot_sync(FULL, mk && is_row_major(type));
-            if (all & ~rows) half_stream<DT, false>(d.payload, d.ws.x_dense, idx, w, xm, rb, all & ~rows, lane, emit);
-            if (rows) half_stream<DT, true>(d.payload, d.ws.x_dense, idx, w, xm, rb, rows, lane, emit);
-            if (have && xm && type <= DBSPMSPV_BLK_COO) {       // the odd hypersparse block: its own lane
-                const float *xb = d.ws.x_dense + (size_t)(idx & IDX_MASK) * 16;
-                float *row0 = y + (size_t)rb * 16;
-                if (type == DBSPMSPV_BLK_INLINE) {
-                    if ((xm >> (aux & 15)) & 1u) atomicAdd(row0 + (aux >> 4), Val<DT>::inline_value(w) * xb[aux & 15]);
-                } else {
-                    const int nnz = (int)aux + 1;
-                    const uint8_t *blk = d.payload + (size_t)w * 4, *vals = blk + ((nnz + 3) & ~3);
-                    for (int k = 0; k < nnz; ++k) {
-                        const int c = blk[k] & 15, r = blk[k] >> 4;
-                        if ((xm >> c) & 1u) atomicAdd(row0 + r, Val<DT>::load(vals, k) * xb[c]);
-                    }
+    for (int task = gwarp; task < n_tasks; task += nwarps) {
+        const int p = task * 32 + lane;
+        const bool have = p < d.n_entries;
+        uint32_t idx = 0, w = 0, aux = 0, xm = 0;
+        int rb = -1;
+        if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; rb = entry_row[p]; xm = mask_of(d.ws.x_mask32, idx & IDX_MASK); }
+        const int type = idx >> TYPE_SHIFT;
+        const bool mk = have && xm && type > DBSPMSPV_BLK_COO;
+        const bool rowm = mk && is_row_major(type);
+        const float *xb = d.ws.x_dense + (size_t)(idx & IDX_MASK) * 16;
+        float acc[16];
+#pragma unroll
+        for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+        if (mk && !rowm) lane_block_columns<DT>(d.payload + (size_t)w * 4, type == DBSPMSPV_BLK_DENSE, xm, xb, acc, slot);
+        __syncwarp();
+        const int rb0 = __shfl_sync(FULL, rb, 0);
+        if (__all_sync(FULL, rb == rb0)) {
+            const float total = fold_rows(acc, lane);
+            if (!(lane & 1) && total != 0.f) atomicAdd(y + (size_t)rb0 * 16 + folded_row(lane), total);
+        } else if (mk && !rowm) {
+#pragma unroll
+            for (int r = 0; r < 16; ++r)
+                if (acc[r] != 0.f) atomicAdd(y + (size_t)rb * 16 + r, acc[r]);
+        }
+        const uint32_t rows = __ballot_sync(FULL, rowm);
+        if (rows) half_stream<DT, true>(d.payload, d.ws.x_dense, idx, w, xm, rb, rows, lane, emit);
+        if (have && xm && type <= DBSPMSPV_BLK_COO) {       // the odd hypersparse block: its own lane
+            float *row0 = y + (size_t)rb * 16;
+            if (type == DBSPMSPV_BLK_INLINE) {
+                if ((xm >> (aux & 15)) & 1u) atomicAdd(row0 + (aux >> 4), Val<DT>::inline_value(w) * xb[aux & 15]);
+            } else {
+                const int nnz = (int)aux + 1;
+                const uint8_t *blk = d.payload + (size_t)w * 4, *vals = blk + ((nnz + 3) & ~3);
+                for (int k = 0; k < nnz; ++k) {
+                    const int c = blk[k] & 15, r = blk[k] >> 4;
+                    if ((xm >> c) & 1u) atomicAdd(row0 + r, Val<DT>::load(vals, k) * xb[c]);
                 }
             }
         }
@@ -1110,7 +1247,7 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
                 if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_decode_pull<DT>, CTA, 0) != cudaSuccess || per_sm < 1) return DBSPMSPV_ERR_CUDA;
                 grid = per_sm * h->sm_count;
             }
-            DBS_CUDA(launch_pdl(k_decode_pull<DT>, grid, CTA, 0, st, d, y, h->ropts.th3_decode, h->ropts.force_path));
+            DBS_CUDA(launch_pdl(k_decode_pull<DT>, grid, CTA, 0, st, d, (const int32_t *)h->block_row, y, h->ropts.th3_decode, h->ropts.force_path));
             ++h->kernel_launches;
             s = launch_compute<DT, OutDense, 1>(h, out, h->ropts.th3_decode, true, st, 1);
         } else {

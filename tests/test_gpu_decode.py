@@ -47,6 +47,31 @@ def test_decode_parity_bf16(shape, prune, zf):
     h.close()
 
 
+@pytest.mark.parametrize("dtype", [B.BF16, B.F32])
+def test_decode_non_finite_activations_reach_only_stored_elements(dtype):
+    # Dense blocks keep explicit zeros for absent elements: an infinite or NaN activation must
+    # not leak through them (0 * inf), only through the stored elements of its column
+    m, n = 192, 256
+    w = wl.pruned_weight(m, n, 0.5, seed=5, stream=11)
+    x = wl.relu_activation(n, 0.8, seed=5, stream=61)
+    act = np.flatnonzero(x)
+    x[act[0]] = np.inf
+    x[act[3]] = np.nan
+    h = Handle(w, dtype)
+    assert h.get_stats().class_blocks[B.BLK_DENSE] > 0
+    want, scale = oracle.ref_decode(ref_matrix(w), x)
+    nan, inf = np.isnan(want), np.isinf(want)
+    assert nan.any() and inf.any() and (~nan & ~inf).any()
+    for p in PATHS:
+        h.set_opts(force_path=p)
+        y = decode(h, x)
+        assert (np.isnan(y) == nan).all()
+        assert (y[inf] == want[inf]).all()
+        fin = ~nan & ~inf
+        check(y[fin], want[fin], scale[fin])
+    h.close()
+
+
 def test_decode_fp32_handle_small_integers_exact_and_negative_zero():
     a = (wl.rand_below(3, 0, np.arange(64 * 48, dtype=np.uint64), 7).reshape(64, 48) - 3).astype(np.float32)
     w = wl.csr_from_dense(a)
