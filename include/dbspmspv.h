@@ -114,7 +114,11 @@ typedef struct {
                                 a push level pays one atomic per reached entry)             */
     float th3_decode;        /* dbspmspv_decode: same rule; the output is dense and every row block
                                 takes part, so pull wins much earlier (0.01, the paper's value) */
-    int32_t reserved[9];
+    int32_t no_fused_decode; /* 1: dbspmspv_decode never uses its single-kernel form (which serves
+                                handles whose elements sit mostly in mask-based blocks and whose
+                                x fits in shared memory) but the blocking / traversal / cleanup
+                                kernels of dbspmspv_run                              (0)    */
+    int32_t reserved[8];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64

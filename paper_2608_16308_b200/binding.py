@@ -45,7 +45,8 @@ class RunOpts(ctypes.Structure):
     _fields_ = [("th3", ctypes.c_float), ("force_path", ctypes.c_int32),
                 ("popc_threshold", ctypes.c_int32), ("validate", ctypes.c_int32),
                 ("timing", ctypes.c_int32), ("th3_bfs", ctypes.c_float),
-                ("th3_decode", ctypes.c_float), ("reserved", ctypes.c_int32 * 9)]
+                ("th3_decode", ctypes.c_float), ("no_fused_decode", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 8)]
 
 
 class Stats(ctypes.Structure):

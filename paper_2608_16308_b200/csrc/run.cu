@@ -930,6 +930,264 @@ __global__ void __launch_bounds__(CTA) k_decode_pull(Device d, const int32_t *__
     }
 }
 
+// Active columns of the column-major and Dense blocks of one warp step, when all 32 blocks lie in
+// ONE row block: then any lane may take any (block, column) pair -- its 16 sums go into the
+// same rows -- and the pairs are dealt out evenly, 32 per round, instead of every lane walking
+// the columns of its own block (with activations 10 % dense a block has 1.6 active columns on
+// average but the busiest of 32 has five).  `cols` is the lane's own block's active-column mask
+// (0: not a block of these classes).  Column values are fetched and expanded as in
+// lane_block_columns, Dense columns through the same staged form.
+template <int DT>
+__device__ __forceinline__ void warp_columns(const uint8_t *payload, const float *x_blocks, uint32_t idx, uint32_t w,
+                                             uint32_t cols, int lane, float (&acc)[16], uint4 *slot) {
+    int incl = __popc(cols);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(FULL, incl, o);
+        if (lane >= o) incl += t;
+    }
+    const int excl = incl - __popc(cols);
+    const int total = __shfl_sync(FULL, incl, 31);
+    for (int k0 = 0; k0 < total; k0 += 32) {
+        const int k = k0 + lane;
+        int b = 0;                       // owner of pair k: the last lane whose exclusive prefix is <= k
+#pragma unroll
+        for (int s = 16; s; s >>= 1) {
+            const int t = __shfl_sync(FULL, excl, b + s);
+            if (t <= k) b += s;
+        }
+        uint32_t m = __shfl_sync(FULL, cols, b);
+        const int j = k - __shfl_sync(FULL, excl, b);
+        const uint32_t bidx = __shfl_sync(FULL, idx, b), bw = __shfl_sync(FULL, w, b);
+        if (k >= total) continue;
+        for (int t = 0; t < j; ++t) m &= m - 1;
+        const int c = __ffs(m) - 1;       // the j-th active column of that block
+        const bool dense = (bidx >> TYPE_SHIFT) == DBSPMSPV_BLK_DENSE;
+        const uint8_t *blk = payload + (size_t)bw * 4;
+        const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+        const float xv = x_blocks[(size_t)(bidx & IDX_MASK) * 16 + c];
+        // absent elements of a Dense block are stored as zeros: only a non-finite x needs its mask
+        const bool finite = (__float_as_uint(xv) & 0x7F800000u) != 0x7F800000u;
+        const uint32_t gate = dense && finite ? 0xFFFFu : masks[c];
+        const int pos = dense ? c * 16 : blk[32 + c];
+        const int step_all = dense ? 1 : 0;
+        if (DT == DBSPMSPV_BF16) {
+            const int nvals = dense ? 16 : __popc(gate), off = pos & 7;
+            const uint4 *src = reinterpret_cast<const uint4 *>(blk + (dense ? 32 : HDR_BYTES) + ((pos * 2) & ~15));
+            const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+            const uint4 q0 = src[0], q1 = off + nvals > 8 ? src[1] : zero, q2 = off + nvals > 16 ? src[2] : zero;
+            slot[0] = q0; slot[1] = q1; slot[2] = q2;
+            asm volatile("" ::: "memory");
+            const uint16_t *sv = reinterpret_cast<const uint16_t *>(slot) + off;
+            int i = 0;
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                const uint32_t bit = (gate >> r) & 1u;
+                if (bit) acc[r] += __uint_as_float((uint32_t)sv[i] << 16) * xv;
+                i += (int)bit | step_all;
+            }
+            asm volatile("" ::: "memory");
+        } else {
+            const uint8_t *vals = blk + (dense ? 32 : HDR_BYTES);
+            int i = pos;
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                const uint32_t bit = (gate >> r) & 1u;
+                if (bit) acc[r] += Val<DT>::load(vals, i) * xv;
+                i += (int)bit | step_all;
+            }
+        }
+    }
+}
+
+// The whole decode call in one kernel, for payload-dominated handles whose x fits in shared
+// memory (Section 4.3: one layer, one token).  One thread block per row block.  Every block
+// first reads the dense activation vector itself -- a few KB -- into shared memory as the
+// vector-block masks and the fp32 x blocks the microkernels expect, counts the nonzero vector
+// blocks and evaluates the selector; nothing of that touches the handle's workspace, so there
+// is no blocking kernel before and no cleanup after.
+//   pull: the warps take the row block's view entries 32 at a time, one block per lane (see
+//         k_decode_pull);
+//   push: the lanes take the nonzero vector blocks instead and look their column block up in
+//         the row block's entries (sorted by column block) by bisection, so only blocks under a
+//         nonzero vector block are fetched.
+// The 16 row sums are folded over the warp, added up over the warps in shared memory and
+// stored: a thread block owns its rows, so y needs neither zeroing nor atomics.
+struct FusedLayout {
+    int x_bytes, slot_off, part_off, y_off, cnt_off, active_off, xm_off, total;
+    __host__ __device__ FusedLayout(int nb, int threads) {
+        x_bytes = nb * 64;
+        slot_off = x_bytes;
+        part_off = slot_off + threads * LBC_SLOT_BYTES;
+        y_off = part_off + (threads / 32) * 64;
+        cnt_off = y_off + 64;
+        active_off = cnt_off + 16;
+        xm_off = active_off + nb * 4;
+        total = (xm_off + nb * 2 + 15) & ~15;
+    }
+};
+constexpr int FUSED_MAX_SMEM = 96 * 1024;
+
+template <int DT, int NW>
+__global__ void __launch_bounds__(NW * 32, 768 / (NW * 32))
+k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, float th3, int force_path) {
+    extern __shared__ __align__(16) uint8_t s_dyn[];
+    constexpr int T = NW * 32;
+    const FusedLayout lay(d.nb, T);
+    float *s_x = reinterpret_cast<float *>(s_dyn);
+    float *s_part = reinterpret_cast<float *>(s_dyn + lay.part_off);
+    float *s_y = reinterpret_cast<float *>(s_dyn + lay.y_off);
+    int *s_cnt = reinterpret_cast<int *>(s_dyn + lay.cnt_off);       // [0] nonzero vector blocks
+    int *s_active = reinterpret_cast<int *>(s_dyn + lay.active_off);  // their indices, ascending (push)
+    uint16_t *s_xm = reinterpret_cast<uint16_t *>(s_dyn + lay.xm_off);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint4 *slot = reinterpret_cast<uint4 *>(s_dyn + lay.slot_off + tid * LBC_SLOT_BYTES);
+    if (tid == 0) s_cnt[0] = 0;
+    if (tid < 16) s_y[tid] = 0.f;
+    __syncthreads();
+
+    // ---- x -> masks and fp32 blocks (absent entries carry the marker)
+    {
+        const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
+        int mine = 0;
+        for (int cb = tid; cb < d.nb; cb += T) {
+            const int64_t j0 = (int64_t)cb * 16;
+            float v[16];
+            if (aligned && j0 + 16 <= d.n) {
+                if (DT == DBSPMSPV_BF16) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(x) + j0);
+                    const uint4 a = src[0], b = src[1];
+                    const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) { v[2 * q] = __uint_as_float(u[q] << 16); v[2 * q + 1] = __uint_as_float(u[q] & 0xFFFF0000u); }
+                } else {
+                    const float4 *src = reinterpret_cast<const float4 *>(static_cast<const float *>(x) + j0);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) { const float4 f = src[q]; v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w; }
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    v[k] = 0.f;
+                    if (j0 + k < d.n) v[k] = DT == DBSPMSPV_BF16 ? __uint_as_float((uint32_t) static_cast<const uint16_t *>(x)[j0 + k] << 16)
+                                                                 : static_cast<const float *>(x)[j0 + k];
+                }
+            }
+            uint32_t bits = 0;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const bool nz = v[k] != 0.0f;
+                bits |= (nz ? 1u : 0u) << k;
+                v[k] = nz ? (__float_as_uint(v[k]) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v[k]) : __uint_as_float(X_ABSENT);
+            }
+            float4 *dst = reinterpret_cast<float4 *>(s_x + j0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            s_xm[cb] = (uint16_t)bits;
+            mine += bits != 0;
+        }
+        mine = __reduce_add_sync(FULL, mine);
+        if (lane == 0 && mine) atomicAdd(&s_cnt[0], mine);
+    }
+    __syncthreads();
+    const int n_nzblk = s_cnt[0];
+    int path = force_path;
+    if (path != DBSPMSPV_PATH_PUSH && path != DBSPMSPV_PATH_PULL)
+        path = (float)n_nzblk / (float)d.nb < th3 ? DBSPMSPV_PATH_PUSH : DBSPMSPV_PATH_PULL;
+    if (blockIdx.x == 0 && tid == 0) {
+        Counters *c = d.ws.ctr;
+        c->last_n_nzblk = n_nzblk; c->last_n_tasks = 0; c->last_path = path; c->last_y_nnz = (int32_t)d.m;
+    }
+    if (path == DBSPMSPV_PATH_PUSH) {
+        if (warp == 0) {
+            int count = 0;
+            for (int base = 0; base < d.nb; base += 32) {
+                const bool on = base + lane < d.nb && s_xm[base + lane] != 0;
+                const uint32_t m = __ballot_sync(FULL, on);
+                if (on) s_active[count + __popc(m & below(lane))] = base + lane;
+                count += __popc(m);
+            }
+        }
+        __syncthreads();
+    }
+
+    const int rb = blockIdx.x;
+    const int begin = d.csr.ptr[rb], end = d.csr.ptr[rb + 1];
+    float acc[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+    auto emit = [&](int, int erow, float esum) { atomicAdd(&s_y[erow], esum); };
+    // one step: the lane's entry (idx, w, aux), if `have`
+    auto step = [&](uint32_t idx, uint32_t w, uint32_t aux, bool have) {
+        const uint32_t xm = have ? s_xm[idx & IDX_MASK] : 0u;
+        const int type = idx >> TYPE_SHIFT;
+        const bool mk = have && xm && type > DBSPMSPV_BLK_COO;
+        const bool rowm = mk && is_row_major(type);
+        const float *xb = s_x + (size_t)(idx & IDX_MASK) * 16;
+        warp_columns<DT>(d.payload, s_x, idx, w, mk && !rowm ? xm : 0u, lane, acc, slot);
+        __syncwarp();
+        const uint32_t rows = __ballot_sync(FULL, rowm);
+        if (rows) half_stream<DT, true>(d.payload, s_x, idx, w, xm, rb, rows, lane, emit);
+        if (have && xm && type <= DBSPMSPV_BLK_COO) {       // the odd hypersparse block: its own lane
+            if (type == DBSPMSPV_BLK_INLINE) {
+                if ((xm >> (aux & 15)) & 1u) atomicAdd(&s_y[aux >> 4], Val<DT>::inline_value(w) * xb[aux & 15]);
+            } else {
+                const int nnz = (int)aux + 1;
+                const uint8_t *blk = d.payload + (size_t)w * 4, *vals = blk + ((nnz + 3) & ~3);
+                for (int k = 0; k < nnz; ++k) {
+                    const int c = blk[k] & 15, r = blk[k] >> 4;
+                    if ((xm >> c) & 1u) atomicAdd(&s_y[r], Val<DT>::load(vals, k) * xb[c]);
+                }
+            }
+        }
+    };
+    auto fetch = [&](int p, bool have, uint32_t &idx, uint32_t &w, uint32_t &aux) {
+        idx = 0; w = 0; aux = 0;
+        if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; }
+    };
+    if (path == DBSPMSPV_PATH_PULL) {
+        // the next step's entries are fetched before this step's blocks are worked on
+        uint32_t idx, w, aux, n_idx, n_w, n_aux;
+        int base = begin + warp * 32;
+        fetch(base + lane, base + lane < end, idx, w, aux);
+        for (; base < end; base += T) {
+            const int nb_ = base + T;
+            fetch(nb_ + lane, nb_ + lane < end, n_idx, n_w, n_aux);
+            step(idx, w, aux, base + lane < end);
+            idx = n_idx; w = n_w; aux = n_aux;
+        }
+    } else {
+        for (int i0 = warp * 32; i0 < n_nzblk; i0 += T) {
+            int lo = 0, hi = 0;
+            if (i0 + lane < n_nzblk) {
+                const uint32_t cb = (uint32_t)s_active[i0 + lane];
+                int a = begin, b = end;           // first entry with column block >= cb
+                while (a < b) { const int mid = a + ((b - a) >> 1); if ((d.csr.idx[mid] & IDX_MASK) < cb) a = mid + 1; else b = mid; }
+                lo = a; b = end;                  // first entry with column block > cb
+                while (a < b) { const int mid = a + ((b - a) >> 1); if ((d.csr.idx[mid] & IDX_MASK) <= cb) a = mid + 1; else b = mid; }
+                hi = a;
+            }
+            for (int t = 0; __any_sync(FULL, lo + t < hi); ++t) {
+                uint32_t idx, w, aux;
+                fetch(lo + t, lo + t < hi, idx, w, aux);
+                step(idx, w, aux, lo + t < hi);
+            }
+        }
+    }
+    {
+        const float total = fold_rows(acc, lane);
+        if (!(lane & 1)) s_part[warp * 16 + folded_row(lane)] = total;
+    }
+    __syncthreads();
+    if (tid < 16) {
+        float sum = s_y[tid];
+#pragma unroll
+        for (int k = 0; k < NW; ++k) sum += s_part[k * 16 + tid];
+        const int64_t row = (int64_t)rb * 16 + tid;
+        if (row < d.m) y[row] = sum;
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // Output compaction: the hit masks of the row blocks are scanned in order, so y comes out
 // sorted.  Pass 1 counts per tile, pass 2 places the entries, clears the accumulator and the
@@ -1230,6 +1488,27 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
 template <int DT>
 static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStream_t st) {
     const Device &d = h->d;
+    if (h->heavy_stage && !h->ropts.no_fused_decode) {
+        // one kernel for the whole call, when x fits in shared memory
+        const int per_rb = d.mb ? d.n_entries / d.mb : 0;
+        const int nw = per_rb <= 384 ? 4 : per_rb <= 1024 ? 8 : 16;
+        const FusedLayout lay(d.nb, nw * 32);
+        if (lay.total <= FUSED_MAX_SMEM) {
+            auto kernel = nw == 4 ? k_decode_fused<DT, 4> : nw == 8 ? k_decode_fused<DT, 8> : k_decode_fused<DT, 16>;
+            static bool configured[3] = {false, false, false};
+            bool &done = configured[nw == 4 ? 0 : nw == 8 ? 1 : 2];
+            if (!done) {
+                DBS_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED_MAX_SMEM));
+                done = true;
+            }
+            if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
+            kernel<<<d.mb, nw * 32, lay.total, st>>>(d, x, y, h->ropts.th3_decode, h->ropts.force_path);
+            if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
+            ++h->kernel_launches;
+            DBS_CUDA(cudaGetLastError());
+            return DBSPMSPV_OK;
+        }
+    }
     const int64_t padded = (int64_t)((d.nb + 1) / 2) * 32;
     int64_t work = padded > d.m ? padded : d.m;
     int g = (int)((work + 255) / 256);

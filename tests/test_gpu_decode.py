@@ -40,8 +40,11 @@ def test_decode_parity_bf16(shape, prune, zf):
     want, scale = oracle.ref_decode(ref_matrix(w), x)
     for p in PATHS:
         for thr in (1, 8):
-            h.set_opts(force_path=p, popc_threshold=thr)
-            check(decode(h, x), want, scale)
+            for legacy in (0, 1):     # the single-kernel form (where the handle qualifies) and the general kernels
+                h.set_opts(force_path=p, popc_threshold=thr, no_fused_decode=legacy)
+                check(decode(h, x), want, scale)
+                if p != B.PATH_AUTO:
+                    assert h.get_stats().last_path == p
     assert h.get_stats().last_n_nzblk == int((x.reshape(-1)[: (n // 16) * 16].reshape(-1, 16) != 0).any(axis=1).sum()
                                              + (1 if n % 16 and (x[(n // 16) * 16:] != 0).any() else 0))
     h.close()
@@ -62,8 +65,8 @@ def test_decode_non_finite_activations_reach_only_stored_elements(dtype):
     want, scale = oracle.ref_decode(ref_matrix(w), x)
     nan, inf = np.isnan(want), np.isinf(want)
     assert nan.any() and inf.any() and (~nan & ~inf).any()
-    for p in PATHS:
-        h.set_opts(force_path=p)
+    for p, legacy in [(p, l) for p in PATHS for l in (0, 1)]:
+        h.set_opts(force_path=p, no_fused_decode=legacy)
         y = decode(h, x)
         assert (np.isnan(y) == nan).all()
         assert (y[inf] == want[inf]).all()
@@ -81,8 +84,9 @@ def test_decode_fp32_handle_small_integers_exact_and_negative_zero():
         h = Handle(w, dtype)
         want, _ = oracle.ref_decode(ref_matrix(w), x)
         for p in PATHS:
-            h.set_opts(force_path=p)
-            assert np.array_equal(decode(h, x).astype(np.float64), want)
+            for legacy in (0, 1):
+                h.set_opts(force_path=p, no_fused_decode=legacy)
+                assert np.array_equal(decode(h, x).astype(np.float64), want)
         h.close()
 
 
@@ -115,8 +119,8 @@ def test_decode_rejects_pattern_handles():
 @pytest.mark.parametrize("inline_max", [31, 3])
 def test_decode_on_a_matrix_with_every_block_class(inline_max):
     """Planted dense, row-skewed, column-skewed and banded blocks over a sparse background
-    (with inline_max = 3 also packed-COO blocks): the decode entry's own pull kernel meets every
-    class, row-major and column-major, and the push goes through the general kernel."""
+    (with inline_max = 3 also packed-COO blocks): the decode entry's own kernels meet every
+    class, row-major and column-major, on both paths."""
     from test_gpu_format import mixed_matrix
     a = mixed_matrix(160, 176, 9)
     o = B.default_create_opts()
@@ -126,6 +130,7 @@ def test_decode_on_a_matrix_with_every_block_class(inline_max):
         h = Handle(a, dtype, opts=o)
         want, scale = oracle.ref_decode(ref_matrix(a, bf16=dtype == B.BF16), x if dtype == B.F32 else wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x)))
         for p in PATHS:
-            h.set_opts(force_path=p)
-            check(decode(h, x), want, scale)
+            for legacy in (0, 1):
+                h.set_opts(force_path=p, no_fused_decode=legacy)
+                check(decode(h, x), want, scale)
         h.close()
