@@ -202,6 +202,8 @@ def main() -> None:
     ap.add_argument("--bfs-scale", type=int, default=22)
     ap.add_argument("--bfs-only", action="store_true",
                     help="run only the DB-BFS leg and print its record (the command ncu captures k_bfs from)")
+    ap.add_argument("--decode-only", action="store_true",
+                    help="run only the decode layers and print their records (the command ncu captures k_decode_fused from)")
     ap.add_argument("--crossover", action="store_true",
                     help="print the measured push/pull crossover table (forced paths) and exit")
     args = ap.parse_args()
@@ -226,6 +228,11 @@ def main() -> None:
         if rank == 0:
             flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
             print(json.dumps(bench_bfs(args, B, torch, dev, flush)))
+        return
+    if args.decode_only:
+        if rank == 0:
+            flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+            print(json.dumps(decode_layers(B, torch, dev, cold_call_timer(torch, flush))))
         return
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
@@ -455,14 +462,8 @@ def crossover_table() -> None:
         B.dbspmspv_destroy(h)
 
 
-def other_configs(B, torch, dev, flush, peak):
-    """The remaining workload shapes, one record each (whole call, cold L2, median of 12 after 3
-    warm-ups): the uniform matrix with a 1 % x, the 27-point stencil with clustered x at 0.1 %
-    and 5 %, and single-token decode on three pruned layer shapes next to a dense bf16 GEMV of
-    the same shape on the same box."""
-    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
-    out = []
-
+def cold_call_timer(torch, flush):
+    """us of one call: L2 flushed before every call, median of 12 after 3 warm-ups, CUDA events."""
     def timed(fn):
         ts = []
         for it in range(15):
@@ -474,6 +475,18 @@ def other_configs(B, torch, dev, flush, peak):
             torch.cuda.synchronize()
             ts.append(e0.elapsed_time(e1) * 1e3)
         return float(np.median(ts[3:]))
+    return timed
+
+
+def other_configs(B, torch, dev, flush, peak):
+    """The remaining workload shapes, one record each (whole call, cold L2, median of 12 after 3
+    warm-ups): the uniform matrix with a 1 % x, the 27-point stencil with clustered x at 0.1 %
+    and 5 %, and single-token decode on three pruned layer shapes next to a dense bf16 GEMV of
+    the same shape on the same box."""
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    out = []
+
+    timed = cold_call_timer(torch, flush)
 
     def spmspv_case(name, a, xs):
         h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(a.val), B.F32)
@@ -504,6 +517,15 @@ def other_configs(B, torch, dev, flush, peak):
     spmspv_case("stencil27_160cubed_fp32", a3, [("0.1 % in runs of 64", wl.clustered_x(a3.n, 64)),
                                                  ("5 % in runs of 64", wl.clustered_x(a3.n, 3200))])
     del a3
+    out += decode_layers(B, torch, dev, timed)
+    return out
+
+
+def decode_layers(B, torch, dev, timed):
+    """Single-token decode on the three pruned layer shapes (bf16, 50 % magnitude-pruned) at
+    70 % and 90 % activation zeros, whole call, next to a dense bf16 GEMV of the same shape."""
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    out = []
     for (m, n) in wl.DECODE_SHAPES:
         wgt = wl.pruned_weight(m, n, 0.5)
         bits = wl.f32_to_bf16_bits(wgt.val).view(np.int16)
