@@ -1078,7 +1078,9 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
             for (int k = 0; k < 16; ++k) {
                 const bool nz = v[k] != 0.0f;
                 bits |= (nz ? 1u : 0u) << k;
-                v[k] = nz ? (__float_as_uint(v[k]) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v[k]) : __uint_as_float(X_ABSENT);
+                // (a widened bf16 has zero low bits: it cannot collide with the marker)
+                if (DT != DBSPMSPV_BF16 && __float_as_uint(v[k]) == X_ABSENT) v[k] = __uint_as_float(0x7FC00000u);
+                v[k] = nz ? v[k] : __uint_as_float(X_ABSENT);
             }
             float4 *dst = reinterpret_cast<float4 *>(s_x + j0);
 #pragma unroll
