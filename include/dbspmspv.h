@@ -15,7 +15,9 @@
  *   - `stream` is a cudaStream_t (passed as an opaque pointer; NULL = the legacy default
  *     stream).  dbspmspv_run / db_bfs / dbspmspv_decode only enqueue work on it: they allocate
  *     nothing, never synchronise, and return as soon as the kernels are queued.  Calls on the
- *     same handle must be stream ordered (the handle owns one workspace).
+ *     same handle must be stream ordered (the handle owns one workspace).  A handle lives on
+ *     the device that was current when it was created; run / db_bfs / decode return
+ *     DBSPMSPV_ERR_INVALID_ARG when the calling thread's current device is another one.
  *   - Functions return a dbspmspv_status_t.  Argument errors are reported synchronously.
  *     Conditions detected on the device (output capacity, a bounded wait that ran out) are
  *     recorded in the handle and returned by the next dbspmspv_get_stats; a kernel never traps.

@@ -506,6 +506,7 @@ extern "C" int db_bfs(dbspmspv_handle_t h, int32_t src, int32_t *levels, dbspmsp
     if (!h || !levels) return DBSPMSPV_ERR_INVALID_ARG;
     if (h->d.m != h->d.n) return DBSPMSPV_ERR_UNSUPPORTED;
     if (src < 0 || src >= h->d.n) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     switch (h->d.dtype) {
         case DBSPMSPV_F32: return dbs::bfs_typed<DBSPMSPV_F32>(h, src, levels, st);

@@ -245,4 +245,10 @@ template <> struct Val<DBSPMSPV_PATTERN> {
     __device__ static __forceinline__ float inline_value(uint32_t) { return 1.0f; }
 };
 
+// The entry points enqueue on the calling thread's current device: it has to be the handle's.
+inline bool on_handle_device(const dbspmspv_handle_s *h) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
+
 }  // namespace dbs

@@ -1381,6 +1381,8 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, siz
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+constexpr int MAX_DEVICES = 64;   // per-device caches of launch configurations (device ordinal modulo this)
+
 // Persistent grid of the traversal kernel: as many thread blocks as fit (0 on error).
 template <int DT, typename Out, int MODE> static int compute_grid(int sm_count) {
     const size_t smem = compute_dyn_smem<MODE>();
@@ -1392,7 +1394,8 @@ template <int DT, typename Out, int MODE> static int compute_grid(int sm_count) 
 
 template <int DT, typename Out, int MODE>
 static int launch_compute(dbspmspv_handle_s *h, Out out, float th3, bool pdl, cudaStream_t st, int pull_done = 0) {
-    static int grid = 0;
+    static int grids[MAX_DEVICES] = {};     // function attributes and occupancy are per device
+    int &grid = grids[h->device % MAX_DEVICES];
     if (!grid) grid = compute_grid<DT, Out, MODE>(h->sm_count);
     if (!grid) return DBSPMSPV_ERR_CUDA;
     const size_t smem = compute_dyn_smem<MODE>();
@@ -1497,8 +1500,8 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
         const FusedLayout lay(d.nb, nw * 32);
         if (lay.total <= FUSED_MAX_SMEM) {
             auto kernel = nw == 4 ? k_decode_fused<DT, 4> : nw == 8 ? k_decode_fused<DT, 8> : k_decode_fused<DT, 16>;
-            static bool configured[3] = {false, false, false};
-            bool &done = configured[nw == 4 ? 0 : nw == 8 ? 1 : 2];
+            static bool configured[MAX_DEVICES][3] = {};
+            bool &done = configured[h->device % MAX_DEVICES][nw == 4 ? 0 : nw == 8 ? 1 : 2];
             if (!done) {
                 DBS_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED_MAX_SMEM));
                 done = true;
@@ -1522,7 +1525,8 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
         int s;
         if (h->heavy_stage) {
             // pull by the lean kernel of its own; the general kernel then only runs a push
-            static int grid = 0;
+            static int grids[MAX_DEVICES] = {};
+            int &grid = grids[h->device % MAX_DEVICES];
             if (!grid) {
                 int per_sm = 0;
                 if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_decode_pull<DT>, CTA, 0) != cudaSuccess || per_sm < 1) return DBSPMSPV_ERR_CUDA;
@@ -1580,6 +1584,7 @@ int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, i
         if ((nnz_x > 0 && !x_val) || (y_capacity > 0 && !y_val)) return DBSPMSPV_ERR_INVALID_ARG;
     }
     if ((int64_t)nnz_x > h->d.n) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     switch (h->d.dtype) {
         case DBSPMSPV_F32: return dbs::run_typed<DBSPMSPV_F32>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
@@ -1590,6 +1595,7 @@ int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, i
 
 int dbspmspv_decode(dbspmspv_handle_t h, const void *x, float *y, dbspmspv_stream_t stream) {
     if (!h || !x || !y) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     switch (h->d.dtype) {
         case DBSPMSPV_F32: return dbs::decode_typed<DBSPMSPV_F32>(h, x, y, st);
