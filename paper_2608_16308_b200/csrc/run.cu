@@ -937,7 +937,14 @@ __global__ void __launch_bounds__(CTA) k_decode_pull(Device d, const int32_t *__
 // average but the busiest of 32 has five).  `cols` is the lane's own block's active-column mask
 // (0: not a block of these classes).  Column values are fetched and expanded as in
 // lane_block_columns, Dense columns through the same staged form.
-template <int DT>
+// WC_ILP = (block, column) pairs a lane works on at a time: 2 where a warp has several steps per
+// row block (wide layers: measured 45 -> 41 us on 4096 x 11008), 1 where it has one or two
+// (12288 x 4096: 2 measured 10 % slower).
+__host__ __device__ constexpr int wc_ilp(int warps_per_block) { return warps_per_block >= 8 ? 2 : 1; }
+// staging bytes per lane; the stride keeps 16-byte stores conflict-free
+__host__ __device__ constexpr int wc_slot_bytes(int ilp) { return 48 * ilp + (ilp > 1 ? 16 : 0); }
+
+template <int DT, int WC_ILP>
 __device__ __forceinline__ void warp_columns(const uint8_t *payload, const float *x_blocks, uint32_t idx, uint32_t w,
                                              uint32_t cols, int lane, float (&acc)[16], uint4 *slot) {
     int incl = __popc(cols);
@@ -948,53 +955,84 @@ __device__ __forceinline__ void warp_columns(const uint8_t *payload, const float
     }
     const int excl = incl - __popc(cols);
     const int total = __shfl_sync(FULL, incl, 31);
-    for (int k0 = 0; k0 < total; k0 += 32) {
-        const int k = k0 + lane;
-        int b = 0;                       // owner of pair k: the last lane whose exclusive prefix is <= k
+    for (int k0 = 0; k0 < total; k0 += 32 * WC_ILP) {
+        // WC_ILP pairs per lane and round, worked on side by side: their dependent loads (header ->
+        // values -> staged expansion) overlap
+        bool on[WC_ILP], dense[WC_ILP];
+        uint32_t m[WC_ILP], bidx[WC_ILP], bw[WC_ILP], gate[WC_ILP];
+        int j[WC_ILP], pos[WC_ILP];
+        float xv[WC_ILP];
+        const uint8_t *blk[WC_ILP];
 #pragma unroll
-        for (int s = 16; s; s >>= 1) {
-            const int t = __shfl_sync(FULL, excl, b + s);
-            if (t <= k) b += s;
+        for (int u = 0; u < WC_ILP; ++u) {
+            const int k = k0 + 32 * u + lane;
+            int b = 0;                   // owner of pair k: the last lane whose exclusive prefix is <= k
+#pragma unroll
+            for (int s = 16; s; s >>= 1) {
+                const int t = __shfl_sync(FULL, excl, b + s);
+                if (t <= k) b += s;
+            }
+            m[u] = __shfl_sync(FULL, cols, b);
+            j[u] = k - __shfl_sync(FULL, excl, b);
+            bidx[u] = __shfl_sync(FULL, idx, b);
+            bw[u] = __shfl_sync(FULL, w, b);
+            on[u] = k < total;
         }
-        uint32_t m = __shfl_sync(FULL, cols, b);
-        const int j = k - __shfl_sync(FULL, excl, b);
-        const uint32_t bidx = __shfl_sync(FULL, idx, b), bw = __shfl_sync(FULL, w, b);
-        if (k >= total) continue;
-        for (int t = 0; t < j; ++t) m &= m - 1;
-        const int c = __ffs(m) - 1;       // the j-th active column of that block
-        const bool dense = (bidx >> TYPE_SHIFT) == DBSPMSPV_BLK_DENSE;
-        const uint8_t *blk = payload + (size_t)bw * 4;
-        const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
-        const float xv = x_blocks[(size_t)(bidx & IDX_MASK) * 16 + c];
-        // absent elements of a Dense block are stored as zeros: only a non-finite x needs its mask
-        const bool finite = (__float_as_uint(xv) & 0x7F800000u) != 0x7F800000u;
-        const uint32_t gate = dense && finite ? 0xFFFFu : masks[c];
-        const int pos = dense ? c * 16 : blk[32 + c];
-        const int step_all = dense ? 1 : 0;
+#pragma unroll
+        for (int u = 0; u < WC_ILP; ++u) {
+            gate[u] = 0u; pos[u] = 0; xv[u] = 0.f; dense[u] = false; blk[u] = payload;
+            if (on[u]) {
+                uint32_t mm = m[u];
+                for (int t = 0; t < j[u]; ++t) mm &= mm - 1;
+                const int c = __ffs(mm) - 1;   // the j-th active column of that block
+                dense[u] = (bidx[u] >> TYPE_SHIFT) == DBSPMSPV_BLK_DENSE;
+                blk[u] = payload + (size_t)bw[u] * 4;
+                xv[u] = x_blocks[(size_t)(bidx[u] & IDX_MASK) * 16 + c];
+                // absent elements of a Dense block are stored as zeros: only a non-finite x needs its mask
+                const bool finite = (__float_as_uint(xv[u]) & 0x7F800000u) != 0x7F800000u;
+                gate[u] = dense[u] && finite ? 0xFFFFu : reinterpret_cast<const uint16_t *>(blk[u])[c];
+                pos[u] = dense[u] ? c * 16 : blk[u][32 + c];
+            }
+        }
         if (DT == DBSPMSPV_BF16) {
-            const int nvals = dense ? 16 : __popc(gate), off = pos & 7;
-            const uint4 *src = reinterpret_cast<const uint4 *>(blk + (dense ? 32 : HDR_BYTES) + ((pos * 2) & ~15));
-            const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-            const uint4 q0 = src[0], q1 = off + nvals > 8 ? src[1] : zero, q2 = off + nvals > 16 ? src[2] : zero;
-            slot[0] = q0; slot[1] = q1; slot[2] = q2;
+            int off[WC_ILP];
+#pragma unroll
+            for (int u = 0; u < WC_ILP; ++u) {
+                off[u] = pos[u] & 7;
+                if (on[u]) {
+                    const int nvals = dense[u] ? 16 : __popc(gate[u]);
+                    const uint4 *src = reinterpret_cast<const uint4 *>(blk[u] + (dense[u] ? 32 : HDR_BYTES) + ((pos[u] * 2) & ~15));
+                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                    const uint4 q0 = src[0], q1 = off[u] + nvals > 8 ? src[1] : zero, q2 = off[u] + nvals > 16 ? src[2] : zero;
+                    slot[3 * u] = q0; slot[3 * u + 1] = q1; slot[3 * u + 2] = q2;
+                }
+            }
             asm volatile("" ::: "memory");
-            const uint16_t *sv = reinterpret_cast<const uint16_t *>(slot) + off;
-            int i = 0;
+            int i[WC_ILP];
+#pragma unroll
+            for (int u = 0; u < WC_ILP; ++u) i[u] = 0;
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
-                const uint32_t bit = (gate >> r) & 1u;
-                if (bit) acc[r] += __uint_as_float((uint32_t)sv[i] << 16) * xv;
-                i += (int)bit | step_all;
+#pragma unroll
+                for (int u = 0; u < WC_ILP; ++u) {
+                    const uint16_t *sv = reinterpret_cast<const uint16_t *>(slot + 3 * u) + off[u];
+                    const uint32_t bit = (gate[u] >> r) & 1u;
+                    if (bit) acc[r] += __uint_as_float((uint32_t)sv[i[u]] << 16) * xv[u];
+                    i[u] += (int)bit | (dense[u] ? 1 : 0);
+                }
             }
             asm volatile("" ::: "memory");
         } else {
-            const uint8_t *vals = blk + (dense ? 32 : HDR_BYTES);
-            int i = pos;
 #pragma unroll
-            for (int r = 0; r < 16; ++r) {
-                const uint32_t bit = (gate >> r) & 1u;
-                if (bit) acc[r] += Val<DT>::load(vals, i) * xv;
-                i += (int)bit | step_all;
+            for (int u = 0; u < WC_ILP; ++u) {
+                const uint8_t *vals = blk[u] + (dense[u] ? 32 : HDR_BYTES);
+                int i = pos[u];
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    const uint32_t bit = (gate[u] >> r) & 1u;
+                    if (bit) acc[r] += Val<DT>::load(vals, i) * xv[u];
+                    i += (int)bit | (dense[u] ? 1 : 0);
+                }
             }
         }
     }
@@ -1018,7 +1056,7 @@ struct FusedLayout {
     __host__ __device__ FusedLayout(int nb, int threads) {
         x_bytes = nb * 64;
         slot_off = x_bytes;
-        part_off = slot_off + threads * LBC_SLOT_BYTES;
+        part_off = slot_off + threads * wc_slot_bytes(wc_ilp(threads / 32));
         y_off = part_off + (threads / 32) * 64;
         cnt_off = y_off + 64;
         active_off = cnt_off + 16;
@@ -1041,7 +1079,7 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
     int *s_active = reinterpret_cast<int *>(s_dyn + lay.active_off);  // their indices, ascending (push)
     uint16_t *s_xm = reinterpret_cast<uint16_t *>(s_dyn + lay.xm_off);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint4 *slot = reinterpret_cast<uint4 *>(s_dyn + lay.slot_off + tid * LBC_SLOT_BYTES);
+    uint4 *slot = reinterpret_cast<uint4 *>(s_dyn + lay.slot_off + tid * wc_slot_bytes(wc_ilp(NW)));
     if (tid == 0) s_cnt[0] = 0;
     if (tid < 16) s_y[tid] = 0.f;
     __syncthreads();
@@ -1126,7 +1164,7 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
         const bool mk = have && xm && type > DBSPMSPV_BLK_COO;
         const bool rowm = mk && is_row_major(type);
         const float *xb = s_x + (size_t)(idx & IDX_MASK) * 16;
-        warp_columns<DT>(d.payload, s_x, idx, w, mk && !rowm ? xm : 0u, lane, acc, slot);
+        warp_columns<DT, wc_ilp(NW)>(d.payload, s_x, idx, w, mk && !rowm ? xm : 0u, lane, acc, slot);
         __syncwarp();
         const uint32_t rows = __ballot_sync(FULL, rowm);
         if (rows) half_stream<DT, true>(d.payload, s_x, idx, w, xm, rb, rows, lane, emit);
