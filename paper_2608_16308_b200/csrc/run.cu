@@ -1064,7 +1064,7 @@ struct FusedLayout {
         total = (xm_off + nb * 2 + 15) & ~15;
     }
 };
-constexpr int FUSED_MAX_SMEM = 96 * 1024;
+constexpr int FUSED_MAX_SMEM = 200 * 1024;   // of the 227 KB a thread block may have
 
 template <int DT, int NW>
 __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32))

@@ -75,6 +75,21 @@ def test_decode_non_finite_activations_reach_only_stored_elements(dtype):
     h.close()
 
 
+def test_decode_wide_layer_many_entries_per_row_block():
+    # more than 1024 view entries per row block: the single-kernel form runs 16 warps per row
+    # block and keeps 80 KB of x in shared memory
+    m, n = 48, 20000
+    w = wl.pruned_weight(m, n, 0.5, seed=5, stream=21)
+    x = wl.relu_activation(n, 0.9, seed=5, stream=62)
+    h = Handle(w, B.BF16)
+    want, scale = oracle.ref_decode(ref_matrix(w), x)
+    for p in PATHS:
+        for legacy in (0, 1):
+            h.set_opts(force_path=p, no_fused_decode=legacy)
+            check(decode(h, x), want, scale)
+    h.close()
+
+
 def test_decode_fp32_handle_small_integers_exact_and_negative_zero():
     a = (wl.rand_below(3, 0, np.arange(64 * 48, dtype=np.uint64), 7).reshape(64, 48) - 3).astype(np.float32)
     w = wl.csr_from_dense(a)

@@ -93,9 +93,12 @@ def test_c5_decode_layers(shape):
             x = wl.relu_activation(n, zf)
             xd = torch.from_numpy(wl.f32_to_bf16_bits(x).view(np.int16)).to(DEV)
             y = torch.empty(m, dtype=torch.float32, device=DEV)
-            B.dbspmspv_decode(h.h, xd, y)
-            torch.cuda.synchronize()
             want, scale = oracle.ref_decode(A, x)
-            err = np.abs(y.cpu().numpy().astype(np.float64) - want)
-            assert (err <= TOL * scale).all(), f"prune {prune} zeros {zf}: worst {np.max(err / np.maximum(scale, 1e-300)):.2e}"
+            for legacy in (0, 1):          # the single-kernel form, and the general kernels
+                h.set_opts(no_fused_decode=legacy)
+                y.fill_(7.0)
+                B.dbspmspv_decode(h.h, xd, y)
+                torch.cuda.synchronize()
+                err = np.abs(y.cpu().numpy().astype(np.float64) - want)
+                assert (err <= TOL * scale).all(), f"prune {prune} zeros {zf} legacy {legacy}: worst {np.max(err / np.maximum(scale, 1e-300)):.2e}"
         h.close()
