@@ -103,7 +103,7 @@ typedef struct {
 typedef struct {
     float th3;               /* dbspmspv_run: push iff the nonempty-vector-block ratio is
                                 below th3.  0.01 in the paper; default 0.9, the crossover
-                                measured on B200 (profiles/selector_crossover.md)            */
+                                measured on B200 (the table `bench.py --crossover` prints)    */
     int32_t force_path;      /* DBSPMSPV_PATH_*                                              */
     int32_t popc_threshold;  /* CSR-class blocks: popc(mask) >= this -> row-driven (pull-style)
                                 microkernel, below -> column-driven (push-style)             */
