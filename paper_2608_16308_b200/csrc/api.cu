@@ -195,9 +195,7 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     cudaFree(const_cast<int32_t *>(d.rowrun_ptr)); cudaFree(const_cast<uint32_t *>(d.rowrun_idx));
     cudaFree(const_cast<int32_t *>(d.payload_ptr)); cudaFree(const_cast<int32_t *>(d.payload_pos));
     cudaFree(h->csc2csr); cudaFree(h->block_row);
-    dbs::Workspace &ws = d.ws;
-    cudaFree(ws.x_dense); cudaFree(ws.x_mask32); cudaFree(ws.tasks); cudaFree(ws.hubs); cudaFree(ws.bfs_words); cudaFree(ws.z_mask32); cudaFree(ws.y_acc);
-    cudaFree(ws.y_mask32); cudaFree(ws.y_hit8); cudaFree(ws.tile_count); cudaFree(ws.visited32); cudaFree(ws.ctr);
+    cudaFree(h->ws_arena);
     if (h->ev[0]) cudaEventDestroy(h->ev[0]);
     if (h->ev[1]) cudaEventDestroy(h->ev[1]);
     delete h;

@@ -193,6 +193,7 @@ struct dbspmspv_handle_s {
     bool timed;
     int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)
     int64_t bfs_index_bytes;
+    void *ws_arena;             // the one allocation that holds the whole workspace
 };
 
 namespace dbs {

@@ -1460,20 +1460,36 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     ws.task_capacity = (int64_t)d.n_entries / d.payload_chunk + 17 * (int64_t)d.nb + 32;
     ws.n_tiles = (int32_t)ceil_div<int64_t>((d.mb + 1) / 2, TILE_WORDS);
     if (ws.n_tiles < 1) ws.n_tiles = 1;
-#define DBS_WS(expr) do { int s__ = (expr); if (s__ != DBSPMSPV_OK) return s__; } while (0)
-    DBS_WS(dev_alloc_zero(&ws.x_dense, xwords * 32, &total));
-    DBS_WS(dev_alloc_zero(&ws.x_mask32, xwords, &total));
-    DBS_WS(dev_alloc_zero(&ws.tasks, (size_t)ws.task_capacity, &total));
-    DBS_WS(dev_alloc_zero(&ws.hubs, (size_t)3 * HUB_CAP, &total));
-    DBS_WS(dev_alloc_zero(&ws.bfs_words, xwords, &total));
-    DBS_WS(dev_alloc_zero(&ws.z_mask32, xwords > ywords ? xwords : ywords, &total));
-    DBS_WS(dev_alloc_zero(&ws.y_acc, ywords * 32, &total));
-    DBS_WS(dev_alloc_zero(&ws.y_mask32, ywords, &total));
-    DBS_WS(dev_alloc_zero(&ws.y_hit8, ywords * 32, &total));
-    DBS_WS(dev_alloc_zero(&ws.tile_count, (size_t)ws.n_tiles, &total));
-    DBS_WS(dev_alloc_zero(&ws.visited32, d.m == d.n ? ywords : 1, &total));
-    DBS_WS(dev_alloc_zero(&ws.ctr, 1, &total));
-#undef DBS_WS
+    // One allocation for the whole workspace, carved at 512-byte boundaries (a dozen cudaMalloc
+    // calls fewer per handle).  Where the driver places its pages still matters: the same push
+    // kernel measured 68 .. 83 us on the same data from one allocation history to the next.
+    size_t off = 0;
+    auto carve = [&](size_t bytes) { const size_t o = off; off += (bytes + 511) & ~(size_t)511; return o; };
+    const size_t zwords = xwords > ywords ? xwords : ywords;
+    const size_t o_xd = carve(xwords * 32 * sizeof(float)), o_yacc = carve(ywords * 32 * sizeof(float)),
+                 o_hit = carve(ywords * 32), o_tasks = carve((size_t)ws.task_capacity * sizeof(*ws.tasks)),
+                 o_xm = carve(xwords * 4), o_ym = carve(ywords * 4), o_zm = carve(zwords * 4),
+                 o_words = carve(xwords * sizeof(*ws.bfs_words)), o_vis = carve((d.m == d.n ? ywords : 1) * 4),
+                 o_hubs = carve((size_t)3 * HUB_CAP * sizeof(*ws.hubs)), o_tile = carve((size_t)ws.n_tiles * sizeof(*ws.tile_count)),
+                 o_ctr = carve(sizeof(*ws.ctr));
+    void *arena = nullptr;
+    if (cudaMalloc(&arena, off) != cudaSuccess) return DBSPMSPV_ERR_ALLOC;
+    h->ws_arena = arena;
+    if (cudaMemset(arena, 0, off) != cudaSuccess) return DBSPMSPV_ERR_CUDA;
+    uint8_t *base = static_cast<uint8_t *>(arena);
+    ws.x_dense = reinterpret_cast<decltype(ws.x_dense)>(base + o_xd);
+    ws.y_acc = reinterpret_cast<decltype(ws.y_acc)>(base + o_yacc);
+    ws.y_hit8 = reinterpret_cast<decltype(ws.y_hit8)>(base + o_hit);
+    ws.tasks = reinterpret_cast<decltype(ws.tasks)>(base + o_tasks);
+    ws.x_mask32 = reinterpret_cast<decltype(ws.x_mask32)>(base + o_xm);
+    ws.y_mask32 = reinterpret_cast<decltype(ws.y_mask32)>(base + o_ym);
+    ws.z_mask32 = reinterpret_cast<decltype(ws.z_mask32)>(base + o_zm);
+    ws.bfs_words = reinterpret_cast<decltype(ws.bfs_words)>(base + o_words);
+    ws.visited32 = reinterpret_cast<decltype(ws.visited32)>(base + o_vis);
+    ws.hubs = reinterpret_cast<decltype(ws.hubs)>(base + o_hubs);
+    ws.tile_count = reinterpret_cast<decltype(ws.tile_count)>(base + o_tile);
+    ws.ctr = reinterpret_cast<decltype(ws.ctr)>(base + o_ctr);
+    total = (int64_t)off;
     h->stats.workspace_bytes = total;
     if (cudaMemset(ws.x_dense, 0xFF, xwords * 32 * sizeof(float)) != cudaSuccess) return DBSPMSPV_ERR_CUDA;
     {   // 0xFFFFFFFF -> the marker pattern 0x7FFFFFFF needs a kernel; a tiny fill does it
