@@ -1464,7 +1464,14 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     // calls fewer per handle).  Where the driver places its pages still matters: the same push
     // kernel measured 68 .. 83 us on the same data from one allocation history to the next.
     size_t off = 0;
-    auto carve = [&](size_t bytes) { const size_t o = off; off += (bytes + 511) & ~(size_t)511; return o; };
+    // (arrays of a megabyte or more start on a 2 MB boundary, the others on a 512-byte one)
+    auto carve = [&](size_t bytes) {
+        const size_t a = bytes >= ((size_t)1 << 20) ? ((size_t)2 << 20) : 512;
+        off = (off + a - 1) / a * a;
+        const size_t o = off;
+        off += (bytes + 511) & ~(size_t)511;
+        return o;
+    };
     const size_t zwords = xwords > ywords ? xwords : ywords;
     const size_t o_xd = carve(xwords * 32 * sizeof(float)), o_yacc = carve(ywords * 32 * sizeof(float)),
                  o_hit = carve(ywords * 32), o_tasks = carve((size_t)ws.task_capacity * sizeof(*ws.tasks)),
