@@ -260,23 +260,14 @@ __device__ __forceinline__ void mark_rows(uint8_t *hit8, int rb, uint32_t rows16
     }
 }
 
-// Global accumulate of one product (or partial sum) with its structural-hit flag.  The flag is
-// stored only when the atomic returns zero: the first product that reaches a row always sees the
-// cleared accumulator, so the flag is set once per row instead of once per product (a later zero --
-// an explicitly stored zero, a cancellation -- only repeats the store).  The repeated byte stores
-// to the hub rows of a power-law matrix, not the atomics, were what the push waited for: 77 -> 57 us
-// at 10 % x density, 326 -> 170 us at 50 %.
-template <typename Out>
-__device__ __forceinline__ void add_and_flag(Out out, size_t row, float v) {
-    const float old = atomicAdd(out.acc + row, v);
-    if (Out::MASKS && old == 0.0f) out.hit8[row] = 1;
-}
-
 // Writeback of one block handled outside the shared-memory accumulator: lanes 0..15 own the 16
 // rows; one global atomic and one flag store per touched row.
 template <typename Out>
 __device__ __forceinline__ void flush_rows(Out out, int rb, uint32_t hits, float v, int lane) {
-    if (lane < 16 && ((hits >> lane) & 1u)) add_and_flag(out, (size_t)rb * 16 + lane, v);
+    if (lane < 16 && ((hits >> lane) & 1u)) {
+        atomicAdd(out.acc + (size_t)rb * 16 + lane, v);
+        if (Out::MASKS) out.hit8[(size_t)rb * 16 + lane] = 1;
+    }
 }
 
 // Push (Section 3.3.2): every warp takes one task = up to PUSH_CHUNK consecutive block-CSC
@@ -338,10 +329,18 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
             if (have) {
                 if (type == DBSPMSPV_BLK_INLINE) {
                     float *row0 = out.acc + (size_t)brow * 16;
+                    // The structural-hit flag is stored only when the atomic returns zero: the first
+                    // product that reaches a row always sees the cleared accumulator, so the flag is
+                    // set once per row instead of once per product (a later zero -- an explicitly
+                    // stored zero, a cancellation -- only repeats the store).  The repeated byte
+                    // stores to the hub rows of a power-law matrix, not the atomics, were what the
+                    // push waited for: 77 -> 57 us at 10 % x density, 326 -> 170 us at 50 %.  (The
+                    // per-block writebacks of mask-based blocks keep the plain atomic and the
+                    // unconditional store: on the stencil the returning atomic cost 7-15 %.)
                     bool first = DT == DBSPMSPV_PATTERN;     // (no accumulate on pattern matrices: always flag)
                     const uint32_t hit = lane_block<DT>(type, w[u], aux[u], xm, s_x[aux[u] & 15], s_x, d.payload,
                                                         [&](int r, float v) { first |= atomicAdd(row0 + r, v) == 0.0f; });
-                    if (Out::MASKS && hit && first) mark_rows(out.hit8, brow, hit);   // see add_and_flag
+                    if (Out::MASKS && hit && first) mark_rows(out.hit8, brow, hit);
                 } else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
                     coo_cnt = (int)aux[u] + 1;
                 } else {
@@ -368,7 +367,10 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                 const bool mk = heavy && type != DBSPMSPV_BLK_COO;
                 const uint32_t cs = __ballot_sync(FULL, mk);
                 if (__popc(cs) >= HEAVY_LANE_MIN) {
-                    auto emit = [&](int erb, int erow, float esum) { add_and_flag(out, (size_t)erb * 16 + erow, esum); };
+                    auto emit = [&](int erb, int erow, float esum) {
+                        atomicAdd(out.acc + (size_t)erb * 16 + erow, esum);
+                        if (Out::MASKS) out.hit8[(size_t)erb * 16 + erow] = 1;
+                    };
                     const uint32_t rows = __ballot_sync(FULL, mk && is_row_major(type));
                     const uint32_t tagged = (idx[u] & ~IDX_MASK) | (uint32_t)jb;     // class bits + the task's column block
                     if (cs & ~rows) half_stream<DT, false>(d.payload, d.ws.x_dense, tagged, w[u], xm, brow, cs & ~rows, lane, emit);
@@ -1626,7 +1628,7 @@ extern "C" {
 void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
-    o->th3 = 0.9f;
+    o->th3 = 0.98f;
     o->th3_bfs = 0.05f;
     o->th3_decode = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;
