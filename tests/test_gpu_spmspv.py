@@ -285,3 +285,31 @@ def test_dense_but_clustered_x_takes_the_push_with_a_late_worklist():
     h.set_opts()
     check_against_oracle(h.run(dense_x(csr.n, 3, 0.01)), oracle.ref_pull(A, dense_x(csr.n, 3, 0.01).idx, dense_x(csr.n, 3, 0.01).val))
     h.close()
+
+
+def test_rows_that_sum_to_zero_or_hold_stored_zeros_are_still_reported():
+    """The push flags a row when its accumulator was zero before the product arrived.  Rows whose
+    products are zeros (stored zero values), cancel exactly, or arrive by the thousand (a hub
+    row) must all come out as structural hits, on every path."""
+    m, n = 600, 4000
+    rng = np.random.default_rng(7)
+    dense = np.zeros((m, n), dtype=np.float32)
+    bg = wl.random_sparse(m, n, 3000, 9)
+    dense[bg.rows(), bg.col_idx] = bg.val
+    dense[5, :] = 1.0                                  # hub row: every listed column reaches it
+    dense[17, :] = 0.0                                 # row 17: stored zeros only
+    dense[33, :] = 0.0                                 # row 33: +v and -v under two listed columns
+    dense[33, 100], dense[33, 101] = 2.5, -2.5
+    mask = dense != 0
+    cols = rng.choice(n, 40, replace=False)
+    mask[17, cols] = True
+    a = wl.csr_from_dense(dense, keep_zeros_mask=mask)
+    x_idx = np.unique(np.concatenate([cols[:20], [100, 101], rng.choice(n, 300, replace=False)])).astype(np.int32)
+    x = wl.SparseVec(n, x_idx, np.ones(x_idx.size, dtype=np.float32))
+    h = Handle(a, B.F32)
+    want = oracle.ref_pull(ref_matrix(a), x.idx, x.val)
+    assert 17 in want[0] and 33 in want[0] and 5 in want[0]
+    for p in (B.PATH_AUTO, B.PATH_PUSH, B.PATH_PULL):
+        h.set_opts(force_path=p)
+        check_against_oracle(h.run(x), want)
+    h.close()
