@@ -337,9 +337,12 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                     // push waited for: 77 -> 57 us at 10 % x density, 326 -> 170 us at 50 %.  (The
                     // per-block writebacks of mask-based blocks keep the plain atomic and the
                     // unconditional store: on the stencil the returning atomic cost 7-15 %.)
-                    bool first = DT == DBSPMSPV_PATTERN;     // (no accumulate on pattern matrices: always flag)
+                    bool first = false;
                     const uint32_t hit = lane_block<DT>(type, w[u], aux[u], xm, s_x[aux[u] & 15], s_x, d.payload,
                                                         [&](int r, float v) { first |= atomicAdd(row0 + r, v) == 0.0f; });
+                    // (pattern matrices have no product: they count the hits in the accumulator,
+                    // which the compaction clears like any other, to get the same first-touch test)
+                    if (DT == DBSPMSPV_PATTERN && hit) first = atomicAdd(row0 + (aux[u] >> 4), 1.0f) == 0.0f;
                     if (Out::MASKS && hit && first) mark_rows(out.hit8, brow, hit);
                 } else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
                     coo_cnt = (int)aux[u] + 1;
