@@ -410,7 +410,7 @@ def main() -> None:
 
 # DRAM traffic of that launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
 # summarised in profiles/k_compute_pull_rmat20_x50pct.txt
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 157849344
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 156602880
 
 
 def crossover_table() -> None:
