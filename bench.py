@@ -605,7 +605,10 @@ def bench_bfs(args, B, torch, dev, flush):
     srcs = wl.bfs_sources(g, 16)
     deg = np.diff(g.row_ptr)
     levels = torch.empty(g.n, dtype=torch.int32, device=dev)
-    times, teps, nlev = [], [], []
+    import oracle
+    A = oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx)
+    A.csc()
+    times, teps, nlev, matches, cpu_s, cpu_edges = [], [], [], [], 0.0, 0.0
     for s in srcs:
         best = None
         for rep in range(3):
@@ -622,21 +625,19 @@ def bench_bfs(args, B, torch, dev, flush):
         times.append(best)
         teps.append(edges / (best * 1e-3) / 1e9)
         nlev.append(int(B.dbspmspv_get_stats(h).bfs_levels))
-    import oracle
-    A = oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx)
-    A.csc()
-    t0 = time.perf_counter()
-    ref = oracle.ref_bfs(A, int(srcs[-1]))
-    cpu_s = time.perf_counter() - t0
-    match = bool(np.array_equal(ref, lv))
+        t0 = time.perf_counter()
+        ref = oracle.ref_bfs(A, int(s))               # every timed source is compared with the oracle
+        cpu_s += time.perf_counter() - t0
+        cpu_edges += float(deg[ref >= 0].sum()) / 2.0
+        matches.append(bool(np.array_equal(ref, lv)))
     B.dbspmspv_destroy(h)
     hm = len(teps) / sum(1.0 / t for t in teps)
     return {"workload": f"rmat{args.bfs_scale}_sym_ef16_pattern_16sources", "gteps_harmonic_mean": round(hm, 3),
             "gteps_min": round(min(teps), 3), "gteps_max": round(max(teps), 3),
             "ms_median": round(float(np.median(times)), 4), "levels": nlev, "vertices": int(g.n), "nnz": int(g.nnz),
-            "last_source_matches_oracle": match,
-            "cpu_baseline": {"value": round(float(deg[ref >= 0].sum()) / 2.0 / cpu_s / 1e9, 4), "unit": "GTEPS",
-                             "cores": 1, "kind": "oracle", "sample": "queue BFS from the last source"}}
+            "sources_matching_oracle": int(sum(matches)), "sources": len(matches),
+            "cpu_baseline": {"value": round(cpu_edges / cpu_s / 1e9, 4), "unit": "GTEPS",
+                             "cores": 1, "kind": "oracle", "sample": "queue BFS from each of the sources"}}
 
 
 if __name__ == "__main__":

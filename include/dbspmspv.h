@@ -47,7 +47,7 @@ typedef enum {
     DBSPMSPV_ERR_CUDA = 4,        /* a CUDA runtime call failed                           */
     DBSPMSPV_ERR_CAPACITY = 5,    /* y_capacity too small; nothing was written out of bounds */
     DBSPMSPV_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out                   */
-    DBSPMSPV_ERR_BOUNDS = 7,      /* validate=1: an x index was out of range              */
+    DBSPMSPV_ERR_BOUNDS = 7,      /* an x index was out of range (the entry was skipped)  */
     DBSPMSPV_ERR_TOO_LARGE = 8    /* dbspmspv_compact_noalloc: more rows than its fixed scratch covers */
 } dbspmspv_status_t;
 
@@ -107,7 +107,9 @@ typedef struct {
     int32_t force_path;      /* DBSPMSPV_PATH_*                                              */
     int32_t popc_threshold;  /* CSR-class blocks: popc(mask) >= this -> row-driven (pull-style)
                                 microkernel, below -> column-driven (push-style)             */
-    int32_t validate;        /* 1: range-check x indices on the device (ERR_BOUNDS)          */
+    int32_t validate;        /* x indices outside [0, n) are always skipped and reported as
+                                ERR_BOUNDS; 1: an index listed twice is reported as well
+                                (deferred ERR_INVALID_ARG; it contributes once either way)   */
     int32_t timing;          /* 1: bracket the traversal kernel of run/decode with two CUDA
                                 events (made at create); read back as last_compute_ms      */
     float th3_bfs;           /* db_bfs: same rule per level.  Default 0.05, measured on the
@@ -228,8 +230,9 @@ int db_bfs(dbspmspv_handle_t h, int32_t src, int32_t *levels, dbspmspv_stream_t 
  */
 int dbspmspv_decode(dbspmspv_handle_t h, const void *x, float *y, dbspmspv_stream_t stream);
 
-/* Synchronises `stream`-ordered work of the handle (cudaDeviceSynchronize) and copies the
- * statistics to the HOST struct `out`.  Returns the deferred device status of the last call. */
+/* Waits for the stream the handle's last run / decode / db_bfs call was enqueued on (not for the
+ * whole device) and copies the statistics to the HOST struct `out`.  Returns the deferred
+ * device status of the last call, which is then cleared.                                      */
 int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out);
 
 /* Test hook: decode the blocked format back to coordinates.  row/col/val: device arrays with
@@ -260,10 +263,11 @@ int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *cs
  *
  *   acc         m fp32 values (device); only rows whose bit is set are read
  *   hit_bitmap  ceil(m/32) uint32 words (device): bit (i & 31) of word (i >> 5) set iff row i
- *               belongs to the result; bits at or beyond m must be clear
+ *               belongs to the result; bits at or beyond m in the last word are ignored
  *   y_idx/y_val out: the set rows in ascending order and their values, room for y_capacity
  *               entries (y_val may be NULL); y_nnz out: one int32 on the device, the full count
- *   Inputs are not modified.  Handles are not involved.
+ *   Inputs are not modified.  Handles are not involved.  m must be at least 1 (m = 0 and
+ *   negative sizes return DBSPMSPV_ERR_INVALID_ARG).
  *
  * Scratch: one counter per 8192 rows, kept in a fixed 16 KB __device__ array inside the
  * library (every GPU that loads the library holds it until the process exits).  Hence
@@ -273,13 +277,21 @@ int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *cs
  *   - two calls whose kernels overlap on the GPU (different streams, or threads) race on it:
  *     serialise calls to this entry point on one device;
  *   - the first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress); make that first call before any stream capture begins.
+ *     (cudaGetSymbolAddress) and keeps it for the life of the process; make that first call
+ *     before any stream capture begins, and do not reset the device while the library is in use.
  * It calls no cudaMalloc / cudaFree or other allocating routine, enqueues two kernels on
  * `stream` and returns without synchronising.
  */
 int dbspmspv_compact_noalloc(const float *acc, const uint32_t *hit_bitmap, int64_t m,
                              int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
                              dbspmspv_stream_t stream);
+
+/* Test hook for the bounded device-side waits (Section 3.3.3's asynchronous staging completes
+ * on barriers in shared memory, and every wait on them has an iteration limit): launches one
+ * warp that waits on such a barrier with NO copy in flight, so the wait runs out after
+ * `max_tries` tries (1 .. 4096, about 2 us each) and the kernel records DBSPMSPV_ERR_TIMEOUT,
+ * which the next dbspmspv_get_stats returns.  The context stays usable.                       */
+int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_stream_t stream);
 
 int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts);
 int dbspmspv_destroy(dbspmspv_handle_t h);

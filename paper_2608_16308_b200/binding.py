@@ -28,6 +28,7 @@ EXPORTED_SYMBOLS = (
     "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "dbspmspv_decode", "dbspmspv_get_stats",
     "dbspmspv_export_coo", "dbspmspv_export_blocks", "dbspmspv_export_views",
     "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror", "dbspmspv_compact_noalloc",
+    "dbspmspv_test_bounded_wait",
 )
 
 
@@ -95,6 +96,7 @@ def lib() -> ctypes.CDLL:
         L.dbspmspv_export_blocks.argtypes = [vp, vp, vp, vp, vp]
         L.dbspmspv_export_views.argtypes = [vp, vp, vp, vp, vp]
         L.dbspmspv_compact_noalloc.argtypes = [vp, vp, i64, vp, vp, i64, vp, vp]
+        L.dbspmspv_test_bounded_wait.argtypes = [vp, i32, vp]
         L.dbspmspv_set_run_opts.argtypes = [vp, ctypes.POINTER(RunOpts)]
         L.dbspmspv_destroy.argtypes = [vp]
         L.dbspmspv_strerror.argtypes = [ctypes.c_int]
@@ -211,6 +213,11 @@ def dbspmspv_compact_noalloc(acc, hit_bitmap, m, y_idx, y_val, y_capacity, y_nnz
     _check(lib().dbspmspv_compact_noalloc(_ptr(acc), _ptr(hit_bitmap), m, _ptr(y_idx), _ptr(y_val),
                                           y_capacity, _ptr(y_nnz), _stream() if stream is None else stream),
            "dbspmspv_compact_noalloc")
+
+
+def dbspmspv_test_bounded_wait(h, max_tries: int, stream: Optional[int] = None) -> None:
+    _check(lib().dbspmspv_test_bounded_wait(h, max_tries, _stream() if stream is None else stream),
+           "dbspmspv_test_bounded_wait")
 
 
 def dbspmspv_set_run_opts(h, opts: RunOpts) -> None:

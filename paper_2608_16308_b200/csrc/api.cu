@@ -105,7 +105,9 @@ extern "C" {
 
 int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out) {
     if (!h || !out) return DBSPMSPV_ERR_INVALID_ARG;
-    DBS_CUDA(cudaDeviceSynchronize());
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
+    // wait for the handle's own work only: the stream its last call was enqueued on
+    DBS_CUDA(cudaStreamSynchronize(h->last_stream));
     dbs::Counters c;
     DBS_CUDA(cudaMemcpy(&c, h->d.ws.ctr, sizeof(c), cudaMemcpyDeviceToHost));
     *out = h->stats;

@@ -508,6 +508,7 @@ extern "C" int db_bfs(dbspmspv_handle_t h, int32_t src, int32_t *levels, dbspmsp
     if (src < 0 || src >= h->d.n) return DBSPMSPV_ERR_INVALID_ARG;
     if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
     switch (h->d.dtype) {
         case DBSPMSPV_F32: return dbs::bfs_typed<DBSPMSPV_F32>(h, src, levels, st);
         case DBSPMSPV_BF16: return dbs::bfs_typed<DBSPMSPV_BF16>(h, src, levels, st);

@@ -194,6 +194,7 @@ struct dbspmspv_handle_s {
     int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)
     int64_t bfs_index_bytes;
     void *ws_arena;             // the one allocation that holds the whole workspace
+    cudaStream_t last_stream;   // stream of the last run / decode / bfs call (get_stats waits on it)
 };
 
 namespace dbs {

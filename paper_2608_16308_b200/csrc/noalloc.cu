@@ -22,15 +22,26 @@ constexpr int NA_MAX_TILES = 4096;                // -> at most 33,554,432 rows 
 static __device__ __align__(256) int32_t g_tile_scratch[NA_MAX_TILES];
 
 // Host code must not hand `g_tile_scratch` itself to a kernel: on the host that name is only a
-// stand-in for the symbol.  The real device address is looked up once per device.
+// stand-in for the symbol.  The real device address is looked up once per device and kept for
+// the life of the process (a cudaDeviceReset would invalidate it: not supported while the
+// library is in use).
 constexpr int NA_MAX_DEVICES = 64;
 int32_t *g_scratch_addr[NA_MAX_DEVICES] = {};
 std::mutex g_setup_lock;
 
-__global__ void __launch_bounds__(NA_TPB) k_na_count(const uint32_t *__restrict__ hit, int n_words, int32_t *tiles) {
+// Bits at or beyond row m in the last bitmap word are ignored by both passes (so the count and
+// the placement agree whatever the caller left there).
+__device__ __forceinline__ uint32_t na_word(const uint32_t *hit, int wi, int n_words, int64_t m) {
+    if (wi >= n_words) return 0u;
+    uint32_t word = hit[wi];
+    if (wi == n_words - 1 && (m & 31)) word &= (1u << (m & 31)) - 1u;
+    return word;
+}
+
+__global__ void __launch_bounds__(NA_TPB) k_na_count(const uint32_t *__restrict__ hit, int64_t m, int n_words, int32_t *tiles) {
     __shared__ int s_red[NA_TPB / 32];
     const int wi = blockIdx.x * NA_TPB + threadIdx.x;
-    int c = wi < n_words ? __popc(hit[wi]) : 0;
+    int c = __popc(na_word(hit, wi, n_words, m));
     c = __reduce_add_sync(0xFFFFFFFFu, c);
     if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = c;
     __syncthreads();
@@ -60,7 +71,7 @@ __global__ void __launch_bounds__(NA_TPB) k_na_write(const float *__restrict__ a
     }
     __syncthreads();
     const int wi = blockIdx.x * NA_TPB + threadIdx.x;
-    const uint32_t word = wi < n_words ? hit[wi] : 0u;
+    const uint32_t word = na_word(hit, wi, n_words, m);
     const int c = __popc(word);
     int incl = c;
     for (int o = 1; o < 32; o <<= 1) {
@@ -74,7 +85,7 @@ __global__ void __launch_bounds__(NA_TPB) k_na_write(const float *__restrict__ a
     for (int k = 0; k < warp; ++k) pos += s_red[k];
     for (uint32_t wd = word; wd; wd &= wd - 1) {
         const int64_t row = (int64_t)wi * 32 + (__ffs(wd) - 1);
-        if (row < m && pos < capacity) {
+        if (pos < capacity) {
             y_idx[pos] = (int32_t)row;
             if (y_val) y_val[pos] = acc[row];
         }
@@ -104,7 +115,10 @@ extern "C" int dbspmspv_compact_noalloc(const float *acc, const uint32_t *hit_bi
         std::lock_guard<std::mutex> guard(g_setup_lock);
         if (!g_scratch_addr[dev]) {
             int32_t *p = nullptr;
-            if (cudaGetSymbolAddress((void **)&p, g_tile_scratch) != cudaSuccess || !p) return DBSPMSPV_ERR_CUDA;
+            if (cudaGetSymbolAddress((void **)&p, g_tile_scratch) != cudaSuccess || !p) {
+                cudaGetLastError();          // do not leave the error behind for the caller's next check
+                return DBSPMSPV_ERR_CUDA;
+            }
             g_scratch_addr[dev] = p;
         }
         tiles = g_scratch_addr[dev];
@@ -112,7 +126,7 @@ extern "C" int dbspmspv_compact_noalloc(const float *acc, const uint32_t *hit_bi
     const int n_words = (int)((m + 31) / 32);
     const int n_tiles = (int)n_tiles64;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    k_na_count<<<n_tiles, NA_TPB, 0, st>>>(hit_bitmap, n_words, tiles);
+    k_na_count<<<n_tiles, NA_TPB, 0, st>>>(hit_bitmap, m, n_words, tiles);
     k_na_write<<<n_tiles, NA_TPB, 0, st>>>(acc, hit_bitmap, m, n_words, tiles, y_idx, y_val, y_capacity, y_nnz);
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;

@@ -37,7 +37,9 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
     int first = 0, deg = 0, pfirst = 0, pdeg = 0;
     if (t < nnz_x) {
         const int j = x_idx[t];
-        if (validate && (j < 0 || j >= d.n)) {
+        // an index outside [0, n) is never written through: the entry is skipped and the call
+        // reports ERR_BOUNDS (the compare is free next to the dependent scatter)
+        if (j < 0 || j >= d.n) {
             d.ws.ctr->status = DBSPMSPV_ERR_BOUNDS;
         } else {
             float v = 1.0f;
@@ -55,6 +57,7 @@ __global__ void k_xblock_sparse(Device d, const int32_t *__restrict__ x_idx, con
             const uint32_t old = atomicOr(&d.ws.x_mask32[j >> 5], 1u << ((j & 15) + sh));
             newly = ((old >> sh) & 0xFFFFu) == 0;
             fresh = ((old >> ((j & 15) + sh)) & 1u) == 0;     // (an index listed twice emits once)
+            if (validate && !fresh) d.ws.ctr->status = DBSPMSPV_ERR_INVALID_ARG;   // optional check: duplicate index
             jb = j >> 4;
             jcol = j;
         }
@@ -1397,6 +1400,18 @@ __global__ void k_decode_cleanup(Device d) {
     }
 }
 
+// Test hook: the bounded wait of the staging code on a barrier that nothing will ever arrive on
+// (no copy is in flight, so there is nothing to drain): the wait gives up after `max_tries`
+// tries and the kernel records DBSPMSPV_ERR_TIMEOUT, exactly as the pull traversal would.
+__global__ void k_wait_probe(Device d, int max_tries) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+        if (!mbar_wait_bounded(&bar, 0u, max_tries)) d.ws.ctr->status = DBSPMSPV_ERR_TIMEOUT;
+    }
+}
+
 __global__ void k_fill_u32(uint32_t *p, int64_t n, uint32_t v) {
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = v;
 }
@@ -1661,6 +1676,7 @@ int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, i
     if ((int64_t)nnz_x > h->d.n) return DBSPMSPV_ERR_INVALID_ARG;
     if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
     switch (h->d.dtype) {
         case DBSPMSPV_F32: return dbs::run_typed<DBSPMSPV_F32>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
         case DBSPMSPV_BF16: return dbs::run_typed<DBSPMSPV_BF16>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
@@ -1668,10 +1684,22 @@ int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, i
     }
 }
 
+int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_stream_t stream) {
+    if (!h || max_tries < 1 || max_tries > 4096) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    dbs::k_wait_probe<<<1, 32, 0, st>>>(h->d, max_tries);
+    ++h->kernel_launches;
+    DBS_CUDA(cudaGetLastError());
+    return DBSPMSPV_OK;
+}
+
 int dbspmspv_decode(dbspmspv_handle_t h, const void *x, float *y, dbspmspv_stream_t stream) {
     if (!h || !x || !y) return DBSPMSPV_ERR_INVALID_ARG;
     if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
     switch (h->d.dtype) {
         case DBSPMSPV_F32: return dbs::decode_typed<DBSPMSPV_F32>(h, x, y, st);
         case DBSPMSPV_BF16: return dbs::decode_typed<DBSPMSPV_BF16>(h, x, y, st);

@@ -163,13 +163,34 @@ def test_capacity_overflow_is_reported_not_written():
     h.close()
 
 
-def test_validate_flags_out_of_range_index():
+def test_out_of_range_index_is_skipped_and_reported():
+    """With the default options too: the bad entry is never written through, the call reports
+    ERR_BOUNDS once, the other entries give their result, and the handle stays usable."""
+    csr = wl.random_sparse(100, 100, 300, 8)
+    A = ref_matrix(csr)
+    good = wl.SparseVec(100, np.array([1, 7], np.int32), np.ones(2, np.float32))
+    want = oracle.ref_pull(A, good.idx, good.val)
+    for validate in (0, 1):
+        h = Handle(csr, B.F32)
+        h.set_opts(validate=validate)
+        for bad in (5000, -3, 100):
+            x = wl.SparseVec(100, np.array([1, bad, 7], np.int32), np.ones(3, np.float32))
+            check_against_oracle(h.run(x), want)
+            assert h.get_stats(raise_on_device_status=False).device_status == B.ERR_BOUNDS
+            assert h.get_stats().device_status == B.OK
+        check_against_oracle(h.run(good), want)
+        h.close()
+
+
+def test_validate_reports_a_duplicate_index():
     csr = wl.random_sparse(100, 100, 300, 8)
     h = Handle(csr, B.F32)
-    h.set_opts(validate=1)
-    x = wl.SparseVec(100, np.array([1, 5000, 7], np.int32), np.ones(3, np.float32))
+    x = wl.SparseVec(100, np.array([4, 9, 4], np.int32), np.ones(3, np.float32))
     h.run(x)
-    assert h.get_stats(raise_on_device_status=False).device_status == B.ERR_BOUNDS
+    assert h.get_stats().device_status == B.OK               # not checked by default
+    h.set_opts(validate=1)
+    h.run(x)
+    assert h.get_stats(raise_on_device_status=False).device_status == B.ERR_INVALID_ARG
     h.close()
 
 
@@ -199,7 +220,9 @@ def test_identity_permutation_and_block_diagonal_dense():
     for path in PATHS:
         h.set_opts(force_path=path)
         yi, yv, k = h.run(x)
-        assert np.allclose(yv, want[yi], rtol=0, atol=2e-5 * (np.abs(a) @ np.abs(xd)).max())
+        assert k == 16 * len(np.unique(x.idx >> 4))
+        scale = np.abs(a).astype(np.float64) @ np.abs(xd)                   # per row: sum |a x|
+        assert (np.abs(yv.astype(np.float64) - want[yi]) <= 2e-5 * scale[yi]).all()
     h.close()
 
 
@@ -312,4 +335,23 @@ def test_rows_that_sum_to_zero_or_hold_stored_zeros_are_still_reported():
     for p in (B.PATH_AUTO, B.PATH_PUSH, B.PATH_PULL):
         h.set_opts(force_path=p)
         check_against_oracle(h.run(x), want)
+    h.close()
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """The staging waits are bounded: a wait on a barrier that nothing arrives on (no copy in
+    flight) gives up, the kernel records ERR_TIMEOUT, get_stats returns it once, and the handle
+    and the context stay usable."""
+    csr = wl.random_sparse(200, 200, 1500, 12)
+    h = Handle(csr, B.F32)
+    B.dbspmspv_test_bounded_wait(h.h, 64)
+    assert h.get_stats(raise_on_device_status=False).device_status == B.ERR_TIMEOUT
+    assert h.get_stats().device_status == B.OK
+    x = dense_x(csr.n, 5, 0.1)
+    for path in PATHS:
+        h.set_opts(force_path=path)
+        check_against_oracle(h.run(x), oracle.ref_pull(ref_matrix(csr), x.idx, x.val))
+    with pytest.raises(B.DbSpmspvError) as e:
+        B.dbspmspv_test_bounded_wait(h.h, 0)
+    assert e.value.status == B.ERR_INVALID_ARG
     h.close()

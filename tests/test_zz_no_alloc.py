@@ -85,3 +85,20 @@ def test_capacity_empty_and_size_limit():
         B.dbspmspv_compact_noalloc(t, t, 33554432 + 1, t, None, 8, t)
     assert e.value.status == B.ERR_TOO_LARGE
     assert "scratch" in B.dbspmspv_strerror(B.ERR_TOO_LARGE)
+
+
+def test_garbage_bits_beyond_the_last_row_are_ignored():
+    """m not a multiple of 32 and the unused high bits of the last bitmap word set: neither the
+    count nor the placement may see them."""
+    m = 1003                                             # last word holds rows 992..1002
+    yi = np.array([0, 5, 991, 992, 1002], dtype=np.int64)
+    yv = np.array([1.0, -2.0, 3.0, 4.5, -0.25], dtype=np.float32)
+    acc, words = dense_and_bitmap(m, yi, yv)
+    words[-1] |= np.uint32(0xFFFFF800)                   # bits for rows 1003..1023
+    gi, gv, gk, raw = compact(m, acc, words)
+    assert gk == yi.size and np.array_equal(gi, yi) and np.array_equal(gv, yv)
+    assert (raw[yi.size:] == -1).all()
+    with pytest.raises(B.DbSpmspvError) as e:            # m = 0 is rejected, as documented
+        t = torch.zeros(8, dtype=torch.int32, device=DEV)
+        B.dbspmspv_compact_noalloc(t, t, 0, t, None, 8, t)
+    assert e.value.status == B.ERR_INVALID_ARG
