@@ -102,7 +102,7 @@ typedef struct {
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
 typedef struct {
     float th3;               /* dbspmspv_run: push iff the nonempty-vector-block ratio is
-                                below th3.  0.01 in the paper; default 0.98, the crossover
+                                below th3.  0.01 in the paper; default 0.9, the crossover
                                 measured on B200 (the table `bench.py --crossover` prints)    */
     int32_t force_path;      /* DBSPMSPV_PATH_*                                              */
     int32_t popc_threshold;  /* CSR-class blocks: popc(mask) >= this -> row-driven (pull-style)
@@ -158,7 +158,8 @@ typedef struct {
                                       else -1                                                 */
     int64_t kernel_launches;       /* kernels launched through this handle so far             */
     int64_t bfs_index_bytes;       /* row-run index of DB-BFS (0 when not built)              */
-    int32_t reserved[2];
+    int64_t lean_index_bytes;      /* row list / chunk table of the streaming pull (hypersparse
+                                      handles; 0 otherwise)                                   */
 } dbspmspv_stats;
 
 /* Paper thresholds (th0 = 32, th1 = 128, th2 = 2.0, Section 3.2.1).  The segment weights keep
@@ -236,13 +237,16 @@ int dbspmspv_decode(dbspmspv_handle_t h, const void *x, float *y, dbspmspv_strea
 int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out);
 
 /* Test hook: decode the blocked format back to coordinates.  row/col/val: device arrays with
- * room for stats.nnz entries (val may be NULL; element type = the handle's dtype).  Order is
- * block-major; sort before comparing.  Synchronises.                                         */
+ * room for stats.nnz entries (val may be NULL; element type = the handle's dtype).  Order: the
+ * elements of every block-CSR view entry together, entries in view order (see
+ * dbspmspv_export_blocks); sort before comparing with a matrix.  Synchronises.               */
 int dbspmspv_export_coo(dbspmspv_handle_t h, int32_t *row, int32_t *col, void *val);
 
-/* Test hook: per view entry, in primary (block-CSR) order: block coordinates, class code
+/* Test hook: per view entry, in block-CSR view order: block coordinates, class code
  * (DBSPMSPV_BLK_*) and stored elements of the entry.  Device arrays of stats.n_view_entries
- * int32 (any may be NULL).  The entries of one INLINE block are adjacent.                    */
+ * int32 (any may be NULL).  Block-CSR view order: by row block; inside a row block the entries
+ * with a payload first (by column block), then the INLINE elements (one entry each) by
+ * (local row, column) -- the elements of one row are adjacent.                               */
 int dbspmspv_export_blocks(dbspmspv_handle_t h, int32_t *block_row, int32_t *block_col,
                            int32_t *block_class, int32_t *block_nnz);
 

@@ -65,7 +65,7 @@ class Stats(ctypes.Structure):
                 ("bfs_level_nzblk", ctypes.c_int32 * MAX_BFS_LEVELS_RECORDED),
                 ("device_status", ctypes.c_int32), ("last_compute_ms", ctypes.c_float),
                 ("kernel_launches", ctypes.c_int64), ("bfs_index_bytes", ctypes.c_int64),
-                ("reserved", ctypes.c_int32 * 2)]
+                ("lean_index_bytes", ctypes.c_int64)]
 
 
 _lib = None

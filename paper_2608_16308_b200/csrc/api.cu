@@ -195,7 +195,8 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     cudaFree(const_cast<int32_t *>(d.seg_rb));
     cudaFree(const_cast<uint32_t *>(d.row_present32));
     cudaFree(const_cast<int32_t *>(d.rowrun_ptr)); cudaFree(const_cast<uint32_t *>(d.rowrun_idx));
-    cudaFree(const_cast<int32_t *>(d.payload_ptr)); cudaFree(const_cast<int32_t *>(d.payload_pos));
+    cudaFree(const_cast<int32_t *>(d.csr_inl)); cudaFree(const_cast<int32_t *>(d.payload_pos));
+    cudaFree(const_cast<int32_t *>(d.lean_rows)); cudaFree(const_cast<int32_t *>(d.lean_chunk_ord));
     cudaFree(h->csc2csr); cudaFree(h->block_row);
     cudaFree(h->ws_arena);
     if (h->ev[0]) cudaEventDestroy(h->ev[0]);

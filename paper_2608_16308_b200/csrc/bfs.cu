@@ -282,10 +282,9 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             const int rb = 2 * wd + hf;
             const uint32_t need16 = (need >> (16 * hf)) & 0xFFFFu;
             if (rb >= d.mb || !need16) continue;    // warp-uniform
-            const int pbeg = d.payload_ptr[rb], pend = d.payload_ptr[rb + 1];
+            const int pbeg = d.csr.ptr[rb], pend = d.csr_inl[rb];      // the row block's entries with a payload
             uint32_t hit = 0;
-            for (int q = pbeg + lane; q < pend; q += 32) {
-                const int pos = d.payload_pos[q];
+            for (int pos = pbeg + lane; pos < pend; pos += 32) {
                 const uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
                 const uint32_t xm = mask_of(F, idx & IDX_MASK);
                 if (xm) {

@@ -346,6 +346,75 @@ __global__ void k_encode(int32_t n_blocks, const int32_t *blk_start, const uint6
     }
 }
 
+// Sort key of the block-CSR view: row block (27 bits) | group (5 bits: 0 = entry with a payload,
+// 16 + r = INLINE element of local row r) | column block (27 bits) | local column (4 bits).
+// Inside a row block the entries with a payload come first (by column block), then the INLINE
+// elements row by row (by column): the mirror image of the block-CSC order.  The elements of a
+// row are then adjacent, which turns the pull over a hypersparse matrix into a segmented sum.
+constexpr int CSR_KEY_GROUP_SHIFT = 31, CSR_KEY_ROW_SHIFT = 36;
+__global__ void k_csr_keys(int32_t n_entries, const int32_t *entry_row, const uint32_t *idx,
+                           const uint8_t *aux, uint64_t *keys, int32_t *ids) {
+    int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (b >= n_entries) return;
+    const uint32_t v = idx[b];
+    const bool inl = (v >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE;
+    const uint32_t rc = aux[b];
+    const uint64_t group = inl ? 16u + (rc >> 4) : 0u, c = inl ? rc & 15u : 0u;
+    keys[b] = ((uint64_t)entry_row[b] << CSR_KEY_ROW_SHIFT) | (group << CSR_KEY_GROUP_SHIFT) |
+              ((uint64_t)(v & IDX_MASK) << 4) | c;
+    ids[b] = (int32_t)b;
+}
+
+// Moves the entries into their final order; the first INLINE element of every row gets ROW_FLAG.
+__global__ void k_csr_gather(int32_t n_entries, const uint64_t *keys_sorted, const int32_t *ids,
+                             const uint32_t *t_idx, const uint32_t *t_w, const uint8_t *t_aux,
+                             uint32_t *idx, uint32_t *w, uint8_t *aux, int32_t *entry_row) {
+    int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p >= n_entries) return;
+    const int32_t b = ids[p];
+    const uint64_t k = keys_sorted[p];
+    const bool inl = ((k >> CSR_KEY_GROUP_SHIFT) & 31u) >= 16u;
+    const bool head = inl && (p == 0 || (keys_sorted[p - 1] >> CSR_KEY_GROUP_SHIFT) != (k >> CSR_KEY_GROUP_SHIFT));
+    idx[p] = t_idx[b] | (head ? ROW_FLAG : 0u);
+    w[p] = t_w[b];
+    aux[p] = t_aux[b];
+    entry_row[p] = (int32_t)(k >> CSR_KEY_ROW_SHIFT);
+}
+
+// inl[rb], rb = 0..mb: first position whose (row block, group) is >= (rb, 16): the end of row
+// block rb's payload run and the start of its INLINE elements (inl[mb] = n_entries)
+__global__ void k_csr_inl(int32_t mb, const uint64_t *keys_sorted, int32_t n, int32_t *inl) {
+    int64_t rb = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (rb > mb) return;
+    const uint64_t target = ((uint64_t)rb << 5) + 16u;
+    int32_t lo = 0, hi = n;
+    while (lo < hi) {
+        int32_t mid = lo + ((hi - lo) >> 1);
+        if ((keys_sorted[mid] >> CSR_KEY_GROUP_SHIFT) < target) lo = mid + 1; else hi = mid;
+    }
+    inl[rb] = lo;
+}
+
+// Row list of the streaming pull: flag[p] = 1 at the first INLINE element of a row;
+// rows[rank[p]] = that row; chunk_ord[c] = row heads before entry c * LEAN_CHUNK.
+__global__ void k_lean_flags(int32_t n_entries, const uint32_t *idx, int32_t *flag) {
+    int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p <= n_entries) flag[p] = (p < n_entries && (idx[p] & ROW_FLAG)) ? 1 : 0;
+}
+__global__ void k_lean_rows(int32_t n_entries, const uint32_t *idx, const uint8_t *aux, const int32_t *entry_row,
+                            const int32_t *rank, int32_t *rows, int32_t n_chunks, int32_t *chunk_ord) {
+    int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p < n_entries && (idx[p] & ROW_FLAG)) rows[rank[p]] = entry_row[p] * 16 + (int32_t)(aux[p] >> 4);
+    if (p <= n_chunks) {
+        const int64_t e = p * (int64_t)LEAN_CHUNK;
+        chunk_ord[p] = rank[e < n_entries ? e : n_entries];
+    }
+}
+
+__global__ void k_fill_words(uint32_t *p, int64_t n, uint32_t v) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = v;
+}
+
 // first position p in a sorted int array with a[p] >= v, for v = 0..count (pointer arrays)
 __global__ void k_lower_bounds(int32_t count, const int32_t *sorted, int32_t n, int32_t *ptr) {
     int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
@@ -395,7 +464,7 @@ __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
     if (p >= n_blocks) return;
     int32_t b = csc2csr[p];
     uint64_t k = keys_sorted[p];
-    csc_idx[p] = (uint32_t)((k >> 4) & IDX_MASK) | (csr_idx[b] & ~IDX_MASK);
+    csc_idx[p] = (uint32_t)((k >> 4) & IDX_MASK) | (csr_idx[b] & (7u << TYPE_SHIFT));   // class, without the CSR view's flags
     csc_w[p] = csr_w[b];
     csc_aux[p] = csr_aux[b];
     bcol_sorted[p] = (int32_t)(k >> CSC_KEY_COL_SHIFT);
@@ -403,7 +472,7 @@ __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
 
 // ---- row-run index of the INLINE elements (DB-BFS pull levels)
 __global__ void k_rowrun_keys(int32_t n_entries, int64_t m, const int32_t *entry_row, const uint32_t *csr_idx,
-                              const uint8_t *csr_aux, uint64_t *keys, uint32_t *vals, int32_t *is_payload) {
+                              const uint8_t *csr_aux, uint64_t *keys, uint32_t *vals) {
     int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (p >= n_entries) return;
     const uint32_t idx = csr_idx[p], rc = csr_aux[p];
@@ -412,7 +481,6 @@ __global__ void k_rowrun_keys(int32_t n_entries, int64_t m, const int32_t *entry
     const uint64_t col = inl ? (uint64_t)(idx & IDX_MASK) * 16 + (rc & 15u) : 0u;
     keys[p] = (row << 31) | col;
     vals[p] = (idx & IDX_MASK) | ((rc & 15u) << 27);
-    is_payload[p] = inl ? 0 : 1;
 }
 
 // ptr[i] = first position whose row is >= i, i = 0..m
@@ -427,11 +495,13 @@ __global__ void k_rowrun_ptr(int64_t m, const uint64_t *keys_sorted, int32_t n, 
     ptr[i] = lo;
 }
 
-__global__ void k_payload_list(int32_t n_entries, int32_t mb, const int32_t *is_payload, const int32_t *rank,
-                               const int32_t *csr_ptr, int32_t *payload_pos, int32_t *payload_ptr) {
+__global__ void k_payload_flags(int32_t n_entries, const uint32_t *idx, int32_t *flag) {
+    int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p <= n_entries) flag[p] = (p < n_entries && (idx[p] >> TYPE_SHIFT) != DBSPMSPV_BLK_INLINE) ? 1 : 0;
+}
+__global__ void k_payload_list(int32_t n_entries, const int32_t *is_payload, const int32_t *rank, int32_t *payload_pos) {
     int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (p < n_entries && is_payload[p]) payload_pos[rank[p]] = (int32_t)p;
-    if (p <= mb) payload_ptr[p] = rank[csr_ptr[p]];
 }
 
 // ---- pull segments (Section 3.3.2): greedy walk along each row block; a segment closes
@@ -724,28 +794,60 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         DBS_CUDA(cudaMemsetAsync(p, 0, h->payload_bytes + 256, st));
         h->payload_alloc = p; d.payload = p;
     }
+    // class census -> which kernel variant the handle uses, hence what a mask-based block costs
+    unsigned long long cls_h[2 * DBSPMSPV_BLK_NCLASS];
+    DBS_CUDA(cudaMemcpy(cls_h, cls, sizeof(cls_h), cudaMemcpyDeviceToHost));
+    {
+        unsigned long long heavy_nnz = 0;
+        for (int c = DBSPMSPV_BLK_FCSR; c <= DBSPMSPV_BLK_DENSE; ++c) heavy_nnz += cls_h[DBSPMSPV_BLK_NCLASS + c];
+        h->heavy_stage = heavy_nnz * 2 > (unsigned long long)nnzu;
+    }
     DBS_KEEP(d.csr.ptr, d.mb + 1); DBS_KEEP(d.csr.idx, n_entries + VIEW_PAD); DBS_KEEP(d.csr.w, n_entries + VIEW_PAD); DBS_KEEP(d.csr.aux, n_entries + VIEW_PAD);
-    DBS_CUDA(cudaMemsetAsync(d.csr.idx + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.aux + n_entries, 0, VIEW_PAD, st));
+    // the slack behind the last entry is read by whole-group staging copies: a class code that no
+    // kernel acts on
+    k_fill_words<<<1, VIEW_PAD, 0, st>>>(d.csr.idx + n_entries, VIEW_PAD, PAD_IDX);
+    DBS_CUDA(cudaMemsetAsync(d.csr.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csr.aux + n_entries, 0, VIEW_PAD, st));
     DBS_KEEP(d.csc.colptr, (int64_t)d.nb * 17); d.csr.colptr = nullptr;
     DBS_KEEP(d.csc.ptr, d.nb + 1); DBS_KEEP(d.csc.idx, n_entries + VIEW_PAD); DBS_KEEP(d.csc.w, n_entries + VIEW_PAD); DBS_KEEP(d.csc.aux, n_entries + VIEW_PAD);
     DBS_CUDA(cudaMemsetAsync(d.csc.idx + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csc.w + n_entries, 0, VIEW_PAD * 4, st)); DBS_CUDA(cudaMemsetAsync(d.csc.aux + n_entries, 0, VIEW_PAD, st));
     DBS_KEEP(h->csc2csr, n_entries);
     DBS_KEEP(h->block_row, n_entries);
-    if (n_blocks) {
-        uint8_t *pl = static_cast<uint8_t *>(h->payload_alloc);
-        const int g = grid_for(n_blocks, TPB), gi = grid_for(nnzu);
+    { int32_t *t; DBS_KEEP(t, (int64_t)d.mb + 1); d.csr_inl = t; }
+    d.entry_row = h->block_row;
+    {
+        // The entries are encoded block by block -- (row block, column block) order -- into
+        // temporaries and then moved into the block-CSR order (see k_csr_keys).
+        uint32_t *t_idx, *t_w;
+        uint8_t *t_aux;
+        int32_t *t_row, *ids, *ids_alt;
+        uint64_t *k1, *k1_alt;
+        DBS_GET(t_idx, n_entries); DBS_GET(t_w, n_entries); DBS_GET(t_aux, n_entries); DBS_GET(t_row, n_entries);
+        if (n_blocks) {
+            uint8_t *pl = static_cast<uint8_t *>(h->payload_alloc);
+            const int g = grid_for(n_blocks, TPB), gi = grid_for(nnzu);
 #define DBS_ENCODE(DT) do { \
-            k_encode_inline<DT><<<gi, TPB, 0, st>>>(nnzu, block_of, blk_start, ukey, uval, type, eoff, brow, bcol, d.csr.idx, d.csr.w, d.csr.aux, h->block_row); \
-            k_encode<DT><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, d.csr.idx, d.csr.w, d.csr.aux, h->block_row); } while (0)
-        if (dt == DBSPMSPV_F32) DBS_ENCODE(DBSPMSPV_F32);
-        else if (dt == DBSPMSPV_BF16) DBS_ENCODE(DBSPMSPV_BF16);
-        else DBS_ENCODE(DBSPMSPV_PATTERN);
+            k_encode_inline<DT><<<gi, TPB, 0, st>>>(nnzu, block_of, blk_start, ukey, uval, type, eoff, brow, bcol, t_idx, t_w, t_aux, t_row); \
+            k_encode<DT><<<g, TPB, 0, st>>>(n_blocks, blk_start, ukey, uval, type, poff, eoff, brow, bcol, pl, t_idx, t_w, t_aux, t_row); } while (0)
+            if (dt == DBSPMSPV_F32) DBS_ENCODE(DBSPMSPV_F32);
+            else if (dt == DBSPMSPV_BF16) DBS_ENCODE(DBSPMSPV_BF16);
+            else DBS_ENCODE(DBSPMSPV_PATTERN);
 #undef DBS_ENCODE
+        }
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(ukey); tp.release(uval); tp.release(blk_start); tp.release(block_of); tp.release(poff); tp.release(psize);
+        tp.release(brow); tp.release(bcol); tp.release(ecount); tp.release(eoff); tp.release(type);
+        DBS_GET(k1, n_entries); DBS_GET(k1_alt, n_entries); DBS_GET(ids, n_entries); DBS_GET(ids_alt, n_entries);
+        if (n_entries) {
+            k_csr_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, t_row, t_idx, t_aux, k1, ids);
+            DBS_TRY(sort_pairs(tp, k1, k1_alt, ids, ids_alt, (int64_t)n_entries, CSR_KEY_ROW_SHIFT + bits_for((uint64_t)d.mb), st));
+            k_csr_gather<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, k1, ids, t_idx, t_w, t_aux, d.csr.idx, d.csr.w, d.csr.aux, h->block_row);
+        }
+        k_csr_inl<<<grid_for((int64_t)d.mb + 1), TPB, 0, st>>>(d.mb, k1, n_entries, const_cast<int32_t *>(d.csr_inl));
+        k_lower_bounds<<<grid_for(d.mb + 1), TPB, 0, st>>>(d.mb, h->block_row, n_entries, d.csr.ptr);
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(t_idx); tp.release(t_w); tp.release(t_aux); tp.release(t_row);
+        tp.release(k1); tp.release(k1_alt); tp.release(ids); tp.release(ids_alt);
     }
-    k_lower_bounds<<<grid_for(d.mb + 1), TPB, 0, st>>>(d.mb, h->block_row, n_entries, d.csr.ptr);
-    DBS_CUDA(cudaStreamSynchronize(st));
-    tp.release(ukey); tp.release(uval); tp.release(blk_start); tp.release(block_of); tp.release(poff); tp.release(psize);
-    tp.release(brow); tp.release(bcol); tp.release(ecount); tp.release(eoff); tp.release(type);
 
     // block-CSC view: sort the primary entries by column block, and inside it payload entries
     // first (by row block), then the INLINE elements column by column
@@ -767,42 +869,61 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     }
 
     // row-run index for the pull levels of DB-BFS
-    d.rowrun_ptr = nullptr; d.rowrun_idx = nullptr; d.payload_ptr = nullptr; d.payload_pos = nullptr;
+    d.rowrun_ptr = nullptr; d.rowrun_idx = nullptr;
     if (m == n && !h->copts.no_bfs_index) {
         uint64_t *rk, *rk_alt;
         uint32_t *rv, *rv_alt;
-        int32_t *isp, *rank;
         DBS_GET(rk, n_entries); DBS_GET(rk_alt, n_entries); DBS_GET(rv, n_entries); DBS_GET(rv_alt, n_entries);
-        DBS_GET(isp, (int64_t)n_entries + 1); DBS_GET(rank, (int64_t)n_entries + 1);
-        DBS_CUDA(cudaMemsetAsync(isp, 0, ((size_t)n_entries + 1) * 4, st));
         if (n_entries) {
-            k_rowrun_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, m, h->block_row, d.csr.idx, d.csr.aux, rk, rv, isp);
+            k_rowrun_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, m, h->block_row, d.csr.idx, d.csr.aux, rk, rv);
             DBS_TRY(sort_pairs(tp, rk, rk_alt, rv, rv_alt, (int64_t)n_entries, 31 + bits_for((uint64_t)m), st));
         }
-        DBS_TRY(exclusive_sum(tp, isp, rank, (int64_t)n_entries + 1, st));
-        int32_t n_payload = 0;
-        DBS_CUDA(cudaMemcpy(&n_payload, rank + n_entries, 4, cudaMemcpyDeviceToHost));
-        const int32_t n_inline = n_entries - n_payload;
-        int32_t *rp, *pp, *ppos;
-        uint32_t *ri;
-        DBS_KEEP(rp, m + 1); DBS_KEEP(ri, n_inline); DBS_KEEP(pp, (int64_t)d.mb + 1); DBS_KEEP(ppos, n_payload);
-        d.rowrun_ptr = rp; d.rowrun_idx = ri; d.payload_ptr = pp; d.payload_pos = ppos;
+        int32_t *rp;
+        DBS_KEEP(rp, m + 1);
+        d.rowrun_ptr = rp;
         k_rowrun_ptr<<<grid_for(m + 1), TPB, 0, st>>>(m, rk, n_entries, rp);
-        if (n_inline) DBS_CUDA(cudaMemcpyAsync(ri, rv, (size_t)n_inline * 4, cudaMemcpyDeviceToDevice, st));
-        const int64_t span = (int64_t)n_entries > d.mb + 1 ? n_entries : d.mb + 1;
-        k_payload_list<<<grid_for(span), TPB, 0, st>>>(n_entries, d.mb, isp, rank, d.csr.ptr, ppos, pp);
+        int32_t n_inline = 0;      // the entries with a payload sort behind every row
+        DBS_CUDA(cudaMemcpyAsync(&n_inline, rp + m, 4, cudaMemcpyDeviceToHost, st));
         DBS_CUDA(cudaStreamSynchronize(st));
-        tp.release(rk); tp.release(rk_alt); tp.release(rv); tp.release(rv_alt); tp.release(isp); tp.release(rank);
-        h->bfs_index_bytes = ((int64_t)m + 1) * 4 + (int64_t)n_inline * 4 + ((int64_t)d.mb + 1) * 4 + (int64_t)n_payload * 4;
+        uint32_t *ri;
+        DBS_KEEP(ri, n_inline);
+        d.rowrun_idx = ri;
+        if (n_inline) DBS_CUDA(cudaMemcpyAsync(ri, rv, (size_t)n_inline * 4, cudaMemcpyDeviceToDevice, st));
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(rk); tp.release(rk_alt); tp.release(rv); tp.release(rv_alt);
+        h->bfs_index_bytes = ((int64_t)m + 1) * 4 + (int64_t)n_inline * 4;
     }
 
-    // class census -> which kernel variant the handle uses, hence what a mask-based block costs
-    unsigned long long cls_h[2 * DBSPMSPV_BLK_NCLASS];
-    DBS_CUDA(cudaMemcpy(cls_h, cls, sizeof(cls_h), cudaMemcpyDeviceToHost));
-    {
-        unsigned long long heavy_nnz = 0;
-        for (int c = DBSPMSPV_BLK_FCSR; c <= DBSPMSPV_BLK_DENSE; ++c) heavy_nnz += cls_h[DBSPMSPV_BLK_NCLASS + c];
-        h->heavy_stage = heavy_nnz * 2 > (unsigned long long)nnzu;
+    // Streaming pull of hypersparse handles: the list of rows that hold INLINE elements (the
+    // stream itself carries one flag bit per row start), the number of row starts before every
+    // chunk of the stream, and the positions of the few entries with a payload.
+    d.lean_rows = nullptr; d.lean_chunk_ord = nullptr; d.payload_pos = nullptr;
+    d.n_lean_chunks = 0; d.n_payload = 0; d.n_lean_rows = 0;
+    if (!h->heavy_stage) {
+        int32_t *flag, *rank;
+        DBS_GET(flag, (int64_t)n_entries + 1); DBS_GET(rank, (int64_t)n_entries + 1);
+        k_lean_flags<<<grid_for((int64_t)n_entries + 1), TPB, 0, st>>>(n_entries, d.csr.idx, flag);
+        DBS_TRY(exclusive_sum(tp, flag, rank, (int64_t)n_entries + 1, st));
+        int32_t n_rows = 0;
+        DBS_CUDA(cudaMemcpy(&n_rows, rank + n_entries, 4, cudaMemcpyDeviceToHost));
+        d.n_lean_rows = n_rows;
+        d.n_lean_chunks = (int32_t)(((int64_t)n_entries + LEAN_CHUNK - 1) / LEAN_CHUNK);
+        int32_t *rows, *ord;
+        DBS_KEEP(rows, n_rows); DBS_KEEP(ord, (int64_t)d.n_lean_chunks + 1);
+        d.lean_rows = rows; d.lean_chunk_ord = ord;
+        const int64_t span = (int64_t)n_entries > d.n_lean_chunks + 1 ? n_entries : d.n_lean_chunks + 1;
+        k_lean_rows<<<grid_for(span), TPB, 0, st>>>(n_entries, d.csr.idx, d.csr.aux, h->block_row, rank, rows, d.n_lean_chunks, ord);
+        // entries with a payload, in view order
+        k_payload_flags<<<grid_for((int64_t)n_entries + 1), TPB, 0, st>>>(n_entries, d.csr.idx, flag);
+        DBS_TRY(exclusive_sum(tp, flag, rank, (int64_t)n_entries + 1, st));
+        DBS_CUDA(cudaMemcpy(&d.n_payload, rank + n_entries, 4, cudaMemcpyDeviceToHost));
+        int32_t *ppos;
+        DBS_KEEP(ppos, d.n_payload);
+        d.payload_pos = ppos;
+        if (n_entries) k_payload_list<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, flag, rank, ppos);
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(flag); tp.release(rank);
+        h->lean_index_bytes = (int64_t)n_rows * 4 + ((int64_t)d.n_lean_chunks + 1) * 4 + (int64_t)d.n_payload * 4;
     }
 
     // pull segments.  Where mask-based blocks are the bulk of the matrix the lanes of a warp each
@@ -851,10 +972,11 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     s.n_row_blocks = d.mb; s.n_col_blocks = d.nb; s.n_segments = d.n_segments;
     s.payload_bytes = h->payload_bytes;
     s.n_view_entries = d.n_entries;
-    s.csr_view_bytes = ((int64_t)d.mb + 1) * 4 + (int64_t)d.n_entries * 9;
+    s.csr_view_bytes = ((int64_t)d.mb + 1) * 8 + (int64_t)d.n_entries * 9;
     s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.nb * 17 * 4 + (int64_t)d.n_entries * 9;
     s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment) + ((int64_t)d.n_chunks + 1) * 8 + (int64_t)d.n_segments * 4;
     s.bfs_index_bytes = h->bfs_index_bytes;
+    s.lean_index_bytes = h->lean_index_bytes;
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }

@@ -16,6 +16,7 @@ namespace dbs {
 // A "view" is three parallel arrays with one entry per nonempty block:
 //   idx[p]  bits 0..26  the block's index along the *other* dimension (column block in the
 //                       block-CSR view, row block in the block-CSC view)
+//           bit  27     block-CSR view only: first INLINE element of its row (ROW_FLAG)
 //           bit  28     block-CSR view only: first entry of a pull segment
 //           bits 29..31 block class (DBSPMSPV_BLK_*)
 //   w[p]    payload offset in 4-byte words -- or, for INLINE entries, the stored value itself
@@ -25,9 +26,14 @@ namespace dbs {
 // per element (adjacent in both views).
 // A packed local coordinate is one byte: (row << 4) | col.
 // Both views carry the same (w, aux) for a block, so either traversal direction reaches the
-// payload in one hop; the payload itself is stored once, in block-CSR ("primary") order.
-// The block-CSR view is ordered by (row block, column block, local row, local column); the
-// block-CSC view by column block, and inside it as described at View::colptr.
+// payload in one hop; the payload itself is stored once, in (row block, column block) order.
+// The two views mirror each other.  Block-CSR: by row block; inside a row block first the
+// entries with a payload (by column block), then the INLINE elements row by row (by column),
+// with Device::csr_inl marking where they start.  Block-CSC: by column block; inside it the
+// entries with a payload (by row block), then the INLINE elements column by column (by row),
+// see View::colptr.  So the elements of one row are adjacent in the block-CSR view (a pull is a
+// segmented sum over a stream) and those of one column in the block-CSC view (a push visits
+// the listed columns only).
 //
 // Payload per class (V = value size: 4 fp32, 2 bf16, 0 pattern; every block starts on a
 // 16-byte boundary and is padded to a multiple of 16 bytes):
@@ -50,6 +56,14 @@ __host__ __device__ inline bool is_row_major(int type) { return type == DBSPMSPV
 __host__ __device__ inline int public_class(int type) { return type == BLK_CSR_ROWMAJOR ? DBSPMSPV_BLK_CSR : type; }
 constexpr uint32_t IDX_MASK = 0x07FFFFFFu;  // 27 bits
 constexpr int TYPE_SHIFT = 29;
+constexpr uint32_t ROW_FLAG = 1u << 27;     // block-CSR view: first INLINE element of its row
+constexpr uint32_t PAD_IDX = 7u << TYPE_SHIFT;   // class code of the slack behind the last view entry: no kernel acts on it
+// The streaming pull of hypersparse handles takes the block-CSR view in chunks of LEAN_CHUNK
+// entries, one chunk (eight entries per lane) per warp pass.
+#ifndef DBS_LEAN_CHUNK
+#define DBS_LEAN_CHUNK 256
+#endif
+constexpr int LEAN_CHUNK = DBS_LEAN_CHUNK;
 #ifndef DBS_PUSH_CHUNK
 #define DBS_PUSH_CHUNK 32
 #endif
@@ -105,7 +119,7 @@ struct Segment {     // pull work unit: a run of consecutive view entries inside
 constexpr int PULL_CH = DBS_PULL_CH;
 constexpr int MAX_SEG_ENTRIES = 128;
 constexpr int STAGE_CAP = PULL_CH + MAX_SEG_ENTRIES + 32;   // + alignment slack (16 each side)
-constexpr int VIEW_PAD = 64;                                // view arrays are over-allocated by this
+constexpr int VIEW_PAD = LEAN_CHUNK + 32;                    // view arrays are over-allocated by this (a whole staging chunk and alignment slack)
 
 // Dense-x marker for "not listed": a NaN bit pattern that listed values never take (listed
 // NaNs are stored as the canonical quiet NaN), so one gather yields presence and value.
@@ -163,12 +177,22 @@ struct Device {           // everything the kernels need, passed by value
     // Row-run index for the pull levels of DB-BFS (square matrices, unless switched off): the
     // INLINE elements once more, row by row -- rowrun_idx[k] = column block | local column << 27
     // for k in [rowrun_ptr[i], rowrun_ptr[i + 1]) -- so that a row can stop at its first frontier
-    // neighbour; and the block-CSR positions of the entries with a payload, per row block
-    // (payload_pos[payload_ptr[rb] .. payload_ptr[rb + 1])).  Null when not built.
+    // neighbour.  Null when not built.
     const int32_t *rowrun_ptr;
     const uint32_t *rowrun_idx;
-    const int32_t *payload_ptr;
+    // Block-CSR view: csr_inl[rb] = first INLINE element of row block rb; its entries with a
+    // payload are [csr.ptr[rb], csr_inl[rb]), its INLINE elements [csr_inl[rb], csr.ptr[rb + 1]).
+    const int32_t *csr_inl;
+    const int32_t *entry_row;   // row block of every block-CSR view entry
+    // Streaming pull (hypersparse handles only, else null): lean_rows[k] = the k-th row that
+    // holds INLINE elements (the k-th ROW_FLAG of the view); lean_chunk_ord[c] = ROW_FLAGs before
+    // entry c * LEAN_CHUNK; payload_pos[0 .. n_payload) = view positions of the entries with a payload.
+    const int32_t *lean_rows;
+    const int32_t *lean_chunk_ord;
     const int32_t *payload_pos;
+    int32_t n_lean_chunks;
+    int32_t n_lean_rows;
+    int32_t n_payload;
     const uint32_t *row_present32;  // per row block: rows that hold a stored element (two 16-bit masks per word)
     Workspace ws;
 };
@@ -188,11 +212,17 @@ struct dbspmspv_handle_s {
     void *payload_alloc;
     int64_t payload_bytes;
     int bfs_grid;               // co-resident grid size of the BFS kernel
+    // launch configurations, worked out on first use (function attributes and occupancy are per
+    // device, and a handle lives on one device; calls on a handle are stream ordered, so plain fields)
+    int grid_compute, grid_compute_dense, grid_decode_pull;
+    bool lean_configured, lean_configured_dense;
+    bool fused_configured[3];
     bool heavy_stage;           // most stored elements sit in mask-based blocks: MODE 1 kernels
     cudaEvent_t ev[2];          // optional timing of the traversal kernel (run_opts.timing)
     bool timed;
     int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)
     int64_t bfs_index_bytes;
+    int64_t lean_index_bytes;
     void *ws_arena;             // the one allocation that holds the whole workspace
     cudaStream_t last_stream;   // stream of the last run / decode / bfs call (get_stats waits on it)
 };

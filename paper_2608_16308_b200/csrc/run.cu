@@ -8,6 +8,11 @@
 #include "worklist.cuh"
 
 namespace dbs {
+__device__ __forceinline__ int select_path(const Device &d, float th3, int force_path);
+}
+#include "lean_pull.cuh"
+
+namespace dbs {
 
 constexpr int CTA = 128;            // four warps per thread block (Section 3.3.2)
 constexpr int WARPS = CTA / 32;
@@ -734,19 +739,19 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
 #define DBS_MIN_CTAS 1
 #endif
 // Variants of the traversal kernel, chosen per handle from the class census at create:
-//   MODE 0  hypersparse matrices (power-law graphs): no lane-owned / streaming code, smallest
-//           footprint
+//   MODE 0  hypersparse matrices (power-law graphs): the push only -- their pull is the
+//           streaming kernel k_pull_lean, launched next in the stream
 //   MODE 1  matrices whose elements sit mostly in mask-based blocks (pruned layers, banded
 //           matrices): half-warp streaming and lane-owned microkernels
 // Dynamic shared memory: per-warp pull stages | lane scratch of the lane-owned form (MODE 1).
 template <int MODE> constexpr size_t compute_dyn_smem() {
-    return WARPS * sizeof(PullWarp) + (MODE >= 1 ? WARPS * 16 * LANE_ACC_STRIDE * sizeof(float) : 0);
+    return MODE >= 1 ? WARPS * sizeof(PullWarp) + WARPS * 16 * LANE_ACC_STRIDE * sizeof(float) : 0;
 }
 
 template <int DT, typename Out, int MODE>
 __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold, int pull_done) {
     constexpr bool HV = MODE >= 1;
-    __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[WARPS][16 * SY_COPIES];
+    __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[HV ? WARPS : 1][16 * SY_COPIES];
     extern __shared__ __align__(128) uint8_t s_dyn[];
     PullWarp *s_pull = reinterpret_cast<PullWarp *>(s_dyn);
     float *s_lacc = reinterpret_cast<float *>(s_dyn + WARPS * sizeof(PullWarp));
@@ -758,7 +763,8 @@ __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out
     float *lacc = HV ? s_lacc + warp * 16 * LANE_ACC_STRIDE : nullptr;
     if (pull_done && path == DBSPMSPV_PATH_PULL) return;     // (the decode entry's own pull kernel has run)
     if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], lacc);
-    else pull_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], lacc, &s_pull[warp]);
+    else if (HV) pull_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], lacc, &s_pull[warp]);
+    // (MODE 0: the pull is k_pull_lean's)
 }
 
 // Pull of the decode entry for matrices whose elements sit mostly in mask-based blocks (pruned
@@ -1212,13 +1218,15 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
             idx = n_idx; w = n_w; aux = n_aux;
         }
     } else {
+        // the row block's entries with a payload are sorted by column block: [begin, pend)
+        const int pend = d.csr_inl[rb];
         for (int i0 = warp * 32; i0 < n_nzblk; i0 += T) {
             int lo = 0, hi = 0;
             if (i0 + lane < n_nzblk) {
                 const uint32_t cb = (uint32_t)s_active[i0 + lane];
-                int a = begin, b = end;           // first entry with column block >= cb
+                int a = begin, b = pend;          // first entry with column block >= cb
                 while (a < b) { const int mid = a + ((b - a) >> 1); if ((d.csr.idx[mid] & IDX_MASK) < cb) a = mid + 1; else b = mid; }
-                lo = a; b = end;                  // first entry with column block > cb
+                lo = a; b = pend;                 // first entry with column block > cb
                 while (a < b) { const int mid = a + ((b - a) >> 1); if ((d.csr.idx[mid] & IDX_MASK) <= cb) a = mid + 1; else b = mid; }
                 hi = a;
             }
@@ -1227,6 +1235,12 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
                 fetch(lo + t, lo + t < hi, idx, w, aux);
                 step(idx, w, aux, lo + t < hi);
             }
+        }
+        // its INLINE elements (row by row, rare in these handles): each tested against its mask
+        for (int base = pend + warp * 32; base < end; base += T) {
+            uint32_t idx, w, aux;
+            fetch(base + lane, base + lane < end, idx, w, aux);
+            step(idx, w, aux, base + lane < end);
         }
     }
     {
@@ -1446,8 +1460,6 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, siz
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-constexpr int MAX_DEVICES = 64;   // per-device caches of launch configurations (device ordinal modulo this)
-
 // Persistent grid of the traversal kernel: as many thread blocks as fit (0 on error).
 template <int DT, typename Out, int MODE> static int compute_grid(int sm_count) {
     const size_t smem = compute_dyn_smem<MODE>();
@@ -1459,8 +1471,9 @@ template <int DT, typename Out, int MODE> static int compute_grid(int sm_count) 
 
 template <int DT, typename Out, int MODE>
 static int launch_compute(dbspmspv_handle_s *h, Out out, float th3, bool pdl, cudaStream_t st, int pull_done = 0) {
-    static int grids[MAX_DEVICES] = {};     // function attributes and occupancy are per device
-    int &grid = grids[h->device % MAX_DEVICES];
+    // (one handle launches one instantiation per output kind; the decode entry of a handle and its
+    // run entry differ in Out, hence the two slots)
+    int &grid = Out::MASKS ? h->grid_compute : h->grid_compute_dense;
     if (!grid) grid = compute_grid<DT, Out, MODE>(h->sm_count);
     if (!grid) return DBSPMSPV_ERR_CUDA;
     const size_t smem = compute_dyn_smem<MODE>();
@@ -1471,6 +1484,36 @@ static int launch_compute(dbspmspv_handle_s *h, Out out, float th3, bool pdl, cu
     }
     ++h->kernel_launches;
     return DBSPMSPV_OK;
+}
+
+// The streaming pull of hypersparse handles (lean_pull.cuh), launched behind k_compute.
+template <int DT, typename Out>
+static int launch_lean(dbspmspv_handle_s *h, Out out, float th3, cudaStream_t st) {
+    bool &configured = Out::MASKS ? h->lean_configured : h->lean_configured_dense;
+    // filter size: the power of two that holds one bit per column, capped
+    const int n_words = (h->d.nb + 1) / 2;
+    int filter_words = 32;
+    while (filter_words < n_words && filter_words < LEAN_FILTER_MAX_WORDS) filter_words <<= 1;
+    const size_t smem = (size_t)filter_words * 4 + LEAN_WARPS * sizeof(LeanScratch);
+    if (!configured) {
+        auto kernel = k_pull_lean<DT, Out>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DBSPMSPV_ERR_CUDA;
+        configured = true;
+    }
+    DBS_CUDA(launch_pdl(k_pull_lean<DT, Out>, h->sm_count, LEAN_CTA, smem, st, h->d, out, th3, h->ropts.force_path,
+                        h->ropts.popc_threshold, filter_words));
+    ++h->kernel_launches;
+    return DBSPMSPV_OK;
+}
+
+// Upper bound of the selector's ratio known on the host: with at most `nnz_x` listed columns no
+// more than min(nnz_x, nb) vector blocks are nonempty.  When even that stays below th3 the push
+// is certain and the pull kernel need not be launched.
+static bool pull_possible(const dbspmspv_handle_s *h, int64_t nnz_x, float th3) {
+    if (h->ropts.force_path == DBSPMSPV_PATH_PUSH) return false;
+    if (h->ropts.force_path == DBSPMSPV_PATH_PULL) return true;
+    const int64_t most = nnz_x < h->d.nb ? nnz_x : h->d.nb;
+    return !((float)most / (float)h->d.nb < th3);
 }
 
 int allocate_workspace(dbspmspv_handle_s *h) {
@@ -1561,8 +1604,16 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     OutSparse out{d.ws.y_acc, d.ws.y_hit8};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
     if (nnz_x > 0 && d.n_entries > 0) {
-        const int s = h->heavy_stage ? launch_compute<DT, OutSparse, 1>(h, out, h->ropts.th3, true, st)
-                                     : launch_compute<DT, OutSparse, 0>(h, out, h->ropts.th3, true, st);
+        int s = DBSPMSPV_OK;
+        if (h->heavy_stage) {
+            s = launch_compute<DT, OutSparse, 1>(h, out, h->ropts.th3, true, st);
+        } else {
+            // push by k_compute, pull by the streaming kernel: each returns at once when the
+            // selector (evaluated on the device) chose the other; a kernel whose path cannot be
+            // chosen is not launched at all
+            if (h->ropts.force_path != DBSPMSPV_PATH_PULL) s = launch_compute<DT, OutSparse, 0>(h, out, h->ropts.th3, true, st);
+            if (s == DBSPMSPV_OK && pull_possible(h, nnz_x, h->ropts.th3)) s = launch_lean<DT, OutSparse>(h, out, h->ropts.th3, st);
+        }
         if (s != DBSPMSPV_OK) return s;
     }
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
@@ -1590,8 +1641,7 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
         const FusedLayout lay(d.nb, nw * 32);
         if (lay.total <= FUSED_MAX_SMEM) {
             auto kernel = nw == 4 ? k_decode_fused<DT, 4> : nw == 8 ? k_decode_fused<DT, 8> : k_decode_fused<DT, 16>;
-            static bool configured[MAX_DEVICES][3] = {};
-            bool &done = configured[h->device % MAX_DEVICES][nw == 4 ? 0 : nw == 8 ? 1 : 2];
+            bool &done = h->fused_configured[nw == 4 ? 0 : nw == 8 ? 1 : 2];
             if (!done) {
                 DBS_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED_MAX_SMEM));
                 done = true;
@@ -1615,8 +1665,7 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
         int s;
         if (h->heavy_stage) {
             // pull by the lean kernel of its own; the general kernel then only runs a push
-            static int grids[MAX_DEVICES] = {};
-            int &grid = grids[h->device % MAX_DEVICES];
+            int &grid = h->grid_decode_pull;
             if (!grid) {
                 int per_sm = 0;
                 if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_decode_pull<DT>, CTA, 0) != cudaSuccess || per_sm < 1) return DBSPMSPV_ERR_CUDA;
@@ -1626,7 +1675,9 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
             ++h->kernel_launches;
             s = launch_compute<DT, OutDense, 1>(h, out, h->ropts.th3_decode, true, st, 1);
         } else {
-            s = launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, true, st);
+            s = DBSPMSPV_OK;
+            if (h->ropts.force_path != DBSPMSPV_PATH_PULL) s = launch_compute<DT, OutDense, 0>(h, out, h->ropts.th3_decode, true, st);
+            if (s == DBSPMSPV_OK && pull_possible(h, d.n, h->ropts.th3_decode)) s = launch_lean<DT, OutDense>(h, out, h->ropts.th3_decode, st);
         }
         if (s != DBSPMSPV_OK) return s;
     }
@@ -1646,7 +1697,7 @@ extern "C" {
 void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
-    o->th3 = 0.98f;
+    o->th3 = 0.9f;
     o->th3_bfs = 0.05f;
     o->th3_decode = 0.01f;
     o->force_path = DBSPMSPV_PATH_AUTO;

@@ -64,7 +64,9 @@ class Handle:
         kk = min(k, cap)
         return self.y_idx[:kk].cpu().numpy(), self.y_val[:kk].cpu().numpy(), k
 
-    def export_coo(self):
+    def export_coo(self, sort=True):
+        """Stored elements as (row, col, value); sorted by (row, col), or -- sort=False -- in the
+        order of the block-CSR view entries that hold them."""
         nnz = int(self.stats.nnz)
         r = torch.empty(max(nnz, 1), dtype=torch.int32, device=DEV)
         c = torch.empty(max(nnz, 1), dtype=torch.int32, device=DEV)
@@ -76,6 +78,8 @@ class Handle:
         B.dbspmspv_export_coo(self.h, r, c, v)
         r, c = r[:nnz].cpu().numpy(), c[:nnz].cpu().numpy()
         v = None if v is None else v[:nnz].cpu().numpy()
+        if not sort:
+            return r, c, v
         order = np.lexsort((c, r))
         return r[order], c[order], (None if v is None else v[order])
 

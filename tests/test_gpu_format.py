@@ -87,25 +87,27 @@ def test_export_equals_input_and_census(name, make, dtype):
         assert np.array_equal(v.view(np.uint32), csr.val.view(np.uint32))      # bit exact
     elif dtype == B.BF16:
         assert np.array_equal(v.view(np.uint16), to_bf16_bits(csr.val))
-    er, ec, ecls, en = h.export_blocks()                 # per view entry, primary order
+    er, ec, ecls, en = h.export_blocks()                 # per view entry, block-CSR view order
     wr, wc, wcls, wn = cpu_classify(csr.rows(), csr.col_idx, dtype)
-    # entries -> blocks: the entries of one block are adjacent
+    # entries -> blocks: group the entries by (row block, column block)
     ekey = er.astype(np.int64) << 32 | ec
-    assert (np.diff(ekey) >= 0).all()                                           # primary order
-    first = np.r_[True, np.diff(ekey) != 0]
-    br, bc, cls = er[first], ec[first], ecls[first]
-    bn = np.add.reduceat(en, np.flatnonzero(first)) if en.size else en
+    assert (np.diff(er) >= 0).all()                                             # row-block major
+    by_block = np.argsort(ekey, kind="stable")
+    skey = ekey[by_block]
+    first = np.r_[True, np.diff(skey) != 0]
+    br, bc, cls = er[by_block][first], ec[by_block][first], ecls[by_block][first]
+    bn = np.add.reduceat(en[by_block], np.flatnonzero(first)) if en.size else en
     assert np.array_equal(br, wr) and np.array_equal(bc, wc)
     assert np.array_equal(bn, wn) and int(bn.sum()) == csr.nnz
     assert np.array_equal(cls, wcls)
-    assert (en[ecls == B.BLK_INLINE] == 1).all() and first[ecls != B.BLK_INLINE].all()
+    assert np.array_equal(ecls[by_block], np.repeat(cls, np.diff(np.r_[np.flatnonzero(first), skey.size])))  # one class per block
+    inl = ecls == B.BLK_INLINE
+    assert (en[inl] == 1).all() and first[~inl[by_block]].all()                 # a payload block is one entry
     assert s.n_blocks == wr.size and s.n_view_entries == er.size
     for k in range(6):
         assert s.class_blocks[k] == int((wcls == k).sum())
         assert s.class_nnz[k] == int(wn[wcls == k].sum())
-    # dual view: same entry set, consistent pointers, and the block-CSC order: by column block;
-    # inside it the entries with a payload first (by row block), then the INLINE elements column
-    # by column (by row), so that a push can visit single columns
+    # dual view: same entry set and consistent pointers
     rp, cp, crow, c2r = h.export_views()
     ne = er.size
     assert rp[0] == 0 and rp[-1] == ne and cp[0] == 0 and cp[-1] == ne
@@ -113,16 +115,22 @@ def test_export_equals_input_and_census(name, make, dtype):
     assert np.array_equal(np.diff(cp), np.bincount(ec, minlength=s.n_col_blocks))
     assert np.array_equal(np.sort(c2r), np.arange(ne))                          # a permutation
     assert np.array_equal(crow, er[c2r])
-    # the stored elements in primary order: by (row block, column block, local row, local column)
-    prim = np.lexsort((c & 15, r & 15, c >> 4, r >> 4))
-    pr, pc = r[prim], c[prim]
-    elem0 = np.r_[0, np.cumsum(en)[:-1]] if ne else np.zeros(0, np.int64)       # first element of every entry
-    inl = ecls == B.BLK_INLINE
-    lr = np.where(inl, pr[elem0] & 15, 0) if ne else elem0
-    lc = np.where(inl, pc[elem0] & 15, 0) if ne else elem0
-    group = np.where(inl, 16 + lc, 0)
-    key = ((ec.astype(np.int64) << 36) | (group.astype(np.int64) << 31) | (er.astype(np.int64) << 4) | lr)[c2r]
-    assert (np.diff(key) > 0).all()                                             # strictly ascending: the order above
+    # The two orders mirror each other.  Block-CSR: by row block; inside it the entries with a
+    # payload first (by column block), then the INLINE elements row by row (by column), so that
+    # a pull sums each row from adjacent entries.  Block-CSC: by column block; inside it the
+    # entries with a payload (by row block), then the INLINE elements column by column (by row),
+    # so that a push can visit single columns.
+    ur, uc, _ = h.export_coo(sort=False)                 # elements in the order of their entries
+    elem0 = np.r_[0, np.cumsum(en)[:-1]].astype(np.int64) if ne else np.zeros(0, np.int64)
+    lr = np.where(inl, ur[elem0] & 15, 0) if ne else elem0
+    lc = np.where(inl, uc[elem0] & 15, 0) if ne else elem0
+    if ne:
+        assert np.array_equal(ur[elem0] >> 4, er) and np.array_equal(uc[elem0] >> 4, ec)
+    e64, c64 = er.astype(np.int64), ec.astype(np.int64)
+    key_csr = (e64 << 36) | (np.where(inl, 16 + lr, 0).astype(np.int64) << 31) | (c64 << 4) | lc
+    assert (np.diff(key_csr) > 0).all()
+    key_csc = ((c64 << 36) | (np.where(inl, 16 + lc, 0).astype(np.int64) << 31) | (e64 << 4) | lr)[c2r]
+    assert (np.diff(key_csc) > 0).all()
     h.close()
 
 
@@ -151,7 +159,7 @@ def test_threshold_edges():
     """31 / 32 entries (COO vs mid), 128 / 129 (mid vs Dense), skew exactly 2.0 vs above."""
     def cls_of(entries):
         h = Handle(_block(entries), B.F32)
-        c = h.export_blocks()[2][0]
+        c = h.export_blocks()[2][0]                    # (a single block: every entry has its class)
         h.close()
         return c
     full = [(r, c) for r in range(16) for c in range(16)]
