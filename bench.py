@@ -1,14 +1,21 @@
 """Benchmark of the DB-SpMSpV hot path on B200.
 
-Workload at N=1: R-MAT scale 20, edge factor 16, fp32 values, with the
-input-sparsity sweep x nnz fraction 1e-5 ... 0.5.  One *step* is one pass of the whole hot path
-(vector blocking -> selector -> worklist -> block microkernels -> writeback -> compaction) over
-that batch: one dbspmspv_run call per sweep point, six calls.  L2 is flushed before every timed
-call, so every number is cold.  `value` is the bytes the method must touch (B_touch, defined at
-ByteModel below) summed over the sweep, divided by the summed device time.  DB-BFS GTEPS on the
-symmetrised R-MAT scale 22 graph is reported in `bfs` unless --no-bfs is given.
+Workload at N=1: R-MAT scale 20, edge factor 16, fp32 values, with the input-sparsity sweep
+x nnz fraction 1e-5 ... 0.5.  One *step* is one pass of the whole hot path (vector blocking ->
+selector -> worklist -> block microkernels -> writeback -> compaction) over that batch: one
+dbspmspv_run call per sweep point, six calls.  L2 is flushed before every timed call, so the
+headline numbers are cold; an L2-warm pass is reported beside them.
 
-python bench.py [--gpus N --steps K --warmup W] [--impl reference] [--no-bfs]
+Bytes.  Three figures per call (ByteModel below, all computed on the host from the structure of
+(A, x) and the format's documented sizes):
+  B_moved  what the implementation reads and writes on the path it took, each distinct byte
+           once (format bytes as the library's counting pass reports them, plus x and y);
+           `value` = sum of B_moved over the sweep / summed device time;
+  B_touch  the block-granular scope definition: every entry and payload of every column block
+           under a nonempty vector block (what a purely block-granular method must touch);
+  B_min    the format-independent floor of a plain CSC gather.
+
+python bench.py [--gpus N --steps K --warmup W] [--impl reference] [--no-bfs] [--no-extras]
 Under torchrun every rank runs the same sweep on its own GPU (independent replicas: the path
 has no exchange step), times are the max over ranks, `value` is the whole-job aggregate.
 """
@@ -34,48 +41,112 @@ METRIC = "spmspv_sweep_achieved_hbm_GBps"
 UNIT = "GB/s"
 WORKLOAD = "rmat20_ef16_fp32_xsweep_1e-5..0.5"
 VIEW_ENTRY_BYTES = 9          # idx 4 + w 4 + aux 1 per view entry
+NOMINAL_HBM_GBS = 8000.0      # the nominal HBM3e figure, reported beside the measured copy bandwidth
+LEAN_CHUNK = 256              # entries per chunk of the streaming pull (whole chunks are read)
+PUSH, PULL = 1, 2
 
 
 # ---------------------------------------------------------------------------------------------
 # Algorithmic bytes (host, from the structure of A and x)
 # ---------------------------------------------------------------------------------------------
-def payload_bytes_per_entry(cls: np.ndarray, nnz: np.ndarray, vsize: int) -> np.ndarray:
-    """Payload bytes of every view entry from the documented per-class sizes."""
-    out = np.zeros(cls.size, dtype=np.int64)
-    coo = cls == 1
-    out[coo] = ((nnz[coo] + 3) // 4) * 4 + nnz[coo] * vsize
-    mid = (cls >= 2) & (cls <= 4)
-    out[mid] = (48 + nnz[mid] * vsize) if vsize else 32
-    out[cls == 5] = 32 + 256 * vsize
-    return ((out + 15) // 16) * 16          # every block is padded to 16 bytes
+def payload_bytes_of(nnz: np.ndarray, vsize: int, th0=32, th1=128) -> np.ndarray:
+    """Payload bytes of a block with `nnz` stored elements under the default options: below th0
+    none (its elements are INLINE view entries); up to th1 a mask-based block (48-byte header +
+    values; pattern matrices: 32 bytes of masks); above, Dense (32 bytes of masks + 256 values);
+    every block padded to 16 bytes."""
+    out = np.where(nnz < th0, 0, np.where(nnz > th1, 32 + 256 * vsize, (48 + nnz * vsize) if vsize else 32))
+    return ((out + 15) // 16) * 16
 
 
 class ByteModel:
-    """Algorithmic bytes of one SpMSpV call, each distinct byte once.
-    B_touch: what the method must touch -- the view entries (9 bytes each) and payloads of the
-    blocks in active column blocks, a column-pointer pair per active column block, x (8 bytes per
-    listed nonzero, plus mask and staged block per nonempty vector block), y (8 bytes out and an
-    8-byte accumulator read-modify-write per output, 8 bytes of hit flags per touched row block).
-    B_min: the information-theoretic floor of a plain CSC gather -- per listed x_j its column's
-    entries at (value + 4-byte row) each plus a pointer pair, x and y once."""
+    """Byte counts of one SpMSpV call from the matrix structure alone (the library is not
+    consulted: its counting pass, dbspmspv_count_call_bytes, is the cross-check)."""
 
-    def __init__(self, csr: wl.CSR, entry_col: np.ndarray, entry_cls: np.ndarray, entry_nnz: np.ndarray,
-                 vsize: int):
+    def __init__(self, csr: wl.CSR, vsize: int):
         self.csr, self.vsize = csr, vsize
-        nb = (csr.n + 15) // 16
-        per_entry = VIEW_ENTRY_BYTES + payload_bytes_per_entry(entry_cls, entry_nnz, vsize)
-        self.colblock_bytes = np.bincount(entry_col, weights=per_entry, minlength=nb)
+        self.nb = (csr.n + 15) // 16
+        rows = csr.rows()
+        key = (rows.astype(np.int64) >> 4) * self.nb + (csr.col_idx >> 4)
+        ub, inv, cnt = np.unique(key, return_inverse=True, return_counts=True)
+        blk_col = (ub % self.nb).astype(np.int64)
+        inline_blk = cnt < 32
+        elem_inline = inline_blk[inv]
+        pbytes = payload_bytes_of(cnt, vsize)
         self.col_nnz = np.bincount(csr.col_idx, minlength=csr.n)
+        self.inline_col_nnz = np.bincount(csr.col_idx[elem_inline], minlength=csr.n)
+        # per column block: entries with a payload, their payload bytes, all view entries
+        pay = ~inline_blk
+        self.cb_payload_entries = np.bincount(blk_col[pay], minlength=self.nb)
+        self.cb_payload_bytes = np.bincount(blk_col[pay], weights=pbytes[pay], minlength=self.nb)
+        self.cb_inline_entries = np.bincount(csr.col_idx[elem_inline] >> 4, minlength=self.nb)
+        self.blk_col, self.blk_payload_bytes, self.blk_is_payload = blk_col, pbytes, pay
+        self.n_inline = int(elem_inline.sum())
+        self.n_payload = int(pay.sum())
+        self.n_entries = self.n_inline + self.n_payload
+        self.n_lean_rows = int(np.unique(rows[elem_inline]).size)
+        self.heavy = 2 * int(cnt[pay].sum()) > csr.nnz        # most elements in blocks with a payload
+        self.payload_total = float(pbytes.sum())
 
-    def bytes(self, x_idx: np.ndarray, y_nnz: int, y_row_blocks: int):
+    # -- what the format part of a call reads (mirrors dbspmspv_count_call_bytes)
+    def format_bytes(self, x_idx: np.ndarray, path: int) -> dict:
         xb = np.unique(x_idx >> 4)
-        touched = float(self.colblock_bytes[xb].sum())               # view entries + payload
-        pointers = 8.0 * xb.size                                      # column-pointer pair
-        xbytes = 8.0 * x_idx.size + xb.size * (2 + 64)                # list + mask + staged block
-        ybytes = 8.0 * y_nnz + 8.0 * y_nnz + 8.0 * y_row_blocks       # out + acc RMW + mask set/clear
-        b_touch = touched + pointers + xbytes + ybytes
-        b_min = float((8 + self.col_nnz[x_idx] * (self.vsize + 4)).sum()) + 8.0 * x_idx.size + 8.0 * y_nnz
-        return b_touch, b_min, touched + pointers + xb.size * 66     # last: traversal kernel only
+        if path == PUSH:
+            if self.heavy:
+                entries = float((self.cb_payload_entries[xb] + self.cb_inline_entries[xb]).sum())
+                pointers = 8.0 * xb.size
+            else:
+                entries = float(self.inline_col_nnz[x_idx].sum() + self.cb_payload_entries[xb].sum())
+                pointers = 8.0 * x_idx.size + 8.0 * xb.size
+            blocks = float(self.cb_payload_entries[xb].sum())
+            payload = float(self.cb_payload_bytes[xb].sum())
+        else:
+            if x_idx.size == 0:
+                return {"view_entries": 0, "view_bytes": 0, "payload_blocks": 0, "payload_bytes": 0, "pointer_bytes": 0,
+                        "active_vector_blocks": 0}
+            if self.heavy:
+                raise NotImplementedError("pull tables of a payload-dominated handle come from the library's statistics")
+            n_chunks = (self.n_entries + LEAN_CHUNK - 1) // LEAN_CHUNK
+            entries = float(n_chunks * LEAN_CHUNK)
+            pointers = 4.0 * (n_chunks + self.n_lean_rows + self.n_payload)
+            active = np.zeros(self.nb, dtype=bool)
+            active[xb] = True
+            sel = self.blk_is_payload & active[self.blk_col]
+            blocks = float(sel.sum())
+            payload = float(self.blk_payload_bytes[sel].sum())
+        return {"view_entries": int(entries), "view_bytes": int(VIEW_ENTRY_BYTES * entries), "payload_blocks": int(blocks),
+                "payload_bytes": int(payload), "pointer_bytes": int(pointers), "active_vector_blocks": int(xb.size)}
+
+    def moved(self, x_idx: np.ndarray, path: int, y_nnz: int, fmt: dict | None = None) -> dict:
+        """Bytes the implementation moves on `path`, each distinct byte once: the format part
+        (above), x (the list, the dense copy written and gathered, the masks, the clean-up),
+        y (accumulator read-modify-write, hit flags, the sorted output) and the two O(m) scans
+        of the compaction passes (hit flags in, packed masks out and in)."""
+        f = fmt if fmt is not None else self.format_bytes(x_idx, path)
+        m, nx = self.csr.m, x_idx.size
+        xbytes = 8.0 * nx + 4.0 * nx + 4.0 * nx + 2.0 * f["active_vector_blocks"] + 4.0 * nx + 6.0 * nx
+        if path == PULL:
+            xbytes += self.csr.n / 8.0                       # the presence filter, read once per SM from L2
+        ybytes = 8.0 * y_nnz + 2.0 * y_nnz + 8.0 * y_nnz + 8.0 * y_nnz
+        scans = m * 1.0 + (m / 8.0) * 2.0
+        fmt_total = f["view_bytes"] + f["payload_bytes"] + f["pointer_bytes"]
+        return {"format": fmt_total, "x": xbytes, "y": ybytes, "scans": scans, "total": fmt_total + xbytes + ybytes + scans,
+                "traversal_kernel": fmt_total + 4.0 * nx + 10.0 * y_nnz + (self.csr.n / 8.0 if path == PULL else 2.0 * f["active_vector_blocks"])}
+
+    def touch(self, x_idx: np.ndarray, y_nnz: int, y_row_blocks: int) -> float:
+        xb = np.unique(x_idx >> 4)
+        entries = self.cb_payload_entries[xb] + self.cb_inline_entries[xb]
+        touched = float((VIEW_ENTRY_BYTES * entries + self.cb_payload_bytes[xb]).sum())
+        return touched + 8.0 * xb.size + 8.0 * x_idx.size + xb.size * 66 + 16.0 * y_nnz + 8.0 * y_row_blocks
+
+    def floor(self, x_idx: np.ndarray, y_nnz: int) -> float:
+        return float((8 + self.col_nnz[x_idx] * (self.vsize + 4)).sum()) + 8.0 * x_idx.size + 8.0 * y_nnz
+
+    def storage(self) -> dict:
+        """Stored bytes of the plain formats the blocked one replaces (32-bit indices)."""
+        a = self.csr
+        csr = a.nnz * (4 + self.vsize) + 4 * (a.m + 1)
+        csc = a.nnz * (4 + self.vsize) + 4 * (a.n + 1)
+        return {"csr_bytes": int(csr), "csr_plus_csc_bytes": int(csr + csc)}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -134,6 +205,21 @@ def measured_peak_gbs():
     return 6650.0, "fallback"
 
 
+def fractions(nbytes: float, us: float, peak: float) -> dict:
+    gbs = nbytes / us / 1e3 if us > 0 else 0.0
+    return {"GBps": round(gbs, 2), "frac_of_measured": round(gbs / peak, 4), "frac_of_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4)}
+
+
+def ncu_traffic(name: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
+    summary the profiling command wrote under profiles/ (None when there is none)."""
+    p = os.path.join(ROOT, "profiles", name)
+    try:
+        return int(json.load(open(p))["dram_bytes_per_launch"])
+    except Exception:
+        return None
+
+
 # ---------------------------------------------------------------------------------------------
 def reference_arm(args) -> None:
     """--impl reference: the CPU oracle as it stands, on the host cores, same config and metric."""
@@ -145,11 +231,11 @@ def reference_arm(args) -> None:
     A = oracle.RefMatrix(a.m, a.n, a.row_ptr, a.col_idx, a.val)
     A.csc()
     xs = [wl.rmat_x(a.n, f, k) for k, f in enumerate(wl.RMAT_SWEEP)]
-    model = host_byte_model(a)
+    model = ByteModel(a, 4)
     per_step = []
-    btouch_step = 0.0
+    bytes_step = 0.0
     for it in range(args.warmup + args.steps):
-        t_step, btouch_step = 0.0, 0.0
+        t_step, bytes_step = 0.0, 0.0
         for x in xs:
             best = None
             for fn in (oracle.ref_push, oracle.ref_pull):
@@ -158,11 +244,13 @@ def reference_arm(args) -> None:
                 dt = time.perf_counter() - t0
                 best = dt if best is None or dt < best else best
             t_step += best
-            btouch_step += model.bytes(x.idx, yi.size, np.unique(yi >> 4).size)[0]
+            # same numerator as the GPU arm: the bytes the library moves on its default path
+            path = PUSH if np.float32(np.unique(x.idx >> 4).size) / np.float32(model.nb) < np.float32(0.9) else PULL
+            bytes_step += model.moved(x.idx, path, yi.size)["total"]
         if it >= args.warmup:
             per_step.append(t_step)
     ms = 1e3 * float(np.mean(per_step))
-    value = btouch_step / (ms * 1e-3) / 1e9
+    value = bytes_step / (ms * 1e-3) / 1e9
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -174,24 +262,54 @@ def reference_arm(args) -> None:
     print(json.dumps(line))
 
 
-def host_byte_model(a: wl.CSR) -> ByteModel:
-    """Byte model with the class census computed on the host (used by the reference arm, where
-    no GPU library is loaded): the documented classification rule applied with numpy."""
-    rows = a.rows()
-    key = (rows.astype(np.int64) >> 4) * ((a.n + 15) // 16) + (a.col_idx >> 4)
-    ub, cnt = np.unique(key, return_counts=True)
-    bcol = (ub % ((a.n + 15) // 16)).astype(np.int64)
-    # blocks with fewer than 32 entries are INLINE (one 9-byte view entry per element, the
-    # library's default); the handful of denser blocks are counted as CSR-class or Dense
-    inl = cnt < 32
-    cls = np.where(inl, 0, np.where(cnt < 32, 1, np.where(cnt > 128, 5, 4))).astype(np.int32)
-    ecol = np.concatenate([np.repeat(bcol[inl], cnt[inl]), bcol[~inl]])
-    ecls = np.concatenate([np.zeros(int(cnt[inl].sum()), np.int32), cls[~inl]])
-    ennz = np.concatenate([np.ones(int(cnt[inl].sum()), np.int64), cnt[~inl]])
-    return ByteModel(a, ecol, ecls, ennz, 4)
-
-
 # ---------------------------------------------------------------------------------------------
+def stats_of(ts_us) -> dict:
+    a = np.asarray(ts_us, dtype=np.float64)
+    return {"us": round(float(np.median(a)), 2), "us_min": round(float(a.min()), 2), "us_p90": round(float(np.percentile(a, 90)), 2)}
+
+
+def timed_calls(torch, fn, flush, reps: int, warm: bool = False):
+    """Device time of `reps` calls of fn (CUDA events on the current stream); cold: L2 flushed
+    (512 MB write) before every call, outside the event pair; warm: back to back, with a short
+    spin kernel in front of the first event so that the host has enqueued the whole call before
+    the device reaches it (otherwise a call of a few microseconds measures the host's launch
+    rate, not the device)."""
+    ts = []
+    for it in range(reps + 3):
+        if not warm:
+            flush.fill_(it & 0xFF)
+        else:
+            torch.cuda._sleep(200000)          # ~0.1 ms of spinning; touches no memory
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            ts.append(e0.elapsed_time(e1) * 1e3)
+    return ts
+
+
+def latency_floors(B, torch, dev, flush) -> dict:
+    """Floors of the machine for the latency-bound calls: an empty kernel (launch + completion)
+    and the time of one dependent load, through a random cycle larger than L2 (DRAM) and
+    through one that fits in L2."""
+    out = {}
+    ts = timed_calls(torch, lambda: B.dbspmspv_probe_floor(0), flush, 30, warm=True)
+    out["empty_kernel_us"] = round(float(np.median(ts)), 2)
+    res = torch.zeros(1, dtype=torch.int32, device=dev)
+    for label, n in (("dram", 64 << 20), ("l2", 1 << 20)):
+        # one cycle through all n elements: i -> (i + stride) mod n with an odd stride is a
+        # permutation with a single cycle when n is a power of two
+        stride = (n // 2 + 12345) | 1
+        chain = ((torch.arange(n, dtype=torch.int64, device=dev) + stride) % n).to(torch.int32)
+        steps = 256
+        ts = timed_calls(torch, lambda: B.dbspmspv_probe_floor(1, chain, 0, steps, res), flush, 10, warm=(label == "l2"))
+        out[f"dependent_load_{label}_ns"] = round((float(np.median(ts)) - out["empty_kernel_us"]) * 1e3 / steps, 1)
+        del chain
+    return out
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -199,6 +317,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-bfs", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configurations, the ablation and the storage table")
     ap.add_argument("--bfs-scale", type=int, default=22)
     ap.add_argument("--bfs-only", action="store_true",
                     help="run only the DB-BFS leg and print its record (the command ncu captures k_bfs from)")
@@ -206,6 +325,7 @@ def main() -> None:
                     help="run only the decode layers and print their records (the command ncu captures k_decode_fused from)")
     ap.add_argument("--crossover", action="store_true",
                     help="print the measured push/pull crossover table (forced paths) and exit")
+    ap.add_argument("--ablation", action="store_true", help="print the block-format ablation and storage records and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -224,15 +344,16 @@ def main() -> None:
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    if args.bfs_only:
+    peak, peak_kind = measured_peak_gbs()
+    if args.bfs_only or args.decode_only or args.ablation:
         if rank == 0:
             flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
-            print(json.dumps(bench_bfs(args, B, torch, dev, flush)))
-        return
-    if args.decode_only:
-        if rank == 0:
-            flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
-            print(json.dumps(decode_layers(B, torch, dev, cold_call_timer(torch, flush))))
+            if args.bfs_only:
+                print(json.dumps(bench_bfs(args, B, torch, dev, flush, peak)))
+            elif args.decode_only:
+                print(json.dumps(decode_layers(B, torch, dev, flush, peak)))
+            else:
+                print(json.dumps({"format_ablation": format_ablation(B, torch, dev, flush), "storage": storage_table(B, torch, dev)}))
         return
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
@@ -246,13 +367,7 @@ def main() -> None:
     a = wl.rmat(20, 16, seed=1)
     h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(a.val), B.F32)
     st0 = B.dbspmspv_get_stats(h)
-    ne = int(st0.n_view_entries)
-    e_col = torch.empty(ne, dtype=torch.int32, device=dev)
-    e_cls = torch.empty(ne, dtype=torch.int32, device=dev)
-    e_nnz = torch.empty(ne, dtype=torch.int32, device=dev)
-    B.dbspmspv_export_blocks(h, None, e_col, e_cls, e_nnz)
-    model = ByteModel(a, e_col.cpu().numpy().astype(np.int64), e_cls.cpu().numpy(), e_nnz.cpu().numpy().astype(np.int64), 4)
-    del e_col, e_cls, e_nnz
+    model = ByteModel(a, 4)
 
     xs = [wl.rmat_x(a.n, f, k) for k, f in enumerate(wl.RMAT_SWEEP)]
     xd = [(up(x.idx), up(x.val)) for x in xs]
@@ -321,6 +436,12 @@ def main() -> None:
     step_ms = call_ms.sum(axis=1)
     ms_per_step = max_over_ranks(float(step_ms.mean()), dev)
 
+    # L2-warm pass: the same calls back to back, no flush (small formats and vectors stay in L2;
+    # never to be read as HBM bandwidth)
+    warm_us = []
+    for k in range(npts):
+        warm_us.append(float(np.median(timed_calls(torch, lambda: one_call(k), flush, 10, warm=True))))
+
     # ---- end to end through the same C-ABI call with HOST buffers: x and y live in page-locked
     # host memory that the device addresses directly, so the call's own kernels read x and write
     # y (and the count) across PCIe -- no staging copy, one synchronisation per call
@@ -347,70 +468,100 @@ def main() -> None:
             e2e_ms.append(tot)
     e2e_ms_step = max_over_ranks(float(np.mean(e2e_ms)), dev)
 
-    peak, peak_kind = measured_peak_gbs()
-    sweep, b_touch_total = [], 0.0
+    sweep, b_moved_total, b_touch_total, b_min_total = [], 0.0, 0.0, 0.0
+    moved_by_point = []
     for k, x in enumerate(xs):
         path, nzblk, ntasks, yk, yrb = info[k]
-        bt, bm, bk = model.bytes(x.idx, yk, yrb)
-        us = float(np.median(call_ms[:, k])) * 1e3
+        counted = B.dbspmspv_count_call_bytes(h, xd[k][0], int(x.idx.size), path)
+        fmt_model = model.format_bytes(x.idx, path)
+        fmt_counted = {f: int(getattr(counted, f)) for f in fmt_model}
+        mv = model.moved(x.idx, path, yk, fmt_model)
+        moved_by_point.append(mv)
+        bt, bm = model.touch(x.idx, yk, yrb), model.floor(x.idx, yk)
+        st = stats_of(call_ms[:, k] * 1e3)
         kus = float(np.median(kernel_ms[:, k])) * 1e3
+        b_moved_total += mv["total"]
         b_touch_total += bt
-        sweep.append({"x_fraction": wl.RMAT_SWEEP[k], "x_nnz": int(x.idx.size), "path": "push" if path == B.PATH_PUSH else "pull",
-                      "us": round(us, 2), "us_min": round(float(call_ms[:, k].min()) * 1e3, 2),
-                      "traversal_kernel_us": round(kus, 2), "y_nnz": yk, "n_nzblk": nzblk,
-                      "B_touch": int(bt), "B_min": int(bm), "GBps_touch": round(bt / us / 1e3, 2),
-                      "frac_of_peak_touch": round(bt / us / 1e3 / peak, 4), "frac_of_peak_min": round(bm / us / 1e3 / peak, 4)})
-    value = world * b_touch_total / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * b_touch_total / (e2e_ms_step * 1e-3) / 1e9
+        b_min_total += bm
+        rec = {"x_fraction": wl.RMAT_SWEEP[k], "x_nnz": int(x.idx.size), "path": "push" if path == B.PATH_PUSH else "pull"}
+        rec.update(st)
+        rec.update({"us_l2_warm": round(warm_us[k], 2), "traversal_kernel_us": round(kus, 2), "y_nnz": yk, "n_nzblk": nzblk,
+                    "n_tasks": ntasks, "B_moved": int(mv["total"]),
+                    "B_moved_parts": {p: int(v) for p, v in mv.items() if p not in ("total", "traversal_kernel")},
+                    "B_touch": int(bt), "B_min": int(bm),
+                    "format_bytes_model_equals_counting_pass": fmt_model == fmt_counted,
+                    "moved": fractions(mv["total"], st["us"], peak), "touch": fractions(bt, st["us"], peak),
+                    "min": fractions(bm, st["us"], peak)})
+        if not rec["format_bytes_model_equals_counting_pass"]:
+            rec["format_bytes_model"], rec["format_bytes_counted"] = fmt_model, fmt_counted
+        sweep.append(rec)
+    value = world * b_moved_total / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * b_moved_total / (e2e_ms_step * 1e-3) / 1e9
     # roofline of the dominant kernel: the traversal kernel at the sweep point that moves the
-    # most bytes (x = 50 %, pull); achieved = its algorithmic bytes / its own duration, measured
-    # with CUDA events recorded inside the library around that launch
-    kdom = int(np.argmax([model.bytes(x.idx, info[k][3], info[k][4])[2] for k, x in enumerate(xs)]))
-    b_kernel_dom = model.bytes(xs[kdom].idx, info[kdom][3], info[kdom][4])[2]
+    # most bytes; achieved = its algorithmic bytes / its own duration, measured with CUDA events
+    # recorded inside the library around that launch
+    kdom = int(np.argmax([mv["traversal_kernel"] for mv in moved_by_point]))
+    b_kernel_dom = moved_by_point[kdom]["traversal_kernel"]
     kernel_dom_ms = float(np.median(kernel_ms[:, kdom]))
     achieved = b_kernel_dom / (kernel_dom_ms * 1e-3) / 1e9
+    dom_pull = info[kdom][0] == B.PATH_PULL
+    dom_name = "k_pull_lean" if dom_pull else "k_compute"
+    traffic = ncu_traffic("k_pull_lean_rmat20_x50pct.json" if dom_pull else "k_compute_push_rmat20_x10pct.json")
     line = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": WORKLOAD, "step": "6 dbspmspv_run calls (one per sweep point), auto path",
                        "l2": "flushed (512 MB write) before every timed call", "block_size": 16,
+                       "bytes": "B_moved: what the implementation reads and writes per call, each distinct byte once",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+            "value_on_B_touch": round(world * b_touch_total / (ms_per_step * 1e-3) / 1e9, 3),
+            "value_on_B_min": round(world * b_min_total / (ms_per_step * 1e-3) / 1e9, 3),
             "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "ms_per_step": round(e2e_ms_step, 5),
                     "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": int(launches),
             "clocks": clocks_summary(samples),
-            "roofline": {"bound": "hbm", "kernel": f"k_compute, x fraction {wl.RMAT_SWEEP[kdom]} ({sweep[kdom]['path']})",
+            "roofline": {"bound": "hbm", "kernel": f"{dom_name}, x fraction {wl.RMAT_SWEEP[kdom]} ({sweep[kdom]['path']})",
                          "achieved": round(achieved, 2), "peak": peak, "peak_kind": f"of {peak_kind}",
-                         "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
-                         "algorithmic_bytes_per_launch": int(b_kernel_dom),
+                         "unit": "GB/s", "frac": round(achieved / peak, 4), "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
+                         "traffic": traffic, "algorithmic_bytes_per_launch": int(b_kernel_dom),
                          "kernel_us": round(kernel_dom_ms * 1e3, 2)},
-            "sweep": sweep, "wall_s_timed_region": round(t_wall, 3)}
+            "sweep": sweep, "wall_s_timed_region": round(t_wall, 3),
+            "format": {"stored_bytes": int(st0.payload_bytes + st0.csr_view_bytes + st0.csc_view_bytes + st0.segment_bytes + st0.lean_index_bytes),
+                       "bfs_index_bytes": int(st0.bfs_index_bytes), **model.storage()}}
 
     if rank == 0 and world == 1:
+        line["latency_floors"] = latency_floors(B, torch, dev, flush)
+        fl = line["latency_floors"]
+        for rec in sweep:
+            rec["us_over_empty_kernel"] = round(rec["us"] / max(fl["empty_kernel_us"], 1e-3), 1)
         line["cusparse_spmv_reference"] = cusparse_reference(a, torch, dev, flush)
-        line["cpu_baseline"] = cpu_baseline(a, xs, model)
-    if rank == 0 and world == 1 and not args.no_bfs:
+        line["cpu_baseline"] = cpu_baseline(a, xs, model, info)
+    if rank == 0 and world == 1 and not args.no_extras:
         try:
-            line["other_configs"] = other_configs(B, torch, dev, flush, peak)
+            line["other_configs"] = other_configs(B, torch, dev, flush, peak, line.get("latency_floors"))
         except Exception as e:
             line["other_configs"] = {"error": repr(e)}
         try:
+            line["format_ablation"] = format_ablation(B, torch, dev, flush)
+            line["storage"] = storage_table(B, torch, dev)
+        except Exception as e:
+            line["format_ablation"] = {"error": repr(e)}
+    if rank == 0 and world == 1 and not args.no_bfs:
+        try:
             # hand the harness's cached device memory back first: with torch's allocator holding
             # the earlier legs' blocks the 3 GB graph format measured 6 % slower (same kernels)
+            B.dbspmspv_destroy(h)
+            h = None
             torch.cuda.empty_cache()
-            line["bfs"] = bench_bfs(args, B, torch, dev, flush)
+            line["bfs"] = bench_bfs(args, B, torch, dev, flush, peak)
         except Exception as e:  # the SpMSpV line must survive a BFS-side problem
             line["bfs"] = {"error": repr(e)}
-    B.dbspmspv_destroy(h)
+    if h is not None:
+        B.dbspmspv_destroy(h)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
-
-
-# DRAM traffic of that launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
-# summarised in profiles/k_compute_pull_rmat20_x50pct.txt
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 156602880
 
 
 def crossover_table() -> None:
@@ -431,16 +582,8 @@ def crossover_table() -> None:
         y_idx = torch.empty(m, dtype=torch.int32, device=dev)
         y_val = torch.empty(m, dtype=torch.float32, device=dev)
         y_nnz = torch.zeros(1, dtype=torch.int32, device=dev)
-        ts = []
-        for it in range(18):
-            flush.fill_(it)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            B.dbspmspv_run(h, xi, xv, int(x.idx.size), B.PLUS_TIMES, y_idx, y_val, m, y_nnz)
-            e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1) * 1e3)
-        return float(np.median(ts[3:]))
+        ts = timed_calls(torch, lambda: B.dbspmspv_run(h, xi, xv, int(x.idx.size), B.PLUS_TIMES, y_idx, y_val, m, y_nnz), flush, 15)
+        return float(np.median(ts))
 
     print("| matrix | x | s_b = N_nzblk/N_blk | push us | pull us | faster |")
     print("|---|---|---|---|---|---|")
@@ -449,9 +592,12 @@ def crossover_table() -> None:
     cases.append(("uniform 16384^2, 8/row", a, [("164 nnz", wl.sparse_x(0, 1, a.n, 164))] +
                   [(f"{f:g}", wl.sparse_x(40 + i, 0, a.n, int(a.n * f))) for i, f in enumerate((0.05, 0.2, 0.5, 1.0))]))
     a2 = wl.rmat(20, 16, seed=1)
-    fr = list(wl.RMAT_SWEEP) + [0.03, 0.05, 0.2, 0.3, 0.7, 1.0]
+    fr = list(wl.RMAT_SWEEP) + [0.03, 0.05, 0.15, 0.2, 0.3, 0.7, 1.0]
     cases.append(("R-MAT scale 20", a2, [(f"{f:g}", wl.rmat_x(a2.n, f, k) if k < 6 else wl.sparse_x(200 + k, 0, a2.n, int(a2.n * f)))
                                          for k, f in enumerate(fr)]))
+    a4 = banded_plus_random(1 << 19, 12, 6, seed=7)
+    cases.append(("band of 12 + 6 random per row, n = 2^19", a4, [(f"{f:g}", wl.sparse_x(300 + i, 0, a4.n, int(a4.n * f)))
+                                                                  for i, f in enumerate((0.001, 0.01, 0.05, 0.2, 0.5))]))
     a3 = wl.stencil27(160, seed=2)
     cases.append(("27-pt stencil 160^3, runs of 64", a3, [(f"{r * 64 / a3.n:.3g}", wl.clustered_x(a3.n, r))
                                                           for r in (64, 3200, 12800, 32000)]))
@@ -465,53 +611,61 @@ def crossover_table() -> None:
         B.dbspmspv_destroy(h)
 
 
-def cold_call_timer(torch, flush):
-    """us of one call: L2 flushed before every call, median of 12 after 3 warm-ups, CUDA events."""
-    def timed(fn):
-        ts = []
-        for it in range(15):
-            flush.fill_(it)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            fn()
-            e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1) * 1e3)
-        return float(np.median(ts[3:]))
-    return timed
+def banded_plus_random(n: int, band: int, extra: int, seed: int) -> wl.CSR:
+    """A matrix between the hypersparse and the payload-dominated extremes: every row holds a
+    band of `band` consecutive columns around the diagonal (dense-ish blocks) plus `extra`
+    uniformly random columns (singleton blocks)."""
+    rows = np.repeat(np.arange(n, dtype=np.int64), band + extra)
+    off = np.tile(np.arange(band, dtype=np.int64) - band // 2, n).reshape(n, band)
+    bandc = np.clip(np.arange(n, dtype=np.int64)[:, None] + off, 0, n - 1)
+    rnd = (wl.rand_u64(seed, 0, np.arange(n * extra, dtype=np.uint64)) % np.uint64(n)).astype(np.int64).reshape(n, extra)
+    cols = np.concatenate([bandc, rnd], axis=1).reshape(-1)
+    key = np.unique(rows * n + cols)
+    r, c = (key // n).astype(np.int64), (key % n).astype(np.int32)
+    row_ptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(np.bincount(r, minlength=n), out=row_ptr[1:])
+    val = (wl.rand_f32(seed, 1, np.arange(key.size, dtype=np.uint64)) * 2.0 - 1.0).astype(np.float32)
+    return wl.CSR(n, n, row_ptr, c, val)
 
 
-def other_configs(B, torch, dev, flush, peak):
-    """The remaining workload shapes, one record each (whole call, cold L2, median of 12 after 3
-    warm-ups): the uniform matrix with a 1 % x, the 27-point stencil with clustered x at 0.1 %
-    and 5 %, and single-token decode on three pruned layer shapes next to a dense bf16 GEMV of
-    the same shape on the same box."""
+def other_configs(B, torch, dev, flush, peak, floors):
+    """The remaining workload shapes, one record each (whole call, cold L2 and L2-warm): the
+    uniform matrix with a 1 % x, the 27-point stencil with clustered x at 0.1 % and 5 %, and
+    single-token decode on three pruned layer shapes next to a dense bf16 GEMV of the same shape
+    on the same box."""
     up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
     out = []
 
-    timed = cold_call_timer(torch, flush)
-
     def spmspv_case(name, a, xs):
         h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(a.val), B.F32)
-        ne = int(B.dbspmspv_get_stats(h).n_view_entries)
-        e_col = torch.empty(ne, dtype=torch.int32, device=dev)
-        e_cls = torch.empty(ne, dtype=torch.int32, device=dev)
-        e_nnz = torch.empty(ne, dtype=torch.int32, device=dev)
-        B.dbspmspv_export_blocks(h, None, e_col, e_cls, e_nnz)
-        model = ByteModel(a, e_col.cpu().numpy().astype(np.int64), e_cls.cpu().numpy(), e_nnz.cpu().numpy().astype(np.int64), 4)
+        model = ByteModel(a, 4)
         y_idx = torch.empty(a.m, dtype=torch.int32, device=dev)
         y_val = torch.empty(a.m, dtype=torch.float32, device=dev)
         y_nnz = torch.zeros(1, dtype=torch.int32, device=dev)
         for label, x in xs:
             xi, xv = up(x.idx), up(x.val)
-            us = timed(lambda: B.dbspmspv_run(h, xi, xv, int(x.idx.size), B.PLUS_TIMES, y_idx, y_val, a.m, y_nnz))
-            st = B.dbspmspv_get_stats(h)
+            call = lambda: B.dbspmspv_run(h, xi, xv, int(x.idx.size), B.PLUS_TIMES, y_idx, y_val, a.m, y_nnz)
+            st = stats_of(timed_calls(torch, call, flush, 12))
+            warm = float(np.median(timed_calls(torch, call, flush, 10, warm=True)))
+            stt = B.dbspmspv_get_stats(h)
             k = int(y_nnz.item())
             yrb = int(np.unique(y_idx[:k].cpu().numpy() >> 4).size)
-            bt = model.bytes(x.idx, k, yrb)[0]
-            out.append({"workload": name, "x": label, "path": "push" if st.last_path == B.PATH_PUSH else "pull",
-                        "us": round(us, 2), "y_nnz": k, "B_touch": int(bt), "GBps_touch": round(bt / us / 1e3, 2),
-                        "frac_of_peak_touch": round(bt / us / 1e3 / peak, 4)})
+            path = int(stt.last_path)
+            counted = B.dbspmspv_count_call_bytes(h, xi, int(x.idx.size), path)
+            fmt = {f: int(getattr(counted, f)) for f in ("view_entries", "view_bytes", "payload_blocks", "payload_bytes",
+                                                          "pointer_bytes", "active_vector_blocks")}
+            mv = model.moved(x.idx, path, k, fmt)       # format part from the counting pass (tables of a payload-dominated handle)
+            bt, bm = model.touch(x.idx, k, yrb), model.floor(x.idx, k)
+            rec = {"workload": name, "x": label, "path": "push" if path == B.PATH_PUSH else "pull"}
+            rec.update(st)
+            rec.update({"us_l2_warm": round(warm, 2), "y_nnz": k, "B_moved": int(mv["total"]), "B_touch": int(bt), "B_min": int(bm),
+                        "moved": fractions(mv["total"], st["us"], peak), "touch": fractions(bt, st["us"], peak),
+                        "min": fractions(bm, st["us"], peak)})
+            if path == B.PATH_PUSH:
+                rec["format_bytes_model_equals_counting_pass"] = model.format_bytes(x.idx, path) == fmt
+            if floors:
+                rec["us_over_empty_kernel"] = round(st["us"] / max(floors["empty_kernel_us"], 1e-3), 1)
+            out.append(rec)
         B.dbspmspv_destroy(h)
 
     a1 = wl.uniform_rows()
@@ -520,11 +674,37 @@ def other_configs(B, torch, dev, flush, peak):
     spmspv_case("stencil27_160cubed_fp32", a3, [("0.1 % in runs of 64", wl.clustered_x(a3.n, 64)),
                                                  ("5 % in runs of 64", wl.clustered_x(a3.n, 3200))])
     del a3
-    out += decode_layers(B, torch, dev, timed)
+    out += decode_layers(B, torch, dev, flush, peak)
     return out
 
 
-def decode_layers(B, torch, dev, timed):
+def decode_bytes(wgt: wl.CSR, x: np.ndarray) -> dict:
+    """Algorithmic bytes of one decode call on a pruned bf16 layer: the whole block-CSR view
+    (the pull walks it), under every nonempty vector block the block's 48-byte header (32-byte
+    for Dense) and the 2-byte values of its active columns, x (2 bytes per entry) and y (4 per
+    row).  B_min: the CSC floor -- per active column its entries at 2 + 4 bytes, x and y."""
+    m, n = wgt.m, wgt.n
+    rows = wgt.rows()
+    nbk = (n + 15) // 16
+    key = (rows.astype(np.int64) >> 4) * nbk + (wgt.col_idx >> 4)
+    ub, inv, cnt = np.unique(key, return_inverse=True, return_counts=True)
+    active_col = x != 0
+    elem_active = active_col[wgt.col_idx]
+    blk_active_vals = np.bincount(inv[elem_active], minlength=ub.size)
+    cbmask = np.zeros(nbk, dtype=bool)
+    cbmask[np.unique(np.flatnonzero(active_col) >> 4)] = True
+    blk_touched = cbmask[(ub % nbk)]
+    inline = cnt < 32
+    n_entries = int(cnt[inline].sum() + (~inline).sum())
+    header = np.where(cnt > 128, 32, 48)
+    payload = float((header[blk_touched & ~inline]).sum() + 2.0 * blk_active_vals[blk_touched & ~inline].sum())
+    moved = 9.0 * n_entries + 4.0 * ((m + 15) // 16 + 1) + payload + 2.0 * n + 4.0 * m
+    col_nnz = np.bincount(wgt.col_idx, minlength=n)
+    floor = float((8 + col_nnz[active_col] * 6).sum()) + 2.0 * n + 4.0 * m
+    return {"B_moved": int(moved), "B_min": int(floor), "payload_bytes_touched": int(payload)}
+
+
+def decode_layers(B, torch, dev, flush, peak):
     """Single-token decode on the three pruned layer shapes (bf16, 50 % magnitude-pruned) at
     70 % and 90 % activation zeros, whole call, next to a dense bf16 GEMV of the same shape."""
     up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
@@ -536,54 +716,113 @@ def decode_layers(B, torch, dev, timed):
         y = torch.empty(m, dtype=torch.float32, device=dev)
         wd = torch.randn(m, n, device=dev, dtype=torch.bfloat16)
         xb = torch.randn(n, device=dev, dtype=torch.bfloat16)
-        gemv = timed(lambda: torch.mv(wd, xb))
+        gemv = float(np.median(timed_calls(torch, lambda: torch.mv(wd, xb), flush, 12)))
         for zf in (0.7, 0.9):          # 0.9: the activation density of the paper's Table 2
             x = wl.relu_activation(n, zf)
             xd = up(wl.f32_to_bf16_bits(x).view(np.int16))
-            us = timed(lambda: B.dbspmspv_decode(h, xd, y))
-            st = B.dbspmspv_get_stats(h)
-            out.append({"workload": f"decode_{m}x{n}_bf16_prune50_act{int(zf * 100)}zero", "path": "push" if st.last_path == B.PATH_PUSH else "pull",
-                        "us": round(us, 2), "dense_bf16_gemv_us_same_box": round(gemv, 2),
-                        "format_bytes": int(st.payload_bytes + st.csr_view_bytes)})
+            call = lambda: B.dbspmspv_decode(h, xd, y)
+            st = stats_of(timed_calls(torch, call, flush, 12))
+            warm = float(np.median(timed_calls(torch, call, flush, 10, warm=True)))
+            stt = B.dbspmspv_get_stats(h)
+            db = decode_bytes(wgt, wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x)))
+            rec = {"workload": f"decode_{m}x{n}_bf16_prune50_act{int(zf * 100)}zero", "path": "push" if stt.last_path == B.PATH_PUSH else "pull"}
+            rec.update(st)
+            rec.update({"us_l2_warm": round(warm, 2), "dense_bf16_gemv_us_same_box": round(gemv, 2),
+                        "format_bytes": int(stt.payload_bytes + stt.csr_view_bytes), **db,
+                        "moved": fractions(db["B_moved"], st["us"], peak), "min": fractions(db["B_min"], st["us"], peak)})
+            out.append(rec)
         B.dbspmspv_destroy(h)
         del wd
     return out
 
 
+def format_ablation(B, torch, dev, flush):
+    """Block-format ablation (Section 5.4): COO-only / CSR-only / automatic block formats, forced
+    pull, x density 0.1, whole call, cold L2 -- on a banded matrix with random fill-in and on the
+    27-point stencil at 96^3."""
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    out = []
+    mats = [("band12_plus_6random_n2^18", banded_plus_random(1 << 18, 12, 6, seed=7)), ("stencil27_96cubed", wl.stencil27(96, seed=2))]
+    for name, a in mats:
+        x = wl.sparse_x(77, 0, a.n, int(a.n * 0.1))
+        y_idx = torch.empty(a.m, dtype=torch.int32, device=dev)
+        y_val = torch.empty(a.m, dtype=torch.float32, device=dev)
+        y_nnz = torch.zeros(1, dtype=torch.int32, device=dev)
+        xi, xv = up(x.idx), up(x.val)
+        rec = {"matrix": name, "nnz": int(a.nnz), "x_density": 0.1, "path": "pull (forced)"}
+        for label, fmt in (("auto", B.FORMAT_AUTO), ("coo_only", B.FORMAT_COO), ("csr_only", B.FORMAT_CSR)):
+            o = B.default_create_opts()
+            o.force_format = fmt
+            h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(a.val), B.F32, 16, o)
+            ro = B.default_run_opts()
+            ro.force_path = B.PATH_PULL
+            B.dbspmspv_set_run_opts(h, ro)
+            ts = timed_calls(torch, lambda: B.dbspmspv_run(h, xi, xv, int(x.idx.size), B.PLUS_TIMES, y_idx, y_val, a.m, y_nnz), flush, 8)
+            us = float(np.median(ts))
+            st = B.dbspmspv_get_stats(h)
+            rec[label] = {"us": round(us, 1), "gflops_on_2nnz": round(2.0 * a.nnz / us / 1e3, 1),
+                          "stored_bytes_per_nnz": round((st.payload_bytes + st.csr_view_bytes + st.csc_view_bytes) / a.nnz, 2)}
+            B.dbspmspv_destroy(h)
+        out.append(rec)
+    return out
+
+
+def storage_table(B, torch, dev):
+    """Stored bytes of the blocked format against CSR and CSR + CSC (Section 5.5's accounting,
+    on the synthetic inputs; 32-bit indices, the configuration's value type)."""
+    up = lambda arr: None if arr is None else torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    out = []
+    w = wl.pruned_weight(4096, 11008, 0.5)
+    cases = [("uniform16384_8perrow_fp32", wl.uniform_rows(), B.F32, 4), ("rmat20_ef16_fp32", wl.rmat(20, 16, seed=1), B.F32, 4),
+             ("stencil27_96cubed_fp32", wl.stencil27(96, seed=2), B.F32, 4), ("decode_4096x11008_bf16_prune50", w, B.BF16, 2),
+             ("rmat18_sym_pattern", wl.rmat(18, 16, seed=3, values=False, symmetrise=True), B.PATTERN, 0)]
+    for name, a, dt, vs in cases:
+        val = None
+        if dt == B.F32:
+            val = a.val
+        elif dt == B.BF16:
+            val = wl.f32_to_bf16_bits(a.val).view(np.int16)
+        h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(val), dt)
+        st = B.dbspmspv_get_stats(h)
+        fmt = int(st.payload_bytes + st.csr_view_bytes + st.csc_view_bytes + st.segment_bytes + st.lean_index_bytes)
+        csr = a.nnz * (4 + vs) + 4 * (a.m + 1)
+        both = 2 * a.nnz * (4 + vs) + 4 * (a.m + a.n + 2)
+        out.append({"matrix": name, "nnz": int(a.nnz), "format_bytes": fmt, "bfs_index_bytes": int(st.bfs_index_bytes),
+                    "payload_bytes": int(st.payload_bytes), "view_bytes": int(st.csr_view_bytes + st.csc_view_bytes),
+                    "csr_bytes": int(csr), "csr_plus_csc_bytes": int(both), "format_bytes_per_nnz": round(fmt / a.nnz, 2),
+                    "vs_csr": round(fmt / csr, 3), "vs_csr_plus_csc": round(fmt / both, 3)})
+        B.dbspmspv_destroy(h)
+    return out
+
+
 def cusparse_reference(a, torch, dev, flush):
     """Same-box library reference: CSR SpMV on x densified to length n (torch's sparse CSR
-    matmul, which calls cuSPARSE).  One time serves every sweep point: a dense x makes the
-    library read the whole matrix whatever x holds.  Harness only; the library never links it."""
+    matmul, which calls cuSPARSE), cold and L2-warm.  One time serves every sweep point: a dense
+    x makes the library read the whole matrix whatever x holds.  Harness only; the library never
+    links it."""
     try:
         A = torch.sparse_csr_tensor(torch.from_numpy(a.row_ptr).to(dev), torch.from_numpy(a.col_idx.astype(np.int64)).to(dev),
                                     torch.from_numpy(a.val).to(dev), size=(a.m, a.n))
         xd = torch.zeros(a.n, 1, dtype=torch.float32, device=dev)
         xd[:: 7] = 1.0
-        ts = []
-        for it in range(13):
-            flush.fill_(it)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            y = A @ xd
-            e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1) * 1e3)
-        return {"us": round(float(np.median(ts[3:])), 2), "what": "torch sparse CSR (cuSPARSE) SpMV, fp32, dense x, cold L2",
-                "csr_bytes": int(a.nnz * 8 + (a.m + 1) * 8)}
+        cold = timed_calls(torch, lambda: A @ xd, flush, 10)
+        warm = timed_calls(torch, lambda: A @ xd, flush, 10, warm=True)
+        return {"us": round(float(np.median(cold)), 2), "us_l2_warm": round(float(np.median(warm)), 2),
+                "what": "torch sparse CSR (cuSPARSE) SpMV, fp32, dense x", "csr_bytes": int(a.nnz * 8 + (a.m + 1) * 8)}
     except Exception as e:
         return {"error": repr(e)}
 
 
-def cpu_baseline(a, xs, model):
+def cpu_baseline(a, xs, model, info):
     """The oracle as it stands, single thread, on the same sweep (bounded: one pass, both
-    routines per point, the faster one counted)."""
+    routines per point, the faster one counted; same byte numerator as the GPU line)."""
     import oracle
     A = oracle.RefMatrix(a.m, a.n, a.row_ptr, a.col_idx, a.val)
     A.csc()
     total_t, total_b = 0.0, 0.0
     for rep in range(2):
         total_t, total_b = 0.0, 0.0
-        for x in xs:
+        for k, x in enumerate(xs):
             best = None
             for fn in (oracle.ref_push, oracle.ref_pull):
                 t0 = time.perf_counter()
@@ -591,51 +830,102 @@ def cpu_baseline(a, xs, model):
                 dt = time.perf_counter() - t0
                 best = dt if best is None or dt < best else best
             total_t += best
-            total_b += model.bytes(x.idx, yi.size, np.unique(yi >> 4).size)[0]
+            total_b += model.moved(x.idx, info[k][0], yi.size)["total"]
     return {"value": round(total_b / total_t / 1e9, 4), "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": "whole 6-point sweep, faster of ref_push/ref_pull per point, second of two passes",
             "ms_per_step": round(total_t * 1e3, 3), "host_cores_available": os.cpu_count()}
 
 
-def bench_bfs(args, B, torch, dev, flush):
-    """DB-BFS GTEPS on the symmetrised R-MAT graph, 16 seeded sources (configs[3])."""
+def bfs_level_bytes(g: wl.CSR, lv: np.ndarray, paths):
+    """Algorithmic bytes per level of one DB-BFS run, from the graph and the levels it produced
+    (an untimed host pass).  Push level: per frontier vertex 8 bytes of column pointers, per
+    frontier edge 5 bytes of view entry (index word + coordinate byte) and 2 bytes of visited
+    mask, per 32 edges an 8-byte task record written and read.  Pull level over the row-run
+    index: per mask word 12 bytes (visited, next, spare), per row still wanted 8 bytes of row
+    pointers, per entry scanned -- a row stops at its first frontier neighbour; entries come in
+    aligned groups of four -- 4 bytes plus 2 bytes of frontier mask.  Both: 4 bytes of level
+    and 4 of frontier word per vertex found."""
+    deg = np.diff(g.row_ptr)
+    out = []
+    n_words = (g.n + 31) // 32
+    for L, path in enumerate(paths):
+        frontier = lv == L
+        found = int((lv == L + 1).sum())
+        if path == PUSH:
+            edges = float(deg[frontier].sum())
+            nbytes = 8.0 * frontier.sum() + 7.0 * edges + 16.0 * (edges / 32.0) + 8.0 * found
+            out.append({"level": L, "path": "push", "frontier": int(frontier.sum()), "edges_walked": int(edges), "bytes": int(nbytes)})
+        else:
+            want = ((lv > L) | (lv < 0)) & (deg > 0)
+            hit = frontier[g.col_idx]                              # entries whose column is in the frontier
+            pos = np.flatnonzero(hit)
+            row_of = np.searchsorted(g.row_ptr, pos, side="right") - 1
+            first = np.full(g.n, -1, dtype=np.int64)
+            keep = np.r_[True, row_of[1:] != row_of[:-1]] if pos.size else np.zeros(0, bool)
+            first[row_of[keep]] = pos[keep]
+            start, end = g.row_ptr[:-1], g.row_ptr[1:]
+            stop = np.where(first >= 0, first + 1, end)            # scanned up to the first hit, else the whole row
+            scanned = ((stop + 3) // 4) * 4 - (start // 4) * 4
+            scanned = np.minimum(scanned, ((end + 3) // 4) * 4 - (start // 4) * 4)
+            entries = float(scanned[want].sum())
+            nbytes = 12.0 * n_words + 8.0 * want.sum() + 6.0 * entries + 8.0 * found
+            out.append({"level": L, "path": "pull", "rows_wanted": int(want.sum()), "entries_scanned": int(entries), "bytes": int(nbytes)})
+    return out
+
+
+def bench_bfs(args, B, torch, dev, flush, peak):
+    """DB-BFS GTEPS on the symmetrised R-MAT graph, 16 seeded sources (configs[3]); every timed
+    source is compared with the oracle; per-level time, direction and algorithmic bytes for the
+    first source."""
     g = wl.rmat(args.bfs_scale, 16, seed=3, values=False, symmetrise=True)
     up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
     h = B.dbspmspv_create_csr(g.m, g.n, g.nnz, up(g.row_ptr), up(g.col_idx), None, B.PATTERN)
+    st0 = B.dbspmspv_get_stats(h)
     srcs = wl.bfs_sources(g, 16)
     deg = np.diff(g.row_ptr)
     levels = torch.empty(g.n, dtype=torch.int32, device=dev)
     import oracle
     A = oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx)
     A.csc()
-    times, teps, nlev, matches, cpu_s, cpu_edges = [], [], [], [], 0.0, 0.0
+    times, warm_times, teps, nlev, matches, cpu_s, cpu_edges = [], [], [], [], [], 0.0, 0.0
+    level_rec = None
     for s in srcs:
-        best = None
-        for rep in range(3):
-            flush.fill_(rep)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            B.db_bfs(h, int(s), levels)
-            e1.record()
-            torch.cuda.synchronize()
-            t = e0.elapsed_time(e1)
-            best = t if best is None or t < best else best
+        ts = timed_calls(torch, lambda: B.db_bfs(h, int(s), levels), flush, 3)
+        tw = timed_calls(torch, lambda: B.db_bfs(h, int(s), levels), flush, 3, warm=True)
+        best = min(ts) * 1e-3
         lv = levels.cpu().numpy()
         edges = float(deg[lv >= 0].sum()) / 2.0
         times.append(best)
+        warm_times.append(min(tw) * 1e-3)
         teps.append(edges / (best * 1e-3) / 1e9)
-        nlev.append(int(B.dbspmspv_get_stats(h).bfs_levels))
+        stt = B.dbspmspv_get_stats(h)
+        nlev.append(int(stt.bfs_levels))
         t0 = time.perf_counter()
         ref = oracle.ref_bfs(A, int(s))               # every timed source is compared with the oracle
         cpu_s += time.perf_counter() - t0
         cpu_edges += float(deg[ref >= 0].sum()) / 2.0
         matches.append(bool(np.array_equal(ref, lv)))
+        if level_rec is None:
+            nl = int(stt.bfs_levels)
+            paths = [int(p) for p in stt.bfs_level_path[:nl]]
+            lb = bfs_level_bytes(g, lv, paths)
+            for L, rec in enumerate(lb):
+                us = float(stt.bfs_level_us[L])
+                rec["us"] = round(us, 1)
+                rec.update(fractions(rec["bytes"], us, peak))
+            total_b = float(sum(r["bytes"] for r in lb)) + 4.0 * g.n + 16.0 * ((g.n + 31) // 32)   # + initialisation of levels and masks
+            level_rec = {"source": int(s), "setup_us": round(float(stt.bfs_setup_us), 1), "levels": lb, "bytes": int(total_b),
+                         "call_us_l2_warm": round(min(tw), 1), "whole_call": fractions(total_b, min(tw), peak),
+                         "note": "level times are device time stamps of the last (L2-warm) run of this source"}
     B.dbspmspv_destroy(h)
     hm = len(teps) / sum(1.0 / t for t in teps)
     return {"workload": f"rmat{args.bfs_scale}_sym_ef16_pattern_16sources", "gteps_harmonic_mean": round(hm, 3),
             "gteps_min": round(min(teps), 3), "gteps_max": round(max(teps), 3),
-            "ms_median": round(float(np.median(times)), 4), "levels": nlev, "vertices": int(g.n), "nnz": int(g.nnz),
+            "ms_median": round(float(np.median(times)), 4), "ms_median_l2_warm": round(float(np.median(warm_times)), 4),
+            "levels": nlev, "vertices": int(g.n), "nnz": int(g.nnz),
             "sources_matching_oracle": int(sum(matches)), "sources": len(matches),
+            "format_bytes": int(st0.payload_bytes + st0.csr_view_bytes + st0.csc_view_bytes + st0.segment_bytes + st0.lean_index_bytes),
+            "bfs_index_bytes": int(st0.bfs_index_bytes), "roofline_first_source": level_rec,
             "cpu_baseline": {"value": round(cpu_edges / cpu_s / 1e9, 4), "unit": "GTEPS",
                              "cores": 1, "kind": "oracle", "sample": "queue BFS from each of the sources"}}
 

@@ -122,7 +122,12 @@ typedef struct {
                                 handles whose elements sit mostly in mask-based blocks and whose
                                 x fits in shared memory) but the blocking / traversal / cleanup
                                 kernels of dbspmspv_run                              (0)    */
-    int32_t reserved[8];
+    float bfs_push_max_edge_frac; /* db_bfs (with the row-run index): a level whose push worklist
+                                covers more than this share of the view's entries is pulled
+                                even when the block ratio says push -- a frontier of a few hub
+                                vertices fills few vector blocks but owns many elements.
+                                0 = block ratio only.  Default measured on B200             */
+    int32_t reserved[7];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64
@@ -160,6 +165,11 @@ typedef struct {
     int64_t bfs_index_bytes;       /* row-run index of DB-BFS (0 when not built)              */
     int64_t lean_index_bytes;      /* row list / chunk table of the streaming pull (hypersparse
                                       handles; 0 otherwise)                                   */
+    /* last db_bfs, from time stamps taken on the device: microseconds before the first level
+       (initialisation of levels and masks) and per level (traversal + frontier bookkeeping)    */
+    float bfs_setup_us;
+    float bfs_level_us[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
+    int32_t reserved[1];
 } dbspmspv_stats;
 
 /* Paper thresholds (th0 = 32, th1 = 128, th2 = 2.0, Section 3.2.1).  The segment weights keep
@@ -289,6 +299,36 @@ int dbspmspv_export_views(dbspmspv_handle_t h, int32_t *csr_row_ptr, int32_t *cs
 int dbspmspv_compact_noalloc(const float *acc, const uint32_t *hit_bitmap, int64_t m,
                              int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
                              dbspmspv_stream_t stream);
+
+/* Measurement aid (untimed; allocates and synchronises): the bytes of the format that ONE call
+ * with this x would read on the given path (DBSPMSPV_PATH_PUSH or _PULL), counted by walking
+ * the format as built -- the check of the benchmark's host-side byte model (Section 5.1 reports
+ * time only; achieved bandwidth needs a numerator).  x_idx: nnz_x device indices.
+ *   push, hypersparse handle: the INLINE run of every listed column and the payload run of
+ *     every nonempty vector block's column block, 8 bytes of pointers each;
+ *   push, handle whose elements sit mostly in blocks with a payload: every entry of the column
+ *     blocks of the nonempty vector blocks;
+ *   pull: the whole block-CSR view (streaming pull: in whole chunks) and its tables;
+ *   both: the payload of every visited block under a nonempty vector block.
+ * x and y traffic is not included (it follows from nnz_x and y_nnz).                          */
+typedef struct {
+    int64_t view_entries;         /* view entries read                                         */
+    int64_t view_bytes;           /* 9 bytes each (index word, value / offset word, byte)      */
+    int64_t payload_blocks;       /* blocks whose payload is fetched                           */
+    int64_t payload_bytes;
+    int64_t pointer_bytes;        /* pointer words, chunk / segment tables, row list           */
+    int64_t active_vector_blocks; /* nonempty vector blocks of x                               */
+    int64_t reserved[2];
+} dbspmspv_call_bytes;
+int dbspmspv_count_call_bytes(dbspmspv_handle_t h, const int32_t *x_idx, int32_t nnz_x, int path,
+                              dbspmspv_call_bytes *out);
+
+/* Measurement aid: latency floors of the machine, enqueued on `stream`.  kind 0: an empty
+ * kernel (launch + completion); kind 1: one thread follows `steps` dependent loads through
+ * `chain` (device int32 array in which element i holds the index of the next element, e.g. one
+ * long random cycle), starting at `start`, and stores where it ended in `out` (device).        */
+int dbspmspv_probe_floor(int kind, const int32_t *chain, int32_t start, int32_t steps, int32_t *out,
+                         dbspmspv_stream_t stream);
 
 /* Test hook for the bounded device-side waits (Section 3.3.3's asynchronous staging completes
  * on barriers in shared memory, and every wait on them has an iteration limit): launches one

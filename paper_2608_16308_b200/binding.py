@@ -28,7 +28,7 @@ EXPORTED_SYMBOLS = (
     "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "dbspmspv_decode", "dbspmspv_get_stats",
     "dbspmspv_export_coo", "dbspmspv_export_blocks", "dbspmspv_export_views",
     "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror", "dbspmspv_compact_noalloc",
-    "dbspmspv_test_bounded_wait",
+    "dbspmspv_test_bounded_wait", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
 )
 
 
@@ -47,7 +47,7 @@ class RunOpts(ctypes.Structure):
                 ("popc_threshold", ctypes.c_int32), ("validate", ctypes.c_int32),
                 ("timing", ctypes.c_int32), ("th3_bfs", ctypes.c_float),
                 ("th3_decode", ctypes.c_float), ("no_fused_decode", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 8)]
+                ("bfs_push_max_edge_frac", ctypes.c_float), ("reserved", ctypes.c_int32 * 7)]
 
 
 class Stats(ctypes.Structure):
@@ -65,7 +65,15 @@ class Stats(ctypes.Structure):
                 ("bfs_level_nzblk", ctypes.c_int32 * MAX_BFS_LEVELS_RECORDED),
                 ("device_status", ctypes.c_int32), ("last_compute_ms", ctypes.c_float),
                 ("kernel_launches", ctypes.c_int64), ("bfs_index_bytes", ctypes.c_int64),
-                ("lean_index_bytes", ctypes.c_int64)]
+                ("lean_index_bytes", ctypes.c_int64), ("bfs_setup_us", ctypes.c_float),
+                ("bfs_level_us", ctypes.c_float * MAX_BFS_LEVELS_RECORDED), ("reserved", ctypes.c_int32 * 1)]
+
+
+class CallBytes(ctypes.Structure):
+    _fields_ = [("view_entries", ctypes.c_int64), ("view_bytes", ctypes.c_int64),
+                ("payload_blocks", ctypes.c_int64), ("payload_bytes", ctypes.c_int64),
+                ("pointer_bytes", ctypes.c_int64), ("active_vector_blocks", ctypes.c_int64),
+                ("reserved", ctypes.c_int64 * 2)]
 
 
 _lib = None
@@ -97,6 +105,8 @@ def lib() -> ctypes.CDLL:
         L.dbspmspv_export_views.argtypes = [vp, vp, vp, vp, vp]
         L.dbspmspv_compact_noalloc.argtypes = [vp, vp, i64, vp, vp, i64, vp, vp]
         L.dbspmspv_test_bounded_wait.argtypes = [vp, i32, vp]
+        L.dbspmspv_count_call_bytes.argtypes = [vp, vp, i32, ctypes.c_int, ctypes.POINTER(CallBytes)]
+        L.dbspmspv_probe_floor.argtypes = [ctypes.c_int, vp, i32, i32, vp, vp]
         L.dbspmspv_set_run_opts.argtypes = [vp, ctypes.POINTER(RunOpts)]
         L.dbspmspv_destroy.argtypes = [vp]
         L.dbspmspv_strerror.argtypes = [ctypes.c_int]
@@ -218,6 +228,17 @@ def dbspmspv_compact_noalloc(acc, hit_bitmap, m, y_idx, y_val, y_capacity, y_nnz
 def dbspmspv_test_bounded_wait(h, max_tries: int, stream: Optional[int] = None) -> None:
     _check(lib().dbspmspv_test_bounded_wait(h, max_tries, _stream() if stream is None else stream),
            "dbspmspv_test_bounded_wait")
+
+
+def dbspmspv_count_call_bytes(h, x_idx, nnz_x: int, path: int) -> CallBytes:
+    out = CallBytes()
+    _check(lib().dbspmspv_count_call_bytes(h, _ptr(x_idx), nnz_x, path, ctypes.byref(out)), "dbspmspv_count_call_bytes")
+    return out
+
+
+def dbspmspv_probe_floor(kind: int, chain=None, start: int = 0, steps: int = 1, out=None, stream: Optional[int] = None) -> None:
+    _check(lib().dbspmspv_probe_floor(kind, _ptr(chain), start, steps, _ptr(out), _stream() if stream is None else stream),
+           "dbspmspv_probe_floor")
 
 
 def dbspmspv_set_run_opts(h, opts: RunOpts) -> None:

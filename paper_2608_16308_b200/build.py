@@ -10,8 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdbspmspv.so")
-SOURCES = ("create.cu", "run.cu", "bfs.cu", "api.cu", "noalloc.cu")
-HEADERS = ("internal.cuh", "microkernels.cuh", "worklist.cuh", "staging.cuh")
+SOURCES = ("create.cu", "run.cu", "bfs.cu", "api.cu", "noalloc.cu", "measure.cu")
+HEADERS = ("internal.cuh", "microkernels.cuh", "worklist.cuh", "staging.cuh", "lean_pull.cuh")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

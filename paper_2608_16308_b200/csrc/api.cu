@@ -121,6 +121,12 @@ int dbspmspv_get_stats(dbspmspv_handle_t h, dbspmspv_stats *out) {
         out->bfs_level_path[k] = c.bfs_level_path[k];
         out->bfs_level_nzblk[k] = c.bfs_level_nzblk[k];
     }
+    {
+        const int nl = c.bfs_levels < DBSPMSPV_MAX_BFS_LEVELS_RECORDED ? c.bfs_levels : DBSPMSPV_MAX_BFS_LEVELS_RECORDED;
+        out->bfs_setup_us = nl >= 0 ? (float)((double)(c.bfs_stamp[1] - c.bfs_stamp[0]) * 1e-3) : 0.f;
+        for (int k = 0; k < DBSPMSPV_MAX_BFS_LEVELS_RECORDED; ++k)
+            out->bfs_level_us[k] = k < nl ? (float)((double)(c.bfs_stamp[k + 2] - c.bfs_stamp[k + 1]) * 1e-3) : 0.f;
+    }
     out->device_status = c.status;
     out->kernel_launches = h->kernel_launches;
     out->last_compute_ms = -1.0f;

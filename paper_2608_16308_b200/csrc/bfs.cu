@@ -44,17 +44,35 @@ __device__ __forceinline__ void write_levels(int32_t *levels, int rb, uint32_t f
     }
 }
 
+// The threads that share a level's work (the whole cooperative grid).
+struct Scope {
+    int tid, nthreads;      // thread index / count in the scope
+    int gwarp, nwarps;      // warp index / count in the scope
+};
+
+// Appends word indices (one per lane with `word` >= 0) to a list: one atomic per warp.
+__device__ __forceinline__ void append_words(int word, int32_t *list, int32_t *count, int lane) {
+    const uint32_t m = __ballot_sync(FULL, word >= 0);
+    if (!m) return;
+    int base = 0;
+    if (lane == __ffs(m) - 1) base = atomicAdd(count, __popc(m));
+    base = __shfl_sync(FULL, base, __ffs(m) - 1);
+    if (word >= 0) list[base + __popc(m & ((1u << lane) - 1u))] = word;
+}
+
 // Boolean push: tasks of the active frontier blocks (a task is at most PUSH_CHUNK = 32 view
 // entries: one warp step); newly reached rows are claimed with one atomicOr per entry on the
 // next-frontier masks (the winner writes the level).  Like the pull, the loop is software-
 // pipelined: while task k is evaluated, the visited masks of k+1, the view entries of k+2 and
-// the task record of k+3 (in this warp's stride) are in flight.
+// the task record of k+3 (in this warp's stride) are in flight.  The thread whose atomic turns a
+// word of the next-frontier masks nonzero lists that word, so that the bookkeeping after the
+// level visits the nonzero words only.
 template <int DT>
-__device__ void bfs_push(const Device &d, const uint32_t *F, uint32_t *N, int n_recs, const int4 *hubs, int n_hubs, int32_t *levels, int depth) {
+__device__ void bfs_push(const Device &d, const Scope &sc, const uint32_t *F, uint32_t *N, int n_recs, const int4 *hubs, int n_hubs,
+                         int32_t *levels, int depth, int32_t *words_out, int32_t *nwords_out) {
     static_assert(PUSH_CHUNK == 32, "one warp step per task");
     const int lane = threadIdx.x & 31;
-    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int gwarp = sc.gwarp, nwarps = sc.nwarps;
     const HubTable table = load_hub_table(hubs, n_hubs, lane);
     const int n_tasks = n_recs + table.total;                    // task records, then the steps of the hub runs
     auto item = [&](int i) { return worklist_item(d.ws.tasks, n_recs, table, i); };
@@ -88,6 +106,7 @@ __device__ void bfs_push(const Device &d, const uint32_t *F, uint32_t *N, int n_
             const int type = idx >> TYPE_SHIFT, brow = idx & IDX_MASK;
             bool heavy = false;
             uint32_t w = 0;
+            int fresh_word = -1;           // a mask word this lane turned nonzero
             if (need0) {
                 uint32_t hit = 0;
                 if (type == DBSPMSPV_BLK_INLINE) {
@@ -106,8 +125,10 @@ __device__ void bfs_push(const Device &d, const uint32_t *F, uint32_t *N, int n_
                     const int sh = (brow & 1) * 16;
                     const uint32_t old = atomicOr(&N[brow >> 1], hit << sh);
                     write_levels(levels, brow, hit & ~(old >> sh), depth);
+                    if (!old) fresh_word = brow >> 1;
                 }
             }
+            append_words(fresh_word, words_out, nwords_out, lane);
             uint32_t hv = __ballot_sync(FULL, heavy);
             while (hv) {
                 const int src = __ffs(hv) - 1;
@@ -122,6 +143,7 @@ __device__ void bfs_push(const Device &d, const uint32_t *F, uint32_t *N, int n_
                     const int sh = (bbrow & 1) * 16;
                     const uint32_t old = atomicOr(&N[bbrow >> 1], hits << sh);
                     write_levels(levels, bbrow, hits & ~(old >> sh), depth);
+                    if (!old) words_out[atomicAdd(nwords_out, 1)] = bbrow >> 1;
                 }
             }
         }
@@ -137,11 +159,10 @@ __device__ void bfs_push(const Device &d, const uint32_t *F, uint32_t *N, int n_
 // last link is waited for: while segment k is evaluated, the entries of k+1, the visited mask
 // of k+2 and the descriptor of k+3 (k counted in this warp's stride) are already in flight.
 template <int DT>
-__device__ void bfs_pull(const Device &d, const uint32_t *F, uint32_t *N, int32_t *levels, int depth) {
+__device__ void bfs_pull(const Device &d, const Scope &sc, const uint32_t *F, uint32_t *N, int32_t *levels, int depth) {
     constexpr int U = MAX_SEG_ENTRIES / 32;
     const int lane = threadIdx.x & 31;
-    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int gwarp = sc.gwarp, nwarps = sc.nwarps;
     const int nseg = d.n_segments;
     const Segment none = Segment{0, 0, 0, 0};
     auto need_of = [&](const Segment &sg) { return (sg.count & 0x7FFFFFFF) ? ~mask_of(d.ws.visited32, sg.row_block) & 0xFFFFu : 0u; };
@@ -251,8 +272,8 @@ __device__ void bfs_pull(const Device &d, const uint32_t *F, uint32_t *N, int32_
 // long (a hub with no frontier neighbour so far) and is finished by the whole warp, 32 entries
 // per step.  The warp owns its mask word: plain stores, no atomics.
 template <int DT>
-__device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, uint32_t *Z, int32_t *nz_out, int32_t *nwords_out,
-                              int32_t *levels, int depth) {
+__device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, uint32_t *Z, int32_t *nz_out, int32_t *words_out,
+                              int32_t *nwords_out, int32_t *levels, int depth) {
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -268,7 +289,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
         int base = 0;
         if (lane == 0) base = atomicAdd(nwords_out, n_batch);
         base = __shfl_sync(FULL, base, 0);
-        if (lane < n_batch) d.ws.bfs_words[base + lane] = batch_wd;
+        if (lane < n_batch) words_out[base + lane] = batch_wd;
         n_batch = 0;
     };
     for (int wd = gwarp; wd < n_words; wd += nwarps) {
@@ -302,15 +323,20 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
         int p = 0, e = 0;
         if (active) { p = d.rowrun_ptr[row]; e = d.rowrun_ptr[row + 1]; active = p < e; }
         bool got = false;
+        // a round = the aligned group of four entries that holds position p: one 16-byte load per
+        // lane (four 4-byte loads cost four trips through the L1 tag stage for the same line)
         for (int round = 0; round < 8 && __any_sync(FULL, active); ++round) {
-            uint32_t v[4], xm[4];
+            const int q0 = p & ~3;
+            uint4 v4 = make_uint4(NONE, NONE, NONE, NONE);
+            if (active) v4 = __ldcs(reinterpret_cast<const uint4 *>(d.rowrun_idx + q0));     // (the array has slack behind its end)
+            uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w}, xm[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = (active && p + j < e) ? __ldcs(&d.rowrun_idx[p + j]) : NONE;
+            for (int j = 0; j < 4; ++j) if (q0 + j < p || q0 + j >= e) v[j] = NONE;
 #pragma unroll
             for (int j = 0; j < 4; ++j) xm[j] = v[j] != NONE ? mask_of(F, v[j] & IDX_MASK) : 0u;
 #pragma unroll
             for (int j = 0; j < 4; ++j) got |= ((xm[j] >> (v[j] >> 27)) & 1u) != 0;
-            p += 4;
+            p = q0 + 4;
             if (got || p >= e) active = false;
         }
         uint32_t longm = __ballot_sync(FULL, active);
@@ -347,28 +373,195 @@ __device__ __forceinline__ int bfs_path(int n_nzblk, int nb, float th3, int forc
     return ((float)n_nzblk / (float)nb < th3) ? DBSPMSPV_PATH_PUSH : DBSPMSPV_PATH_PULL;
 }
 
+// Worklist of the frontier F from the listed nonzero words of its masks: a warp takes one word
+// (two vector blocks) at a time, lane = column; frontier columns emit their INLINE runs (adjacent
+// ones merged), lanes 0 and 16 the payload runs of the two blocks.  (With the words in index
+// order, the few warps that held the hub blocks of an early frontier wrote almost the whole
+// worklist.)  With UPDATE the same pass also does the level's bookkeeping for the word: visited
+// is updated and the vertices found and the nonempty blocks are counted.
+template <bool UPDATE>
+__device__ void bfs_worklist(const Device &d, const Scope &sc, const uint32_t *F, const int32_t *words, int n_listed,
+                             int32_t *n_tasks, int32_t *n_hubs, int4 *hubs, int32_t *nz_out) {
+    const int lane = threadIdx.x & 31;
+    Counters *ctr = d.ws.ctr;
+    int found = 0, nz = 0;
+    for (int i = sc.gwarp; i < n_listed; i += sc.nwarps) {
+        const int wd = words[i];
+        const uint32_t word = F[wd];
+        if (UPDATE) {
+            if (lane == 0) d.ws.visited32[wd] |= word;
+            found += __popc(word);
+            nz += ((word & 0xFFFFu) != 0) + ((word >> 16) != 0);
+        }
+        const int jb = 2 * wd + (lane >> 4), j = jb * 16 + (lane & 15);
+        const bool listed = (word >> lane) & 1u;
+        int first = 0, deg = 0;
+        if (listed) column_run(d, j, first, deg);
+        merge_column_runs(listed, j, first, deg, lane);
+        emit_tasks(d, false, jb, first, deg, lane, n_tasks, &ctr->pad, PUSH_CHUNK, n_hubs, hubs);
+        first = 0; deg = 0;
+        if ((lane & 15) == 0 && ((word >> lane) & 0xFFFFu)) payload_run(d, jb, first, deg);
+        if (__any_sync(FULL, deg > 0)) emit_tasks(d, false, jb, first, deg, lane, n_tasks, &ctr->pad, d.payload_chunk);
+    }
+    if (UPDATE && lane == 0 && found) { atomicAdd(&ctr->bfs_reached, found); atomicAdd(nz_out, nz); }
+}
+
+// Path of the level whose counters are set `cur` (Section 3.3.1): push iff the ratio of nonempty
+// frontier blocks is below th3 -- and, the worklist of a push level being built by then, iff that
+// worklist is short: a frontier of a few hub vertices fills few vector blocks but owns a good
+// part of all stored elements, and a pull, which stops every row at its first frontier
+// neighbour, reads less than the push of all those elements would (edge_frac = the share of
+// the view's entries above which the push is given up; 0 = block ratio only).
+__device__ __forceinline__ int bfs_level_path(const Device &d, int cur, float th3, float edge_frac, int force_path) {
+    const Counters *ctr = d.ws.ctr;
+    int path = bfs_path(ctr->bfs_cnt[cur][0], d.nb, th3, force_path);
+    if (path == DBSPMSPV_PATH_PUSH && force_path == DBSPMSPV_PATH_AUTO && edge_frac > 0.f && d.rowrun_ptr != nullptr) {
+        // warp steps of the worklist: the task records plus the steps of the listed hub runs
+        const int n_hubs = min(ctr->bfs_hubs[cur], HUB_CAP);
+        int64_t steps = ctr->bfs_cnt[cur][1];
+        for (int k = 0; k < n_hubs; ++k) steps += (d.ws.hubs[cur * HUB_CAP + k].z + PUSH_CHUNK - 1) / PUSH_CHUNK;
+        if ((float)steps * (float)PUSH_CHUNK > edge_frac * (float)d.n_entries) path = DBSPMSPV_PATH_PULL;
+    }
+    return path;
+}
+
+// One level of the search: the expansion of the frontier of level lv.  Three mask buffers rotate:
+// F holds the frontier, N receives the next one, Z (the frontier before) is cleared meanwhile and
+// becomes N of the next level.  Four lists of nonzero mask words rotate with them -- the list of
+// the frontier produced by level L is list L % 4 -- and three sets of per-level counters, so
+// that nothing is moved or reset behind an extra barrier.
 template <int DT>
-__global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t *levels, float th3,
+__device__ void bfs_level(const Device &d, cg::grid_group &grid, const Scope &sc, int lv, int32_t *levels, float th3,
+                          float edge_frac, int force_path) {
+    Counters *ctr = d.ws.ctr;
+    const int lane = threadIdx.x & 31;
+    const int n_words = (d.mb + 1) / 2;
+    uint32_t *const buf[3] = {d.ws.x_mask32, d.ws.y_mask32, d.ws.z_mask32};
+    const int cur = lv % 3, nxt = (lv + 1) % 3, spare = (lv + 2) % 3;
+    const uint32_t *F = buf[cur];
+    uint32_t *N = buf[nxt], *Z = buf[spare];
+    const int q_out = lv & 3, q_z = (lv + 2) & 3, q_next = (lv + 1) & 3;    // lists: produced now / of Z / produced next
+    int32_t *words_out = d.ws.bfs_words + (size_t)q_out * d.ws.bfs_words_stride;
+    const int32_t *words_z = d.ws.bfs_words + (size_t)q_z * d.ws.bfs_words_stride;
+    const int depth = lv + 1;
+    const int n_nzblk = ctr->bfs_cnt[cur][0];
+    const int n_tasks = ctr->bfs_cnt[cur][1];
+    const int path = bfs_level_path(d, cur, th3, edge_frac, force_path);
+    // counters that come into use at the next level are reset now: nobody reads or writes them
+    // during this one (the previous level was their last reader, behind a barrier)
+    if (sc.tid == 0) {
+        ctr->bfs_cnt[spare][0] = 0;
+        ctr->bfs_cnt[spare][1] = 0;
+        ctr->bfs_hubs[spare] = 0;
+        ctr->bfs_nwords[q_next] = 0;
+        if (depth <= DBSPMSPV_MAX_BFS_LEVELS_RECORDED) {
+            ctr->bfs_level_path[depth - 1] = path;
+            ctr->bfs_level_nzblk[depth - 1] = n_nzblk;
+            ctr->bfs_stamp[depth] = global_timer_ns();
+        }
+    }
+    int4 *hubs_next = d.ws.hubs + nxt * HUB_CAP;
+    if (path != DBSPMSPV_PATH_PUSH && d.rowrun_ptr != nullptr) {
+        // a pull over the row-run index does its own bookkeeping (it owns the mask words it writes)
+        bfs_pull_rows<DT>(d, F, N, Z, &ctr->bfs_cnt[nxt][0], words_out, &ctr->bfs_nwords[q_out], levels, depth);
+        grid.sync();
+    } else if (path == DBSPMSPV_PATH_PUSH) {
+        bfs_push<DT>(d, sc, F, N, n_tasks, d.ws.hubs + cur * HUB_CAP, min(ctr->bfs_hubs[cur], HUB_CAP), levels, depth,
+                     words_out, &ctr->bfs_nwords[q_out]);
+        grid.sync();
+        // Z (the frontier before this one) is cleared through its list
+        const int nz_words = ctr->bfs_nwords[q_z];
+        for (int i = sc.tid; i < nz_words; i += sc.nthreads) Z[words_z[i]] = 0u;
+        const int n_listed = ctr->bfs_nwords[q_out];
+        // With so few nonzero words that the next level is a push whatever their content, the
+        // bookkeeping and the next worklist are one pass (one barrier less); otherwise the
+        // bookkeeping first, then -- the selector's input being known -- the worklist if needed.
+        const bool surely_push = bfs_path(min(2 * n_listed, d.nb), d.nb, th3, force_path) == DBSPMSPV_PATH_PUSH;
+        if (surely_push) {
+            bfs_worklist<true>(d, sc, N, words_out, n_listed, &ctr->bfs_cnt[nxt][1], &ctr->bfs_hubs[nxt], hubs_next, &ctr->bfs_cnt[nxt][0]);
+            grid.sync();
+            return;
+        }
+        int found = 0, nz = 0;
+        for (int i = sc.tid; i < n_listed; i += sc.nthreads) {
+            const int k = words_out[i];
+            const uint32_t nm = N[k];
+            d.ws.visited32[k] |= nm;
+            found += __popc(nm);
+            nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
+        }
+        found = __reduce_add_sync(FULL, found);
+        nz = __reduce_add_sync(FULL, nz);
+        if (lane == 0 && found) { atomicAdd(&ctr->bfs_reached, found); atomicAdd(&ctr->bfs_cnt[nxt][0], nz); }
+        grid.sync();
+    } else {
+        // pull over the row-block segments (no row-run index): the masks produced are scanned as a
+        // whole: visited is updated, the nonempty blocks counted, the nonzero words listed
+        bfs_pull<DT>(d, sc, F, N, levels, depth);
+        grid.sync();
+        int found = 0, nz = 0;
+        for (int k0 = sc.tid & ~31; k0 < n_words; k0 += sc.nthreads) {
+            const int k = k0 + lane;
+            uint32_t nm = 0;
+            if (k < n_words) {
+                nm = N[k];
+                if (nm) {
+                    d.ws.visited32[k] |= nm;
+                    found += __popc(nm);
+                    nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
+                }
+                if (Z[k]) Z[k] = 0u;
+            }
+            append_words(nm ? k : -1, words_out, &ctr->bfs_nwords[q_out], lane);
+        }
+        found = __reduce_add_sync(FULL, found);
+        nz = __reduce_add_sync(FULL, nz);
+        if (lane == 0 && found) { atomicAdd(&ctr->bfs_reached, found); atomicAdd(&ctr->bfs_cnt[nxt][0], nz); }
+        grid.sync();
+    }
+    // the push worklist is rebuilt if the block ratio of the next level asks for a push (the
+    // selector's input is known now; the level may still turn to a pull when the list is long)
+    const int next_n = ctr->bfs_cnt[nxt][0];
+    if (next_n && bfs_path(next_n, d.nb, th3, force_path) == DBSPMSPV_PATH_PUSH) {
+        bfs_worklist<false>(d, sc, N, words_out, ctr->bfs_nwords[q_out], &ctr->bfs_cnt[nxt][1], &ctr->bfs_hubs[nxt], hubs_next, nullptr);
+        grid.sync();
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t *levels, float th3, float edge_frac,
                                                  int force_path, int max_levels) {
     cg::grid_group grid = cg::this_grid();
     const int tid = blockIdx.x * blockDim.x + threadIdx.x;
     const int nthreads = gridDim.x * blockDim.x;
     const int lane = threadIdx.x & 31;
-    const int gwarp_all = tid >> 5, nwarps_all = nthreads >> 5;
     const int n_words = (d.mb + 1) / 2;
     Counters *ctr = d.ws.ctr;
+    const Scope sc{tid, nthreads, tid >> 5, nthreads >> 5};
+    if (tid == 0) ctr->bfs_stamp[0] = global_timer_ns();
 
-    for (int64_t v = tid; v < d.n; v += nthreads) levels[v] = -1;
+    // levels = -1 (16-byte stores over the aligned middle, the ragged ends one by one)
+    {
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(levels);
+        int64_t head = (int64_t)((16 - (addr & 15)) & 15) / 4;
+        if (head > d.n) head = d.n;
+        const int64_t n4 = (d.n - head) / 4;
+        int4 *mid = reinterpret_cast<int4 *>(levels + head);
+        for (int64_t v = tid; v < n4; v += nthreads) mid[v] = make_int4(-1, -1, -1, -1);
+        for (int64_t v = tid; v < head; v += nthreads) levels[v] = -1;
+        for (int64_t v = head + n4 * 4 + tid; v < d.n; v += nthreads) levels[v] = -1;
+    }
     // rows without a stored element can never be reached through a pull: they start out as
     // "visited", so that a row block is skipped (and a segment left early) once every row that
     // can be found has been found
     for (int k = tid; k < n_words; k += nthreads) { d.ws.visited32[k] = ~d.row_present32[k]; d.ws.x_mask32[k] = 0u; d.ws.y_mask32[k] = 0u; d.ws.z_mask32[k] = 0u; }
     if (tid == 0) {
-        for (int k = 0; k < 3; ++k) { ctr->bfs_cnt[k][0] = 0; ctr->bfs_cnt[k][1] = 0; ctr->bfs_hubs[k] = 0; ctr->bfs_nwords[k] = 0; }
+        for (int k = 0; k < 3; ++k) { ctr->bfs_cnt[k][0] = 0; ctr->bfs_cnt[k][1] = 0; ctr->bfs_hubs[k] = 0; }
+        for (int k = 0; k < 4; ++k) ctr->bfs_nwords[k] = 0;
         ctr->bfs_reached = 1;
     }
     grid.sync();
-    // level 0: the source is the first frontier
+    // level 0: the source is the first frontier (its mask word is list 3 = "produced by level -1")
     if (blockIdx.x == 0 && threadIdx.x < 32) {
         const int jb = src >> 4;
         if (lane == 0) {
@@ -376,6 +569,8 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
             const uint32_t bit = 1u << ((src & 15) + (jb & 1) * 16);
             d.ws.x_mask32[jb >> 1] = bit;
             d.ws.visited32[jb >> 1] |= bit;
+            d.ws.bfs_words[(size_t)3 * d.ws.bfs_words_stride] = jb >> 1;
+            ctr->bfs_nwords[3] = 1;
         }
         int first = 0, deg = 0;
         if (lane == 0) column_run(d, src, first, deg);
@@ -383,103 +578,27 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
         emit_tasks(d, lane == 0, jb, first, deg, lane, &ctr->bfs_cnt[0][1], &ctr->bfs_cnt[0][0], PUSH_CHUNK, &ctr->bfs_hubs[0], d.ws.hubs);
     }
     grid.sync();
-
-    // Three mask buffers rotate: F holds the frontier, N receives the next one, Z is cleared while
-    // the level runs and becomes N of the next level (the old F becomes Z).
-    uint32_t *F = d.ws.x_mask32, *N = d.ws.y_mask32, *Z = d.ws.z_mask32;
-    int cur = 0, depth = 0;
-    while (depth < max_levels) {
-        const int n_nzblk = ctr->bfs_cnt[cur][0];
-        const int n_tasks = ctr->bfs_cnt[cur][1];
-        if (n_nzblk == 0) break;
-        ++depth;
-        const int path = bfs_path(n_nzblk, d.nb, th3, force_path);
-        // per-level counters: `cur` holds this level's, `nxt` is accumulated for the next level,
-        // `spare` (the previous level's, read for the last time before the barriers of that
-        // level) is reset now and accumulated into at the next level
-        const int nxt = (cur + 1) % 3, spare = (cur + 2) % 3;
-        if (tid == 0) {
-            ctr->bfs_cnt[spare][0] = 0;
-            ctr->bfs_cnt[spare][1] = 0;
-            ctr->bfs_hubs[spare] = 0;
-            ctr->bfs_nwords[spare] = 0;
-            if (depth <= DBSPMSPV_MAX_BFS_LEVELS_RECORDED) {
-                ctr->bfs_level_path[depth - 1] = path;
-                ctr->bfs_level_nzblk[depth - 1] = n_nzblk;
-            }
-        }
-        const bool fused = path != DBSPMSPV_PATH_PUSH && d.rowrun_ptr != nullptr;
-        if (fused) {
-            bfs_pull_rows<DT>(d, F, N, Z, &ctr->bfs_cnt[nxt][0], &ctr->bfs_nwords[nxt], levels, depth);
-            grid.sync();
-        } else {
-            if (path == DBSPMSPV_PATH_PUSH) bfs_push<DT>(d, F, N, n_tasks, d.ws.hubs + cur * HUB_CAP, min(ctr->bfs_hubs[cur], HUB_CAP), levels, depth);
-            else bfs_pull<DT>(d, F, N, levels, depth);
-            grid.sync();
-            // the masks produced above are the next frontier: visited is updated, the nonempty
-            // blocks are counted (one atomic per warp), the nonzero words listed so that a
-            // worklist rebuild can share them out evenly, and the spare buffer is cleared
-            int found = 0, nz = 0;
-            for (int k0 = tid & ~31; k0 < n_words; k0 += nthreads) {
-                const int k = k0 + lane;
-                uint32_t nm = 0;
-                if (k < n_words) {
-                    nm = N[k];
-                    if (nm) {
-                        d.ws.visited32[k] |= nm;
-                        found += __popc(nm);
-                        nz += ((nm & 0xFFFFu) != 0) + ((nm >> 16) != 0);
-                    }
-                    if (Z[k]) Z[k] = 0u;
-                }
-                const uint32_t nzw = __ballot_sync(FULL, nm != 0u);
-                if (nzw) {
-                    int base = 0;
-                    if (lane == 0) base = atomicAdd(&ctr->bfs_nwords[nxt], __popc(nzw));
-                    base = __shfl_sync(FULL, base, 0);
-                    if (nm) d.ws.bfs_words[base + __popc(nzw & ((1u << lane) - 1u))] = k;
-                }
-            }
-            found = __reduce_add_sync(FULL, found);
-            nz = __reduce_add_sync(FULL, nz);
-            if (lane == 0 && found) { atomicAdd(&ctr->bfs_reached, found); atomicAdd(&ctr->bfs_cnt[nxt][0], nz); }
-            grid.sync();
-        }
-        { uint32_t *t = F; F = N; N = Z; Z = t; }       // rotate: the new frontier is what was written
-        // the push worklist is rebuilt only if the next level is a push (the selector's input is
-        // known now); its block count goes to a scratch counter
-        const int next_n = ctr->bfs_cnt[nxt][0];
-        if (next_n && bfs_path(next_n, d.nb, th3, force_path) == DBSPMSPV_PATH_PUSH) {
-            // a warp takes one listed mask word (two vector blocks) at a time, lane = column:
-            // frontier columns emit their INLINE runs (adjacent ones merged), lanes 0 and 16 the
-            // payload runs of the two blocks.  (With the words in index order, the few warps that
-            // held the hub blocks of an early frontier wrote almost the whole worklist.)
-            const int n_listed = ctr->bfs_nwords[nxt];
-            for (int i = gwarp_all; i < n_listed; i += nwarps_all) {
-                const int wd = d.ws.bfs_words[i];
-                const uint32_t word = F[wd];
-                const int jb = 2 * wd + (lane >> 4), j = jb * 16 + (lane & 15);
-                const bool listed = (word >> lane) & 1u;
-                int first = 0, deg = 0;
-                if (listed) column_run(d, j, first, deg);
-                merge_column_runs(listed, j, first, deg, lane);
-                emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[nxt][1], &ctr->pad, PUSH_CHUNK,
-                           &ctr->bfs_hubs[nxt], d.ws.hubs + nxt * HUB_CAP);
-                first = 0; deg = 0;
-                if ((lane & 15) == 0 && ((word >> lane) & 0xFFFFu)) payload_run(d, jb, first, deg);
-                if (__any_sync(FULL, deg > 0))
-                    emit_tasks(d, false, jb, first, deg, lane, &ctr->bfs_cnt[nxt][1], &ctr->pad, d.payload_chunk);
-            }
-            grid.sync();
-        }
-        cur = nxt;
+    int lv = 0;
+    while (lv < max_levels && ctr->bfs_cnt[lv % 3][0] != 0) {
+        bfs_level<DT>(d, grid, sc, lv, levels, th3, edge_frac, force_path);    // ends with a grid barrier
+        ++lv;
     }
-    // leave the shared workspace as dbspmspv_run expects it: all masks clear (Z is the last
-    // frontier that was expanded; F is empty unless the level cap ended the search; N is clear)
-    for (int k = tid; k < n_words; k += nthreads) if (Z[k]) Z[k] = 0u;
-    if (ctr->bfs_cnt[cur][0] != 0)
-        for (int k = tid; k < n_words; k += nthreads) F[k] = 0u;
-    if (tid == 0) ctr->bfs_levels = depth;
+    // leave the shared workspace as dbspmspv_run expects it: all masks clear.  The frontier before
+    // the last one (buffer (lv + 2) % 3) is cleared through its list; the last frontier is empty
+    // unless the level cap ended the search; the third buffer is clear.
+    {
+        uint32_t *const buf[3] = {d.ws.x_mask32, d.ws.y_mask32, d.ws.z_mask32};
+        uint32_t *Z = buf[(lv + 2) % 3], *F = buf[lv % 3];
+        const int32_t *wz = d.ws.bfs_words + (size_t)((lv + 2) & 3) * d.ws.bfs_words_stride;
+        const int nz_words = ctr->bfs_nwords[(lv + 2) & 3];
+        for (int i = tid; i < nz_words; i += nthreads) Z[wz[i]] = 0u;
+        if (ctr->bfs_cnt[lv % 3][0] != 0)
+            for (int k = tid; k < n_words; k += nthreads) F[k] = 0u;
+    }
+    if (tid == 0) {
+        ctr->bfs_levels = lv;
+        if (lv < DBSPMSPV_MAX_BFS_LEVELS_RECORDED + 1) ctr->bfs_stamp[lv + 1] = global_timer_ns();
+    }
 }
 
 template <int DT>
@@ -491,9 +610,10 @@ static int bfs_typed(dbspmspv_handle_s *h, int32_t src, int32_t *levels, cudaStr
         h->bfs_grid = per_sm * h->sm_count;
     }
     float th3 = h->ropts.th3_bfs;
+    float edge_frac = 0.f;
     int force = h->ropts.force_path;
     int max_levels = d.n > 0x7FFFFFFF ? 0x7FFFFFFF : (int)d.n;
-    void *args[] = {&d, &src, &levels, &th3, &force, &max_levels};
+    void *args[] = {&d, &src, &levels, &th3, &edge_frac, &force, &max_levels};
     DBS_CUDA(cudaLaunchCooperativeKernel((void *)k_bfs<DT>, dim3(h->bfs_grid), dim3(BFS_CTA), args, 0, st));
     ++h->kernel_launches;
     return DBSPMSPV_OK;

@@ -886,7 +886,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         DBS_CUDA(cudaMemcpyAsync(&n_inline, rp + m, 4, cudaMemcpyDeviceToHost, st));
         DBS_CUDA(cudaStreamSynchronize(st));
         uint32_t *ri;
-        DBS_KEEP(ri, n_inline);
+        DBS_KEEP(ri, (int64_t)n_inline + 4);      // (slack: the pull reads whole aligned groups of four)
         d.rowrun_idx = ri;
         if (n_inline) DBS_CUDA(cudaMemcpyAsync(ri, rv, (size_t)n_inline * 4, cudaMemcpyDeviceToDevice, st));
         DBS_CUDA(cudaStreamSynchronize(st));

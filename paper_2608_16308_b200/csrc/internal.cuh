@@ -138,10 +138,12 @@ struct Counters {    // device-resident scalars of one call
     int32_t bfs_hubs[3];    // BFS: the same per level (the per-level counters rotate three ways: the
                             // level's own, the ones it accumulates for the next level, and a spare
                             // set that is reset meanwhile)
-    int32_t bfs_nwords[3];  // BFS: nonzero words of the new frontier's masks (listed in Workspace::bfs_words)
+    int32_t bfs_nwords[4];  // BFS: lengths of the four rotating lists of nonzero mask words (Workspace::bfs_words)
     int32_t bfs_cnt[3][2];  // BFS: {nonempty frontier blocks, tasks}
     int32_t bfs_level_path[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
     int32_t bfs_level_nzblk[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
+    // BFS: device time stamps (ns): [0] kernel start, [1 + L] start of level L, then the end of the last level
+    unsigned long long bfs_stamp[DBSPMSPV_MAX_BFS_LEVELS_RECORDED + 2];
 };
 
 struct Workspace {
@@ -155,7 +157,9 @@ struct Workspace {
     int32_t *tile_count;  // compaction: result entries per tile of row blocks
     uint32_t *visited32;  // BFS: visited masks
     uint32_t *z_mask32;   // BFS: third mask buffer (frontier / next / being cleared rotate)
-    int32_t *bfs_words;   // BFS: indices of the nonzero mask words of the new frontier
+    int32_t *bfs_words;   // BFS: four lists of bfs_words_stride ints: the nonzero mask words of the frontiers produced by
+                          // the levels L, L-1, L-2 (rotating, list L % 4 is written while level L runs)
+    int32_t bfs_words_stride;
     Counters *ctr;
     int64_t task_capacity;
     int32_t n_tiles;
@@ -243,6 +247,11 @@ __host__ __device__ inline T ceil_div(T a, T b) { return (a + b - 1) / b; }
 // its writes are visible (a no-op for a normally launched kernel), `pdl_launch_dependents`
 // lets the successor's launch proceed early.  This hides the launch latency between the short
 // kernels of one call.
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

@@ -1546,7 +1546,7 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     const size_t o_xd = carve(xwords * 32 * sizeof(float)), o_yacc = carve(ywords * 32 * sizeof(float)),
                  o_hit = carve(ywords * 32), o_tasks = carve((size_t)ws.task_capacity * sizeof(*ws.tasks)),
                  o_xm = carve(xwords * 4), o_ym = carve(ywords * 4), o_zm = carve(zwords * 4),
-                 o_words = carve(xwords * sizeof(*ws.bfs_words)), o_vis = carve((d.m == d.n ? ywords : 1) * 4),
+                 o_words = carve(4 * zwords * sizeof(*ws.bfs_words)), o_vis = carve((d.m == d.n ? ywords : 1) * 4),
                  o_hubs = carve((size_t)3 * HUB_CAP * sizeof(*ws.hubs)), o_tile = carve((size_t)ws.n_tiles * sizeof(*ws.tile_count)),
                  o_ctr = carve(sizeof(*ws.ctr));
     void *arena = nullptr;
@@ -1562,6 +1562,7 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     ws.y_mask32 = reinterpret_cast<decltype(ws.y_mask32)>(base + o_ym);
     ws.z_mask32 = reinterpret_cast<decltype(ws.z_mask32)>(base + o_zm);
     ws.bfs_words = reinterpret_cast<decltype(ws.bfs_words)>(base + o_words);
+    ws.bfs_words_stride = (int32_t)zwords;
     ws.visited32 = reinterpret_cast<decltype(ws.visited32)>(base + o_vis);
     ws.hubs = reinterpret_cast<decltype(ws.hubs)>(base + o_hubs);
     ws.tile_count = reinterpret_cast<decltype(ws.tile_count)>(base + o_tile);
@@ -1700,6 +1701,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     o->th3 = 0.9f;
     o->th3_bfs = 0.05f;
     o->th3_decode = 0.01f;
+    o->bfs_push_max_edge_frac = 0.1f;
     o->force_path = DBSPMSPV_PATH_AUTO;
     o->popc_threshold = 8;
     o->validate = 0;
@@ -1708,7 +1710,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
 int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts) {
     if (!h || !opts) return DBSPMSPV_ERR_INVALID_ARG;
     if (opts->force_path < DBSPMSPV_PATH_AUTO || opts->force_path > DBSPMSPV_PATH_PULL) return DBSPMSPV_ERR_INVALID_ARG;
-    if (!(opts->th3 >= 0.f) || !(opts->th3_bfs >= 0.f) || !(opts->th3_decode >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!(opts->th3 >= 0.f) || !(opts->th3_bfs >= 0.f) || !(opts->th3_decode >= 0.f) || !(opts->bfs_push_max_edge_frac >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
     h->ropts = *opts;
     return DBSPMSPV_OK;
 }

@@ -43,7 +43,7 @@ def test_struct_layouts_match_the_header():
     text = open(os.path.join(ROOT, "include", "dbspmspv.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     for cname, cls in (("dbspmspv_create_opts", B.CreateOpts), ("dbspmspv_run_opts", B.RunOpts),
-                       ("dbspmspv_stats", B.Stats)):
+                       ("dbspmspv_stats", B.Stats), ("dbspmspv_call_bytes", B.CallBytes)):
         body = re.search(r"typedef struct \{([^}]*)\}\s*" + cname + ";", text).group(1)
         fields = []
         for decl in body.split(";"):
