@@ -124,10 +124,14 @@ typedef struct {
                                 kernels of dbspmspv_run                              (0)    */
     float bfs_push_max_edge_frac; /* db_bfs (with the row-run index): a level whose push worklist
                                 covers more than this share of the view's entries is pulled
-                                even when the block ratio says push -- a frontier of a few hub
-                                vertices fills few vector blocks but owns many elements.
-                                0 = block ratio only.  Default measured on B200             */
-    int32_t reserved[7];
+                                even when the block ratio says push.  0 = block ratio only,
+                                the paper's rule and the default: on the R-MAT scale 22 graph
+                                the one level this moved to the pull (a frontier of hub
+                                vertices) took 389 us instead of 66                        */
+    int32_t hub_min_nnz_x;   /* dbspmspv_run: shortest x list for which the push adds into the
+                                private accumulators of hub row blocks (they cost one more
+                                kernel in the chain); 0 = default (32768), < 0 = never     */
+    int32_t reserved[6];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64
@@ -144,7 +148,8 @@ typedef struct {
     int64_t n_segments;            /* pull segments                                           */
     int64_t payload_bytes;         /* the single block payload                                */
     int64_t csr_view_bytes;        /* block-CSR view: row pointers + per-block entries        */
-    int64_t csc_view_bytes;        /* block-CSC view: column pointers + per-block entries     */
+    int64_t csc_view_bytes;        /* block-CSC view: column pointers + per-block entries (+ the
+                                      slot table and private accumulators of hub row blocks)  */
     int64_t segment_bytes;
     int64_t workspace_bytes;       /* per-call scratch owned by the handle                    */
     /* last dbspmspv_run / dbspmspv_decode */
@@ -169,7 +174,7 @@ typedef struct {
        (initialisation of levels and masks) and per level (traversal + frontier bookkeeping)    */
     float bfs_setup_us;
     float bfs_level_us[DBSPMSPV_MAX_BFS_LEVELS_RECORDED];
-    int32_t reserved[1];
+    int32_t n_hub_row_blocks;      /* row blocks with private push accumulators (0: none)     */
 } dbspmspv_stats;
 
 /* Paper thresholds (th0 = 32, th1 = 128, th2 = 2.0, Section 3.2.1).  The segment weights keep

@@ -47,7 +47,8 @@ class RunOpts(ctypes.Structure):
                 ("popc_threshold", ctypes.c_int32), ("validate", ctypes.c_int32),
                 ("timing", ctypes.c_int32), ("th3_bfs", ctypes.c_float),
                 ("th3_decode", ctypes.c_float), ("no_fused_decode", ctypes.c_int32),
-                ("bfs_push_max_edge_frac", ctypes.c_float), ("reserved", ctypes.c_int32 * 7)]
+                ("bfs_push_max_edge_frac", ctypes.c_float), ("hub_min_nnz_x", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 6)]
 
 
 class Stats(ctypes.Structure):
@@ -66,7 +67,7 @@ class Stats(ctypes.Structure):
                 ("device_status", ctypes.c_int32), ("last_compute_ms", ctypes.c_float),
                 ("kernel_launches", ctypes.c_int64), ("bfs_index_bytes", ctypes.c_int64),
                 ("lean_index_bytes", ctypes.c_int64), ("bfs_setup_us", ctypes.c_float),
-                ("bfs_level_us", ctypes.c_float * MAX_BFS_LEVELS_RECORDED), ("reserved", ctypes.c_int32 * 1)]
+                ("bfs_level_us", ctypes.c_float * MAX_BFS_LEVELS_RECORDED), ("n_hub_row_blocks", ctypes.c_int32)]
 
 
 class CallBytes(ctypes.Structure):

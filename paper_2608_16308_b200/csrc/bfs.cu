@@ -610,7 +610,7 @@ static int bfs_typed(dbspmspv_handle_s *h, int32_t src, int32_t *levels, cudaStr
         h->bfs_grid = per_sm * h->sm_count;
     }
     float th3 = h->ropts.th3_bfs;
-    float edge_frac = 0.f;
+    float edge_frac = h->ropts.bfs_push_max_edge_frac;
     int force = h->ropts.force_path;
     int max_levels = d.n > 0x7FFFFFFF ? 0x7FFFFFFF : (int)d.n;
     void *args[] = {&d, &src, &levels, &th3, &edge_frac, &force, &max_levels};

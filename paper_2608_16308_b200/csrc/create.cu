@@ -4,6 +4,7 @@
 // Radix sort and prefix sums are CUB library primitives; everything else is written here.
 #include <cub/cub.cuh>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -459,12 +460,14 @@ __global__ void k_csc_colptr(int32_t nb, const uint64_t *keys_sorted, int32_t n,
 __global__ void k_csc_gather(int32_t n_blocks, const uint64_t *keys_sorted,
                              const int32_t *csc2csr, const uint32_t *csr_idx,
                              const uint32_t *csr_w, const uint8_t *csr_aux, uint32_t *csc_idx,
-                             uint32_t *csc_w, uint8_t *csc_aux, int32_t *bcol_sorted) {
+                             uint32_t *csc_w, uint8_t *csc_aux, int32_t *bcol_sorted, const uint16_t *hub_slot) {
     int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (p >= n_blocks) return;
     int32_t b = csc2csr[p];
     uint64_t k = keys_sorted[p];
-    csc_idx[p] = (uint32_t)((k >> 4) & IDX_MASK) | (csr_idx[b] & (7u << TYPE_SHIFT));   // class, without the CSR view's flags
+    const uint32_t rb = (uint32_t)((k >> 4) & IDX_MASK), cls = csr_idx[b] & (7u << TYPE_SHIFT);   // class, without the CSR view's flags
+    const bool hub = hub_slot && (cls >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE && hub_slot[rb] != HUB_NONE;
+    csc_idx[p] = rb | cls | (hub ? HUB_FLAG : 0u);
     csc_w[p] = csr_w[b];
     csc_aux[p] = csr_aux[b];
     bcol_sorted[p] = (int32_t)(k >> CSC_KEY_COL_SHIFT);
@@ -849,6 +852,39 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         tp.release(k1); tp.release(k1_alt); tp.release(ids); tp.release(ids_alt);
     }
 
+    // Hub row blocks: the (at most HUB_BLOCKS_MAX) row blocks with the most view entries, if
+    // they hold HUB_BLOCK_MIN_ENTRIES or more.  Chosen on the host from the row block pointers.
+    d.hub_slot = nullptr; d.hub_rb = nullptr; d.hub_acc = nullptr; d.n_hub_blocks = 0; d.hub_on = 0;
+    if (d.mb > 0 && n_entries >= HUB_BLOCK_MIN_ENTRIES) {
+        std::vector<int32_t> ptr((size_t)d.mb + 1);
+        DBS_CUDA(cudaMemcpyAsync(ptr.data(), d.csr.ptr, ((size_t)d.mb + 1) * 4, cudaMemcpyDeviceToHost, st));
+        DBS_CUDA(cudaStreamSynchronize(st));
+        std::vector<int32_t> big;
+        for (int32_t rb = 0; rb < d.mb; ++rb)
+            if (ptr[rb + 1] - ptr[rb] >= HUB_BLOCK_MIN_ENTRIES) big.push_back(rb);
+        auto deg = [&](int32_t rb) { return ptr[rb + 1] - ptr[rb]; };
+        auto heavier = [&](int32_t a, int32_t b) { return deg(a) != deg(b) ? deg(a) > deg(b) : a < b; };
+        if ((int)big.size() > HUB_BLOCKS_MAX) {
+            std::nth_element(big.begin(), big.begin() + HUB_BLOCKS_MAX, big.end(), heavier);
+            big.resize(HUB_BLOCKS_MAX);
+        }
+        std::sort(big.begin(), big.end(), heavier);
+        if (!big.empty()) {
+            std::vector<uint16_t> slot((size_t)d.mb + 2, HUB_NONE);     // padded: read two at a time
+            for (size_t k = 0; k < big.size(); ++k) slot[big[k]] = (uint16_t)k;
+            uint16_t *hs; float *ha; int32_t *hr;
+            DBS_KEEP(hr, big.size());
+            DBS_CUDA(cudaMemcpyAsync(hr, big.data(), big.size() * 4, cudaMemcpyHostToDevice, st));
+            const int64_t n_acc = (int64_t)HUB_COPIES * (int64_t)big.size() * 16;
+            DBS_KEEP(hs, (int64_t)d.mb + 2); DBS_KEEP(ha, n_acc);
+            DBS_CUDA(cudaMemcpyAsync(hs, slot.data(), ((size_t)d.mb + 2) * 2, cudaMemcpyHostToDevice, st));
+            k_fill_words<<<grid_for(n_acc), TPB, 0, st>>>(reinterpret_cast<uint32_t *>(ha), n_acc, HUB_CLEAR);
+            DBS_CUDA(cudaStreamSynchronize(st));
+            d.hub_slot = hs; d.hub_rb = hr; d.hub_acc = ha; d.n_hub_blocks = (int32_t)big.size();
+            h->hub_bytes = ((int64_t)d.mb + 2) * 2 + (int64_t)big.size() * 4 + n_acc * 4;
+        }
+    }
+
     // block-CSC view: sort the primary entries by column block, and inside it payload entries
     // first (by row block), then the INLINE elements column by column
     {
@@ -860,7 +896,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
             k_csc_keys<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, h->block_row, d.csr.idx, d.csr.aux, k2, ids);
             DBS_TRY(sort_pairs(tp, k2, k2_alt, ids, ids_alt, (int64_t)n_entries, CSC_KEY_COL_SHIFT + bits_for((uint64_t)d.nb), st));
             DBS_CUDA(cudaMemcpyAsync(h->csc2csr, ids, (size_t)n_entries * 4, cudaMemcpyDeviceToDevice, st));
-            k_csc_gather<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, k2, h->csc2csr, d.csr.idx, d.csr.w, d.csr.aux, d.csc.idx, d.csc.w, d.csc.aux, bcol_sorted);
+            k_csc_gather<<<grid_for(n_entries), TPB, 0, st>>>(n_entries, k2, h->csc2csr, d.csr.idx, d.csr.w, d.csr.aux, d.csc.idx, d.csc.w, d.csc.aux, bcol_sorted, d.hub_slot);
         }
         k_lower_bounds<<<grid_for(d.nb + 1), TPB, 0, st>>>(d.nb, bcol_sorted, n_entries, d.csc.ptr);
         k_csc_colptr<<<grid_for((int64_t)d.nb * 17), TPB, 0, st>>>(d.nb, k2, n_entries, d.csc.colptr);
@@ -973,10 +1009,11 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     s.payload_bytes = h->payload_bytes;
     s.n_view_entries = d.n_entries;
     s.csr_view_bytes = ((int64_t)d.mb + 1) * 8 + (int64_t)d.n_entries * 9;
-    s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.nb * 17 * 4 + (int64_t)d.n_entries * 9;
+    s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.nb * 17 * 4 + (int64_t)d.n_entries * 9 + h->hub_bytes;
     s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment) + ((int64_t)d.n_chunks + 1) * 8 + (int64_t)d.n_segments * 4;
     s.bfs_index_bytes = h->bfs_index_bytes;
     s.lean_index_bytes = h->lean_index_bytes;
+    s.n_hub_row_blocks = d.n_hub_blocks;
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }

@@ -16,7 +16,8 @@ namespace dbs {
 // A "view" is three parallel arrays with one entry per nonempty block:
 //   idx[p]  bits 0..26  the block's index along the *other* dimension (column block in the
 //                       block-CSR view, row block in the block-CSC view)
-//           bit  27     block-CSR view only: first INLINE element of its row (ROW_FLAG)
+//           bit  27     block-CSR view: first INLINE element of its row (ROW_FLAG);
+//                       block-CSC view: INLINE element of a hub row block (HUB_FLAG)
 //           bit  28     block-CSR view only: first entry of a pull segment
 //           bits 29..31 block class (DBSPMSPV_BLK_*)
 //   w[p]    payload offset in 4-byte words -- or, for INLINE entries, the stored value itself
@@ -57,6 +58,25 @@ __host__ __device__ inline int public_class(int type) { return type == BLK_CSR_R
 constexpr uint32_t IDX_MASK = 0x07FFFFFFu;  // 27 bits
 constexpr int TYPE_SHIFT = 29;
 constexpr uint32_t ROW_FLAG = 1u << 27;     // block-CSR view: first INLINE element of its row
+// Hub row blocks: the few row blocks that hold a large share of a power-law matrix.  Atomics on
+// one line are served one after the other by the L2 slice that owns it, so the push gives
+// every hub row block HUB_COPIES private accumulators (Device::hub_acc); the compaction folds them.
+constexpr uint32_t HUB_FLAG = 1u << 27;     // block-CSC view: INLINE element whose row block is a hub
+#ifndef DBS_HUB_COPIES
+#define DBS_HUB_COPIES 16
+#endif
+#ifndef DBS_HUB_BLOCKS_MAX
+#define DBS_HUB_BLOCKS_MAX 256
+#endif
+#ifndef DBS_HUB_MIN_ENTRIES
+#define DBS_HUB_MIN_ENTRIES 4096
+#endif
+constexpr int HUB_COPIES = DBS_HUB_COPIES;              // private accumulator copies per hub row block (power of two)
+constexpr int HUB_BLOCKS_MAX = DBS_HUB_BLOCKS_MAX;      // hub row blocks per handle, at most
+constexpr int HUB_BLOCK_MIN_ENTRIES = DBS_HUB_MIN_ENTRIES; // view entries that make a row block a hub
+constexpr uint16_t HUB_NONE = 0xFFFFu;
+constexpr int HUB_MIN_NNZ_X = 32768;        // shorter x: too few products for a queue, and the fold kernel is one more step in the chain
+constexpr uint32_t HUB_CLEAR = 0x80000000u; // an untouched private accumulator: -0.0f (see push_private)
 constexpr uint32_t PAD_IDX = 7u << TYPE_SHIFT;   // class code of the slack behind the last view entry: no kernel acts on it
 // The streaming pull of hypersparse handles takes the block-CSR view in chunks of LEAN_CHUNK
 // entries, one chunk (eight entries per lane) per warp pass.
@@ -197,6 +217,15 @@ struct Device {           // everything the kernels need, passed by value
     int32_t n_lean_chunks;
     int32_t n_lean_rows;
     int32_t n_payload;
+    // Hub row blocks (null / 0 when the matrix has none): hub_slot[rb] = slot of row block rb or
+    // HUB_NONE; hub_acc[(copy * n_hub_blocks + slot) * 16 + row] = private accumulators, all
+    // HUB_CLEAR between calls.
+    // hub_rb[slot] = the row block; hub_on: this call's push uses them (set per call by the host).
+    const uint16_t *hub_slot;
+    const int32_t *hub_rb;
+    float *hub_acc;
+    int32_t n_hub_blocks;
+    int32_t hub_on;
     const uint32_t *row_present32;  // per row block: rows that hold a stored element (two 16-bit masks per word)
     Workspace ws;
 };
@@ -227,6 +256,7 @@ struct dbspmspv_handle_s {
     int64_t kernel_launches;    // kernels this handle has launched (run / decode / bfs)
     int64_t bfs_index_bytes;
     int64_t lean_index_bytes;
+    int64_t hub_bytes;
     void *ws_arena;             // the one allocation that holds the whole workspace
     cudaStream_t last_stream;   // stream of the last run / decode / bfs call (get_stats waits on it)
 };

@@ -278,6 +278,24 @@ __device__ __forceinline__ void flush_rows(Out out, int rb, uint32_t hits, float
     }
 }
 
+// One product of an INLINE element whose row block is a hub (HUB_FLAG): added to one of the
+// HUB_COPIES private accumulators of that row block, picked by the CTA, with an atomic whose
+// reply nobody reads.  The L2 serves atomics on one line one after the other: on an R-MAT
+// matrix one line of the accumulator receives 1-2 % of ALL products, and that queue, not the
+// traversal, set the duration of the push (58 -> 35 us at 10 % x density when the same atomics
+// go to distinct lines).  A private accumulator that nothing touched holds -0.0f: any sum of
+// finite products that are neither zero nor subnormal differs from it in its bits (x + -x is
+// +0 in round-to-nearest), so the fold of the compaction needs no flags.  Products that are
+// zero or subnormal (an atomic may flush them to a signed zero) return false and take the
+// ordinary path.
+template <typename Out>
+__device__ __forceinline__ bool push_private(const Device &d, uint32_t idx, uint32_t aux, float prod) {
+    if (!Out::MASKS || !d.hub_on || !(idx & HUB_FLAG) || !(fabsf(prod) >= 1.17549435e-38f)) return false;
+    const int slot = d.hub_slot[idx & IDX_MASK];
+    atomicAdd(d.hub_acc + (((size_t)(blockIdx.x & (HUB_COPIES - 1)) * d.n_hub_blocks + slot) * 16 + (aux >> 4)), prod);
+    return true;
+}
+
 // Push (Section 3.3.2): every warp takes one task = up to PUSH_CHUNK consecutive block-CSC
 // entries of one active column block (32 per step, all fetched up front); the vector block is staged once per task (Section 3.3.3).  Lanes
 // own hypersparse blocks; heavier blocks are then processed by the whole warp one at a time.
@@ -347,10 +365,10 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                     // unconditional store: on the stencil the returning atomic cost 7-15 %.)
                     bool first = false;
                     const uint32_t hit = lane_block<DT>(type, w[u], aux[u], xm, s_x[aux[u] & 15], s_x, d.payload,
-                                                        [&](int r, float v) { first |= atomicAdd(row0 + r, v) == 0.0f; });
+                                                        [&](int r, float v) { if (!push_private<Out>(d, idx[u], aux[u], v)) first |= atomicAdd(row0 + r, v) == 0.0f; });
                     // (pattern matrices have no product: they count the hits in the accumulator,
                     // which the compaction clears like any other, to get the same first-touch test)
-                    if (DT == DBSPMSPV_PATTERN && hit) first = atomicAdd(row0 + (aux[u] >> 4), 1.0f) == 0.0f;
+                    if (DT == DBSPMSPV_PATTERN && hit && !push_private<Out>(d, idx[u], aux[u], 1.0f)) first = atomicAdd(row0 + (aux[u] >> 4), 1.0f) == 0.0f;
                     if (Out::MASKS && hit && first) mark_rows(out.hit8, brow, hit);
                 } else if (type == DBSPMSPV_BLK_COO && aux[u] < COO_SERIAL_MAX) {
                     coo_cnt = (int)aux[u] + 1;
@@ -1262,6 +1280,53 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
 // sorted.  Pass 1 counts per tile, pass 2 places the entries, clears the accumulator and the
 // masks it read, clears the vector-block state of this call's x, and rolls the counters over.
 // ------------------------------------------------------------------------------------------
+// Fold of the private accumulators of one hub row block (see push_private), by a whole warp:
+// every lane takes four rows of two copies, a shuffle tree adds the copies up in a fixed
+// order, the totals go into the accumulator proper (no atomics: every push has ended) and the
+// rows that any copy touched get their structural-hit flag; touched copies are put back to
+// HUB_CLEAR.  A kernel of its own, one warp per hub row block, between the traversal and the
+// compaction: hub row blocks are neighbours (the low vertex numbers of an R-MAT graph), so a
+// fold inside the compaction, by the warp that owns the rows, took 40 folds one after the other.
+static_assert(HUB_COPIES % 8 == 0, "a warp folds eight copies per step");
+__device__ __forceinline__ void fold_hub_block(const Device &d, int rb, int slot, int lane) {
+    const int q = lane & 3;
+    float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint32_t touched = 0u;
+#pragma unroll
+    for (int k = 0; k < HUB_COPIES / 8; ++k) {
+        const int c = (lane >> 2) + 8 * k;
+        float4 *p = reinterpret_cast<float4 *>(d.hub_acc + ((size_t)c * d.n_hub_blocks + slot) * 16) + q;
+        const float4 v = __ldcg(p);
+        const uint32_t t = (__float_as_uint(v.x) != HUB_CLEAR ? 1u : 0u) | (__float_as_uint(v.y) != HUB_CLEAR ? 2u : 0u) |
+                           (__float_as_uint(v.z) != HUB_CLEAR ? 4u : 0u) | (__float_as_uint(v.w) != HUB_CLEAR ? 8u : 0u);
+        // (an untouched -0.0f adds nothing)
+        tot.x += v.x; tot.y += v.y; tot.z += v.z; tot.w += v.w;
+        if (t) { const float z = __uint_as_float(HUB_CLEAR); *p = make_float4(z, z, z, z); }
+        touched |= t;
+    }
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+        tot.x += __shfl_xor_sync(FULL, tot.x, o); tot.y += __shfl_xor_sync(FULL, tot.y, o);
+        tot.z += __shfl_xor_sync(FULL, tot.z, o); tot.w += __shfl_xor_sync(FULL, tot.w, o);
+        touched |= __shfl_xor_sync(FULL, touched, o);
+    }
+    if (lane < 4 && touched) {
+        float *a = d.ws.y_acc + (size_t)rb * 16 + 4 * q;
+        uint8_t *f = d.ws.y_hit8 + (size_t)rb * 16 + 4 * q;
+        if (touched & 1u) { a[0] += tot.x; f[0] = 1; }
+        if (touched & 2u) { a[1] += tot.y; f[1] = 1; }
+        if (touched & 4u) { a[2] += tot.z; f[2] = 1; }
+        if (touched & 8u) { a[3] += tot.w; f[3] = 1; }
+    }
+}
+
+__global__ void __launch_bounds__(128) k_fold_hubs(Device d) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int slot = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (slot < d.n_hub_blocks) fold_hub_block(d, d.hub_rb[slot], slot, threadIdx.x & 31);
+}
+
 __global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d) {
     __shared__ int s_red[TILE_WORDS / 32];
     pdl_wait();
@@ -1604,6 +1669,11 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     }
     OutSparse out{d.ws.y_acc, d.ws.y_hit8};
     if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
+    // private accumulators for the hub row blocks: when x is long enough for their atomics to
+    // queue up, and not so long that the call will most likely pull
+    const int hub_min = h->ropts.hub_min_nnz_x ? h->ropts.hub_min_nnz_x : HUB_MIN_NNZ_X;
+    h->d.hub_on = d.n_hub_blocks > 0 && hub_min > 0 && nnz_x >= hub_min && h->ropts.force_path != DBSPMSPV_PATH_PULL &&
+                  (!late_emit || h->heavy_stage);
     if (nnz_x > 0 && d.n_entries > 0) {
         int s = DBSPMSPV_OK;
         if (h->heavy_stage) {
@@ -1616,6 +1686,10 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
             if (s == DBSPMSPV_OK && pull_possible(h, nnz_x, h->ropts.th3)) s = launch_lean<DT, OutSparse>(h, out, h->ropts.th3, st);
         }
         if (s != DBSPMSPV_OK) return s;
+        if (d.hub_on) {
+            DBS_CUDA(launch_pdl(k_fold_hubs, (d.n_hub_blocks + 3) / 4, 128, 0, st, d));
+            ++h->kernel_launches;
+        }
     }
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
     h->kernel_launches += 2;
@@ -1701,7 +1775,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     o->th3 = 0.9f;
     o->th3_bfs = 0.05f;
     o->th3_decode = 0.01f;
-    o->bfs_push_max_edge_frac = 0.1f;
+    o->bfs_push_max_edge_frac = 0.f;
     o->force_path = DBSPMSPV_PATH_AUTO;
     o->popc_threshold = 8;
     o->validate = 0;

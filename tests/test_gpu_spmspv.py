@@ -338,6 +338,58 @@ def test_rows_that_sum_to_zero_or_hold_stored_zeros_are_still_reported():
     h.close()
 
 
+def test_hub_row_blocks_add_into_private_accumulators_and_fold_exactly():
+    """Two row blocks hold 10,000 INLINE elements each, so the handle gives them private push
+    accumulators (an untouched one holds -0.0).  Rows whose products are stored zeros, partly
+    subnormal, or cancel exactly must still come out as structural hits with the oracle's values, and the
+    result must not depend on whether the private accumulators are used."""
+    m, n = 640, 10000
+    rng = np.random.default_rng(3)
+    dense = np.zeros((m, n), dtype=np.float32)
+    bg = wl.random_sparse(m, n, 6000, 13)
+    dense[bg.rows(), bg.col_idx] = bg.val
+    mask = dense != 0
+    for r in range(32):                                # one element per 16 x 16 block: INLINE class
+        cols = np.arange(r % 16, n, 16)
+        dense[r, :] = 0.0
+        mask[r, :] = False
+        dense[r, cols] = rng.uniform(0.5, 1.5, cols.size).astype(np.float32) * rng.choice([-1.0, 1.0], cols.size)
+        mask[r, cols] = True
+    dense[3, :] = 0.0                                  # row 3: stored zeros only
+    c9 = np.arange(9, n, 16)
+    dense[9, c9] = np.where(np.arange(c9.size) % 2 == 0, 2.5, -2.5)   # row 9: cancels under x = 1
+    c20 = np.arange(4, n, 16)
+    dense[20, c20] = np.where(np.arange(c20.size) % 2 == 0, 1e-41, 1.0)   # row 20: every other product subnormal
+    a = wl.csr_from_dense(dense, keep_zeros_mask=mask)
+    x_idx = np.arange(0, 8000, dtype=np.int32)
+    x = wl.SparseVec(n, x_idx, np.ones(x_idx.size, dtype=np.float32))
+    h = Handle(a, B.F32)
+    assert h.stats.n_hub_row_blocks == 2
+    want = oracle.ref_pull(ref_matrix(a), x.idx, x.val)
+    assert {3, 9, 20} <= set(want[0].tolist())
+    got = {}
+    for hub_min in (1, -1):
+        h.set_opts(force_path=B.PATH_PUSH, hub_min_nnz_x=hub_min)
+        got[hub_min] = h.run(x)
+        check_against_oracle(got[hub_min], want)
+        assert h.get_stats().last_path == B.PATH_PUSH
+    assert np.array_equal(got[1][0], got[-1][0])
+    i9 = int(np.searchsorted(got[1][0], 9))
+    assert got[1][1][i9] == 0.0
+    # the private accumulators are clean again: a second, different call
+    x2 = wl.SparseVec(n, np.arange(5, 9000, 3, dtype=np.int32), np.linspace(-1.0, 1.0, len(range(5, 9000, 3)), dtype=np.float32))
+    h.set_opts(force_path=B.PATH_PUSH, hub_min_nnz_x=1)
+    check_against_oracle(h.run(x2), oracle.ref_pull(ref_matrix(a), x2.idx, x2.val))
+    h.set_opts(hub_min_nnz_x=1)
+    check_against_oracle(h.run(x2), oracle.ref_pull(ref_matrix(a), x2.idx, x2.val))
+    # pattern handle: the products are counts
+    hp = Handle(wl.CSR(a.m, a.n, a.row_ptr, a.col_idx, None), B.PATTERN)
+    hp.set_opts(force_path=B.PATH_PUSH, hub_min_nnz_x=1)
+    wp = oracle.ref_pull(oracle.RefMatrix(a.m, a.n, a.row_ptr, a.col_idx, None), x.idx, None)
+    check_against_oracle(hp.run(x, semiring=B.OR_AND), wp, boolean=True)
+    h.close(); hp.close()
+
+
 def test_bounded_wait_runs_out_and_reports_timeout():
     """The staging waits are bounded: a wait on a barrier that nothing arrives on (no copy in
     flight) gives up, the kernel records ERR_TIMEOUT, get_stats returns it once, and the handle
