@@ -118,10 +118,15 @@ typedef struct {
                                 a push level pays one atomic per reached entry)             */
     float th3_decode;        /* dbspmspv_decode: same rule; the output is dense and every row block
                                 takes part, so pull wins much earlier (0.01, the paper's value) */
-    int32_t no_fused_decode; /* 1: dbspmspv_decode never uses its single-kernel form (which serves
-                                handles whose elements sit mostly in mask-based blocks and whose
-                                x fits in shared memory) but the blocking / traversal / cleanup
-                                kernels of dbspmspv_run                              (0)    */
+    int32_t no_fused_decode; /* dbspmspv_decode on handles whose elements sit mostly in blocks with
+                                a payload and whose x fits in shared memory has two one-kernel
+                                forms: a streaming one (the whole payload is moved through
+                                shared memory by bulk copies) and a selective one (only the
+                                block columns x reaches are fetched).
+                                0: streaming, or selective when the x of the handle's previous
+                                   decode call had fewer than 15 % nonzero elements (default);
+                                1: neither -- the blocking / traversal / cleanup kernels of
+                                   dbspmspv_run;   2: selective only;   3: streaming only      */
     float bfs_push_max_edge_frac; /* db_bfs (with the row-run index): a level whose push worklist
                                 covers more than this share of the view's entries is pulled
                                 even when the block ratio says push.  0 = block ratio only,

@@ -203,6 +203,8 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     cudaFree(const_cast<int32_t *>(d.rowrun_ptr)); cudaFree(const_cast<uint32_t *>(d.rowrun_idx));
     cudaFree(const_cast<int32_t *>(d.csr_inl)); cudaFree(const_cast<int32_t *>(d.payload_pos));
     cudaFree(const_cast<int32_t *>(d.lean_rows)); cudaFree(const_cast<int32_t *>(d.lean_chunk_ord));
+    cudaFree(const_cast<int4 *>(d.stage_chunks));
+    if (h->x_nnz_seen_host) cudaFreeHost(h->x_nnz_seen_host);
     cudaFree(const_cast<uint16_t *>(d.hub_slot)); cudaFree(const_cast<int32_t *>(d.hub_rb)); cudaFree(d.hub_acc);
     cudaFree(h->csc2csr); cudaFree(h->block_row);
     cudaFree(h->ws_arena);

@@ -396,6 +396,29 @@ __global__ void k_csr_inl(int32_t mb, const uint64_t *keys_sorted, int32_t n, in
     inl[rb] = lo;
 }
 
+// Payload chunks of the staged decode: one thread per row block walks its entries with a payload
+// ([ptr[rb], inl[rb]), contiguous in the payload) and cuts them greedily into chunks of at most
+// cap_entries entries and cap_bytes bytes.  out == nullptr: count only.
+__global__ void k_stage_chunks(int32_t mb, const int32_t *ptr, const int32_t *inl, const uint32_t *idx, const uint32_t *w,
+                               const uint8_t *aux, int vsize, int cap_entries, int cap_bytes, int32_t *count,
+                               const int32_t *first, int4 *out) {
+    const int rb = blockIdx.x * blockDim.x + threadIdx.x;
+    if (rb >= mb) return;
+    int n = 0, e0 = ptr[rb], words = 0;
+    const int end = inl[rb];
+    int4 *o = out ? out + first[rb] : nullptr;
+    for (int p = e0; p < end; ++p) {
+        const int sz = payload_words((int)(idx[p] >> TYPE_SHIFT), (int)aux[p] + 1, vsize);
+        if (p > e0 && (p - e0 >= cap_entries || (words + sz) * 4 > cap_bytes)) {
+            if (o) o[n] = make_int4(e0, rb, (int)w[e0], words | ((p - e0) << 24));
+            ++n; e0 = p; words = 0;
+        }
+        words += sz;
+    }
+    if (end > e0) { if (o) o[n] = make_int4(e0, rb, (int)w[e0], words | ((end - e0) << 24)); ++n; }
+    if (!out) count[rb] = n;
+}
+
 // Row list of the streaming pull: flag[p] = 1 at the first INLINE element of a row;
 // rows[rank[p]] = that row; chunk_ord[c] = row heads before entry c * LEAN_CHUNK.
 __global__ void k_lean_flags(int32_t n_entries, const uint32_t *idx, int32_t *flag) {
@@ -930,6 +953,39 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
         h->bfs_index_bytes = ((int64_t)m + 1) * 4 + (int64_t)n_inline * 4;
     }
 
+    // Streaming decode of payload-dominated handles: the chunk table
+    d.stage_chunks = nullptr; d.n_stage_chunks = 0;
+    d.has_inline = cls_h[DBSPMSPV_BLK_INLINE] > 0;
+    d.x_nnz_seen = nullptr; h->x_nnz_seen_host = nullptr; d.x_sparse_believed = 0;
+    if (h->heavy_stage) {
+        // one word of mapped host memory through which the decode kernels report the x they saw
+        void *hp = nullptr, *dp = nullptr;
+        if (cudaHostAlloc(&hp, 64, cudaHostAllocMapped) == cudaSuccess && cudaHostGetDevicePointer(&dp, hp, 0) == cudaSuccess) {
+            h->x_nnz_seen_host = static_cast<int32_t *>(hp);
+            *h->x_nnz_seen_host = -1;
+            d.x_nnz_seen = static_cast<int32_t *>(dp);
+        } else {
+            if (hp) cudaFreeHost(hp);
+            cudaGetLastError();
+        }
+    }
+    d.stage_bytes = h->heavy_stage ? decode_stage_bytes(d) : 0;
+    if (d.stage_bytes > 0 && d.mb > 0) {
+        int32_t *cnt, *first;
+        DBS_GET(cnt, (int64_t)d.mb + 1); DBS_GET(first, (int64_t)d.mb + 1);
+        DBS_CUDA(cudaMemsetAsync(cnt, 0, ((size_t)d.mb + 1) * 4, st));
+        k_stage_chunks<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr_inl, d.csr.idx, d.csr.w, d.csr.aux, vsize, 32, d.stage_bytes, cnt, nullptr, nullptr);
+        DBS_TRY(exclusive_sum(tp, cnt, first, (int64_t)d.mb + 1, st));
+        DBS_CUDA(cudaMemcpy(&d.n_stage_chunks, first + d.mb, 4, cudaMemcpyDeviceToHost));
+        int4 *chunks;
+        DBS_KEEP(chunks, d.n_stage_chunks);
+        k_stage_chunks<<<grid_for(d.mb), TPB, 0, st>>>(d.mb, d.csr.ptr, d.csr_inl, d.csr.idx, d.csr.w, d.csr.aux, vsize, 32, d.stage_bytes, cnt, first, chunks);
+        DBS_CUDA(cudaStreamSynchronize(st));
+        tp.release(cnt); tp.release(first);
+        d.stage_chunks = chunks;
+        h->stage_index_bytes = (int64_t)d.n_stage_chunks * 16;
+    }
+
     // Streaming pull of hypersparse handles: the list of rows that hold INLINE elements (the
     // stream itself carries one flag bit per row start), the number of row starts before every
     // chunk of the stream, and the positions of the few entries with a payload.
@@ -1010,7 +1066,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     s.n_view_entries = d.n_entries;
     s.csr_view_bytes = ((int64_t)d.mb + 1) * 8 + (int64_t)d.n_entries * 9;
     s.csc_view_bytes = ((int64_t)d.nb + 1) * 4 + (int64_t)d.nb * 17 * 4 + (int64_t)d.n_entries * 9 + h->hub_bytes;
-    s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment) + ((int64_t)d.n_chunks + 1) * 8 + (int64_t)d.n_segments * 4;
+    s.segment_bytes = (int64_t)d.n_segments * (int64_t)sizeof(Segment) + ((int64_t)d.n_chunks + 1) * 8 + (int64_t)d.n_segments * 4 + h->stage_index_bytes;
     s.bfs_index_bytes = h->bfs_index_bytes;
     s.lean_index_bytes = h->lean_index_bytes;
     s.n_hub_row_blocks = d.n_hub_blocks;

@@ -93,6 +93,12 @@ static_assert(PUSH_CHUNK == 32, "a push task is one warp step; its record stores
 // into tasks: it is listed once and every warp of the traversal strides over its 32-entry steps.
 constexpr int HUB_MIN_ENTRIES = 8192;
 constexpr int HUB_CAP = 32;
+// Stage of the single-kernel decode: payload bytes per chunk, at most (a chunk also has at
+// most 32 view entries: one per lane)
+#ifndef DBS_STAGE_BYTES
+#define DBS_STAGE_BYTES (6 * 1024)
+#endif
+constexpr int STAGE_BYTES = DBS_STAGE_BYTES;
 constexpr int HDR_BYTES = 48;               // masks + starts of a valued mid-class block
 
 // Payload size in 4-byte words; every block is padded to 16 bytes so that it can be moved with
@@ -217,6 +223,16 @@ struct Device {           // everything the kernels need, passed by value
     int32_t n_lean_chunks;
     int32_t n_lean_rows;
     int32_t n_payload;
+    // Streaming decode (handles whose elements sit mostly in blocks with a payload; null
+    // otherwise): the payload of a row block is one contiguous byte range, cut into chunks of
+    // whole blocks that fit a warp's shared-memory stage.  stage_chunks[c] = {first view entry,
+    // row block, payload offset in words, words | entries << 24}, in payload order.
+    const int4 *stage_chunks;
+    int32_t n_stage_chunks;
+    int32_t stage_bytes;        // payload bytes of one stage (a multiple of 512)
+    int32_t has_inline;         // the handle holds INLINE elements at all
+    int32_t x_sparse_believed;  // per call: what the host currently takes x for (1: sparse)
+    int32_t *x_nnz_seen;        // mapped host word: nonzero elements of the x of the last single-kernel decode (null: none)
     // Hub row blocks (null / 0 when the matrix has none): hub_slot[rb] = slot of row block rb or
     // HUB_NONE; hub_acc[(copy * n_hub_blocks + slot) * 16 + row] = private accumulators, all
     // HUB_CLEAR between calls.
@@ -250,6 +266,8 @@ struct dbspmspv_handle_s {
     int grid_compute, grid_compute_dense, grid_decode_pull;
     bool lean_configured, lean_configured_dense;
     bool fused_configured[3];
+    int stream_grid;            // thread blocks of the streaming decode (0: not configured yet)
+    int32_t *x_nnz_seen_host;   // host view of Device::x_nnz_seen (page-locked, mapped)
     bool heavy_stage;           // most stored elements sit in mask-based blocks: MODE 1 kernels
     cudaEvent_t ev[2];          // optional timing of the traversal kernel (run_opts.timing)
     bool timed;
@@ -257,6 +275,7 @@ struct dbspmspv_handle_s {
     int64_t bfs_index_bytes;
     int64_t lean_index_bytes;
     int64_t hub_bytes;
+    int64_t stage_index_bytes;
     void *ws_arena;             // the one allocation that holds the whole workspace
     cudaStream_t last_stream;   // stream of the last run / decode / bfs call (get_stats waits on it)
 };
@@ -271,6 +290,10 @@ namespace dbs {
 
 template <typename T>
 __host__ __device__ inline T ceil_div(T a, T b) { return (a + b - 1) / b; }
+
+// Streaming decode (run.cu): the payload bytes of one stage that shared memory leaves room for
+// on this handle (0: none).
+int decode_stage_bytes(const Device &d);
 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
 // start while its predecessor drains; `pdl_wait` blocks until the predecessor has completed and

@@ -983,7 +983,8 @@ __host__ __device__ constexpr int wc_ilp(int warps_per_block) { return warps_per
 // staging bytes per lane; the stride keeps 16-byte stores conflict-free
 __host__ __device__ constexpr int wc_slot_bytes(int ilp) { return 48 * ilp + (ilp > 1 ? 16 : 0); }
 
-template <int DT, int WC_ILP>
+// DIRECT: the payload lies in shared memory, so the values are indexed where they are (no staging slot).
+template <int DT, int WC_ILP, bool DIRECT = false>
 __device__ __forceinline__ void warp_columns(const uint8_t *payload, const float *x_blocks, uint32_t idx, uint32_t w,
                                              uint32_t cols, int lane, float (&acc)[16], uint4 *slot) {
     int incl = __popc(cols);
@@ -1033,7 +1034,7 @@ __device__ __forceinline__ void warp_columns(const uint8_t *payload, const float
                 pos[u] = dense[u] ? c * 16 : blk[u][32 + c];
             }
         }
-        if (DT == DBSPMSPV_BF16) {
+        if (DT == DBSPMSPV_BF16 && !DIRECT) {
             int off[WC_ILP];
 #pragma unroll
             for (int u = 0; u < WC_ILP; ++u) {
@@ -1077,6 +1078,65 @@ __device__ __forceinline__ void warp_columns(const uint8_t *payload, const float
     }
 }
 
+// x -> 16-bit masks and fp32 blocks in shared memory (absent entries carry the marker), by all
+// `threads` threads of the block; s_cnt[0] and s_cnt[1] (zeroed by the caller, barrier in
+// between) receive the numbers of nonzero vector blocks and of nonzero elements.  The caller synchronises afterwards.
+template <int DT>
+__device__ __forceinline__ void stage_x_blocks(const Device &d, const void *__restrict__ x, float *s_x, uint16_t *s_xm,
+                                               int *s_cnt, int tid, int T) {
+    const int lane = tid & 31;
+    const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
+    int mine = 0;
+    for (int cb = tid; cb < d.nb; cb += T) {
+        const int64_t j0 = (int64_t)cb * 16;
+        float v[16];
+        if (aligned && j0 + 16 <= d.n) {
+            if (DT == DBSPMSPV_BF16) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(x) + j0);
+                const uint4 a = src[0], b = src[1];
+                const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { v[2 * q] = __uint_as_float(u[q] << 16); v[2 * q + 1] = __uint_as_float(u[q] & 0xFFFF0000u); }
+            } else {
+                const float4 *src = reinterpret_cast<const float4 *>(static_cast<const float *>(x) + j0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { const float4 f = src[q]; v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w; }
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                v[k] = 0.f;
+                if (j0 + k < d.n) v[k] = DT == DBSPMSPV_BF16 ? __uint_as_float((uint32_t) static_cast<const uint16_t *>(x)[j0 + k] << 16)
+                                                             : static_cast<const float *>(x)[j0 + k];
+            }
+        }
+        uint32_t bits = 0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const bool nz = v[k] != 0.0f;
+            bits |= (nz ? 1u : 0u) << k;
+            // (a widened bf16 has zero low bits: it cannot collide with the marker)
+            if (DT != DBSPMSPV_BF16 && __float_as_uint(v[k]) == X_ABSENT) v[k] = __uint_as_float(0x7FC00000u);
+            v[k] = nz ? v[k] : __uint_as_float(X_ABSENT);
+        }
+        float4 *dst = reinterpret_cast<float4 *>(s_x + j0);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        s_xm[cb] = (uint16_t)bits;
+        mine += (bits != 0) | (__popc(bits) << 16);           // nonzero blocks, nonzero elements
+    }
+    mine = __reduce_add_sync(FULL, mine);
+    if (lane == 0 && mine) { atomicAdd(&s_cnt[0], mine & 0xFFFF); atomicAdd(&s_cnt[1], mine >> 16); }
+}
+
+// Streaming reads the whole payload whatever x holds; the single-kernel form above fetches only
+// the columns x reaches, which is less than half of the bytes once x has fewer nonzero elements
+// than this share (measured on the three layer shapes: 22.6 against 27.6 us at 10 %, 37.9
+// against 33.8 us at 30 %).  The choice follows the x of the handle's previous decode call --
+// both kernels report the number of nonzero elements they saw through a word of mapped host
+// memory, read without waiting: activations of one layer keep their sparsity from token to token.
+constexpr float STREAM_MIN_X_DENSITY = 0.15f;
+
 // The whole decode call in one kernel, for payload-dominated handles whose x fits in shared
 // memory (Section 4.3: one layer, one token).  One thread block per row block.  Every block
 // first reads the dense activation vector itself -- a few KB -- into shared memory as the
@@ -1119,55 +1179,11 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
     uint16_t *s_xm = reinterpret_cast<uint16_t *>(s_dyn + lay.xm_off);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint4 *slot = reinterpret_cast<uint4 *>(s_dyn + lay.slot_off + tid * wc_slot_bytes(wc_ilp(NW)));
-    if (tid == 0) s_cnt[0] = 0;
+    if (tid == 0) { s_cnt[0] = 0; s_cnt[1] = 0; }
     if (tid < 16) s_y[tid] = 0.f;
     __syncthreads();
 
-    // ---- x -> masks and fp32 blocks (absent entries carry the marker)
-    {
-        const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
-        int mine = 0;
-        for (int cb = tid; cb < d.nb; cb += T) {
-            const int64_t j0 = (int64_t)cb * 16;
-            float v[16];
-            if (aligned && j0 + 16 <= d.n) {
-                if (DT == DBSPMSPV_BF16) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(x) + j0);
-                    const uint4 a = src[0], b = src[1];
-                    const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) { v[2 * q] = __uint_as_float(u[q] << 16); v[2 * q + 1] = __uint_as_float(u[q] & 0xFFFF0000u); }
-                } else {
-                    const float4 *src = reinterpret_cast<const float4 *>(static_cast<const float *>(x) + j0);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) { const float4 f = src[q]; v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w; }
-                }
-            } else {
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    v[k] = 0.f;
-                    if (j0 + k < d.n) v[k] = DT == DBSPMSPV_BF16 ? __uint_as_float((uint32_t) static_cast<const uint16_t *>(x)[j0 + k] << 16)
-                                                                 : static_cast<const float *>(x)[j0 + k];
-                }
-            }
-            uint32_t bits = 0;
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const bool nz = v[k] != 0.0f;
-                bits |= (nz ? 1u : 0u) << k;
-                // (a widened bf16 has zero low bits: it cannot collide with the marker)
-                if (DT != DBSPMSPV_BF16 && __float_as_uint(v[k]) == X_ABSENT) v[k] = __uint_as_float(0x7FC00000u);
-                v[k] = nz ? v[k] : __uint_as_float(X_ABSENT);
-            }
-            float4 *dst = reinterpret_cast<float4 *>(s_x + j0);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-            s_xm[cb] = (uint16_t)bits;
-            mine += bits != 0;
-        }
-        mine = __reduce_add_sync(FULL, mine);
-        if (lane == 0 && mine) atomicAdd(&s_cnt[0], mine);
-    }
+    stage_x_blocks<DT>(d, x, s_x, s_xm, s_cnt, tid, T);
     __syncthreads();
     const int n_nzblk = s_cnt[0];
     int path = force_path;
@@ -1176,6 +1192,8 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
     if (blockIdx.x == 0 && tid == 0) {
         Counters *c = d.ws.ctr;
         c->last_n_nzblk = n_nzblk; c->last_n_tasks = 0; c->last_path = path; c->last_y_nnz = (int32_t)d.m;
+        // (a store to host memory: only when it changes what the host goes by)
+        if (d.x_nnz_seen && ((float)s_cnt[1] < STREAM_MIN_X_DENSITY * (float)d.n) != (d.x_sparse_believed != 0)) *d.x_nnz_seen = s_cnt[1];
     }
     if (path == DBSPMSPV_PATH_PUSH) {
         if (warp == 0) {
@@ -1272,6 +1290,248 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
         for (int k = 0; k < NW; ++k) sum += s_part[k * 16 + tid];
         const int64_t row = (int64_t)rb * 16 + tid;
         if (row < d.m) y[row] = sum;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Streaming decode (Section 4.3: one layer, one token) for payload-dominated handles: the whole
+// call in one persistent kernel that reads the payload as a stream.
+//   * The payload of a row block is one contiguous byte range; at create it is cut into chunks
+//     of whole blocks (a few KB, at most 32 blocks).  The chunk list is split evenly over all
+//     warps of the grid, every warp taking a contiguous piece.
+//   * Every warp runs its own ring of STREAM_DEPTH stages in shared memory: one lane moves a
+//     chunk's payload bytes with one bulk copy while the warp works on an earlier chunk (the
+//     chunk's view entries, 9 bytes per block, are loaded into registers a round ahead).  The microkernels' chains of
+//     dependent loads (entry -> header -> column start -> values) then cost shared-memory
+//     latency, no load goes through the L1 tag stage one sector at a time, and HBM sees
+//     sequential reads whatever the activation sparsity.
+//   * x is read once per thread block (a few KB) into masks and fp32 blocks, as in the
+//     single-kernel form above; the 16 row sums of a warp stay in registers while its chunks
+//     belong to one row block and go to y with one atomic per row when the row block changes
+//     (y is zeroed by a memset in front of the kernel).
+// A call whose x fills few vector blocks (push) walks the row blocks' entries by bisection
+// straight from global memory, as the single-kernel form does.
+#ifndef DBS_STREAM_WARPS
+#define DBS_STREAM_WARPS 16
+#endif
+#ifndef DBS_STREAM_BUDGET
+#define DBS_STREAM_BUDGET (220 * 1024)
+#endif
+constexpr int STREAM_WARPS = DBS_STREAM_WARPS;
+constexpr int STREAM_CTA = STREAM_WARPS * 32;
+#ifndef DBS_STREAM_DEPTH
+#define DBS_STREAM_DEPTH 2
+#endif
+constexpr int STREAM_DEPTH = DBS_STREAM_DEPTH;
+constexpr int STREAM_MAX_SMEM = 220 * 1024;
+__host__ __device__ constexpr int stream_stride(int stage_bytes) { return (stage_bytes + 127) & ~127; }
+struct StreamLayout {
+    int xm_off, cnt_off, active_off, bar_off, ring_off, total;
+    __host__ __device__ StreamLayout(int nb, int stage_bytes) {
+        xm_off = nb * 64;
+        cnt_off = (xm_off + nb * 2 + 15) & ~15;
+        active_off = cnt_off + 16;
+        bar_off = (active_off + nb * 4 + 15) & ~15;
+        ring_off = (bar_off + STREAM_WARPS * STREAM_DEPTH * 8 + 127) & ~127;
+        total = ring_off + STREAM_WARPS * STREAM_DEPTH * stream_stride(stage_bytes);
+    }
+};
+
+template <int DT>
+__global__ void __launch_bounds__(STREAM_CTA, STREAM_WARPS <= 8 ? 2 : 1)
+k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, float th3, int force_path) {
+    extern __shared__ __align__(128) uint8_t s_dyn[];
+    constexpr int T = STREAM_CTA, NW = STREAM_WARPS;
+    const StreamLayout lay(d.nb, d.stage_bytes);
+    float *s_x = reinterpret_cast<float *>(s_dyn);
+    uint16_t *s_xm = reinterpret_cast<uint16_t *>(s_dyn + lay.xm_off);
+    int *s_cnt = reinterpret_cast<int *>(s_dyn + lay.cnt_off);
+    int *s_active = reinterpret_cast<int *>(s_dyn + lay.active_off);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int stride = stream_stride(d.stage_bytes);
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(s_dyn + lay.bar_off) + warp * STREAM_DEPTH;
+    uint8_t *s_ring = s_dyn + lay.ring_off + (size_t)warp * STREAM_DEPTH * stride;
+    if (tid == 0) { s_cnt[0] = 0; s_cnt[1] = 0; }
+
+    // this warp's piece of the chunk list; lane i keeps the descriptor of its i-th chunk (32 at a time)
+    const int gw = blockIdx.x * NW + warp, W = gridDim.x * NW;
+    const int lo = (int)((int64_t)d.n_stage_chunks * gw / W), hi = (int)((int64_t)d.n_stage_chunks * (gw + 1) / W);
+    const int n_mine = hi - lo;
+    int4 my_desc = make_int4(0, 0, 0, 0);
+    if (lane < n_mine) my_desc = d.stage_chunks[lo + lane];
+    auto desc_of = [&](int k) {                               // (whole warp)
+        return make_int4(__shfl_sync(FULL, my_desc.x, k & 31), __shfl_sync(FULL, my_desc.y, k & 31),
+                         __shfl_sync(FULL, my_desc.z, k & 31), __shfl_sync(FULL, my_desc.w, k & 31));
+    };
+    // descriptor: x = first view entry, y = row block, z = payload offset in words, w = words | entries << 24
+    auto issue = [&](const int4 &ch, int st) {               // lane 0 only
+        uint8_t *base = s_ring + (size_t)st * stride;
+        const uint32_t pb = ((uint32_t)ch.w & 0xFFFFFFu) * 4u;
+        fence_proxy_async_smem();
+        mbar_arrive_expect_tx(&s_bar[st], pb);
+        bulk_copy_g2s(base, d.payload + (size_t)(uint32_t)ch.z * 4, pb, &s_bar[st]);
+    };
+    // the chunk's view entries, one per lane, by plain loads a round ahead of their use (they
+    // are 9 bytes per block; bulk copies of 48-256 bytes cost the copy engine as much as the payload's)
+    auto entries_of = [&](const int4 &ch, uint32_t &idx, uint32_t &w, uint32_t &aux) {
+        idx = 0; w = 0; aux = 0;
+        if (lane < (int)((uint32_t)ch.w >> 24)) { const int p_ = ch.x + lane; idx = d.csr.idx[p_]; w = d.csr.w[p_]; aux = d.csr.aux[p_]; }
+    };
+    int issued = 0;                                           // chunks of mine whose copies were started
+    if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < STREAM_DEPTH; ++k) mbar_init(&s_bar[k], 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+    // the first copies start before x is even looked at
+    for (; issued < STREAM_DEPTH - 1 && issued < n_mine; ++issued) {
+        const int4 ch = desc_of(issued);
+        if (lane == 0) issue(ch, issued);
+    }
+    __syncthreads();
+    stage_x_blocks<DT>(d, x, s_x, s_xm, s_cnt, tid, T);
+    __syncthreads();
+    const int n_nzblk = s_cnt[0];
+    int path = force_path;
+    if (path != DBSPMSPV_PATH_PUSH && path != DBSPMSPV_PATH_PULL)
+        path = (float)n_nzblk / (float)d.nb < th3 ? DBSPMSPV_PATH_PUSH : DBSPMSPV_PATH_PULL;
+    if (blockIdx.x == 0 && tid == 0) {
+        Counters *c = d.ws.ctr;
+        c->last_n_nzblk = n_nzblk; c->last_n_tasks = 0; c->last_path = path; c->last_y_nnz = (int32_t)d.m;
+        // (a store to host memory: only when it changes what the host goes by)
+        if (d.x_nnz_seen && ((float)s_cnt[1] < STREAM_MIN_X_DENSITY * (float)d.n) != (d.x_sparse_believed != 0)) *d.x_nnz_seen = s_cnt[1];
+    }
+
+    // y is zeroed by the kernel in front, which this one may overlap up to here
+    pdl_wait();
+
+    float acc[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+    int cur_rb = -1;
+    // the warp's 16 row sums -> y (rows past m hold nothing: their sums are exact zeros)
+    auto flush = [&]() {
+        if (cur_rb >= 0) {
+            const float total = fold_rows(acc, lane);
+            if (!(lane & 1) && total != 0.f) atomicAdd(y + (size_t)cur_rb * 16 + folded_row(lane), total);
+#pragma unroll
+            for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+        }
+    };
+    auto emit = [&](int erb, int erow, float esum) { atomicAdd(y + (size_t)erb * 16 + erow, esum); };
+    // one step: the lane's entry (idx, w, aux) of row block cur_rb, if `have`; the payload pointer
+    // is the staged copy (shifted so that the entry's offset applies) or, on the rare paths that
+    // read global memory, the payload itself -- the values are indexed where they are either way
+    auto step = [&](const uint8_t *payload, uint32_t idx, uint32_t w, uint32_t aux, bool have) {
+        const uint32_t xm = have ? s_xm[idx & IDX_MASK] : 0u;
+        const int type = idx >> TYPE_SHIFT;
+        const bool mk = have && xm && type > DBSPMSPV_BLK_COO;
+        const bool rowm = mk && is_row_major(type);
+        const float *xb = s_x + (size_t)(idx & IDX_MASK) * 16;
+        warp_columns<DT, 2, true>(payload, s_x, idx, w, mk && !rowm ? xm : 0u, lane, acc, static_cast<uint4 *>(nullptr));
+        __syncwarp();
+        const uint32_t rows = __ballot_sync(FULL, rowm);
+        if (rows) half_stream<DT, true>(payload, s_x, idx, w, xm, cur_rb, rows, lane, emit);
+        if (have && xm && type <= DBSPMSPV_BLK_COO) {       // the odd hypersparse block: its own lane
+            float *row0 = y + (size_t)cur_rb * 16;
+            if (type == DBSPMSPV_BLK_INLINE) {
+                if ((xm >> (aux & 15)) & 1u) atomicAdd(row0 + (aux >> 4), Val<DT>::inline_value(w) * xb[aux & 15]);
+            } else {
+                const int nnz = (int)aux + 1;
+                const uint8_t *blk = payload + (size_t)w * 4, *vals = blk + ((nnz + 3) & ~3);
+                for (int k = 0; k < nnz; ++k) {
+                    const int c = blk[k] & 15, r = blk[k] >> 4;
+                    if ((xm >> c) & 1u) atomicAdd(row0 + r, Val<DT>::load(vals, k) * xb[c]);
+                }
+            }
+        }
+    };
+    auto fetch = [&](int p, bool have, uint32_t &idx, uint32_t &w, uint32_t &aux) {
+        idx = 0; w = 0; aux = 0;
+        if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; }
+    };
+
+    if (path == DBSPMSPV_PATH_PULL) {
+        bool timed_out = false;
+        uint32_t idx = 0, w = 0, aux = 0, n_idx, n_w, n_aux;
+        if (n_mine > 0) entries_of(desc_of(0), idx, w, aux);
+        for (int k = 0; k < n_mine; ++k) {
+            // keep STREAM_DEPTH - 1 chunks in flight beside this one: chunk i goes into the stage
+            // that chunk i - STREAM_DEPTH was read from, in a round before this one
+            for (const int lim = min(n_mine, min(k + STREAM_DEPTH, (k & ~31) + 32)); issued < lim; ++issued) {
+                const int4 nch = desc_of(issued);
+                if (lane == 0) issue(nch, issued % STREAM_DEPTH);
+            }
+            const int st = k % STREAM_DEPTH;
+            const int4 ch = desc_of(k);
+            n_idx = 0; n_w = 0; n_aux = 0;
+            if (k + 1 < n_mine && ((k + 1) & 31)) entries_of(desc_of(k + 1), n_idx, n_w, n_aux);
+            if (!mbar_wait_bounded(&s_bar[st], (uint32_t)(k / STREAM_DEPTH) & 1u)) { timed_out = true; break; }
+            if (ch.y != cur_rb) { flush(); cur_rb = ch.y; }
+            const uint8_t *base = s_ring + (size_t)st * stride;
+            step(base - (size_t)(uint32_t)ch.z * 4, idx, w, aux, lane < (int)((uint32_t)ch.w >> 24));
+            __syncwarp();
+            idx = n_idx; w = n_w; aux = n_aux;
+            if (k + 1 < n_mine && !((k + 1) & 31)) {           // first chunk of the next descriptor batch: fetched late
+                my_desc = make_int4(0, 0, 0, 0);
+                if (k + 1 + lane < n_mine) my_desc = d.stage_chunks[lo + k + 1 + lane];
+                entries_of(desc_of(k + 1), idx, w, aux);
+            }
+        }
+        flush();
+        if (timed_out) { d.ws.ctr->status = DBSPMSPV_ERR_TIMEOUT; return; }
+        // the INLINE elements of the row blocks (row by row, rare in these handles)
+        for (int rb = gw; rb < d.mb && d.has_inline; rb += W) {
+            const int b0 = d.csr_inl[rb], b1 = d.csr.ptr[rb + 1];
+            cur_rb = rb;
+            for (int base = b0; base < b1; base += 32) {
+                uint32_t idx, w, aux;
+                fetch(base + lane, base + lane < b1, idx, w, aux);
+                step(d.payload, idx, w, aux, base + lane < b1);
+            }
+            if (b1 > b0) flush();
+        }
+    } else {
+        // copies of the first chunks are in flight: they must have landed before the block ends
+        for (int k = 0; k < issued; ++k) mbar_wait_bounded(&s_bar[k], 0u);
+        if (warp == 0) {
+            int count = 0;
+            for (int base = 0; base < d.nb; base += 32) {
+                const bool on = base + lane < d.nb && s_xm[base + lane] != 0;
+                const uint32_t m = __ballot_sync(FULL, on);
+                if (on) s_active[count + __popc(m & below(lane))] = base + lane;
+                count += __popc(m);
+            }
+        }
+        __syncthreads();
+        for (int rb = blockIdx.x; rb < d.mb; rb += gridDim.x) {
+            const int begin = d.csr.ptr[rb], pend = d.csr_inl[rb], end = d.csr.ptr[rb + 1];
+            cur_rb = rb;
+            // the row block's entries with a payload are sorted by column block: [begin, pend)
+            for (int i0 = warp * 32; i0 < n_nzblk; i0 += T) {
+                int lo_ = 0, hi_ = 0;
+                if (i0 + lane < n_nzblk) {
+                    const uint32_t cb = (uint32_t)s_active[i0 + lane];
+                    int a = begin, b = pend;          // first entry with column block >= cb
+                    while (a < b) { const int mid = a + ((b - a) >> 1); if ((d.csr.idx[mid] & IDX_MASK) < cb) a = mid + 1; else b = mid; }
+                    lo_ = a; b = pend;                // first entry with column block > cb
+                    while (a < b) { const int mid = a + ((b - a) >> 1); if ((d.csr.idx[mid] & IDX_MASK) <= cb) a = mid + 1; else b = mid; }
+                    hi_ = a;
+                }
+                for (int t = 0; __any_sync(FULL, lo_ + t < hi_); ++t) {
+                    uint32_t idx, w, aux;
+                    fetch(lo_ + t, lo_ + t < hi_, idx, w, aux);
+                    step(d.payload, idx, w, aux, lo_ + t < hi_);
+                }
+            }
+            for (int base = pend + warp * 32; base < end; base += T) {
+                uint32_t idx, w, aux;
+                fetch(base + lane, base + lane < end, idx, w, aux);
+                step(d.payload, idx, w, aux, base + lane < end);
+            }
+            flush();
+        }
     }
 }
 
@@ -1704,10 +1964,48 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     return DBSPMSPV_OK;
 }
 
+// payload bytes of one stage of a warp's ring in the streaming decode: what shared memory leaves
+// when two thread blocks share an SM (else one), at most STAGE_BYTES; 0 = no room (a block must fit)
+int decode_stage_bytes(const Device &d) {
+    const StreamLayout lay(d.nb, 0);
+    for (int budget : {DBS_STREAM_BUDGET, STREAM_MAX_SMEM}) {
+        const int room = budget - lay.ring_off;
+        if (room <= 0) continue;
+        int sb = (room / (STREAM_WARPS * STREAM_DEPTH)) & ~511;
+        if (sb > STAGE_BYTES) sb = STAGE_BYTES;
+        if (sb >= 2048) return sb;
+    }
+    return 0;
+}
+
 template <int DT>
 static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStream_t st) {
     const Device &d = h->d;
-    if (h->heavy_stage && !h->ropts.no_fused_decode) {
+    // (-1: no decode call has reported yet)
+    const int seen = h->x_nnz_seen_host ? *const_cast<volatile int32_t *>(h->x_nnz_seen_host) : -1;
+    const bool sparse_x = seen >= 0 && (float)seen < STREAM_MIN_X_DENSITY * (float)d.n;
+    h->d.x_sparse_believed = sparse_x;
+    if (h->heavy_stage && d.stage_chunks != nullptr && (h->ropts.no_fused_decode == 3 || (h->ropts.no_fused_decode == 0 && !sparse_x))) {
+        // the streaming form: one persistent kernel behind a memset of y
+        const StreamLayout lay(d.nb, d.stage_bytes);
+        if (!h->stream_grid) {
+            // (the attribute belongs to the kernel, not to the handle: always the largest size)
+            DBS_CUDA(cudaFuncSetAttribute(k_decode_stream<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, STREAM_MAX_SMEM));
+            int per_sm = 0;
+            DBS_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_decode_stream<DT>, STREAM_CTA, lay.total));
+            if (per_sm < 1) return DBSPMSPV_ERR_CUDA;
+            h->stream_grid = per_sm * h->sm_count;
+        }
+        if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
+        k_fill_u32<<<(int)((d.m + 1023) / 1024), 256, 0, st>>>(reinterpret_cast<uint32_t *>(y), d.m, 0u);
+        DBS_CUDA(launch_pdl(k_decode_stream<DT>, h->stream_grid, STREAM_CTA, (size_t)lay.total, st, d, x, y, h->ropts.th3_decode, h->ropts.force_path));
+        ++h->kernel_launches;
+        if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
+        ++h->kernel_launches;
+        DBS_CUDA(cudaGetLastError());
+        return DBSPMSPV_OK;
+    }
+    if (h->heavy_stage && h->ropts.no_fused_decode != 1) {
         // one kernel for the whole call, when x fits in shared memory
         const int per_rb = d.mb ? d.n_entries / d.mb : 0;
         // warps per thread block from the entries per row block (measured on the three layer

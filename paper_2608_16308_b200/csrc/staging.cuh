@@ -47,8 +47,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // Bounded wait (each try suspends for at most ~2 us): false when the limit ran out.
 constexpr int MBAR_WAIT_LIMIT = 1 << 20;
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, int limit = MBAR_WAIT_LIMIT) {
-    for (int i = 0; i < limit; ++i)
+    for (int i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(32);             // a waiting warp leaves the issue slots to the working ones
+    }
     return false;
 }
 

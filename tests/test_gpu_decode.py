@@ -40,7 +40,7 @@ def test_decode_parity_bf16(shape, prune, zf):
     want, scale = oracle.ref_decode(ref_matrix(w), x)
     for p in PATHS:
         for thr in (1, 8):
-            for legacy in (0, 1):     # the single-kernel form (where the handle qualifies) and the general kernels
+            for legacy in (0, 3, 2, 1):  # auto / streaming / selective one-kernel forms (where the handle qualifies), general kernels
                 h.set_opts(force_path=p, popc_threshold=thr, no_fused_decode=legacy)
                 check(decode(h, x), want, scale)
                 if p != B.PATH_AUTO:
@@ -65,7 +65,7 @@ def test_decode_non_finite_activations_reach_only_stored_elements(dtype):
     want, scale = oracle.ref_decode(ref_matrix(w), x)
     nan, inf = np.isnan(want), np.isinf(want)
     assert nan.any() and inf.any() and (~nan & ~inf).any()
-    for p, legacy in [(p, l) for p in PATHS for l in (0, 1)]:
+    for p, legacy in [(p, l) for p in PATHS for l in (0, 3, 2, 1)]:
         h.set_opts(force_path=p, no_fused_decode=legacy)
         y = decode(h, x)
         assert (np.isnan(y) == nan).all()
@@ -84,7 +84,7 @@ def test_decode_wide_layer_many_entries_per_row_block():
     h = Handle(w, B.BF16)
     want, scale = oracle.ref_decode(ref_matrix(w), x)
     for p in PATHS:
-        for legacy in (0, 1):
+        for legacy in (0, 3, 2, 1):
             h.set_opts(force_path=p, no_fused_decode=legacy)
             check(decode(h, x), want, scale)
     h.close()
@@ -99,7 +99,7 @@ def test_decode_fp32_handle_small_integers_exact_and_negative_zero():
         h = Handle(w, dtype)
         want, _ = oracle.ref_decode(ref_matrix(w), x)
         for p in PATHS:
-            for legacy in (0, 1):
+            for legacy in (0, 3, 2, 1):
                 h.set_opts(force_path=p, no_fused_decode=legacy)
                 assert np.array_equal(decode(h, x).astype(np.float64), want)
         h.close()
@@ -119,6 +119,26 @@ def test_decode_all_zero_x_and_interleaving_with_run():
     xs.val = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(xs.val))
     check_against_oracle(h.run(xs), oracle.ref_pull(ref_matrix(w), xs.idx, xs.val))
     check(decode(h, x), want, scale)
+    h.close()
+
+
+def test_decode_choice_follows_the_previous_x_and_every_form_agrees():
+    """Automatic mode streams the payload unless the x of the handle's previous decode call had
+    fewer than 15 % nonzero elements; whichever form runs, the result is the oracle's -- for a
+    dense x after a sparse one and the other way round."""
+    m, n = 512, 2048
+    w = wl.pruned_weight(m, n, 0.5, seed=5, stream=31)
+    h = Handle(w, B.BF16)
+    assert h.get_stats().class_blocks[B.BLK_DENSE] + h.get_stats().class_blocks[B.BLK_FCSC] > 0
+    xs = {zf: wl.relu_activation(n, zf, seed=5, stream=70 + i) for i, zf in enumerate((0.5, 0.95, 0.99, 0.7))}
+    refs = {zf: oracle.ref_decode(ref_matrix(w), x) for zf, x in xs.items()}
+    launches = []
+    for zf in (0.5, 0.95, 0.95, 0.99, 0.7, 0.7, 0.5):
+        before = h.get_stats().kernel_launches
+        check(decode(h, xs[zf]), *refs[zf])
+        launches.append(h.get_stats().kernel_launches - before)
+    # streaming = zero kernel + stream kernel; selective = one kernel.  The call after a sparse x is selective.
+    assert launches == [2, 2, 1, 1, 1, 2, 2]
     h.close()
 
 
@@ -145,7 +165,7 @@ def test_decode_on_a_matrix_with_every_block_class(inline_max):
         h = Handle(a, dtype, opts=o)
         want, scale = oracle.ref_decode(ref_matrix(a, bf16=dtype == B.BF16), x if dtype == B.F32 else wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x)))
         for p in PATHS:
-            for legacy in (0, 1):
+            for legacy in (0, 3, 2, 1):
                 h.set_opts(force_path=p, no_fused_decode=legacy)
                 check(decode(h, x), want, scale)
         h.close()
