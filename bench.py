@@ -679,10 +679,11 @@ def other_configs(B, torch, dev, flush, peak, floors):
 
 
 def decode_bytes(wgt: wl.CSR, x: np.ndarray) -> dict:
-    """Algorithmic bytes of one decode call on a pruned bf16 layer: the whole block-CSR view
-    (the pull walks it), under every nonempty vector block the block's 48-byte header (32-byte
-    for Dense) and the 2-byte values of its active columns, x (2 bytes per entry) and y (4 per
-    row).  B_min: the CSC floor -- per active column its entries at 2 + 4 bytes, x and y."""
+    """Bytes of one decode call on a pruned bf16 layer in its selective form: the whole block-CSR
+    view (the pull walks it), under every nonempty vector block the block's 48-byte header
+    (32-byte for Dense) and the 2-byte values of its active columns, x (2 bytes per entry) and
+    y (4 per row).  (The streaming form moves the whole payload instead: see decode_layers.)
+    B_min: the CSC floor -- per active column its entries at 2 + 4 bytes, x and y."""
     m, n = wgt.m, wgt.n
     rows = wgt.rows()
     nbk = (n + 15) // 16
@@ -701,7 +702,7 @@ def decode_bytes(wgt: wl.CSR, x: np.ndarray) -> dict:
     moved = 9.0 * n_entries + 4.0 * ((m + 15) // 16 + 1) + payload + 2.0 * n + 4.0 * m
     col_nnz = np.bincount(wgt.col_idx, minlength=n)
     floor = float((8 + col_nnz[active_col] * 6).sum()) + 2.0 * n + 4.0 * m
-    return {"B_moved": int(moved), "B_min": int(floor), "payload_bytes_touched": int(payload)}
+    return {"B_moved_selective": int(moved), "B_min": int(floor), "payload_bytes_touched": int(payload), "view_entries": n_entries}
 
 
 def decode_layers(B, torch, dev, flush, peak):
@@ -723,9 +724,18 @@ def decode_layers(B, torch, dev, flush, peak):
             call = lambda: B.dbspmspv_decode(h, xd, y)
             st = stats_of(timed_calls(torch, call, flush, 12))
             warm = float(np.median(timed_calls(torch, call, flush, 10, warm=True)))
+            before = B.dbspmspv_get_stats(h).kernel_launches
+            call()
+            torch.cuda.synchronize()
             stt = B.dbspmspv_get_stats(h)
+            streamed = stt.kernel_launches - before == 2       # zero kernel + streaming kernel; the selective form is one kernel
             db = decode_bytes(wgt, wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x)))
-            rec = {"workload": f"decode_{m}x{n}_bf16_prune50_act{int(zf * 100)}zero", "path": "push" if stt.last_path == B.PATH_PUSH else "pull"}
+            # streaming form: the whole payload, the view entries with a payload (9 bytes), the
+            # chunk table (16 bytes per chunk, part of segment_bytes), x once per thread block
+            # (from L2 after the first: counted once), y zeroed and added to (4 + 8 bytes per row)
+            db["B_moved"] = int(stt.payload_bytes + 9 * db["view_entries"] + stt.segment_bytes + 2 * n + 12 * m) if streamed else db["B_moved_selective"]
+            rec = {"workload": f"decode_{m}x{n}_bf16_prune50_act{int(zf * 100)}zero", "path": "push" if stt.last_path == B.PATH_PUSH else "pull",
+                   "form": "streaming" if streamed else "selective"}
             rec.update(st)
             rec.update({"us_l2_warm": round(warm, 2), "dense_bf16_gemv_us_same_box": round(gemv, 2),
                         "format_bytes": int(stt.payload_bytes + stt.csr_view_bytes), **db,

@@ -181,6 +181,8 @@ struct Workspace {
     uint32_t *y_mask32;   // run: hit masks packed by the compaction pass; BFS: next-frontier masks
     uint8_t *y_hit8;      // run: one structural-hit flag byte per row, all zero between calls
     int32_t *tile_count;  // compaction: result entries per tile of row blocks
+    int32_t *tile_group;  // compaction: [2][n_tile_groups] totals of groups of 32 tiles, by call parity
+    int32_t n_tile_groups;
     uint32_t *visited32;  // BFS: visited masks
     uint32_t *z_mask32;   // BFS: third mask buffer (frontier / next / being cleared rotate)
     int32_t *bfs_words;   // BFS: four lists of bfs_words_stride ints: the nonzero mask words of the frontiers produced by
@@ -266,6 +268,7 @@ struct dbspmspv_handle_s {
     int grid_compute, grid_compute_dense, grid_decode_pull;
     bool lean_configured, lean_configured_dense;
     bool fused_configured[3];
+    uint32_t compact_calls;     // compaction launches so far (their parity picks the group-total buffer)
     int stream_grid;            // thread blocks of the streaming decode (0: not configured yet)
     int32_t *x_nnz_seen_host;   // host view of Device::x_nnz_seen (page-locked, mapped)
     bool heavy_stage;           // most stored elements sit in mask-based blocks: MODE 1 kernels

@@ -1587,7 +1587,7 @@ __global__ void __launch_bounds__(128) k_fold_hubs(Device d) {
     if (slot < d.n_hub_blocks) fold_hub_block(d, d.hub_rb[slot], slot, threadIdx.x & 31);
 }
 
-__global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d) {
+__global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d, int parity) {
     __shared__ int s_red[TILE_WORDS / 32];
     pdl_wait();
     pdl_launch_dependents();
@@ -1616,12 +1616,16 @@ __global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d) {
         int t = 0;
         for (int k = 0; k < TILE_WORDS / 32; ++k) t += s_red[k];
         d.ws.tile_count[blockIdx.x] = t;
+        // totals of groups of 32 tiles, so that pass 2 adds up a few dozen numbers per tile
+        // instead of one per earlier tile (all thread blocks reading the same few lines of
+        // counts was most of pass 2 on a large m: 2,100 tiles -> 2.2 M loads on 64 lines)
+        if (t) atomicAdd(d.ws.tile_group + parity * d.ws.n_tile_groups + (blockIdx.x >> 5), t);
     }
 }
 
 __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__restrict__ y_idx, float *__restrict__ y_val,
                                                            int64_t y_capacity, int32_t *__restrict__ y_nnz, int boolean,
-                                                           const int32_t *__restrict__ x_idx, int32_t nnz_x, int clear_all) {
+                                                           const int32_t *__restrict__ x_idx, int32_t nnz_x, int clear_all, int parity) {
     __shared__ int s_before[CMP_TPB / 32], s_cnt[CMP_TPB / 32];
     __shared__ int32_t s_oidx[TILE_WORDS * 32];
     __shared__ float s_oval[TILE_WORDS * 32];
@@ -1639,8 +1643,15 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
         const int wi = blockIdx.x * TILE_WORDS + (threadIdx.x >> 2);
         const int sub = threadIdx.x & 3;
         const uint32_t word = wi < n_words ? d.ws.y_mask32[wi] : 0u;
-        int before = 0;               // entries in all earlier tiles
-        for (int k = threadIdx.x; k < (int)blockIdx.x; k += CMP_TPB) before += d.ws.tile_count[k];
+        int before = 0;               // entries in all earlier tiles: whole groups of 32, then the tiles of this group
+        {
+            const int g = (int)blockIdx.x >> 5, r = (int)blockIdx.x & 31;
+            const int32_t *grp = d.ws.tile_group + parity * d.ws.n_tile_groups;
+            for (int k = threadIdx.x; k < g + r; k += CMP_TPB) before += k < g ? grp[k] : d.ws.tile_count[g * 32 + (k - g)];
+            // the group totals of the other parity served the call before: cleared for the next one
+            if (blockIdx.x == 0)
+                for (int k = threadIdx.x; k < d.ws.n_tile_groups; k += CMP_TPB) d.ws.tile_group[(parity ^ 1) * d.ws.n_tile_groups + k] = 0;
+        }
         const uint32_t bits = (word >> (8 * sub)) & 0xFFu;
         const int c = __popc(bits);
         const int row0 = wi * 32 + sub * 8;
@@ -1873,6 +1884,7 @@ int allocate_workspace(dbspmspv_handle_s *h) {
                  o_xm = carve(xwords * 4), o_ym = carve(ywords * 4), o_zm = carve(zwords * 4),
                  o_words = carve(4 * zwords * sizeof(*ws.bfs_words)), o_vis = carve((d.m == d.n ? ywords : 1) * 4),
                  o_hubs = carve((size_t)3 * HUB_CAP * sizeof(*ws.hubs)), o_tile = carve((size_t)ws.n_tiles * sizeof(*ws.tile_count)),
+                 o_group = carve((size_t)2 * ((ws.n_tiles + 31) / 32) * sizeof(*ws.tile_group)),
                  o_ctr = carve(sizeof(*ws.ctr));
     void *arena = nullptr;
     if (cudaMalloc(&arena, off) != cudaSuccess) return DBSPMSPV_ERR_ALLOC;
@@ -1891,6 +1903,8 @@ int allocate_workspace(dbspmspv_handle_s *h) {
     ws.visited32 = reinterpret_cast<decltype(ws.visited32)>(base + o_vis);
     ws.hubs = reinterpret_cast<decltype(ws.hubs)>(base + o_hubs);
     ws.tile_count = reinterpret_cast<decltype(ws.tile_count)>(base + o_tile);
+    ws.tile_group = reinterpret_cast<decltype(ws.tile_group)>(base + o_group);
+    ws.n_tile_groups = (ws.n_tiles + 31) / 32;
     ws.ctr = reinterpret_cast<decltype(ws.ctr)>(base + o_ctr);
     total = (int64_t)off;
     h->stats.workspace_bytes = total;
@@ -1954,12 +1968,13 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
     h->kernel_launches += 2;
     const int nt = d.ws.n_tiles;
-    DBS_CUDA(launch_pdl(k_compact_count, nt, TILE_WORDS, 0, st, d));
+    const int parity = (int)(++h->compact_calls & 1u);
+    DBS_CUDA(launch_pdl(k_compact_count, nt, TILE_WORDS, 0, st, d, parity));
     int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
     if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
     const int clear_all = (int64_t)nnz_x * 8 > d.n;     // scattered clears cost more than a full sweep
     DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, 0, st, d, y_idx, y_val, y_capacity, y_nnz,
-                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x, clear_all));
+                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x, clear_all, parity));
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }
