@@ -48,7 +48,9 @@ typedef enum {
     DBSPMSPV_ERR_CAPACITY = 5,    /* y_capacity too small; nothing was written out of bounds */
     DBSPMSPV_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out                   */
     DBSPMSPV_ERR_BOUNDS = 7,      /* an x index was out of range (the entry was skipped)  */
-    DBSPMSPV_ERR_TOO_LARGE = 8    /* dbspmspv_compact_noalloc: more rows than its fixed scratch covers */
+    DBSPMSPV_ERR_TOO_LARGE = 8,   /* dbspmspv_compact_noalloc: more rows than its fixed scratch covers */
+    DBSPMSPV_ERR_INTERNAL = 9     /* range-checked build only (-DDBS_BOUNDS_CHECK): an index read from the
+                                     handle's own arrays was out of range; the access was skipped   */
 } dbspmspv_status_t;
 
 typedef enum {
@@ -346,6 +348,13 @@ int dbspmspv_probe_floor(int kind, const int32_t *chain, int32_t start, int32_t 
  * `max_tries` tries (1 .. 4096, about 2 us each) and the kernel records DBSPMSPV_ERR_TIMEOUT,
  * which the next dbspmspv_get_stats returns.  The context stays usable.                       */
 int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_stream_t stream);
+
+/* Test hook of the range-checked build (-DDBS_BOUNDS_CHECK; any other build returns
+ * DBSPMSPV_ERR_UNSUPPORTED and does nothing): overwrites the other-dimension block index of
+ * block-CSR view entry `position` with `block_index` (27 bits), so that a test can show that a
+ * kernel which meets the entry records DBSPMSPV_ERR_INTERNAL and skips it.  Synchronous.  The
+ * handle is meant to be destroyed afterwards.                                                  */
+int dbspmspv_test_corrupt_entry(dbspmspv_handle_t h, int32_t position, uint32_t block_index);
 
 int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts);
 int dbspmspv_destroy(dbspmspv_handle_t h);

@@ -12,9 +12,10 @@ import os
 from typing import Optional
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libdbspmspv.so")
+# DBSPMSPV_LIBRARY: another build of the same library (the range-checked one, for the tests)
+LIB_PATH = os.environ.get("DBSPMSPV_LIBRARY") or os.path.join(HERE, "libdbspmspv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_CAPACITY, ERR_TIMEOUT, ERR_BOUNDS, ERR_TOO_LARGE = range(9)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_CAPACITY, ERR_TIMEOUT, ERR_BOUNDS, ERR_TOO_LARGE, ERR_INTERNAL = range(10)
 F32, BF16, PATTERN = 0, 1, 2
 PLUS_TIMES, OR_AND = 0, 1
 PATH_AUTO, PATH_PUSH, PATH_PULL = 0, 1, 2
@@ -28,7 +29,7 @@ EXPORTED_SYMBOLS = (
     "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "dbspmspv_decode", "dbspmspv_get_stats",
     "dbspmspv_export_coo", "dbspmspv_export_blocks", "dbspmspv_export_views",
     "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror", "dbspmspv_compact_noalloc",
-    "dbspmspv_test_bounded_wait", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
+    "dbspmspv_test_bounded_wait", "dbspmspv_test_corrupt_entry", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
 )
 
 
@@ -106,6 +107,7 @@ def lib() -> ctypes.CDLL:
         L.dbspmspv_export_views.argtypes = [vp, vp, vp, vp, vp]
         L.dbspmspv_compact_noalloc.argtypes = [vp, vp, i64, vp, vp, i64, vp, vp]
         L.dbspmspv_test_bounded_wait.argtypes = [vp, i32, vp]
+        L.dbspmspv_test_corrupt_entry.argtypes = [vp, i32, ctypes.c_uint32]
         L.dbspmspv_count_call_bytes.argtypes = [vp, vp, i32, ctypes.c_int, ctypes.POINTER(CallBytes)]
         L.dbspmspv_probe_floor.argtypes = [ctypes.c_int, vp, i32, i32, vp, vp]
         L.dbspmspv_set_run_opts.argtypes = [vp, ctypes.POINTER(RunOpts)]
@@ -229,6 +231,10 @@ def dbspmspv_compact_noalloc(acc, hit_bitmap, m, y_idx, y_val, y_capacity, y_nnz
 def dbspmspv_test_bounded_wait(h, max_tries: int, stream: Optional[int] = None) -> None:
     _check(lib().dbspmspv_test_bounded_wait(h, max_tries, _stream() if stream is None else stream),
            "dbspmspv_test_bounded_wait")
+
+
+def dbspmspv_test_corrupt_entry(h, position: int, block_index: int) -> None:
+    _check(lib().dbspmspv_test_corrupt_entry(h, position, block_index), "dbspmspv_test_corrupt_entry")
 
 
 def dbspmspv_count_call_bytes(h, x_idx, nnz_x: int, path: int) -> CallBytes:

@@ -10,6 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdbspmspv.so")
+LIB_CHECKED = os.path.join(HERE, "libdbspmspv_check.so")   # the range-checked build (-DDBS_BOUNDS_CHECK)
 SOURCES = ("create.cu", "run.cu", "bfs.cu", "api.cu", "noalloc.cu", "measure.cu")
 HEADERS = ("internal.cuh", "microkernels.cuh", "worklist.cuh", "staging.cuh", "lean_pull.cuh")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -28,16 +29,20 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
+def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compiles the sources that changed and links the library; checked=True builds the
+    range-checked variant beside it (own object files, own .so)."""
+    lib = LIB_CHECKED if checked else LIB
+    extra = ["-DDBS_BOUNDS_CHECK"] if checked else []
     deps_common = [os.path.join(CSRC, h) for h in HEADERS] + [os.path.join(ROOT, "include", "dbspmspv.h"),
                                                               os.path.abspath(__file__)]
     objs, jobs = [], []
     for src in SOURCES:
         s = os.path.join(CSRC, src)
-        o = os.path.join(CSRC, src.replace(".cu", ".o"))
+        o = os.path.join(CSRC, src.replace(".cu", ".chk.o" if checked else ".o"))
         objs.append(o)
         if force or _stale(o, [s] + deps_common):
-            cmd = [_nvcc()] + NVCC_FLAGS + os.environ.get("DBS_EXTRA_NVCC_FLAGS", "").split() \
+            cmd = [_nvcc()] + NVCC_FLAGS + extra + os.environ.get("DBS_EXTRA_NVCC_FLAGS", "").split() \
                 + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
@@ -52,10 +57,10 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
             for out in ex.map(run, jobs):
                 if verbose:
                     sys.stderr.write(out)
-    if jobs or force or _stale(LIB, objs):
-        run([_nvcc(), "-shared", "-o", LIB] + objs + ["-lcudart"])
-    return LIB
+    if jobs or force or _stale(lib, objs):
+        run([_nvcc(), "-shared", "-o", lib] + objs + ["-lcudart"])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

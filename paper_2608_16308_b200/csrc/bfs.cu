@@ -84,7 +84,11 @@ __device__ void bfs_push(const Device &d, const Scope &sc, const uint32_t *F, ui
             const int jb = (int)(task.x & IDX_MASK), start = (int)task.y;
             e.n = (int)(task.x >> 27) + 1;
             e.start = start;
-            if (lane < e.n) { e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane]; }
+            if (lane < e.n && DBS_CHK_RANGE(d, start, e.n) && DBS_CHK_INDEX(d, jb, d.nb)) {
+                e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane];
+                uint32_t w_ = d.csc.w[start + lane];
+                DBS_CHK_ENTRY(d, false, e.idx, w_, e.aux);
+            }
             e.xm = mask_of(F, jb);
         }
         return e;
@@ -176,7 +180,7 @@ __device__ void bfs_pull(const Device &d, const Scope &sc, const uint32_t *F, ui
     auto fetch = [&](const Segment &sg, uint32_t need, uint32_t (&idx)[U], uint32_t (&aux)[U]) {
         const uint32_t *ip = d.csr.idx + sg.start + lane;
         const uint8_t *ap = d.csr.aux + sg.start + lane;
-        const int rem = need ? (sg.count & 0x7FFFFFFF) - lane : 0;
+        const int rem = need && DBS_CHK_RANGE(d, sg.start, sg.count & 0x7FFFFFFF) ? (sg.count & 0x7FFFFFFF) - lane : 0;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             idx[u] = 0; aux[u] = 0;
@@ -306,7 +310,8 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             const int pbeg = d.csr.ptr[rb], pend = d.csr_inl[rb];      // the row block's entries with a payload
             uint32_t hit = 0;
             for (int pos = pbeg + lane; pos < pend; pos += 32) {
-                const uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
+                uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
+                { uint32_t w_ = d.csr.w[pos]; DBS_CHK_ENTRY(d, true, idx, w_, aux); }
                 const uint32_t xm = mask_of(F, idx & IDX_MASK);
                 if (xm) {
                     const int type = idx >> TYPE_SHIFT;
@@ -331,7 +336,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             if (active) v4 = __ldcs(reinterpret_cast<const uint4 *>(d.rowrun_idx + q0));     // (the array has slack behind its end)
             uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w}, xm[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) if (q0 + j < p || q0 + j >= e) v[j] = NONE;
+            for (int j = 0; j < 4; ++j) if (q0 + j < p || q0 + j >= e || (v[j] != NONE && !DBS_CHK_INDEX(d, v[j] & IDX_MASK, d.nb))) v[j] = NONE;
 #pragma unroll
             for (int j = 0; j < 4; ++j) xm[j] = v[j] != NONE ? mask_of(F, v[j] & IDX_MASK) : 0u;
 #pragma unroll
@@ -346,7 +351,8 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             const int lp = __shfl_sync(FULL, p, src), le = __shfl_sync(FULL, e, src);
             bool hit = false;
             for (int q = lp; q < le && !hit; q += 32) {
-                const uint32_t v = q + lane < le ? d.rowrun_idx[q + lane] : NONE;
+                uint32_t v = q + lane < le ? d.rowrun_idx[q + lane] : NONE;
+                if (v != NONE && !DBS_CHK_INDEX(d, v & IDX_MASK, d.nb)) v = NONE;
                 const uint32_t xm = v != NONE ? mask_of(F, v & IDX_MASK) : 0u;
                 hit = __any_sync(FULL, (xm >> (v >> 27)) & 1u);
             }

@@ -818,7 +818,7 @@ int build(dbspmspv_handle_s *h, int64_t m, int64_t n, int64_t nnz, const int64_t
     {
         uint8_t *p; DBS_KEEP(p, h->payload_bytes + 256);  // slack: staged copies may over-read
         DBS_CUDA(cudaMemsetAsync(p, 0, h->payload_bytes + 256, st));
-        h->payload_alloc = p; d.payload = p;
+        h->payload_alloc = p; d.payload = p; d.payload_words = (uint32_t)total_words;
     }
     // class census -> which kernel variant the handle uses, hence what a mask-based block costs
     unsigned long long cls_h[2 * DBSPMSPV_BLK_NCLASS];

@@ -201,6 +201,7 @@ struct Device {           // everything the kernels need, passed by value
     int32_t dtype;
     View csr, csc;
     const uint8_t *payload;
+    uint32_t payload_words;   // its size in 4-byte words
     const Segment *segments;
     const int32_t *seg_rb;  // row block of every segment (compact copy for the pull kernel)
     const int2 *chunks;   // n_chunks + 1: {first segment, first entry} of every pull chunk
@@ -310,6 +311,39 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Range-checked build (-DDBS_BOUNDS_CHECK; it stands in for a memory checker on the small parity
+// cases): every index that a kernel READS from the handle's arrays -- the other-dimension block
+// index and the payload offset of a view entry, the entry range of a task, a column run, a
+// segment or a chunk, a listed row -- is tested before it is used; a violation records
+// DBSPMSPV_ERR_INTERNAL in the status word and the access is skipped (the entry is replaced
+// by a harmless one, the range is emptied).  Nothing traps.  In the normal build these compile to nothing.
+#ifdef DBS_BOUNDS_CHECK
+__device__ __forceinline__ bool chk_fail(const Device &d) { d.ws.ctr->status = DBSPMSPV_ERR_INTERNAL; return false; }
+__device__ __forceinline__ bool chk_index(const Device &d, int64_t i, int64_t n) { return (i >= 0 && i < n) || chk_fail(d); }
+// entries [first, first + count) of a view
+__device__ __forceinline__ bool chk_range(const Device &d, int64_t first, int64_t count) {
+    return (first >= 0 && count >= 0 && first + count <= (int64_t)d.n_entries) || chk_fail(d);
+}
+// a view entry as loaded: one that points outside the handle is replaced by an INLINE element
+// (0, 0) of block 0 with the value 0 -- every access it leads to is in range
+template <typename A>
+__device__ __forceinline__ void chk_entry(const Device &d, bool csr_view, uint32_t &idx, uint32_t &w, A &aux) {
+    const int type = (int)(idx >> TYPE_SHIFT);
+    if (type == 7) return;                                       // padding behind the last entry
+    const int vsize = d.dtype == DBSPMSPV_F32 ? 4 : d.dtype == DBSPMSPV_BF16 ? 2 : 0;
+    bool ok = (int)(idx & IDX_MASK) < (csr_view ? d.nb : d.mb) && type <= BLK_CSR_ROWMAJOR;
+    if (ok && type != DBSPMSPV_BLK_INLINE) ok = (uint64_t)w + (uint64_t)payload_words(type, (int)aux + 1, vsize) <= (uint64_t)d.payload_words;
+    if (!ok) { chk_fail(d); idx = (uint32_t)DBSPMSPV_BLK_INLINE << TYPE_SHIFT; w = 0u; aux = 0; }
+}
+#define DBS_CHK_INDEX(d, i, n) dbs::chk_index((d), (int64_t)(i), (int64_t)(n))
+#define DBS_CHK_RANGE(d, first, count) dbs::chk_range((d), (int64_t)(first), (int64_t)(count))
+#define DBS_CHK_ENTRY(d, csr_view, idx, w, aux) dbs::chk_entry((d), (csr_view), (idx), (w), (aux))
+#else
+#define DBS_CHK_INDEX(d, i, n) true
+#define DBS_CHK_RANGE(d, first, count) true
+#define DBS_CHK_ENTRY(d, csr_view, idx, w, aux) ((void)0)
+#endif
 
 // 16-bit mask of one block.  The mask arrays are updated as 32-bit words (two blocks per word,
 // the even block in the low half: atomics need the word) but read as the halfword itself: one

@@ -136,7 +136,7 @@ __device__ __forceinline__ void lean_chunk(const Device &d, Out out, const LeanR
 #pragma unroll
     for (int k = 0; k < K; ++k) {
         // INLINE is class 0: any other entry (a block with a payload, the slack) is skipped here
-        bool go = idx[k] < (1u << TYPE_SHIFT);
+        bool go = idx[k] < (1u << TYPE_SHIFT) && DBS_CHK_INDEX(d, idx[k] & IDX_MASK, d.nb);
         const uint32_t a = k < 4 ? r.a.x : r.a.y;
         const uint32_t col = (idx[k] & IDX_MASK) * 16u + ((a >> (8 * (k & 3))) & 15u);
 #if DBS_LEAN_FILTER
@@ -261,7 +261,13 @@ k_pull_lean(Device d, Out out, float th3, int force_path, int popc_threshold, in
     // entries with a payload: one block per warp at a time (they are the exception in these handles)
     for (int q = gwarp; q < d.n_payload; q += nwarps) {
         const int pos = d.payload_pos[q];
-        const uint32_t idx = d.csr.idx[pos];
+        if (!DBS_CHK_INDEX(d, pos, d.n_entries)) continue;            // warp-uniform
+        uint32_t idx = d.csr.idx[pos];
+        {
+            uint32_t w_ = d.csr.w[pos], a_ = d.csr.aux[pos];
+            DBS_CHK_ENTRY(d, true, idx, w_, a_);
+            if ((idx >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE || !DBS_CHK_INDEX(d, d.entry_row[pos], d.mb)) continue;   // (only a replaced entry is INLINE here)
+        }
         const int cb = idx & IDX_MASK, type = idx >> TYPE_SHIFT;
         const uint32_t xm = mask_of(d.ws.x_mask32, cb);
         if (!xm) continue;                                            // warp-uniform

@@ -292,6 +292,7 @@ template <typename Out>
 __device__ __forceinline__ bool push_private(const Device &d, uint32_t idx, uint32_t aux, float prod) {
     if (!Out::MASKS || !d.hub_on || !(idx & HUB_FLAG) || !(fabsf(prod) >= 1.17549435e-38f)) return false;
     const int slot = d.hub_slot[idx & IDX_MASK];
+    if (!DBS_CHK_INDEX(d, slot, d.n_hub_blocks)) return false;
     atomicAdd(d.hub_acc + (((size_t)(blockIdx.x & (HUB_COPIES - 1)) * d.n_hub_blocks + slot) * 16 + (aux >> 4)), prod);
     return true;
 }
@@ -324,7 +325,10 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
             l.jb = jb;
             const int cnt = (int)(task.x >> 27) + 1;              // entries of the task
             l.start = (int)task.y;
-            if (lane < cnt) { const int p = l.start + lane; l.idx = d.csc.idx[p]; l.w = d.csc.w[p]; l.aux = d.csc.aux[p]; }
+            if (lane < cnt && DBS_CHK_RANGE(d, l.start, cnt) && DBS_CHK_INDEX(d, jb, d.nb)) {
+                const int p = l.start + lane; l.idx = d.csc.idx[p]; l.w = d.csc.w[p]; l.aux = d.csc.aux[p];
+                DBS_CHK_ENTRY(d, false, l.idx, l.w, l.aux);
+            }
             l.end = l.start + cnt;
             l.xm = mask_of(d.ws.x_mask32, jb);
             if (lane < 16) l.xv = d.ws.x_dense[jb * 16 + lane];
@@ -487,7 +491,7 @@ constexpr uint32_t SEG_FLAG = 1u << 28;   // view entry starts a pull segment (b
 // lane 0 issues the copies of the chunk [e0, e1) into stage st
 __device__ __forceinline__ void pull_issue(const Device &d, int e0, int e1, PullStage *st, uint64_t *bar, int lane) {
     const int a0 = e0 & ~15, a1 = (e1 + 15) & ~15;
-    if (lane == 0 && e1 > e0) {      // same condition as the consumer's wait
+    if (lane == 0 && e1 > e0 && DBS_CHK_RANGE(d, e0, e1 - e0)) {      // same condition as the consumer's wait
         const uint32_t n = (uint32_t)(a1 - a0);
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(bar, n * 9u);
@@ -546,7 +550,7 @@ __device__ void pull_body(const Device &d, Out out, int popc_threshold, float *s
             for (int u = 0; u < PULL_UNROLL; ++u) {
                 const int p = base + u * 32 + lane;
                 idx[u] = 0; w[u] = 0; aux[u] = 0;
-                if (p < e1) { const int o = p - a0; idx[u] = st->idx[o]; w[u] = st->w[o]; aux[u] = st->aux[o]; }
+                if (p < e1) { const int o = p - a0; idx[u] = st->idx[o]; w[u] = st->w[o]; aux[u] = st->aux[o]; DBS_CHK_ENTRY(d, true, idx[u], w[u], aux[u]); }
             }
 #pragma unroll
             for (int u = 0; u < PULL_UNROLL; ++u) {
@@ -932,7 +936,12 @@ __global__ void __launch_bounds__(CTA) k_decode_pull(Device d, const int32_t *__
         const bool have = p < d.n_entries;
         uint32_t idx = 0, w = 0, aux = 0, xm = 0;
         int rb = -1;
-        if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; rb = entry_row[p]; xm = mask_of(d.ws.x_mask32, idx & IDX_MASK); }
+        if (have) {
+            idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; rb = entry_row[p];
+            DBS_CHK_ENTRY(d, true, idx, w, aux);
+            if (!DBS_CHK_INDEX(d, rb, d.mb)) rb = 0;
+            xm = mask_of(d.ws.x_mask32, idx & IDX_MASK);
+        }
         const int type = idx >> TYPE_SHIFT;
         const bool mk = have && xm && type > DBSPMSPV_BLK_COO;
         const bool rowm = mk && is_row_major(type);
@@ -1240,7 +1249,7 @@ k_decode_fused(Device d, const void *__restrict__ x, float *__restrict__ y, floa
     };
     auto fetch = [&](int p, bool have, uint32_t &idx, uint32_t &w, uint32_t &aux) {
         idx = 0; w = 0; aux = 0;
-        if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; }
+        if (have && DBS_CHK_INDEX(d, p, d.n_entries)) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; DBS_CHK_ENTRY(d, true, idx, w, aux); }
     };
     if (path == DBSPMSPV_PATH_PULL) {
         // the next step's entries are fetched before this step's blocks are worked on
@@ -1366,16 +1375,22 @@ k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, flo
     // descriptor: x = first view entry, y = row block, z = payload offset in words, w = words | entries << 24
     auto issue = [&](const int4 &ch, int st) {               // lane 0 only
         uint8_t *base = s_ring + (size_t)st * stride;
-        const uint32_t pb = ((uint32_t)ch.w & 0xFFFFFFu) * 4u;
+        uint32_t pb = ((uint32_t)ch.w & 0xFFFFFFu) * 4u;
+        if (!DBS_CHK_INDEX(d, pb, d.stage_bytes + 1) || !DBS_CHK_INDEX(d, (uint64_t)(uint32_t)ch.z + (pb >> 2), (uint64_t)d.payload_words + 1)) pb = 0u;
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(&s_bar[st], pb);
-        bulk_copy_g2s(base, d.payload + (size_t)(uint32_t)ch.z * 4, pb, &s_bar[st]);
+        if (pb) bulk_copy_g2s(base, d.payload + (size_t)(uint32_t)ch.z * 4, pb, &s_bar[st]);
     };
     // the chunk's view entries, one per lane, by plain loads a round ahead of their use (they
     // are 9 bytes per block; bulk copies of 48-256 bytes cost the copy engine as much as the payload's)
     auto entries_of = [&](const int4 &ch, uint32_t &idx, uint32_t &w, uint32_t &aux) {
         idx = 0; w = 0; aux = 0;
-        if (lane < (int)((uint32_t)ch.w >> 24)) { const int p_ = ch.x + lane; idx = d.csr.idx[p_]; w = d.csr.w[p_]; aux = d.csr.aux[p_]; }
+        if (lane < (int)((uint32_t)ch.w >> 24) && DBS_CHK_RANGE(d, ch.x, (uint32_t)ch.w >> 24)) {
+            const int p_ = ch.x + lane; idx = d.csr.idx[p_]; w = d.csr.w[p_]; aux = d.csr.aux[p_];
+            DBS_CHK_ENTRY(d, true, idx, w, aux);
+            // (the staged copy holds exactly the chunk's words: the block must start inside them)
+            if ((idx >> TYPE_SHIFT) != DBSPMSPV_BLK_INLINE && !DBS_CHK_INDEX(d, (int64_t)w - (uint32_t)ch.z, (uint32_t)ch.w & 0xFFFFFFu)) { idx = 0u; w = 0u; aux = 0u; }
+        }
     };
     int issued = 0;                                           // chunks of mine whose copies were started
     if (lane == 0) {
@@ -1449,7 +1464,7 @@ k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, flo
     };
     auto fetch = [&](int p, bool have, uint32_t &idx, uint32_t &w, uint32_t &aux) {
         idx = 0; w = 0; aux = 0;
-        if (have) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; }
+        if (have && DBS_CHK_INDEX(d, p, d.n_entries)) { idx = d.csr.idx[p]; w = d.csr.w[p]; aux = d.csr.aux[p]; DBS_CHK_ENTRY(d, true, idx, w, aux); }
     };
 
     if (path == DBSPMSPV_PATH_PULL) {
@@ -1468,7 +1483,7 @@ k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, flo
             n_idx = 0; n_w = 0; n_aux = 0;
             if (k + 1 < n_mine && ((k + 1) & 31)) entries_of(desc_of(k + 1), n_idx, n_w, n_aux);
             if (!mbar_wait_bounded(&s_bar[st], (uint32_t)(k / STREAM_DEPTH) & 1u)) { timed_out = true; break; }
-            if (ch.y != cur_rb) { flush(); cur_rb = ch.y; }
+            if (ch.y != cur_rb) { flush(); cur_rb = DBS_CHK_INDEX(d, ch.y, d.mb) ? ch.y : 0; }
             const uint8_t *base = s_ring + (size_t)st * stride;
             step(base - (size_t)(uint32_t)ch.z * 4, idx, w, aux, lane < (int)((uint32_t)ch.w >> 24));
             __syncwarp();
@@ -1584,7 +1599,7 @@ __global__ void __launch_bounds__(128) k_fold_hubs(Device d) {
     pdl_wait();
     pdl_launch_dependents();
     const int slot = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (slot < d.n_hub_blocks) fold_hub_block(d, d.hub_rb[slot], slot, threadIdx.x & 31);
+    if (slot < d.n_hub_blocks && DBS_CHK_INDEX(d, d.hub_rb[slot], d.mb)) fold_hub_block(d, d.hub_rb[slot], slot, threadIdx.x & 31);
 }
 
 __global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d, int parity) {
@@ -2133,6 +2148,21 @@ int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_
     ++h->kernel_launches;
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
+}
+
+int dbspmspv_test_corrupt_entry(dbspmspv_handle_t h, int32_t position, uint32_t block_index) {
+#ifdef DBS_BOUNDS_CHECK
+    if (!h || position < 0 || position >= h->d.n_entries || block_index > dbs::IDX_MASK) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
+    uint32_t v = 0;
+    DBS_CUDA(cudaMemcpy(&v, h->d.csr.idx + position, 4, cudaMemcpyDeviceToHost));
+    v = (v & ~dbs::IDX_MASK) | block_index;
+    DBS_CUDA(cudaMemcpy(h->d.csr.idx + position, &v, 4, cudaMemcpyHostToDevice));
+    return DBSPMSPV_OK;
+#else
+    (void)h; (void)position; (void)block_index;
+    return DBSPMSPV_ERR_UNSUPPORTED;
+#endif
 }
 
 int dbspmspv_decode(dbspmspv_handle_t h, const void *x, float *y, dbspmspv_stream_t stream) {

@@ -122,11 +122,13 @@ __device__ __forceinline__ uint2 worklist_item(const uint2 *tasks, int n_tasks, 
 __device__ __forceinline__ void payload_run(const Device &d, int jb, int &first, int &deg) {
     first = d.csc.ptr[jb];
     deg = d.csc.colptr[17 * jb] - first;
+    if (!DBS_CHK_RANGE(d, first, deg)) deg = 0;
 }
 __device__ __forceinline__ void column_run(const Device &d, int j, int &first, int &deg) {
     const int32_t *cp = d.csc.colptr + 17 * (j >> 4) + (j & 15);
     first = cp[0];
     deg = cp[1] - first;
+    if (!DBS_CHK_RANGE(d, first, deg)) deg = 0;
 }
 
 // Runs of consecutive columns of one column block are adjacent in the view, so lanes that hold

@@ -1,5 +1,7 @@
 """Helpers shared by the GPU parity tests: upload a generated matrix, call the C ABI through
 the binding, fetch results, and compare against the CPU oracle."""
+import os
+
 import numpy as np
 import torch
 
@@ -104,6 +106,10 @@ class Handle:
 
     def close(self):
         if self.h:
+            if os.environ.get("DBSPMSPV_LIBRARY"):
+                # a run with the range-checked library: no kernel may have met a bad index
+                st = B.dbspmspv_get_stats(self.h, raise_on_device_status=False)
+                assert st.device_status != B.ERR_INTERNAL, "range check failed inside a kernel"
             B.dbspmspv_destroy(self.h)
             self.h = None
 
