@@ -211,13 +211,19 @@ def fractions(nbytes: float, us: float, peak: float) -> dict:
 
 
 def ncu_traffic(name: str):
-    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
-    summary the profiling command wrote under profiles/ (None when there is none)."""
-    p = os.path.join(ROOT, "profiles", name)
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, parsed from
+    the text summary of its ncu capture under profiles/ (None when there is none)."""
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    total, seen = 0.0, 0
     try:
-        return int(json.load(open(p))["dram_bytes_per_launch"])
-    except Exception:
+        for line in open(os.path.join(ROOT, "profiles", name)):
+            f = line.split()
+            if len(f) == 3 and f[0] in ("dram__bytes_read.sum", "dram__bytes_write.sum") and f[1] in scale:
+                total += float(f[2]) * scale[f[1]]
+                seen += 1
+    except OSError:
         return None
+    return int(total) if seen == 2 else None
 
 
 # ---------------------------------------------------------------------------------------------
@@ -506,7 +512,7 @@ def main() -> None:
     achieved = b_kernel_dom / (kernel_dom_ms * 1e-3) / 1e9
     dom_pull = info[kdom][0] == B.PATH_PULL
     dom_name = "k_pull_lean" if dom_pull else "k_compute"
-    traffic = ncu_traffic("k_pull_lean_rmat20_x50pct.json" if dom_pull else "k_compute_push_rmat20_x10pct.json")
+    traffic = ncu_traffic("k_pull_lean_rmat20_x50pct.txt" if dom_pull else "k_compute_push_rmat20_x10pct.txt")
     line = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
