@@ -104,7 +104,7 @@ typedef struct {
 /* Run-time options; may be changed between calls with dbspmspv_set_run_opts.               */
 typedef struct {
     float th3;               /* dbspmspv_run: push iff the nonempty-vector-block ratio is
-                                below th3.  0.01 in the paper; default 0.9, the crossover
+                                below th3.  0.01 in the paper; default 0.95, the crossover
                                 measured on B200 (the table `bench.py --crossover` prints)    */
     int32_t force_path;      /* DBSPMSPV_PATH_*                                              */
     int32_t popc_threshold;  /* CSR-class blocks: popc(mask) >= this -> row-driven (pull-style)

@@ -2100,7 +2100,7 @@ extern "C" {
 void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     if (!o) return;
     *o = dbspmspv_run_opts();
-    o->th3 = 0.9f;
+    o->th3 = 0.95f;
     o->th3_bfs = 0.05f;
     o->th3_decode = 0.01f;
     o->bfs_push_max_edge_frac = 0.f;
