@@ -12,10 +12,10 @@
 //     column) in shared memory and tests it before every gather: an absent x_j costs a
 //     shared-memory load instead of a trip through the L1 tag stage, which is what bounds this
 //     kernel (one 4-byte gather per stored element, one cache line each).
-//   * A warp pass covers one chunk, eight CONSECUTIVE entries per lane (16-byte shared-memory
-//     loads).  A lane gathers its four x entries (one load each: the dense
-//     copy of x carries a "not listed" marker), multiplies, and sums runs of equal row inside
-//     its eight entries in registers; ROW_FLAG in the entry marks where a row starts.
+//   * A warp pass covers one chunk, eight CONSECUTIVE entries per lane.  A lane gathers the x
+//     entries that pass the filter (one load each: the dense copy of x carries a "not listed"
+//     marker), multiplies, and sums runs of equal row inside its eight entries in registers;
+//     ROW_FLAG in the entry marks where a row starts.
 //   * Across the lanes a segmented shuffle scan adds up the pieces of every row that spans
 //     several lanes (Section 3.3.3: registers, then warp shuffle), and one lane per row adds the
 //     sum to global memory -- a row cut by a pass or chunk boundary simply contributes one atomic
