@@ -296,18 +296,32 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
         if (lane < n_batch) words_out[base + lane] = batch_wd;
         n_batch = 0;
     };
+    // A word is a chain of dependent loads (visited word -> row pointers -> entries -> frontier
+    // masks): the visited word of the warp's next word is fetched a word ahead, and all pointers
+    // of a word -- both row blocks' payload ranges and the lane's row run -- in one round.
+    uint32_t need_next = gwarp < n_words ? ~d.ws.visited32[gwarp] : 0u;
     for (int wd = gwarp; wd < n_words; wd += nwarps) {
-        const uint32_t need = ~d.ws.visited32[wd];   // (rows without stored elements and rows past m count as visited)
+        const uint32_t need = need_next;             // (rows without stored elements and rows past m count as visited)
+        if (wd + nwarps < n_words) need_next = ~d.ws.visited32[wd + nwarps];
         if (lane == 0) Z[wd] = 0u;
         if (!need) { if (lane == 0) N[wd] = 0u; continue; }
         uint32_t found = 0;
+        const int row = wd * 32 + lane;
+        int p = 0, e = 0;
+        if ((need >> lane) & 1u) { p = d.rowrun_ptr[row]; e = d.rowrun_ptr[row + 1]; }
+        int pb2[2] = {0, 0}, pe2[2] = {0, 0};
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            const int rb = 2 * wd + hf;
+            if (rb < d.mb && ((need >> (16 * hf)) & 0xFFFFu)) { pb2[hf] = d.csr.ptr[rb]; pe2[hf] = d.csr_inl[rb]; }
+        }
         // entries with a payload, one per lane
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
             const int rb = 2 * wd + hf;
             const uint32_t need16 = (need >> (16 * hf)) & 0xFFFFu;
             if (rb >= d.mb || !need16) continue;    // warp-uniform
-            const int pbeg = d.csr.ptr[rb], pend = d.csr_inl[rb];      // the row block's entries with a payload
+            const int pbeg = pb2[hf], pend = pe2[hf];                  // the row block's entries with a payload
             uint32_t hit = 0;
             for (int pos = pbeg + lane; pos < pend; pos += 32) {
                 uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
@@ -323,10 +337,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             if (pend > pbeg) found |= (__reduce_or_sync(FULL, hit) & need16) << (16 * hf);
         }
         // row runs
-        const int row = wd * 32 + lane;
-        bool active = ((need & ~found) >> lane) & 1u;
-        int p = 0, e = 0;
-        if (active) { p = d.rowrun_ptr[row]; e = d.rowrun_ptr[row + 1]; active = p < e; }
+        bool active = (((need & ~found) >> lane) & 1u) && p < e;
         bool got = false;
         // a round = the aligned group of four entries that holds position p: one 16-byte load per
         // lane (four 4-byte loads cost four trips through the L1 tag stage for the same line)
