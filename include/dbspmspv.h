@@ -138,7 +138,11 @@ typedef struct {
     int32_t hub_min_nnz_x;   /* dbspmspv_run: shortest x list for which the push adds into the
                                 private accumulators of hub row blocks (they cost one more
                                 kernel in the chain); 0 = default (32768), < 0 = never     */
-    int32_t reserved[6];
+    float decode_threshold;  /* dbspmspv_decode: activation magnitude cut fused into the vector
+                                blocking (Section 5.3: activation sparsity by magnitude
+                                thresholding) -- x_j takes part iff |x_j| > decode_threshold;
+                                0 (default): iff x_j is not zero.  A NaN always takes part.  */
+    int32_t reserved[5];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64

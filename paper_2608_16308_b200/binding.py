@@ -49,7 +49,7 @@ class RunOpts(ctypes.Structure):
                 ("timing", ctypes.c_int32), ("th3_bfs", ctypes.c_float),
                 ("th3_decode", ctypes.c_float), ("no_fused_decode", ctypes.c_int32),
                 ("bfs_push_max_edge_frac", ctypes.c_float), ("hub_min_nnz_x", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 6)]
+                ("decode_threshold", ctypes.c_float), ("reserved", ctypes.c_int32 * 5)]
 
 
 class Stats(ctypes.Structure):

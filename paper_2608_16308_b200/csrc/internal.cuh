@@ -234,6 +234,7 @@ struct Device {           // everything the kernels need, passed by value
     int32_t n_stage_chunks;
     int32_t stage_bytes;        // payload bytes of one stage (a multiple of 512)
     int32_t has_inline;         // the handle holds INLINE elements at all
+    float decode_tau;           // per call: activation magnitude cut of dbspmspv_decode (run option)
     int32_t x_sparse_believed;  // per call: what the host currently takes x for (1: sparse)
     int32_t *x_nnz_seen;        // mapped host word: nonzero elements of the x of the last single-kernel decode (null: none)
     // Hub row blocks (null / 0 when the matrix has none): hub_slot[rb] = slot of row block rb or

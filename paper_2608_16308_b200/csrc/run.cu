@@ -134,14 +134,16 @@ __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__re
         float v = 0.f;
         if (j < d.n) v = DT == DBSPMSPV_BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(x)[j])
                                              : static_cast<const float *>(x)[j];
+        // an entry takes part iff |x_j| > tau (tau = 0: iff it is not zero; a NaN always does)
+        const bool in = !(fabsf(v) <= d.decode_tau);
         if (j < (int64_t)d.nb * 16)
-            d.ws.x_dense[j] = v != 0.0f ? (__float_as_uint(v) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v)
-                                        : __uint_as_float(X_ABSENT);
-        const uint32_t bits = __ballot_sync(FULL, v != 0.0f);
+            d.ws.x_dense[j] = in ? (__float_as_uint(v) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v)
+                                 : __uint_as_float(X_ABSENT);
+        const uint32_t bits = __ballot_sync(FULL, in);
         if (lane == 0) d.ws.x_mask32[j >> 5] = bits;
         const bool newly = (lane == 0 && (bits & 0xFFFFu)) || (lane == 16 && (bits >> 16));
         int first = 0, deg = 0;
-        const bool listed = v != 0.0f && j < d.n;
+        const bool listed = in && j < d.n;
         if (d.payload_chunk == PUSH_CHUNK) {                 // whole column blocks, as in the sparse-x kernel
             if (newly) { first = d.csc.ptr[j >> 4]; deg = d.csc.ptr[(j >> 4) + 1] - first; }
             emit_tasks(d, newly, (int)(j >> 4), first, deg, lane, &d.ws.ctr->n_tasks, &d.ws.ctr->n_nzblk, PUSH_CHUNK, &d.ws.ctr->n_hubs, d.ws.hubs);
@@ -1122,7 +1124,7 @@ __device__ __forceinline__ void stage_x_blocks(const Device &d, const void *__re
         uint32_t bits = 0;
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
-            const bool nz = v[k] != 0.0f;
+            const bool nz = !(fabsf(v[k]) <= d.decode_tau);      // |x_j| > tau; tau = 0: not zero; NaN takes part
             bits |= (nz ? 1u : 0u) << k;
             // (a widened bf16 has zero low bits: it cannot collide with the marker)
             if (DT != DBSPMSPV_BF16 && __float_as_uint(v[k]) == X_ABSENT) v[k] = __uint_as_float(0x7FC00000u);
@@ -2011,6 +2013,7 @@ int decode_stage_bytes(const Device &d) {
 template <int DT>
 static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStream_t st) {
     const Device &d = h->d;
+    h->d.decode_tau = h->ropts.decode_threshold;
     // (-1: no decode call has reported yet)
     const int seen = h->x_nnz_seen_host ? *const_cast<volatile int32_t *>(h->x_nnz_seen_host) : -1;
     const bool sparse_x = seen >= 0 && (float)seen < STREAM_MIN_X_DENSITY * (float)d.n;
@@ -2112,7 +2115,8 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
 int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts) {
     if (!h || !opts) return DBSPMSPV_ERR_INVALID_ARG;
     if (opts->force_path < DBSPMSPV_PATH_AUTO || opts->force_path > DBSPMSPV_PATH_PULL) return DBSPMSPV_ERR_INVALID_ARG;
-    if (!(opts->th3 >= 0.f) || !(opts->th3_bfs >= 0.f) || !(opts->th3_decode >= 0.f) || !(opts->bfs_push_max_edge_frac >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!(opts->th3 >= 0.f) || !(opts->th3_bfs >= 0.f) || !(opts->th3_decode >= 0.f) || !(opts->bfs_push_max_edge_frac >= 0.f) ||
+        !(opts->decode_threshold >= 0.f)) return DBSPMSPV_ERR_INVALID_ARG;
     h->ropts = *opts;
     return DBSPMSPV_OK;
 }

@@ -142,6 +142,31 @@ def test_decode_choice_follows_the_previous_x_and_every_form_agrees():
     h.close()
 
 
+@pytest.mark.parametrize("dtype", [B.BF16, B.F32])
+def test_decode_magnitude_threshold_is_fused_into_the_blocking(dtype):
+    """decode_threshold = tau: x_j takes part iff |x_j| > tau (Section 5.3's activation sparsity
+    by magnitude thresholding), on a dense activation vector without a single zero; every form
+    and path must equal the oracle run on the thresholded vector."""
+    m, n = 512, 1024
+    w = wl.pruned_weight(m, n, 0.5, seed=5, stream=41)
+    x = wl.rand_normal_f32(5, 77, np.arange(n, dtype=np.uint64))
+    assert (x != 0).all()
+    xr = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x)) if dtype == B.BF16 else x
+    h = Handle(w, dtype)
+    for keep in (0.1, 0.6):
+        tau = float(np.quantile(np.abs(xr), 1.0 - keep))
+        xt = np.where(np.abs(xr) > np.float32(tau), xr, 0.0).astype(np.float32)
+        want, scale = oracle.ref_decode(ref_matrix(w, bf16=dtype == B.BF16), xt)
+        for p in PATHS:
+            for legacy in (0, 3, 2, 1):
+                h.set_opts(force_path=p, no_fused_decode=legacy, decode_threshold=tau)
+                check(decode(h, x), want, scale)
+        assert h.get_stats().last_n_nzblk == int((xt.reshape(-1, 16) != 0).any(axis=1).sum())
+    with pytest.raises(B.DbSpmspvError):
+        h.set_opts(decode_threshold=-1.0)
+    h.close()
+
+
 def test_decode_rejects_pattern_handles():
     h = Handle(wl.random_sparse(32, 32, 50, 1, values=False), B.PATTERN)
     t = torch.zeros(32, device=DEV)
