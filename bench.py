@@ -357,7 +357,7 @@ def main() -> None:
             if args.bfs_only:
                 print(json.dumps(bench_bfs(args, B, torch, dev, flush, peak)))
             elif args.decode_only:
-                print(json.dumps(decode_layers(B, torch, dev, flush, peak)))
+                print(json.dumps(decode_layers(B, torch, dev, flush, peak) + [decode_chain(B, torch, dev, flush)]))
             else:
                 print(json.dumps({"format_ablation": format_ablation(B, torch, dev, flush), "storage": storage_table(B, torch, dev)}))
         return
@@ -681,6 +681,7 @@ def other_configs(B, torch, dev, flush, peak, floors):
                                                  ("5 % in runs of 64", wl.clustered_x(a3.n, 3200))])
     del a3
     out += decode_layers(B, torch, dev, flush, peak)
+    out.append(decode_chain(B, torch, dev, flush))
     return out
 
 
@@ -709,6 +710,58 @@ def decode_bytes(wgt: wl.CSR, x: np.ndarray) -> dict:
     col_nnz = np.bincount(wgt.col_idx, minlength=n)
     floor = float((8 + col_nnz[active_col] * 6).sum()) + 2.0 * n + 4.0 * m
     return {"B_moved_selective": int(moved), "B_min": int(floor), "payload_bytes_touched": int(payload), "view_entries": n_entries}
+
+
+def decode_chain(B, torch, dev, flush):
+    """A feed-forward pair chained on the device (Section 4.3 / 5.3): up projection 11008x4096,
+    then down projection 4096x11008 whose x is the up projection's fp32 y with ReLU and a
+    magnitude cut fused into the blocking (cut chosen for 10 % dense activations) -- two
+    dbspmspv_decode calls, nothing in between.  Beside it: two dense bf16 GEMVs of the same
+    shapes with torch's relu / cut / cast between them."""
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    n0, n1 = 4096, 11008
+    hs = []
+    for (m, n, stream) in ((n1, n0, 0), (n0, n1, 1)):
+        wgt = wl.pruned_weight(m, n, 0.5, stream=stream)
+        bits = wl.f32_to_bf16_bits(wgt.val).view(np.int16)
+        hs.append(B.dbspmspv_create_csr(wgt.m, wgt.n, wgt.nnz, up(wgt.row_ptr), up(wgt.col_idx), up(bits), B.BF16))
+        del wgt
+    h_up, h_down = hs
+    x0 = up(wl.f32_to_bf16_bits(wl.relu_activation(n0, 0.9)).view(np.int16))
+    y1 = torch.empty(n1, dtype=torch.float32, device=dev)
+    y2 = torch.empty(n0, dtype=torch.float32, device=dev)
+    B.dbspmspv_decode(h_up, x0, y1)
+    torch.cuda.synchronize()
+    y1h = y1.cpu().numpy()
+    tau = float(np.quantile(y1h, 0.9))                       # 10 % of the entries lie above it
+    o = B.default_run_opts()
+    o.decode_x_f32, o.decode_relu, o.decode_threshold = 1, 1, max(tau, 0.0)
+    B.dbspmspv_set_run_opts(h_down, o)
+
+    def chain():
+        B.dbspmspv_decode(h_up, x0, y1)
+        B.dbspmspv_decode(h_down, y1, y2)
+
+    st = stats_of(timed_calls(torch, chain, flush, 12))
+    warm = float(np.median(timed_calls(torch, chain, flush, 10, warm=True)))
+    w1 = torch.randn(n1, n0, device=dev, dtype=torch.bfloat16)
+    w2 = torch.randn(n0, n1, device=dev, dtype=torch.bfloat16)
+    xb = torch.randn(n0, device=dev, dtype=torch.bfloat16)
+
+    def dense():
+        t = torch.mv(w1, xb)
+        t = torch.where(t > tau, t, torch.zeros_like(t))
+        return torch.mv(w2, t)
+
+    gd = float(np.median(timed_calls(torch, dense, flush, 12)))
+    density = float((wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(y1h)) > max(tau, 0.0)).mean())
+    for h in hs:
+        B.dbspmspv_destroy(h)
+    rec = {"workload": "decode_chain_up11008x4096_relu_cut_down4096x11008_bf16_prune50", "calls": 2,
+           "x0_zero_fraction": 0.9, "x1_density_after_cut": round(density, 4), "us_l2_warm": round(warm, 2),
+           "dense_bf16_gemv_pair_with_torch_relu_cut_us": round(gd, 2)}
+    rec.update(st)
+    return rec
 
 
 def decode_layers(B, torch, dev, flush, peak):

@@ -142,7 +142,12 @@ typedef struct {
                                 blocking (Section 5.3: activation sparsity by magnitude
                                 thresholding) -- x_j takes part iff |x_j| > decode_threshold;
                                 0 (default): iff x_j is not zero.  A NaN always takes part.  */
-    int32_t reserved[5];
+    int32_t decode_relu;     /* dbspmspv_decode: 1 = ReLU fused into the cut: x_j takes part iff
+                                x_j > decode_threshold (negative entries are zeros)        (0) */
+    int32_t decode_x_f32;    /* dbspmspv_decode on a bf16 handle: 1 = x is given as n fp32 values
+                                (e.g. the y of the layer before, fed straight back in) and
+                                rounded to bf16, to nearest even, while it is blocked      (0) */
+    int32_t reserved[3];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64

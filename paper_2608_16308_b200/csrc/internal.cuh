@@ -235,6 +235,8 @@ struct Device {           // everything the kernels need, passed by value
     int32_t stage_bytes;        // payload bytes of one stage (a multiple of 512)
     int32_t has_inline;         // the handle holds INLINE elements at all
     float decode_tau;           // per call: activation magnitude cut of dbspmspv_decode (run option)
+    int32_t decode_relu;        // per call: ReLU fused into the cut (x_j > tau instead of |x_j| > tau)
+    int32_t decode_x_f32;       // per call: x of a bf16 handle is given in fp32 (rounded to bf16 here)
     int32_t x_sparse_believed;  // per call: what the host currently takes x for (1: sparse)
     int32_t *x_nnz_seen;        // mapped host word: nonzero elements of the x of the last single-kernel decode (null: none)
     // Hub row blocks (null / 0 when the matrix has none): hub_slot[rb] = slot of row block rb or

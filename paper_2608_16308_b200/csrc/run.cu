@@ -124,6 +124,12 @@ __global__ void k_emit_from_masks(Device d, float th3, int force_path) {
 
 // Dense input (Sections 4.1, 4.3): every warp reads 32 elements, one ballot gives the two
 // 16-bit masks of its two vector blocks.  Also clears the dense output.
+// Which entries of a dense activation vector take part in a decode call: |x_j| > tau, or, with
+// the ReLU fused in, x_j > tau (tau = 0: x_j not zero / positive).  A NaN always takes part.
+__device__ __forceinline__ bool decode_takes_part(const Device &d, float v) {
+    return d.decode_relu ? !(v <= d.decode_tau) : !(fabsf(v) <= d.decode_tau);
+}
+
 template <int DT>
 __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__restrict__ y) {
     pdl_launch_dependents();
@@ -132,10 +138,12 @@ __global__ void k_xblock_dense(Device d, const void *__restrict__ x, float *__re
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < padded; j += stride) {
         float v = 0.f;
-        if (j < d.n) v = DT == DBSPMSPV_BF16 ? __bfloat162float(static_cast<const __nv_bfloat16 *>(x)[j])
-                                             : static_cast<const float *>(x)[j];
-        // an entry takes part iff |x_j| > tau (tau = 0: iff it is not zero; a NaN always does)
-        const bool in = !(fabsf(v) <= d.decode_tau);
+        if (j < d.n) {
+            if (DT == DBSPMSPV_BF16 && !d.decode_x_f32) v = __bfloat162float(static_cast<const __nv_bfloat16 *>(x)[j]);
+            else v = static_cast<const float *>(x)[j];
+            if (DT == DBSPMSPV_BF16 && d.decode_x_f32) v = __bfloat162float(__float2bfloat16_rn(v));
+        }
+        const bool in = j < d.n && decode_takes_part(d, v);
         if (j < (int64_t)d.nb * 16)
             d.ws.x_dense[j] = in ? (__float_as_uint(v) == X_ABSENT ? __uint_as_float(0x7FC00000u) : v)
                                  : __uint_as_float(X_ABSENT);
@@ -1097,12 +1105,15 @@ __device__ __forceinline__ void stage_x_blocks(const Device &d, const void *__re
                                                int *s_cnt, int tid, int T) {
     const int lane = tid & 31;
     const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
+    // (a bf16 handle may be given its x in fp32 -- the fp32 output of the layer before --, which
+    // is rounded to bf16 here, to nearest even, so that the products stay exact)
+    const bool x16 = DT == DBSPMSPV_BF16 && !d.decode_x_f32;
     int mine = 0;
     for (int cb = tid; cb < d.nb; cb += T) {
         const int64_t j0 = (int64_t)cb * 16;
         float v[16];
         if (aligned && j0 + 16 <= d.n) {
-            if (DT == DBSPMSPV_BF16) {
+            if (x16) {
                 const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(x) + j0);
                 const uint4 a = src[0], b = src[1];
                 const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
@@ -1117,14 +1128,15 @@ __device__ __forceinline__ void stage_x_blocks(const Device &d, const void *__re
 #pragma unroll
             for (int k = 0; k < 16; ++k) {
                 v[k] = 0.f;
-                if (j0 + k < d.n) v[k] = DT == DBSPMSPV_BF16 ? __uint_as_float((uint32_t) static_cast<const uint16_t *>(x)[j0 + k] << 16)
-                                                             : static_cast<const float *>(x)[j0 + k];
+                if (j0 + k < d.n) v[k] = x16 ? __uint_as_float((uint32_t) static_cast<const uint16_t *>(x)[j0 + k] << 16)
+                                             : static_cast<const float *>(x)[j0 + k];
             }
         }
         uint32_t bits = 0;
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
-            const bool nz = !(fabsf(v[k]) <= d.decode_tau);      // |x_j| > tau; tau = 0: not zero; NaN takes part
+            if (DT == DBSPMSPV_BF16 && !x16) v[k] = __bfloat162float(__float2bfloat16_rn(v[k]));
+            const bool nz = decode_takes_part(d, v[k]);
             bits |= (nz ? 1u : 0u) << k;
             // (a widened bf16 has zero low bits: it cannot collide with the marker)
             if (DT != DBSPMSPV_BF16 && __float_as_uint(v[k]) == X_ABSENT) v[k] = __uint_as_float(0x7FC00000u);
@@ -2014,6 +2026,8 @@ template <int DT>
 static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStream_t st) {
     const Device &d = h->d;
     h->d.decode_tau = h->ropts.decode_threshold;
+    h->d.decode_relu = h->ropts.decode_relu != 0;
+    h->d.decode_x_f32 = h->ropts.decode_x_f32 != 0;
     // (-1: no decode call has reported yet)
     const int seen = h->x_nnz_seen_host ? *const_cast<volatile int32_t *>(h->x_nnz_seen_host) : -1;
     const bool sparse_x = seen >= 0 && (float)seen < STREAM_MIN_X_DENSITY * (float)d.n;

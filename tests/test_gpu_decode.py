@@ -167,6 +167,39 @@ def test_decode_magnitude_threshold_is_fused_into_the_blocking(dtype):
     h.close()
 
 
+def test_decode_chain_up_relu_cut_down_without_leaving_the_device():
+    """Two bf16 layers chained on the device: the fp32 output of the first decode call is the x
+    of the second (decode_x_f32), with the ReLU and the magnitude cut fused into its blocking
+    (decode_relu, decode_threshold) -- no kernel in between.  Each layer is checked against the
+    oracle on the operands it was given: the second one on the bf16-rounded, rectified and cut
+    output of the first as the GPU produced it."""
+    n0, n1, n2 = 512, 1408, 512
+    w_up = wl.pruned_weight(n1, n0, 0.5, seed=5, stream=51)
+    w_down = wl.pruned_weight(n2, n1, 0.5, seed=5, stream=52)
+    h_up, h_down = Handle(w_up, B.BF16), Handle(w_down, B.BF16)
+    x0 = wl.relu_activation(n0, 0.7, seed=5, stream=63)
+    want1, scale1 = oracle.ref_decode(ref_matrix(w_up, bf16=True), wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x0)))
+    x0d = torch.from_numpy(wl.f32_to_bf16_bits(x0).view(np.int16)).to(DEV)
+    y1 = torch.empty(n1, dtype=torch.float32, device=DEV)
+    y2 = torch.full((n2,), 7.0, dtype=torch.float32, device=DEV)
+    for legacy in (0, 3, 2, 1):
+        h_up.set_opts(no_fused_decode=legacy)
+        B.dbspmspv_decode(h_up.h, x0d, y1)
+        torch.cuda.synchronize()
+        y1h = y1.cpu().numpy()
+        check(y1h, want1, scale1)
+        x1 = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(y1h))
+        for tau in (0.0, float(np.quantile(x1[x1 > 0], 0.5))):
+            x1t = np.where(x1 > np.float32(tau), x1, 0.0).astype(np.float32)
+            want2, scale2 = oracle.ref_decode(ref_matrix(w_down, bf16=True), x1t)
+            h_down.set_opts(no_fused_decode=legacy, decode_x_f32=1, decode_relu=1, decode_threshold=tau)
+            B.dbspmspv_decode(h_down.h, y1, y2)          # y1 never left the device
+            torch.cuda.synchronize()
+            check(y2.cpu().numpy(), want2, scale2)
+            assert h_down.get_stats().last_n_nzblk == int((x1t.reshape(-1, 16) != 0).any(axis=1).sum())
+    h_up.close(); h_down.close()
+
+
 def test_decode_rejects_pattern_handles():
     h = Handle(wl.random_sparse(32, 32, 50, 1, values=False), B.PATTERN)
     t = torch.zeros(32, device=DEV)
