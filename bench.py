@@ -357,7 +357,7 @@ def main() -> None:
             if args.bfs_only:
                 print(json.dumps(bench_bfs(args, B, torch, dev, flush, peak)))
             elif args.decode_only:
-                print(json.dumps(decode_layers(B, torch, dev, flush, peak) + [decode_chain(B, torch, dev, flush)]))
+                print(json.dumps(decode_layers(B, torch, dev, flush, peak) + [decode_chain(B, torch, dev, flush)] + decode_batch(B, torch, dev, flush)))
             else:
                 print(json.dumps({"format_ablation": format_ablation(B, torch, dev, flush), "storage": storage_table(B, torch, dev)}))
         return
@@ -682,6 +682,7 @@ def other_configs(B, torch, dev, flush, peak, floors):
     del a3
     out += decode_layers(B, torch, dev, flush, peak)
     out.append(decode_chain(B, torch, dev, flush))
+    out += decode_batch(B, torch, dev, flush)
     return out
 
 
@@ -762,6 +763,41 @@ def decode_chain(B, torch, dev, flush):
            "dense_bf16_gemv_pair_with_torch_relu_cut_us": round(gd, 2)}
     rec.update(st)
     return rec
+
+
+def decode_batch(B, torch, dev, flush):
+    """Multi-vector decode (the paper's stated limitation, Section 6): 2 and 4 activation vectors
+    through the 12288x4096 bf16 layer in one dbspmspv_decode_batch call (one pass over the
+    payload), beside the same vectors as single calls and a dense bf16 GEMM of the same shape."""
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    m, n = wl.DECODE_SHAPES[0]
+    wgt = wl.pruned_weight(m, n, 0.5)
+    bits = wl.f32_to_bf16_bits(wgt.val).view(np.int16)
+    h = B.dbspmspv_create_csr(wgt.m, wgt.n, wgt.nnz, up(wgt.row_ptr), up(wgt.col_idx), up(bits), B.BF16)
+    wd = torch.randn(m, n, device=dev, dtype=torch.bfloat16)
+    out = []
+    for zf in (0.7, 0.9):
+        xs = np.stack([wl.f32_to_bf16_bits(wl.relu_activation(n, zf, stream=50 + b)).view(np.int16) for b in range(4)])
+        xd = up(xs)
+        for batch in (2, 4):
+            y = torch.empty(batch, m, dtype=torch.float32, device=dev)
+            call = lambda: B.dbspmspv_decode_batch(h, xd, n, y, m, batch)
+
+            def singles():
+                for b in range(batch):
+                    B.dbspmspv_decode(h, xd[b], y[b])
+
+            st = stats_of(timed_calls(torch, call, flush, 12))
+            one = float(np.median(timed_calls(torch, singles, flush, 12)))
+            xb = torch.randn(n, batch, device=dev, dtype=torch.bfloat16)
+            gemm = float(np.median(timed_calls(torch, lambda: torch.mm(wd, xb), flush, 12)))
+            rec = {"workload": f"decode_batch{batch}_{m}x{n}_bf16_prune50_act{int(zf * 100)}zero", "vectors": batch,
+                   "single_calls_us": round(one, 2), "dense_bf16_gemm_us_same_box": round(gemm, 2)}
+            rec.update(st)
+            rec["us_per_vector"] = round(st["us"] / batch, 2)
+            out.append(rec)
+    B.dbspmspv_destroy(h)
+    return out
 
 
 def decode_layers(B, torch, dev, flush, peak):

@@ -358,6 +358,20 @@ int dbspmspv_probe_floor(int kind, const int32_t *chain, int32_t start, int32_t 
  * which the next dbspmspv_get_stats returns.  The context stays usable.                       */
 int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_stream_t stream);
 
+/* Several activation vectors through one layer (multi-vector input: the extension the paper
+ * leaves open in its limitations).  x holds `batch` dense vectors of n entries each, vector b
+ * at x + b * ldx entries (the handle's value type; fp32 with run option decode_x_f32); y
+ * receives `batch` dense fp32 vectors of m entries, vector b at y + b * ldy.  ldx >= n,
+ * ldy >= m.  Every y vector equals what dbspmspv_decode gives for its x vector (up to the
+ * order of the fp32 additions).  Where the handle has the streaming decode form, groups of up
+ * to four vectors share one pass over the payload (the selector is not evaluated for them: the
+ * payload is streamed whatever the vectors hold); otherwise the vectors are taken one by one.
+ * The activation options (decode_threshold, decode_relu, decode_x_f32) apply to every vector.
+ * Device pointers; allocates nothing; asynchronous on `stream`.  Pattern handles:
+ * DBSPMSPV_ERR_UNSUPPORTED.                                                                   */
+int dbspmspv_decode_batch(dbspmspv_handle_t h, const void *x, int64_t ldx, float *y, int64_t ldy, int32_t batch,
+                          dbspmspv_stream_t stream);
+
 /* Test hook of the range-checked build (-DDBS_BOUNDS_CHECK; any other build returns
  * DBSPMSPV_ERR_UNSUPPORTED and does nothing): overwrites the other-dimension block index of
  * block-CSR view entry `position` with `block_index` (27 bits), so that a test can show that a

@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = (
     "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "dbspmspv_decode", "dbspmspv_get_stats",
     "dbspmspv_export_coo", "dbspmspv_export_blocks", "dbspmspv_export_views",
     "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror", "dbspmspv_compact_noalloc",
-    "dbspmspv_test_bounded_wait", "dbspmspv_test_corrupt_entry", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
+    "dbspmspv_test_bounded_wait", "dbspmspv_test_corrupt_entry", "dbspmspv_decode_batch", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
 )
 
 
@@ -102,6 +102,7 @@ def lib() -> ctypes.CDLL:
         L.dbspmspv_run.argtypes = [vp, vp, vp, i32, ctypes.c_int, vp, vp, i64, vp, vp]
         L.db_bfs.argtypes = [vp, i32, vp, vp]
         L.dbspmspv_decode.argtypes = [vp, vp, vp, vp]
+        L.dbspmspv_decode_batch.argtypes = [vp, vp, i64, vp, i64, i32, vp]
         L.dbspmspv_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
         L.dbspmspv_export_coo.argtypes = [vp, vp, vp, vp]
         L.dbspmspv_export_blocks.argtypes = [vp, vp, vp, vp, vp]
@@ -232,6 +233,11 @@ def dbspmspv_compact_noalloc(acc, hit_bitmap, m, y_idx, y_val, y_capacity, y_nnz
 def dbspmspv_test_bounded_wait(h, max_tries: int, stream: Optional[int] = None) -> None:
     _check(lib().dbspmspv_test_bounded_wait(h, max_tries, _stream() if stream is None else stream),
            "dbspmspv_test_bounded_wait")
+
+
+def dbspmspv_decode_batch(h, x, ldx: int, y, ldy: int, batch: int, stream: Optional[int] = None) -> None:
+    _check(lib().dbspmspv_decode_batch(h, _ptr(x), ldx, _ptr(y), ldy, batch, _stream() if stream is None else stream),
+           "dbspmspv_decode_batch")
 
 
 def dbspmspv_test_corrupt_entry(h, position: int, block_index: int) -> None:

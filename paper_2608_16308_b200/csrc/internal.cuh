@@ -272,6 +272,7 @@ struct dbspmspv_handle_s {
     int grid_compute, grid_compute_dense, grid_decode_pull;
     bool lean_configured, lean_configured_dense;
     bool fused_configured[3];
+    bool batch_configured[2];
     uint32_t compact_calls;     // compaction launches so far (their parity picks the group-total buffer)
     int stream_grid;            // thread blocks of the streaming decode (0: not configured yet)
     int32_t *x_nnz_seen_host;   // host view of Device::x_nnz_seen (page-locked, mapped)

@@ -1564,6 +1564,10 @@ k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, flo
     }
 }
 
+}  // namespace dbs
+#include "decode_batch.cuh"
+namespace dbs {
+
 // ------------------------------------------------------------------------------------------
 // Output compaction: the hit masks of the row blocks are scanned in order, so y comes out
 // sorted.  Pass 1 counts per tile, pass 2 places the entries, clears the accumulator and the
@@ -2110,6 +2114,52 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
     return DBSPMSPV_OK;
 }
 
+// dbspmspv_decode_batch: groups of up to four vectors share one pass over the payload where the
+// handle has the streaming form and shared memory holds the staged vectors; what is left over
+// (and every vector of a handle without the streaming form) goes through decode_typed.
+template <int DT>
+static int decode_batch_typed(dbspmspv_handle_s *h, const void *x, int64_t ldx, float *y, int64_t ldy, int32_t batch,
+                              cudaStream_t st) {
+    const Device &d = h->d;
+    const size_t esize = (DT == DBSPMSPV_BF16 && !h->ropts.decode_x_f32) ? 2 : 4;
+    const bool stream_ok = h->heavy_stage && d.stage_chunks != nullptr && (h->ropts.no_fused_decode == 0 || h->ropts.no_fused_decode == 3);
+    int max_nb = 1;
+    if (stream_ok) {
+        if (BatchLayout(d.nb, 4, d.stage_bytes).total <= STREAM_MAX_SMEM) max_nb = 4;
+        else if (BatchLayout(d.nb, 2, d.stage_bytes).total <= STREAM_MAX_SMEM) max_nb = 2;
+    }
+    for (int32_t b0 = 0; b0 < batch;) {
+        const int left = batch - b0;
+        const int g = left >= 3 && max_nb >= 4 ? (left < 4 ? left : 4) : (left >= 2 && max_nb >= 2 ? 2 : 1);
+        const void *xg = static_cast<const uint8_t *>(x) + (size_t)b0 * (size_t)ldx * esize;
+        float *yg = y + (size_t)b0 * (size_t)ldy;
+        if (g == 1) {
+            const int s = decode_typed<DT>(h, xg, yg, st);
+            if (s != DBSPMSPV_OK) return s;
+        } else {
+            const int nb = g == 2 ? 2 : 4;
+            const BatchLayout lay(d.nb, nb, d.stage_bytes);
+            auto kernel = nb == 2 ? k_decode_stream_batch<DT, 2> : k_decode_stream_batch<DT, 4>;
+            bool &done = h->batch_configured[nb == 2 ? 0 : 1];
+            if (!done) {
+                DBS_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, STREAM_MAX_SMEM));
+                done = true;
+            }
+            h->d.decode_tau = h->ropts.decode_threshold;
+            h->d.decode_relu = h->ropts.decode_relu != 0;
+            h->d.decode_x_f32 = h->ropts.decode_x_f32 != 0;
+            if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
+            k_zero_rows<<<(int)((d.m + 1023) / 1024), 256, 0, st>>>(yg, ldy, d.m, g);
+            DBS_CUDA(launch_pdl(kernel, h->sm_count, BATCH_CTA, (size_t)lay.total, st, d, xg, ldx, yg, ldy, g));
+            if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
+            h->kernel_launches += 2;
+            DBS_CUDA(cudaGetLastError());
+        }
+        b0 += g;
+    }
+    return DBSPMSPV_OK;
+}
+
 }  // namespace dbs
 
 extern "C" {
@@ -2166,6 +2216,17 @@ int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_
     ++h->kernel_launches;
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
+}
+
+int dbspmspv_decode_batch(dbspmspv_handle_t h, const void *x, int64_t ldx, float *y, int64_t ldy, int32_t batch,
+                          dbspmspv_stream_t stream) {
+    if (!h || !x || !y || batch < 1 || ldx < h->d.n || ldy < h->d.m) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
+    if (h->d.dtype == DBSPMSPV_PATTERN) return DBSPMSPV_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    return h->d.dtype == DBSPMSPV_F32 ? dbs::decode_batch_typed<DBSPMSPV_F32>(h, x, ldx, y, ldy, batch, st)
+                                      : dbs::decode_batch_typed<DBSPMSPV_BF16>(h, x, ldx, y, ldy, batch, st);
 }
 
 int dbspmspv_test_corrupt_entry(dbspmspv_handle_t h, int32_t position, uint32_t block_index) {

@@ -200,6 +200,46 @@ def test_decode_chain_up_relu_cut_down_without_leaving_the_device():
     h_up.close(); h_down.close()
 
 
+@pytest.mark.parametrize("shape,dtype", [((512, 1024), B.BF16), ((333, 1000), B.BF16), ((512, 1024), B.F32), ((48, 20000), B.BF16)])
+def test_decode_batch_equals_the_oracle_vector_by_vector(shape, dtype):
+    """dbspmspv_decode_batch: 1 to 7 vectors of different activation densities (one all zero),
+    leading dimensions larger than n and m, with and without the fused ReLU cut; groups of up
+    to four vectors share one pass over the payload, the rest goes through the single-vector
+    forms.  Every y vector is checked against the oracle for its own x vector."""
+    m, n = shape
+    w = wl.pruned_weight(m, n, 0.5, seed=5, stream=71)
+    h = Handle(w, dtype)
+    ldx, ldy = n + 24, m + 8
+    zfs = [0.7, 0.9, 0.5, 1.0, 0.99, 0.3, 0.8]
+    xs = np.zeros((7, ldx), dtype=np.float32)
+    for b, zf in enumerate(zfs):
+        if zf < 1.0:
+            xs[b, :n] = wl.relu_activation(n, zf, seed=5, stream=80 + b)
+    xs[2, :n] *= np.where(np.arange(n) % 3 == 0, -1.0, 1.0)        # negative entries for the ReLU case
+    xr = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(xs)) if dtype == B.BF16 else xs
+    xd = torch.from_numpy(wl.f32_to_bf16_bits(xs).view(np.int16)).to(DEV) if dtype == B.BF16 else torch.from_numpy(xs).to(DEV)
+    A = ref_matrix(w, bf16=dtype == B.BF16)
+    for relu, tau in ((0, 0.0), (1, 0.3)):
+        refs = []
+        for b in range(7):
+            xt = xr[b, :n]
+            xt = np.where(xt > np.float32(tau), xt, 0.0).astype(np.float32) if relu else xt
+            refs.append(oracle.ref_decode(A, xt))
+        for legacy in (0, 1):
+            for batch in (1, 2, 3, 4, 7):
+                h.set_opts(no_fused_decode=legacy, decode_relu=relu, decode_threshold=tau)
+                y = torch.full((batch, ldy), 55.0, dtype=torch.float32, device=DEV)
+                B.dbspmspv_decode_batch(h.h, xd, ldx, y, ldy, batch)
+                torch.cuda.synchronize()
+                yh = y.cpu().numpy()
+                for b in range(batch):
+                    check(yh[b, :m], *refs[b])
+                assert (yh[:, m:] == 55.0).all()                 # nothing is written past m
+    with pytest.raises(B.DbSpmspvError):
+        B.dbspmspv_decode_batch(h.h, xd, n - 1, y, ldy, 2)
+    h.close()
+
+
 def test_decode_rejects_pattern_handles():
     h = Handle(wl.random_sparse(32, 32, 50, 1, values=False), B.PATTERN)
     t = torch.zeros(32, device=DEV)
