@@ -766,9 +766,10 @@ def decode_chain(B, torch, dev, flush):
 
 
 def decode_batch(B, torch, dev, flush):
-    """Multi-vector decode (the paper's stated limitation, Section 6): 2 and 4 activation vectors
-    through the 12288x4096 bf16 layer in one dbspmspv_decode_batch call (one pass over the
-    payload), beside the same vectors as single calls and a dense bf16 GEMM of the same shape."""
+    """Multi-vector decode (the paper's stated limitation, Section 6): 2, 4 and 8 activation
+    vectors through the 12288x4096 bf16 layer in one dbspmspv_decode_batch call (one pass over
+    the payload, block products on the tensor cores), beside the same vectors as single calls
+    and a dense bf16 GEMM of the same shape."""
     up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
     m, n = wl.DECODE_SHAPES[0]
     wgt = wl.pruned_weight(m, n, 0.5)
@@ -777,9 +778,9 @@ def decode_batch(B, torch, dev, flush):
     wd = torch.randn(m, n, device=dev, dtype=torch.bfloat16)
     out = []
     for zf in (0.7, 0.9):
-        xs = np.stack([wl.f32_to_bf16_bits(wl.relu_activation(n, zf, stream=50 + b)).view(np.int16) for b in range(4)])
+        xs = np.stack([wl.f32_to_bf16_bits(wl.relu_activation(n, zf, stream=50 + b)).view(np.int16) for b in range(8)])
         xd = up(xs)
-        for batch in (2, 4):
+        for batch in (2, 4, 8):
             y = torch.empty(batch, m, dtype=torch.float32, device=dev)
             call = lambda: B.dbspmspv_decode_batch(h, xd, n, y, m, batch)
 

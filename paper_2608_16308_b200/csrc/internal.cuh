@@ -160,6 +160,7 @@ struct Counters {    // device-resident scalars of one call
     int32_t last_n_nzblk, last_n_tasks, last_path, last_y_nnz;
     int32_t bfs_levels, bfs_reached;
     int32_t pad;
+    int32_t batch_fallback;   // decode_batch: the tensor-core kernel left its vectors to the per-column kernel behind it
     int32_t n_hubs;         // hub runs of this call's push worklist (may exceed HUB_CAP: the rest became tasks)
     int32_t bfs_hubs[3];    // BFS: the same per level (the per-level counters rotate three ways: the
                             // level's own, the ones it accumulates for the next level, and a spare
@@ -273,6 +274,7 @@ struct dbspmspv_handle_s {
     bool lean_configured, lean_configured_dense;
     bool fused_configured[3];
     bool batch_configured[2];
+    bool batch_mma_configured[3];
     uint32_t compact_calls;     // compaction launches so far (their parity picks the group-total buffer)
     int stream_grid;            // thread blocks of the streaming decode (0: not configured yet)
     int32_t *x_nnz_seen_host;   // host view of Device::x_nnz_seen (page-locked, mapped)

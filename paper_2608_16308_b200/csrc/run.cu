@@ -6,6 +6,7 @@
 #include "microkernels.cuh"
 #include "staging.cuh"
 #include "worklist.cuh"
+#include "mma_block.cuh"
 
 namespace dbs {
 __device__ __forceinline__ int select_path(const Device &d, float th3, int force_path);
@@ -2114,47 +2115,80 @@ static int decode_typed(dbspmspv_handle_s *h, const void *x, float *y, cudaStrea
     return DBSPMSPV_OK;
 }
 
-// dbspmspv_decode_batch: groups of up to four vectors share one pass over the payload where the
-// handle has the streaming form and shared memory holds the staged vectors; what is left over
-// (and every vector of a handle without the streaming form) goes through decode_typed.
+// dbspmspv_decode_batch: where the handle has the streaming form, groups of vectors share one
+// pass over the payload -- bf16 handles: up to eight per group on the tensor cores
+// (k_decode_batch_mma), with the per-column kernel launched behind it as the fallback for
+// non-finite activations; fp32 handles: up to four per group in the per-column kernel.  What is
+// left over (and every vector of a handle without the streaming form) goes through decode_typed.
 template <int DT>
 static int decode_batch_typed(dbspmspv_handle_s *h, const void *x, int64_t ldx, float *y, int64_t ldy, int32_t batch,
                               cudaStream_t st) {
     const Device &d = h->d;
     const size_t esize = (DT == DBSPMSPV_BF16 && !h->ropts.decode_x_f32) ? 2 : 4;
     const bool stream_ok = h->heavy_stage && d.stage_chunks != nullptr && (h->ropts.no_fused_decode == 0 || h->ropts.no_fused_decode == 3);
-    int max_nb = 1;
+    int max_nb = 1, max_mma = 1;
     if (stream_ok) {
-        if (BatchLayout(d.nb, 4, d.stage_bytes).total <= STREAM_MAX_SMEM) max_nb = 4;
-        else if (BatchLayout(d.nb, 2, d.stage_bytes).total <= STREAM_MAX_SMEM) max_nb = 2;
+        for (int nb : {2, 4})
+            if (BatchLayout(d.nb, nb, d.stage_bytes).total <= STREAM_MAX_SMEM) max_nb = nb;
+        if (DT == DBSPMSPV_BF16)
+            for (int nb : {2, 4, 8})
+                if (max_nb >= (nb < 4 ? nb : 4) && BatchMmaLayout(d.nb, nb, d.stage_bytes).total <= STREAM_MAX_SMEM) max_mma = nb;
     }
+    h->d.decode_tau = h->ropts.decode_threshold;
+    h->d.decode_relu = h->ropts.decode_relu != 0;
+    h->d.decode_x_f32 = h->ropts.decode_x_f32 != 0;
+    // the per-column kernel on vectors [b0, b0 + g), g <= 4
+    auto scalar_group = [&](const void *xg, float *yg, int g, int only_as_fallback) -> int {
+        const int nb = g <= 2 ? 2 : 4;
+        const BatchLayout lay(d.nb, nb, d.stage_bytes);
+        auto kernel = nb == 2 ? k_decode_stream_batch<DT, 2> : k_decode_stream_batch<DT, 4>;
+        bool &done = h->batch_configured[nb == 2 ? 0 : 1];
+        if (!done) {
+            DBS_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, STREAM_MAX_SMEM));
+            done = true;
+        }
+        DBS_CUDA(launch_pdl(kernel, h->sm_count, BATCH_CTA, (size_t)lay.total, st, d, xg, ldx, yg, ldy, g, only_as_fallback));
+        ++h->kernel_launches;
+        return DBSPMSPV_OK;
+    };
     for (int32_t b0 = 0; b0 < batch;) {
         const int left = batch - b0;
-        const int g = left >= 3 && max_nb >= 4 ? (left < 4 ? left : 4) : (left >= 2 && max_nb >= 2 ? 2 : 1);
         const void *xg = static_cast<const uint8_t *>(x) + (size_t)b0 * (size_t)ldx * esize;
         float *yg = y + (size_t)b0 * (size_t)ldy;
+        const int cap = DT == DBSPMSPV_BF16 && max_mma > 1 ? max_mma : max_nb;
+        const int g = left < cap ? left : cap;
         if (g == 1) {
             const int s = decode_typed<DT>(h, xg, yg, st);
             if (s != DBSPMSPV_OK) return s;
-        } else {
-            const int nb = g == 2 ? 2 : 4;
-            const BatchLayout lay(d.nb, nb, d.stage_bytes);
-            auto kernel = nb == 2 ? k_decode_stream_batch<DT, 2> : k_decode_stream_batch<DT, 4>;
-            bool &done = h->batch_configured[nb == 2 ? 0 : 1];
+            b0 += 1;
+            continue;
+        }
+        if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
+        k_zero_rows<<<(int)((d.m + 1023) / 1024), 256, 0, st>>>(yg, ldy, d.m, g);
+        ++h->kernel_launches;
+        if (DT == DBSPMSPV_BF16 && max_mma > 1) {
+            const int nb = g <= 2 ? 2 : g <= 4 ? 4 : 8;
+            const BatchMmaLayout lay(d.nb, nb, d.stage_bytes);
+            auto kernel = nb == 2 ? k_decode_batch_mma<2> : nb == 4 ? k_decode_batch_mma<4> : k_decode_batch_mma<8>;
+            bool &done = h->batch_mma_configured[nb == 2 ? 0 : nb == 4 ? 1 : 2];
             if (!done) {
                 DBS_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, STREAM_MAX_SMEM));
                 done = true;
             }
-            h->d.decode_tau = h->ropts.decode_threshold;
-            h->d.decode_relu = h->ropts.decode_relu != 0;
-            h->d.decode_x_f32 = h->ropts.decode_x_f32 != 0;
-            if (h->ropts.timing) DBS_CUDA(cudaEventRecord(h->ev[0], st));
-            k_zero_rows<<<(int)((d.m + 1023) / 1024), 256, 0, st>>>(yg, ldy, d.m, g);
-            DBS_CUDA(launch_pdl(kernel, h->sm_count, BATCH_CTA, (size_t)lay.total, st, d, xg, ldx, yg, ldy, g));
-            if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
-            h->kernel_launches += 2;
-            DBS_CUDA(cudaGetLastError());
+            DBS_CUDA(launch_pdl(kernel, h->sm_count, BATCH_MMA_CTA, (size_t)lay.total, st, d, xg, ldx, yg, ldy, g));
+            ++h->kernel_launches;
+            // the fallback for non-finite activations: returns at once unless the kernel above asked for it
+            for (int q = 0; q < g; q += 4) {
+                const int gq = g - q < 4 ? g - q : 4;
+                const int s = scalar_group(static_cast<const uint8_t *>(xg) + (size_t)q * (size_t)ldx * esize, yg + (size_t)q * (size_t)ldy, gq, 1);
+                if (s != DBSPMSPV_OK) return s;
+            }
+        } else {
+            const int s = scalar_group(xg, yg, g, 0);
+            if (s != DBSPMSPV_OK) return s;
         }
+        if (h->ropts.timing) { DBS_CUDA(cudaEventRecord(h->ev[1], st)); h->timed = true; }
+        DBS_CUDA(cudaGetLastError());
         b0 += g;
     }
     return DBSPMSPV_OK;

@@ -202,31 +202,40 @@ def test_decode_chain_up_relu_cut_down_without_leaving_the_device():
 
 @pytest.mark.parametrize("shape,dtype", [((512, 1024), B.BF16), ((333, 1000), B.BF16), ((512, 1024), B.F32), ((48, 20000), B.BF16)])
 def test_decode_batch_equals_the_oracle_vector_by_vector(shape, dtype):
-    """dbspmspv_decode_batch: 1 to 7 vectors of different activation densities (one all zero),
-    leading dimensions larger than n and m, with and without the fused ReLU cut; groups of up
-    to four vectors share one pass over the payload, the rest goes through the single-vector
-    forms.  Every y vector is checked against the oracle for its own x vector."""
+    """dbspmspv_decode_batch: 1 to 9 vectors of different activation densities (one all zero),
+    leading dimensions larger than n and m, with and without the fused ReLU cut; groups of
+    vectors share one pass over the payload (bf16: up to eight, on the tensor cores), the rest
+    goes through the single-vector forms.  Every y vector is checked against the oracle for its
+    own x vector.  Then one vector gets an infinite and a NaN entry: the tensor-core kernel hands
+    the group over to the per-column kernel, and non-finite values reach only stored elements."""
     m, n = shape
     w = wl.pruned_weight(m, n, 0.5, seed=5, stream=71)
     h = Handle(w, dtype)
     ldx, ldy = n + 24, m + 8
-    zfs = [0.7, 0.9, 0.5, 1.0, 0.99, 0.3, 0.8]
-    xs = np.zeros((7, ldx), dtype=np.float32)
+    zfs = [0.7, 0.9, 0.5, 1.0, 0.99, 0.3, 0.8, 0.6, 0.95]
+    nv = len(zfs)
+    xs = np.zeros((nv, ldx), dtype=np.float32)
     for b, zf in enumerate(zfs):
         if zf < 1.0:
             xs[b, :n] = wl.relu_activation(n, zf, seed=5, stream=80 + b)
     xs[2, :n] *= np.where(np.arange(n) % 3 == 0, -1.0, 1.0)        # negative entries for the ReLU case
-    xr = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(xs)) if dtype == B.BF16 else xs
-    xd = torch.from_numpy(wl.f32_to_bf16_bits(xs).view(np.int16)).to(DEV) if dtype == B.BF16 else torch.from_numpy(xs).to(DEV)
     A = ref_matrix(w, bf16=dtype == B.BF16)
+
+    def upload(a):
+        return torch.from_numpy(wl.f32_to_bf16_bits(a).view(np.int16)).to(DEV) if dtype == B.BF16 else torch.from_numpy(a).to(DEV)
+
+    def rounded(a):
+        return wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(a)) if dtype == B.BF16 else a
+
+    xr, xd = rounded(xs), upload(xs)
     for relu, tau in ((0, 0.0), (1, 0.3)):
         refs = []
-        for b in range(7):
+        for b in range(nv):
             xt = xr[b, :n]
             xt = np.where(xt > np.float32(tau), xt, 0.0).astype(np.float32) if relu else xt
             refs.append(oracle.ref_decode(A, xt))
         for legacy in (0, 1):
-            for batch in (1, 2, 3, 4, 7):
+            for batch in (1, 2, 3, 4, 5, 8, 9):
                 h.set_opts(no_fused_decode=legacy, decode_relu=relu, decode_threshold=tau)
                 y = torch.full((batch, ldy), 55.0, dtype=torch.float32, device=DEV)
                 B.dbspmspv_decode_batch(h.h, xd, ldx, y, ldy, batch)
@@ -235,6 +244,23 @@ def test_decode_batch_equals_the_oracle_vector_by_vector(shape, dtype):
                 for b in range(batch):
                     check(yh[b, :m], *refs[b])
                 assert (yh[:, m:] == 55.0).all()                 # nothing is written past m
+    # non-finite activations in one vector of the group
+    act = np.flatnonzero(xs[1, :n])
+    xs[1, act[0]], xs[1, act[2]] = np.inf, np.nan
+    xr, xd = rounded(xs), upload(xs)
+    h.set_opts()
+    for batch in (4, 8):
+        y = torch.full((batch, ldy), 55.0, dtype=torch.float32, device=DEV)
+        B.dbspmspv_decode_batch(h.h, xd, ldx, y, ldy, batch)
+        torch.cuda.synchronize()
+        yh = y.cpu().numpy()
+        for b in range(batch):
+            want, scale = oracle.ref_decode(A, xr[b, :n])
+            nan, inf = np.isnan(want), np.isinf(want)
+            assert (np.isnan(yh[b, :m]) == nan).all() and (yh[b, :m][inf] == want[inf]).all()
+            fin = ~nan & ~inf
+            check(yh[b, :m][fin], want[fin], scale[fin])
+        assert np.isnan(yh[1, :m]).any()
     with pytest.raises(B.DbSpmspvError):
         B.dbspmspv_decode_batch(h.h, xd, n - 1, y, ldy, 2)
     h.close()
