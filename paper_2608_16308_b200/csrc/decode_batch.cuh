@@ -363,13 +363,27 @@ k_decode_batch_mma(Device d, const void *__restrict__ x, int64_t ldx, float *__r
                 for (int k = 0; k < 16; ++k) hv[k] = 0;
                 if (v < nvec) {
                     const int64_t j0 = (int64_t)cb * 16;
+                    float fv[16];
+                    const uint16_t *xh_g = static_cast<const uint16_t *>(x) + (size_t)v * ldx + j0;
+                    if (!d.decode_x_f32 && j0 + 16 <= d.n && (reinterpret_cast<uintptr_t>(xh_g) & 15u) == 0) {
+                        // sixteen bf16 entries with two 16-byte loads
+                        const uint4 a = reinterpret_cast<const uint4 *>(xh_g)[0], b = reinterpret_cast<const uint4 *>(xh_g)[1];
+                        const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) { fv[2 * q] = __uint_as_float(u[q] << 16); fv[2 * q + 1] = __uint_as_float(u[q] & 0xFFFF0000u); }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            fv[k] = 0.f;
+                            if (j0 + k < d.n) {
+                                if (d.decode_x_f32) fv[k] = __bfloat162float(__float2bfloat16_rn(static_cast<const float *>(x)[(size_t)v * ldx + j0 + k]));
+                                else fv[k] = __uint_as_float((uint32_t)xh_g[k] << 16);
+                            }
+                        }
+                    }
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        float f = 0.f;
-                        if (j0 + k < d.n) {
-                            if (d.decode_x_f32) f = __bfloat162float(__float2bfloat16_rn(static_cast<const float *>(x)[(size_t)v * ldx + j0 + k]));
-                            else f = __uint_as_float((uint32_t) static_cast<const uint16_t *>(x)[(size_t)v * ldx + j0 + k] << 16);
-                        }
+                        const float f = fv[k];
                         if (decode_takes_part(d, f)) {
                             bits |= 1u << k;
                             hv[k] = (uint16_t)(__float_as_uint(f) >> 16);

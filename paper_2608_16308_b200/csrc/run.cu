@@ -1347,7 +1347,7 @@ constexpr int STREAM_CTA = STREAM_WARPS * 32;
 #define DBS_STREAM_DEPTH 2
 #endif
 constexpr int STREAM_DEPTH = DBS_STREAM_DEPTH;
-constexpr int STREAM_MAX_SMEM = 220 * 1024;
+constexpr int STREAM_MAX_SMEM = 227 * 1024;   // all a thread block may have
 __host__ __device__ constexpr int stream_stride(int stage_bytes) { return (stage_bytes + 127) & ~127; }
 struct StreamLayout {
     int xm_off, cnt_off, active_off, bar_off, ring_off, total;
