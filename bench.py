@@ -680,6 +680,11 @@ def other_configs(B, torch, dev, flush, peak, floors):
     spmspv_case("stencil27_160cubed_fp32", a3, [("0.1 % in runs of 64", wl.clustered_x(a3.n, 64)),
                                                  ("5 % in runs of 64", wl.clustered_x(a3.n, 3200))])
     del a3
+    # the sweep's matrix with its vertices relabelled by a seeded permutation (hubs scattered
+    # instead of packed at the low indices): the 1 %, 10 % and 50 % points
+    a2 = wl.rmat(20, 16, seed=1, relabel=True)
+    spmspv_case("rmat20_ef16_relabelled_fp32", a2, [(f"x fraction {f:g}", wl.rmat_x(a2.n, f, k)) for k, f in ((3, 1e-2), (4, 1e-1), (5, 0.5))])
+    del a2
     out += decode_layers(B, torch, dev, flush, peak)
     out.append(decode_chain(B, torch, dev, flush))
     out += decode_batch(B, torch, dev, flush)

@@ -219,13 +219,25 @@ def rmat_keys(scale: int, edge_factor: int, seed: int,
     return keys
 
 
+def vertex_permutation(n: int, seed: int, stream: int = 9) -> np.ndarray:
+    """A seeded permutation of 0..n-1 (argsort of counter-based random keys, ties by index)."""
+    return np.argsort(rand_u64(seed, stream, np.arange(n, dtype=np.uint64)), kind="stable").astype(np.int64)
+
+
 def rmat(scale: int = 20, edge_factor: int = 16, seed: int = 1, values: bool = True,
-         symmetrise: bool = False) -> CSR:
+         symmetrise: bool = False, relabel: bool = False) -> CSR:
     """R-MAT power-law matrix; duplicates merged.  With `symmetrise`, self loops are dropped
     and every edge gets its reverse (the BFS graph of the paper's DB-BFS experiments is
-    symmetric, Section 5.1)."""
+    symmetric, Section 5.1).  With `relabel`, rows and columns are renumbered by one seeded
+    permutation (the Graph500 habit): the hubs no longer sit next to each other at the low
+    indices.  The configurations of the paper's workloads use no relabelling."""
     n = 1 << scale
     keys = rmat_keys(scale, edge_factor, seed)
+    if relabel:
+        perm = vertex_permutation(n, seed)
+        r = keys // n
+        keys = perm[r] * n + perm[keys - r * n]
+        del r, perm
     if symmetrise:
         r = keys // n
         c = keys - r * n

@@ -110,3 +110,17 @@ def test_bf16_rounding_is_nearest_even():
     # 1 + 2^-8 is a tie between 1.0 and 1 + 2^-7 -> even mantissa (1.0); 1 + 3*2^-8 -> 1 + 2^-6
     got = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(a))
     assert got.tolist() == [1.0, 1.0, 1.015625, -2.5, 3.140625]
+
+
+def test_rmat_relabelled_is_the_same_graph_under_a_permutation():
+    a = wl.rmat(10, 8, seed=7)
+    b = wl.rmat(10, 8, seed=7, relabel=True)
+    perm = wl.vertex_permutation(1 << 10, 7)
+    assert sorted(perm.tolist()) == list(range(1 << 10))
+    assert a.nnz == b.nnz
+    ka = np.sort(perm[a.rows().astype(np.int64)] * (1 << 10) + perm[a.col_idx.astype(np.int64)])
+    kb = np.sort(b.rows().astype(np.int64) * (1 << 10) + b.col_idx.astype(np.int64))
+    assert np.array_equal(ka, kb)
+    # the degree multiset survives, the hubs move away from the low indices
+    assert np.array_equal(np.sort(np.diff(a.row_ptr)), np.sort(np.diff(b.row_ptr)))
+    assert np.argmax(np.diff(a.row_ptr)) == 0 and np.argmax(np.diff(b.row_ptr)) == perm[0]
