@@ -358,6 +358,18 @@ int dbspmspv_probe_floor(int kind, const int32_t *chain, int32_t start, int32_t 
  * which the next dbspmspv_get_stats returns.  The context stays usable.                       */
 int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_stream_t stream);
 
+/* y<mask> = A x: dbspmspv_run with an output mask (the GraphBLAS form of the primitive; the
+ * "strip the visited vertices" step of DB-BFS, Section 4.2, as an option of the call).
+ * row_mask is a device bitmap over the rows, bit i of word i / 32 = row i, at least
+ * ceil(ceil(m / 16) / 2) words (the last one padded with anything).  complement = 0: a row goes
+ * to y iff its bit is set; complement = 1: iff its bit is clear (the mask then names what is
+ * already known, e.g. a visited set).  y holds the structural result restricted to those rows,
+ * ascending; y_nnz counts them.  The mask is applied where y is compacted: the traversal does
+ * the same work as dbspmspv_run.  Everything else as dbspmspv_run.                             */
+int dbspmspv_run_masked(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
+                        int semiring, const uint32_t *row_mask, int complement, int32_t *y_idx, float *y_val,
+                        int64_t y_capacity, int32_t *y_nnz, dbspmspv_stream_t stream);
+
 /* Several activation vectors through one layer (multi-vector input: the extension the paper
  * leaves open in its limitations).  x holds `batch` dense vectors of n entries each, vector b
  * at x + b * ldx entries (the handle's value type; fp32 with run option decode_x_f32); y

@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = (
     "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "dbspmspv_decode", "dbspmspv_get_stats",
     "dbspmspv_export_coo", "dbspmspv_export_blocks", "dbspmspv_export_views",
     "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror", "dbspmspv_compact_noalloc",
-    "dbspmspv_test_bounded_wait", "dbspmspv_test_corrupt_entry", "dbspmspv_decode_batch", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
+    "dbspmspv_test_bounded_wait", "dbspmspv_test_corrupt_entry", "dbspmspv_decode_batch", "dbspmspv_run_masked", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
 )
 
 
@@ -100,6 +100,7 @@ def lib() -> ctypes.CDLL:
                                           ctypes.c_int, ctypes.POINTER(CreateOpts), vp]
         L.dbspmspv_create_coo.argtypes = L.dbspmspv_create_csr.argtypes
         L.dbspmspv_run.argtypes = [vp, vp, vp, i32, ctypes.c_int, vp, vp, i64, vp, vp]
+        L.dbspmspv_run_masked.argtypes = [vp, vp, vp, i32, ctypes.c_int, vp, ctypes.c_int, vp, vp, i64, vp, vp]
         L.db_bfs.argtypes = [vp, i32, vp, vp]
         L.dbspmspv_decode.argtypes = [vp, vp, vp, vp]
         L.dbspmspv_decode_batch.argtypes = [vp, vp, i64, vp, i64, i32, vp]
@@ -233,6 +234,13 @@ def dbspmspv_compact_noalloc(acc, hit_bitmap, m, y_idx, y_val, y_capacity, y_nnz
 def dbspmspv_test_bounded_wait(h, max_tries: int, stream: Optional[int] = None) -> None:
     _check(lib().dbspmspv_test_bounded_wait(h, max_tries, _stream() if stream is None else stream),
            "dbspmspv_test_bounded_wait")
+
+
+def dbspmspv_run_masked(h, x_idx, x_val, nnz_x: int, semiring: int, row_mask, complement: int, y_idx, y_val,
+                        y_capacity: int, y_nnz, stream: Optional[int] = None) -> None:
+    _check(lib().dbspmspv_run_masked(h, _ptr(x_idx), _ptr(x_val), nnz_x, semiring, _ptr(row_mask), complement, _ptr(y_idx),
+                                     _ptr(y_val), y_capacity, _ptr(y_nnz), _stream() if stream is None else stream),
+           "dbspmspv_run_masked")
 
 
 def dbspmspv_decode_batch(h, x, ldx: int, y, ldy: int, batch: int, stream: Optional[int] = None) -> None:

@@ -1621,7 +1621,7 @@ __global__ void __launch_bounds__(128) k_fold_hubs(Device d) {
     if (slot < d.n_hub_blocks && DBS_CHK_INDEX(d, d.hub_rb[slot], d.mb)) fold_hub_block(d, d.hub_rb[slot], slot, threadIdx.x & 31);
 }
 
-__global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d, int parity) {
+__global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d, int parity, const uint32_t *__restrict__ row_mask, int complement) {
     __shared__ int s_red[TILE_WORDS / 32];
     pdl_wait();
     pdl_launch_dependents();
@@ -1641,7 +1641,8 @@ __global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d, int pari
             f4[1] = make_uint4(0u, 0u, 0u, 0u);
         }
         d.ws.y_mask32[wi] = word;
-        c = __popc(word);
+        // (an output mask drops rows from y; their accumulator entries are still cleared by pass 2)
+        c = __popc(row_mask ? word & (complement ? ~row_mask[wi] : row_mask[wi]) : word);
     }
     c = __reduce_add_sync(FULL, c);
     if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = c;
@@ -1659,7 +1660,8 @@ __global__ void __launch_bounds__(TILE_WORDS) k_compact_count(Device d, int pari
 
 __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__restrict__ y_idx, float *__restrict__ y_val,
                                                            int64_t y_capacity, int32_t *__restrict__ y_nnz, int boolean,
-                                                           const int32_t *__restrict__ x_idx, int32_t nnz_x, int clear_all, int parity) {
+                                                           const int32_t *__restrict__ x_idx, int32_t nnz_x, int clear_all, int parity,
+                                                           const uint32_t *__restrict__ row_mask, int complement) {
     __shared__ int s_before[CMP_TPB / 32], s_cnt[CMP_TPB / 32];
     __shared__ int32_t s_oidx[TILE_WORDS * 32];
     __shared__ float s_oval[TILE_WORDS * 32];
@@ -1686,11 +1688,13 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
             if (blockIdx.x == 0)
                 for (int k = threadIdx.x; k < d.ws.n_tile_groups; k += CMP_TPB) d.ws.tile_group[(parity ^ 1) * d.ws.n_tile_groups + k] = 0;
         }
-        const uint32_t bits = (word >> (8 * sub)) & 0xFFu;
+        const uint32_t keep = row_mask && wi < n_words ? (complement ? ~row_mask[wi] : row_mask[wi]) : 0xFFFFFFFFu;
+        const uint32_t hits = (word >> (8 * sub)) & 0xFFu;    // rows to clear
+        const uint32_t bits = hits & (keep >> (8 * sub));     // rows that go to y
         const int c = __popc(bits);
         const int row0 = wi * 32 + sub * 8;
         float4 v4[2];
-        if (bits) {                   // two independent 16-byte loads fetch the 8 accumulator entries
+        if (hits) {                   // two independent 16-byte loads fetch the 8 accumulator entries
             float4 *acc4 = reinterpret_cast<float4 *>(d.ws.y_acc + row0);
             v4[0] = acc4[0]; v4[1] = acc4[1];
             acc4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1956,7 +1960,7 @@ int allocate_workspace(dbspmspv_handle_s *h) {
 template <int DT>
 static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
                      int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
-                     cudaStream_t st) {
+                     cudaStream_t st, const uint32_t *row_mask = nullptr, int complement = 0) {
     const Device &d = h->d;
     // x lists a quarter of the columns or more: a pull is likely (on hypersparse matrices), so
     // the worklist is built afterwards from the masks, and only if the selector does choose the push
@@ -2003,12 +2007,12 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     h->kernel_launches += 2;
     const int nt = d.ws.n_tiles;
     const int parity = (int)(++h->compact_calls & 1u);
-    DBS_CUDA(launch_pdl(k_compact_count, nt, TILE_WORDS, 0, st, d, parity));
+    DBS_CUDA(launch_pdl(k_compact_count, nt, TILE_WORDS, 0, st, d, parity, row_mask, complement));
     int extra = (nnz_x + CMP_TPB * 8 - 1) / (CMP_TPB * 8);
     if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
     const int clear_all = (int64_t)nnz_x * 8 > d.n;     // scattered clears cost more than a full sweep
     DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, 0, st, d, y_idx, y_val, y_capacity, y_nnz,
-                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x, clear_all, parity));
+                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x, clear_all, parity, row_mask, complement));
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }
@@ -2219,9 +2223,9 @@ int dbspmspv_set_run_opts(dbspmspv_handle_t h, const dbspmspv_run_opts *opts) {
     return DBSPMSPV_OK;
 }
 
-int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
-                 int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
-                 dbspmspv_stream_t stream) {
+static int run_checked(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
+                       int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
+                       dbspmspv_stream_t stream, const uint32_t *row_mask, int complement) {
     if (!h || nnz_x < 0 || y_capacity < 0 || !y_nnz) return DBSPMSPV_ERR_INVALID_ARG;
     if (nnz_x > 0 && !x_idx) return DBSPMSPV_ERR_INVALID_ARG;
     if (y_capacity > 0 && !y_idx) return DBSPMSPV_ERR_INVALID_ARG;
@@ -2235,10 +2239,23 @@ int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     h->last_stream = st;
     switch (h->d.dtype) {
-        case DBSPMSPV_F32: return dbs::run_typed<DBSPMSPV_F32>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
-        case DBSPMSPV_BF16: return dbs::run_typed<DBSPMSPV_BF16>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
-        default: return dbs::run_typed<DBSPMSPV_PATTERN>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st);
+        case DBSPMSPV_F32: return dbs::run_typed<DBSPMSPV_F32>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st, row_mask, complement);
+        case DBSPMSPV_BF16: return dbs::run_typed<DBSPMSPV_BF16>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st, row_mask, complement);
+        default: return dbs::run_typed<DBSPMSPV_PATTERN>(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, st, row_mask, complement);
     }
+}
+
+int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
+                 int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
+                 dbspmspv_stream_t stream) {
+    return run_checked(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, stream, nullptr, 0);
+}
+
+int dbspmspv_run_masked(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, int32_t nnz_x,
+                        int semiring, const uint32_t *row_mask, int complement, int32_t *y_idx, float *y_val,
+                        int64_t y_capacity, int32_t *y_nnz, dbspmspv_stream_t stream) {
+    if (!row_mask || (complement != 0 && complement != 1)) return DBSPMSPV_ERR_INVALID_ARG;
+    return run_checked(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, stream, row_mask, complement);
 }
 
 int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_stream_t stream) {

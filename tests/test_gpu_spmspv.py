@@ -390,6 +390,52 @@ def test_hub_row_blocks_add_into_private_accumulators_and_fold_exactly():
     h.close(); hp.close()
 
 
+def test_masked_output_keeps_exactly_the_rows_the_mask_names():
+    """dbspmspv_run_masked: y<mask> and y<not mask> are the oracle's y restricted to the rows
+    whose bit is set / clear, on every path, and the handle is clean afterwards (the dropped
+    rows' sums must not leak into the next call).  As a BFS step: one OR-AND product of the
+    frontier masked by the complement of the visited set is the oracle's next level."""
+    csr = wl.rmat(12, 16, seed=5)
+    A = ref_matrix(csr)
+    h = Handle(csr, B.F32)
+    rng = np.random.default_rng(11)
+    bits = rng.random(csr.m) < 0.4
+    n_words = ((csr.m + 15) // 16 + 1) // 2
+    words = np.zeros(n_words, dtype=np.uint32)
+    rows = np.flatnonzero(bits)
+    np.bitwise_or.at(words, rows >> 5, np.uint32(1) << (rows & 31).astype(np.uint32))
+    maskd = torch.from_numpy(words.view(np.int32)).to("cuda")
+    x = dense_x(csr.n, 3, 0.05)
+    xi = torch.from_numpy(x.idx).to("cuda"); xv = torch.from_numpy(x.val).to("cuda")
+    ri, rv, rs = oracle.ref_pull(A, x.idx, x.val)
+    for path in PATHS:
+        h.set_opts(force_path=path)
+        for complement in (0, 1):
+            keep = bits[ri] if complement == 0 else ~bits[ri]
+            h.y_nnz.fill_(-7)
+            B.dbspmspv_run_masked(h.h, xi, xv, int(x.idx.size), B.PLUS_TIMES, maskd, complement, h.y_idx, h.y_val, csr.m, h.y_nnz)
+            torch.cuda.synchronize()
+            k = int(h.y_nnz.item())
+            got = (h.y_idx[:k].cpu().numpy(), h.y_val[:k].cpu().numpy(), k)
+            check_against_oracle(got, (ri[keep], rv[keep], rs[keep]))
+            check_against_oracle(h.run(x), (ri, rv, rs))          # nothing left behind
+    # one BFS level from the oracle's levels
+    g = wl.rmat(11, 8, seed=5, values=False, symmetrise=True)
+    hg = Handle(g, B.PATTERN)
+    src = int(wl.bfs_sources(g, 1)[0])
+    levels = oracle.ref_bfs(oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx, None), src)
+    frontier = np.flatnonzero(levels == 1).astype(np.int32)
+    visited = np.flatnonzero((levels >= 0) & (levels <= 1))
+    vw = np.zeros(((g.m + 15) // 16 + 1) // 2, dtype=np.uint32)
+    np.bitwise_or.at(vw, visited >> 5, np.uint32(1) << (visited & 31).astype(np.uint32))
+    B.dbspmspv_run_masked(hg.h, torch.from_numpy(frontier).to("cuda"), None, int(frontier.size), B.OR_AND,
+                          torch.from_numpy(vw.view(np.int32)).to("cuda"), 1, hg.y_idx, None, g.m, hg.y_nnz)
+    torch.cuda.synchronize()
+    k = int(hg.y_nnz.item())
+    assert np.array_equal(hg.y_idx[:k].cpu().numpy(), np.flatnonzero(levels == 2))
+    h.close(); hg.close()
+
+
 def test_bounded_wait_runs_out_and_reports_timeout():
     """The staging waits are bounded: a wait on a barrier that nothing arrives on (no copy in
     flight) gives up, the kernel records ERR_TIMEOUT, get_stats returns it once, and the handle
