@@ -2208,7 +2208,7 @@ void dbspmspv_default_run_opts(dbspmspv_run_opts *o) {
     o->th3 = 0.95f;
     o->th3_bfs = 0.05f;
     o->th3_decode = 0.01f;
-    o->bfs_push_max_edge_frac = 0.f;
+    o->bfs_push_max_edge_frac = 0.08f;
     o->force_path = DBSPMSPV_PATH_AUTO;
     o->popc_threshold = 8;
     o->validate = 0;
