@@ -86,8 +86,10 @@ __device__ void bfs_push(const Device &d, const Scope &sc, const uint32_t *F, ui
             e.start = start;
             if (lane < e.n && DBS_CHK_RANGE(d, start, e.n) && DBS_CHK_INDEX(d, jb, d.nb)) {
                 e.idx = d.csc.idx[start + lane]; e.aux = d.csc.aux[start + lane];
+#ifdef DBS_BOUNDS_CHECK
                 uint32_t w_ = d.csc.w[start + lane];
                 DBS_CHK_ENTRY(d, false, e.idx, w_, e.aux);
+#endif
             }
             e.xm = mask_of(F, jb);
         }
@@ -337,7 +339,9 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
                 const int pos = base + lane;
                 if (pos < pend) {
                     uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
+#ifdef DBS_BOUNDS_CHECK
                     { uint32_t w_ = d.csr.w[pos]; DBS_CHK_ENTRY(d, true, idx, w_, aux); }
+#endif
                     const uint32_t xm = mask_of(F, idx & IDX_MASK);
                     if (xm) {
                         const int type = idx >> TYPE_SHIFT;

@@ -263,11 +263,13 @@ k_pull_lean(Device d, Out out, float th3, int force_path, int popc_threshold, in
         const int pos = d.payload_pos[q];
         if (!DBS_CHK_INDEX(d, pos, d.n_entries)) continue;            // warp-uniform
         uint32_t idx = d.csr.idx[pos];
+#ifdef DBS_BOUNDS_CHECK
         {
             uint32_t w_ = d.csr.w[pos], a_ = d.csr.aux[pos];
             DBS_CHK_ENTRY(d, true, idx, w_, a_);
             if ((idx >> TYPE_SHIFT) == DBSPMSPV_BLK_INLINE || !DBS_CHK_INDEX(d, d.entry_row[pos], d.mb)) continue;   // (only a replaced entry is INLINE here)
         }
+#endif
         const int cb = idx & IDX_MASK, type = idx >> TYPE_SHIFT;
         const uint32_t xm = mask_of(d.ws.x_mask32, cb);
         if (!xm) continue;                                            // warp-uniform
