@@ -421,6 +421,180 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
     if (lane == 0 && n_found) { atomicAdd(&d.ws.ctr->bfs_reached, n_found); atomicAdd(nz_out, n_nz); }
 }
 
+// The same pull, transposed: a warp takes a block of 32 consecutive mask words (1024 rows) and
+// lane l walks row l of every word, one row after the other, each lane at its own pace.  With
+// lane = row inside ONE word (bfs_pull_rows above) a word costs as many dependent rounds as its
+// slowest row -- and at the levels with a small frontier almost every word holds a row without
+// a frontier neighbour, which is walked to its end -- so a warp's time is the sum over its words
+// of the maximum; here it is the maximum over the lanes of the sum, about a third of the rounds.
+// Found rows are collected as one bit per (lane, word) and transposed back with ballots, so the
+// warp still owns its mask words: plain stores, no atomics, and the level's bookkeeping as above.
+template <int DT>
+__device__ void bfs_pull_rows_t(const Device &d, const uint32_t *F, uint32_t *N, uint32_t *Z, int32_t *nz_out, int32_t *words_out,
+                                int32_t *nwords_out, int32_t *levels, int depth, bool wide, uint32_t *s_need) {
+    const int lane = threadIdx.x & 31;
+    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int n_words = (d.mb + 1) / 2;
+    constexpr uint32_t NONE = 0xFFFFFFFFu;          // no entry: local column 31 never matches a 16-bit mask
+    constexpr int LONG_UNROLL = 8, MAX_ROUNDS = 8;
+    const int per_round = wide ? 8 : 4;
+    int n_found = 0, n_nz = 0;
+    for (int w0 = gwarp * 32; w0 < n_words; w0 += nwarps * 32) {
+        const int wd = w0 + lane;                    // this lane's word (bookkeeping); rows: lane = row of every word
+        const bool in = wd < n_words;
+        const uint32_t need = in ? ~d.ws.visited32[wd] : 0u;   // (rows without stored elements and rows past m count as visited)
+        if (in) Z[wd] = 0u;
+        if (!__any_sync(FULL, need != 0u)) { if (in) N[wd] = 0u; continue; }
+        uint32_t found = 0u;
+        // entries with a payload: the words that have any (their two row blocks' ranges), one word at a time
+        {
+            int pb0 = 0, pe0 = 0, pb1 = 0, pe1 = 0;
+            if (need) {
+                const int rb = 2 * wd;
+                if (rb < d.mb) { pb0 = d.csr.ptr[rb]; pe0 = d.csr_inl[rb]; }
+                if (rb + 1 < d.mb) { pb1 = d.csr.ptr[rb + 1]; pe1 = d.csr_inl[rb + 1]; }
+            }
+            uint32_t todo = __ballot_sync(FULL, need && (pe0 > pb0 || pe1 > pb1));
+            while (todo) {
+                const int k = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const uint32_t need_k = __shfl_sync(FULL, need, k);
+                uint32_t fk = 0u;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const uint32_t need16 = (need_k >> (16 * hf)) & 0xFFFFu;
+                    const int pbeg = __shfl_sync(FULL, hf ? pb1 : pb0, k), pend = __shfl_sync(FULL, hf ? pe1 : pe0, k);
+                    if (!need16 || pend <= pbeg) continue;        // warp-uniform
+                    uint32_t hit = 0;
+                    for (int base = pbeg; base < pend; base += 32) {
+                        const int pos = base + lane;
+                        if (pos < pend) {
+                            uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
+#ifdef DBS_BOUNDS_CHECK
+                            { uint32_t w_ = d.csr.w[pos]; DBS_CHK_ENTRY(d, true, idx, w_, aux); }
+#endif
+                            const uint32_t xm = mask_of(F, idx & IDX_MASK);
+                            if (xm) {
+                                const int type = idx >> TYPE_SHIFT;
+                                const uint32_t w = d.csr.w[pos];
+                                hit |= type == DBSPMSPV_BLK_COO ? lane_block_bool<DT>(type, w, aux, xm, d.payload)
+                                                                : lane_heavy_bool(type, d.payload + (size_t)w * 4, xm);
+                            }
+                        }
+                        hit = __reduce_or_sync(FULL, hit);
+                        if ((hit & need16) == need16) break;      // every wanted row of the block has a parent
+                    }
+                    fk |= (hit & need16) << (16 * hf);
+                }
+                if ((fk >> lane) & 1u) levels[(size_t)(w0 + k) * 32 + lane] = depth;
+                if (lane == k) found |= fk;
+            }
+        }
+        // rows: bit k of `mine` = row `lane` of word w0 + k is still wanted
+        __syncwarp();
+        s_need[lane] = need & ~found;
+        __syncwarp();
+        uint32_t mine = 0u;
+#pragma unroll 8
+        for (int k = 0; k < 32; ++k) mine |= ((s_need[k] >> lane) & 1u) << k;
+        uint32_t res = 0u, longm = 0u;
+        int k = 0, p = 0, e = 0, rounds = 0;
+        bool active = false;
+        // (the run of the lane's next row is fetched while the current one is walked)
+        int kn = 0, pn = 0, en = 0;
+        bool have_next = false;
+        auto fetch_next = [&]() {
+            have_next = mine != 0u;
+            if (have_next) {
+                kn = __ffs(mine) - 1;
+                mine &= mine - 1;
+                const size_t row = (size_t)(w0 + kn) * 32 + lane;
+                pn = d.rowrun_ptr[row];
+                en = d.rowrun_ptr[row + 1];
+            }
+        };
+        fetch_next();
+        while (__any_sync(FULL, active || have_next)) {
+            if (!active && have_next) {               // next row of this lane
+                k = kn; p = pn; e = en;
+                active = p < e;
+                rounds = 0;
+                fetch_next();
+            }
+            if (active) {
+                // a round = the aligned group(s) of four entries from position p on: 16-byte loads
+                const int q0 = p & ~3;
+                uint4 v4 = __ldcs(reinterpret_cast<const uint4 *>(d.rowrun_idx + q0)), w4 = make_uint4(NONE, NONE, NONE, NONE);   // (the array has slack behind its end)
+                if (wide && q0 + 4 < e) w4 = __ldcs(reinterpret_cast<const uint4 *>(d.rowrun_idx + q0 + 4));
+                uint32_t v[8] = {v4.x, v4.y, v4.z, v4.w, w4.x, w4.y, w4.z, w4.w}, xm[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) if (q0 + j < p || q0 + j >= e || (v[j] != NONE && !DBS_CHK_INDEX(d, v[j] & IDX_MASK, d.nb))) v[j] = NONE;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) xm[j] = v[j] != NONE ? mask_of(F, v[j] & IDX_MASK) : 0u;
+                bool got = false;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) got |= ((xm[j] >> (v[j] >> 27)) & 1u) != 0;
+                p = q0 + per_round;
+                if (got) { res |= 1u << k; levels[(size_t)(w0 + k) * 32 + lane] = depth; active = false; }
+                else if (p >= e) active = false;
+                else if (++rounds == MAX_ROUNDS) { longm |= 1u << k; active = false; }     // a long row: finished by the whole warp below
+            }
+        }
+        // long rows (hubs with no frontier neighbour among their first entries): the whole warp, 32 * LONG_UNROLL entries per round
+        uint32_t lanes_long = __ballot_sync(FULL, longm != 0u);
+        while (lanes_long) {
+            const int src = __ffs(lanes_long) - 1;
+            lanes_long &= lanes_long - 1;
+            uint32_t lm = __shfl_sync(FULL, longm, src);
+            while (lm) {
+                const int kk = __ffs(lm) - 1;
+                lm &= lm - 1;
+                const size_t row = (size_t)(w0 + kk) * 32 + src;
+                const int lp = (d.rowrun_ptr[row] & ~3) + MAX_ROUNDS * per_round, le = d.rowrun_ptr[row + 1];
+                bool hit = false;
+                for (int q = lp; q < le && !hit; q += 32 * LONG_UNROLL) {
+                    uint32_t v[LONG_UNROLL], xm[LONG_UNROLL];
+#pragma unroll
+                    for (int u = 0; u < LONG_UNROLL; ++u) {
+                        const int p_ = q + 32 * u + lane;
+                        v[u] = p_ < le ? d.rowrun_idx[p_] : NONE;
+                        if (v[u] != NONE && !DBS_CHK_INDEX(d, v[u] & IDX_MASK, d.nb)) v[u] = NONE;
+                    }
+#pragma unroll
+                    for (int u = 0; u < LONG_UNROLL; ++u) xm[u] = v[u] != NONE ? mask_of(F, v[u] & IDX_MASK) : 0u;
+                    bool m1 = false;
+#pragma unroll
+                    for (int u = 0; u < LONG_UNROLL; ++u) m1 |= ((xm[u] >> (v[u] >> 27)) & 1u) != 0;
+                    hit = __any_sync(FULL, m1);
+                }
+                if (hit && lane == src) { res |= 1u << kk; levels[row] = depth; }
+            }
+        }
+        // back to one word per lane: bit l of word w0 + k <- bit k of lane l's result
+#pragma unroll 8
+        for (int kk = 0; kk < 32; ++kk) {
+            const uint32_t fk = __ballot_sync(FULL, (res >> kk) & 1u);
+            if (lane == kk) found |= fk;
+        }
+        found &= need;
+        if (in) N[wd] = found;
+        if (found) d.ws.visited32[wd] |= found;
+        n_found += __popc(found);
+        n_nz += ((found & 0xFFFFu) != 0) + ((found >> 16) != 0);
+        const uint32_t listed = __ballot_sync(FULL, found != 0u);
+        if (listed) {
+            int base = 0;
+            if (lane == 0) base = atomicAdd(nwords_out, __popc(listed));
+            base = __shfl_sync(FULL, base, 0);
+            if (found) words_out[base + __popc(listed & ((1u << lane) - 1u))] = wd;
+        }
+    }
+    n_found = __reduce_add_sync(FULL, n_found);
+    n_nz = __reduce_add_sync(FULL, n_nz);
+    if (lane == 0 && n_found) { atomicAdd(&d.ws.ctr->bfs_reached, n_found); atomicAdd(nz_out, n_nz); }
+}
+
 // Per-level selector (Section 3.3.1): push iff N_nzblk / N_blk < th3.  Monotone in n_nzblk.
 __device__ __forceinline__ int bfs_path(int n_nzblk, int nb, float th3, int force_path) {
     if (force_path == DBSPMSPV_PATH_PUSH || force_path == DBSPMSPV_PATH_PULL) return force_path;
@@ -486,7 +660,7 @@ __device__ __forceinline__ int bfs_level_path(const Device &d, int cur, float th
 // that nothing is moved or reset behind an extra barrier.
 template <int DT>
 __device__ void bfs_level(const Device &d, cg::grid_group &grid, const Scope &sc, int lv, int32_t *levels, float th3,
-                          float edge_frac, int force_path) {
+                          float edge_frac, int force_path, uint32_t *s_need) {
     Counters *ctr = d.ws.ctr;
     const int lane = threadIdx.x & 31;
     const int n_words = (d.mb + 1) / 2;
@@ -517,8 +691,13 @@ __device__ void bfs_level(const Device &d, cg::grid_group &grid, const Scope &sc
     int4 *hubs_next = d.ws.hubs + nxt * HUB_CAP;
     if (path != DBSPMSPV_PATH_PUSH && d.rowrun_ptr != nullptr) {
         // a pull over the row-run index does its own bookkeeping (it owns the mask words it writes)
+#ifdef DBS_BFS_PULL_BY_WORD
         bfs_pull_rows<DT>(d, F, N, Z, &ctr->bfs_cnt[nxt][0], words_out, &ctr->bfs_nwords[q_out], levels, depth,
                           (float)n_nzblk < BFS_WIDE_PULL * (float)d.nb);
+#else
+        bfs_pull_rows_t<DT>(d, F, N, Z, &ctr->bfs_cnt[nxt][0], words_out, &ctr->bfs_nwords[q_out], levels, depth,
+                            (float)n_nzblk < BFS_WIDE_PULL * (float)d.nb, s_need + (threadIdx.x >> 5) * 32);
+#endif
         grid.sync();
     } else if (path == DBSPMSPV_PATH_PUSH) {
         bfs_push<DT>(d, sc, F, N, n_tasks, d.ws.hubs + cur * HUB_CAP, min(ctr->bfs_hubs[cur], HUB_CAP), levels, depth,
@@ -586,6 +765,7 @@ __device__ void bfs_level(const Device &d, cg::grid_group &grid, const Scope &sc
 template <int DT>
 __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t *levels, float th3, float edge_frac,
                                                  int force_path, int max_levels) {
+    __shared__ uint32_t s_need[BFS_CTA];                      // per warp: the wanted rows of its 32 words (transposed pull)
     cg::grid_group grid = cg::this_grid();
     const int tid = blockIdx.x * blockDim.x + threadIdx.x;
     const int nthreads = gridDim.x * blockDim.x;
@@ -635,7 +815,7 @@ __global__ void __launch_bounds__(BFS_CTA) k_bfs(Device d, int32_t src, int32_t 
     grid.sync();
     int lv = 0;
     while (lv < max_levels && ctr->bfs_cnt[lv % 3][0] != 0) {
-        bfs_level<DT>(d, grid, sc, lv, levels, th3, edge_frac, force_path);    // ends with a grid barrier
+        bfs_level<DT>(d, grid, sc, lv, levels, th3, edge_frac, force_path, s_need);    // ends with a grid barrier
         ++lv;
     }
     // leave the shared workspace as dbspmspv_run expects it: all masks clear.  The frontier before
