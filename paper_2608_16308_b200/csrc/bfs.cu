@@ -268,15 +268,23 @@ __device__ void bfs_pull(const Device &d, const Scope &sc, const uint32_t *F, ui
     }
 }
 
-// Boolean pull over the row-run index (square matrices, unless the index was switched off): a
-// warp takes the 32 rows of one mask word (two row blocks), lane = row.  Entries with a payload
-// are evaluated first, from the per-row-block position list; then every row that is still wanted
-// walks its own INLINE run and stops at its first frontier neighbour -- the early exit of
+// Boolean pull over the row-run index (square matrices, unless the index was switched off).
+// Entries with a payload are evaluated first, from the per-row-block position list, and a row
+// block is left as soon as each of its wanted rows has a parent; then every row that is still
+// wanted walks its own INLINE run and stops at its first frontier neighbour -- the early exit of
 // Algorithm 5 per row instead of per row block: in the big levels a row finds a parent within a
-// few entries, so a fraction of the edges is read at all.  Four entries are fetched per round
-// and lane (then their four frontier masks); a row that has not finished after eight rounds is
-// long (a hub with no frontier neighbour so far) and is finished by the whole warp, 32 entries
-// per step.  The warp owns its mask word: plain stores, no atomics.
+// few entries, so a fraction of the edges is read at all.
+// A warp takes a block of 32 consecutive mask words (1024 rows) and lane l walks row l of every
+// word, one row after the other, each lane at its own pace.  (With lane = row inside ONE word a
+// word costs as many dependent rounds as its slowest row -- and at the levels with a small
+// frontier almost every word holds a row without a frontier neighbour, which is walked to its
+// end -- so a warp's time would be the sum over its words of the maximum; here it is the maximum
+// over the lanes of the sum, about a third of the rounds.)  Four entries are fetched per round
+// and lane (eight when the frontier is small), then their frontier masks; the run of the lane's
+// next row is fetched meanwhile.  A row that has not finished after eight rounds is long (a hub
+// with no frontier neighbour so far) and is finished by the whole warp, 32 * 8 entries per step.
+// Found rows are collected as one bit per (lane, word) and transposed back with ballots, so the
+// warp owns its mask words: plain stores, no atomics.
 // a pull level over a frontier that fills fewer than this share of the vector blocks reads two groups of four entries per round
 #ifndef DBS_BFS_WIDE_PULL
 #define DBS_BFS_WIDE_PULL 0.3f
@@ -285,152 +293,6 @@ constexpr float BFS_WIDE_PULL = DBS_BFS_WIDE_PULL;
 
 template <int DT>
 __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, uint32_t *Z, int32_t *nz_out, int32_t *words_out,
-                              int32_t *nwords_out, int32_t *levels, int depth, bool wide) {
-    const int lane = threadIdx.x & 31;
-    const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int nwarps = (gridDim.x * blockDim.x) >> 5;
-    const int n_words = (d.mb + 1) / 2;
-    constexpr uint32_t NONE = 0xFFFFFFFFu;          // no entry: local column 31 never matches a 16-bit mask
-    constexpr int LONG_UNROLL = 8;
-    // This traversal also does the level's bookkeeping for its word (it owns it): the new
-    // frontier word is stored whatever its value (the buffer is not cleared beforehand), the
-    // buffer that comes into use two levels on is cleared, visited is updated, and the nonempty
-    // blocks, the vertices found and the nonzero words are counted / listed (in batches of 32
-    // words per warp) -- so a pull level needs no separate update pass and one grid barrier less.
-    int n_found = 0, n_nz = 0, n_batch = 0, batch_wd = 0;
-    auto flush_batch = [&]() {
-        int base = 0;
-        if (lane == 0) base = atomicAdd(nwords_out, n_batch);
-        base = __shfl_sync(FULL, base, 0);
-        if (lane < n_batch) words_out[base + lane] = batch_wd;
-        n_batch = 0;
-    };
-    // A word is a chain of dependent loads (visited word -> row pointers -> entries -> frontier
-    // masks): the visited word of the warp's next word is fetched a word ahead, and all pointers
-    // of a word -- both row blocks' payload ranges and the lane's row run -- in one round.
-    uint32_t need_next = gwarp < n_words ? ~d.ws.visited32[gwarp] : 0u;
-    for (int wd = gwarp; wd < n_words; wd += nwarps) {
-        const uint32_t need = need_next;             // (rows without stored elements and rows past m count as visited)
-        if (wd + nwarps < n_words) need_next = ~d.ws.visited32[wd + nwarps];
-        if (lane == 0) Z[wd] = 0u;
-        if (!need) { if (lane == 0) N[wd] = 0u; continue; }
-        uint32_t found = 0;
-        const int row = wd * 32 + lane;
-        int p = 0, e = 0;
-        if ((need >> lane) & 1u) { p = d.rowrun_ptr[row]; e = d.rowrun_ptr[row + 1]; }
-        int pb2[2] = {0, 0}, pe2[2] = {0, 0};
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-            const int rb = 2 * wd + hf;
-            if (rb < d.mb && ((need >> (16 * hf)) & 0xFFFFu)) { pb2[hf] = d.csr.ptr[rb]; pe2[hf] = d.csr_inl[rb]; }
-        }
-        // entries with a payload, one per lane
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-            const int rb = 2 * wd + hf;
-            const uint32_t need16 = (need >> (16 * hf)) & 0xFFFFu;
-            if (rb >= d.mb || !need16) continue;    // warp-uniform
-            const int pbeg = pb2[hf], pend = pe2[hf];                  // the row block's entries with a payload
-            // (32 entries per step; the walk stops as soon as every wanted row of the block has a
-            // parent -- the early exit of Algorithm 5: the row blocks of the hubs hold thousands of
-            // entries with a payload, and while the hubs are still unvisited one warp walked them all)
-            uint32_t hit = 0;
-            for (int base = pbeg; base < pend; base += 32) {
-                const int pos = base + lane;
-                if (pos < pend) {
-                    uint32_t idx = d.csr.idx[pos], aux = d.csr.aux[pos];
-#ifdef DBS_BOUNDS_CHECK
-                    { uint32_t w_ = d.csr.w[pos]; DBS_CHK_ENTRY(d, true, idx, w_, aux); }
-#endif
-                    const uint32_t xm = mask_of(F, idx & IDX_MASK);
-                    if (xm) {
-                        const int type = idx >> TYPE_SHIFT;
-                        const uint32_t w = d.csr.w[pos];
-                        hit |= type == DBSPMSPV_BLK_COO ? lane_block_bool<DT>(type, w, aux, xm, d.payload)
-                                                        : lane_heavy_bool(type, d.payload + (size_t)w * 4, xm);
-                    }
-                }
-                hit = __reduce_or_sync(FULL, hit);
-                if ((hit & need16) == need16) break;
-            }
-            if (pend > pbeg) found |= (hit & need16) << (16 * hf);
-        }
-        // row runs
-        bool active = (((need & ~found) >> lane) & 1u) && p < e;
-        bool got = false;
-        // a round = the aligned group of four entries that holds position p: one 16-byte load per
-        // lane (four 4-byte loads cost four trips through the L1 tag stage for the same line)
-        // (`wide`: the frontier is small, so a row that has a frontier neighbour at all finds it
-        // late and most rows are walked to their end -- two groups per round then halve the
-        // number of dependent rounds a word costs; with a large frontier the second group would
-        // mostly be read for nothing)
-        for (int round = 0; round < 8 && __any_sync(FULL, active); ++round) {
-            const int q0 = p & ~3;
-            uint4 v4 = make_uint4(NONE, NONE, NONE, NONE), w4 = make_uint4(NONE, NONE, NONE, NONE);
-            if (active) v4 = __ldcs(reinterpret_cast<const uint4 *>(d.rowrun_idx + q0));     // (the array has slack behind its end)
-            if (wide && active && q0 + 4 < e) w4 = __ldcs(reinterpret_cast<const uint4 *>(d.rowrun_idx + q0 + 4));
-            uint32_t v[8] = {v4.x, v4.y, v4.z, v4.w, w4.x, w4.y, w4.z, w4.w}, xm[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) if (q0 + j < p || q0 + j >= e || (v[j] != NONE && !DBS_CHK_INDEX(d, v[j] & IDX_MASK, d.nb))) v[j] = NONE;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) xm[j] = v[j] != NONE ? mask_of(F, v[j] & IDX_MASK) : 0u;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) got |= ((xm[j] >> (v[j] >> 27)) & 1u) != 0;
-            p = q0 + (wide ? 8 : 4);
-            if (got || p >= e) active = false;
-        }
-        uint32_t longm = __ballot_sync(FULL, active);
-        while (longm) {
-            const int src = __ffs(longm) - 1;
-            longm &= longm - 1;
-            const int lp = __shfl_sync(FULL, p, src), le = __shfl_sync(FULL, e, src);
-            bool hit = false;
-            // (eight steps of 32 entries per round: the entry loads of a round, then its mask
-            // gathers, are in flight together -- one step at a time costs two dependent round
-            // trips per 32 entries, and an unvisited hub row with few frontier neighbours has
-            // tens of thousands of entries)
-            for (int q = lp; q < le && !hit; q += 32 * LONG_UNROLL) {
-                uint32_t v[LONG_UNROLL], xm[LONG_UNROLL];
-#pragma unroll
-                for (int u = 0; u < LONG_UNROLL; ++u) {
-                    const int p_ = q + 32 * u + lane;
-                    v[u] = p_ < le ? d.rowrun_idx[p_] : NONE;
-                    if (v[u] != NONE && !DBS_CHK_INDEX(d, v[u] & IDX_MASK, d.nb)) v[u] = NONE;
-                }
-#pragma unroll
-                for (int u = 0; u < LONG_UNROLL; ++u) xm[u] = v[u] != NONE ? mask_of(F, v[u] & IDX_MASK) : 0u;
-                bool mine = false;
-#pragma unroll
-                for (int u = 0; u < LONG_UNROLL; ++u) mine |= ((xm[u] >> (v[u] >> 27)) & 1u) != 0;
-                hit = __any_sync(FULL, mine);
-            }
-            if (lane == src) got = hit;
-        }
-        found = (found | __ballot_sync(FULL, got)) & need;
-        if (lane == 0) N[wd] = found;
-        if (found) {
-            if (lane == 0) d.ws.visited32[wd] |= found;
-            if ((found >> lane) & 1u) levels[row] = depth;
-            n_found += __popc(found);
-            n_nz += ((found & 0xFFFFu) != 0) + ((found >> 16) != 0);
-            if (lane == n_batch) batch_wd = wd;
-            if (++n_batch == 32) flush_batch();
-        }
-    }
-    if (n_batch) flush_batch();
-    if (lane == 0 && n_found) { atomicAdd(&d.ws.ctr->bfs_reached, n_found); atomicAdd(nz_out, n_nz); }
-}
-
-// The same pull, transposed: a warp takes a block of 32 consecutive mask words (1024 rows) and
-// lane l walks row l of every word, one row after the other, each lane at its own pace.  With
-// lane = row inside ONE word (bfs_pull_rows above) a word costs as many dependent rounds as its
-// slowest row -- and at the levels with a small frontier almost every word holds a row without
-// a frontier neighbour, which is walked to its end -- so a warp's time is the sum over its words
-// of the maximum; here it is the maximum over the lanes of the sum, about a third of the rounds.
-// Found rows are collected as one bit per (lane, word) and transposed back with ballots, so the
-// warp still owns its mask words: plain stores, no atomics, and the level's bookkeeping as above.
-template <int DT>
-__device__ void bfs_pull_rows_t(const Device &d, const uint32_t *F, uint32_t *N, uint32_t *Z, int32_t *nz_out, int32_t *words_out,
                                 int32_t *nwords_out, int32_t *levels, int depth, bool wide, uint32_t *s_need) {
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -691,13 +553,8 @@ __device__ void bfs_level(const Device &d, cg::grid_group &grid, const Scope &sc
     int4 *hubs_next = d.ws.hubs + nxt * HUB_CAP;
     if (path != DBSPMSPV_PATH_PUSH && d.rowrun_ptr != nullptr) {
         // a pull over the row-run index does its own bookkeeping (it owns the mask words it writes)
-#ifdef DBS_BFS_PULL_BY_WORD
         bfs_pull_rows<DT>(d, F, N, Z, &ctr->bfs_cnt[nxt][0], words_out, &ctr->bfs_nwords[q_out], levels, depth,
-                          (float)n_nzblk < BFS_WIDE_PULL * (float)d.nb);
-#else
-        bfs_pull_rows_t<DT>(d, F, N, Z, &ctr->bfs_cnt[nxt][0], words_out, &ctr->bfs_nwords[q_out], levels, depth,
-                            (float)n_nzblk < BFS_WIDE_PULL * (float)d.nb, s_need + (threadIdx.x >> 5) * 32);
-#endif
+                          (float)n_nzblk < BFS_WIDE_PULL * (float)d.nb, s_need + (threadIdx.x >> 5) * 32);
         grid.sync();
     } else if (path == DBSPMSPV_PATH_PUSH) {
         bfs_push<DT>(d, sc, F, N, n_tasks, d.ws.hubs + cur * HUB_CAP, min(ctr->bfs_hubs[cur], HUB_CAP), levels, depth,
