@@ -274,8 +274,8 @@ __device__ void bfs_pull(const Device &d, const Scope &sc, const uint32_t *F, ui
 // wanted walks its own INLINE run and stops at its first frontier neighbour -- the early exit of
 // Algorithm 5 per row instead of per row block: in the big levels a row finds a parent within a
 // few entries, so a fraction of the edges is read at all.
-// A warp takes a block of 32 consecutive mask words (1024 rows) and lane l walks row l of every
-// word, one row after the other, each lane at its own pace.  (With lane = row inside ONE word a
+// A warp takes a block of 32 consecutive mask words (1024 rows) and lane l walks one row of
+// every word (row (l + k) mod 32 of the block's word k), one row after the other, each lane at its own pace.  (With lane = row inside ONE word a
 // word costs as many dependent rounds as its slowest row -- and at the levels with a small
 // frontier almost every word holds a row without a frontier neighbour, which is walked to its
 // end -- so a warp's time would be the sum over its words of the maximum; here it is the maximum
@@ -353,13 +353,15 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
                 if (lane == k) found |= fk;
             }
         }
-        // rows: bit k of `mine` = row `lane` of word w0 + k is still wanted
+        // rows: bit k of `mine` = row (lane + k) mod 32 of word w0 + k is still wanted.  (The rotation matters where
+        // the degree goes with the low bits of the row number, as in an R-MAT graph that was not relabelled: with
+        // row = lane, lane 0 would own the heaviest row of every word.)
         __syncwarp();
         s_need[lane] = need & ~found;
         __syncwarp();
         uint32_t mine = 0u;
 #pragma unroll 8
-        for (int k = 0; k < 32; ++k) mine |= ((s_need[k] >> lane) & 1u) << k;
+        for (int k = 0; k < 32; ++k) mine |= ((s_need[k] >> ((lane + k) & 31)) & 1u) << k;
         uint32_t res = 0u, longm = 0u;
         int k = 0, p = 0, e = 0, rounds = 0;
         bool active = false;
@@ -371,7 +373,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             if (have_next) {
                 kn = __ffs(mine) - 1;
                 mine &= mine - 1;
-                const size_t row = (size_t)(w0 + kn) * 32 + lane;
+                const size_t row = (size_t)(w0 + kn) * 32 + ((lane + kn) & 31);
                 pn = d.rowrun_ptr[row];
                 en = d.rowrun_ptr[row + 1];
             }
@@ -398,7 +400,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
 #pragma unroll
                 for (int j = 0; j < 8; ++j) got |= ((xm[j] >> (v[j] >> 27)) & 1u) != 0;
                 p = q0 + per_round;
-                if (got) { res |= 1u << k; levels[(size_t)(w0 + k) * 32 + lane] = depth; active = false; }
+                if (got) { res |= 1u << k; levels[(size_t)(w0 + k) * 32 + ((lane + k) & 31)] = depth; active = false; }
                 else if (p >= e) active = false;
                 else if (++rounds == MAX_ROUNDS) { longm |= 1u << k; active = false; }     // a long row: finished by the whole warp below
             }
@@ -412,7 +414,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             while (lm) {
                 const int kk = __ffs(lm) - 1;
                 lm &= lm - 1;
-                const size_t row = (size_t)(w0 + kk) * 32 + src;
+                const size_t row = (size_t)(w0 + kk) * 32 + ((src + kk) & 31);
                 const int lp = (d.rowrun_ptr[row] & ~3) + MAX_ROUNDS * per_round, le = d.rowrun_ptr[row + 1];
                 bool hit = false;
                 for (int q = lp; q < le && !hit; q += 32 * LONG_UNROLL) {
@@ -433,11 +435,11 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
                 if (hit && lane == src) { res |= 1u << kk; levels[row] = depth; }
             }
         }
-        // back to one word per lane: bit l of word w0 + k <- bit k of lane l's result
+        // back to one word per lane: bit (l + k) mod 32 of word w0 + k <- bit k of lane l's result
 #pragma unroll 8
         for (int kk = 0; kk < 32; ++kk) {
             const uint32_t fk = __ballot_sync(FULL, (res >> kk) & 1u);
-            if (lane == kk) found |= fk;
+            if (lane == kk) found |= __funnelshift_l(fk, fk, kk);
         }
         found &= need;
         if (in) N[wd] = found;
