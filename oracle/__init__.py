@@ -3,7 +3,7 @@ cpu_baseline leg).  The product path never imports this package.
 
 Thin ctypes wrapper over ``ref_spmspv.c``: the textbook push and pull SpMSpV loops of
 Algorithm 1 (Section 2.1) in fp64, a queue BFS, and the dense-output decode variant
-(Section 4.3).  The C file is compiled with gcc on first use (``build()``).  Shares no code
+(Section 4.3), and the (min, +) product with a Bellman-Ford search.  The C file is compiled with gcc on first use (``build()``).  Shares no code
 with the CUDA library and does not import it.
 """
 from __future__ import annotations
@@ -39,6 +39,8 @@ def _load():
         _lib.ref_bfs.restype = ctypes.c_int64
         _lib.ref_csr_to_csc.restype = None
         _lib.ref_decode.restype = None
+        _lib.ref_minplus.restype = ctypes.c_int64
+        _lib.ref_sssp.restype = ctypes.c_int64
     return _lib
 
 
@@ -150,3 +152,51 @@ def ref_decode(A: RefMatrix, x_dense):
     _load().ref_decode(_i64(A.m), _i64(A.n), _p(A.row_ptr), _p(A.col_idx), _p(A.val), _p(x),
                        _p(y), _p(s))
     return y, s
+
+
+def ref_minplus(A: RefMatrix, x_idx, x_val=None):
+    """(min, +) SpMSpV: y_i = min_j (A[i][j] + x_j) over stored A[i][j] and listed x_j.
+    x_val None -> every listed entry is 0; a pattern matrix -> every weight is 1.
+    Returns (y_idx int32 ascending, y_val fp64)."""
+    x_idx = _prep(x_idx, np.int32)
+    x_val = _prep(x_val, np.float32)
+    y_idx = np.empty(A.m, dtype=np.int32)
+    y_val = np.empty(A.m, dtype=np.float64)
+    cnt = _load().ref_minplus(_i64(A.m), _i64(A.n), _p(A.row_ptr), _p(A.col_idx), _p(A.val),
+                              _i64(x_idx.size), _p(x_idx), _p(x_val), _p(y_idx), _p(y_val))
+    if cnt < 0:
+        raise MemoryError("oracle allocation failed")
+    return y_idx[:cnt].copy(), y_val[:cnt].copy()
+
+
+def ref_sssp(A: RefMatrix, src: int) -> np.ndarray:
+    """Bellman-Ford sweeps; A[i][j] stored = edge j -> i of weight A[i][j] (1 for a pattern
+    matrix).  fp64 distances, source 0, unreachable +inf."""
+    if A.m != A.n:
+        raise ValueError("SSSP needs a square matrix")
+    col_ptr, row_idx, cval = A.csc()
+    dist = np.empty(A.n, dtype=np.float64)
+    sweeps = _load().ref_sssp(_i64(A.n), _p(col_ptr), _p(row_idx), _p(cval), ctypes.c_int32(int(src)), _p(dist))
+    if sweeps < 0:
+        raise ValueError("negative cycle")
+    return dist
+
+
+def ref_sssp_frontier(A: RefMatrix, src: int) -> np.ndarray:
+    """The same search as the iteration of (min, +) SpMSpV steps a frontier-driven driver
+    makes: x = the vertices whose distance improved in the last step, with their distances;
+    y = A (min,+) x; every y_i below dist_i replaces it and puts i on the next frontier.
+    Cross-check for ref_sssp."""
+    dist = np.full(A.n, np.inf, dtype=np.float64)
+    dist[src] = 0.0
+    frontier = np.asarray([src], dtype=np.int32)
+    steps = 0
+    while frontier.size:
+        steps += 1
+        if steps > A.n + 1:
+            raise ValueError("negative cycle")
+        y_idx, y_val = ref_minplus(A, frontier, dist[frontier].astype(np.float32))
+        better = y_val < dist[y_idx]
+        dist[y_idx[better]] = y_val[better]
+        frontier = y_idx[better]
+    return dist

@@ -161,3 +161,68 @@ void ref_decode(int64_t m, int64_t n, const int64_t *row_ptr, const int32_t *col
         if (y_scale) y_scale[i] = scale;
     }
 }
+
+/* (min, +) SpMSpV: Algorithm 1 (pull half) with the sum of products replaced by the minimum
+ * of sums, y_i = min over stored A[i][j] with x_j listed of (A[i][j] + x_j) -- the product
+ * that GraphBLAS-style systems (Sections 1 and 6) iterate for single-source shortest paths.
+ * A listed x_j = 0 takes part (an absent entry is +infinity, not 0); val == NULL: every
+ * stored element has weight 1.  Row i is reported iff a stored element meets a listed entry.
+ * Pins: brute force over a dense matrix, x = {j: 0} returns column j, pattern matrix with a
+ * zero-valued frontier gives hop counts (BFS levels).                                       */
+int64_t ref_minplus(int64_t m, int64_t n, const int64_t *row_ptr, const int32_t *col_idx,
+                    const float *val, int64_t nnz_x, const int32_t *x_idx, const float *x_val,
+                    int32_t *y_idx, double *y_val)
+{
+    uint8_t *present = (uint8_t *)calloc((size_t)(n > 0 ? n : 1), 1);
+    double *xs = (double *)calloc((size_t)(n > 0 ? n : 1), sizeof(double));
+    if (!present || !xs) { free(present); free(xs); return -1; }
+    for (int64_t k = 0; k < nnz_x; ++k) {
+        present[x_idx[k]] = 1;
+        xs[x_idx[k]] = x_val ? (double)x_val[k] : 0.0;
+    }
+    int64_t cnt = 0;
+    for (int64_t i = 0; i < m; ++i) {
+        double best = INFINITY;
+        int hit = 0;
+        for (int64_t p = row_ptr[i]; p < row_ptr[i + 1]; ++p) {
+            int32_t j = col_idx[p];
+            if (present[j]) {
+                double t = (val ? (double)val[p] : 1.0) + xs[j];
+                if (!hit || t < best) best = t;
+                hit = 1;
+            }
+        }
+        if (hit) {
+            y_idx[cnt] = (int32_t)i;
+            y_val[cnt] = best;
+            ++cnt;
+        }
+    }
+    free(present);
+    free(xs);
+    return cnt;
+}
+
+/* Single-source shortest paths by Bellman-Ford sweeps: dist[src] = 0, everything else
+ * +infinity; every sweep relaxes every edge (a stored A[i][j] is the edge j -> i of weight
+ * A[i][j], as in ref_bfs) until a sweep changes nothing.  Weights must not close a negative
+ * cycle (at most n sweeps are made).  Returns the number of sweeps, -1 if it did not settle.
+ * Pins: a library Dijkstra, path and star graphs in closed form, unit weights == BFS levels. */
+int64_t ref_sssp(int64_t n, const int64_t *col_ptr, const int32_t *row_idx, const float *cval,
+                 int32_t src, double *dist)
+{
+    for (int64_t v = 0; v < n; ++v) dist[v] = INFINITY;
+    dist[src] = 0.0;
+    for (int64_t sweep = 1; sweep <= n + 1; ++sweep) {
+        int changed = 0;
+        for (int64_t j = 0; j < n; ++j) {
+            if (isinf(dist[j])) continue;
+            for (int64_t p = col_ptr[j]; p < col_ptr[j + 1]; ++p) {
+                double t = dist[j] + (cval ? (double)cval[p] : 1.0);
+                if (t < dist[row_idx[p]]) { dist[row_idx[p]] = t; changed = 1; }
+            }
+        }
+        if (!changed) return sweep;
+    }
+    return -1;
+}

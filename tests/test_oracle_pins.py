@@ -206,3 +206,89 @@ def test_decode_small_integers_exact_and_negative_zero_is_zero():
     y, s = oracle.ref_decode(_mat(wl.csr_from_dense(a)), x)
     assert y.tolist() == [6.0, 0.0, 10.0]
     assert s.tolist() == [6.0, 0.0, 10.0]
+
+
+# ---- (min, +) product and shortest paths -------------------------------------------------
+
+@pytest.mark.parametrize("m,n,nnz,k,seed", [(1, 1, 1, 1, 0), (7, 5, 12, 3, 1), (33, 64, 300, 9, 2),
+                                            (64, 64, 900, 64, 3), (50, 50, 60, 0, 5)])
+def test_minplus_brute_force_dense(m, n, nnz, k, seed):
+    """(min, +) product vs the definition on a dense copy with explicit structure masks (numpy):
+    absent entries are +inf, not 0; rows with no (stored, listed) pair are absent."""
+    csr = wl.random_sparse(m, n, nnz, seed)
+    a, s = _dense(csr)
+    rng = np.random.default_rng(100 + seed)
+    x_idx = np.sort(rng.choice(n, size=k, replace=False)).astype(np.int32)
+    x_val = rng.standard_normal(k).astype(np.float32)
+    y_idx, y_val = oracle.ref_minplus(_mat(csr), x_idx, x_val)
+    big = np.where(s[:, x_idx], a[:, x_idx] + x_val.astype(np.float64)[None, :], np.inf) if k else np.full((m, 0), np.inf)
+    want_rows = np.flatnonzero(s[:, x_idx].any(axis=1)) if k else np.zeros(0, dtype=np.int64)
+    assert np.array_equal(y_idx, want_rows)
+    if k:
+        assert np.array_equal(y_val, big.min(axis=1)[want_rows])
+
+
+def test_minplus_single_zero_entry_returns_the_column():
+    """x = {j: 0}: y is column j of A, stored zeros and negative weights included (a listed 0
+    takes part; with 0 read as "absent" the result would be empty)."""
+    a = np.zeros((5, 4))
+    a[0, 2], a[3, 2], a[4, 2], a[1, 1] = 2.5, -1.0, 7.0, 3.0
+    csr = wl.csr_from_dense(a)
+    y_idx, y_val = oracle.ref_minplus(_mat(csr), np.asarray([2], np.int32), np.asarray([0.0], np.float32))
+    assert y_idx.tolist() == [0, 3, 4] and y_val.tolist() == [2.5, -1.0, 7.0]
+    # the minimum, not the sum and not the last one: two listed columns meet row 0
+    a[0, 1] = 1.0
+    csr = wl.csr_from_dense(a)
+    y_idx, y_val = oracle.ref_minplus(_mat(csr), np.asarray([1, 2], np.int32), np.asarray([0.25, 0.0], np.float32))
+    assert y_idx.tolist() == [0, 1, 3, 4] and y_val.tolist() == [1.25, 3.25, -1.0, 7.0]
+
+
+def _weighted(n, edges):
+    a = np.zeros((n, n))
+    for u, v, w in edges:
+        a[v, u] = w
+    return _mat(wl.csr_from_dense(a))
+
+
+def test_sssp_path_star_and_orientation():
+    n = 30
+    w = [(i % 5) + 0.5 for i in range(n - 1)]
+    g = _weighted(n, [(i, i + 1, w[i]) for i in range(n - 1)])          # directed path 0 -> 1 -> ...
+    want = np.concatenate([[0.0], np.cumsum(w)])
+    assert np.array_equal(oracle.ref_sssp(g, 0), want)
+    d5 = oracle.ref_sssp(g, 5)
+    assert np.all(np.isinf(d5[:5])) and np.array_equal(d5[5:], want[5:] - want[5])   # nothing upstream is reached
+    # a shortcut that is longer in hops but shorter in weight wins: 0 -> 1 (10), 0 -> 2 (1), 2 -> 3 (1), 3 -> 1 (1)
+    g = _weighted(4, [(0, 1, 10.0), (0, 2, 1.0), (2, 3, 1.0), (3, 1, 1.0)])
+    assert oracle.ref_sssp(g, 0).tolist() == [0.0, 3.0, 1.0, 2.0]
+    assert oracle.ref_sssp_frontier(g, 0).tolist() == [0.0, 3.0, 1.0, 2.0]
+
+
+def test_sssp_unit_weights_equal_bfs_levels():
+    csr = wl.random_sparse(300, 300, 800, 77, values=False)
+    g = _mat(csr)
+    for src in (0, 150):
+        lv = oracle.ref_bfs(g, src).astype(np.float64)
+        lv[lv < 0] = np.inf
+        assert np.array_equal(oracle.ref_sssp(g, src), lv)
+        assert np.array_equal(oracle.ref_sssp_frontier(g, src), lv)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_sssp_equals_library_dijkstra_and_frontier_form(seed):
+    """Bellman-Ford sweeps vs scipy's Dijkstra on positive weights that are exact in binary
+    (multiples of 1/8: every path sum is exact, so the comparison is for equality), and vs the
+    frontier-driven iteration of (min, +) products."""
+    import scipy.sparse as sp
+    from scipy.sparse.csgraph import dijkstra
+    n = 500
+    csr = wl.random_sparse(n, n, 3000, 300 + seed)
+    rng = np.random.default_rng(seed)
+    val = (rng.integers(1, 64, size=csr.nnz) / 8.0).astype(np.float32)
+    g = oracle.RefMatrix(n, n, csr.row_ptr, csr.col_idx, val)
+    # scipy: entry [u, v] = edge u -> v; the stored A[i][j] is the edge j -> i, so pass the transpose
+    m_lib = sp.csr_matrix((val.astype(np.float64), csr.col_idx, csr.row_ptr), shape=(n, n)).T.tocsr()
+    for src in (0, 123):
+        want = dijkstra(m_lib, directed=True, indices=src)
+        assert np.array_equal(oracle.ref_sssp(g, src), want)
+        assert np.array_equal(oracle.ref_sssp_frontier(g, src), want)
