@@ -61,7 +61,9 @@ typedef enum {
 
 typedef enum {
     DBSPMSPV_PLUS_TIMES = 0,
-    DBSPMSPV_OR_AND = 1 /* Boolean: only reachability is computed (Section 4.2)            */
+    DBSPMSPV_OR_AND = 1, /* Boolean: only reachability is computed (Section 4.2)           */
+    DBSPMSPV_MIN_PLUS = 2 /* y_i = min_j (A[i][j] + x_j): the shortest-path product of
+                             GraphBLAS-style systems (Sections 1, 6)                       */
 } dbspmspv_semiring_t;
 
 enum { DBSPMSPV_PATH_AUTO = 0, DBSPMSPV_PATH_PUSH = 1, DBSPMSPV_PATH_PULL = 2 };
@@ -230,7 +232,11 @@ int dbspmspv_create_coo(dbspmspv_handle_t *out, int64_t m, int64_t n, int64_t nn
  *   x_idx    nnz_x distinct indices in [0, n), any order; x_val nnz_x values of the handle's
  *            dtype (float, or bf16 bit patterns; ignored/NULL for OR_AND).  Both must stay
  *            valid and unchanged until the call has finished on the stream.
- *   semiring PLUS_TIMES (F32/BF16 handles) or OR_AND (any handle; values are then 1.0f)
+ *   semiring PLUS_TIMES (F32/BF16 handles), OR_AND (any handle; values are then 1.0f) or
+ *            MIN_PLUS (any handle; a pattern handle's elements weigh 1): y_i is the smallest
+ *            A[i][j] + x_j over the stored elements of row i whose x_j is listed, in fp32; a
+ *            listed 0 takes part like any other value; NaN operands give unspecified values.
+ *            MIN_PLUS always takes the push path (force_path is ignored).
  *   y_idx    out: row indices of the structural result, ascending; y_val out: fp32 sums
  *            (may be NULL for OR_AND); both with room for y_capacity entries
  *   y_nnz    out: one int32, the number of result entries (the full count even when it

@@ -17,7 +17,7 @@ LIB_PATH = os.environ.get("DBSPMSPV_LIBRARY") or os.path.join(HERE, "libdbspmspv
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_CAPACITY, ERR_TIMEOUT, ERR_BOUNDS, ERR_TOO_LARGE, ERR_INTERNAL = range(10)
 F32, BF16, PATTERN = 0, 1, 2
-PLUS_TIMES, OR_AND = 0, 1
+PLUS_TIMES, OR_AND, MIN_PLUS = 0, 1, 2
 PATH_AUTO, PATH_PUSH, PATH_PULL = 0, 1, 2
 FORMAT_AUTO, FORMAT_COO, FORMAT_CSR = 0, 1, 2
 BLK_INLINE, BLK_COO, BLK_FCSR, BLK_FCSC, BLK_CSR, BLK_DENSE = range(6)

@@ -1567,6 +1567,7 @@ k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, flo
 
 }  // namespace dbs
 #include "decode_batch.cuh"
+#include "minplus.cuh"
 namespace dbs {
 
 // ------------------------------------------------------------------------------------------
@@ -1724,7 +1725,8 @@ __global__ void __launch_bounds__(CMP_TPB) k_compact_write(Device d, int32_t *__
             for (int bit = 0; bit < 8; ++bit) {
                 if ((bits >> bit) & 1u) {
                     s_oidx[pos] = row0 + bit;
-                    s_oval[pos] = boolean ? 1.0f : v[bit];
+                    // boolean 1: a Boolean result; 2: the accumulator holds (min, +) keys
+                    s_oval[pos] = boolean == 1 ? 1.0f : boolean == 2 ? minplus_value(__float_as_uint(v[bit])) : v[bit];
                     ++pos;
                 }
             }
@@ -1964,7 +1966,8 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     const Device &d = h->d;
     // x lists a quarter of the columns or more: a pull is likely (on hypersparse matrices), so
     // the worklist is built afterwards from the masks, and only if the selector does choose the push
-    const bool late_emit = !h->heavy_stage && h->ropts.force_path != DBSPMSPV_PATH_PUSH && (int64_t)nnz_x * 4 >= d.n;
+    const bool minplus = semiring == DBSPMSPV_MIN_PLUS;     // always the push: the worklist is built with the vector blocking
+    const bool late_emit = !minplus && !h->heavy_stage && h->ropts.force_path != DBSPMSPV_PATH_PUSH && (int64_t)nnz_x * 4 >= d.n;
     const void *xv = semiring == DBSPMSPV_OR_AND ? nullptr : x_val;
     if (nnz_x > 0) {
         const int g = (nnz_x + XB_TPB - 1) / XB_TPB;
@@ -1984,9 +1987,12 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     // private accumulators for the hub row blocks: when x is long enough for their atomics to
     // queue up, and not so long that the call will most likely pull
     const int hub_min = h->ropts.hub_min_nnz_x ? h->ropts.hub_min_nnz_x : HUB_MIN_NNZ_X;
-    h->d.hub_on = d.n_hub_blocks > 0 && hub_min > 0 && nnz_x >= hub_min && h->ropts.force_path != DBSPMSPV_PATH_PULL &&
+    h->d.hub_on = !minplus && d.n_hub_blocks > 0 && hub_min > 0 && nnz_x >= hub_min && h->ropts.force_path != DBSPMSPV_PATH_PULL &&
                   (!late_emit || h->heavy_stage);
-    if (nnz_x > 0 && d.n_entries > 0) {
+    if (minplus && nnz_x > 0 && d.n_entries > 0) {
+        DBS_CUDA(launch_pdl(k_minplus_push<DT>, 4 * h->sm_count, MINPLUS_CTA, 0, st, d));
+        ++h->kernel_launches;
+    } else if (nnz_x > 0 && d.n_entries > 0) {
         int s = DBSPMSPV_OK;
         if (h->heavy_stage) {
             s = launch_compute<DT, OutSparse, 1>(h, out, h->ropts.th3, true, st);
@@ -2012,7 +2018,7 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     if (extra > 4 * h->sm_count) extra = 4 * h->sm_count;
     const int clear_all = (int64_t)nnz_x * 8 > d.n;     // scattered clears cost more than a full sweep
     DBS_CUDA(launch_pdl(k_compact_write, nt + extra, CMP_TPB, 0, st, d, y_idx, y_val, y_capacity, y_nnz,
-                        (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x, clear_all, parity, row_mask, complement));
+                        minplus ? 2 : (int)(semiring == DBSPMSPV_OR_AND || DT == DBSPMSPV_PATTERN), x_idx, nnz_x, clear_all, parity, row_mask, complement));
     DBS_CUDA(cudaGetLastError());
     return DBSPMSPV_OK;
 }
@@ -2229,11 +2235,9 @@ static int run_checked(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_
     if (!h || nnz_x < 0 || y_capacity < 0 || !y_nnz) return DBSPMSPV_ERR_INVALID_ARG;
     if (nnz_x > 0 && !x_idx) return DBSPMSPV_ERR_INVALID_ARG;
     if (y_capacity > 0 && !y_idx) return DBSPMSPV_ERR_INVALID_ARG;
-    if (semiring != DBSPMSPV_PLUS_TIMES && semiring != DBSPMSPV_OR_AND) return DBSPMSPV_ERR_INVALID_ARG;
-    if (semiring == DBSPMSPV_PLUS_TIMES) {
-        if (h->d.dtype == DBSPMSPV_PATTERN) return DBSPMSPV_ERR_UNSUPPORTED;
-        if ((nnz_x > 0 && !x_val) || (y_capacity > 0 && !y_val)) return DBSPMSPV_ERR_INVALID_ARG;
-    }
+    if (semiring != DBSPMSPV_PLUS_TIMES && semiring != DBSPMSPV_OR_AND && semiring != DBSPMSPV_MIN_PLUS) return DBSPMSPV_ERR_INVALID_ARG;
+    if (semiring == DBSPMSPV_PLUS_TIMES && h->d.dtype == DBSPMSPV_PATTERN) return DBSPMSPV_ERR_UNSUPPORTED;
+    if (semiring != DBSPMSPV_OR_AND && ((nnz_x > 0 && !x_val) || (y_capacity > 0 && !y_val))) return DBSPMSPV_ERR_INVALID_ARG;
     if ((int64_t)nnz_x > h->d.n) return DBSPMSPV_ERR_INVALID_ARG;
     if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

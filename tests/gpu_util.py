@@ -53,7 +53,7 @@ class Handle:
     def run(self, x: wl.SparseVec, semiring=B.PLUS_TIMES, capacity=None):
         xi = torch.from_numpy(np.ascontiguousarray(x.idx, dtype=np.int32)).to(DEV)
         xv = None
-        if x.val is not None and semiring == B.PLUS_TIMES:
+        if x.val is not None and semiring != B.OR_AND:
             if self.dtype == B.BF16:
                 xv = torch.from_numpy(to_bf16_bits(x.val).view(np.int16)).to(DEV)
             else:
