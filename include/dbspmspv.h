@@ -262,6 +262,23 @@ int dbspmspv_run(dbspmspv_handle_t h, const int32_t *x_idx, const void *x_val, i
 int db_bfs(dbspmspv_handle_t h, int32_t src, int32_t *levels, dbspmspv_stream_t stream);
 
 /*
+ * Single-source shortest paths as the iteration of MIN_PLUS products (SpMSpV as the primitive
+ * of GraphBLAS-style graph algorithms, Sections 1 and 6): x holds the vertices whose distance
+ * improved in the last step, y = A (min,+) x relaxes their out-edges, the improved rows of y
+ * become the next x.  A stored A[i][j] is the edge j -> i of weight A[i][j] (1 on a pattern
+ * handle), as in db_bfs.  Weights may be negative as long as no cycle is.
+ *   src      source vertex in [0, n); square F32 or PATTERN handle (BF16: ERR_UNSUPPORTED)
+ *   dist     out: n fp32 on the device; source 0, unreachable +infinity.  Every path sum is
+ *            accumulated in fp32 in path order.
+ *   n_steps  out (host, may be NULL): products made, the last one with an empty result
+ * Unlike the other calls this one is a host loop: it waits on `stream` once per step to read
+ * the size of the next x (4 bytes), and the first call on a handle allocates 24 n bytes of
+ * device memory and one page-locked word (freed by dbspmspv_destroy).  More than n + 1 steps
+ * (a negative cycle) end the search with ERR_UNSUPPORTED.
+ */
+int db_sssp(dbspmspv_handle_t h, int32_t src, float *dist, int32_t *n_steps, dbspmspv_stream_t stream);
+
+/*
  * Single-token linear layer (Section 4.3): dense x in, dense y out.  The nonzero mask of x is
  * generated on the GPU by warp ballot (Section 4.1) and drives the same engine.
  *   x        n values of the handle's dtype (F32 or BF16 handles); zeros (+0.0 and -0.0) are

@@ -26,7 +26,7 @@ MAX_BFS_LEVELS_RECORDED = 64
 
 EXPORTED_SYMBOLS = (
     "dbspmspv_default_create_opts", "dbspmspv_default_run_opts", "dbspmspv_create_csr",
-    "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "dbspmspv_decode", "dbspmspv_get_stats",
+    "dbspmspv_create_coo", "dbspmspv_run", "db_bfs", "db_sssp", "dbspmspv_decode", "dbspmspv_get_stats",
     "dbspmspv_export_coo", "dbspmspv_export_blocks", "dbspmspv_export_views",
     "dbspmspv_set_run_opts", "dbspmspv_destroy", "dbspmspv_strerror", "dbspmspv_compact_noalloc",
     "dbspmspv_test_bounded_wait", "dbspmspv_test_corrupt_entry", "dbspmspv_decode_batch", "dbspmspv_run_masked", "dbspmspv_count_call_bytes", "dbspmspv_probe_floor",
@@ -102,6 +102,7 @@ def lib() -> ctypes.CDLL:
         L.dbspmspv_run.argtypes = [vp, vp, vp, i32, ctypes.c_int, vp, vp, i64, vp, vp]
         L.dbspmspv_run_masked.argtypes = [vp, vp, vp, i32, ctypes.c_int, vp, ctypes.c_int, vp, vp, i64, vp, vp]
         L.db_bfs.argtypes = [vp, i32, vp, vp]
+        L.db_sssp.argtypes = [vp, i32, vp, ctypes.POINTER(ctypes.c_int32), vp]
         L.dbspmspv_decode.argtypes = [vp, vp, vp, vp]
         L.dbspmspv_decode_batch.argtypes = [vp, vp, i64, vp, i64, i32, vp]
         L.dbspmspv_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
@@ -192,6 +193,13 @@ def dbspmspv_run(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_n
 
 def db_bfs(h, src, levels, stream: Optional[int] = None) -> None:
     _check(lib().db_bfs(h, src, _ptr(levels), _stream() if stream is None else stream), "db_bfs")
+
+
+def db_sssp(h, src, dist, stream: Optional[int] = None) -> int:
+    """Returns the number of (min, +) products the search made."""
+    steps = ctypes.c_int32(0)
+    _check(lib().db_sssp(h, src, _ptr(dist), ctypes.byref(steps), _stream() if stream is None else stream), "db_sssp")
+    return int(steps.value)
 
 
 def dbspmspv_decode(h, x, y, stream: Optional[int] = None) -> None:

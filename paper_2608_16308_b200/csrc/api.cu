@@ -208,6 +208,8 @@ int dbspmspv_destroy(dbspmspv_handle_t h) {
     cudaFree(const_cast<uint16_t *>(d.hub_slot)); cudaFree(const_cast<int32_t *>(d.hub_rb)); cudaFree(d.hub_acc);
     cudaFree(h->csc2csr); cudaFree(h->block_row);
     cudaFree(h->ws_arena);
+    cudaFree(h->sssp_arena);
+    if (h->sssp_host) cudaFreeHost(h->sssp_host);
     if (h->ev[0]) cudaEventDestroy(h->ev[0]);
     if (h->ev[1]) cudaEventDestroy(h->ev[1]);
     delete h;
@@ -225,6 +227,7 @@ const char *dbspmspv_strerror(int status) {
         case DBSPMSPV_ERR_TIMEOUT: return "bounded device wait ran out";
         case DBSPMSPV_ERR_BOUNDS: return "x index out of range";
         case DBSPMSPV_ERR_TOO_LARGE: return "more rows than the fixed scratch of the no-allocation entry point covers";
+        case DBSPMSPV_ERR_INTERNAL: return "a range check failed inside a kernel (range-checked build)";
         default: return "unknown status";
     }
 }

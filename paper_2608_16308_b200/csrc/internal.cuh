@@ -287,6 +287,8 @@ struct dbspmspv_handle_s {
     int64_t hub_bytes;
     int64_t stage_index_bytes;
     void *ws_arena;             // the one allocation that holds the whole workspace
+    void *sssp_arena;           // db_sssp: frontier lists, y and counters (allocated by the first search)
+    int32_t *sssp_host;         // db_sssp: page-locked word the size of the next frontier is copied to
     cudaStream_t last_stream;   // stream of the last run / decode / bfs call (get_stats waits on it)
 };
 

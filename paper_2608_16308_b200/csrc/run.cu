@@ -2204,6 +2204,86 @@ static int decode_batch_typed(dbspmspv_handle_s *h, const void *x, int64_t ldx, 
     return DBSPMSPV_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// db_sssp: single-source shortest paths as the iteration of (min, +) products (Sections 1, 6:
+// SpMSpV as the primitive of GraphBLAS-style graph algorithms).  x = the vertices whose
+// distance improved in the last step, with their distances; y = A (min,+) x; every y_i below
+// dist_i replaces it and puts i on the next x.  The rows of y are distinct, so the relaxation
+// needs no atomics on dist.
+// ------------------------------------------------------------------------------------------
+__global__ void k_sssp_init(float *dist, int64_t n, int32_t src, int32_t *x_idx, float *x_val, int32_t *count) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < n; v += stride) dist[v] = v == src ? 0.0f : __int_as_float(0x7F800000);
+    if (blockIdx.x == 0 && threadIdx.x == 0) { x_idx[0] = src; x_val[0] = 0.0f; *count = 0; }
+}
+
+__global__ void k_sssp_relax(const int32_t *__restrict__ y_idx, const float *__restrict__ y_val, const int32_t *__restrict__ y_nnz,
+                             float *__restrict__ dist, int32_t *__restrict__ x_idx, float *__restrict__ x_val, int32_t *count) {
+    const int n = *y_nnz;
+    const int lane = threadIdx.x & 31;
+    const int stride = gridDim.x * blockDim.x;
+    for (int k0 = (blockIdx.x * blockDim.x + threadIdx.x) - lane; k0 < n; k0 += stride) {     // warp-uniform trip count
+        const int k = k0 + lane;
+        bool better = false;
+        int i = 0;
+        float v = 0.f;
+        if (k < n) { i = y_idx[k]; v = y_val[k]; better = v < dist[i]; }
+        const uint32_t m = __ballot_sync(0xFFFFFFFFu, better);
+        if (!m) continue;
+        int base = 0;
+        if (lane == 0) base = atomicAdd(count, __popc(m));
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if (better) {
+            const int pos = base + __popc(m & ((1u << lane) - 1u));
+            dist[i] = v;
+            x_idx[pos] = i;
+            x_val[pos] = v;
+        }
+    }
+}
+
+template <int DT>
+static int sssp_typed(dbspmspv_handle_s *h, int32_t src, float *dist, int32_t *n_steps, cudaStream_t st) {
+    const Device &d = h->d;
+    const int64_t n = d.n;
+    if (!h->sssp_arena) {
+        // two x lists (the relaxation writes the one the running product does not read), y, two counters
+        const size_t bytes = (size_t)n * (4 * sizeof(int32_t) + 2 * sizeof(float)) + 64;
+        if (cudaMalloc(&h->sssp_arena, bytes) != cudaSuccess) { h->sssp_arena = nullptr; return DBSPMSPV_ERR_ALLOC; }
+        if (cudaHostAlloc(reinterpret_cast<void **>(&h->sssp_host), sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) return DBSPMSPV_ERR_ALLOC;
+    }
+    int32_t *xi[2], *y_idx, *ctr;
+    float *xv[2], *y_val;
+    {
+        uint8_t *p = static_cast<uint8_t *>(h->sssp_arena);
+        xi[0] = reinterpret_cast<int32_t *>(p); p += n * sizeof(int32_t);
+        xi[1] = reinterpret_cast<int32_t *>(p); p += n * sizeof(int32_t);
+        y_idx = reinterpret_cast<int32_t *>(p); p += n * sizeof(int32_t);
+        xv[0] = reinterpret_cast<float *>(p); p += n * sizeof(float);
+        xv[1] = reinterpret_cast<float *>(p); p += n * sizeof(float);
+        y_val = reinterpret_cast<float *>(p); p += n * sizeof(float);
+        ctr = reinterpret_cast<int32_t *>(p);                 // [0] next x count, [1] y_nnz
+    }
+    k_sssp_init<<<4 * h->sm_count, 256, 0, st>>>(dist, n, src, xi[0], xv[0], ctr);
+    ++h->kernel_launches;
+    int32_t nnz_x = 1;
+    int steps = 0, cur = 0;
+    while (nnz_x > 0) {
+        if (++steps > n + 1) return DBSPMSPV_ERR_UNSUPPORTED;          // a cycle of negative weight
+        const int s = run_typed<DT>(h, xi[cur], xv[cur], nnz_x, DBSPMSPV_MIN_PLUS, y_idx, y_val, n, ctr + 1, st);
+        if (s != DBSPMSPV_OK) return s;
+        k_sssp_relax<<<2 * h->sm_count, 256, 0, st>>>(y_idx, y_val, ctr + 1, dist, xi[cur ^ 1], xv[cur ^ 1], ctr);
+        ++h->kernel_launches;
+        DBS_CUDA(cudaMemcpyAsync(h->sssp_host, ctr, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        DBS_CUDA(cudaMemsetAsync(ctr, 0, sizeof(int32_t), st));
+        DBS_CUDA(cudaStreamSynchronize(st));
+        nnz_x = *h->sssp_host;
+        cur ^= 1;
+    }
+    if (n_steps) *n_steps = steps;
+    return DBSPMSPV_OK;
+}
+
 }  // namespace dbs
 
 extern "C" {
@@ -2260,6 +2340,18 @@ int dbspmspv_run_masked(dbspmspv_handle_t h, const int32_t *x_idx, const void *x
                         int64_t y_capacity, int32_t *y_nnz, dbspmspv_stream_t stream) {
     if (!row_mask || (complement != 0 && complement != 1)) return DBSPMSPV_ERR_INVALID_ARG;
     return run_checked(h, x_idx, x_val, nnz_x, semiring, y_idx, y_val, y_capacity, y_nnz, stream, row_mask, complement);
+}
+
+int db_sssp(dbspmspv_handle_t h, int32_t src, float *dist, int32_t *n_steps, dbspmspv_stream_t stream) {
+    if (!h || !dist) return DBSPMSPV_ERR_INVALID_ARG;
+    if (h->d.m != h->d.n) return DBSPMSPV_ERR_UNSUPPORTED;
+    if (h->d.dtype == DBSPMSPV_BF16) return DBSPMSPV_ERR_UNSUPPORTED;    // distances are fp32; x would have to be bf16
+    if (src < 0 || src >= h->d.n) return DBSPMSPV_ERR_INVALID_ARG;
+    if (!dbs::on_handle_device(h)) return DBSPMSPV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    return h->d.dtype == DBSPMSPV_F32 ? dbs::sssp_typed<DBSPMSPV_F32>(h, src, dist, n_steps, st)
+                                      : dbs::sssp_typed<DBSPMSPV_PATTERN>(h, src, dist, n_steps, st);
 }
 
 int dbspmspv_test_bounded_wait(dbspmspv_handle_t h, int32_t max_tries, dbspmspv_stream_t stream) {

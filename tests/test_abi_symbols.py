@@ -13,7 +13,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "dbspmspv.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"\b(dbspmspv_[a-z_]+|db_bfs)\s*\(", text)
+    names = re.findall(r"\b(dbspmspv_[a-z_]+|db_bfs|db_sssp)\s*\(", text)
     return sorted(set(names))
 
 

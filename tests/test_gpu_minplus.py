@@ -113,3 +113,76 @@ def test_minplus_argument_errors():
     with pytest.raises(B.DbSpmspvError):
         B.dbspmspv_run(h.h, xi, xi.float(), 1, 3, h.y_idx, h.y_val, 64, h.y_nnz)          # unknown semiring
     h.close()
+
+
+# ---- db_sssp ------------------------------------------------------------------------------
+
+def _sssp(h, src):
+    dist = torch.empty(h.csr.n, dtype=torch.float32, device="cuda")
+    steps = B.db_sssp(h.h, int(src), dist)
+    torch.cuda.synchronize()
+    return dist.cpu().numpy(), steps
+
+
+@pytest.mark.parametrize("make", [lambda: wl.rmat(12, 16, seed=2, symmetrise=True), lambda: wl.rmat(14, 8, seed=3),
+                                  lambda: wl.stencil27(12, seed=1), lambda: wl.random_sparse(3000, 3000, 9000, 8)],
+                         ids=["rmat12_sym", "rmat14_directed", "stencil12", "uniform3000"])
+def test_sssp_exact_on_dyadic_weights(make):
+    """Weights that are multiples of 1/8 below 8: every path sum is exact in fp32 and in the
+    oracle's fp64, so the distances must be identical, unreachable vertices +inf."""
+    csr = make()
+    csr.val = (1 + (wl.rand_u64(11, 3, np.arange(csr.nnz)) % 63)).astype(np.float32) / 8.0
+    h = Handle(csr, B.F32)
+    A = ref_matrix(csr)
+    deg = np.bincount(csr.col_idx, minlength=csr.n)
+    srcs = [int(np.argmax(deg)), int(np.flatnonzero(deg > 0)[0]), int(np.flatnonzero(deg > 0)[-1])]
+    for src in srcs:
+        got, steps = _sssp(h, src)
+        want = oracle.ref_sssp(A, src)
+        assert np.array_equal(got.astype(np.float64), want)
+        assert steps >= 1
+    h.close()
+
+
+def test_sssp_general_weights_within_rounding():
+    """Arbitrary fp32 weights: a path of k edges accumulates k roundings of 2^-24 relative."""
+    csr = wl.rmat(13, 16, seed=5, symmetrise=True)
+    csr.val = (0.05 + wl.rand_f32(7, 1, np.arange(csr.nnz))).astype(np.float32)
+    h = Handle(csr, B.F32)
+    A = ref_matrix(csr)
+    for src in wl.bfs_sources(csr, 3):
+        got, steps = _sssp(h, src)
+        want = oracle.ref_sssp(A, int(src))
+        assert np.array_equal(np.isinf(got), np.isinf(want))
+        fin = np.isfinite(want)
+        assert np.all(np.abs(got[fin] - want[fin]) <= 64 * 2.0 ** -24 * want[fin] + 1e-30)
+    h.close()
+
+
+def test_sssp_pattern_handle_gives_bfs_levels_and_negative_edges():
+    g = wl.rmat(12, 8, seed=9, values=False, symmetrise=True)
+    h = Handle(g, B.PATTERN)
+    src = int(wl.bfs_sources(g, 1)[0])
+    lv = oracle.ref_bfs(oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx, None), src).astype(np.float64)
+    lv[lv < 0] = np.inf
+    got, _ = _sssp(h, src)
+    assert np.array_equal(got.astype(np.float64), lv)
+    h.close()
+    # negative edges without a negative cycle; then one with: 0 -> 1 -> 2 -> 0 of total weight -1
+    a = np.zeros((5, 5), dtype=np.float32)
+    a[1, 0], a[2, 1], a[3, 2], a[3, 0], a[4, 3] = 4.0, -2.0, 1.0, 5.0, -1.0
+    csr = wl.csr_from_dense(a)
+    h = Handle(csr, B.F32)
+    got, steps = _sssp(h, 0)
+    assert got.tolist() == [0.0, 4.0, 2.0, 3.0, 2.0]
+    assert np.array_equal(got.astype(np.float64), oracle.ref_sssp(ref_matrix(csr), 0))
+    got, steps = _sssp(h, 4)                                  # no out-edges: one product, nothing reached
+    assert got.tolist() == [np.inf] * 4 + [0.0] and steps == 1
+    h.close()
+    a = np.zeros((3, 3), dtype=np.float32)
+    a[1, 0], a[2, 1], a[0, 2] = 1.0, 1.0, -3.0
+    h = Handle(wl.csr_from_dense(a), B.F32)
+    with pytest.raises(B.DbSpmspvError):
+        _sssp(h, 0)
+    torch.cuda.synchronize()
+    h.close()
