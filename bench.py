@@ -634,6 +634,68 @@ def banded_plus_random(n: int, band: int, extra: int, seed: int) -> wl.CSR:
     return wl.CSR(n, n, row_ptr, c, val)
 
 
+def minplus_rows(B, torch, dev, flush, peak):
+    """The (min, +) semiring: one product on the sweep's matrix at three x densities next to the
+    (+, *) push on the same x, and db_sssp on the symmetrised weighted R-MAT scale 20 graph (four
+    sources; one checked against the CPU Bellman-Ford oracle, which is timed on that source)."""
+    import oracle
+    up = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    out = []
+    a = wl.rmat(20, 16, seed=1)
+    h = B.dbspmspv_create_csr(a.m, a.n, a.nnz, up(a.row_ptr), up(a.col_idx), up(a.val), B.F32)
+    model = ByteModel(a, 4)
+    y_idx = torch.empty(a.m, dtype=torch.int32, device=dev)
+    y_val = torch.empty(a.m, dtype=torch.float32, device=dev)
+    y_nnz = torch.zeros(1, dtype=torch.int32, device=dev)
+    o = B.default_run_opts()
+    o.force_path = B.PATH_PUSH
+    B.dbspmspv_set_run_opts(h, o)
+    for k, f in ((2, 1e-3), (3, 1e-2), (4, 1e-1)):
+        x = wl.rmat_x(a.n, f, k)
+        xi, xv = up(x.idx), up(x.val)
+        rec = {"workload": "rmat20_ef16_fp32 (min,+) product", "x": f"x fraction {f:g}", "path": "push"}
+        for name, sr in (("minplus", B.MIN_PLUS), ("plus_times_forced_push", B.PLUS_TIMES)):
+            call = lambda: B.dbspmspv_run(h, xi, xv, int(x.idx.size), sr, y_idx, y_val, a.m, y_nnz)
+            st = stats_of(timed_calls(torch, call, flush, 12))
+            rec[name + "_us"] = st["us"]
+            if sr == B.MIN_PLUS:
+                kk = int(y_nnz.item())
+                mv = model.moved(x.idx, B.PATH_PUSH, kk, None)
+                rec.update({"y_nnz": kk, "B_moved": int(mv["total"]), "moved": fractions(mv["total"], st["us"], peak)})
+        out.append(rec)
+    B.dbspmspv_destroy(h)
+    del a
+    g = wl.rmat(20, 16, seed=3, symmetrise=True)
+    g.val = (0.05 + wl.rand_f32(7, 1, np.arange(g.nnz))).astype(np.float32)
+    h = B.dbspmspv_create_csr(g.m, g.n, g.nnz, up(g.row_ptr), up(g.col_idx), up(g.val), B.F32)
+    dist = torch.empty(g.n, dtype=torch.float32, device=dev)
+    srcs = wl.bfs_sources(g, 4)
+    ms, steps, edges = [], [], []
+    deg = np.diff(g.row_ptr)
+    for s_ in srcs:
+        B.db_sssp(h, int(s_), dist)                         # warm-up (the first call allocates)
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); n_steps = B.db_sssp(h, int(s_), dist); e1.record()
+        torch.cuda.synchronize()
+        dv = dist.cpu().numpy()
+        ms.append(e0.elapsed_time(e1)); steps.append(n_steps); edges.append(int(deg[np.isfinite(dv)].sum()))
+    t0 = time.perf_counter()
+    want = oracle.ref_sssp(oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx, g.val), int(srcs[-1]))
+    cpu_s = time.perf_counter() - t0
+    fin = np.isfinite(want)
+    ok = bool(np.array_equal(np.isfinite(dv), fin) and np.all(np.abs(dv[fin] - want[fin]) <= 64 * 2.0 ** -24 * want[fin] + 1e-30))
+    out.append({"workload": "rmat20_ef16_symmetrised_weighted_fp32 db_sssp", "sources": len(srcs),
+                "ms_per_search_median": round(float(np.median(ms)), 3), "ms_min": round(min(ms), 3), "ms_max": round(max(ms), 3),
+                "products_per_search": steps, "edges_in_component": edges[-1],
+                "GTEPS_edges_of_component_over_time": round(float(np.mean([e / (t * 1e-3) / 1e9 for e, t in zip(edges, ms)])), 3),
+                "cpu_bellman_ford_s": round(cpu_s, 3), "matches_oracle": ok})
+    if not ok:
+        raise SystemExit("db_sssp disagrees with the oracle")
+    B.dbspmspv_destroy(h)
+    return out
+
+
 def other_configs(B, torch, dev, flush, peak, floors):
     """The remaining workload shapes, one record each (whole call, cold L2 and L2-warm): the
     uniform matrix with a 1 % x, the 27-point stencil with clustered x at 0.1 % and 5 %, and
@@ -688,6 +750,7 @@ def other_configs(B, torch, dev, flush, peak, floors):
     out += decode_layers(B, torch, dev, flush, peak)
     out.append(decode_chain(B, torch, dev, flush))
     out += decode_batch(B, torch, dev, flush)
+    out += minplus_rows(B, torch, dev, flush, peak)
     return out
 
 

@@ -271,8 +271,11 @@ int db_bfs(dbspmspv_handle_t h, int32_t src, int32_t *levels, dbspmspv_stream_t 
  *   dist     out: n fp32 on the device; source 0, unreachable +infinity.  Every path sum is
  *            accumulated in fp32 in path order.
  *   n_steps  out (host, may be NULL): products made, the last one with an empty result
+ * Direction per step: run_opts.force_path if set; else a step whose x holds more than a tenth
+ * of the stored elements as out-edges is pulled (hypersparse F32 handles; the others always
+ * push), the rest pushed.
  * Unlike the other calls this one is a host loop: it waits on `stream` once per step to read
- * the size of the next x (4 bytes), and the first call on a handle allocates 24 n bytes of
+ * the size of the next x and its out-edge count (16 bytes), and the first call on a handle allocates 24 n bytes of
  * device memory and one page-locked word (freed by dbspmspv_destroy).  More than n + 1 steps
  * (a negative cycle) end the search with ERR_UNSUPPORTED.
  */

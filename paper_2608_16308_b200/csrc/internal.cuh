@@ -271,7 +271,7 @@ struct dbspmspv_handle_s {
     // launch configurations, worked out on first use (function attributes and occupancy are per
     // device, and a handle lives on one device; calls on a handle are stream ordered, so plain fields)
     int grid_compute, grid_compute_dense, grid_decode_pull;
-    bool lean_configured, lean_configured_dense;
+    bool lean_configured, lean_configured_dense, lean_configured_min;
     bool fused_configured[3];
     bool batch_configured[2];
     bool batch_mma_configured[3];

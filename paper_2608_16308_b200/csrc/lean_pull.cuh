@@ -23,10 +23,13 @@
 //     running count of ROW_FLAGs; structural hits are tracked as bit masks beside the sums.
 //   * The few entries with a payload are skipped by the stream and taken afterwards, one block
 //     per warp at a time, from the list of their positions.
+//   * The same kernel serves the (min, +) semiring (Out::MINPLUS): products become sums, sums
+//     minima with identity +infinity, and the writeback keeps the smaller value (minplus.cuh).
 #pragma once
 
 #include "internal.cuh"
 #include "microkernels.cuh"
+#include "minplus.cuh"
 
 namespace dbs {
 
@@ -83,9 +86,18 @@ __device__ __forceinline__ LeanRegs lean_fetch(const Device &d, int c, int lane)
 
 template <int DT, typename Out>
 __device__ __forceinline__ void lean_add(Out out, int row, float v) {
+    if (Out::MINPLUS) {          // keep the smaller sum (an atomic whose reply nobody waits for)
+        atomicMax(reinterpret_cast<uint32_t *>(out.acc) + row, minplus_key(v));
+        out.hit8[row] = 1;
+        return;
+    }
     if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + row, v);
     if (Out::MASKS) out.hit8[row] = 1;
 }
+// The semiring of the segmented reduction: (+, *) or, for Out::MINPLUS, (min, +).
+template <typename Out> __device__ __forceinline__ float lean_identity() { return Out::MINPLUS ? __int_as_float(0x7F800000) : 0.f; }
+template <typename Out> __device__ __forceinline__ float lean_mul(float a, float x) { return Out::MINPLUS ? a + x : a * x; }
+template <typename Out> __device__ __forceinline__ float lean_sum(float s, float p) { return Out::MINPLUS ? fminf(s, p) : s + p; }
 
 // One chunk = one warp pass, eight consecutive entries per lane, arranged so that the chunk costs
 // one exposed memory latency: first what needs the entries only (the row-start bits and, from a
@@ -153,7 +165,8 @@ __device__ __forceinline__ void lean_chunk(const Device &d, Out out, const LeanR
     // ---- sums.  Thread-serial part: `lead` = sum of the lane's entries before its first row
     // start (they belong to the row that was open when the lane began), `seg` = sum from its last
     // row start on; rows that lie wholly inside the lane are added to global memory by the lane.
-    float lead = 0.f, seg = 0.f;
+    const float ID = lean_identity<Out>();
+    float lead = ID, seg = ID;
     uint32_t lead_hit = 0u, seg_hit = 0u;
     if (!multi) {
         // at most one row start per lane (the usual case): entries below it, entries from it on
@@ -164,8 +177,8 @@ __device__ __forceinline__ void lean_chunk(const Device &d, Out out, const LeanR
             if (__float_as_uint(xin[k]) != X_ABSENT) {
                 pb |= 1u << k;
                 if (VAL) {
-                    const float p = Val<DT>::inline_value(wv[k]) * xin[k];
-                    if (k < f) lead += p; else seg += p;
+                    const float p = lean_mul<Out>(Val<DT>::inline_value(wv[k]), xin[k]);
+                    if (k < f) lead = lean_sum<Out>(lead, p); else seg = lean_sum<Out>(seg, p);
                 }
             }
         }
@@ -180,14 +193,14 @@ __device__ __forceinline__ void lean_chunk(const Device &d, Out out, const LeanR
                 if (nh == 0) { lead = seg; lead_hit = seg_hit; }
                 else if (seg_hit) lean_add<DT>(out, row_of(excl + nh), seg);   // a whole row inside the lane
                 ++nh;
-                seg = 0.f; seg_hit = 0u;
+                seg = ID; seg_hit = 0u;
             }
             if (__float_as_uint(xin[k]) != X_ABSENT) {
-                if (VAL) seg += Val<DT>::inline_value(wv[k]) * xin[k];
+                if (VAL) seg = lean_sum<Out>(seg, lean_mul<Out>(Val<DT>::inline_value(wv[k]), xin[k]));
                 seg_hit = 1u;
             }
         }
-        if (nh == 0) { lead = seg; lead_hit = seg_hit; seg = 0.f; seg_hit = 0u; }
+        if (nh == 0) { lead = seg; lead_hit = seg_hit; seg = ID; seg_hit = 0u; }
     }
     // Warp part.  A lane with a row start closes the row that was open before it.  S = inclusive
     // sum of `lead` over the lanes since the last lane with a row start (exclusive): at a lane with
@@ -199,7 +212,7 @@ __device__ __forceinline__ void lean_chunk(const Device &d, Out out, const LeanR
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float t = __shfl_up_sync(FULL, S, o);
-            if (reach >= o) S += t;
+            if (reach >= o) S = lean_sum<Out>(S, t);
         }
     }
     // (a) the row that runs into the chunk: closed by the first lane with a row start (lane 31 if none)
@@ -209,11 +222,11 @@ __device__ __forceinline__ void lean_chunk(const Device &d, Out out, const LeanR
     // lanes up to and including the next lane with a row start (or lane 31)
     const uint32_t above = hm & ~lt & ~(1u << lane);
     const int nx = above ? __ffs(above) - 1 : 31;
-    float tail = 0.f;
-    if (VAL) { tail = __shfl_sync(FULL, S, nx); if (lane == 31) tail = 0.f; }
+    float tail = ID;
+    if (VAL) { tail = __shfl_sync(FULL, S, nx); if (lane == 31) tail = ID; }
     if (cnt) {
         const uint32_t tail_hit = ((lh >> 1) >> lane) & ((1u << (nx - lane)) - 1u);
-        if (seg_hit | tail_hit) lean_add<DT>(out, row_of(excl + cnt), seg + tail);
+        if (seg_hit | tail_hit) lean_add<DT>(out, row_of(excl + cnt), lean_sum<Out>(seg, tail));
     }
 }
 
@@ -276,6 +289,12 @@ k_pull_lean(Device d, Out out, float th3, int force_path, int popc_threshold, in
         const uint8_t *blk = d.payload + (size_t)d.csr.w[pos] * 4;
         const int nnz = (int)d.csr.aux[pos] + 1;
         const int rb = d.entry_row[pos];
+        if (Out::MINPLUS) {
+            block_elements_warp<DT>(type, d.csr.w[pos], d.csr.aux[pos], xm, d.payload, lane, [&](int r, int c, float a) {
+                lean_add<DT>(out, rb * 16 + r, a + d.ws.x_dense[(size_t)cb * 16 + c]);
+            });
+            continue;
+        }
         uint32_t hits;
         float sum = 0.f;
         if (DT == DBSPMSPV_PATTERN) {

@@ -13,10 +13,12 @@
 // value whose key would be 0 is the NaN 0x7FFFFFFF; NaN has no place in a (min, +) product and
 // its key is stored as 1.  The compaction turns the keys back into values.
 //
-// Traversal: always the push over the block-CSC view (a listed x_j meets exactly the stored
-// elements of column j; there is no row-wise form here).  A warp takes one task of the push
-// worklist, 32 view entries, lane = entry; a lane walks all stored elements of its block that
-// sit in listed columns, whatever the block's class.
+// Traversal.  Push (this file): a warp takes one task of the push worklist, 32 entries of the
+// block-CSC view, lane = entry; a lane walks all stored elements of its block that sit in
+// listed columns, whatever the block's class.  Pull: on hypersparse valued handles the streaming
+// pull kernel runs with the semiring swapped (lean_pull.cuh); the selector is the same
+// vector-block ratio as for (+, *).  Pattern handles and handles whose elements sit mostly in
+// mask-based blocks always push.
 #pragma once
 
 #include "internal.cuh"
@@ -81,12 +83,53 @@ __device__ __forceinline__ void block_elements(int type, uint32_t w, uint32_t au
     }
 }
 
+// The same for one block with a payload taken by a whole warp: a lane owns half a row (row-major
+// classes) or half a column (column-major classes, Dense), COO entries are dealt out in turn.
+template <int DT, typename F>
+__device__ __forceinline__ void block_elements_warp(int type, uint32_t w, uint32_t aux, uint32_t xm, const uint8_t *payload, int lane, F f) {
+    const uint8_t *blk = payload + (size_t)w * 4;
+    if (type == DBSPMSPV_BLK_COO) {
+        const int nnz = (int)aux + 1;
+        const uint8_t *vals = blk + ((nnz + 3) & ~3);
+        for (int k = lane; k < nnz; k += 32) {
+            const uint32_t rc = blk[k];
+            if ((xm >> (rc & 15)) & 1u) f((int)(rc >> 4), (int)(rc & 15), Val<DT>::load(vals, k));
+        }
+        return;
+    }
+    constexpr bool HAS_STARTS = Val<DT>::SIZE != 0;
+    const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
+    const int major = lane >> 1;
+    const uint32_t half = 0xFFu << (8 * (lane & 1));
+    const uint32_t full = masks[major];
+    if (is_row_major(type)) {
+        const uint8_t *vals = blk + HDR_BYTES;
+        const int base = HAS_STARTS ? blk[32 + major] : 0;
+        for (uint32_t act = full & xm & half; act; act &= act - 1) {
+            const int c = __ffs(act) - 1;
+            f(major, c, Val<DT>::load(vals, base + __popc(full & ((1u << c) - 1u))));
+        }
+        return;
+    }
+    if (!((xm >> major) & 1u)) return;
+    const bool dense = type == DBSPMSPV_BLK_DENSE;
+    const uint8_t *vals = blk + (dense ? 32 : HDR_BYTES);
+    const int base = dense ? major * 16 : (HAS_STARTS ? blk[32 + major] : 0);
+    for (uint32_t cm = full & half; cm; cm &= cm - 1) {
+        const int r = __ffs(cm) - 1;
+        f(r, major, Val<DT>::load(vals, dense ? base + r : base + __popc(full & ((1u << r) - 1u))));
+    }
+}
+
 constexpr int MINPLUS_CTA = 256;
 
+__device__ __forceinline__ int select_path(const Device &d, float th3, int force_path);
+
 template <int DT>
-__global__ void __launch_bounds__(MINPLUS_CTA, 4) k_minplus_push(Device d) {
+__global__ void __launch_bounds__(MINPLUS_CTA, 4) k_minplus_push(Device d, float th3, int force_path) {
     pdl_wait();
     pdl_launch_dependents();
+    if (select_path(d, th3, force_path) != DBSPMSPV_PATH_PUSH) return;
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;

@@ -177,11 +177,20 @@ struct OutSparse {
     float *acc;
     uint8_t *hit8;     // one byte per row: 1 = structurally hit (plain idempotent stores, no atomics)
     static constexpr bool MASKS = true;
+    static constexpr bool MINPLUS = false;
 };
 struct OutDense {
     float *acc;
     uint8_t *hit8;
     static constexpr bool MASKS = false;
+    static constexpr bool MINPLUS = false;
+};
+// (min, +) semiring: the accumulator holds keys of the smallest sum so far (minplus.cuh)
+struct OutSparseMin {
+    float *acc;
+    uint8_t *hit8;
+    static constexpr bool MASKS = true;
+    static constexpr bool MINPLUS = true;
 };
 
 // One lane owns one hypersparse block (INLINE or COO).  `emit(r, v)` receives the products,
@@ -1567,7 +1576,6 @@ k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, flo
 
 }  // namespace dbs
 #include "decode_batch.cuh"
-#include "minplus.cuh"
 namespace dbs {
 
 // ------------------------------------------------------------------------------------------
@@ -1865,7 +1873,7 @@ static int launch_compute(dbspmspv_handle_s *h, Out out, float th3, bool pdl, cu
 // The streaming pull of hypersparse handles (lean_pull.cuh), launched behind k_compute.
 template <int DT, typename Out>
 static int launch_lean(dbspmspv_handle_s *h, Out out, float th3, cudaStream_t st) {
-    bool &configured = Out::MASKS ? h->lean_configured : h->lean_configured_dense;
+    bool &configured = Out::MINPLUS ? h->lean_configured_min : Out::MASKS ? h->lean_configured : h->lean_configured_dense;
     // filter size: the power of two that holds one bit per column, capped
     const int n_words = (h->d.nb + 1) / 2;
     int filter_words = 32;
@@ -1966,8 +1974,10 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     const Device &d = h->d;
     // x lists a quarter of the columns or more: a pull is likely (on hypersparse matrices), so
     // the worklist is built afterwards from the masks, and only if the selector does choose the push
-    const bool minplus = semiring == DBSPMSPV_MIN_PLUS;     // always the push: the worklist is built with the vector blocking
-    const bool late_emit = !minplus && !h->heavy_stage && h->ropts.force_path != DBSPMSPV_PATH_PUSH && (int64_t)nnz_x * 4 >= d.n;
+    const bool minplus = semiring == DBSPMSPV_MIN_PLUS;
+    // (min, +) pulls only with the streaming kernel of hypersparse valued handles
+    const bool minplus_pull = minplus && !h->heavy_stage && DT != DBSPMSPV_PATTERN;
+    const bool late_emit = (!minplus || minplus_pull) && !h->heavy_stage && h->ropts.force_path != DBSPMSPV_PATH_PUSH && (int64_t)nnz_x * 4 >= d.n;
     const void *xv = semiring == DBSPMSPV_OR_AND ? nullptr : x_val;
     if (nnz_x > 0) {
         const int g = (nnz_x + XB_TPB - 1) / XB_TPB;
@@ -1990,8 +2000,15 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
     h->d.hub_on = !minplus && d.n_hub_blocks > 0 && hub_min > 0 && nnz_x >= hub_min && h->ropts.force_path != DBSPMSPV_PATH_PULL &&
                   (!late_emit || h->heavy_stage);
     if (minplus && nnz_x > 0 && d.n_entries > 0) {
-        DBS_CUDA(launch_pdl(k_minplus_push<DT>, 4 * h->sm_count, MINPLUS_CTA, 0, st, d));
-        ++h->kernel_launches;
+        const int fp = minplus_pull ? h->ropts.force_path : DBSPMSPV_PATH_PUSH;
+        if (fp != DBSPMSPV_PATH_PULL) {
+            DBS_CUDA(launch_pdl(k_minplus_push<DT>, 4 * h->sm_count, MINPLUS_CTA, 0, st, d, h->ropts.th3, fp));
+            ++h->kernel_launches;
+        }
+        if (minplus_pull && pull_possible(h, nnz_x, h->ropts.th3)) {
+            const int s = launch_lean<DT, OutSparseMin>(h, OutSparseMin{d.ws.y_acc, d.ws.y_hit8}, h->ropts.th3, st);
+            if (s != DBSPMSPV_OK) return s;
+        }
     } else if (nnz_x > 0 && d.n_entries > 0) {
         int s = DBSPMSPV_OK;
         if (h->heavy_stage) {
@@ -2214,10 +2231,18 @@ static int decode_batch_typed(dbspmspv_handle_s *h, const void *x, int64_t ldx, 
 __global__ void k_sssp_init(float *dist, int64_t n, int32_t src, int32_t *x_idx, float *x_val, int32_t *count) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; v < n; v += stride) dist[v] = v == src ? 0.0f : __int_as_float(0x7F800000);
-    if (blockIdx.x == 0 && threadIdx.x == 0) { x_idx[0] = src; x_val[0] = 0.0f; *count = 0; }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { x_idx[0] = src; x_val[0] = 0.0f; count[0] = 0; count[2] = 0; count[3] = 0; }
 }
 
-__global__ void k_sssp_relax(const int32_t *__restrict__ y_idx, const float *__restrict__ y_val, const int32_t *__restrict__ y_nnz,
+// A step whose x reaches more than this share of the stored elements is pulled (where the handle
+// has a (min, +) pull): such an x is a handful of hubs or half the graph, its push is a queue of
+// atomics on the hub rows, and the streaming pull reads the matrix once whatever x holds.
+#ifndef DBS_SSSP_PULL_EDGE_FRAC
+#define DBS_SSSP_PULL_EDGE_FRAC 0.1f
+#endif
+
+// count[0]: entries of the next x; count[2..3]: the out-edges they hold (64 bits; INLINE runs of the block-CSC view)
+__global__ void k_sssp_relax(Device d, const int32_t *__restrict__ y_idx, const float *__restrict__ y_val, const int32_t *__restrict__ y_nnz,
                              float *__restrict__ dist, int32_t *__restrict__ x_idx, float *__restrict__ x_val, int32_t *count) {
     const int n = *y_nnz;
     const int lane = threadIdx.x & 31;
@@ -2233,12 +2258,17 @@ __global__ void k_sssp_relax(const int32_t *__restrict__ y_idx, const float *__r
         int base = 0;
         if (lane == 0) base = atomicAdd(count, __popc(m));
         base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        int deg = 0;
         if (better) {
             const int pos = base + __popc(m & ((1u << lane) - 1u));
             dist[i] = v;
             x_idx[pos] = i;
             x_val[pos] = v;
+            int first;
+            column_run(d, i, first, deg);
         }
+        deg = __reduce_add_sync(0xFFFFFFFFu, deg);
+        if (lane == 0 && deg) atomicAdd(reinterpret_cast<unsigned long long *>(count + 2), (unsigned long long)deg);
     }
 }
 
@@ -2250,7 +2280,7 @@ static int sssp_typed(dbspmspv_handle_s *h, int32_t src, float *dist, int32_t *n
         // two x lists (the relaxation writes the one the running product does not read), y, two counters
         const size_t bytes = (size_t)n * (4 * sizeof(int32_t) + 2 * sizeof(float)) + 64;
         if (cudaMalloc(&h->sssp_arena, bytes) != cudaSuccess) { h->sssp_arena = nullptr; return DBSPMSPV_ERR_ALLOC; }
-        if (cudaHostAlloc(reinterpret_cast<void **>(&h->sssp_host), sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) return DBSPMSPV_ERR_ALLOC;
+        if (cudaHostAlloc(reinterpret_cast<void **>(&h->sssp_host), 4 * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) return DBSPMSPV_ERR_ALLOC;
     }
     int32_t *xi[2], *y_idx, *ctr;
     float *xv[2], *y_val;
@@ -2262,24 +2292,34 @@ static int sssp_typed(dbspmspv_handle_s *h, int32_t src, float *dist, int32_t *n
         xv[0] = reinterpret_cast<float *>(p); p += n * sizeof(float);
         xv[1] = reinterpret_cast<float *>(p); p += n * sizeof(float);
         y_val = reinterpret_cast<float *>(p); p += n * sizeof(float);
-        ctr = reinterpret_cast<int32_t *>(p);                 // [0] next x count, [1] y_nnz
+        ctr = reinterpret_cast<int32_t *>(p);                 // [0] next x count, [1] y_nnz, [2..3] out-edges of the next x
     }
     k_sssp_init<<<4 * h->sm_count, 256, 0, st>>>(dist, n, src, xi[0], xv[0], ctr);
     ++h->kernel_launches;
     int32_t nnz_x = 1;
-    int steps = 0, cur = 0;
+    int64_t edges = 0;
+    int steps = 0, cur = 0, status = DBSPMSPV_OK;
+    const int user_path = h->ropts.force_path;
     while (nnz_x > 0) {
-        if (++steps > n + 1) return DBSPMSPV_ERR_UNSUPPORTED;          // a cycle of negative weight
-        const int s = run_typed<DT>(h, xi[cur], xv[cur], nnz_x, DBSPMSPV_MIN_PLUS, y_idx, y_val, n, ctr + 1, st);
-        if (s != DBSPMSPV_OK) return s;
-        k_sssp_relax<<<2 * h->sm_count, 256, 0, st>>>(y_idx, y_val, ctr + 1, dist, xi[cur ^ 1], xv[cur ^ 1], ctr);
+        if (++steps > n + 1) { status = DBSPMSPV_ERR_UNSUPPORTED; break; }          // a cycle of negative weight
+        // direction of this step: the caller's, else by the share of the stored elements x reaches
+        if (user_path == DBSPMSPV_PATH_AUTO)
+            h->ropts.force_path = (double)edges > (double)DBS_SSSP_PULL_EDGE_FRAC * (double)d.n_entries ? DBSPMSPV_PATH_PULL : DBSPMSPV_PATH_PUSH;
+        status = run_typed<DT>(h, xi[cur], xv[cur], nnz_x, DBSPMSPV_MIN_PLUS, y_idx, y_val, n, ctr + 1, st);
+        if (status != DBSPMSPV_OK) break;
+        k_sssp_relax<<<2 * h->sm_count, 256, 0, st>>>(d, y_idx, y_val, ctr + 1, dist, xi[cur ^ 1], xv[cur ^ 1], ctr);
         ++h->kernel_launches;
-        DBS_CUDA(cudaMemcpyAsync(h->sssp_host, ctr, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-        DBS_CUDA(cudaMemsetAsync(ctr, 0, sizeof(int32_t), st));
-        DBS_CUDA(cudaStreamSynchronize(st));
-        nnz_x = *h->sssp_host;
+        if (cudaMemcpyAsync(h->sssp_host, ctr, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaMemsetAsync(ctr, 0, 4 * sizeof(int32_t), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+            status = DBSPMSPV_ERR_CUDA;
+            break;
+        }
+        nnz_x = h->sssp_host[0];
+        edges = (int64_t)(uint32_t)h->sssp_host[2] | ((int64_t)h->sssp_host[3] << 32);
         cur ^= 1;
     }
+    h->ropts.force_path = user_path;
+    if (status != DBSPMSPV_OK) return status;
     if (n_steps) *n_steps = steps;
     return DBSPMSPV_OK;
 }

@@ -39,9 +39,16 @@ def test_minplus_parity(name, make, dtype, inline_max):
         if dtype == B.BF16:
             x.val = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x.val))
         want = oracle.ref_minplus(A, x.idx, x.val)
-        check_exact(h.run(x, semiring=B.MIN_PLUS), want)
-        st = h.get_stats()
-        assert st.last_path == B.PATH_PUSH and st.last_y_nnz == want[0].size
+        for path in (B.PATH_AUTO, B.PATH_PUSH, B.PATH_PULL):
+            h.set_opts(force_path=path)
+            check_exact(h.run(x, semiring=B.MIN_PLUS), want)
+            st = h.get_stats()
+            assert st.last_y_nnz == want[0].size
+            # the pull is the streaming kernel of hypersparse valued handles; everything else pushes
+            if name == "rmat12" and dtype != B.PATTERN and path == B.PATH_PULL:
+                assert st.last_path == B.PATH_PULL
+            if path == B.PATH_PUSH or dtype == B.PATTERN:
+                assert st.last_path == B.PATH_PUSH
     h.close()
 
 
