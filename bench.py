@@ -116,13 +116,21 @@ class ByteModel:
         return {"view_entries": int(entries), "view_bytes": int(VIEW_ENTRY_BYTES * entries), "payload_blocks": int(blocks),
                 "payload_bytes": int(payload), "pointer_bytes": int(pointers), "active_vector_blocks": int(xb.size)}
 
-    def moved(self, x_idx: np.ndarray, path: int, y_nnz: int, fmt: dict | None = None) -> dict:
+    def moved(self, x_idx: np.ndarray, path: int, y_nnz: int, fmt: dict | None = None, one_kernel: bool = False) -> dict:
         """Bytes the implementation moves on `path`, each distinct byte once: the format part
         (above), x (the list, the dense copy written and gathered, the masks, the clean-up),
         y (accumulator read-modify-write, hit flags, the sorted output) and the two O(m) scans
-        of the compaction passes (hit flags in, packed masks out and in)."""
+        of the compaction passes (hit flags in, packed masks out and in).  one_kernel: the
+        single-kernel form of a short call -- x is read once as a list, the row bitmap lives in
+        shared memory (no scans), y is the accumulator read-modify-write, the row list written
+        and read back, the gather-and-clear and the output."""
         f = fmt if fmt is not None else self.format_bytes(x_idx, path)
         m, nx = self.csr.m, x_idx.size
+        if one_kernel:
+            fmt_total = f["view_bytes"] + f["payload_bytes"] + f["pointer_bytes"]
+            xbytes, ybytes = 8.0 * nx, 8.0 * y_nnz + 8.0 * y_nnz + 8.0 * y_nnz + 8.0 * y_nnz
+            return {"format": fmt_total, "x": xbytes, "y": ybytes, "scans": 0.0, "total": fmt_total + xbytes + ybytes,
+                    "traversal_kernel": fmt_total + xbytes + ybytes}
         xbytes = 8.0 * nx + 4.0 * nx + 4.0 * nx + 2.0 * f["active_vector_blocks"] + 4.0 * nx + 6.0 * nx
         if path == PULL:
             xbytes += self.csr.n / 8.0                       # the presence filter, read once per SM from L2
@@ -252,7 +260,7 @@ def reference_arm(args) -> None:
             t_step += best
             # same numerator as the GPU arm: the bytes the library moves on its default path
             path = PUSH if np.float32(np.unique(x.idx >> 4).size) / np.float32(model.nb) < np.float32(0.9) else PULL
-            bytes_step += model.moved(x.idx, path, yi.size)["total"]
+            bytes_step += model.moved(x.idx, path, yi.size, None, path == PUSH and x.idx.size <= 256)["total"]    # (short calls: the one-kernel form)
         if it >= args.warmup:
             per_step.append(t_step)
     ms = 1e3 * float(np.mean(per_step))
@@ -402,6 +410,12 @@ def main() -> None:
             flush.fill_(1)
             one_call(k)
     torch.cuda.synchronize()
+    # which points run in the one-kernel form of a short call (one launch)
+    one_kernel = []
+    for k in range(npts):
+        l0 = B.dbspmspv_get_stats(h).kernel_launches
+        one_call(k)
+        one_kernel.append(B.dbspmspv_get_stats(h).kernel_launches - l0 == 1)
     # separate pass with the library's kernel timing on (two extra event records per call):
     # duration of the traversal kernel alone, and the per-point facts for the byte model
     opts.timing = 1
@@ -481,7 +495,7 @@ def main() -> None:
         counted = B.dbspmspv_count_call_bytes(h, xd[k][0], int(x.idx.size), path)
         fmt_model = model.format_bytes(x.idx, path)
         fmt_counted = {f: int(getattr(counted, f)) for f in fmt_model}
-        mv = model.moved(x.idx, path, yk, fmt_model)
+        mv = model.moved(x.idx, path, yk, fmt_model, one_kernel[k])
         moved_by_point.append(mv)
         bt, bm = model.touch(x.idx, yk, yrb), model.floor(x.idx, yk)
         st = stats_of(call_ms[:, k] * 1e3)
@@ -492,7 +506,7 @@ def main() -> None:
         rec = {"x_fraction": wl.RMAT_SWEEP[k], "x_nnz": int(x.idx.size), "path": "push" if path == B.PATH_PUSH else "pull"}
         rec.update(st)
         rec.update({"us_l2_warm": round(warm_us[k], 2), "traversal_kernel_us": round(kus, 2), "y_nnz": yk, "n_nzblk": nzblk,
-                    "n_tasks": ntasks, "B_moved": int(mv["total"]),
+                    "n_tasks": ntasks, "one_kernel_form": bool(one_kernel[k]), "B_moved": int(mv["total"]),
                     "B_moved_parts": {p: int(v) for p, v in mv.items() if p not in ("total", "traversal_kernel")},
                     "B_touch": int(bt), "B_min": int(bm),
                     "format_bytes_model_equals_counting_pass": fmt_model == fmt_counted,
@@ -541,7 +555,7 @@ def main() -> None:
         for rec in sweep:
             rec["us_over_empty_kernel"] = round(rec["us"] / max(fl["empty_kernel_us"], 1e-3), 1)
         line["cusparse_spmv_reference"] = cusparse_reference(a, torch, dev, flush)
-        line["cpu_baseline"] = cpu_baseline(a, xs, model, info)
+        line["cpu_baseline"] = cpu_baseline(a, xs, model, info, one_kernel)
     if rank == 0 and world == 1 and not args.no_extras:
         try:
             line["other_configs"] = other_configs(B, torch, dev, flush, peak, line.get("latency_floors"))
@@ -987,7 +1001,7 @@ def cusparse_reference(a, torch, dev, flush):
         return {"error": repr(e)}
 
 
-def cpu_baseline(a, xs, model, info):
+def cpu_baseline(a, xs, model, info, one_kernel):
     """The oracle as it stands, single thread, on the same sweep (bounded: one pass, both
     routines per point, the faster one counted; same byte numerator as the GPU line)."""
     import oracle
@@ -1004,7 +1018,7 @@ def cpu_baseline(a, xs, model, info):
                 dt = time.perf_counter() - t0
                 best = dt if best is None or dt < best else best
             total_t += best
-            total_b += model.moved(x.idx, info[k][0], yi.size)["total"]
+            total_b += model.moved(x.idx, info[k][0], yi.size, None, one_kernel[k])["total"]
     return {"value": round(total_b / total_t / 1e9, 4), "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": "whole 6-point sweep, faster of ref_push/ref_pull per point, second of two passes",
             "ms_per_step": round(total_t * 1e3, 3), "host_cores_available": os.cpu_count()}

@@ -151,7 +151,13 @@ typedef struct {
     int32_t decode_x_f32;    /* dbspmspv_decode on a bf16 handle: 1 = x is given as n fp32 values
                                 (e.g. the y of the layer before, fed straight back in) and
                                 rounded to bf16, to nearest even, while it is blocked      (0) */
-    int32_t reserved[3];
+    int32_t no_small_call;   /* dbspmspv_run on a hypersparse handle with at most 256 entries in x
+                                (and a selector that is certain to say push, up to ~2.5 M rows,
+                                validate and timing off) runs as one kernel of one cluster of
+                                eight thread blocks that keep the result's row bitmap in their
+                                shared memories; 1 = use
+                                the general chain of kernels instead                      (0) */
+    int32_t reserved[2];
 } dbspmspv_run_opts;
 
 #define DBSPMSPV_MAX_BFS_LEVELS_RECORDED 64

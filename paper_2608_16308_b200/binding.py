@@ -50,7 +50,8 @@ class RunOpts(ctypes.Structure):
                 ("th3_decode", ctypes.c_float), ("no_fused_decode", ctypes.c_int32),
                 ("bfs_push_max_edge_frac", ctypes.c_float), ("hub_min_nnz_x", ctypes.c_int32),
                 ("decode_threshold", ctypes.c_float), ("decode_relu", ctypes.c_int32),
-                ("decode_x_f32", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
+                ("decode_x_f32", ctypes.c_int32), ("no_small_call", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 2)]
 
 
 class Stats(ctypes.Structure):

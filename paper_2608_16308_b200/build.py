@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdbspmspv.so")
 LIB_CHECKED = os.path.join(HERE, "libdbspmspv_check.so")   # the range-checked build (-DDBS_BOUNDS_CHECK)
 SOURCES = ("create.cu", "run.cu", "bfs.cu", "api.cu", "noalloc.cu", "measure.cu")
-HEADERS = ("internal.cuh", "microkernels.cuh", "worklist.cuh", "staging.cuh", "lean_pull.cuh", "decode_batch.cuh", "mma_block.cuh", "minplus.cuh")
+HEADERS = ("internal.cuh", "microkernels.cuh", "worklist.cuh", "staging.cuh", "lean_pull.cuh", "decode_batch.cuh", "mma_block.cuh", "minplus.cuh", "small_call.cuh")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

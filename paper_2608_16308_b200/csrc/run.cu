@@ -1576,6 +1576,7 @@ k_decode_stream(Device d, const void *__restrict__ x, float *__restrict__ y, flo
 
 }  // namespace dbs
 #include "decode_batch.cuh"
+#include "small_call.cuh"
 namespace dbs {
 
 // ------------------------------------------------------------------------------------------
@@ -1972,6 +1973,20 @@ static int run_typed(dbspmspv_handle_s *h, const int32_t *x_idx, const void *x_v
                      int semiring, int32_t *y_idx, float *y_val, int64_t y_capacity, int32_t *y_nnz,
                      cudaStream_t st, const uint32_t *row_mask = nullptr, int complement = 0) {
     const Device &d = h->d;
+    // a short x on a hypersparse handle: the whole call as one kernel of one thread-block cluster (small_call.cuh)
+    {
+        const size_t ywords = (size_t)(d.mb + 1) / 2, cbwords = (size_t)(d.nb + 31) / 32;
+        const size_t smem = ((ywords + SMALL_CLUSTER - 1) / SMALL_CLUSTER + (cbwords + SMALL_CLUSTER - 1) / SMALL_CLUSTER) * sizeof(uint32_t);
+        if (nnz_x > 0 && nnz_x <= SMALL_MAX_NNZ_X && d.n_entries > 0 && !h->heavy_stage && !h->ropts.validate && !h->ropts.timing &&
+            !h->ropts.no_small_call && h->ropts.force_path != DBSPMSPV_PATH_PULL && !pull_possible(h, nnz_x, h->ropts.th3) &&
+            smem <= SMALL_MAX_SMEM && (int64_t)ywords * 32 * (int64_t)sizeof(int32_t) <= d.ws.task_capacity * (int64_t)sizeof(*d.ws.tasks)) {
+            const int mode = semiring == DBSPMSPV_OR_AND ? 1 : semiring == DBSPMSPV_MIN_PLUS ? 2 : 0;
+            k_run_small<DT><<<SMALL_CLUSTER, SMALL_CTA, smem, st>>>(d, x_idx, x_val, nnz_x, mode, y_idx, y_val, y_capacity, y_nnz, row_mask, complement);
+            ++h->kernel_launches;
+            DBS_CUDA(cudaGetLastError());
+            return DBSPMSPV_OK;
+        }
+    }
     // x lists a quarter of the columns or more: a pull is likely (on hypersparse matrices), so
     // the worklist is built afterwards from the masks, and only if the selector does choose the push
     const bool minplus = semiring == DBSPMSPV_MIN_PLUS;

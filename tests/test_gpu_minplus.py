@@ -39,8 +39,10 @@ def test_minplus_parity(name, make, dtype, inline_max):
         if dtype == B.BF16:
             x.val = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x.val))
         want = oracle.ref_minplus(A, x.idx, x.val)
-        for path in (B.PATH_AUTO, B.PATH_PUSH, B.PATH_PULL):
-            h.set_opts(force_path=path)
+        for path in (B.PATH_AUTO, B.PATH_PUSH, B.PATH_PULL, -1):
+            # (-1: the push once more with the one-kernel form of a short call switched off)
+            h.set_opts(force_path=B.PATH_PUSH if path < 0 else path, no_small_call=int(path < 0))
+            path = B.PATH_PUSH if path < 0 else path
             check_exact(h.run(x, semiring=B.MIN_PLUS), want)
             st = h.get_stats()
             assert st.last_y_nnz == want[0].size

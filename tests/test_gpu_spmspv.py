@@ -47,13 +47,15 @@ def test_parity_all_paths(name, make, dtype, inline_max):
         want = oracle.ref_pull(A, x.idx, x.val)
         for path in PATHS:
             for thr in (1, 8, 17):
-                h.set_opts(force_path=path, popc_threshold=thr)
-                check_against_oracle(h.run(x), want)
-                st = h.get_stats()
-                if path != B.PATH_AUTO:
-                    assert st.last_path == path
-                assert st.last_n_nzblk == np.unique(x.idx >> 4).size
-                assert st.last_y_nnz == want[0].size
+                # (a short x may take the one-kernel form of the call: both forms are checked)
+                for no_small in ((0, 1) if path != B.PATH_PULL and thr == 8 else (0,)):
+                    h.set_opts(force_path=path, popc_threshold=thr, no_small_call=no_small)
+                    check_against_oracle(h.run(x), want)
+                    st = h.get_stats()
+                    if path != B.PATH_AUTO:
+                        assert st.last_path == path
+                    assert st.last_n_nzblk == np.unique(x.idx >> 4).size
+                    assert st.last_y_nnz == want[0].size
     h.close()
 
 
@@ -452,4 +454,57 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     with pytest.raises(B.DbSpmspvError) as e:
         B.dbspmspv_test_bounded_wait(h.h, 0)
     assert e.value.status == B.ERR_INVALID_ARG
+    h.close()
+
+
+def test_one_kernel_form_of_a_short_call():
+    """A short x on a hypersparse handle runs as one kernel of one thread block: one launch
+    instead of four, same result as the general chain; Boolean and masked output, capacity
+    overflow (full count reported, nothing written beyond, the handle clean afterwards), a hub
+    column shared out over the warp, a column block with payload entries, and the switch back
+    to the chain when x is long or an option asks for it."""
+    csr = wl.rmat(14, 16, seed=4)
+    A = ref_matrix(csr)
+    h = Handle(csr, B.F32)
+    rng = np.random.default_rng(3)
+    hub = int(np.argmax(np.bincount(csr.col_idx, minlength=csr.n)))
+    for k in (1, 17, 256, 257, 5000):
+        idx = rng.choice(csr.n, size=k, replace=False).astype(np.int32)
+        if hub not in idx:
+            idx[0] = hub
+        x = wl.SparseVec(csr.n, idx, rng.standard_normal(k).astype(np.float32))
+        want = oracle.ref_pull(A, x.idx, x.val)
+        launches = []
+        for no_small in (0, 1):
+            h.set_opts(no_small_call=no_small)
+            before = h.get_stats().kernel_launches
+            check_against_oracle(h.run(x), want)
+            launches.append(h.get_stats().kernel_launches - before)
+            check_against_oracle(h.run(x, semiring=B.OR_AND), want, boolean=True)
+        assert launches[0] == (1 if k <= 256 else launches[1]) and launches[1] >= 3
+    # capacity
+    h.set_opts()
+    x = wl.SparseVec(csr.n, np.asarray([hub, 5, 77], np.int32), np.ones(3, np.float32))
+    want = oracle.ref_pull(A, x.idx, x.val)
+    cap = want[0].size // 2
+    h.y_idx.fill_(-1)
+    yi, yv, k = h.run(x, capacity=cap)
+    assert k == want[0].size and np.array_equal(yi, want[0][:cap])
+    assert (h.y_idx[cap:].cpu().numpy() == -1).all()
+    assert h.get_stats(raise_on_device_status=False).device_status == B.ERR_CAPACITY
+    check_against_oracle(h.run(x), want)
+    # output mask and its complement
+    bits = rng.random(csr.m) < 0.5
+    words = np.zeros(((csr.m + 15) // 16 + 1) // 2, dtype=np.uint32)
+    r = np.flatnonzero(bits)
+    np.bitwise_or.at(words, r >> 5, np.uint32(1) << (r & 31).astype(np.uint32))
+    maskd = torch.from_numpy(words.view(np.int32)).to("cuda")
+    xi = torch.from_numpy(x.idx).to("cuda"); xv = torch.from_numpy(x.val).to("cuda")
+    for complement in (0, 1):
+        keep = bits[want[0]] if complement == 0 else ~bits[want[0]]
+        B.dbspmspv_run_masked(h.h, xi, xv, 3, B.PLUS_TIMES, maskd, complement, h.y_idx, h.y_val, csr.m, h.y_nnz)
+        torch.cuda.synchronize()
+        kk = int(h.y_nnz.item())
+        check_against_oracle((h.y_idx[:kk].cpu().numpy(), h.y_val[:kk].cpu().numpy(), kk), tuple(a[keep] for a in want))
+        check_against_oracle(h.run(x), want)                  # the dropped rows left nothing behind
     h.close()
