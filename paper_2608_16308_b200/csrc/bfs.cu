@@ -274,7 +274,7 @@ __device__ void bfs_pull(const Device &d, const Scope &sc, const uint32_t *F, ui
 // wanted walks its own INLINE run and stops at its first frontier neighbour -- the early exit of
 // Algorithm 5 per row instead of per row block: in the big levels a row finds a parent within a
 // few entries, so a fraction of the edges is read at all.
-// A warp takes a block of 32 consecutive mask words (1024 rows) and lane l walks one row of
+// A warp takes a block of W = 32 consecutive mask words (1024 rows; fewer on small graphs) and lane l walks one row of
 // every word (row (l + k) mod 32 of the block's word k), one row after the other, each lane at its own pace.  (With lane = row inside ONE word a
 // word costs as many dependent rounds as its slowest row -- and at the levels with a small
 // frontier almost every word holds a row without a frontier neighbour, which is walked to its
@@ -302,9 +302,14 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
     constexpr int LONG_UNROLL = 8, MAX_ROUNDS = 8;
     const int per_round = wide ? 8 : 4;
     int n_found = 0, n_nz = 0;
-    for (int w0 = gwarp * 32; w0 < n_words; w0 += nwarps * 32) {
+    // words per warp: 32, or -- on a graph with fewer mask words than that keeps every warp busy --
+    // the smallest power of two with which one pass of all warps covers the words (a lane then
+    // walks W rows; with 32-word blocks a graph of 2^18 vertices gave work to 256 of 4736 warps)
+    int W = 32;
+    while (W > 1 && (int64_t)nwarps * (W / 2) >= n_words) W >>= 1;
+    for (int w0 = gwarp * W; w0 < n_words; w0 += nwarps * W) {
         const int wd = w0 + lane;                    // this lane's word (bookkeeping); rows: lane = row of every word
-        const bool in = wd < n_words;
+        const bool in = lane < W && wd < n_words;
         const uint32_t need = in ? ~d.ws.visited32[wd] : 0u;   // (rows without stored elements and rows past m count as visited)
         if (in) Z[wd] = 0u;
         if (!__any_sync(FULL, need != 0u)) { if (in) N[wd] = 0u; continue; }
@@ -436,8 +441,7 @@ __device__ void bfs_pull_rows(const Device &d, const uint32_t *F, uint32_t *N, u
             }
         }
         // back to one word per lane: bit (l + k) mod 32 of word w0 + k <- bit k of lane l's result
-#pragma unroll 8
-        for (int kk = 0; kk < 32; ++kk) {
+        for (int kk = 0; kk < W; ++kk) {
             const uint32_t fk = __ballot_sync(FULL, (res >> kk) & 1u);
             if (lane == kk) found |= __funnelshift_l(fk, fk, kk);
         }

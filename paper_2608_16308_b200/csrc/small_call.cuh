@@ -218,8 +218,7 @@ k_run_small(Device d, const int32_t *__restrict__ x_idx, const void *__restrict_
             else { if ((keep >> bit) & 1u) ++pos; d.ws.y_acc[row] = 0.f; }
         }
     }
-    __threadfence();
-    cluster.sync();
+    cluster.sync();          // (release / acquire at cluster scope: the row list is visible to every block)
     STAMP();
     // every thread of the cluster takes result positions in turn: the gathers of a round are independent
     for (int64_t p0 = rank * SMALL_CTA + tid; p0 < room; p0 += (int64_t)SMALL_ILP * SMALL_CLUSTER * SMALL_CTA) {

@@ -1,6 +1,6 @@
 // Asynchronous staging into shared memory (Section 3.3.3): 1-D bulk copies issued by one lane
 // (the TMA engine moves the bytes; no registers are held while they fly) that complete on an
-// mbarrier.  Only the plain, non-multicast form is used, and only on this GPU's own memory.
+// mbarrier.  Only the plain form with one destination is used, and only on this GPU's own memory.
 // Every wait is bounded: on expiry the caller records DBSPMSPV_ERR_TIMEOUT and leaves.
 #pragma once
 
