@@ -1,6 +1,6 @@
 """The range-checked build of the library (-DDBS_BOUNDS_CHECK: every index a kernel reads from
 the handle's arrays is tested, a violation records ERR_INTERNAL and skips the access) runs the
-small parity cases of run, decode and BFS in a child process; every handle's status must stay
+small parity cases of run (all semirings), decode, BFS and shortest paths in a child process; every handle's status must stay
 clean and every parity check must hold.  It stands in for a memory checker."""
 import os
 import subprocess
@@ -17,7 +17,8 @@ def test_small_parity_cases_pass_under_the_range_checked_library():
     lib = build.build_library(checked=True)
     env = dict(os.environ, DBSPMSPV_LIBRARY=lib)
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
-           "tests/test_gpu_spmspv.py", "tests/test_gpu_decode.py", "tests/test_gpu_bfs.py", "tests/test_gpu_format.py"]
+           "tests/test_gpu_spmspv.py", "tests/test_gpu_decode.py", "tests/test_gpu_bfs.py", "tests/test_gpu_format.py",
+           "tests/test_gpu_minplus.py"]
     r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)
     assert r.returncode == 0, r.stdout[-4000:] + r.stderr[-2000:]
 
