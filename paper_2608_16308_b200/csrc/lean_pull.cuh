@@ -290,8 +290,9 @@ k_pull_lean(Device d, Out out, float th3, int force_path, int popc_threshold, in
         const int nnz = (int)d.csr.aux[pos] + 1;
         const int rb = d.entry_row[pos];
         if (Out::MINPLUS) {
-            block_elements_warp<DT>(type, d.csr.w[pos], d.csr.aux[pos], xm, d.payload, lane, [&](int r, int c, float a) {
-                lean_add<DT>(out, rb * 16 + r, a + d.ws.x_dense[(size_t)cb * 16 + c]);
+            block_rows_min_warp<DT>(type, d.csr.w[pos], d.csr.aux[pos], xm, d.ws.x_dense + (size_t)cb * 16, d.payload, lane, [&](int r, uint32_t key) {
+                atomicMax(reinterpret_cast<uint32_t *>(out.acc) + (size_t)rb * 16 + r, key);
+                out.hit8[(size_t)rb * 16 + r] = 1;
             });
             continue;
         }

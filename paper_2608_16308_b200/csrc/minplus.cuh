@@ -83,41 +83,70 @@ __device__ __forceinline__ void block_elements(int type, uint32_t w, uint32_t au
     }
 }
 
-// The same for one block with a payload taken by a whole warp: a lane owns half a row (row-major
-// classes) or half a column (column-major classes, Dense), COO entries are dealt out in turn.
+// One block with a payload taken by a whole warp, (min, +): row r's smallest a + x over the listed
+// columns, reduced across the lanes, then `f(r, key)` once per row that has one (lane r calls
+// it) -- one atomic per row instead of one per element (the payload blocks of a power-law
+// matrix are its hub corner: their rows are the ones whose atomics queue up).  `xb`: the 16 x
+// entries of the block's vector block.  A lane owns half a row (row-major classes) or half a
+// column (column-major classes, Dense); COO entries are dealt out in turn.
 template <int DT, typename F>
-__device__ __forceinline__ void block_elements_warp(int type, uint32_t w, uint32_t aux, uint32_t xm, const uint8_t *payload, int lane, F f) {
+__device__ __forceinline__ void block_rows_min_warp(int type, uint32_t w, uint32_t aux, uint32_t xm, const float *xb,
+                                                    const uint8_t *payload, int lane, F f) {
     const uint8_t *blk = payload + (size_t)w * 4;
+    constexpr uint32_t FULLW = 0xFFFFFFFFu;
     if (type == DBSPMSPV_BLK_COO) {
+        // (entries of a row are adjacent but few: one reduction per row present in the block)
         const int nnz = (int)aux + 1;
         const uint8_t *vals = blk + ((nnz + 3) & ~3);
-        for (int k = lane; k < nnz; k += 32) {
+        uint32_t key[2] = {0u, 0u};
+        int row[2] = {-1, -1};
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {               // nnz <= 64 in this class
+            const int k = lane + 32 * u;
+            if (k < nnz) {
+                const uint32_t rc = blk[k];
+                if ((xm >> (rc & 15)) & 1u) { row[u] = (int)(rc >> 4); key[u] = minplus_key(Val<DT>::load(vals, k) + xb[rc & 15]); }
+            }
+        }
+        for (int r = 0; r < 16; ++r) {
+            const uint32_t mine = max(row[0] == r ? key[0] : 0u, row[1] == r ? key[1] : 0u);
+            const uint32_t m = __reduce_max_sync(FULLW, mine);
+            if (lane == r && m) f(r, m);
+        }
+        for (int k = lane + 64; k < nnz; k += 32) {  // (forced-format blocks may be longer: element-wise)
             const uint32_t rc = blk[k];
-            if ((xm >> (rc & 15)) & 1u) f((int)(rc >> 4), (int)(rc & 15), Val<DT>::load(vals, k));
+            if ((xm >> (rc & 15)) & 1u) f((int)(rc >> 4), minplus_key(Val<DT>::load(vals, k) + xb[rc & 15]));
         }
         return;
     }
     constexpr bool HAS_STARTS = Val<DT>::SIZE != 0;
     const uint16_t *masks = reinterpret_cast<const uint16_t *>(blk);
-    const int major = lane >> 1;
-    const uint32_t half = 0xFFu << (8 * (lane & 1));
+    const int major = lane >> 1, hf = lane & 1;
     const uint32_t full = masks[major];
     if (is_row_major(type)) {
         const uint8_t *vals = blk + HDR_BYTES;
         const int base = HAS_STARTS ? blk[32 + major] : 0;
-        for (uint32_t act = full & xm & half; act; act &= act - 1) {
+        uint32_t key = 0u;
+        for (uint32_t act = full & xm & (0xFFu << (8 * hf)); act; act &= act - 1) {
             const int c = __ffs(act) - 1;
-            f(major, c, Val<DT>::load(vals, base + __popc(full & ((1u << c) - 1u))));
+            key = max(key, minplus_key(Val<DT>::load(vals, base + __popc(full & ((1u << c) - 1u))) + xb[c]));
         }
+        key = max(key, __shfl_xor_sync(FULLW, key, 1));
+        if (hf == 0 && key) f(major, key);           // lane 2r holds row r
         return;
     }
-    if (!((xm >> major) & 1u)) return;
     const bool dense = type == DBSPMSPV_BLK_DENSE;
     const uint8_t *vals = blk + (dense ? 32 : HDR_BYTES);
     const int base = dense ? major * 16 : (HAS_STARTS ? blk[32 + major] : 0);
-    for (uint32_t cm = full & half; cm; cm &= cm - 1) {
-        const int r = __ffs(cm) - 1;
-        f(r, major, Val<DT>::load(vals, dense ? base + r : base + __popc(full & ((1u << r) - 1u))));
+    const bool listed = (xm >> major) & 1u;
+    const float xc = listed ? xb[major] : 0.f;
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+        uint32_t key = 0u;
+        if (listed && (r >> 3) == hf && ((full >> r) & 1u))
+            key = minplus_key(Val<DT>::load(vals, dense ? base + r : base + __popc(full & ((1u << r) - 1u))) + xc);
+        const uint32_t m = __reduce_max_sync(FULLW, key);
+        if (lane == r && m) f(r, m);
     }
 }
 
