@@ -1,7 +1,8 @@
 // One SpMSpV call (Sections 3.3 and 4.1): vector blocking + push worklist, device-side path
 // selection, push / pull traversal with per-block microkernels, hierarchical writeback, and
 // compaction of the dense accumulator into a sorted sparse y.  Also the dense-in / dense-out
-// decode entry (Section 4.3).  Nothing here allocates or synchronises.
+// decode entry (Section 4.3).  Nothing here allocates or synchronises, except db_sssp (a host
+// loop over (min, +) products, at the end of the file).
 #include "internal.cuh"
 #include "microkernels.cuh"
 #include "staging.cuh"
