@@ -37,6 +37,34 @@ def test_c2_rmat20_sweep():
             for path in (B.PATH_PUSH, B.PATH_PULL):
                 h.set_opts(force_path=path)
                 check_against_oracle(h.run(x), want)
+        if x.idx.size <= 256:                     # the short points once more as the general chain of kernels
+            h.set_opts(no_small_call=1)
+            check_against_oracle(h.run(x), want)
+        if f in (1e-5, 1e-2, 0.5):                # (min, +) on the same x: one-kernel form, push, streaming pull
+            h.set_opts()
+            wi, wv = oracle.ref_minplus(A, x.idx, x.val)
+            gi, gv, kk = h.run(x, semiring=B.MIN_PLUS)
+            assert kk == wi.size and np.array_equal(gi, wi)
+            assert np.array_equal(gv.view(np.uint32), wv.astype(np.float32).view(np.uint32))
+    h.close()
+
+
+def test_sssp_rmat20_symmetric_weighted():
+    """db_sssp at the size the benchmark times: distances against the Bellman-Ford oracle."""
+    import torch
+    g = wl.rmat(20, 16, seed=3, symmetrise=True)
+    g.val = (0.05 + wl.rand_f32(7, 1, np.arange(g.nnz))).astype(np.float32)
+    h = Handle(g, B.F32)
+    A = ref_matrix(g)
+    for src in wl.bfs_sources(g, 2):
+        dist = torch.empty(g.n, dtype=torch.float32, device="cuda")
+        steps = B.db_sssp(h.h, int(src), dist)
+        torch.cuda.synchronize()
+        got = dist.cpu().numpy()
+        want = oracle.ref_sssp(A, int(src))
+        fin = np.isfinite(want)
+        assert np.array_equal(np.isfinite(got), fin) and steps >= 2
+        assert np.all(np.abs(got[fin] - want[fin]) <= 64 * 2.0 ** -24 * want[fin] + 1e-30)
     h.close()
 
 
