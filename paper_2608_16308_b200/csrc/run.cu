@@ -318,6 +318,18 @@ __device__ __forceinline__ bool push_private(const Device &d, uint32_t idx, uint
     return true;
 }
 
+// Per-warp staging area in shared memory: two stages of view entries for the pull; the push
+// uses the same bytes as one stage for the payload of a task's blocks.
+struct PullStage {
+    uint32_t idx[STAGE_CAP];
+    uint32_t w[STAGE_CAP];
+    uint8_t aux[STAGE_CAP];
+};
+struct PullWarp {
+    PullStage stage[2];
+    uint64_t bar[2];
+};
+
 // Push (Section 3.3.2): every warp takes one task = up to PUSH_CHUNK consecutive block-CSC
 // entries of one active column block (32 per step, all fetched up front); the vector block is staged once per task (Section 3.3.3).  Lanes
 // own hypersparse blocks; heavier blocks are then processed by the whole warp one at a time.
@@ -325,7 +337,7 @@ __device__ __forceinline__ bool push_private(const Device &d, uint32_t idx, uint
 // the row block's hit mask.  The task record carries its length, so the view entries, the mask
 // and the x block are all fetched in one round of independent loads.
 template <int DT, typename Out, bool HV>
-__device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp, float *s_lacc) {
+__device__ void push_body(const Device &d, Out out, int popc_threshold, float *s_x, float *s_tmp, float *s_lacc, PullWarp *pw) {
     constexpr int U = PUSH_CHUNK / 32;
     const int lane = threadIdx.x & 31;
     const int gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -359,10 +371,44 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
     const uint2 none = make_uint2(0u, 0u);
     uint2 rec1 = gwarp + nwarps < n_tasks ? item(gwarp + nwarps) : none;
     Loads cur = loads_of(gwarp, gwarp < n_tasks ? item(gwarp) : none);
+    // Payload staging (Section 3.3.3) on handles whose elements sit mostly in blocks with a payload:
+    // when the payload of all blocks of a task fits the warp's staging area, every lane moves its
+    // block there with one bulk copy and the microkernels read shared memory.  The point is the
+    // bytes in flight: 32 blocks per warp at once instead of the two a half-warp pair walks
+    // (header -> values, two dependent trips each) -- at 14 warps per SM the latter keeps about
+    // 6 KB per SM in flight where the memory system wants 35.  (A second area per warp, so that
+    // the next task's copies fly while this one is computed, was measured slower: the shared
+    // memory it takes costs a resident thread block per SM.)
+    constexpr int STAGE_AREA = (int)sizeof(PullStage) * 2;
+    uint32_t stage_parity = 0u;
+    // issues the copies of one task; returns the lane's byte offset in the area, or -1 (not staged)
+    auto stage_issue = [&](const Loads &l) {
+        const bool have = l.start + lane < l.end;
+        const int type = l.idx >> TYPE_SHIFT;
+        const int bytes = have && type != DBSPMSPV_BLK_INLINE ? payload_words(type, (int)l.aux + 1, Val<DT>::SIZE) * 4 : 0;
+        int incl = bytes;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(FULL, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int total = __shfl_sync(FULL, incl, 31);
+        if (total <= 0 || total > STAGE_AREA) return -1;          // warp-uniform
+        uint8_t *area = reinterpret_cast<uint8_t *>(pw->stage);
+        if (lane == 0) mbar_arrive_expect_tx(&pw->bar[0], (uint32_t)total);
+        __syncwarp();
+        if (bytes) bulk_copy_g2s(area + incl - bytes, d.payload + (size_t)l.w * 4, (uint32_t)bytes, &pw->bar[0]);
+        return incl - bytes;
+    };
+    if (HV) {
+        if (lane == 0) { mbar_init(&pw->bar[0], 1); fence_barrier_init(); }
+        __syncwarp();
+    }
     for (int t = gwarp; t < n_tasks; t += nwarps) {
         const uint2 rec2 = t + 2 * nwarps < n_tasks ? item(t + 2 * nwarps) : none;
         const Loads nxt = loads_of(t + nwarps, rec1);
         rec1 = rec2;
+        const int off_cur = HV ? stage_issue(cur) : -1;         // (the area is free: the last task's reads ended at the warp barrier)
         uint32_t idx[U] = {cur.idx}, w[U] = {cur.w}, aux[U] = {cur.aux};
         const int start = cur.start, end = cur.end, jb = cur.jb;
         const uint32_t xm = cur.xm;
@@ -377,6 +423,18 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
             int coo_cnt = 0;
             const int type = idx[u] >> TYPE_SHIFT;
             const int brow = idx[u] & IDX_MASK;
+            const uint8_t *pl = d.payload;        // where this task's payload is read from (w[u] counts 4-byte words from it)
+            if (HV && off_cur >= 0) {            // warp-uniform: this task's payload was staged
+                if (!mbar_wait_bounded(&pw->bar[0], stage_parity)) {
+                    // (never seen; the copies in flight get a second, equally bounded chance to land before the warp leaves)
+                    d.ws.ctr->status = DBSPMSPV_ERR_TIMEOUT;
+                    mbar_wait_bounded(&pw->bar[0], stage_parity);
+                    return;
+                }
+                stage_parity ^= 1u;
+                pl = reinterpret_cast<const uint8_t *>(pw->stage);
+                if (have && type != DBSPMSPV_BLK_INLINE) w[u] = (uint32_t)off_cur >> 2;
+            }
             if (have) {
                 if (type == DBSPMSPV_BLK_INLINE) {
                     float *row0 = out.acc + (size_t)brow * 16;
@@ -389,7 +447,7 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                     // per-block writebacks of mask-based blocks keep the plain atomic and the
                     // unconditional store: on the stencil the returning atomic cost 7-15 %.)
                     bool first = false;
-                    const uint32_t hit = lane_block<DT>(type, w[u], aux[u], xm, s_x[aux[u] & 15], s_x, d.payload,
+                    const uint32_t hit = lane_block<DT>(type, w[u], aux[u], xm, s_x[aux[u] & 15], s_x, pl,
                                                         [&](int r, float v) { if (!push_private<Out>(d, idx[u], aux[u], v)) first |= atomicAdd(row0 + r, v) == 0.0f; });
                     // (pattern matrices have no product: they count the hits in the accumulator,
                     // which the compaction clears like any other, to get the same first-touch test)
@@ -405,7 +463,7 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                 uint32_t *s_hit = reinterpret_cast<uint32_t *>(s_tmp);   // per-owner-lane hit masks
                 s_hit[lane] = 0u;
                 __syncwarp();
-                warp_flat_coo<DT>(coo_cnt, w[u], xm, (uint32_t)brow, 0u, d.payload, lane,
+                warp_flat_coo<DT>(coo_cnt, w[u], xm, (uint32_t)brow, 0u, pl, lane,
                                   [&](uint32_t tag, uint32_t, int r, int c, float a, int owner) {
                                       if (DT != DBSPMSPV_PATTERN) atomicAdd(out.acc + (size_t)tag * 16 + r, a * s_x[c]);
                                       if (Out::MASKS) atomicOr(&s_hit[owner], 1u << r);
@@ -427,8 +485,8 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                     };
                     const uint32_t rows = __ballot_sync(FULL, mk && is_row_major(type));
                     const uint32_t tagged = (idx[u] & ~IDX_MASK) | (uint32_t)jb;     // class bits + the task's column block
-                    if (cs & ~rows) half_stream<DT, false>(d.payload, d.ws.x_dense, tagged, w[u], xm, brow, cs & ~rows, lane, emit);
-                    if (rows) half_stream<DT, true>(d.payload, d.ws.x_dense, tagged, w[u], xm, brow, rows, lane, emit);
+                    if (cs & ~rows) half_stream<DT, false>(pl, d.ws.x_dense, tagged, w[u], xm, brow, cs & ~rows, lane, emit);
+                    if (rows) half_stream<DT, true>(pl, d.ws.x_dense, tagged, w[u], xm, brow, rows, lane, emit);
                     if (mk) heavy = false;
                     __syncwarp();
                 }
@@ -441,7 +499,7 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
             if (HV && __popc(hv_mask) >= HEAVY_LANE_MIN) {
                 // many mask-based blocks side by side: every lane walks its own block
                 if (lane_form) {
-                    const uint8_t *blk = d.payload + (size_t)w[u] * 4;
+                    const uint8_t *blk = pl + (size_t)w[u] * 4;
                     float *acc = s_lacc + lane;
                     uint32_t hits;
                     if (DT == DBSPMSPV_PATTERN) {
@@ -468,7 +526,7 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
                 const int nnz = (int)__shfl_sync(FULL, aux[u], src) + 1;
                 const int btype = bidx >> TYPE_SHIFT;
                 const int bbrow = bidx & IDX_MASK;
-                const uint8_t *blk = d.payload + (size_t)bw * 4;
+                const uint8_t *blk = pl + (size_t)bw * 4;
                 uint32_t hits;
                 float sum = 0.f;
                 if (DT == DBSPMSPV_PATTERN) hits = warp_block_bool<DT>(btype, blk, nnz, xm, lane);
@@ -490,15 +548,6 @@ __device__ void push_body(const Device &d, Out out, int popc_threshold, float *s
 // (long hub row blocks stay there over many steps); products of the other, short segments met
 // in the same step go straight to global atomics.  INLINE entries need one gather only: the
 // dense copy of x carries a "not listed" marker, so presence and value come from one load.
-struct PullStage {
-    uint32_t idx[STAGE_CAP];
-    uint32_t w[STAGE_CAP];
-    uint8_t aux[STAGE_CAP];
-};
-struct PullWarp {
-    PullStage stage[2];
-    uint64_t bar[2];
-};
 #ifndef DBS_PULL_UNROLL
 #define DBS_PULL_UNROLL 2
 #endif
@@ -781,18 +830,23 @@ __device__ __forceinline__ int select_path(const Device &d, float th3, int force
 #ifndef DBS_MIN_CTAS
 #define DBS_MIN_CTAS 1
 #endif
+// (MODE 1: five resident thread blocks per SM -- a cap of 102 registers -- measured 7 - 10 % faster
+// than the compiler's own 107 registers and four thread blocks once the push stages its payload)
+#ifndef DBS_MIN_CTAS_HEAVY
+#define DBS_MIN_CTAS_HEAVY 5
+#endif
 // Variants of the traversal kernel, chosen per handle from the class census at create:
 //   MODE 0  hypersparse matrices (power-law graphs): the push only -- their pull is the
 //           streaming kernel k_pull_lean, launched next in the stream
 //   MODE 1  matrices whose elements sit mostly in mask-based blocks (pruned layers, banded
 //           matrices): half-warp streaming and lane-owned microkernels
-// Dynamic shared memory: per-warp pull stages | lane scratch of the lane-owned form (MODE 1).
+// Dynamic shared memory: per-warp pull stages (the push stages payload there) | lane scratch of the lane-owned form (MODE 1).
 template <int MODE> constexpr size_t compute_dyn_smem() {
     return MODE >= 1 ? WARPS * sizeof(PullWarp) + WARPS * 16 * LANE_ACC_STRIDE * sizeof(float) : 0;
 }
 
 template <int DT, typename Out, int MODE>
-__global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold, int pull_done) {
+__global__ void __launch_bounds__(CTA, MODE >= 1 ? DBS_MIN_CTAS_HEAVY : DBS_MIN_CTAS) k_compute(Device d, Out out, float th3, int force_path, int popc_threshold, int pull_done) {
     constexpr bool HV = MODE >= 1;
     __shared__ float s_x[WARPS][16], s_tmp[WARPS][32], s_y[HV ? WARPS : 1][16 * SY_COPIES];
     extern __shared__ __align__(128) uint8_t s_dyn[];
@@ -805,7 +859,7 @@ __global__ void __launch_bounds__(CTA, DBS_MIN_CTAS) k_compute(Device d, Out out
     if (blockIdx.x == 0 && threadIdx.x == 0) d.ws.ctr->path = path;
     float *lacc = HV ? s_lacc + warp * 16 * LANE_ACC_STRIDE : nullptr;
     if (pull_done && path == DBSPMSPV_PATH_PULL) return;     // (the decode entry's own pull kernel has run)
-    if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], lacc);
+    if (path == DBSPMSPV_PATH_PUSH) push_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], lacc, HV ? &s_pull[warp] : nullptr);
     else if (HV) pull_body<DT, Out, HV>(d, out, popc_threshold, s_x[warp], s_tmp[warp], s_y[warp], lacc, &s_pull[warp]);
     // (MODE 0: the pull is k_pull_lean's)
 }
