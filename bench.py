@@ -337,6 +337,9 @@ def main() -> None:
                     help="run only the DB-BFS leg and print its record (the command ncu captures k_bfs from)")
     ap.add_argument("--decode-only", action="store_true",
                     help="run only the decode layers and print their records (the command ncu captures k_decode_fused from)")
+    ap.add_argument("--stencil-only", action="store_true",
+                    help="run only the 27-point stencil records (the command ncu captures the payload-staging push from)")
+    ap.add_argument("--stencil-d", type=int, default=160, help="edge length of the stencil grid for --stencil-only")
     ap.add_argument("--crossover", action="store_true",
                     help="print the measured push/pull crossover table (forced paths) and exit")
     ap.add_argument("--ablation", action="store_true", help="print the block-format ablation and storage records and exit")
@@ -359,11 +362,13 @@ def main() -> None:
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
     peak, peak_kind = measured_peak_gbs()
-    if args.bfs_only or args.decode_only or args.ablation:
+    if args.bfs_only or args.decode_only or args.ablation or args.stencil_only:
         if rank == 0:
             flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
             if args.bfs_only:
                 print(json.dumps(bench_bfs(args, B, torch, dev, flush, peak)))
+            elif args.stencil_only:
+                print(json.dumps(other_configs(B, torch, dev, flush, peak, None, args.stencil_d)))
             elif args.decode_only:
                 print(json.dumps(decode_layers(B, torch, dev, flush, peak) + [decode_chain(B, torch, dev, flush)] + decode_batch(B, torch, dev, flush)))
             else:
@@ -710,7 +715,7 @@ def minplus_rows(B, torch, dev, flush, peak):
     return out
 
 
-def other_configs(B, torch, dev, flush, peak, floors):
+def other_configs(B, torch, dev, flush, peak, floors, stencil_only_d=None):
     """The remaining workload shapes, one record each (whole call, cold L2 and L2-warm): the
     uniform matrix with a 1 % x, the 27-point stencil with clustered x at 0.1 % and 5 %, and
     single-token decode on three pruned layer shapes next to a dense bf16 GEMV of the same shape
@@ -750,6 +755,12 @@ def other_configs(B, torch, dev, flush, peak, floors):
             out.append(rec)
         B.dbspmspv_destroy(h)
 
+    if stencil_only_d:          # (--stencil-only: the 27-point stencil alone, at a chosen edge length)
+        a3 = wl.stencil27(stencil_only_d, seed=2)
+        r1, r2 = max(1, round(1e-3 * a3.n / 64)), max(1, round(5e-2 * a3.n / 64))
+        spmspv_case(f"stencil27_{stencil_only_d}cubed_fp32", a3, [("0.1 % in runs of 64", wl.clustered_x(a3.n, r1)),
+                                                                   ("5 % in runs of 64", wl.clustered_x(a3.n, r2))])
+        return out
     a1 = wl.uniform_rows()
     spmspv_case("uniform16384_8perrow_fp32", a1, [("164 nnz (1 %)", wl.sparse_x(0, 1, a1.n, 164))])
     a3 = wl.stencil27(160, seed=2)
