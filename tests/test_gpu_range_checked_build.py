@@ -18,7 +18,7 @@ def test_small_parity_cases_pass_under_the_range_checked_library():
     env = dict(os.environ, DBSPMSPV_LIBRARY=lib)
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
            "tests/test_gpu_spmspv.py", "tests/test_gpu_decode.py", "tests/test_gpu_bfs.py", "tests/test_gpu_format.py",
-           "tests/test_gpu_minplus.py"]
+           "tests/test_gpu_minplus.py", "tests/test_gpu_randomised.py"]
     r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)
     assert r.returncode == 0, r.stdout[-4000:] + r.stderr[-2000:]
 
