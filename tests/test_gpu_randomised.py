@@ -84,3 +84,32 @@ def test_random_cases(seed):
         else:
             check_against_oracle(got, (wi, wv, ws), boolean=semiring == B.OR_AND)
     h.close()
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("DBS_RANDOM_CASES", "24")) // 2))
+def test_random_graph_drivers(seed):
+    """db_bfs (levels bit-exact) and db_sssp (dyadic weights: distances exact) on random square
+    graphs, directed and symmetrised, from random sources including isolated ones."""
+    rng = np.random.default_rng(5000 + seed)
+    kind = int(rng.integers(0, 3))
+    if kind == 0:
+        n = int(rng.integers(2, 4000))
+        g = wl.random_sparse(n, n, min(n * n, int(rng.integers(1, 5 * n))), int(rng.integers(1 << 30)))
+    elif kind == 1:
+        g = wl.rmat(int(rng.integers(6, 13)), int(rng.integers(2, 16)), seed=int(rng.integers(1 << 30)), symmetrise=bool(rng.integers(0, 2)))
+    else:
+        g = wl.stencil27(int(rng.integers(3, 12)), seed=int(rng.integers(1 << 30)))
+    g.val = (1 + (wl.rand_u64(seed, 3, np.arange(g.nnz)) % 63)).astype(np.float32) / 8.0
+    hv = Handle(g, B.F32)
+    hp = Handle(wl.CSR(g.m, g.n, g.row_ptr, g.col_idx, None), B.PATTERN)
+    A = ref_matrix(g)
+    P = oracle.RefMatrix(g.m, g.n, g.row_ptr, g.col_idx, None)
+    levels = torch.empty(g.n, dtype=torch.int32, device="cuda")
+    dist = torch.empty(g.n, dtype=torch.float32, device="cuda")
+    for src in rng.integers(0, g.n, size=3):
+        B.db_bfs(hp.h, int(src), levels)
+        B.db_sssp(hv.h, int(src), dist)
+        torch.cuda.synchronize()
+        assert np.array_equal(levels.cpu().numpy(), oracle.ref_bfs(P, int(src)))
+        assert np.array_equal(dist.cpu().numpy().astype(np.float64), oracle.ref_sssp(A, int(src)))
+    hv.close(); hp.close()
