@@ -966,6 +966,37 @@ def format_ablation(B, torch, dev, flush):
     return out
 
 
+def modelled_block_size_bytes(a, vs: int, bs: int) -> dict:
+    """Storage of the blocked format at block size `bs`, MODELLED on the host from the per-block
+    element counts (the kernels exist for 16 x 16 blocks only; 32 and 64 are what the same layout
+    rules would store): the class thresholds scale with the block area (no payload up to
+    bs^2/8 - 1 elements, Dense above bs^2/2), a view entry is 8 bytes + the packed local
+    coordinates, a mask-based block carries bs masks of bs bits and bs start offsets, a Dense
+    block bs masks and bs^2 values; both views, their pointer arrays and the per-column
+    pointers are counted.  At bs = 16 this is the library's own layout (checked against its
+    statistics by the caller)."""
+    rows = np.repeat(np.arange(a.m, dtype=np.int64), np.diff(a.row_ptr))
+    nbc = (a.n + bs - 1) // bs
+    key = (rows // bs) * nbc + (a.col_idx.astype(np.int64) // bs)
+    cnt = np.unique(key, return_counts=True)[1]
+    area = bs * bs
+    th0, th1 = area // 8, area // 2
+    coord = (2 * int(np.log2(bs)) + 7) // 8                 # bytes of a packed (row, column) pair
+    start = 1 if area <= 256 else 2                         # bytes of a start offset
+    inline = cnt < th0
+    mid = (~inline) & (cnt <= th1)
+    dense = cnt > th1
+    r16 = lambda b: (b + 15) // 16 * 16
+    payload = int(r16(bs * bs // 8 + bs * start + cnt[mid] * vs).sum()) if vs else int(r16(np.full(int(mid.sum()), bs * bs // 8)).sum())
+    payload += int(dense.sum()) * int(r16(bs * bs // 8 + area * vs))
+    entries = int(cnt[inline].sum()) + int(mid.sum()) + int(dense.sum())
+    mb, nb = (a.m + bs - 1) // bs, nbc
+    views = 2 * entries * (8 + coord) + 4 * (mb + 1) + 4 * (nb + 1) + 4 * (bs + 1) * nb
+    return {"block": bs, "blocks": int(cnt.size), "no_payload_blocks": int(inline.sum()), "mask_blocks": int(mid.sum()),
+            "dense_blocks": int(dense.sum()), "payload_bytes": payload, "view_bytes": int(views),
+            "bytes_per_nnz": round((payload + views) / max(a.nnz, 1), 2)}
+
+
 def storage_table(B, torch, dev):
     """Stored bytes of the blocked format against CSR and CSR + CSC (Section 5.5's accounting,
     on the synthetic inputs; 32-bit indices, the configuration's value type)."""
@@ -986,7 +1017,10 @@ def storage_table(B, torch, dev):
         fmt = int(st.payload_bytes + st.csr_view_bytes + st.csc_view_bytes + st.segment_bytes + st.lean_index_bytes)
         csr = a.nnz * (4 + vs) + 4 * (a.m + 1)
         both = 2 * a.nnz * (4 + vs) + 4 * (a.m + a.n + 2)
+        sweep = [modelled_block_size_bytes(a, vs, bs) for bs in (16, 32, 64)]
+        sweep[0]["payload_bytes_equals_library"] = sweep[0]["payload_bytes"] == int(st.payload_bytes)
         out.append({"matrix": name, "nnz": int(a.nnz), "format_bytes": fmt, "bfs_index_bytes": int(st.bfs_index_bytes),
+                    "block_size_sweep_modelled": sweep,
                     "payload_bytes": int(st.payload_bytes), "view_bytes": int(st.csr_view_bytes + st.csc_view_bytes),
                     "csr_bytes": int(csr), "csr_plus_csc_bytes": int(both), "format_bytes_per_nnz": round(fmt / a.nnz, 2),
                     "vs_csr": round(fmt / csr, 3), "vs_csr_plus_csc": round(fmt / both, 3)})
